@@ -1,0 +1,245 @@
+"""ctypes front end of the CPU oracle (``memoracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+CPU-baseline leg of the benchmark.  The CUDA library and its Python binding never
+import this package, and this package imports nothing from them.
+
+Every function marshals numpy arrays into the C routines and returns numpy
+arrays; no arithmetic of the method happens in Python here.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_DIR = Path(__file__).resolve().parent
+_SRC = _DIR / "memoracle.c"
+_LIB = _DIR / "libmemoracle.so"
+
+F32, F16 = 0, 1
+
+OK = 0
+ERR_ARG, ERR_BLOCK_TABLE, ERR_BLOCK_ID, ERR_FACT_ID, ERR_NOMEM = -1, -2, -3, -4, -5
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle returned {code}")
+        self.code = code
+
+
+def build(force: bool = False) -> Path:
+    """Compile ``memoracle.c`` into ``libmemoracle.so`` next to it (gcc, -O3, OpenMP)."""
+    if not force and _LIB.exists() and _LIB.stat().st_mtime >= _SRC.stat().st_mtime:
+        return _LIB
+    tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+    cmd = ["gcc", "-std=c11", "-O3", "-fPIC", "-shared", "-fopenmp", "-Wall", "-Wextra", str(_SRC), "-o", str(tmp), "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(str(_LIB))
+        p, i32, i64, dbl = C.c_void_p, C.c_int, C.c_int64, C.c_double
+        L.oracle_kv_bytes.restype = i64
+        L.oracle_kv_bytes.argtypes = [i64] * 5
+        L.oracle_max_threads.restype = i32
+        L.oracle_scores.restype = i32
+        L.oracle_scores.argtypes = [p, i32, i64, i32, p, p, i32]
+        L.oracle_retrieve.restype = i32
+        L.oracle_retrieve.argtypes = [p, i32, i64, i32, p, p, i32, i32, p, p, i32]
+        L.oracle_inv_freq.restype = None
+        L.oracle_inv_freq.argtypes = [i32, dbl, p]
+        L.oracle_rope_rows.restype = i32
+        L.oracle_rope_rows.argtypes = [p, i64, i32, p, dbl, i32, p, p]
+        L.oracle_inject.restype = i32
+        L.oracle_inject.argtypes = (
+            [p, i32, i64, p, p, p, p, i64, i32, i32, i32, dbl, i32, p, i64, p, i64, i32, i64, i32, i32]
+            + [p] * 7
+            + [i64] * 4
+            + [i32]
+        )
+        for name in ("oracle_bf16_from_double", "oracle_bf16_to_double", "oracle_f16_to_double"):
+            getattr(L, name).restype = None
+            getattr(L, name).argtypes = [p, i64, p]
+        _lib = L
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _emb_dtype(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.float16:
+        return F16
+    raise TypeError(f"embeddings must be float32 or float16, got {a.dtype}")
+
+
+def max_threads() -> int:
+    return int(lib().oracle_max_threads())
+
+
+def kv_bytes(L: int, c: int, h: int, d: int, b: int) -> int:
+    return int(lib().oracle_kv_bytes(L, c, h, d, b))
+
+
+def bf16_from_double(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib().oracle_bf16_from_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def bf16_to_double(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.uint16)
+    out = np.empty(x.shape, dtype=np.float64)
+    lib().oracle_bf16_to_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def f16_to_double(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x).view(np.uint16)
+    out = np.empty(x.shape, dtype=np.float64)
+    lib().oracle_f16_to_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def scores(emb: np.ndarray, query: np.ndarray, n_threads: int = 0) -> np.ndarray:
+    """Double-precision inner product of one query with every row of ``emb``."""
+    emb = np.ascontiguousarray(emb)
+    query = np.ascontiguousarray(query, dtype=emb.dtype).reshape(-1)
+    n, e = emb.shape
+    assert query.size == e
+    out = np.empty(n, dtype=np.float64)
+    if n:
+        rc = lib().oracle_scores(_ptr(emb), _emb_dtype(emb), n, e, _ptr(query), _ptr(out), n_threads)
+        if rc:
+            raise OracleError(rc)
+    return out
+
+
+def retrieve(emb: np.ndarray, queries: np.ndarray, k: int, row_ids: np.ndarray | None = None, n_threads: int = 0):
+    """Top-k by (score descending, id ascending); returns (ids int32 [nq,k], scores float32 [nq,k])."""
+    emb = np.ascontiguousarray(emb)
+    queries = np.ascontiguousarray(queries, dtype=emb.dtype)
+    if queries.ndim == 1:
+        queries = queries[None]
+    n, e = emb.shape
+    nq = queries.shape[0]
+    if row_ids is not None:
+        row_ids = np.ascontiguousarray(row_ids, dtype=np.int32)
+        assert row_ids.size == n
+    ids = np.empty((nq, k), dtype=np.int32)
+    sc = np.empty((nq, k), dtype=np.float32)
+    rc = lib().oracle_retrieve(
+        _ptr(emb), _emb_dtype(emb), n, e, _ptr(row_ids), _ptr(queries), nq, k, _ptr(ids), _ptr(sc), n_threads
+    )
+    if rc:
+        raise OracleError(rc)
+    return ids, sc
+
+
+def inv_freq(D: int, theta: float) -> np.ndarray:
+    out = np.empty(D // 2, dtype=np.float32)
+    lib().oracle_inv_freq(D, float(theta), _ptr(out))
+    return out
+
+
+def rope_rows(x: np.ndarray, pos: np.ndarray, theta: float, style: int = 0, inv_freq_override=None) -> np.ndarray:
+    """Rotate rows of ``x`` ([n, D] float64), row r at position ``pos[r]``."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    n, D = x.shape
+    pos = np.ascontiguousarray(np.broadcast_to(np.asarray(pos, dtype=np.int64), (n,)))
+    if inv_freq_override is not None:
+        inv_freq_override = np.ascontiguousarray(inv_freq_override, dtype=np.float32)
+        assert inv_freq_override.size == D // 2
+    y = np.empty_like(x)
+    rc = lib().oracle_rope_rows(_ptr(x), n, D, _ptr(pos), float(theta), style, _ptr(inv_freq_override), _ptr(y))
+    if rc:
+        raise OracleError(rc)
+    return y
+
+
+class InjectResult:
+    """m, slots [m], k_ref float64 / k_bf16 uint16 / v uint16, each [nl, m, H, D]."""
+
+    def __init__(self, m, slots, k_ref, k_bf16, v):
+        self.m, self.slots, self.k_ref, self.k_bf16, self.v = m, slots, k_ref, k_bf16, v
+
+
+def inject(
+    ids,
+    fact_offset,
+    fact_len,
+    k_pre,
+    v,
+    theta,
+    start_pos,
+    block_table,
+    bs,
+    num_blocks,
+    style=0,
+    inv_freq_override=None,
+    layers=None,
+    want_ref=True,
+    k_cache=None,
+    v_cache=None,
+    cache_strides=None,
+    n_threads=0,
+) -> InjectResult:
+    """Compose facts ``ids`` (placement order) at ``start_pos`` and place them through ``block_table``.
+
+    ``k_pre`` / ``v``: uint16 (bf16 bits) arrays [n_layers, store_tokens, H, D] on the host.
+    ``k_cache`` / ``v_cache``: optional uint16 host images of the paged cache, written in place using
+    ``cache_strides = (layer, block, token, head)`` in elements.
+    """
+    ids = np.ascontiguousarray(ids, dtype=np.int32).reshape(-1)
+    fact_offset = np.ascontiguousarray(fact_offset, dtype=np.int64)
+    fact_len = np.ascontiguousarray(fact_len, dtype=np.int32)
+    assert k_pre.dtype == np.uint16 and v.dtype == np.uint16 and k_pre.shape == v.shape
+    k_pre = np.ascontiguousarray(k_pre)
+    v = np.ascontiguousarray(v)
+    n_layers, store_tokens, H, D = k_pre.shape
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32).reshape(-1)
+    l0, l1 = (0, n_layers) if layers is None else layers
+    nl = l1 - l0
+    if inv_freq_override is not None:
+        inv_freq_override = np.ascontiguousarray(inv_freq_override, dtype=np.float32)
+    valid = ids[(ids >= 0) & (ids < fact_len.size)]
+    m_guess = int(fact_len[valid].sum())
+    slots = np.empty(m_guess, dtype=np.int64)
+    shape = (nl, m_guess, H, D)
+    k_ref = np.empty(shape, dtype=np.float64) if want_ref else None
+    k_bf16 = np.empty(shape, dtype=np.uint16)
+    v_out = np.empty(shape, dtype=np.uint16)
+    m = C.c_int64(0)
+    strides = (0, 0, 0, 0)
+    if k_cache is not None or v_cache is not None:
+        assert cache_strides is not None
+        strides = tuple(int(s) for s in cache_strides)
+        for c_ in (k_cache, v_cache):
+            assert c_ is None or (c_.dtype == np.uint16 and c_.flags.c_contiguous)
+    rc = lib().oracle_inject(
+        _ptr(ids), ids.size, fact_len.size, _ptr(fact_offset), _ptr(fact_len), _ptr(k_pre), _ptr(v), store_tokens,
+        n_layers, H, D, float(theta), style, _ptr(inv_freq_override), int(start_pos), _ptr(block_table),
+        block_table.size, bs, num_blocks, l0, l1, C.byref(m), _ptr(slots), _ptr(k_ref), _ptr(k_bf16), _ptr(v_out),
+        _ptr(k_cache), _ptr(v_cache), *strides, n_threads,
+    )  # fmt: skip
+    if rc:
+        raise OracleError(rc)
+    assert m.value == m_guess
+    return InjectResult(m.value, slots, k_ref, k_bf16, v_out)

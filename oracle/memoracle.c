@@ -1,0 +1,367 @@
+/*
+ * CPU oracle for the retrieve + Chunked-RoPE KV-injection path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+ * CUDA library is compared against.  It shares no code, header, table or
+ * constant with the CUDA path and must never be called from the product path;
+ * only the tests, the smoke check and the CPU-baseline leg of the benchmark
+ * may load it.
+ *
+ * Everything is computed in double precision, one pass, no blocking, no
+ * fusion.  The optional OpenMP pragmas only split the outermost independent
+ * loop (facts, or tokens); they do not change any value.
+ *
+ * What follows which passage of the paper:
+ *   - scoring / top-k:  "Persistent memory store and retrieval" (Sec. 3.2):
+ *     a top-k search by inner product over the fact embeddings that returns
+ *     fact ids.  Exact search replaces the graph index; ties go to the lower id.
+ *   - RoPE:             "Rotary position embeddings" (Sec. 2.4) and the proof
+ *     sketch of Theorem 2 (Chunked RoPE Injection): a block-diagonal rotation
+ *     R_p with one frequency per 2-d pair, applied after the key projection.
+ *   - positions:        "Position policy" (Sec. 5.2): facts are contiguous,
+ *     fact i starts at b_i = sum_{j<i} |C_j|, total m = sum_i |C_i|.
+ *   - paged placement:  "Paged attention and KV cache management" (Sec. 2.2)
+ *     and the worker side of the connector (Sec. 3.4): a token at position
+ *     pos lives in slot block_table[pos / bs] * bs + pos % bs.
+ *   - V is stored raw and copied unchanged (Sec. 5.1, closing paragraph).
+ *   - bytes per fact:   "Storage cost" (Sec. 3.5): 2 * L * c * h * d * b.
+ *
+ * Parity pins: every exported function is pinned by the CPU tests
+ * (closed forms, group law, brute-force joint rotation, numpy float64
+ * cross-checks, full-sort comparison); none is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG -1
+#define ORACLE_ERR_BLOCK_TABLE -2 /* position needs a block-table entry that is not there */
+#define ORACLE_ERR_BLOCK_ID -3    /* block id outside the pool */
+#define ORACLE_ERR_FACT_ID -4     /* id outside the fact table */
+#define ORACLE_ERR_NOMEM -5
+
+enum { ORACLE_F32 = 0, ORACLE_F16 = 1 };
+
+/* ---------------------------------------------------------------- number formats */
+
+/* IEEE binary16 -> double, exact. */
+static double f16_to_double(uint16_t h) {
+  int sign = (h >> 15) & 1;
+  int exp = (h >> 10) & 0x1f;
+  int man = h & 0x3ff;
+  double v;
+  if (exp == 0) {
+    v = ldexp((double)man, -24); /* subnormal: man * 2^-10 * 2^-14 */
+  } else if (exp == 31) {
+    v = man ? NAN : INFINITY;
+  } else {
+    v = ldexp((double)(man | 0x400), exp - 25); /* (1024+man) * 2^(exp-15-10) */
+  }
+  return sign ? -v : v;
+}
+
+/* bfloat16 -> double, exact (bfloat16 is the upper half of a binary32). */
+static double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* double -> bfloat16 with ONE round-to-nearest-even (no intermediate float). */
+static uint16_t double_to_bf16_rne(double x) {
+  if (isnan(x)) return 0x7fc0;
+  uint16_t sign = signbit(x) ? 0x8000 : 0;
+  double a = fabs(x);
+  if (isinf(a)) return sign | 0x7f80;
+  if (a == 0.0) return sign;
+  int e;
+  (void)frexp(a, &e);       /* a = f * 2^e, f in [0.5, 1): leading bit has weight 2^(e-1) */
+  int lead = e - 1;
+  if (lead < -126) lead = -126; /* subnormal range of bfloat16 shares the quantum of 2^-126 */
+  double quantum = ldexp(1.0, lead - 7); /* 8 significant bits */
+  double q = nearbyint(a / quantum);     /* default rounding mode: ties to even */
+  double y = q * quantum;
+  float f = (float)y; /* exact: y has at most 8 significant bits */
+  if (isinf(f) || y >= ldexp(1.0, 128)) return sign | 0x7f80;
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return sign | (uint16_t)(u >> 16);
+}
+
+void oracle_bf16_from_double(const double* x, int64_t n, uint16_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = double_to_bf16_rne(x[i]);
+}
+void oracle_bf16_to_double(const uint16_t* x, int64_t n, double* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = bf16_to_double(x[i]);
+}
+void oracle_f16_to_double(const uint16_t* x, int64_t n, double* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = f16_to_double(x[i]);
+}
+
+static void set_threads(int n_threads) {
+#ifdef _OPENMP
+  if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+  (void)n_threads;
+#endif
+}
+int oracle_max_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------- storage cost */
+
+/* Sec. 3.5: a fact of c tokens stores 2 * L * c * h * d * b bytes of KV. */
+int64_t oracle_kv_bytes(int64_t L, int64_t c, int64_t h, int64_t d, int64_t b) {
+  return 2 * L * c * h * d * b;
+}
+
+/* ---------------------------------------------------------------- retrieval */
+
+static double emb_at(const void* emb, int dtype, int64_t idx) {
+  if (dtype == ORACLE_F32) return (double)((const float*)emb)[idx];
+  return f16_to_double(((const uint16_t*)emb)[idx]);
+}
+
+/* s[f] = sum_d q[d] * emb[f][d], accumulated left to right in double. */
+int oracle_scores(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim, const void* query,
+                  double* out_scores, int n_threads) {
+  if (!emb || !query || !out_scores || n_facts < 0 || emb_dim <= 0) return ORACLE_ERR_ARG;
+  if (emb_dtype != ORACLE_F32 && emb_dtype != ORACLE_F16) return ORACLE_ERR_ARG;
+  set_threads(n_threads);
+#pragma omp parallel for schedule(static)
+  for (int64_t f = 0; f < n_facts; ++f) {
+    double s = 0.0;
+    for (int d = 0; d < emb_dim; ++d) s += emb_at(query, emb_dtype, d) * emb_at(emb, emb_dtype, f * emb_dim + d);
+    out_scores[f] = s;
+  }
+  return ORACLE_OK;
+}
+
+typedef struct {
+  double s;
+  int32_t id;
+} scored_t;
+
+static int cmp_scored(const void* a, const void* b) {
+  const scored_t* x = (const scored_t*)a;
+  const scored_t* y = (const scored_t*)b;
+  if (x->s > y->s) return -1; /* higher score first */
+  if (x->s < y->s) return 1;
+  if (x->id < y->id) return -1; /* equal score: lower id first */
+  if (x->id > y->id) return 1;
+  return 0;
+}
+
+/*
+ * For each of nq queries: score every fact, sort ALL facts by (score desc, id asc),
+ * return the first k ids and their scores rounded to float; pad with id -1 / score 0
+ * when there are fewer than k facts.  row_ids[f] is the fact id of embedding row f
+ * (NULL: the row index is the id).
+ */
+int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim, const int32_t* row_ids,
+                    const void* queries, int nq, int k, int32_t* out_ids, float* out_scores, int n_threads) {
+  if (nq < 0 || k < 0 || !out_ids) return ORACLE_ERR_ARG;
+  if (n_facts > 0 && (!emb || !queries)) return ORACLE_ERR_ARG;
+  size_t esz = emb_dtype == ORACLE_F32 ? 4 : 2;
+  double* s = (double*)malloc(sizeof(double) * (size_t)(n_facts > 0 ? n_facts : 1));
+  scored_t* all = (scored_t*)malloc(sizeof(scored_t) * (size_t)(n_facts > 0 ? n_facts : 1));
+  if (!s || !all) {
+    free(s);
+    free(all);
+    return ORACLE_ERR_NOMEM;
+  }
+  for (int q = 0; q < nq; ++q) {
+    if (n_facts > 0) {
+      int rc = oracle_scores(emb, emb_dtype, n_facts, emb_dim, (const char*)queries + (size_t)q * emb_dim * esz, s,
+                             n_threads);
+      if (rc != ORACLE_OK) {
+        free(s);
+        free(all);
+        return rc;
+      }
+    }
+    for (int64_t f = 0; f < n_facts; ++f) {
+      all[f].s = s[f];
+      all[f].id = row_ids ? row_ids[f] : (int32_t)f;
+    }
+    qsort(all, (size_t)n_facts, sizeof(scored_t), cmp_scored);
+    for (int r = 0; r < k; ++r) {
+      if (r < n_facts) {
+        out_ids[(size_t)q * k + r] = all[r].id;
+        if (out_scores) out_scores[(size_t)q * k + r] = (float)all[r].s;
+      } else {
+        out_ids[(size_t)q * k + r] = -1;
+        if (out_scores) out_scores[(size_t)q * k + r] = 0.0f;
+      }
+    }
+  }
+  free(s);
+  free(all);
+  return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------- RoPE */
+
+/*
+ * Frequency of pair i: theta^(-2i/D), evaluated in double and rounded ONCE to
+ * binary32 (models keep this vector in fp32).  An override vector replaces it.
+ */
+static double pair_freq(int i, int D, double theta, const float* inv_freq_override) {
+  if (inv_freq_override) return (double)inv_freq_override[i];
+  return (double)(float)pow(theta, -(double)(2 * i) / (double)D);
+}
+
+void oracle_inv_freq(int D, double theta, float* out) {
+  for (int i = 0; i < D / 2; ++i) out[i] = (float)pair_freq(i, D, theta, NULL);
+}
+
+/*
+ * Rotate one head vector x[0..D) at position pos into y.
+ * style 0 (half-split): pair i is (x[i], x[i + D/2]);  style 1 (interleaved): (x[2i], x[2i+1]).
+ * (x1, x2) -> (x1 cos a - x2 sin a,  x2 cos a + x1 sin a),  a = pos * freq_i.
+ */
+static void rope_head(const double* x, double* y, int D, int64_t pos, double theta, int style,
+                      const float* inv_freq_override) {
+  int half = D / 2;
+  for (int i = 0; i < half; ++i) {
+    int i1 = style == 0 ? i : 2 * i;
+    int i2 = style == 0 ? i + half : 2 * i + 1;
+    double angle = (double)pos * pair_freq(i, D, theta, inv_freq_override);
+    double c = cos(angle), s = sin(angle);
+    double x1 = x[i1], x2 = x[i2];
+    y[i1] = x1 * c - x2 * s;
+    y[i2] = x2 * c + x1 * s;
+  }
+}
+
+/* Rotate n_rows independent head vectors (row r at position pos[r]). */
+int oracle_rope_rows(const double* x, int64_t n_rows, int D, const int64_t* pos, double theta, int style,
+                     const float* inv_freq_override, double* y) {
+  if (!x || !y || !pos || D <= 0 || (D & 1) || (style != 0 && style != 1)) return ORACLE_ERR_ARG;
+  for (int64_t r = 0; r < n_rows; ++r) rope_head(x + r * D, y + r * D, D, pos[r], theta, style, inv_freq_override);
+  return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------- injection */
+
+/*
+ * Compose the facts `ids` (placement order; negative ids are skipped) at positions
+ * start_pos, start_pos+1, ... and place every token in the paged cache.
+ *
+ * Store side (host arrays): fact f owns tokens [fact_offset[f], fact_offset[f] + fact_len[f])
+ * of k_pre / v, both bf16 with layout [n_layers][store_tokens][H][D].
+ *
+ * Only layers [layer_begin, layer_end) are produced (lets a caller bound memory); nl = their count.
+ * Outputs, all optional except out_m:
+ *   out_slots   [m]              slot of every composed token
+ *   out_k_ref   [nl][m][H][D]    rotated keys in double (before any rounding)
+ *   out_k_bf16  [nl][m][H][D]    the same rounded once to bf16 (round-to-nearest-even)
+ *   out_v       [nl][m][H][D]    values, bit copies
+ *   k_cache / v_cache            a host image of the paged cache (bf16), written in place at
+ *                                layer*layer_stride + block*block_stride + (slot % bs)*token_stride
+ *                                + head*head_stride + d   (strides in elements; layer = absolute index)
+ * Returns ORACLE_OK or a negative error; on error the outputs are unspecified.
+ */
+int oracle_inject(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
+                  const uint16_t* k_pre, const uint16_t* v, int64_t store_tokens, int n_layers, int H, int D,
+                  double theta, int style, const float* inv_freq_override, int64_t start_pos,
+                  const int32_t* block_table, int64_t n_table, int bs, int64_t num_blocks, int layer_begin,
+                  int layer_end, int64_t* out_m, int64_t* out_slots, double* out_k_ref, uint16_t* out_k_bf16,
+                  uint16_t* out_v, uint16_t* k_cache, uint16_t* v_cache, int64_t layer_stride, int64_t block_stride,
+                  int64_t token_stride, int64_t head_stride, int n_threads) {
+  if (!out_m || k < 0 || (k > 0 && !ids) || !fact_offset || !fact_len || H <= 0 || D <= 0 || (D & 1) || D > 1024 ||
+      bs <= 0)
+    return ORACLE_ERR_ARG;
+  if (layer_begin < 0 || layer_end > n_layers || layer_begin > layer_end) return ORACLE_ERR_ARG;
+  if (start_pos < 0) return ORACLE_ERR_ARG;
+
+  /* Position policy: m = sum of the lengths of the facts that are placed. */
+  int64_t m = 0;
+  for (int i = 0; i < k; ++i) {
+    if (ids[i] < 0) continue;
+    if (ids[i] >= n_facts) return ORACLE_ERR_FACT_ID;
+    m += fact_len[ids[i]];
+  }
+  *out_m = m;
+  if (m == 0) return ORACLE_OK;
+  if (!block_table || !k_pre || !v) return ORACLE_ERR_ARG;
+
+  /* token t of the composed segment comes from store token src[t] */
+  int64_t* src = (int64_t*)malloc(sizeof(int64_t) * (size_t)m);
+  int64_t* slots = (int64_t*)malloc(sizeof(int64_t) * (size_t)m);
+  if (!src || !slots) {
+    free(src);
+    free(slots);
+    return ORACLE_ERR_NOMEM;
+  }
+  int64_t t = 0;
+  for (int i = 0; i < k; ++i) {
+    if (ids[i] < 0) continue;
+    int32_t f = ids[i];
+    for (int32_t j = 0; j < fact_len[f]; ++j, ++t) {
+      int64_t pos = start_pos + t; /* = start_pos + b_i + j */
+      int64_t bi = pos / bs;
+      if (bi >= n_table) {
+        free(src);
+        free(slots);
+        return ORACLE_ERR_BLOCK_TABLE;
+      }
+      int64_t blk = block_table[bi];
+      if (blk < 0 || blk >= num_blocks) {
+        free(src);
+        free(slots);
+        return ORACLE_ERR_BLOCK_ID;
+      }
+      if (fact_offset[f] + j >= store_tokens) {
+        free(src);
+        free(slots);
+        return ORACLE_ERR_ARG;
+      }
+      src[t] = fact_offset[f] + j;
+      slots[t] = blk * bs + pos % bs;
+    }
+  }
+  if (out_slots) memcpy(out_slots, slots, sizeof(int64_t) * (size_t)m);
+
+  int64_t row = (int64_t)H * D;
+  set_threads(n_threads);
+#pragma omp parallel for schedule(static)
+  for (int64_t tt = 0; tt < m; ++tt) {
+    double xin[1024], yout[1024]; /* one head */
+    int64_t pos = start_pos + tt;
+    for (int l = layer_begin; l < layer_end; ++l) {
+      const uint16_t* ksrc = k_pre + ((int64_t)l * store_tokens + src[tt]) * row;
+      const uint16_t* vsrc = v + ((int64_t)l * store_tokens + src[tt]) * row;
+      int64_t o = ((int64_t)(l - layer_begin) * m + tt) * row; /* compact outputs */
+      int64_t blk = slots[tt] / bs, inb = slots[tt] % bs;
+      int64_t cbase = (int64_t)l * layer_stride + blk * block_stride + inb * token_stride;
+      for (int h = 0; h < H; ++h) {
+        for (int d = 0; d < D; ++d) xin[d] = bf16_to_double(ksrc[h * D + d]);
+        rope_head(xin, yout, D, pos, theta, style, inv_freq_override);
+        for (int d = 0; d < D; ++d) {
+          uint16_t kb = double_to_bf16_rne(yout[d]);
+          uint16_t vb = vsrc[h * D + d];
+          if (out_k_ref) out_k_ref[o + h * D + d] = yout[d];
+          if (out_k_bf16) out_k_bf16[o + h * D + d] = kb;
+          if (out_v) out_v[o + h * D + d] = vb;
+          if (k_cache) k_cache[cbase + h * head_stride + d] = kb;
+          if (v_cache) v_cache[cbase + h * head_stride + d] = vb;
+        }
+      }
+    }
+  }
+  free(src);
+  free(slots);
+  return ORACLE_OK;
+}
