@@ -1,0 +1,190 @@
+/*
+ * memstore.h - C ABI of libmemstore.so: an HBM-resident fact store with exact top-k
+ * retrieval and fused Chunked-RoPE injection into a paged KV cache (NVIDIA B200, sm_100a).
+ *
+ * The calls follow the paper's statement of the serving path:
+ *   - a store keyed by fact id that holds, per fact, one retrieval embedding and the fact's
+ *     PRE-rotation keys and raw values for every layer, with no positional metadata
+ *     ("Persistent memory store and retrieval", Sec. 3.2; "Position-agnostic storage", Sec. 5.1);
+ *   - a top-k search by inner product that returns fact ids (Sec. 3.2);
+ *   - composition of the retrieved facts at contiguous positions with RoPE applied to the stored
+ *     keys at those positions ("Chunked-RoPE composition", Sec. 3.3; Theorem 2; "Position policy",
+ *     Sec. 5.2), and a scatter of K and V into the request's paged blocks through the slot mapping
+ *     (Sec. 2.2; worker side of the connector, Sec. 3.4).
+ *
+ * Conventions
+ *   - Every call returns an ms_status and never throws or aborts.  memstore_last_error() gives text.
+ *   - "device" pointers are CUDA device pointers on the store's device; "host" pointers are ordinary
+ *     host memory.  Nothing here takes a framework tensor.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  retrieve and
+ *     inject only ENQUEUE work on it and never synchronise with the host; ids flow device to device.
+ *   - Errors the host can see (bad arguments, capacity) are returned at once and enqueue nothing.
+ *     Errors that depend on device data (a bad id inside a request, a block table that is too
+ *     short ...) set bits in that request's status word and SKIP the offending tokens; the kernels
+ *     never read or write out of bounds, never trap and contain no unbounded wait.
+ *   - The store copies what add_fact(s) is given; the caller keeps ownership of its buffers.  The
+ *     caller owns queries, id lists, block tables and the paged cache.
+ *   - Fact ids are dense int32 numbers assigned in insertion order, global across users.  The store
+ *     is append-only (the paper's store is built once and then read).
+ *   - Calls on one store may be issued from several streams; the store orders them on the device
+ *     (they share scratch memory).  add_fact(s) must not run concurrently with other calls from
+ *     another host thread.
+ *   - There is no CPU fallback: every step runs in CUDA kernels of this library.
+ */
+#ifndef MEMSTORE_H
+#define MEMSTORE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct memstore memstore_t;
+typedef void* ms_stream; /* cudaStream_t */
+
+typedef enum {
+  MS_OK = 0,
+  MS_ERR_INVALID_ARG = 1,
+  MS_ERR_UNSUPPORTED = 2,
+  MS_ERR_OOM = 3,      /* device or host allocation failed */
+  MS_ERR_CAPACITY = 4, /* store full: facts per user or KV arena tokens */
+  MS_ERR_CUDA = 5
+} ms_status;
+
+/* per-request status bits written by memstore_inject (0 = clean) */
+enum {
+  MS_REQ_BAD_FACT_ID = 1,       /* id >= number of facts: contributes no tokens */
+  MS_REQ_NOT_RESIDENT = 2,      /* fact has no K/V in the arena: contributes no tokens */
+  MS_REQ_BLOCK_TABLE_SHORT = 4, /* pos / block_size >= max_blocks: token skipped */
+  MS_REQ_BAD_BLOCK_ID = 8,      /* table entry < 0 or >= num_blocks: token skipped */
+  MS_REQ_POSITION_OVERFLOW = 16 /* pos >= max_position: token skipped */
+};
+
+enum { MS_DTYPE_F32 = 0, MS_DTYPE_F16 = 1, MS_DTYPE_BF16 = 2 };
+enum { MS_ROPE_HALF_SPLIT = 0, MS_ROPE_INTERLEAVED = 1 };
+enum { MS_INJECT_REVERSE = 1u }; /* place ids[k-1] first, so that ids[0] ends next to the query */
+
+typedef struct {
+  int32_t device;         /* CUDA device ordinal */
+  int32_t n_layers;       /* L */
+  int32_t n_kv_heads;     /* h */
+  int32_t head_dim;       /* d: a multiple of 16, at most 512 */
+  int32_t kv_dtype;       /* MS_DTYPE_BF16 only (the paper's cache is bf16) */
+  int32_t emb_dim;        /* a multiple of 8 */
+  int32_t emb_dtype;      /* MS_DTYPE_F32 or MS_DTYPE_F16 */
+  int32_t rope_style;     /* MS_ROPE_HALF_SPLIT pairs (i, i+d/2); MS_ROPE_INTERLEAVED pairs (2i, 2i+1) */
+  double rope_theta;      /* frequency of pair i is theta^(-2i/d), rounded once to fp32 */
+  const float* inv_freq_override; /* host, d/2 floats, or NULL; replaces the formula above (copied) */
+  int64_t max_position;   /* tokens at pos >= max_position are refused; 0 < max_position <= 2^24 */
+  int32_t n_users;        /* number of private embedding segments (>= 1) */
+  int32_t reserved0;
+  int64_t max_facts_per_user; /* capacity of each user's embedding segment */
+  int64_t max_kv_tokens;  /* capacity of the K/V arena in tokens (0: embedding-only store) */
+  void* kv_arena;         /* optional caller-provided DEVICE buffer for the arena, else NULL */
+  size_t kv_arena_bytes;  /* its size; must be >= memstore_arena_bytes(config) */
+} memstore_config;
+
+/* Bytes of the K/V arena for this configuration: 2 * L * max_kv_tokens * h * d * 2
+ * (the paper's storage formula, Sec. 3.5, with c = max_kv_tokens and bf16). */
+size_t memstore_arena_bytes(const memstore_config* config);
+
+/* Create a store on config->device.  Allocates the arena (unless given), the embedding segments
+ * and the fact table with cudaMalloc.  *out is NULL on failure. */
+ms_status memstore_create(const memstore_config* config, memstore_t** out);
+ms_status memstore_destroy(memstore_t* store);
+
+/*
+ * Append one fact to `user`'s segment (Sec. 3.1/3.2: a fact is an embedding plus the fact's slice of
+ * pre-RoPE K and raw V).
+ *   emb    device, [emb_dim] in emb_dtype
+ *   k_pre  device, bf16, [n_layers][n_tokens][n_kv_heads][head_dim], keys BEFORE any rotation
+ *   v      device, bf16, same layout
+ * k_pre == v == NULL with n_tokens == 0 adds an embedding-only fact (not resident: it can be
+ * retrieved but not injected).  *out_fact_id (host, optional) receives the new id.
+ * Copies are enqueued on `stream`; the source buffers may be reused once the stream has passed them.
+ */
+ms_status memstore_add_fact(memstore_t* store, int32_t user, const void* emb, const void* k_pre, const void* v,
+                            int32_t n_tokens, int32_t* out_fact_id, ms_stream stream);
+
+/*
+ * Append n facts to `user`'s segment in one call.
+ *   embs      device, [n][emb_dim]
+ *   n_tokens  HOST, [n]; 0 marks an embedding-only fact
+ *   k_pre, v  device, bf16, [n_layers][T][n_kv_heads][head_dim] with T = sum(n_tokens): the facts' tokens
+ *             one after another along the token axis (NULL allowed when T == 0)
+ * *out_first_id (host, optional) receives the id of the first fact; the others follow densely.
+ */
+ms_status memstore_add_facts(memstore_t* store, int32_t user, int64_t n, const void* embs, const void* k_pre,
+                             const void* v, const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream);
+
+/*
+ * Score each query against every fact of its user by inner product and select the k best
+ * (Sec. 3.2; exact search instead of the paper's graph index).
+ *   queries      device, [nq][emb_dim] in emb_dtype
+ *   query_users  device int32 [nq], or NULL (every query searches user 0)
+ *   out_ids      device int32 [nq][k]: rank 0 = highest score; equal scores: lower fact id first;
+ *                padded with -1 when the user has fewer than k facts
+ *   out_scores   device fp32 [nq][k] or NULL (0 where the id is -1)
+ * Products of the stored values are accumulated in fp32.  1 <= k <= 2048.
+ */
+ms_status memstore_retrieve(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                            int32_t* out_ids, float* out_scores, ms_stream stream);
+
+/* A caller-owned paged KV cache, bf16, described by strides in ELEMENTS:
+ *   element (layer, block, token-in-block, head, d) of K is at
+ *   k_base[layer*layer_stride + block*block_stride + token*token_stride + head*head_stride + d]
+ * and the same for V from v_base.  All strides must be multiples of 8 and the bases 16-byte aligned.
+ * This covers separate K/V planes, stacked planes, token-major and head-major blocks. */
+typedef struct {
+  void* k_base;
+  void* v_base;
+  int64_t layer_stride, block_stride, token_stride, head_stride;
+  int64_t num_blocks;
+  int32_t block_size;
+  int32_t reserved0;
+} ms_paged_cache;
+
+/*
+ * For each of nreq requests, compose its facts and write them into the paged cache
+ * (Sec. 3.3, Theorem 2, Sec. 5.2, Sec. 3.4):
+ *   facts are laid out contiguously in the order given, fact i starting at b_i = sum_{j<i} n_j;
+ *   token j of fact i gets pos = start_pos + b_i + j and slot = block_table[pos / bs] * bs + pos % bs;
+ *   K rows are rotated by RoPE at pos (fp32 arithmetic on the stored bf16 values, cos/sin evaluated
+ *   on the fly, one round-to-nearest-even to bf16), V rows are copied bit for bit.
+ *
+ *   fact_ids      device int32 [nreq][k], placement order; entries < 0 are skipped
+ *   start_pos     device int32 [nreq]
+ *   block_tables  device int32 [nreq][max_blocks]
+ *   out_n_tokens  device int32 [nreq] or NULL: m = number of tokens composed (including skipped ones)
+ *   out_status    device int32 [nreq] or NULL: MS_REQ_* bits
+ *   out_slot_mapping  device int64 [nreq][slot_stride] or NULL: slot of each composed token
+ *                 (-1 for a skipped token; entries beyond min(m, slot_stride) are not written)
+ *   flags         MS_INJECT_REVERSE: place ids in reverse order (the paper's policy for a best-first list)
+ * Two requests that map to the same cache slot race (last writer wins, undetected).
+ */
+ms_status memstore_inject(memstore_t* store, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
+                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
+                          int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
+                          uint32_t flags, ms_stream stream);
+
+/* Counters since creation (host side; bytes are the algorithmic ones, not measured traffic). */
+typedef struct {
+  int64_t n_facts, n_resident_facts, kv_tokens_used;
+  int64_t retrieve_calls, inject_calls;
+  int64_t kernels_launched; /* kernels of this library enqueued so far */
+  int64_t arena_bytes, embedding_bytes;
+} memstore_stats_t;
+ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
+
+/* Text of the last error on this store (never NULL; valid until the next call on the store). */
+const char* memstore_last_error(memstore_t* store);
+
+/* Library version string, e.g. "memstore 0.1 sm_100a". */
+const char* memstore_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEMSTORE_H */

@@ -1,0 +1,56 @@
+// Shared device-side definitions of libmemstore (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ms {
+
+// One row of the device fact table (the paper keeps this id -> location map on the CPU, Sec. 6.7;
+// here it lives in HBM so that ids never leave the device).
+struct FactRec {
+  int32_t tok_off;   // first token of the fact in the K/V arena
+  int32_t n_tokens;  // length of the fact in tokens
+  int32_t user;      // owner segment
+  int32_t resident;  // 1: K/V present in the arena, 0: embedding only
+};
+
+// Tokens per injection tile: 16 consecutive positions aligned to a multiple of 16, so a tile never
+// straddles a cache block whose size is a multiple of 16 (and covers whole smaller power-of-two blocks).
+constexpr int kTileTokens = 16;
+
+// Work description of one tile, written by the plan kernel and read by the copy kernel.
+struct __align__(16) TileDesc {
+  int32_t pos0;                 // position of lane 0 (multiple of kTileTokens)
+  int32_t pad[3];
+  int32_t src_tok[kTileTokens]; // arena token of each lane, -1: nothing to do
+  int64_t dst_off[kTileTokens]; // element offset block*block_stride + token*token_stride in the cache
+};
+
+// Counters shared by the plan and copy kernels of one inject call (reset by the last copy CTA).
+struct InjectCtrl {
+  uint32_t n_tiles;
+  uint32_t work_next;
+  uint32_t done_ctas;
+  uint32_t pad;
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+
+// Programmatic dependent launch: wait until the preceding kernel in the stream has completed and its
+// writes are visible / allow the next kernel in the stream to start its prologue.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::); }
+
+}  // namespace ms

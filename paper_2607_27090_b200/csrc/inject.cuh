@@ -1,0 +1,333 @@
+// Chunked-RoPE injection kernels: a small plan kernel (ids -> positions -> slots) followed by a
+// persistent gather / rotate / scatter kernel.  Paper: Sec. 3.3 (composition), Theorem 2 (chunked RoPE),
+// Sec. 5.2 (position policy), Sec. 2.2 and 3.4 (paged blocks, slot mapping).
+#pragma once
+#include "common.cuh"
+
+namespace ms {
+
+struct InjectParams {
+  // store
+  const FactRec* facts;
+  int32_t n_facts;
+  const __nv_bfloat16* k_arena;  // [L][arena_tokens][H][D]
+  const __nv_bfloat16* v_arena;
+  int64_t arena_tokens;
+  const float* inv_freq;  // [D/2]
+  int32_t n_layers, n_heads, head_dim, rope_style;
+  int32_t max_position;
+  // request
+  const int32_t* fact_ids;  // [nreq][k]
+  int32_t nreq, k;
+  const int32_t* start_pos;
+  const int32_t* block_tables;
+  int32_t max_blocks;
+  uint32_t flags;
+  // cache
+  __nv_bfloat16* k_cache;
+  __nv_bfloat16* v_cache;
+  int64_t layer_stride, block_stride, token_stride, head_stride, num_blocks;
+  int32_t block_size;
+  // outputs
+  int32_t* out_n_tokens;
+  int32_t* out_status;
+  int64_t* out_slot_mapping;
+  int64_t slot_stride;
+  // scratch
+  TileDesc* tiles;
+  uint32_t tiles_capacity;
+  InjectCtrl* ctrl;
+  int32_t layers_per_item;
+};
+
+constexpr int kPlanThreads = 256;
+constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by the plan kernel
+
+// ------------------------------------------------------------------------------------------------
+// Plan kernel: one CTA per request.
+//   I1 fact resolution (id -> arena offset, length), I2 exclusive scan of lengths (b_i, m),
+//   I3 slot = block_table[pos / bs] * bs + pos % bs, validation, tile descriptors.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectParams p) {
+  __shared__ int32_t s_begin[kPlanMaxK];  // b_i: first composed token of placed fact i
+  __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
+  __shared__ int32_t s_scan[kPlanThreads / 32];
+  __shared__ int32_t s_carry, s_status;
+  __shared__ uint32_t s_tile_base;
+
+  const int r = blockIdx.x;
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
+  if (tid == 0) {
+    s_carry = 0;
+    s_status = 0;
+  }
+  __syncthreads();
+
+  // lengths of the facts in placement order, exclusive scan in chunks of kPlanThreads
+  const int32_t* ids = p.fact_ids + (int64_t)r * p.k;
+  for (int base = 0; base < p.k; base += kPlanThreads) {
+    int j = base + tid;
+    int32_t len = 0, src = 0;
+    if (j < p.k) {
+      int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - j) : j];
+      if (id >= 0) {
+        if (id >= p.n_facts) {
+          atomicOr(&s_status, 1 /*MS_REQ_BAD_FACT_ID*/);
+        } else {
+          FactRec f = p.facts[id];
+          if (!f.resident) {
+            atomicOr(&s_status, 2 /*MS_REQ_NOT_RESIDENT*/);
+          } else {
+            len = f.n_tokens;
+            src = f.tok_off;
+          }
+        }
+      }
+    }
+    // block-wide exclusive scan of len
+    int32_t x = len;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) s_scan[warp] = x;
+    __syncthreads();
+    int32_t warp_off = 0;
+    for (int w = 0; w < warp; ++w) warp_off += s_scan[w];
+    int32_t carry = s_carry;
+    if (j < p.k) {
+      s_begin[j] = carry + warp_off + x - len;
+      s_src[j] = src;
+    }
+    __syncthreads();
+    if (tid == kPlanThreads - 1) s_carry = carry + warp_off + x;
+    __syncthreads();
+  }
+  const int32_t m = s_carry;
+  const int32_t start = p.start_pos[r];
+  const int32_t first_tile_pos = (start / kTileTokens) * kTileTokens;
+  const uint32_t n_tiles = m > 0 ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
+  if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->n_tiles, n_tiles) : 0u;
+  __syncthreads();
+  const uint32_t tile_base = s_tile_base;
+
+  const int bs = p.block_size;
+  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += kPlanThreads) {
+    const uint32_t t = e / kTileTokens, ln = e % kTileTokens;
+    const int32_t pos = first_tile_pos + (int32_t)e;
+    const int32_t q = pos - start;  // index in the composed segment
+    int32_t src_tok = -1;
+    int64_t dst = 0, slot = -1;
+    if (q >= 0 && q < m) {
+      // the fact that owns composed token q is the LAST i with b_i <= q: entries of length zero (skipped,
+      // unknown or non-resident ids) share their b_i with the next placed fact, and trailing ones have b_i = m > q
+      int lo = 0, hi = p.k - 1;
+      while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (s_begin[mid] <= q) lo = mid; else hi = mid - 1;
+      }
+      const int i = lo;
+      int32_t st = 0;
+      if (pos >= p.max_position) {
+        st = 16;  // MS_REQ_POSITION_OVERFLOW
+      } else {
+        int32_t bi = pos / bs;
+        if (bi >= p.max_blocks) {
+          st = 4;  // MS_REQ_BLOCK_TABLE_SHORT
+        } else {
+          int32_t blk = p.block_tables[(int64_t)r * p.max_blocks + bi];
+          if (blk < 0 || blk >= p.num_blocks) {
+            st = 8;  // MS_REQ_BAD_BLOCK_ID
+          } else {
+            src_tok = s_src[i] + (q - s_begin[i]);
+            dst = (int64_t)blk * p.block_stride + (int64_t)(pos % bs) * p.token_stride;
+            slot = (int64_t)blk * bs + pos % bs;
+          }
+        }
+      }
+      if (st) atomicOr(&s_status, st);
+      if (p.out_slot_mapping && q < p.slot_stride) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = slot;
+    }
+    if (tile_base + t < p.tiles_capacity) {
+      TileDesc* d = p.tiles + tile_base + t;
+      if (ln == 0) d->pos0 = first_tile_pos + (int32_t)(t * kTileTokens);
+      d->src_tok[ln] = src_tok;
+      d->dst_off[ln] = dst;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    if (p.out_n_tokens) p.out_n_tokens[r] = m;
+    if (p.out_status) p.out_status[r] = s_status;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// RoPE angle: pos * inv_freq formed EXACTLY as hi + lo, reduced by 2*pi with a three-constant
+// Cody-Waite scheme (each fma step is exact up to the last), then sin/cos of the reduced argument.
+// Naive fp32 pos*inv_freq is off by up to 0.5 rad-ulp of a 2^24-sized angle and is not usable.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void rope_sincos(float posf, float inv_freq, float& s, float& c) {
+  const float hi = __fmul_rn(posf, inv_freq);
+  const float lo = __fmaf_rn(posf, inv_freq, -hi);
+  const float n = rintf(hi * 0.15915494309189535f);
+  float r = __fmaf_rn(n, -6.28125f, hi);                  // exact
+  r = __fmaf_rn(n, -0.0019350051879882812f, r);           // exact
+  r = __fmaf_rn(n, -3.019916050561733e-07f, r);           // one rounding
+  r += lo;
+  if (r > 3.14159274f) r -= 6.28318548f;
+  if (r < -3.14159274f) r += 6.28318548f;
+  __sincosf(r, &s, &c);
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (low half), .y = hi
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Rotate one unit = two 16-byte vectors a, b of one head (8 frequencies sn[], cs[]).
+//   half-split : a = x[8j .. 8j+7], b = x[D/2+8j ..]; pair i is (a_i, b_i)
+//   interleaved: a = x[16j .. 16j+7] = pairs 8j..8j+3, b = x[16j+8 ..] = pairs 8j+4..8j+7
+template <int STYLE>
+__device__ __forceinline__ void rotate_unit(uint4& a, uint4& b, const float* sn, const float* cs) {
+  uint32_t* aw = reinterpret_cast<uint32_t*>(&a);
+  uint32_t* bw = reinterpret_cast<uint32_t*>(&b);
+  if (STYLE == 0) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      float x1l = bf16lo(aw[w]), x1h = bf16hi(aw[w]);
+      float x2l = bf16lo(bw[w]), x2h = bf16hi(bw[w]);
+      float y1l = x1l * cs[2 * w] - x2l * sn[2 * w];
+      float y2l = x2l * cs[2 * w] + x1l * sn[2 * w];
+      float y1h = x1h * cs[2 * w + 1] - x2h * sn[2 * w + 1];
+      float y2h = x2h * cs[2 * w + 1] + x1h * sn[2 * w + 1];
+      aw[w] = pack_bf16(y1l, y1h);
+      bw[w] = pack_bf16(y2l, y2h);
+    }
+  } else {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      float x1 = bf16lo(aw[w]), x2 = bf16hi(aw[w]);
+      aw[w] = pack_bf16(x1 * cs[w] - x2 * sn[w], x2 * cs[w] + x1 * sn[w]);
+      float z1 = bf16lo(bw[w]), z2 = bf16hi(bw[w]);
+      bw[w] = pack_bf16(z1 * cs[4 + w] - z2 * sn[4 + w], z2 * cs[4 + w] + z1 * sn[4 + w]);
+    }
+  }
+}
+
+constexpr int kCopyThreads = 256;
+constexpr int kThreadsPerToken = kCopyThreads / kTileTokens;  // 16
+
+// ------------------------------------------------------------------------------------------------
+// Copy kernel (I4 + I5): persistent CTAs over items = (tile, group of layers).
+// 16 threads serve one token; a thread owns units u = lane16, lane16+16, ... of the token's row, a unit
+// being (head, frequency octet): two 16-byte vectors of K (rotated) and the same two of V (copied).
+// UPT = units a thread keeps in flight at once.  Because 16 is a multiple of D/16 every unit of a thread has the
+// same frequency octet, so its 8 sin/cos pairs are computed once per item and reused over heads and layers.
+// ------------------------------------------------------------------------------------------------
+template <int STYLE, int UPT>
+__global__ void __launch_bounds__(kCopyThreads) inject_copy_kernel(const InjectParams p) {
+  const int tid = threadIdx.x;
+  const int tk = tid / kThreadsPerToken;
+  const int l16 = tid % kThreadsPerToken;
+  const int D = p.head_dim, H = p.n_heads;
+  const int G = D >> 4;  // frequency octets per head
+  const int row = H * D;
+  const int n_units = H * G;
+  const int j = l16 % G;  // this thread's octet (requires 16 % G == 0)
+  const int n_lgroups = (p.n_layers + p.layers_per_item - 1) / p.layers_per_item;
+
+  float f8[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) f8[i] = p.inv_freq[8 * j + i];
+  // element offsets of this thread's two vectors inside a head
+  const int offA = STYLE == 0 ? 8 * j : 16 * j;
+  const int offB = STYLE == 0 ? D / 2 + 8 * j : 16 * j + 8;
+
+  grid_dependency_wait();  // tile descriptors come from the plan kernel
+
+  const uint32_t n_tiles = min(p.ctrl->n_tiles, p.tiles_capacity);
+  const uint32_t n_items = n_tiles * (uint32_t)n_lgroups;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t tile = item / n_lgroups;
+    const int l0 = (int)(item % n_lgroups) * p.layers_per_item;
+    const int l1 = min(l0 + p.layers_per_item, p.n_layers);
+    const TileDesc* d = p.tiles + tile;
+    const int32_t src = d->src_tok[tk];
+    if (src < 0) continue;
+    const int64_t dst = d->dst_off[tk];
+    const float posf = (float)(d->pos0 + tk);
+    float sn[8], cs[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) rope_sincos(posf, f8[i], sn[i], cs[i]);
+
+    for (int l = l0; l < l1; ++l) {
+      const int64_t src_row = ((int64_t)l * p.arena_tokens + src) * row;
+      const __nv_bfloat16* ks = p.k_arena + src_row;
+      const __nv_bfloat16* vs = p.v_arena + src_row;
+      const int64_t dbase = (int64_t)l * p.layer_stride + dst;
+      for (int ub = l16; ub < n_units; ub += UPT * kThreadsPerToken) {
+        uint4 ka[UPT], kb[UPT], va[UPT], vb[UPT];
+#pragma unroll
+        for (int u = 0; u < UPT; ++u) {
+          const int unit = ub + u * kThreadsPerToken;
+          if (unit < n_units) {
+            const int h = unit / G;
+            ka[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offA));
+            kb[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offB));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < UPT; ++u) {
+          const int unit = ub + u * kThreadsPerToken;
+          if (unit < n_units) {
+            const int h = unit / G;
+            va[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offA));
+            vb[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offB));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < UPT; ++u) {
+          const int unit = ub + u * kThreadsPerToken;
+          if (unit < n_units) {
+            const int h = unit / G;
+            rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+            __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
+            st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
+            st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < UPT; ++u) {
+          const int unit = ub + u * kThreadsPerToken;
+          if (unit < n_units) {
+            const int h = unit / G;
+            __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
+            st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
+            st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
+          }
+        }
+      }
+    }
+  }
+
+  // Wait-free epilogue: the last CTA to get here clears the counters for the next inject call.
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const uint32_t done = atomicAdd(&p.ctrl->done_ctas, 1u);
+    if (done == gridDim.x - 1) {
+      p.ctrl->n_tiles = 0;
+      p.ctrl->work_next = 0;
+      p.ctrl->done_ctas = 0;
+      __threadfence();
+    }
+  }
+}
+
+}  // namespace ms

@@ -1,0 +1,503 @@
+// Host side of libmemstore.so: the fact store in HBM and the C ABI declared in include/memstore.h.
+// All compute is in the kernels of inject.cuh / retrieve.cuh; this file validates arguments, owns
+// device memory and enqueues launches.  There is no CPU implementation of any step.
+#include "../../include/memstore.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "inject.cuh"
+#include "retrieve.cuh"
+
+using namespace ms;
+
+struct memstore {
+  memstore_config cfg{};
+  int sm_count = 0;
+  // device memory
+  __nv_bfloat16* k_arena = nullptr;  // [L][max_kv_tokens][h][d]
+  __nv_bfloat16* v_arena = nullptr;
+  void* arena_alloc = nullptr;       // non-null when the store owns the arena
+  void* emb = nullptr;               // [n_users][max_facts_per_user][emb_dim]
+  int32_t* emb_fact_id = nullptr;    // [n_users][max_facts_per_user]
+  int32_t* user_count_d = nullptr;   // [n_users]
+  FactRec* facts_d = nullptr;        // [n_users * max_facts_per_user]
+  float* inv_freq_d = nullptr;       // [d/2]
+  // scratch shared by all calls (ordered on the device through `last_done`)
+  float* scores = nullptr;
+  int64_t scores_nq = 0;
+  TileDesc* tiles = nullptr;
+  uint32_t tiles_capacity = 0;
+  InjectCtrl* ctrl = nullptr;
+  cudaEvent_t last_done = nullptr;
+  cudaStream_t last_stream = nullptr;
+  bool have_last = false;
+  // host mirrors
+  std::vector<int64_t> user_count;
+  int64_t n_facts = 0, n_resident = 0, kv_tokens_used = 0;
+  int32_t max_fact_len = 0;
+  int64_t max_user_count = 0;
+  int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
+  int copy_ctas_per_sm = 1;
+  std::mutex mu;
+  std::string err;
+};
+
+namespace {
+
+ms_status fail(memstore* s, ms_status code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (s) s->err = buf;
+  return code;
+}
+
+#define MS_CUDA(s, call)                                                                         \
+  do {                                                                                           \
+    cudaError_t e_ = (call);                                                                     \
+    if (e_ != cudaSuccess)                                                                       \
+      return fail(s, e_ == cudaErrorMemoryAllocation ? MS_ERR_OOM : MS_ERR_CUDA, "%s: %s", #call, \
+                  cudaGetErrorString(e_));                                                       \
+  } while (0)
+
+size_t emb_elem_size(int dtype) { return dtype == MS_DTYPE_F32 ? 4 : 2; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+ms_status check_config(const memstore_config* c) {
+  if (!c) return MS_ERR_INVALID_ARG;
+  if (c->n_layers <= 0 || c->n_kv_heads <= 0 || c->emb_dim <= 0 || c->n_users <= 0) return MS_ERR_INVALID_ARG;
+  if (c->max_facts_per_user <= 0 || c->max_kv_tokens < 0) return MS_ERR_INVALID_ARG;
+  if (c->max_position <= 0 || c->max_position > (1 << 24)) return MS_ERR_INVALID_ARG;
+  if (c->rope_style != MS_ROPE_HALF_SPLIT && c->rope_style != MS_ROPE_INTERLEAVED) return MS_ERR_INVALID_ARG;
+  if (!(c->rope_theta > 0.0) && !c->inv_freq_override) return MS_ERR_INVALID_ARG;
+  if (c->kv_dtype != MS_DTYPE_BF16) return MS_ERR_UNSUPPORTED;
+  if (c->emb_dtype != MS_DTYPE_F32 && c->emb_dtype != MS_DTYPE_F16) return MS_ERR_UNSUPPORTED;
+  if (c->emb_dim % 8) return MS_ERR_UNSUPPORTED;
+  // the copy kernel gives 16 threads to a token and one frequency octet to a thread: d/16 must divide 16
+  const int d = c->head_dim;
+  if (!(d == 16 || d == 32 || d == 64 || d == 128 || d == 256)) return MS_ERR_UNSUPPORTED;
+  if (c->max_kv_tokens >= (1ll << 31) || (int64_t)c->n_users * c->max_facts_per_user >= (1ll << 31))
+    return MS_ERR_UNSUPPORTED;
+  return MS_OK;
+}
+
+// ---- arena append: src [L][T][row] -> arena [L][cap][row] at token offset, K and V in one launch ----
+__global__ void __launch_bounds__(256) arena_append_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
+                                                           uint4* __restrict__ k_dst, uint4* __restrict__ v_dst,
+                                                           int64_t vec_per_layer_src, int64_t vec_per_layer_dst,
+                                                           int64_t dst_vec_off) {
+  const int layer = blockIdx.y;
+  const uint4* s = (blockIdx.z ? v_src : k_src) + (int64_t)layer * vec_per_layer_src;
+  uint4* d = (blockIdx.z ? v_dst : k_dst) + (int64_t)layer * vec_per_layer_dst + dst_vec_off;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vec_per_layer_src; i += (int64_t)gridDim.x * blockDim.x)
+    d[i] = s[i];
+}
+
+template <int STYLE>
+void launch_copy(const InjectParams& p, int upt, dim3 grid, cudaLaunchConfig_t& lc, cudaError_t& e) {
+  lc.gridDim = grid;
+  switch (upt) {
+    case 1: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 1>, p); break;
+    case 2: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 2>, p); break;
+    default: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 4>, p); break;
+  }
+}
+
+// Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
+// stream than the previous one, an event recorded at the tail of the previous stream is waited for.
+ms_status order_after_last(memstore* s, cudaStream_t st) {
+  if (s->have_last && s->last_stream != st) {
+    MS_CUDA(s, cudaEventRecord(s->last_done, s->last_stream));
+    MS_CUDA(s, cudaStreamWaitEvent(st, s->last_done, 0));
+  }
+  return MS_OK;
+}
+ms_status mark_last(memstore* s, cudaStream_t st) {
+  s->last_stream = st;
+  s->have_last = true;
+  return MS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* memstore_version(void) { return "memstore 0.1 sm_100a"; }
+
+size_t memstore_arena_bytes(const memstore_config* c) {
+  if (!c) return 0;
+  return (size_t)2 * c->n_layers * (size_t)c->max_kv_tokens * c->n_kv_heads * c->head_dim * sizeof(__nv_bfloat16);
+}
+
+ms_status memstore_create(const memstore_config* config, memstore_t** out) {
+  if (out) *out = nullptr;
+  if (!out) return MS_ERR_INVALID_ARG;
+  ms_status st = check_config(config);
+  if (st != MS_OK) return st;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || config->device < 0 || config->device >= ndev) return MS_ERR_CUDA;
+  memstore* s = new (std::nothrow) memstore();
+  if (!s) return MS_ERR_OOM;
+  s->cfg = *config;
+  s->cfg.inv_freq_override = nullptr;
+  DeviceGuard g(config->device);
+  auto bail = [&](ms_status code) {
+    memstore_destroy(s);
+    return code;
+  };
+  if (!g.ok) return bail(MS_ERR_CUDA);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, config->device) != cudaSuccess) return bail(MS_ERR_CUDA);
+  s->sm_count = prop.multiProcessorCount;
+
+  const size_t arena_bytes = memstore_arena_bytes(config);
+  if (config->kv_arena) {
+    if (config->kv_arena_bytes < arena_bytes || ((uintptr_t)config->kv_arena & 15)) return bail(MS_ERR_INVALID_ARG);
+    s->k_arena = (__nv_bfloat16*)config->kv_arena;
+  } else if (arena_bytes) {
+    if (cudaMalloc(&s->arena_alloc, arena_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return bail(MS_ERR_OOM);
+    }
+    s->k_arena = (__nv_bfloat16*)s->arena_alloc;
+  }
+  s->v_arena = s->k_arena ? (__nv_bfloat16*)((char*)s->k_arena + arena_bytes / 2) : nullptr;
+
+  const int64_t rows = (int64_t)config->n_users * config->max_facts_per_user;
+  const size_t esz = emb_elem_size(config->emb_dtype);
+  bool ok = cudaMalloc(&s->emb, (size_t)rows * config->emb_dim * esz) == cudaSuccess &&
+            cudaMalloc(&s->emb_fact_id, (size_t)rows * sizeof(int32_t)) == cudaSuccess &&
+            cudaMalloc(&s->facts_d, (size_t)rows * sizeof(FactRec)) == cudaSuccess &&
+            cudaMalloc(&s->user_count_d, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
+            cudaMalloc(&s->inv_freq_d, (size_t)(config->head_dim / 2) * sizeof(float)) == cudaSuccess &&
+            cudaMalloc(&s->ctrl, sizeof(InjectCtrl)) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return bail(MS_ERR_OOM);
+  }
+  // RoPE frequencies: theta^(-2i/d) in double, rounded once to fp32 (Sec. 2.4; models keep this vector in fp32)
+  std::vector<float> f(config->head_dim / 2);
+  for (int i = 0; i < config->head_dim / 2; ++i)
+    f[i] = config->inv_freq_override ? config->inv_freq_override[i]
+                                     : (float)std::pow(config->rope_theta, -(double)(2 * i) / (double)config->head_dim);
+  ok = cudaMemcpy(s->inv_freq_d, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
+       cudaMemset(s->user_count_d, 0, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
+       cudaMemset(s->ctrl, 0, sizeof(InjectCtrl)) == cudaSuccess &&
+       cudaEventCreateWithFlags(&s->last_done, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return bail(MS_ERR_CUDA);
+  }
+  s->user_count.assign(config->n_users, 0);
+  int occ = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0, 4>, kCopyThreads, 0) == cudaSuccess && occ > 0)
+    s->copy_ctas_per_sm = occ;
+  *out = s;
+  return MS_OK;
+}
+
+ms_status memstore_destroy(memstore_t* s) {
+  if (!s) return MS_OK;
+  {
+    DeviceGuard g(s->cfg.device);
+    cudaDeviceSynchronize();
+    cudaFree(s->arena_alloc);
+    cudaFree(s->emb);
+    cudaFree(s->emb_fact_id);
+    cudaFree(s->facts_d);
+    cudaFree(s->user_count_d);
+    cudaFree(s->inv_freq_d);
+    cudaFree(s->ctrl);
+    cudaFree(s->scores);
+    cudaFree(s->tiles);
+    if (s->last_done) cudaEventDestroy(s->last_done);
+    cudaGetLastError();
+  }
+  delete s;
+  return MS_OK;
+}
+
+ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
+                             const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
+  if (n < 0 || (n > 0 && (!embs || !n_tokens))) return fail(s, MS_ERR_INVALID_ARG, "null embeddings or lengths");
+  if (n == 0) {
+    if (out_first_id) *out_first_id = (int32_t)s->n_facts;
+    return MS_OK;
+  }
+  int64_t T = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (n_tokens[i] < 0) return fail(s, MS_ERR_INVALID_ARG, "negative token count");
+    T += n_tokens[i];
+  }
+  if (T > 0 && (!k_pre || !v)) return fail(s, MS_ERR_INVALID_ARG, "null K/V for %lld tokens", (long long)T);
+  if (((uintptr_t)embs & 15) || ((uintptr_t)k_pre & 15) || ((uintptr_t)v & 15))
+    return fail(s, MS_ERR_INVALID_ARG, "device buffers must be 16-byte aligned");
+  if (s->user_count[user] + n > c.max_facts_per_user)
+    return fail(s, MS_ERR_CAPACITY, "user %d segment full (%lld + %lld > %lld)", user, (long long)s->user_count[user],
+                (long long)n, (long long)c.max_facts_per_user);
+  if (s->kv_tokens_used + T > c.max_kv_tokens)
+    return fail(s, MS_ERR_CAPACITY, "K/V arena full (%lld + %lld > %lld tokens)", (long long)s->kv_tokens_used,
+                (long long)T, (long long)c.max_kv_tokens);
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t slot0 = s->user_count[user];
+  const int64_t row0 = (int64_t)user * c.max_facts_per_user + slot0;
+  const size_t esz = emb_elem_size(c.emb_dtype);
+
+  std::vector<FactRec> recs(n);
+  std::vector<int32_t> ids(n);
+  int64_t off = s->kv_tokens_used;
+  int64_t resident = 0;
+  int32_t max_len = s->max_fact_len;
+  for (int64_t i = 0; i < n; ++i) {
+    recs[i] = FactRec{(int32_t)off, n_tokens[i], user, n_tokens[i] > 0 ? 1 : 0};
+    ids[i] = (int32_t)(s->n_facts + i);
+    off += n_tokens[i];
+    resident += n_tokens[i] > 0;
+    if (n_tokens[i] > max_len) max_len = n_tokens[i];
+  }
+  const int32_t new_count = (int32_t)(slot0 + n);
+  MS_CUDA(s, cudaMemcpyAsync((char*)s->emb + (size_t)row0 * c.emb_dim * esz, embs, (size_t)n * c.emb_dim * esz,
+                             cudaMemcpyDeviceToDevice, st));
+  // the three small host arrays are pageable: cudaMemcpyAsync stages them before returning
+  MS_CUDA(s, cudaMemcpyAsync(s->facts_d + s->n_facts, recs.data(), (size_t)n * sizeof(FactRec), cudaMemcpyHostToDevice, st));
+  MS_CUDA(s, cudaMemcpyAsync(s->emb_fact_id + row0, ids.data(), (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  MS_CUDA(s, cudaMemcpyAsync(s->user_count_d + user, &new_count, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  if (T > 0) {
+    const int64_t row_vec = (int64_t)c.n_kv_heads * c.head_dim * 2 / 16;
+    const int64_t src_vec = T * row_vec;
+    int gx = (int)std::min<int64_t>((src_vec + 255) / 256, 4 * s->sm_count);
+    dim3 grid(gx > 0 ? gx : 1, c.n_layers, 2);
+    arena_append_kernel<<<grid, 256, 0, st>>>((const uint4*)k_pre, (const uint4*)v, (uint4*)s->k_arena, (uint4*)s->v_arena,
+                                              src_vec, c.max_kv_tokens * row_vec, s->kv_tokens_used * row_vec);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched++;
+  }
+  if (out_first_id) *out_first_id = (int32_t)s->n_facts;
+  s->user_count[user] += n;
+  if (s->user_count[user] > s->max_user_count) s->max_user_count = s->user_count[user];
+  s->n_facts += n;
+  s->n_resident += resident;
+  s->kv_tokens_used += T;
+  s->max_fact_len = max_len;
+  return MS_OK;
+}
+
+ms_status memstore_add_fact(memstore_t* s, int32_t user, const void* emb, const void* k_pre, const void* v,
+                            int32_t n_tokens, int32_t* out_fact_id, ms_stream stream) {
+  return memstore_add_facts(s, user, 1, emb, k_pre, v, &n_tokens, out_fact_id, stream);
+}
+
+ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                            int32_t* out_ids, float* out_scores, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (nq < 0 || k < 1 || k > kTopkMaxK) return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d (1 <= k <= %d)", nq, k, kTopkMaxK);
+  if (nq == 0) return MS_OK;
+  if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
+  if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (nq > s->scores_nq) {  // grow the score scratch (first call, or a larger batch than ever before)
+    MS_CUDA(s, cudaDeviceSynchronize());
+    cudaFree(s->scores);
+    s->scores = nullptr;
+    s->scores_nq = 0;
+    MS_CUDA(s, cudaMalloc(&s->scores, (size_t)nq * c.max_facts_per_user * sizeof(float)));
+    s->scores_nq = nq;
+  }
+  ms_status rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+
+  RetrieveParams p{};
+  p.emb = s->emb;
+  p.emb_fact_id = s->emb_fact_id;
+  p.user_count = s->user_count_d;
+  p.seg_capacity = c.max_facts_per_user;
+  p.n_users = c.n_users;
+  p.emb_dim = c.emb_dim;
+  p.queries = queries;
+  p.query_users = query_users;
+  p.nq = nq;
+  p.k = k;
+  p.scores = s->scores;
+  p.score_stride = c.max_facts_per_user;
+  p.out_ids = out_ids;
+  p.out_scores = out_scores;
+
+  const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
+  if (n_max > 0) {
+    // enough CTAs to fill the GPU, at least one row per warp
+    int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
+    int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (n_max + target_ctas - 1) / target_ctas);
+    rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
+    dim3 grid((unsigned)((n_max + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+    const size_t smem = (size_t)c.emb_dim * sizeof(float);
+    if (c.emb_dtype == MS_DTYPE_F16)
+      score_rows_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
+    else
+      score_rows_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched++;
+  }
+  topk_kernel<<<nq, kTopkThreads, 0, st>>>(p);
+  MS_CUDA(s, cudaGetLastError());
+  s->kernels_launched++;
+  s->retrieve_calls++;
+  return mark_last(s, st);
+}
+
+ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
+                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
+                          int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
+                          uint32_t flags, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (nreq < 0 || k < 0 || k > kPlanMaxK) return fail(s, MS_ERR_INVALID_ARG, "nreq=%d k=%d (k <= %d)", nreq, k, kPlanMaxK);
+  if (flags & ~(uint32_t)MS_INJECT_REVERSE) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  if (nreq == 0) return MS_OK;
+  if (!start_pos || !block_tables || !cache || (k > 0 && !fact_ids) || max_blocks < 0)
+    return fail(s, MS_ERR_INVALID_ARG, "null request arrays");
+  if (!cache->k_base || !cache->v_base || cache->block_size <= 0 || cache->num_blocks <= 0)
+    return fail(s, MS_ERR_INVALID_ARG, "bad cache description");
+  if (((uintptr_t)cache->k_base & 15) || ((uintptr_t)cache->v_base & 15) || (cache->layer_stride % 8) ||
+      (cache->block_stride % 8) || (cache->token_stride % 8) || (cache->head_stride % 8) || cache->layer_stride < 0 ||
+      cache->block_stride < 0 || cache->token_stride < 0 || cache->head_stride < 0)
+    return fail(s, MS_ERR_INVALID_ARG, "cache bases must be 16-byte aligned and strides non-negative multiples of 8");
+  if (out_slot_mapping && slot_stride < 0) return fail(s, MS_ERR_INVALID_ARG, "negative slot_stride");
+  if (c.max_kv_tokens == 0 || !s->k_arena) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+
+  // upper bound on tiles: each request composes at most k * (longest fact) tokens, plus a ragged first tile
+  const int64_t max_m = (int64_t)k * s->max_fact_len;
+  const int64_t tiles_per_req = (max_m + kTileTokens - 1) / kTileTokens + 1;
+  const int64_t tiles_needed = std::max<int64_t>(1, tiles_per_req * nreq);
+  if (tiles_needed > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
+  if (tiles_needed > s->tiles_capacity) {
+    MS_CUDA(s, cudaDeviceSynchronize());
+    cudaFree(s->tiles);
+    s->tiles = nullptr;
+    s->tiles_capacity = 0;
+    MS_CUDA(s, cudaMalloc(&s->tiles, (size_t)tiles_needed * sizeof(TileDesc)));
+    s->tiles_capacity = (uint32_t)tiles_needed;
+  }
+  ms_status rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+
+  InjectParams p{};
+  p.facts = s->facts_d;
+  p.n_facts = (int32_t)s->n_facts;
+  p.k_arena = s->k_arena;
+  p.v_arena = s->v_arena;
+  p.arena_tokens = c.max_kv_tokens;
+  p.inv_freq = s->inv_freq_d;
+  p.n_layers = c.n_layers;
+  p.n_heads = c.n_kv_heads;
+  p.head_dim = c.head_dim;
+  p.rope_style = c.rope_style;
+  p.max_position = (int32_t)c.max_position;
+  p.fact_ids = fact_ids;
+  p.nreq = nreq;
+  p.k = k;
+  p.start_pos = start_pos;
+  p.block_tables = block_tables;
+  p.max_blocks = max_blocks;
+  p.flags = flags;
+  p.k_cache = (__nv_bfloat16*)cache->k_base;
+  p.v_cache = (__nv_bfloat16*)cache->v_base;
+  p.layer_stride = cache->layer_stride;
+  p.block_stride = cache->block_stride;
+  p.token_stride = cache->token_stride;
+  p.head_stride = cache->head_stride;
+  p.num_blocks = cache->num_blocks;
+  p.block_size = cache->block_size;
+  p.out_n_tokens = out_n_tokens;
+  p.out_status = out_status;
+  p.out_slot_mapping = out_slot_mapping;
+  p.slot_stride = slot_stride;
+  p.tiles = s->tiles;
+  p.tiles_capacity = s->tiles_capacity;
+  p.ctrl = s->ctrl;
+
+  // items = tiles x layer groups; keep at least ~8 items per resident CTA, else one layer per item
+  const int resident_ctas = s->sm_count * s->copy_ctas_per_sm;
+  const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + kTileTokens - 1) / kTileTokens * nreq);
+  int lpi = 1;
+  while (lpi * 2 <= c.n_layers && c.n_layers % (lpi * 2) == 0 && est_tiles * (c.n_layers / (lpi * 2)) >= 8ll * resident_ctas) lpi *= 2;
+  p.layers_per_item = lpi;
+
+  inject_plan_kernel<<<nreq, kPlanThreads, 0, st>>>(p);
+  MS_CUDA(s, cudaGetLastError());
+
+  const int units = c.n_kv_heads * (c.head_dim / 16);
+  const int upt = units >= 64 ? 4 : units >= 32 ? 2 : 1;
+  cudaLaunchConfig_t lc{};
+  lc.blockDim = dim3(kCopyThreads);
+  lc.dynamicSmemBytes = 0;
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaSuccess;
+  dim3 grid((unsigned)resident_ctas);
+  if (c.rope_style == MS_ROPE_HALF_SPLIT)
+    launch_copy<0>(p, upt, grid, lc, e);
+  else
+    launch_copy<1>(p, upt, grid, lc, e);
+  if (e != cudaSuccess) {
+    // the plan kernel has already counted tiles that no copy kernel will clear
+    cudaMemsetAsync(s->ctrl, 0, sizeof(InjectCtrl), st);
+    return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
+  }
+  s->kernels_launched += 2;
+  s->inject_calls++;
+  return mark_last(s, st);
+}
+
+ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
+  if (!s || !out) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  out->n_facts = s->n_facts;
+  out->n_resident_facts = s->n_resident;
+  out->kv_tokens_used = s->kv_tokens_used;
+  out->retrieve_calls = s->retrieve_calls;
+  out->inject_calls = s->inject_calls;
+  out->kernels_launched = s->kernels_launched;
+  out->arena_bytes = (int64_t)memstore_arena_bytes(&s->cfg);
+  out->embedding_bytes = (int64_t)s->cfg.n_users * s->cfg.max_facts_per_user * s->cfg.emb_dim * (int64_t)emb_elem_size(s->cfg.emb_dtype);
+  return MS_OK;
+}
+
+const char* memstore_last_error(memstore_t* s) { return s ? s->err.c_str() : "null store"; }
+
+}  // extern "C"

@@ -1,0 +1,277 @@
+"""Thin Python binding of ``libmemstore.so`` (argument marshalling only).
+
+Every step of the path (scoring, top-k, fact resolution, position assignment, slot mapping, RoPE, the
+K/V scatter) runs in the CUDA kernels behind the C ABI of ``include/memstore.h``; this module converts
+torch tensors to raw device pointers and checks dtypes and shapes.  torch is used for device memory and
+streams only.  If the library has not been built, creating a MemStore raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libmemstore.so"
+
+MS_OK = 0
+STATUS_NAMES = {0: "MS_OK", 1: "MS_ERR_INVALID_ARG", 2: "MS_ERR_UNSUPPORTED", 3: "MS_ERR_OOM", 4: "MS_ERR_CAPACITY", 5: "MS_ERR_CUDA"}
+REQ_BAD_FACT_ID, REQ_NOT_RESIDENT, REQ_BLOCK_TABLE_SHORT, REQ_BAD_BLOCK_ID, REQ_POSITION_OVERFLOW = 1, 2, 4, 8, 16
+DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
+ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
+INJECT_REVERSE = 1
+
+
+class MemStoreError(RuntimeError):
+    def __init__(self, code: int, msg: str = ""):
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+class _Config(C.Structure):
+    _fields_ = [
+        ("device", C.c_int32), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("kv_dtype", C.c_int32), ("emb_dim", C.c_int32), ("emb_dtype", C.c_int32), ("rope_style", C.c_int32),
+        ("rope_theta", C.c_double), ("inv_freq_override", C.POINTER(C.c_float)), ("max_position", C.c_int64),
+        ("n_users", C.c_int32), ("reserved0", C.c_int32), ("max_facts_per_user", C.c_int64),
+        ("max_kv_tokens", C.c_int64), ("kv_arena", C.c_void_p), ("kv_arena_bytes", C.c_size_t),
+    ]  # fmt: skip
+
+
+class _PagedCache(C.Structure):
+    _fields_ = [
+        ("k_base", C.c_void_p), ("v_base", C.c_void_p), ("layer_stride", C.c_int64), ("block_stride", C.c_int64),
+        ("token_stride", C.c_int64), ("head_stride", C.c_int64), ("num_blocks", C.c_int64),
+        ("block_size", C.c_int32), ("reserved0", C.c_int32),
+    ]  # fmt: skip
+
+
+class _Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
+        "arena_bytes", "embedding_bytes")]  # fmt: skip
+
+
+# every symbol include/memstore.h declares
+EXPORTS = (
+    "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
+    "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
+)  # fmt: skip
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen the in-tree CUDA library; raises if it is missing (build it with ``__graft_entry__.build()``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise ImportError(
+            f"{_LIB_PATH} not found: build it with `python -m paper_2607_27090_b200.build` "
+            "(nvcc, sm_100a). This package has no CPU fallback."
+        )
+    L = C.CDLL(str(_LIB_PATH))
+    vp, i32, i64, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32
+    L.memstore_version.restype = C.c_char_p
+    L.memstore_version.argtypes = []
+    L.memstore_arena_bytes.restype = C.c_size_t
+    L.memstore_arena_bytes.argtypes = [C.POINTER(_Config)]
+    L.memstore_create.restype = i32
+    L.memstore_create.argtypes = [C.POINTER(_Config), C.POINTER(vp)]
+    L.memstore_destroy.restype = i32
+    L.memstore_destroy.argtypes = [vp]
+    L.memstore_add_fact.restype = i32
+    L.memstore_add_fact.argtypes = [vp, i32, vp, vp, vp, i32, C.POINTER(i32), vp]
+    L.memstore_add_facts.restype = i32
+    L.memstore_add_facts.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
+    L.memstore_retrieve.restype = i32
+    L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    L.memstore_inject.restype = i32
+    L.memstore_inject.argtypes = [vp, vp, i32, i32, vp, vp, i32, C.POINTER(_PagedCache), vp, vp, vp, i64, u32, vp]
+    L.memstore_stats.restype = i32
+    L.memstore_stats.argtypes = [vp, C.POINTER(_Stats)]
+    L.memstore_last_error.restype = C.c_char_p
+    L.memstore_last_error.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def _dev_ptr(t: torch.Tensor | None, dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise TypeError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+@dataclass
+class PagedCache:
+    """A caller-owned paged KV cache: two bf16 tensors and strides in elements (see ``ms_paged_cache``)."""
+
+    k: torch.Tensor
+    v: torch.Tensor
+    layer_stride: int
+    block_stride: int
+    token_stride: int
+    head_stride: int
+    num_blocks: int
+    block_size: int
+
+    @classmethod
+    def allocate(cls, n_layers, num_blocks, block_size, n_kv_heads, head_dim, device, layout="NHD", stacked=False, fill_bits=None):
+        """Allocate a cache. ``layout`` "NHD": [L][blocks][bs][h][d]; "HND": [L][blocks][h][bs][d].
+        ``stacked``: K and V are planes 0 and 1 of one buffer [L][2][blocks]..., else separate buffers."""
+        shape = (num_blocks, block_size, n_kv_heads, head_dim) if layout == "NHD" else (num_blocks, n_kv_heads, block_size, head_dim)
+        blk = block_size * n_kv_heads * head_dim
+        if stacked:
+            buf = torch.empty((n_layers, 2, *shape), dtype=torch.bfloat16, device=device)
+            k, v = buf[:, 0], buf[:, 1]
+            layer_stride = 2 * num_blocks * blk
+            keep = buf
+        else:
+            k = torch.empty((n_layers, *shape), dtype=torch.bfloat16, device=device)
+            v = torch.empty((n_layers, *shape), dtype=torch.bfloat16, device=device)
+            layer_stride = num_blocks * blk
+            keep = None
+        if fill_bits is not None:
+            for t in ((keep,) if stacked else (k, v)):
+                t.view(torch.int16).fill_(fill_bits - 0x10000 if fill_bits >= 0x8000 else fill_bits)
+        token_stride, head_stride = (n_kv_heads * head_dim, head_dim) if layout == "NHD" else (head_dim, block_size * head_dim)
+        c = cls(k, v, layer_stride, blk, token_stride, head_stride, num_blocks, block_size)
+        c._keep = keep
+        return c
+
+    def _struct(self) -> _PagedCache:
+        for t, n in ((self.k, "k"), (self.v, "v")):
+            if not t.is_cuda or t.dtype != torch.bfloat16:
+                raise TypeError(f"cache.{n} must be a CUDA bfloat16 tensor")
+        return _PagedCache(self.k.data_ptr(), self.v.data_ptr(), self.layer_stride, self.block_stride,
+                           self.token_stride, self.head_stride, self.num_blocks, self.block_size, 0)  # fmt: skip
+
+
+class MemStore:
+    """Handle of one ``memstore_t`` (see ``include/memstore.h`` for the meaning of every argument)."""
+
+    def __init__(self, *, device=0, n_layers, n_kv_heads, head_dim, emb_dim, emb_dtype=torch.float16, rope_theta=1.0e4,
+                 rope_style=ROPE_HALF_SPLIT, inv_freq_override=None, max_position=1 << 24, n_users=1,
+                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None):  # fmt: skip
+        self._lib = load_library()
+        self._h = C.c_void_p()
+        self.device = torch.device("cuda", device if isinstance(device, int) else torch.device(device).index or 0)
+        self.emb_torch_dtype = emb_dtype
+        emb_code = {torch.float32: DTYPE_F32, torch.float16: DTYPE_F16}.get(emb_dtype)
+        if emb_code is None:
+            raise TypeError("emb_dtype must be torch.float32 or torch.float16")
+        ov = None
+        if inv_freq_override is not None:
+            vals = [float(x) for x in inv_freq_override]
+            ov = (C.c_float * len(vals))(*vals)
+            if len(vals) != head_dim // 2:
+                raise ValueError("inv_freq_override needs head_dim/2 entries")
+        self._arena = kv_arena
+        cfg = _Config(self.device.index, n_layers, n_kv_heads, head_dim, DTYPE_BF16, emb_dim, emb_code, rope_style,
+                      float(rope_theta), ov, max_position, n_users, 0, max_facts_per_user, max_kv_tokens,
+                      kv_arena.data_ptr() if kv_arena is not None else None,
+                      kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0)  # fmt: skip
+        self.n_layers, self.n_kv_heads, self.head_dim, self.emb_dim = n_layers, n_kv_heads, head_dim, emb_dim
+        rc = self._lib.memstore_create(C.byref(cfg), C.byref(self._h))
+        if rc != MS_OK:
+            self._h = C.c_void_p()
+            raise MemStoreError(rc, "memstore_create")
+
+    # -- helpers ---------------------------------------------------------------------------------
+    def _check(self, rc: int):
+        if rc != MS_OK:
+            raise MemStoreError(rc, self._lib.memstore_last_error(self._h).decode())
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.memstore_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    # -- the four calls ---------------------------------------------------------------------------
+    def add_fact(self, emb, k_pre=None, v=None, user=0, stream=None) -> int:
+        n_tokens = 0 if k_pre is None else k_pre.shape[1]
+        out = C.c_int32(-1)
+        rc = self._lib.memstore_add_fact(self._h, user, _dev_ptr(emb, self.emb_torch_dtype, "emb"),
+                                         _dev_ptr(k_pre, torch.bfloat16, "k_pre"), _dev_ptr(v, torch.bfloat16, "v"),
+                                         n_tokens, C.byref(out), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out.value
+
+    def add_facts(self, embs, n_tokens, k_pre=None, v=None, user=0, stream=None) -> int:
+        """``n_tokens``: host sequence of ints; ``k_pre``/``v``: [L, sum(n_tokens), h, d] bf16 on the device."""
+        n = embs.shape[0]
+        lens = (C.c_int32 * n)(*[int(x) for x in n_tokens])
+        out = C.c_int32(-1)
+        rc = self._lib.memstore_add_facts(self._h, user, n, _dev_ptr(embs, self.emb_torch_dtype, "embs"),
+                                          _dev_ptr(k_pre, torch.bfloat16, "k_pre"), _dev_ptr(v, torch.bfloat16, "v"),
+                                          lens, C.byref(out), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out.value
+
+    def retrieve(self, queries, k, query_users=None, out_ids=None, out_scores=None, want_scores=True, stream=None):
+        nq = queries.shape[0]
+        if out_ids is None:
+            out_ids = torch.empty((nq, k), dtype=torch.int32, device=queries.device)
+        if out_scores is None and want_scores:
+            out_scores = torch.empty((nq, k), dtype=torch.float32, device=queries.device)
+        rc = self._lib.memstore_retrieve(self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"),
+                                         _dev_ptr(query_users, torch.int32, "query_users"), nq, k,
+                                         _dev_ptr(out_ids, torch.int32, "out_ids"),
+                                         _dev_ptr(out_scores, torch.float32, "out_scores"), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out_ids, out_scores
+
+    def inject(self, fact_ids, start_pos, block_tables, cache: PagedCache, out_n_tokens=None, out_status=None,
+               out_slot_mapping=None, flags=0, stream=None):  # fmt: skip
+        nreq, k = fact_ids.shape
+        dev = fact_ids.device
+        if out_n_tokens is None:
+            out_n_tokens = torch.empty(nreq, dtype=torch.int32, device=dev)
+        if out_status is None:
+            out_status = torch.empty(nreq, dtype=torch.int32, device=dev)
+        cs = cache._struct()
+        rc = self._lib.memstore_inject(self._h, _dev_ptr(fact_ids, torch.int32, "fact_ids"), nreq, k,
+                                       _dev_ptr(start_pos, torch.int32, "start_pos"),
+                                       _dev_ptr(block_tables, torch.int32, "block_tables"), block_tables.shape[1],
+                                       C.byref(cs), _dev_ptr(out_n_tokens, torch.int32, "out_n_tokens"),
+                                       _dev_ptr(out_status, torch.int32, "out_status"),
+                                       _dev_ptr(out_slot_mapping, torch.int64, "out_slot_mapping"),
+                                       out_slot_mapping.shape[1] if out_slot_mapping is not None else 0,
+                                       flags, _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out_n_tokens, out_status
+
+    def stats(self) -> dict:
+        st = _Stats()
+        self._check(self._lib.memstore_stats(self._h, C.byref(st)))
+        return {n: getattr(st, n) for n, _ in _Stats._fields_}
+
+    def last_error(self) -> str:
+        return self._lib.memstore_last_error(self._h).decode()

@@ -1,0 +1,53 @@
+"""CPU-only: the CUDA library builds, loads and exports every function include/memstore.h declares
+(no compute call is made here), and the binding refuses to run without it."""
+import ctypes
+import re
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+def declared_functions():
+    text = (ROOT / "include" / "memstore.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(memstore_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2607_27090_b200 import build, memstore
+
+    lib_path = build.build()
+    names = declared_functions()
+    assert len(names) >= 10 and "memstore_inject" in names and "memstore_retrieve" in names
+    lib = ctypes.CDLL(str(lib_path))
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in memstore.h but not exported"
+    assert set(memstore.EXPORTS) == set(names)
+    assert memstore.load_library().memstore_version().decode().endswith("sm_100a")
+
+
+def test_struct_layouts_match_header_sizes():
+    # the ctypes mirrors must have the C sizes (x86-64 / LP64): config 96 bytes, cache 64, stats 64
+    from paper_2607_27090_b200 import memstore
+
+    assert ctypes.sizeof(memstore._Config) == 96
+    assert ctypes.sizeof(memstore._PagedCache) == 64
+    assert ctypes.sizeof(memstore._Stats) == 64
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    import pytest
+
+    from paper_2607_27090_b200 import memstore
+
+    monkeypatch.setattr(memstore, "_lib", None)
+    monkeypatch.setattr(memstore, "_LIB_PATH", tmp_path / "libmemstore.so")
+    with pytest.raises(ImportError):
+        memstore.load_library()
+
+
+def test_product_path_does_not_import_the_oracle():
+    for f in (ROOT / "paper_2607_27090_b200").rglob("*"):
+        if f.suffix in (".py", ".cu", ".cuh", ".h"):
+            src = f.read_text()
+            assert "import oracle" not in src and "from oracle" not in src and "memoracle" not in src, f

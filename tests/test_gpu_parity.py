@@ -1,0 +1,313 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on small seeded cases that still span several tiles, layers and a ragged tail, plus the edge cases."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_27090_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    import oracle
+    from parity import (HostStore, check_ids, run_inject_and_check, to_dev, untouched_mask_ok)  # noqa: F401
+    from paper_2607_27090_b200 import memstore as M
+    from paper_2607_27090_b200.memstore import MemStore, PagedCache
+
+DEV = "cuda"
+SENT = synth.SENTINEL_BF16
+
+
+def make_cache(hs, num_blocks, bs, **kw):
+    return PagedCache.allocate(hs.L, num_blocks, bs, hs.H, hs.D, DEV, fill_bits=SENT, **kw)
+
+
+# ------------------------------------------------------------------------------------------------ config 1
+def test_tiny_config_end_to_end():
+    """256 facts of 8-32 tokens, 1 layer, 2 heads, d=64, theta 1e4, fp32 64-d embeddings, k=5,
+    injected after a 16-token prefix, block size 16, shuffled block table, the paper's reverse order."""
+    c = synth.CONFIGS["tiny"]
+    hs = HostStore(0, c.n_facts, c.n_layers, c.n_kv_heads, c.head_dim, c.len_lo, c.len_hi, c.emb_dim, c.emb_dtype)
+    ms = hs.to_memstore(c.rope_theta)
+    q = synth.queries(0, 1, c.emb_dim, c.emb_dtype)
+    ids, sc = ms.retrieve(to_dev(q), c.k)
+    torch.cuda.synchronize()
+    ids_np = ids.cpu().numpy()
+    check_ids(ids_np[0], sc.cpu().numpy()[0], hs.emb, q[0], c.k)
+    ids_o, _ = oracle.retrieve(hs.emb, q, c.k)
+    assert np.array_equal(ids_np, ids_o)  # no near-tie in this seed: identical lists
+    nb = 64
+    need = (c.start_pos + c.k * c.len_hi + c.block_size - 1) // c.block_size
+    table = synth.block_tables(0, nb, need, 1)[0]
+    cache = make_cache(hs, nb, c.block_size)
+    out = run_inject_and_check(ms, hs, ids_np[0], c.start_pos, table, cache, c.rope_theta, flags=M.INJECT_REVERSE)
+    assert out["m"] == int(hs.lens[ids_np[0]].sum()) and out["exact_frac"] > 0.999
+
+
+# ------------------------------------------------------------------------------------------------ retrieval
+@pytest.mark.parametrize("dtype,E", [("float32", 64), ("float16", 1024), ("float16", 136)])
+def test_retrieve_k_values_and_padding(dtype, E):
+    N = 777
+    hs = HostStore(1, N, 1, 1, 16, 1, 2, E, dtype)
+    ms = hs.to_memstore(1e4)
+    q = synth.queries(1, 3, E, dtype)
+    for k in (1, 5, 100, N, N + 3, 2048):
+        ids, sc = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        for i in range(3):
+            check_ids(ids[i].cpu().numpy(), sc[i].cpu().numpy(), hs.emb, q[i], k)
+
+
+def test_retrieve_ties_duplicates_and_self_query():
+    hs = HostStore(2, 300, 1, 1, 16, 1, 2, 256, "float16")
+    hs.emb[140] = hs.emb[17]
+    hs.emb[250] = hs.emb[17]
+    hs.emb[5] = hs.emb[4]
+    ms = hs.to_memstore(1e4)
+    q = np.stack([hs.emb[17], hs.emb[4], hs.emb[299]])
+    ids, sc = ms.retrieve(to_dev(q), 10)
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    assert ids[0, :3].tolist() == [17, 140, 250] and sc[0, 0] == sc[0, 1] == sc[0, 2]
+    assert ids[1, :2].tolist() == [4, 5] and ids[2, 0] == 299
+    ids_o, _ = oracle.retrieve(hs.emb, q, 10)
+    assert np.array_equal(ids, ids_o)
+    # all rows identical: every score ties, ids must come back ascending, for k below, at and above a radix bucket
+    same = HostStore(3, 1500, 1, 1, 16, 1, 1, 64, "float16")
+    same.emb[:] = same.emb[0]
+    ms2 = same.to_memstore(1e4)
+    for k in (1, 7, 1024, 1500):
+        ids, _ = ms2.retrieve(to_dev(same.emb[:1]), k)
+        assert ids[0].cpu().tolist() == list(range(k))
+
+
+def test_retrieve_empty_store_and_per_user_segments():
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=64, max_facts_per_user=8, max_kv_tokens=8)
+    ids, sc = ms.retrieve(to_dev(synth.queries(0, 2, 64, "float16")), 4)
+    assert torch.all(ids == -1) and torch.all(sc == 0)
+    # three users with private segments; a query only ever sees its own user's facts; ids are global
+    hs = HostStore(4, 50, 1, 1, 16, 1, 3, 128, "float16", n_users=3)
+    ms = hs.to_memstore(1e4)
+    q = synth.queries(4, 5, 128, "float16")
+    users = np.array([2, 0, 1, 2, 0], np.int32)
+    ids, sc = ms.retrieve(to_dev(q), 60, query_users=to_dev(users))
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    for i, u in enumerate(users):
+        rows = np.arange(u * 50, (u + 1) * 50)
+        check_ids(ids[i], sc[i], hs.emb[rows], q[i], 60, row_ids=rows.astype(np.int32))
+
+
+# ------------------------------------------------------------------------------------------------ injection
+@pytest.mark.parametrize("start,bs", [(0, 16), (13, 16), (16, 16), (4096, 32), (100, 8), (1000003, 16)])
+def test_inject_positions_and_block_sizes(start, bs):
+    # lengths 1 and 128 included; facts straddle up to 9 blocks; several layers and tiles, ragged tail
+    lens = [1, 128, 17, 33, 5, 64, 16, 31]
+    hs = HostStore(5, len(lens), 3, 8, 128, 0, 0, 64, "float16", lens=lens)
+    ms = hs.to_memstore(5e5)
+    ids = [1, 0, 3, -1, 2, 2, 7, 5]
+    m = sum(lens[i] for i in ids if i >= 0)
+    n_table = (start + m + bs - 1) // bs
+    nb = n_table + 7
+    table = synth.block_tables(6, nb, n_table, 1)[0]
+    if start >= 4096:  # only the blocks the request touches need to be real
+        table = np.full(n_table, 0, np.int32)
+        used = np.arange(start // bs, n_table)
+        nb = len(used) + 5
+        table[used] = synth.block_tables(6, nb, len(used), 1)[0]
+    cache = make_cache(hs, nb, bs)
+    out = run_inject_and_check(ms, hs, ids, start, table, cache, 5e5)
+    assert out["m"] == m and out["exact_frac"] > 0.995
+    if start == 0:  # position 0 is the identity: first token's K is bit-identical to the stored K
+        from parity import gather_cache_rows, bits  # noqa: F401
+        slot0 = int(table[0]) * bs
+        kb, _ = gather_cache_rows(cache, np.array([slot0]))
+        assert np.array_equal(kb[:, 0], hs.k[:, hs.offs[1]])
+
+
+@pytest.mark.parametrize("layout,stacked", [("NHD", False), ("NHD", True), ("HND", False), ("HND", True)])
+def test_inject_cache_layouts(layout, stacked):
+    hs = HostStore(7, 10, 2, 4, 64, 3, 40, 64, "float16")
+    ms = hs.to_memstore(1e4)
+    table = synth.block_tables(8, 20, 14, 1)[0]
+    cache = make_cache(hs, 20, 16, layout=layout, stacked=stacked)
+    out = run_inject_and_check(ms, hs, [9, 4, 0, 6], 21, table, cache, 1e4)
+    assert out["exact_frac"] > 0.995
+
+
+@pytest.mark.parametrize("style", [0, 1])
+@pytest.mark.parametrize("H,D", [(2, 64), (8, 128), (1, 256), (4, 32), (3, 16), (32, 128)])
+def test_inject_head_shapes_and_rope_styles(style, H, D):
+    hs = HostStore(9, 6, 2, H, D, 2, 50, 64, "float16")
+    ms = hs.to_memstore(1e6, rope_style=style)
+    table = synth.block_tables(10, 24, 20, 1)[0]
+    cache = make_cache(hs, 24, 16)
+    out = run_inject_and_check(ms, hs, [5, 1, 3, 0], 37, table, cache, 1e6, style=style)
+    assert out["exact_frac"] > 0.995
+
+
+def test_inject_inv_freq_override_and_reverse_flag():
+    D = 64
+    f = (np.linspace(1.0, 0.001, D // 2)).astype(np.float32)
+    hs = HostStore(11, 8, 2, 2, D, 4, 20, 64, "float16")
+    ms = hs.to_memstore(1e4, inv_freq_override=f)
+    table = synth.block_tables(12, 16, 12, 1)[0]
+    for flags in (0, M.INJECT_REVERSE):
+        cache = make_cache(hs, 16, 16)
+        run_inject_and_check(ms, hs, [2, 7, 1, 4], 9, table, cache, 1e4, inv_freq=f, flags=flags)
+
+
+def test_inject_batch_of_requests_shares_one_cache():
+    hs = HostStore(13, 40, 2, 8, 128, 16, 64, 64, "float16")
+    ms = hs.to_memstore(5e5)
+    nreq, k, bs, nb = 5, 6, 16, 200
+    rng = np.random.default_rng(0)
+    ids = rng.integers(0, 40, size=(nreq, k)).astype(np.int32)
+    ids[2, 3] = -1
+    starts = np.array([32, 0, 7, 48, 16], np.int32)
+    per = (48 + k * 64 + bs - 1) // bs
+    tables = synth.block_tables(14, nb, per, nreq)
+    cache = make_cache(hs, nb, bs)
+    n_tok, status = ms.inject(to_dev(ids), to_dev(starts), to_dev(tables), cache)
+    torch.cuda.synchronize()
+    from parity import check_k, gather_cache_rows
+
+    all_slots = []
+    for r in range(nreq):
+        res = oracle.inject(ids[r], hs.offs, hs.lens, hs.k, hs.v, 5e5, int(starts[r]), tables[r], bs, nb)
+        assert int(n_tok[r]) == res.m and int(status[r]) == 0
+        kb, vb = gather_cache_rows(cache, res.slots)
+        assert np.array_equal(vb, res.v)
+        check_k(kb, res.k_ref)
+        all_slots.append(res.slots)
+    assert untouched_mask_ok(cache, np.concatenate(all_slots), SENT)
+
+
+def test_inject_empty_and_degenerate_requests():
+    hs = HostStore(15, 4, 1, 2, 64, 3, 9, 64, "float16")
+    ms = hs.to_memstore(1e4)
+    cache = make_cache(hs, 8, 16)
+    table = np.arange(8, dtype=np.int32)
+    # all ids skipped -> m = 0, nothing written
+    out = run_inject_and_check(ms, hs, [-1, -1, -1], 5, table, cache, 1e4)
+    assert out["m"] == 0
+    # k = 0
+    n_tok, status = ms.inject(torch.empty((2, 0), dtype=torch.int32, device=DEV), to_dev(np.array([0, 3], np.int32)),
+                              to_dev(np.stack([table, table])), cache)  # fmt: skip
+    torch.cuda.synchronize()
+    assert n_tok.cpu().tolist() == [0, 0] and status.cpu().tolist() == [0, 0]
+    assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
+
+
+# ------------------------------------------------------------------------------------------------ safety
+def test_inject_data_errors_set_status_and_skip():
+    lens = [4, 6, 0, 5]
+    hs = HostStore(16, 4, 1, 2, 64, 0, 0, 64, "float16", lens=lens)  # fact 2 is embedding-only
+    ms = hs.to_memstore(1e4, max_position=64)
+    bs, nb = 16, 6
+    cache = make_cache(hs, nb, bs)
+
+    def run(ids, start, table):
+        n, s = ms.inject(to_dev(np.array([ids], np.int32)), to_dev(np.array([start], np.int32)),
+                         to_dev(np.array([table], np.int32)), cache)  # fmt: skip
+        torch.cuda.synchronize()
+        return int(n[0]), int(s[0])
+
+    ok_table = [3, 1, 4, 0]
+    # unknown id and non-resident id contribute nothing; the valid facts are placed as if they were absent
+    n, s = run([0, 99, 2, 3], 2, ok_table)
+    assert n == 9 and s == (M.REQ_BAD_FACT_ID | M.REQ_NOT_RESIDENT)
+    res = oracle.inject([0, 3], hs.offs, hs.lens, hs.k, hs.v, 1e4, 2, ok_table, bs, nb)
+    from parity import check_k, gather_cache_rows
+
+    kb, vb = gather_cache_rows(cache, res.slots)
+    assert np.array_equal(vb, res.v)
+    check_k(kb, res.k_ref)
+    assert untouched_mask_ok(cache, res.slots, SENT)
+    # block table one entry short: tokens beyond it are skipped, the others land
+    cache = make_cache(hs, nb, bs)
+    n, s = run([0, 1, 3], 10, [2])  # positions 10..24, table covers 0..15
+    assert n == 15 and s == M.REQ_BLOCK_TABLE_SHORT
+    assert untouched_mask_ok(cache, np.arange(2 * bs + 10, 3 * bs), SENT)
+    assert not untouched_mask_ok(cache, np.arange(2 * bs + 11, 3 * bs), SENT)
+    # block id == num_blocks and a negative block id
+    cache = make_cache(hs, nb, bs)
+    n, s = run([0, 1, 3], 10, [nb, -1])
+    assert n == 15 and s == M.REQ_BAD_BLOCK_ID
+    assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
+    # position overflow: max_position = 64, tokens at pos >= 64 skipped
+    cache = make_cache(hs, nb, bs)
+    n, s = run([1, 3], 58, [0, 1, 2, 3, 4])
+    assert n == 11 and s == M.REQ_POSITION_OVERFLOW
+    assert untouched_mask_ok(cache, np.arange(3 * bs + 10, 4 * bs), SENT)
+
+
+def test_host_errors_return_codes_and_enqueue_nothing():
+    with pytest.raises(M.MemStoreError) as e:
+        MemStore(n_layers=1, n_kv_heads=1, head_dim=48, emb_dim=64, max_facts_per_user=4, max_kv_tokens=4)
+    assert e.value.code == 2
+    with pytest.raises(M.MemStoreError) as e:
+        MemStore(n_layers=1, n_kv_heads=1, head_dim=64, emb_dim=60, max_facts_per_user=4, max_kv_tokens=4)
+    assert e.value.code == 2
+    with pytest.raises(M.MemStoreError) as e:
+        MemStore(n_layers=0, n_kv_heads=1, head_dim=64, emb_dim=64, max_facts_per_user=4, max_kv_tokens=4)
+    assert e.value.code == 1
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=64, emb_dim=64, max_facts_per_user=2, max_kv_tokens=10)
+    emb = to_dev(synth.embeddings(0, 3, 64, "float16"))
+    kv = torch.zeros((1, 6, 1, 64), dtype=torch.bfloat16, device=DEV)
+    before = ms.stats()["kernels_launched"]
+    with pytest.raises(M.MemStoreError) as e:
+        ms.add_facts(emb, [2, 2, 2], kv, kv)  # three facts into a segment of two
+    assert e.value.code == 4
+    ms.add_fact(emb[0], kv, kv)
+    with pytest.raises(M.MemStoreError) as e:
+        ms.add_fact(emb[1], kv, kv)  # 6 + 6 tokens > 10
+    assert e.value.code == 4 and "arena" in ms.last_error()
+    with pytest.raises(M.MemStoreError) as e:
+        ms.add_fact(emb[1], user=3)
+    assert e.value.code == 1
+    with pytest.raises(M.MemStoreError):
+        ms.retrieve(emb[:1], 0)
+    with pytest.raises(M.MemStoreError):
+        ms.retrieve(emb[:1], 5000)
+    cache = PagedCache.allocate(1, 4, 16, 1, 64, DEV, fill_bits=SENT)
+    bad = PagedCache(cache.k, cache.v, cache.layer_stride, cache.block_stride, 60, cache.head_stride, 4, 16)
+    ids = torch.zeros((1, 1), dtype=torch.int32, device=DEV)
+    z = torch.zeros(1, dtype=torch.int32, device=DEV)
+    with pytest.raises(M.MemStoreError) as e:
+        ms.inject(ids, z, torch.zeros((1, 4), dtype=torch.int32, device=DEV), bad)
+    assert e.value.code == 1
+    st = ms.stats()
+    assert st["n_facts"] == 1 and st["kv_tokens_used"] == 6 and st["kernels_launched"] == before + 1
+    assert M.load_library().memstore_version().decode().startswith("memstore")
+
+
+# ------------------------------------------------------------------------------------------------ determinism
+def test_same_call_twice_and_on_two_streams_is_bit_identical():
+    hs = HostStore(17, 30, 4, 8, 128, 16, 64, 256, "float16")
+    ms = hs.to_memstore(5e5)
+    q = to_dev(synth.queries(17, 4, 256, "float16"))
+    table = to_dev(synth.block_tables(18, 64, 40, 1))
+    start = to_dev(np.array([32], np.int32))
+    results = []
+    streams = [None, None, torch.cuda.Stream(), torch.cuda.Stream()]
+    for st in streams:
+        cache = make_cache(hs, 64, 16)
+        torch.cuda.synchronize()
+        ctx = torch.cuda.stream(st) if st is not None else torch.cuda.stream(torch.cuda.current_stream())
+        with ctx:
+            ids, sc = ms.retrieve(q, 9, stream=st)
+            ms.inject(ids[:1].contiguous(), start, table, cache, flags=M.INJECT_REVERSE, stream=st)
+        torch.cuda.synchronize()
+        results.append((ids.cpu(), sc.cpu(), cache.k.cpu().view(torch.int16), cache.v.cpu().view(torch.int16)))
+    for r in results[1:]:
+        for a, b in zip(results[0], r):
+            assert torch.equal(a, b)
+    # two streams back to back without a host sync in between (the store orders them on the device)
+    c1, c2 = make_cache(hs, 64, 16), make_cache(hs, 64, 16)
+    torch.cuda.synchronize()
+    s1, s2 = streams[2], streams[3]
+    ids1, _ = ms.retrieve(q, 9, stream=s1)
+    ids2, _ = ms.retrieve(q, 9, stream=s2)
+    ms.inject(ids1[:1].contiguous(), start, table, c1, flags=M.INJECT_REVERSE, stream=s1)
+    ms.inject(ids2[1:2].contiguous(), start, table, c2, flags=M.INJECT_REVERSE, stream=s2)
+    torch.cuda.synchronize()
+    assert torch.equal(c1.k.cpu().view(torch.int16), results[0][2]) and torch.equal(ids1.cpu(), ids2.cpu())
