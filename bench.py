@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the retrieve + Chunked-RoPE-inject hot path on the Llama-3.1-8B KV shape at k=50.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--k 50] [--config llama8b]
+
+A step is one request through the whole path: memstore_retrieve (score 2000 fp16 1024-d embeddings, top-k)
+followed by memstore_inject (gather k facts' pre-RoPE K and V, rotate K at the assembled positions,
+scatter both into the paged cache) on one stream, ids flowing device to device.  Requests rotate over a
+pool of queries and block tables; one request moves 2 x m x 128 KiB (about 520 MB at k=50), more than the
+126 MB L2, so every step is cold by construction.
+
+One JSON line is printed by rank 0.  `value` is microseconds per request (whole job: the K steps of all
+ranks divided into the max-over-ranks device time), lower is better.  With N > 1 every rank serves its own
+replica of the store (the path has no exchange step: requests are independent).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "retrieve+inject us per request at k=50 (Llama-3.1-8B KV shape)"
+NOMINAL_HBM_GBS = 8000.0  # the benchmark spec quotes fractions of ~8 TB/s as well
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama8b")
+    ap.add_argument("--k", type=int, default=50)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scale-facts", type=float, default=1.0, help="shrink the store (profiling captures); the request keeps its shape")
+    ap.add_argument("--pool-blocks", type=int, default=0, help="cache pool size in blocks (default: at least 4096)")
+    ap.add_argument("--query-pool", type=int, default=16)
+    ap.add_argument("--sweep-k", action="store_true", help="also report k = 5, 10, 20 (extra keys, same JSON line)")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------- peaks / clocks
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        self.period = period_s
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+            "hw_power_brake": 0x80, "sync_boost": 0x10, "applications_clocks": 0x2,
+        }  # fmt: skip
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}  # fmt: skip
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle arm
+class OracleArm:
+    """Times the CPU oracle, as it stands, on a bounded sample of one request of the workload and scales the
+    result to a whole request.  Sample: the full retrieval (all facts) plus the injection, over all layers, of
+    the first facts of the oracle's own top-k list (placement order), as many tokens as fit the time budget."""
+
+    def __init__(self, shape, k, seed, n_threads=0):
+        import numpy as np
+
+        import oracle
+        from paper_2607_27090_b200 import synth
+
+        oracle.build()
+        self.np, self.oracle, self.synth = np, oracle, synth
+        self.shape, self.k, self.seed, self.n_threads = shape, k, seed, n_threads
+        self.cores = oracle.max_threads() if n_threads <= 0 else n_threads
+        self.emb = synth.embeddings(seed, shape.n_facts, shape.emb_dim, shape.emb_dtype)
+        self.q = synth.queries(seed, 1, shape.emb_dim, shape.emb_dtype)
+        self.lens = synth.fact_lengths(seed, shape.n_facts, shape.len_lo, shape.len_hi)
+        ids, _ = oracle.retrieve(self.emb, self.q, k, n_threads=n_threads)
+        self.ids = ids[0][::-1].copy()  # the paper's placement: best fact last
+        self.m_full = int(self.lens[self.ids].sum())
+        self.table = np.arange((shape.start_pos + self.m_full) // shape.block_size + 2, dtype=np.int32)
+        self._packed = {}
+        t, m = self._inject(1)
+        self.per_token_s = t / max(m, 1)
+
+    def _pack(self, n_take):
+        if n_take not in self._packed:
+            np, s = self.np, self.shape
+            offs = np.zeros(s.n_facts, np.int64)
+            ln = np.zeros(s.n_facts, np.int32)
+            ks, vs, t = [], [], 0
+            for f in dict.fromkeys(int(i) for i in self.ids[:n_take]):
+                kf, vf = self.synth.kv_fact(self.seed, f, s.n_layers, int(self.lens[f]), s.n_kv_heads, s.head_dim)
+                ks.append(kf)
+                vs.append(vf)
+                offs[f], ln[f] = t, self.lens[f]
+                t += int(self.lens[f])
+            self._packed = {n_take: (offs, ln, np.concatenate(ks, axis=1), np.concatenate(vs, axis=1))}
+        return self._packed[n_take]
+
+    def _inject(self, n_take):
+        s = self.shape
+        offs, ln, kk, vv = self._pack(n_take)
+        t0 = time.perf_counter()
+        res = self.oracle.inject(self.ids[:n_take], offs, ln, kk, vv, s.rope_theta, s.start_pos, self.table, s.block_size,
+                                 self.table.size, want_ref=False, n_threads=self.n_threads)  # fmt: skip
+        return time.perf_counter() - t0, res.m
+
+    def facts_for_budget(self, budget_s):
+        n_take, tok = 1, int(self.lens[self.ids[0]])
+        while n_take < len(self.ids) and (tok + self.lens[self.ids[n_take]]) * self.per_token_s < budget_s:
+            tok += int(self.lens[self.ids[n_take]])
+            n_take += 1
+        return n_take
+
+    def time_step(self, n_take):
+        """One sampled request -> (microseconds scaled to the whole request, description of the sample)."""
+        t0 = time.perf_counter()
+        self.oracle.retrieve(self.emb, self.q, self.k, n_threads=self.n_threads)
+        t_retrieve = time.perf_counter() - t0
+        t_inj, m_s = self._inject(n_take)
+        t_req = t_retrieve + t_inj * (self.m_full / m_s)
+        sample = (f"retrieval over all {self.shape.n_facts} facts ({t_retrieve * 1e3:.1f} ms) + injection of the first "
+                  f"{n_take} of {len(self.ids)} facts ({m_s} of {self.m_full} tokens, all {self.shape.n_layers} layers, "
+                  f"{t_inj:.2f} s), injection time scaled by tokens")  # fmt: skip
+        return t_req * 1e6, sample
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_27090_b200 import synth
+
+    shape = synth.CONFIGS[args.config]
+    arm = OracleArm(shape, args.k, args.seed)
+    n_take = arm.facts_for_budget(max(0.02, 100.0 / max(1, args.steps + args.warmup)))
+    vals, sample = [], ""
+    for i in range(args.warmup + args.steps):
+        v, sample = arm.time_step(n_take)
+        if i >= args.warmup:
+            vals.append(v)
+    v = sum(vals) / len(vals)
+    line = {
+        "metric": METRIC, "value": v, "unit": "us", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": v / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "impl": "reference",
+        "config": {"workload": f"{args.config} k={args.k}", "n_facts": shape.n_facts, "emb_dim": shape.emb_dim},
+        "cpu_baseline": {"value": v, "unit": "us", "cores": arm.cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }  # fmt: skip
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_27090_b200 import memstore as M
+    from paper_2607_27090_b200 import synth, workload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = synth.CONFIGS[args.config]
+    k = args.k
+    n_pool = args.query_pool
+    per_req_blocks = workload.blocks_per_request(shape, k)
+    wl = workload.build(args.config, seed=args.seed + rank, device=dev, n_query_pool=n_pool, scale_facts=args.scale_facts,
+                        num_blocks=args.pool_blocks or max(4096, per_req_blocks * n_pool))  # fmt: skip
+    store, cache = wl.store, wl.cache
+    tables = torch.from_numpy(synth.block_tables(args.seed + rank, cache.num_blocks, per_req_blocks, n_pool)).to(dev)
+    queries = torch.from_numpy(wl.queries).to(dev)
+    start = torch.full((1,), shape.start_pos, dtype=torch.int32, device=dev)
+    ids = torch.empty((1, k), dtype=torch.int32, device=dev)
+    n_tok = torch.zeros(n_pool, dtype=torch.int32, device=dev)
+    status = torch.zeros(n_pool, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        j = i % n_pool
+        store.retrieve(queries[j : j + 1], k, out_ids=ids, want_scores=False, stream=stream)
+        store.inject(ids, start, tables[j : j + 1], cache, out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1],
+                     flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert int(status.abs().sum()) == 0, "a request reported a data error"
+    m_pool = n_tok.cpu().numpy().astype(np.int64)
+    if args.warmup < n_pool:  # make sure every pool entry has been seen once for the byte accounting
+        for i in range(n_pool):
+            step(i)
+        barrier()
+        m_pool = n_tok.cpu().numpy().astype(np.int64)
+
+    launches0 = store.stats()["kernels_launched"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = store.stats()["kernels_launched"] - launches0
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+    us_per_request = ms_total * 1e3 / (args.steps * world)
+
+    # ---- per-part timing and the roofline of the dominant kernel (the copy kernel of inject) --------------
+    n_prof = min(args.steps, 400)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+    for a, b in evs:
+        a.record(stream)
+        b.record(stream)
+    r0 = [torch.cuda.Event(enable_timing=True) for _ in range(n_prof)]
+    r1 = [torch.cuda.Event(enable_timing=True) for _ in range(n_prof)]
+    torch.cuda.synchronize()
+    for i in range(n_prof):
+        j = i % n_pool
+        r0[i].record(stream)
+        store.retrieve(queries[j : j + 1], k, out_ids=ids, want_scores=False, stream=stream)
+        r1[i].record(stream)
+        store.set_profile_events(*evs[i])
+        store.inject(ids, start, tables[j : j + 1], cache, out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1],
+                     flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+    store.set_profile_events(None, None)
+    torch.cuda.synchronize()
+    copy_us = np.array([a.elapsed_time(b) * 1e3 for a, b in evs])
+    retr_us = np.array([a.elapsed_time(b) * 1e3 for a, b in zip(r0, r1)])
+    bytes_prof = np.array([workload.kv_bytes_moved(shape, int(m_pool[i % n_pool])) for i in range(n_prof)], dtype=np.float64)
+    copy_gbs = float(bytes_prof.sum() / (copy_us.sum() * 1e-6) / 1e9)
+    peak, peak_kind = measured_peaks()
+    mean_m = float(np.mean([m_pool[i % n_pool] for i in range(args.steps)]))
+    bytes_step = workload.kv_bytes_moved(shape, 1) * mean_m + workload.emb_bytes_scanned(shape, int(wl.lens.size))
+
+    # ---- end to end through the binding with HOST buffers ------------------------------------------------
+    n_e2e = min(args.steps, 500)
+    q_host = torch.from_numpy(wl.queries).pin_memory()
+    t_host = torch.from_numpy(synth.block_tables(args.seed + rank, cache.num_blocks, per_req_blocks, n_pool)).pin_memory()
+    s_host = torch.full((1,), shape.start_pos, dtype=torch.int32).pin_memory()
+    out_host = torch.empty((k + 2,), dtype=torch.int32).pin_memory()
+    q_dev = torch.empty_like(queries[:1])
+    t_dev = torch.empty_like(tables[:1])
+    s_dev = torch.empty_like(start)
+    res_dev = torch.empty((k + 2,), dtype=torch.int32, device=dev)
+    ids_v = res_dev[:k].view(1, k)
+
+    def e2e_step(i):
+        j = i % n_pool
+        q_dev.copy_(q_host[j : j + 1], non_blocking=True)
+        t_dev.copy_(t_host[j : j + 1], non_blocking=True)
+        s_dev.copy_(s_host, non_blocking=True)
+        store.retrieve(q_dev, k, out_ids=ids_v, want_scores=False, stream=stream)
+        store.inject(ids_v, s_dev, t_dev, cache, out_n_tokens=res_dev[k : k + 1], out_status=res_dev[k + 1 : k + 2],
+                     flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+        out_host.copy_(res_dev, non_blocking=True)
+        stream.synchronize()  # the caller needs ids / token count / status before it can schedule the request
+
+    for i in range(5):
+        e2e_step(i)
+    barrier()
+    e0.record(stream)
+    for i in range(n_e2e):
+        e2e_step(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t[0])
+    e2e_us = e2e_ms * 1e3 / (n_e2e * world)
+    h2d = q_host[0:1].numel() * q_host.element_size() + t_host[0:1].numel() * 4 + 4
+    d2h = (k + 2) * 4
+
+    line = {
+        "metric": METRIC, "value": us_per_request, "unit": "us", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 data, f32 arithmetic", "data": "synthetic",
+        "config": {
+            "workload": f"{args.config}: {wl.lens.size} facts of {shape.len_lo}-{shape.len_hi} tokens, L={shape.n_layers} "
+                        f"h={shape.n_kv_heads} d={shape.head_dim}, {shape.emb_dim}-d {shape.emb_dtype} embeddings, k={k}, "
+                        f"start {shape.start_pos}, block {shape.block_size}",
+            "mean_tokens_per_request": mean_m, "bytes_per_request": bytes_step,
+            "l2_policy": "inputs larger than L2: each request moves ~%.0f MB and rotates over %d queries / block tables"
+                         % (bytes_step / 1e6, n_pool),
+            "replicas": world,
+        },
+        "retrieve_us": float(np.median(retr_us)), "inject_copy_kernel_us": float(np.median(copy_us)),
+        "path_gbs": bytes_step / (us_per_request * world * 1e-6) / 1e9,
+        "roofline": {
+            "bound": "hbm", "kernel": "inject_copy_kernel", "achieved": copy_gbs, "peak": peak, "unit": "GB/s",
+            "frac": copy_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": copy_gbs / NOMINAL_HBM_GBS,
+            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.config, k)),
+            "algorithmic_bytes_per_launch": float(bytes_prof.mean()),
+        },
+        "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "clocks": clk.summary(),
+    }  # fmt: skip
+
+    if args.sweep_k:
+        sweep = {}
+        for kk in (5, 10, 20):
+            ids_k = torch.empty((1, kk), dtype=torch.int32, device=dev)
+            for i in range(10):
+                store.retrieve(queries[i % n_pool : i % n_pool + 1], kk, out_ids=ids_k, want_scores=False, stream=stream)
+                store.inject(ids_k, start, tables[i % n_pool : i % n_pool + 1], cache, flags=M.INJECT_REVERSE, stream=stream)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(args.steps):
+                j = i % n_pool
+                store.retrieve(queries[j : j + 1], kk, out_ids=ids_k, want_scores=False, stream=stream)
+                store.inject(ids_k, start, tables[j : j + 1], cache, out_n_tokens=n_tok[j : j + 1],
+                             out_status=status[j : j + 1], flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+            e1.record(stream)
+            torch.cuda.synchronize()
+            sweep[f"k{kk}_us"] = e0.elapsed_time(e1) * 1e3 / args.steps
+        line["sweep"] = sweep
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        arm = OracleArm(shape, k, args.seed)
+        n_take = arm.facts_for_budget(args.cpu_baseline_seconds)
+        vals, t_begin = [], time.perf_counter()
+        while not vals or (time.perf_counter() - t_begin < args.cpu_baseline_seconds and len(vals) < 100):
+            v, sample = arm.time_step(n_take)
+            vals.append(v)
+        line["cpu_baseline"] = {"value": sum(vals) / len(vals), "unit": "us", "cores": arm.cores, "kind": "oracle",
+                                "sample": f"mean of {len(vals)} repeats of: {sample}"}  # fmt: skip
+    if rank == 0:
+        print(json.dumps(line))
+    store.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) per launch of the copy kernel from an ncu capture; see profiles/.  None until measured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {}
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

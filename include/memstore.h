@@ -178,6 +178,15 @@ typedef struct {
 } memstore_stats_t;
 ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
 
+/*
+ * Measurement aid (no counterpart in the paper).  While both events are non-NULL, every memstore_inject
+ * records `before_copy` (a cudaEvent_t) on the call's stream just before the gather/rotate/scatter kernel
+ * and `after_copy` just after it, so that a benchmark can time that kernel alone with CUDA events.  The
+ * record between the plan kernel and the copy kernel removes their launch overlap, so leave this off
+ * (NULL, NULL) when timing whole calls.  The caller owns the events.
+ */
+ms_status memstore_set_profile_events(memstore_t* store, void* before_copy, void* after_copy);
+
 /* Text of the last error on this store (never NULL; valid until the next call on the store). */
 const char* memstore_last_error(memstore_t* store);
 

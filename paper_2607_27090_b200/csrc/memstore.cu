@@ -37,6 +37,7 @@ struct memstore {
   uint32_t tiles_capacity = 0;
   InjectCtrl* ctrl = nullptr;
   cudaEvent_t last_done = nullptr;
+  cudaEvent_t prof_before = nullptr, prof_after = nullptr;  // caller-owned, optional
   cudaStream_t last_stream = nullptr;
   bool have_last = false;
   // host mirrors
@@ -468,6 +469,11 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = 1;
+  const bool prof = s->prof_before && s->prof_after;
+  if (prof) {
+    lc.numAttrs = 0;  // an event between the two kernels: no programmatic overlap
+    MS_CUDA(s, cudaEventRecord(s->prof_before, st));
+  }
   cudaError_t e = cudaSuccess;
   dim3 grid((unsigned)resident_ctas);
   if (c.rope_style == MS_ROPE_HALF_SPLIT)
@@ -479,6 +485,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     cudaMemsetAsync(s->ctrl, 0, sizeof(InjectCtrl), st);
     return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
   }
+  if (prof) MS_CUDA(s, cudaEventRecord(s->prof_after, st));
   s->kernels_launched += 2;
   s->inject_calls++;
   return mark_last(s, st);
@@ -495,6 +502,15 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->kernels_launched = s->kernels_launched;
   out->arena_bytes = (int64_t)memstore_arena_bytes(&s->cfg);
   out->embedding_bytes = (int64_t)s->cfg.n_users * s->cfg.max_facts_per_user * s->cfg.emb_dim * (int64_t)emb_elem_size(s->cfg.emb_dtype);
+  return MS_OK;
+}
+
+ms_status memstore_set_profile_events(memstore_t* s, void* before_copy, void* after_copy) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  if ((before_copy == nullptr) != (after_copy == nullptr)) return fail(s, MS_ERR_INVALID_ARG, "give both events or neither");
+  s->prof_before = (cudaEvent_t)before_copy;
+  s->prof_after = (cudaEvent_t)after_copy;
   return MS_OK;
 }
 

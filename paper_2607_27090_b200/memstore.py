@@ -58,6 +58,7 @@ class _Stats(C.Structure):
 EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
+    "memstore_set_profile_events",
 )  # fmt: skip
 
 _lib = None
@@ -93,6 +94,8 @@ def load_library() -> C.CDLL:
     L.memstore_inject.argtypes = [vp, vp, i32, i32, vp, vp, i32, C.POINTER(_PagedCache), vp, vp, vp, i64, u32, vp]
     L.memstore_stats.restype = i32
     L.memstore_stats.argtypes = [vp, C.POINTER(_Stats)]
+    L.memstore_set_profile_events.restype = i32
+    L.memstore_set_profile_events.argtypes = [vp, vp, vp]
     L.memstore_last_error.restype = C.c_char_p
     L.memstore_last_error.argtypes = [vp]
     _lib = L
@@ -129,6 +132,7 @@ class PagedCache:
     head_stride: int
     num_blocks: int
     block_size: int
+    layout: str = "NHD"  # informational: how `allocate` shaped the tensors
 
     @classmethod
     def allocate(cls, n_layers, num_blocks, block_size, n_kv_heads, head_dim, device, layout="NHD", stacked=False, fill_bits=None):
@@ -152,6 +156,7 @@ class PagedCache:
         token_stride, head_stride = (n_kv_heads * head_dim, head_dim) if layout == "NHD" else (head_dim, block_size * head_dim)
         c = cls(k, v, layer_stride, blk, token_stride, head_stride, num_blocks, block_size)
         c._keep = keep
+        c.layout = layout
         return c
 
     def _struct(self) -> _PagedCache:
@@ -267,6 +272,16 @@ class MemStore:
                                        flags, _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out_n_tokens, out_status
+
+    def set_profile_events(self, before_copy=None, after_copy=None):
+        """torch.cuda.Event pair (created with enable_timing=True and already recorded once so that they own a
+        CUDA event) recorded around the copy kernel of every inject; (None, None) switches it off."""
+        if before_copy is None and after_copy is None:
+            self._check(self._lib.memstore_set_profile_events(self._h, None, None))
+            self._prof = None
+            return
+        self._prof = (before_copy, after_copy)
+        self._check(self._lib.memstore_set_profile_events(self._h, C.c_void_p(before_copy.cuda_event), C.c_void_p(after_copy.cuda_event)))
 
     def stats(self) -> dict:
         st = _Stats()

@@ -139,11 +139,12 @@ def gather_cache_rows(cache: PagedCache, slots: np.ndarray, layers=None):
     bs = cache.block_size
     sl = torch.from_numpy(np.asarray(slots, dtype=np.int64)).to(cache.k.device)
     blk, inb = sl // bs, sl % bs
-    nhd = cache.head_stride < cache.token_stride  # [L][blocks][bs][H][D]
+    nhd = cache.layout == "NHD"  # [L][blocks][bs][H][D]
     out = []
     for t in (cache.k, cache.v):
         x = t[l0:l1]
-        rows = x[:, blk, inb] if nhd else x[:, blk, :, inb]  # [nl, m, H, D] either way
+        # advanced indices split by a slice put the indexed dimension first: [m, nl, H, D] -> [nl, m, H, D]
+        rows = x[:, blk, inb] if nhd else x[:, blk, :, inb].permute(1, 0, 2, 3)
         out.append(bits(rows))
     return out
 
@@ -156,7 +157,7 @@ def untouched_mask_ok(cache: PagedCache, written_slots: np.ndarray, sentinel_bit
     if len(written_slots):
         keep[torch.from_numpy(np.asarray(written_slots, dtype=np.int64)).to(dev)] = False
     keep = keep.view(cache.num_blocks, bs)
-    nhd = cache.head_stride < cache.token_stride
+    nhd = cache.layout == "NHD"
     sent = sentinel_bits - 0x10000 if sentinel_bits >= 0x8000 else sentinel_bits
     for t in (cache.k, cache.v):
         for l in range(t.shape[0]):
