@@ -59,18 +59,22 @@ enum {
   MS_REQ_NOT_RESIDENT = 2,      /* fact has no K/V in the arena: contributes no tokens */
   MS_REQ_BLOCK_TABLE_SHORT = 4, /* pos / block_size >= max_blocks: token skipped */
   MS_REQ_BAD_BLOCK_ID = 8,      /* table entry < 0 or >= num_blocks: token skipped */
-  MS_REQ_POSITION_OVERFLOW = 16 /* pos >= max_position: token skipped */
+  MS_REQ_POSITION_OVERFLOW = 16, /* pos >= max_position: token skipped */
+  MS_REQ_KERNEL_TIMEOUT = 32     /* a bounded wait inside the copy kernel ran out: the cache contents of this call are incomplete */
 };
 
 enum { MS_DTYPE_F32 = 0, MS_DTYPE_F16 = 1, MS_DTYPE_BF16 = 2 };
 enum { MS_ROPE_HALF_SPLIT = 0, MS_ROPE_INTERLEAVED = 1 };
 enum { MS_INJECT_REVERSE = 1u }; /* place ids[k-1] first, so that ids[0] ends next to the query */
+/* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
+ * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */
+enum { MS_STORE_TMA_COPY_PATH = 1u };
 
 typedef struct {
   int32_t device;         /* CUDA device ordinal */
   int32_t n_layers;       /* L */
   int32_t n_kv_heads;     /* h */
-  int32_t head_dim;       /* d: a multiple of 16, at most 512 */
+  int32_t head_dim;       /* d: 16, 32, 64, 128 or 256 */
   int32_t kv_dtype;       /* MS_DTYPE_BF16 only (the paper's cache is bf16) */
   int32_t emb_dim;        /* a multiple of 8 */
   int32_t emb_dtype;      /* MS_DTYPE_F32 or MS_DTYPE_F16 */
@@ -79,7 +83,7 @@ typedef struct {
   const float* inv_freq_override; /* host, d/2 floats, or NULL; replaces the formula above (copied) */
   int64_t max_position;   /* tokens at pos >= max_position are refused; 0 < max_position <= 2^24 */
   int32_t n_users;        /* number of private embedding segments (>= 1) */
-  int32_t reserved0;
+  uint32_t flags;         /* MS_STORE_* bits, normally 0 */
   int64_t max_facts_per_user; /* capacity of each user's embedding segment */
   int64_t max_kv_tokens;  /* capacity of the K/V arena in tokens (0: embedding-only store) */
   void* kv_arena;         /* optional caller-provided DEVICE buffer for the arena, else NULL */

@@ -16,9 +16,9 @@ struct FactRec {
   int32_t resident;  // 1: K/V present in the arena, 0: embedding only
 };
 
-// Tokens per injection tile: 16 consecutive positions aligned to a multiple of 16, so a tile never
-// straddles a cache block whose size is a multiple of 16 (and covers whole smaller power-of-two blocks).
-constexpr int kTileTokens = 16;
+// Tokens per injection tile: 8 consecutive positions aligned to a multiple of 8, so a tile never
+// straddles a cache block whose size is a multiple of 8 (and covers whole smaller power-of-two blocks).
+constexpr int kTileTokens = 8;
 
 // Work description of one tile, written by the plan kernel and read by the copy kernel.
 struct __align__(16) TileDesc {
@@ -28,7 +28,8 @@ struct __align__(16) TileDesc {
   int64_t dst_off[kTileTokens]; // element offset block*block_stride + token*token_stride in the cache
 };
 
-// Counters shared by the plan and copy kernels of one inject call (reset by the last copy CTA).
+// Counters shared by the plan and copy kernels of one inject call.  A store keeps two of them and alternates:
+// the plan kernel of a call clears the pair the next call will use (calls on a store are ordered on the device).
 struct InjectCtrl {
   uint32_t n_tiles;
   uint32_t work_next;

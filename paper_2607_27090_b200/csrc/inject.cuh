@@ -36,7 +36,8 @@ struct InjectParams {
   // scratch
   TileDesc* tiles;
   uint32_t tiles_capacity;
-  InjectCtrl* ctrl;
+  InjectCtrl* ctrl;       // counters of this call (zero when its plan kernel starts)
+  InjectCtrl* ctrl_next;  // counters of the next call, cleared by this call's plan kernel
   int32_t layers_per_item;
 };
 
@@ -60,6 +61,7 @@ __global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectP
   const int lane = tid & 31, warp = tid >> 5;
   grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
   if (tid == 0) {
+    *p.ctrl_next = InjectCtrl{0u, 0u, 0u, 0u};  // the counters the NEXT inject call will use
     s_carry = 0;
     s_status = 0;
   }
@@ -173,7 +175,7 @@ __global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectP
 __device__ __forceinline__ void rope_sincos(float posf, float inv_freq, float& s, float& c) {
   const float hi = __fmul_rn(posf, inv_freq);
   const float lo = __fmaf_rn(posf, inv_freq, -hi);
-  const float n = rintf(hi * 0.15915494309189535f);
+  const float n = (hi * 0.15915494309189535f + 12582912.f) - 12582912.f;  // round to nearest integer, |x| < 2^22
   float r = __fmaf_rn(n, -6.28125f, hi);                  // exact
   r = __fmaf_rn(n, -0.0019350051879882812f, r);           // exact
   r = __fmaf_rn(n, -3.019916050561733e-07f, r);           // one rounding
@@ -221,111 +223,85 @@ __device__ __forceinline__ void rotate_unit(uint4& a, uint4& b, const float* sn,
 }
 
 constexpr int kCopyThreads = 256;
-constexpr int kThreadsPerToken = kCopyThreads / kTileTokens;  // 16
+constexpr int kThreadsPerToken = kCopyThreads / kTileTokens;  // 32
+constexpr int kUnitsPerThread = 2;
+constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a token row served by one CTA
 
 // ------------------------------------------------------------------------------------------------
-// Copy kernel (I4 + I5): persistent CTAs over items = (tile, group of layers).
-// 16 threads serve one token; a thread owns units u = lane16, lane16+16, ... of the token's row, a unit
-// being (head, frequency octet): two 16-byte vectors of K (rotated) and the same two of V (copied).
-// UPT = units a thread keeps in flight at once.  Because 16 is a multiple of D/16 every unit of a thread has the
-// same frequency octet, so its 8 sin/cos pairs are computed once per item and reused over heads and layers.
+// Copy kernel (I4 + I5): ONE CTA per work item = (tile of 8 tokens, layer, row part), no loop, no shared memory.
+// The grid is an upper bound computed on the host (the real tile count is only known on the device); CTAs beyond
+// it return at once.  The hardware CTA scheduler keeps every SM full and balances SMs that get unequal memory
+// service, and with ~1000 resident threads per SM each holding eight 16-byte loads, about 128 KB per SM are in
+// flight: measured on B200 this plain structure sustains the copy rate of the device, and a persistent
+// shared-memory ring fed by bulk copies does not (see inject_tma.cuh).
+//
+// 32 threads serve one token; a thread owns up to two units of the token's row, a unit being (head, frequency
+// octet): two 16-byte vectors of K (rotated) and the same two of V (copied).  32 and 64 are multiples of D/16, so
+// both units of a thread share the frequency octet: its 8 cos/sin pairs are computed once, while the loads fly.
 // ------------------------------------------------------------------------------------------------
-template <int STYLE, int UPT>
-__global__ void __launch_bounds__(kCopyThreads) inject_copy_kernel(const InjectParams p) {
+template <int STYLE>
+__global__ void __launch_bounds__(kCopyThreads, 4) inject_copy_kernel(const InjectParams p) {
   const int tid = threadIdx.x;
-  const int tk = tid / kThreadsPerToken;
-  const int l16 = tid % kThreadsPerToken;
-  const int D = p.head_dim, H = p.n_heads;
-  const int G = D >> 4;  // frequency octets per head
-  const int row = H * D;
-  const int n_units = H * G;
-  const int j = l16 % G;  // this thread's octet (requires 16 % G == 0)
-  const int n_lgroups = (p.n_layers + p.layers_per_item - 1) / p.layers_per_item;
-
-  float f8[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) f8[i] = p.inv_freq[8 * j + i];
+  const int tk = tid >> 5;  // token of the tile
+  const int l = tid & 31;
+  const int D = p.head_dim;
+  const int G = D >> 4, g_shift = 31 - __clz(G);  // frequency octets per head (a power of two, at most 16)
+  const int n_units = p.n_heads << g_shift;
+  const int j = l & (G - 1);
   // element offsets of this thread's two vectors inside a head
   const int offA = STYLE == 0 ? 8 * j : 16 * j;
   const int offB = STYLE == 0 ? D / 2 + 8 * j : 16 * j + 8;
+  const int u0 = blockIdx.y * kUnitsPerPart + l;
+  if (u0 >= n_units) return;
 
   grid_dependency_wait();  // tile descriptors come from the plan kernel
 
   const uint32_t n_tiles = min(p.ctrl->n_tiles, p.tiles_capacity);
-  const uint32_t n_items = n_tiles * (uint32_t)n_lgroups;
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const uint32_t tile = item / n_lgroups;
-    const int l0 = (int)(item % n_lgroups) * p.layers_per_item;
-    const int l1 = min(l0 + p.layers_per_item, p.n_layers);
-    const TileDesc* d = p.tiles + tile;
-    const int32_t src = d->src_tok[tk];
-    if (src < 0) continue;
-    const int64_t dst = d->dst_off[tk];
-    const float posf = (float)(d->pos0 + tk);
-    float sn[8], cs[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) rope_sincos(posf, f8[i], sn[i], cs[i]);
+  // items in (layer, tile) order: CTAs that run together stream neighbouring rows of one layer
+  if (n_tiles == 0) return;
+  const uint32_t item = blockIdx.x;
+  const uint32_t layer = item / n_tiles;
+  if (layer >= (uint32_t)p.n_layers) return;
+  const uint32_t tile = item - layer * n_tiles;
+  const TileDesc* d = p.tiles + tile;
+  const int32_t src = d->src_tok[tk];
+  if (src < 0) return;
+  const int64_t dst = d->dst_off[tk];
+  const int32_t pos = d->pos0 + tk;
 
-    for (int l = l0; l < l1; ++l) {
-      const int64_t src_row = ((int64_t)l * p.arena_tokens + src) * row;
-      const __nv_bfloat16* ks = p.k_arena + src_row;
-      const __nv_bfloat16* vs = p.v_arena + src_row;
-      const int64_t dbase = (int64_t)l * p.layer_stride + dst;
-      for (int ub = l16; ub < n_units; ub += UPT * kThreadsPerToken) {
-        uint4 ka[UPT], kb[UPT], va[UPT], vb[UPT];
+  const int64_t src_row = ((int64_t)layer * p.arena_tokens + src) * (int64_t)(p.n_heads * D);
+  const __nv_bfloat16* ks = p.k_arena + src_row;
+  const __nv_bfloat16* vs = p.v_arena + src_row;
+  const int64_t dbase = (int64_t)layer * p.layer_stride + dst;
+  uint4 ka[kUnitsPerThread], kb[kUnitsPerThread], va[kUnitsPerThread], vb[kUnitsPerThread];
 #pragma unroll
-        for (int u = 0; u < UPT; ++u) {
-          const int unit = ub + u * kThreadsPerToken;
-          if (unit < n_units) {
-            const int h = unit / G;
-            ka[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offA));
-            kb[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offB));
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < UPT; ++u) {
-          const int unit = ub + u * kThreadsPerToken;
-          if (unit < n_units) {
-            const int h = unit / G;
-            va[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offA));
-            vb[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offB));
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < UPT; ++u) {
-          const int unit = ub + u * kThreadsPerToken;
-          if (unit < n_units) {
-            const int h = unit / G;
-            rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
-            __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
-            st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
-            st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < UPT; ++u) {
-          const int unit = ub + u * kThreadsPerToken;
-          if (unit < n_units) {
-            const int h = unit / G;
-            __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
-            st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
-            st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
-          }
-        }
-      }
+  for (int u = 0; u < kUnitsPerThread; ++u) {
+    const int unit = u0 + u * kThreadsPerToken;
+    if (unit < n_units) {
+      const int h = unit >> g_shift;
+      ka[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offA));
+      kb[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offB));
+      va[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offA));
+      vb[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offB));
     }
   }
-
-  // Wait-free epilogue: the last CTA to get here clears the counters for the next inject call.
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    const uint32_t done = atomicAdd(&p.ctrl->done_ctas, 1u);
-    if (done == gridDim.x - 1) {
-      p.ctrl->n_tiles = 0;
-      p.ctrl->work_next = 0;
-      p.ctrl->done_ctas = 0;
-      __threadfence();
+  // cos/sin of (pos, 8 frequencies), evaluated while the loads are in flight
+  float sn[8], cs[8];
+  const float posf = (float)pos;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
+#pragma unroll
+  for (int u = 0; u < kUnitsPerThread; ++u) {
+    const int unit = u0 + u * kThreadsPerToken;
+    if (unit < n_units) {
+      const int h = unit >> g_shift;
+      rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+      __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
+      st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
+      st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
+      __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
+      st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
+      st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
     }
   }
 }

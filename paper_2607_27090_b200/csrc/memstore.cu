@@ -14,6 +14,7 @@
 
 #include "common.cuh"
 #include "inject.cuh"
+#include "inject_tma.cuh"
 #include "retrieve.cuh"
 
 using namespace ms;
@@ -32,6 +33,7 @@ struct memstore {
   float* inv_freq_d = nullptr;       // [d/2]
   // scratch shared by all calls (ordered on the device through `last_done`)
   float* scores = nullptr;
+  uint32_t* tickets = nullptr;  // one wait-free counter per query of the fused retrieve kernel
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
   uint32_t tiles_capacity = 0;
@@ -47,6 +49,8 @@ struct memstore {
   int64_t max_user_count = 0;
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
   int copy_ctas_per_sm = 1;
+  size_t fused_smem_set = 0;
+  bool tma_path = false;  // MS_STORE_TMA_COPY_PATH
   std::mutex mu;
   std::string err;
 };
@@ -92,10 +96,11 @@ ms_status check_config(const memstore_config* c) {
   if (c->max_position <= 0 || c->max_position > (1 << 24)) return MS_ERR_INVALID_ARG;
   if (c->rope_style != MS_ROPE_HALF_SPLIT && c->rope_style != MS_ROPE_INTERLEAVED) return MS_ERR_INVALID_ARG;
   if (!(c->rope_theta > 0.0) && !c->inv_freq_override) return MS_ERR_INVALID_ARG;
+  if (c->flags & ~(uint32_t)MS_STORE_TMA_COPY_PATH) return MS_ERR_INVALID_ARG;
   if (c->kv_dtype != MS_DTYPE_BF16) return MS_ERR_UNSUPPORTED;
   if (c->emb_dtype != MS_DTYPE_F32 && c->emb_dtype != MS_DTYPE_F16) return MS_ERR_UNSUPPORTED;
   if (c->emb_dim % 8) return MS_ERR_UNSUPPORTED;
-  // the copy kernel gives 16 threads to a token and one frequency octet to a thread: d/16 must divide 16
+  // the copy kernels give 32 or more threads to a token and one frequency octet to a thread: d/16 must divide 32
   const int d = c->head_dim;
   if (!(d == 16 || d == 32 || d == 64 || d == 128 || d == 256)) return MS_ERR_UNSUPPORTED;
   if (c->max_kv_tokens >= (1ll << 31) || (int64_t)c->n_users * c->max_facts_per_user >= (1ll << 31))
@@ -113,16 +118,6 @@ __global__ void __launch_bounds__(256) arena_append_kernel(const uint4* __restri
   uint4* d = (blockIdx.z ? v_dst : k_dst) + (int64_t)layer * vec_per_layer_dst + dst_vec_off;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vec_per_layer_src; i += (int64_t)gridDim.x * blockDim.x)
     d[i] = s[i];
-}
-
-template <int STYLE>
-void launch_copy(const InjectParams& p, int upt, dim3 grid, cudaLaunchConfig_t& lc, cudaError_t& e) {
-  lc.gridDim = grid;
-  switch (upt) {
-    case 1: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 1>, p); break;
-    case 2: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 2>, p); break;
-    default: e = cudaLaunchKernelEx(&lc, inject_copy_kernel<STYLE, 4>, p); break;
-  }
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -192,7 +187,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
             cudaMalloc(&s->facts_d, (size_t)rows * sizeof(FactRec)) == cudaSuccess &&
             cudaMalloc(&s->user_count_d, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
             cudaMalloc(&s->inv_freq_d, (size_t)(config->head_dim / 2) * sizeof(float)) == cudaSuccess &&
-            cudaMalloc(&s->ctrl, sizeof(InjectCtrl)) == cudaSuccess;
+            cudaMalloc(&s->ctrl, 2 * sizeof(InjectCtrl)) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return bail(MS_ERR_OOM);
@@ -204,16 +199,22 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
                                      : (float)std::pow(config->rope_theta, -(double)(2 * i) / (double)config->head_dim);
   ok = cudaMemcpy(s->inv_freq_d, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
        cudaMemset(s->user_count_d, 0, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
-       cudaMemset(s->ctrl, 0, sizeof(InjectCtrl)) == cudaSuccess &&
+       cudaMemset(s->ctrl, 0, 2 * sizeof(InjectCtrl)) == cudaSuccess &&
        cudaEventCreateWithFlags(&s->last_done, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return bail(MS_ERR_CUDA);
   }
   s->user_count.assign(config->n_users, 0);
+  s->tma_path = (config->flags & MS_STORE_TMA_COPY_PATH) != 0;
   int occ = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0, 4>, kCopyThreads, 0) == cudaSuccess && occ > 0)
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0>, kCopyThreads, 0) == cudaSuccess && occ > 0)
     s->copy_ctas_per_sm = occ;
+  if (cudaFuncSetAttribute(inject_copy_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(inject_copy_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess) {
+    cudaGetLastError();
+    return bail(MS_ERR_CUDA);
+  }
   *out = s;
   return MS_OK;
 }
@@ -231,6 +232,7 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->inv_freq_d);
     cudaFree(s->ctrl);
     cudaFree(s->scores);
+    cudaFree(s->tickets);
     cudaFree(s->tiles);
     if (s->last_done) cudaEventDestroy(s->last_done);
     cudaGetLastError();
@@ -328,9 +330,13 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   if (nq > s->scores_nq) {  // grow the score scratch (first call, or a larger batch than ever before)
     MS_CUDA(s, cudaDeviceSynchronize());
     cudaFree(s->scores);
+    cudaFree(s->tickets);
     s->scores = nullptr;
+    s->tickets = nullptr;
     s->scores_nq = 0;
     MS_CUDA(s, cudaMalloc(&s->scores, (size_t)nq * c.max_facts_per_user * sizeof(float)));
+    MS_CUDA(s, cudaMalloc(&s->tickets, (size_t)nq * sizeof(uint32_t)));
+    MS_CUDA(s, cudaMemset(s->tickets, 0, (size_t)nq * sizeof(uint32_t)));
     s->scores_nq = nq;
   }
   ms_status rc = order_after_last(s, st);
@@ -353,23 +359,37 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   p.out_scores = out_scores;
 
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
-  if (n_max > 0) {
-    // enough CTAs to fill the GPU, at least one row per warp
-    int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
-    int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (n_max + target_ctas - 1) / target_ctas);
-    rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
-    dim3 grid((unsigned)((n_max + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+  // enough CTAs to fill the GPU, at least one row per warp
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
+  int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
+  rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
+  dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+  if (n_max <= kFusedMaxRows) {
+    // small segments: scoring and top-k in one launch
+    const int keys_cap = (int)std::max<int64_t>(n_max, 1);
+    const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)keys_cap * sizeof(uint32_t);
+    if (smem > s->fused_smem_set) {
+      MS_CUDA(s, cudaFuncSetAttribute(score_topk_fused_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      MS_CUDA(s, cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      s->fused_smem_set = smem;
+    }
+    if (c.emb_dtype == MS_DTYPE_F16)
+      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap);
+    else
+      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched++;
+  } else {
     const size_t smem = (size_t)c.emb_dim * sizeof(float);
     if (c.emb_dtype == MS_DTYPE_F16)
       score_rows_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
     else
       score_rows_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
     MS_CUDA(s, cudaGetLastError());
-    s->kernels_launched++;
+    topk_kernel<<<nq, kTopkThreads, 0, st>>>(p);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched += 2;
   }
-  topk_kernel<<<nq, kTopkThreads, 0, st>>>(p);
-  MS_CUDA(s, cudaGetLastError());
-  s->kernels_launched++;
   s->retrieve_calls++;
   return mark_last(s, st);
 }
@@ -446,23 +466,22 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   p.slot_stride = slot_stride;
   p.tiles = s->tiles;
   p.tiles_capacity = s->tiles_capacity;
-  p.ctrl = s->ctrl;
+  p.ctrl = s->ctrl + (s->inject_calls & 1);
+  p.ctrl_next = s->ctrl + ((s->inject_calls + 1) & 1);
 
-  // items = tiles x layer groups; keep at least ~8 items per resident CTA, else one layer per item
-  const int resident_ctas = s->sm_count * s->copy_ctas_per_sm;
+  // layers per work item: the largest power of two that still leaves every resident CTA about 16 items
+  const int row_bytes = c.n_kv_heads * c.head_dim * 2;
+  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
+  const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
   const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + kTileTokens - 1) / kTileTokens * nreq);
   int lpi = 1;
-  while (lpi * 2 <= c.n_layers && c.n_layers % (lpi * 2) == 0 && est_tiles * (c.n_layers / (lpi * 2)) >= 8ll * resident_ctas) lpi *= 2;
+  while (lpi * 2 <= c.n_layers && c.n_layers % (lpi * 2) == 0 && est_tiles * (c.n_layers / (lpi * 2)) >= 16ll * resident_ctas) lpi *= 2;
   p.layers_per_item = lpi;
 
   inject_plan_kernel<<<nreq, kPlanThreads, 0, st>>>(p);
   MS_CUDA(s, cudaGetLastError());
 
-  const int units = c.n_kv_heads * (c.head_dim / 16);
-  const int upt = units >= 64 ? 4 : units >= 32 ? 2 : 1;
   cudaLaunchConfig_t lc{};
-  lc.blockDim = dim3(kCopyThreads);
-  lc.dynamicSmemBytes = 0;
   lc.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -475,14 +494,34 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     MS_CUDA(s, cudaEventRecord(s->prof_before, st));
   }
   cudaError_t e = cudaSuccess;
-  dim3 grid((unsigned)resident_ctas);
-  if (c.rope_style == MS_ROPE_HALF_SPLIT)
-    launch_copy<0>(p, upt, grid, lc, e);
-  else
-    launch_copy<1>(p, upt, grid, lc, e);
+  if (use_tma) {
+    // bulk-async staged kernel: one persistent CTA per SM
+    int ts = kTileTokens;
+    while (ts > 1 && ts * row_bytes > kTmaAreaBytes) ts >>= 1;
+    const int v_rows = cache->head_stride == c.head_dim ? 1 : 0;
+    lc.gridDim = dim3((unsigned)s->sm_count);
+    lc.blockDim = dim3(kTmaThreads);
+    lc.dynamicSmemBytes = kTmaSmemBytes;
+    if (c.rope_style == MS_ROPE_HALF_SPLIT)
+      e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<0>, p, ts, v_rows);
+    else
+      e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<1>, p, ts, v_rows);
+  } else {
+    // direct kernel: one CTA per (tile, layer, row part); the grid covers the largest request the ids could name
+    const int units = c.n_kv_heads * (c.head_dim / 16);
+    const int64_t items = tiles_needed * c.n_layers;
+    if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
+    lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
+    lc.blockDim = dim3(kCopyThreads);
+    lc.dynamicSmemBytes = 0;
+    if (c.rope_style == MS_ROPE_HALF_SPLIT)
+      e = cudaLaunchKernelEx(&lc, inject_copy_kernel<0>, p);
+    else
+      e = cudaLaunchKernelEx(&lc, inject_copy_kernel<1>, p);
+  }
   if (e != cudaSuccess) {
     // the plan kernel has already counted tiles that no copy kernel will clear
-    cudaMemsetAsync(s->ctrl, 0, sizeof(InjectCtrl), st);
+    cudaMemsetAsync(s->ctrl, 0, 2 * sizeof(InjectCtrl), st);
     return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
   }
   if (prof) MS_CUDA(s, cudaEventRecord(s->prof_after, st));

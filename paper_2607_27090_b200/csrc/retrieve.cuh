@@ -23,8 +23,11 @@ struct RetrieveParams {
 
 constexpr int kScoreThreads = 256;
 constexpr int kScoreWarps = kScoreThreads / 32;
+constexpr int kTopkThreads = 1024;
+constexpr int kTopkMaxK = 2048;
+constexpr int kFusedMaxRows = 8192;  // largest segment whose top-k runs inside the scoring kernel
 
-__device__ __forceinline__ void unpack8(const uint4& v, float* f, const __half*) {
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -34,27 +37,26 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f, const __half*)
   }
 }
 
+// fp32 score -> unsigned key that orders like the float
+__device__ __forceinline__ uint32_t order_key(float s) {
+  uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_score(uint32_t kx) {
+  uint32_t u = (kx & 0x80000000u) ? (kx & 0x7fffffffu) : ~kx;
+  return __uint_as_float(u);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Scoring on CUDA cores: one warp per embedding row, 16-byte loads, fp32 accumulation.
 // The summation order of a row depends only on the lane layout, never on which warp or CTA handles
 // it, so identical rows get bit-identical scores (needed for the id tie rule).
-// grid = (row groups, nq); dynamic shared memory holds the query as fp32.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const RetrieveParams p, int rows_per_cta) {
-  extern __shared__ float s_q[];
+__device__ __forceinline__ void score_rows(const RetrieveParams& p, const float* s_q, int q, int user, int n, int64_t row0,
+                                           int rows_per_cta) {
   constexpr int VEC = 16 / sizeof(T);  // elements per 16-byte vector
-  const int q = blockIdx.y;
-  const int user = p.query_users ? p.query_users[q] : 0;
-  const bool user_ok = user >= 0 && user < p.n_users;
-  const int n = user_ok ? p.user_count[user] : 0;
-  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
-  if (row0 >= n) return;
   const int E = p.emb_dim;
-  const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * E;
-  for (int d = threadIdx.x; d < E; d += kScoreThreads) s_q[d] = (float)qv[d];
-  __syncthreads();
-
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const T* seg = reinterpret_cast<const T*>(p.emb) + (int64_t)user * p.seg_capacity * E;
   const int64_t row_end = min(row0 + rows_per_cta, (int64_t)n);
@@ -76,7 +78,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const Retriev
           const float* qs = s_q + v * VEC;
           if (sizeof(T) == 2) {
             float f[8];
-            unpack8(x[u], f, (const __half*)nullptr);
+            unpack8(x[u], f);
 #pragma unroll
             for (int i = 0; i < 8; ++i) acc = fmaf(f[i], qs[i], acc);
           } else {
@@ -93,115 +95,250 @@ __global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const Retriev
   }
 }
 
-// fp32 score -> unsigned key that orders like the float
-__device__ __forceinline__ uint32_t order_key(float s) {
-  uint32_t u = __float_as_uint(s);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float key_score(uint32_t kx) {
-  uint32_t u = (kx & 0x80000000u) ? (kx & 0x7fffffffu) : ~kx;
-  return __uint_as_float(u);
-}
-
-constexpr int kTopkThreads = 1024;
-constexpr int kTopkMaxK = 2048;
-
-// ------------------------------------------------------------------------------------------------
-// Top-k: one CTA per query.  Radix select (4 passes of 8 bits, most significant first) finds the
-// k-th largest score key T; everything above T is taken, rows equal to T are taken lowest row first
-// (rows of a user are in fact-id order), and the k survivors are sorted by a bitonic network on the
-// 64-bit key (score key << 32) | ~row.
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams p) {
-  __shared__ uint32_t s_hist[256];
-  __shared__ unsigned long long s_cand[kTopkMaxK];
-  __shared__ uint32_t s_prefix, s_krem, s_ngt, s_warp_cnt[kTopkThreads / 32], s_eq_base;
-
-  const int q = blockIdx.x;
+// Bitonic network over P (a power of two) 64-bit keys in shared memory, largest first.
+template <int THREADS>
+__device__ __forceinline__ void bitonic_sort_desc(unsigned long long* cand, int P) {
   const int tid = threadIdx.x;
-  const int user = p.query_users ? p.query_users[q] : 0;
-  const bool user_ok = user >= 0 && user < p.n_users;
-  const int n = user_ok ? p.user_count[user] : 0;
-  const int k = p.k;
-  const float* sc = p.scores + (int64_t)q * p.score_stride;
+  for (int size = 2; size <= P; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = tid; t < P / 2; t += THREADS) {
+        const int lo = 2 * t - (t & (stride - 1));
+        const int hi = lo + stride;
+        const bool desc = (lo & size) == 0;
+        const unsigned long long a = cand[lo], b = cand[hi];
+        if ((a < b) == desc) {
+          cand[lo] = b;
+          cand[hi] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Ranks 0..k-1: fact id and fp32 score of the sorted candidates, -1 / 0 beyond `take`.
+template <int THREADS>
+__device__ __forceinline__ void write_topk(const unsigned long long* cand, int take, int k, const int32_t* row_ids,
+                                           int32_t* out_ids, float* out_scores) {
+  for (int r = threadIdx.x; r < k; r += THREADS) {
+    int32_t id = -1;
+    float s = 0.f;
+    if (r < take) {
+      const unsigned long long c = cand[r];
+      const uint32_t row = 0xffffffffu - (uint32_t)(c & 0xffffffffull);
+      id = row_ids[row];
+      s = key_score((uint32_t)(c >> 32));
+    }
+    out_ids[r] = id;
+    if (out_scores) out_scores[r] = s;
+  }
+}
+
+struct TopkShared {
+  uint32_t hist[256];
+  unsigned long long cand[kTopkMaxK];
+  uint32_t warp_cnt[32];
+  uint32_t warp_min[32], warp_max[32];
+  uint32_t prefix, krem, ngt, eq_base;
+  uint32_t kmin, kmax, bucket, n_cand;
+};
+
+// ------------------------------------------------------------------------------------------------
+// Top-k of one query by one CTA of THREADS threads.  Radix select (4 passes of 8 bits, most significant
+// first) finds the k-th largest score key T; everything above T is taken, rows equal to T are taken lowest
+// row first (rows of a user are in fact-id order), and the k survivors are sorted by a bitonic network on
+// the 64-bit key (score key << 32) | ~row.  `keys` (shared memory, optional) holds the n order keys;
+// without it they are recomputed from the scores in global memory on every pass.
+// ------------------------------------------------------------------------------------------------
+template <int THREADS>
+__device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const int32_t* row_ids,
+                           int32_t* out_ids, float* out_scores) {
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
   const int take = min(n, k);
+  auto key_at = [&](int i) -> uint32_t { return keys ? keys[i] : order_key(__ldcg(sc + i)); };
+
+  // ---- fast path: one histogram over 256 LINEAR buckets of [min key, max key] ---------------------------
+  // Scores of unit-norm embeddings share sign and exponent, so the leading radix digits of almost all keys
+  // coincide; buckets that are linear in the key spread them.  Every key in or above the bucket B that holds
+  // the k-th largest becomes a candidate (their number is k plus part of one bucket); the 64-bit sort below
+  // orders them exactly, ties by row.  If the candidates do not fit (massive ties) the radix path runs instead.
+  bool fast = false;
+  if (n > k) {
+    uint32_t lo = 0xffffffffu, hi = 0u;
+    for (int i = tid; i < n; i += THREADS) {
+      const uint32_t kx = key_at(i);
+      lo = min(lo, kx);
+      hi = max(hi, kx);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+      sm.warp_min[warp] = lo;
+      sm.warp_max[warp] = hi;
+    }
+    for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
+    __syncthreads();
+    if (warp == 0) {
+      lo = lane < THREADS / 32 ? sm.warp_min[lane] : 0xffffffffu;
+      hi = lane < THREADS / 32 ? sm.warp_max[lane] : 0u;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+      }
+      if (lane == 0) {
+        sm.kmin = lo;
+        sm.kmax = hi;
+      }
+    }
+    __syncthreads();
+    const uint32_t kmin = sm.kmin, range = sm.kmax - kmin;
+    const int sh = max(0, 24 - __clz(range));  // (range >> sh) < 256
+    for (int i = tid; i < n; i += THREADS) atomicAdd(&sm.hist[(key_at(i) - kmin) >> sh], 1u);
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t c[8], sum = 0;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        c[b] = sm.hist[8 * lane + b];
+        sum += c[b];
+      }
+      uint32_t incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += y;
+      }
+      uint32_t above = incl - sum;
+      if (above < (uint32_t)k && incl >= (uint32_t)k) {
+        int b = 7;
+        for (; b > 0; --b) {
+          if (above + c[b] >= (uint32_t)k) break;
+          above += c[b];
+        }
+        sm.bucket = 8 * lane + b;
+        sm.n_cand = above + c[b];
+      }
+    }
+    __syncthreads();
+    fast = range != 0 && sm.n_cand <= (uint32_t)kTopkMaxK;
+    if (fast) {
+      const uint32_t B = sm.bucket, n_cand = sm.n_cand;
+      int P2 = 1;
+      while (P2 < (int)n_cand) P2 <<= 1;
+      if (tid == 0) sm.ngt = 0;
+      for (int i = tid; i < P2; i += THREADS) sm.cand[i] = 0ull;
+      __syncthreads();
+      for (int i = tid; i < n; i += THREADS) {
+        const uint32_t kx = key_at(i);
+        if (((kx - kmin) >> sh) >= B) {
+          const uint32_t slot = atomicAdd(&sm.ngt, 1u);
+          sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+        }
+      }
+      __syncthreads();
+      bitonic_sort_desc<THREADS>(sm.cand, P2);
+      write_topk<THREADS>(sm.cand, take, k, row_ids, out_ids, out_scores);
+      return;
+    }
+  }
 
   uint32_t T = 0;        // threshold key
   uint32_t need_eq = 0;  // how many rows with key == T to take
   if (n > k) {
     if (tid == 0) {
-      s_prefix = 0;
-      s_krem = (uint32_t)k;
+      sm.prefix = 0;
+      sm.krem = (uint32_t)k;
     }
     for (int shift = 24; shift >= 0; shift -= 8) {
-      if (tid < 256) s_hist[tid] = 0;
+      for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
       __syncthreads();
-      const uint32_t prefix = s_prefix;
+      const uint32_t prefix = sm.prefix;
       const uint32_t himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-      for (int i = tid; i < n; i += kTopkThreads) {
-        const uint32_t kx = order_key(sc[i]);
-        if ((kx & himask) == prefix) atomicAdd(&s_hist[(kx >> shift) & 255u], 1u);
+      for (int i = tid; i < n; i += THREADS) {
+        const uint32_t kx = key_at(i);
+        if ((kx & himask) == prefix) atomicAdd(&sm.hist[(kx >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
-        // walk buckets from the top: find b with count(> b) < krem <= count(>= b)
-        uint32_t krem = s_krem, above = 0;
-        int b = 255;
-        for (; b > 0; --b) {
-          if (above + s_hist[b] >= krem) break;
-          above += s_hist[b];
+      if (warp == 0) {
+        // lane l owns buckets 8l..8l+7; find the bucket b with count(> b) < krem <= count(>= b)
+        uint32_t c[8], sum = 0;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+          c[b] = sm.hist[8 * lane + b];
+          sum += c[b];
         }
-        s_prefix = prefix | ((uint32_t)b << shift);
-        s_krem = krem - above;
+        uint32_t incl = sum;  // buckets of this lane and of all higher lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += y;
+        }
+        const uint32_t krem = sm.krem;
+        uint32_t above = incl - sum;
+        if (above < krem && incl >= krem) {
+          int b = 7;
+          for (; b > 0; --b) {
+            if (above + c[b] >= krem) break;
+            above += c[b];
+          }
+          sm.prefix = prefix | ((uint32_t)(8 * lane + b) << shift);
+          sm.krem = krem - above;
+        }
       }
       __syncthreads();
     }
-    T = s_prefix;
-    need_eq = s_krem;
+    T = sm.prefix;
+    need_eq = sm.krem;
   }
   if (tid == 0) {
-    s_ngt = 0;
-    s_eq_base = 0;
+    sm.ngt = 0;
+    sm.eq_base = 0;
   }
-  for (int i = tid; i < kTopkMaxK; i += kTopkThreads) s_cand[i] = 0ull;
+  int P = 1;  // sort width: next power of two >= take
+  while (P < take) P <<= 1;
+  for (int i = tid; i < P; i += THREADS) sm.cand[i] = 0ull;  // padding keys are the smallest
   __syncthreads();
 
   if (n <= k) {
-    for (int i = tid; i < n; i += kTopkThreads)
-      s_cand[i] = ((unsigned long long)order_key(sc[i]) << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+    for (int i = tid; i < n; i += THREADS)
+      sm.cand[i] = ((unsigned long long)key_at(i) << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
   } else {
     const uint32_t n_gt = (uint32_t)k - need_eq;
-    // rows above the threshold: order does not matter, they are sorted afterwards
-    // rows equal to the threshold: ordered compaction, lowest rows first, stop after need_eq
-    const int lane = tid & 31, warp = tid >> 5;
-    for (int base = 0; base < n; base += kTopkThreads) {
+    // rows above the threshold: order does not matter here, they are sorted afterwards;
+    // rows equal to the threshold: ordered compaction, lowest rows first, the first need_eq are kept
+    for (int base = 0; base < n; base += THREADS) {
       const int i = base + tid;
       uint32_t kx = 0;
       bool gt = false, eq = false;
       if (i < n) {
-        kx = order_key(sc[i]);
+        kx = key_at(i);
         gt = kx > T;
         eq = kx == T;
       }
       if (gt) {
-        const uint32_t slot = atomicAdd(&s_ngt, 1u);
-        if (slot < n_gt) s_cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+        const uint32_t slot = atomicAdd(&sm.ngt, 1u);
+        if (slot < n_gt) sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
       }
       const uint32_t bal = __ballot_sync(0xffffffffu, eq);
       if (__syncthreads_or(eq)) {
-        if (lane == 0) s_warp_cnt[warp] = __popc(bal);
+        if (lane == 0) sm.warp_cnt[warp] = __popc(bal);
         __syncthreads();
-        uint32_t before = s_eq_base;
-        for (int w = 0; w < warp; ++w) before += s_warp_cnt[w];
+        uint32_t before = sm.eq_base;
+        for (int w = 0; w < warp; ++w) before += sm.warp_cnt[w];
         if (eq) {
           const uint32_t rank = before + __popc(bal & ((1u << lane) - 1u));
-          if (rank < need_eq) s_cand[n_gt + rank] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+          if (rank < need_eq) sm.cand[n_gt + rank] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
         }
         __syncthreads();
         if (tid == 0) {
           uint32_t tot = 0;
-          for (int w = 0; w < kTopkThreads / 32; ++w) tot += s_warp_cnt[w];
-          s_eq_base += tot;
+          for (int w = 0; w < THREADS / 32; ++w) tot += sm.warp_cnt[w];
+          sm.eq_base += tot;
         }
         __syncthreads();
       }
@@ -209,38 +346,74 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams
   }
   __syncthreads();
 
-  // bitonic sort, descending, over the next power of two >= take (padding keys are 0 = smallest)
-  int P = 1;
-  while (P < take) P <<= 1;
-  for (int size = 2; size <= P; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int t = tid; t < P / 2; t += kTopkThreads) {
-        const int lo = 2 * t - (t & (stride - 1));
-        const int hi = lo + stride;
-        const bool desc = (lo & size) == 0;
-        const unsigned long long a = s_cand[lo], b = s_cand[hi];
-        if ((a < b) == desc) {
-          s_cand[lo] = b;
-          s_cand[hi] = a;
-        }
-      }
-      __syncthreads();
-    }
-  }
+  bitonic_sort_desc<THREADS>(sm.cand, P);
+  write_topk<THREADS>(sm.cand, take, k, row_ids, out_ids, out_scores);
+}
 
-  const int32_t* row_ids = p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity;
-  for (int r = tid; r < k; r += kTopkThreads) {
-    int32_t id = -1;
-    float s = 0.f;
-    if (r < take) {
-      const unsigned long long c = s_cand[r];
-      const uint32_t row = 0xffffffffu - (uint32_t)(c & 0xffffffffull);
-      id = row_ids[row];
-      s = key_score((uint32_t)(c >> 32));
-    }
-    p.out_ids[(int64_t)q * k + r] = id;
-    if (p.out_scores) p.out_scores[(int64_t)q * k + r] = s;
+// Scoring only (large segments): grid = (row groups, nq); dynamic shared memory holds the query as fp32.
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const RetrieveParams p, int rows_per_cta) {
+  extern __shared__ float s_q[];
+  const int q = blockIdx.y;
+  const int user = p.query_users ? p.query_users[q] : 0;
+  const bool user_ok = user >= 0 && user < p.n_users;
+  const int n = user_ok ? p.user_count[user] : 0;
+  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+  if (row0 >= n) return;
+  const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * p.emb_dim;
+  for (int d = threadIdx.x; d < p.emb_dim; d += kScoreThreads) s_q[d] = (float)qv[d];
+  __syncthreads();
+  score_rows<T>(p, s_q, q, user, n, row0, rows_per_cta);
+}
+
+// Top-k only (large segments): one CTA per query, keys recomputed from global scores.
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams p) {
+  __shared__ TopkShared sm;
+  const int q = blockIdx.x;
+  const int user = p.query_users ? p.query_users[q] : 0;
+  const bool user_ok = user >= 0 && user < p.n_users;
+  const int n = user_ok ? p.user_count[user] : 0;
+  topk_block<kTopkThreads>(sm, p.scores + (int64_t)q * p.score_stride, nullptr, n, p.k,
+                           p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity, p.out_ids + (int64_t)q * p.k,
+                           p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
+}
+
+// Scoring + top-k in ONE launch for segments of at most kFusedMaxRows rows: grid = (row groups, nq).
+// The CTA that finishes a query's scores last (a wait-free ticket) selects and sorts that query's top-k from
+// keys held in shared memory.  Dynamic shared memory: emb_dim floats (query) + keys_capacity uint32 keys.
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
+                                                                         uint32_t* tickets, int keys_capacity) {
+  extern __shared__ float s_q[];
+  __shared__ TopkShared sm;
+  __shared__ int s_last;
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_q + p.emb_dim);
+  const int q = blockIdx.y;
+  const int user = p.query_users ? p.query_users[q] : 0;
+  const bool user_ok = user >= 0 && user < p.n_users;
+  const int n = user_ok ? min(p.user_count[user], keys_capacity) : 0;
+  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+  if (row0 < n) {
+    const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * p.emb_dim;
+    for (int d = threadIdx.x; d < p.emb_dim; d += kScoreThreads) s_q[d] = (float)qv[d];
+    __syncthreads();
+    score_rows<T>(p, s_q, q, user, n, row0, rows_per_cta);
   }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();  // this CTA's scores are visible before its ticket is
+    const uint32_t t = atomicAdd(&tickets[q], 1u);
+    s_last = t == gridDim.x - 1;
+    if (s_last) tickets[q] = 0;  // ready for the next call (calls on one store are ordered on the device)
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float* sc = p.scores + (int64_t)q * p.score_stride;
+  for (int i = threadIdx.x; i < n; i += kScoreThreads) s_keys[i] = order_key(__ldcg(sc + i));
+  __syncthreads();
+  topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity,
+                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
 }
 
 }  // namespace ms

@@ -22,6 +22,8 @@ REQ_BAD_FACT_ID, REQ_NOT_RESIDENT, REQ_BLOCK_TABLE_SHORT, REQ_BAD_BLOCK_ID, REQ_
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
 ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
 INJECT_REVERSE = 1
+STORE_TMA_COPY_PATH = 1
+REQ_KERNEL_TIMEOUT = 32
 
 
 class MemStoreError(RuntimeError):
@@ -35,7 +37,7 @@ class _Config(C.Structure):
         ("device", C.c_int32), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("kv_dtype", C.c_int32), ("emb_dim", C.c_int32), ("emb_dtype", C.c_int32), ("rope_style", C.c_int32),
         ("rope_theta", C.c_double), ("inv_freq_override", C.POINTER(C.c_float)), ("max_position", C.c_int64),
-        ("n_users", C.c_int32), ("reserved0", C.c_int32), ("max_facts_per_user", C.c_int64),
+        ("n_users", C.c_int32), ("flags", C.c_uint32), ("max_facts_per_user", C.c_int64),
         ("max_kv_tokens", C.c_int64), ("kv_arena", C.c_void_p), ("kv_arena_bytes", C.c_size_t),
     ]  # fmt: skip
 
@@ -172,7 +174,7 @@ class MemStore:
 
     def __init__(self, *, device=0, n_layers, n_kv_heads, head_dim, emb_dim, emb_dtype=torch.float16, rope_theta=1.0e4,
                  rope_style=ROPE_HALF_SPLIT, inv_freq_override=None, max_position=1 << 24, n_users=1,
-                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None):  # fmt: skip
+                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None, flags=0):  # fmt: skip
         self._lib = load_library()
         self._h = C.c_void_p()
         self.device = torch.device("cuda", device if isinstance(device, int) else torch.device(device).index or 0)
@@ -188,7 +190,7 @@ class MemStore:
                 raise ValueError("inv_freq_override needs head_dim/2 entries")
         self._arena = kv_arena
         cfg = _Config(self.device.index, n_layers, n_kv_heads, head_dim, DTYPE_BF16, emb_dim, emb_code, rope_style,
-                      float(rope_theta), ov, max_position, n_users, 0, max_facts_per_user, max_kv_tokens,
+                      float(rope_theta), ov, max_position, n_users, flags, max_facts_per_user, max_kv_tokens,
                       kv_arena.data_ptr() if kv_arena is not None else None,
                       kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0)  # fmt: skip
         self.n_layers, self.n_kv_heads, self.head_dim, self.emb_dim = n_layers, n_kv_heads, head_dim, emb_dim

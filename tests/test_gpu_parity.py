@@ -97,12 +97,16 @@ def test_retrieve_empty_store_and_per_user_segments():
 
 
 # ------------------------------------------------------------------------------------------------ injection
-@pytest.mark.parametrize("start,bs", [(0, 16), (13, 16), (16, 16), (4096, 32), (100, 8), (1000003, 16)])
-def test_inject_positions_and_block_sizes(start, bs):
+PATHS = [0, 1]  # 0: direct copy kernel (default), 1: MS_STORE_TMA_COPY_PATH (bulk-async staged kernel)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("start,bs", [(0, 16), (13, 16), (16, 16), (4096, 32), (100, 8), (1000003, 16), (3, 4)])
+def test_inject_positions_and_block_sizes(start, bs, path):
     # lengths 1 and 128 included; facts straddle up to 9 blocks; several layers and tiles, ragged tail
     lens = [1, 128, 17, 33, 5, 64, 16, 31]
     hs = HostStore(5, len(lens), 3, 8, 128, 0, 0, 64, "float16", lens=lens)
-    ms = hs.to_memstore(5e5)
+    ms = hs.to_memstore(5e5, flags=path)
     ids = [1, 0, 3, -1, 2, 2, 7, 5]
     m = sum(lens[i] for i in ids if i >= 0)
     n_table = (start + m + bs - 1) // bs
@@ -123,21 +127,23 @@ def test_inject_positions_and_block_sizes(start, bs):
         assert np.array_equal(kb[:, 0], hs.k[:, hs.offs[1]])
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("layout,stacked", [("NHD", False), ("NHD", True), ("HND", False), ("HND", True)])
-def test_inject_cache_layouts(layout, stacked):
+def test_inject_cache_layouts(layout, stacked, path):
     hs = HostStore(7, 10, 2, 4, 64, 3, 40, 64, "float16")
-    ms = hs.to_memstore(1e4)
+    ms = hs.to_memstore(1e4, flags=path)
     table = synth.block_tables(8, 20, 14, 1)[0]
     cache = make_cache(hs, 20, 16, layout=layout, stacked=stacked)
     out = run_inject_and_check(ms, hs, [9, 4, 0, 6], 21, table, cache, 1e4)
     assert out["exact_frac"] > 0.995
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("style", [0, 1])
-@pytest.mark.parametrize("H,D", [(2, 64), (8, 128), (1, 256), (4, 32), (3, 16), (32, 128)])
-def test_inject_head_shapes_and_rope_styles(style, H, D):
+@pytest.mark.parametrize("H,D", [(2, 64), (8, 128), (1, 256), (4, 32), (3, 16), (32, 128), (40, 256)])
+def test_inject_head_shapes_and_rope_styles(style, H, D, path):
     hs = HostStore(9, 6, 2, H, D, 2, 50, 64, "float16")
-    ms = hs.to_memstore(1e6, rope_style=style)
+    ms = hs.to_memstore(1e6, rope_style=style, flags=path)
     table = synth.block_tables(10, 24, 20, 1)[0]
     cache = make_cache(hs, 24, 16)
     out = run_inject_and_check(ms, hs, [5, 1, 3, 0], 37, table, cache, 1e6, style=style)
