@@ -174,6 +174,26 @@ def rope_rows(x: np.ndarray, pos: np.ndarray, theta: float, style: int = 0, inv_
     return y
 
 
+def slots(ids, fact_len, start_pos, block_table, bs, num_blocks):
+    """Positions and slots only (no K/V touched): returns (m, slots[m]) for facts ``ids`` in placement order."""
+    ids = np.ascontiguousarray(ids, dtype=np.int32).reshape(-1)
+    fact_len = np.ascontiguousarray(fact_len, dtype=np.int32)
+    fact_offset = np.zeros(fact_len.size, dtype=np.int64)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32).reshape(-1)
+    valid = ids[(ids >= 0) & (ids < fact_len.size)]
+    out = np.empty(int(fact_len[valid].sum()), dtype=np.int64)
+    dummy = np.zeros(1, dtype=np.uint16)
+    m = C.c_int64(0)
+    rc = lib().oracle_inject(
+        _ptr(ids), ids.size, fact_len.size, _ptr(fact_offset), _ptr(fact_len), _ptr(dummy), _ptr(dummy), 1 << 62,
+        1, 1, 2, 1.0, 0, None, int(start_pos), _ptr(block_table), block_table.size, bs, num_blocks, 0, 0,
+        C.byref(m), _ptr(out), None, None, None, None, None, 0, 0, 0, 0, 1,
+    )  # fmt: skip
+    if rc:
+        raise OracleError(rc)
+    return m.value, out
+
+
 class InjectResult:
     """m, slots [m], k_ref float64 / k_bf16 uint16 / v uint16, each [nl, m, H, D]."""
 

@@ -55,11 +55,13 @@ class Workload:
 
 
 def build(name: str, seed: int = 0, device="cuda", n_query_pool: int | None = None, num_blocks: int | None = None,
-          resident_ids=None, scale_facts: float = 1.0, add_batch_tokens: int = 4096, want_cache: bool = True) -> Workload:  # fmt: skip
+          resident_ids=None, hot_per_user: int | None = None, scale_facts: float = 1.0, add_batch_tokens: int = 4096,
+          want_cache: bool = True) -> Workload:  # fmt: skip
     """Create the store of configuration ``name`` and fill it.
 
     ``resident_ids``: for configurations with a hot subset, the global fact ids that must have K/V (the
-    harness passes the ids its requests will inject); random filler ids complete the subset.
+    harness passes the ids its requests will inject); random filler ids complete the subset up to
+    ``hot_per_user`` facts per user (default: the configuration's figure).
     ``scale_facts`` < 1 shrinks the number of facts per user (tests on smaller boxes)."""
     s = synth.CONFIGS[name]
     dev = torch.device(device)
@@ -71,7 +73,7 @@ def build(name: str, seed: int = 0, device="cuda", n_query_pool: int | None = No
         if resident_ids is not None:
             hot[np.asarray(sorted({int(i) for i in resident_ids if i >= 0}), np.int64)] = True
         rng = np.random.default_rng([seed, 6])
-        per_user_hot = max(1, int(round(s.resident_per_user * scale_facts)))
+        per_user_hot = hot_per_user if hot_per_user is not None else max(1, int(round(s.resident_per_user * scale_facts)))
         for u in range(s.n_users):
             seg = np.arange(u * n_per_user, (u + 1) * n_per_user)
             missing = per_user_hot - int(hot[seg].sum())
