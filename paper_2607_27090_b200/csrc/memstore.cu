@@ -49,7 +49,6 @@ struct memstore {
   int64_t max_user_count = 0;
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
   int copy_ctas_per_sm = 1;
-  size_t fused_smem_set = 0;
   bool tma_path = false;  // MS_STORE_TMA_COPY_PATH
   std::mutex mu;
   std::string err;
@@ -118,6 +117,20 @@ __global__ void __launch_bounds__(256) arena_append_kernel(const uint4* __restri
   uint4* d = (blockIdx.z ? v_dst : k_dst) + (int64_t)layer * vec_per_layer_dst + dst_vec_off;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vec_per_layer_src; i += (int64_t)gridDim.x * blockDim.x)
     d[i] = s[i];
+}
+
+// The dynamic shared memory limit of a kernel is a per-device property of the function, shared by all stores:
+// it is only ever raised.
+cudaError_t ensure_fused_smem(int device, size_t bytes) {
+  static std::mutex mu;
+  static size_t set_bytes[64] = {0};
+  std::lock_guard<std::mutex> lock(mu);
+  const int d = device & 63;
+  if (bytes <= set_bytes[d]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(score_topk_fused_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) set_bytes[d] = bytes;
+  return e;
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -368,11 +381,7 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
     // small segments: scoring and top-k in one launch
     const int keys_cap = (int)std::max<int64_t>(n_max, 1);
     const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)keys_cap * sizeof(uint32_t);
-    if (smem > s->fused_smem_set) {
-      MS_CUDA(s, cudaFuncSetAttribute(score_topk_fused_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      MS_CUDA(s, cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      s->fused_smem_set = smem;
-    }
+    MS_CUDA(s, ensure_fused_smem(c.device, smem));
     if (c.emb_dtype == MS_DTYPE_F16)
       score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap);
     else
