@@ -136,6 +136,30 @@ ms_status memstore_add_facts(memstore_t* store, int32_t user, int64_t n, const v
 ms_status memstore_retrieve(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                             int32_t* out_ids, float* out_scores, ms_stream stream);
 
+/*
+ * memstore_retrieve without any allocation (the paper has no counterpart: this exists for callers, not for the
+ * method).  Some callers cannot let a library allocate device memory while they serve requests: an inference
+ * engine that has already claimed almost all of HBM for its KV cache leaves nothing for a later cudaMalloc to
+ * succeed with, and a latency-critical loop cannot afford the device-wide synchronisation a cudaMalloc or
+ * cudaFree may cause.  memstore_retrieve grows its score scratch with cudaMalloc the first time it sees a batch
+ * size; this entry point never allocates or frees anything.  Same arguments, same results as memstore_retrieve.
+ *
+ * Its scratch is a fixed array inside the library: MEMSTORE_STATIC_SCRATCH_BYTES (4 MiB + 4 KiB) of device
+ * memory that every GPU holds from the moment it loads the library until the process exits.  Limits, checked
+ * before anything is enqueued (MS_ERR_CAPACITY with a message otherwise):
+ *     nq <= MEMSTORE_STATIC_MAX_QUERIES  and  nq * max_facts_per_user <= MEMSTORE_STATIC_MAX_SCORES.
+ * The first call on a device looks up the array's device address (no allocation, but a set-up step): make that
+ * first call before any stream capture begins on that device.
+ * The array is shared by EVERY call of this entry point on the device, whichever store or stream: two such calls
+ * whose kernels could overlap on the GPU race on it, so the caller must order them (one stream, or events).  It
+ * keeps the previous call's contents; the part that must start at zero is cleared on the stream by each call.
+ */
+#define MEMSTORE_STATIC_MAX_QUERIES 1024
+#define MEMSTORE_STATIC_MAX_SCORES (1 << 20)
+#define MEMSTORE_STATIC_SCRATCH_BYTES (MEMSTORE_STATIC_MAX_SCORES * 4 + MEMSTORE_STATIC_MAX_QUERIES * 4)
+ms_status memstore_retrieve_static(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq,
+                                   int32_t k, int32_t* out_ids, float* out_scores, ms_stream stream);
+
 /* A caller-owned paged KV cache, bf16, described by strides in ELEMENTS:
  *   element (layer, block, token-in-block, head, d) of K is at
  *   k_base[layer*layer_stride + block*block_stride + token*token_stride + head*head_stride + d]

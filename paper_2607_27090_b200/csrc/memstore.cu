@@ -403,6 +403,101 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   return mark_last(s, st);
 }
 
+// ---- memstore_retrieve_static: the allocation-free variant of retrieve ---------------------------------------
+// Scratch of the variant: fp32 scores first, then one ticket per query.  A file-scope device array: every GPU
+// that loads this library carries it until the process ends.  In HOST code the name below is only a stand-in for
+// the symbol, not a device address; the address each device gives it comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_retrieve_static_scratch[MEMSTORE_STATIC_SCRATCH_BYTES];
+
+namespace {
+// Device address of g_retrieve_static_scratch on `device` (which must be current), looked up once per device.
+cudaError_t static_scratch_address(int device, unsigned char** out) {
+  static std::mutex mu;
+  static unsigned char* addr[64] = {nullptr};
+  if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[device]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_retrieve_static_scratch);
+    if (e != cudaSuccess) return e;
+    addr[device] = static_cast<unsigned char*>(p);
+  }
+  *out = addr[device];
+  return cudaSuccess;
+}
+}  // namespace
+
+ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                                   int32_t* out_ids, float* out_scores, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (nq < 0 || k < 1 || k > kTopkMaxK) return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d (1 <= k <= %d)", nq, k, kTopkMaxK);
+  if (nq == 0) return MS_OK;
+  if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
+  if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
+  if (nq > MEMSTORE_STATIC_MAX_QUERIES || (int64_t)nq * c.max_facts_per_user > MEMSTORE_STATIC_MAX_SCORES)
+    return fail(s, MS_ERR_CAPACITY,
+                "static scratch holds %d queries and %d scores: nq=%d x max_facts_per_user=%lld does not fit "
+                "(use memstore_retrieve)",
+                MEMSTORE_STATIC_MAX_QUERIES, MEMSTORE_STATIC_MAX_SCORES, nq, (long long)c.max_facts_per_user);
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned char* scratch = nullptr;
+  MS_CUDA(s, static_scratch_address(c.device, &scratch));
+  float* scores = reinterpret_cast<float*>(scratch);
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(scratch + (size_t)MEMSTORE_STATIC_MAX_SCORES * sizeof(float));
+  ms_status rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+  // the tickets must start at zero whatever an earlier call (of any store) left behind
+  MS_CUDA(s, cudaMemsetAsync(tickets, 0, (size_t)nq * sizeof(uint32_t), st));
+
+  RetrieveParams p{};
+  p.emb = s->emb;
+  p.emb_fact_id = s->emb_fact_id;
+  p.user_count = s->user_count_d;
+  p.seg_capacity = c.max_facts_per_user;
+  p.n_users = c.n_users;
+  p.emb_dim = c.emb_dim;
+  p.queries = queries;
+  p.query_users = query_users;
+  p.nq = nq;
+  p.k = k;
+  p.scores = scores;
+  p.score_stride = c.max_facts_per_user;
+  p.out_ids = out_ids;
+  p.out_scores = out_scores;
+
+  const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
+  int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
+  rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
+  dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+  if (n_max <= kFusedMaxRows) {
+    const int keys_cap = (int)std::max<int64_t>(n_max, 1);
+    const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)keys_cap * sizeof(uint32_t);
+    MS_CUDA(s, ensure_fused_smem(c.device, smem));  // a function attribute, not an allocation
+    if (c.emb_dtype == MS_DTYPE_F16)
+      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap);
+    else
+      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched++;
+  } else {
+    const size_t smem = (size_t)c.emb_dim * sizeof(float);
+    if (c.emb_dtype == MS_DTYPE_F16)
+      score_rows_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
+    else
+      score_rows_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta);
+    MS_CUDA(s, cudaGetLastError());
+    topk_kernel<<<nq, kTopkThreads, 0, st>>>(p);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched += 2;
+  }
+  s->retrieve_calls++;
+  return mark_last(s, st);
+}
+
 ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
                           const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,

@@ -60,7 +60,7 @@ class _Stats(C.Structure):
 EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
-    "memstore_set_profile_events",
+    "memstore_set_profile_events", "memstore_retrieve_static",
 )  # fmt: skip
 
 _lib = None
@@ -92,6 +92,8 @@ def load_library() -> C.CDLL:
     L.memstore_add_facts.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
     L.memstore_retrieve.restype = i32
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    L.memstore_retrieve_static.restype = i32
+    L.memstore_retrieve_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.memstore_inject.restype = i32
     L.memstore_inject.argtypes = [vp, vp, i32, i32, vp, vp, i32, C.POINTER(_PagedCache), vp, vp, vp, i64, u32, vp]
     L.memstore_stats.restype = i32
@@ -252,6 +254,25 @@ class MemStore:
                                          _dev_ptr(query_users, torch.int32, "query_users"), nq, k,
                                          _dev_ptr(out_ids, torch.int32, "out_ids"),
                                          _dev_ptr(out_scores, torch.float32, "out_scores"), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out_ids, out_scores
+
+    def retrieve_static(self, queries, k, query_users=None, out_ids=None, out_scores=None, want_scores=True, stream=None):
+        """``retrieve`` through the entry point that never allocates device memory, for callers that cannot let the
+        library call cudaMalloc while serving (an engine that has claimed nearly all of HBM, a loop that cannot
+        take the device-wide stall of an allocation).  Scratch is a fixed 4 MiB array inside the library shared by
+        all such calls on the device, so the caller must not let two of them overlap on the GPU; sizes beyond
+        1024 queries or 2^20 scores are refused.  Pass ``out_ids`` / ``out_scores`` to keep torch from allocating
+        too."""
+        nq = queries.shape[0]
+        if out_ids is None:
+            out_ids = torch.empty((nq, k), dtype=torch.int32, device=queries.device)
+        if out_scores is None and want_scores:
+            out_scores = torch.empty((nq, k), dtype=torch.float32, device=queries.device)
+        rc = self._lib.memstore_retrieve_static(self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"),
+                                                _dev_ptr(query_users, torch.int32, "query_users"), nq, k,
+                                                _dev_ptr(out_ids, torch.int32, "out_ids"),
+                                                _dev_ptr(out_scores, torch.float32, "out_scores"), _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out_ids, out_scores
 
