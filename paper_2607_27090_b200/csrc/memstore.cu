@@ -380,12 +380,13 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   if (n_max <= kFusedMaxRows) {
     // small segments: scoring and top-k in one launch
     const int keys_cap = (int)std::max<int64_t>(n_max, 1);
-    const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)keys_cap * sizeof(uint32_t);
+    const size_t smem = (size_t)keys_cap * sizeof(uint32_t);
+    const int n_host = query_users ? -1 : (int)n_max;
     MS_CUDA(s, ensure_fused_smem(c.device, smem));
     if (c.emb_dtype == MS_DTYPE_F16)
-      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap);
+      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host);
     else
-      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap);
+      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host);
     MS_CUDA(s, cudaGetLastError());
     s->kernels_launched++;
   } else {
@@ -475,12 +476,13 @@ ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int
   dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
   if (n_max <= kFusedMaxRows) {
     const int keys_cap = (int)std::max<int64_t>(n_max, 1);
-    const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)keys_cap * sizeof(uint32_t);
+    const size_t smem = (size_t)keys_cap * sizeof(uint32_t);
+    const int n_host = query_users ? -1 : (int)n_max;
     MS_CUDA(s, ensure_fused_smem(c.device, smem));  // a function attribute, not an allocation
     if (c.emb_dtype == MS_DTYPE_F16)
-      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap);
+      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap, n_host);
     else
-      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap);
+      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap, n_host);
     MS_CUDA(s, cudaGetLastError());
     s->kernels_launched++;
   } else {

@@ -95,6 +95,56 @@ __device__ __forceinline__ void score_rows(const RetrieveParams& p, const float*
   }
 }
 
+// The same scoring with the query read straight from global memory (through L1) next to the row, so that one
+// memory round trip serves both and no shared-memory staging or barrier is needed.  Same lane layout and
+// summation order as score_rows.
+template <typename T>
+__device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q, int user, int n, int64_t row0, int rows_per_cta) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int E = p.emb_dim;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const T* seg = reinterpret_cast<const T*>(p.emb) + (int64_t)user * p.seg_capacity * E;
+  const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
+  const int64_t row_end = min(row0 + rows_per_cta, (int64_t)n);
+  const int nvec = E / VEC;
+  for (int64_t row = row0 + warp; row < row_end; row += kScoreWarps) {
+    const uint4* rp = reinterpret_cast<const uint4*>(seg + row * E);
+    float acc = 0.f;
+    for (int v0 = 0; v0 < nvec; v0 += 128) {
+      uint4 x[4], y[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + u * 32 + lane;
+        if (v < nvec) {
+          x[u] = __ldg(rp + v);
+          y[u] = __ldg(qp + v);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + u * 32 + lane;
+        if (v < nvec) {
+          if (sizeof(T) == 2) {
+            float f[8], g[8];
+            unpack8(x[u], f);
+            unpack8(y[u], g);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc = fmaf(f[i], g[i], acc);
+          } else {
+            const float* f = reinterpret_cast<const float*>(&x[u]);
+            const float* g = reinterpret_cast<const float*>(&y[u]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc = fmaf(f[i], g[i], acc);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) p.scores[(int64_t)q * p.score_stride + row] = acc + 0.0f;  // -0 -> +0
+  }
+}
+
 // Bitonic network over P (a power of two) 64-bit keys in shared memory, largest first.
 template <int THREADS>
 __device__ __forceinline__ void bitonic_sort_desc(unsigned long long* cand, int P) {
@@ -152,7 +202,8 @@ struct TopkShared {
 // ------------------------------------------------------------------------------------------------
 template <int THREADS>
 __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const int32_t* row_ids,
-                           int32_t* out_ids, float* out_scores) {
+                           int32_t* out_ids, float* out_scores, bool have_minmax = false, uint32_t my_lo = 0xffffffffu,
+                           uint32_t my_hi = 0u) {
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int take = min(n, k);
@@ -165,11 +216,13 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   // orders them exactly, ties by row.  If the candidates do not fit (massive ties) the radix path runs instead.
   bool fast = false;
   if (n > k) {
-    uint32_t lo = 0xffffffffu, hi = 0u;
-    for (int i = tid; i < n; i += THREADS) {
-      const uint32_t kx = key_at(i);
-      lo = min(lo, kx);
-      hi = max(hi, kx);
+    uint32_t lo = my_lo, hi = my_hi;
+    if (!have_minmax) {
+      for (int i = tid; i < n; i += THREADS) {
+        const uint32_t kx = key_at(i);
+        lo = min(lo, kx);
+        hi = max(hi, kx);
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -241,6 +294,19 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
         }
       }
       __syncthreads();
+      if (n_cand <= (uint32_t)THREADS) {
+        // few candidates: the rank of a candidate is the number of larger ones (keys are distinct); no sorting network
+        if (tid < (int)n_cand) {
+          const unsigned long long mine = sm.cand[tid];
+          uint32_t rank = 0;
+          for (uint32_t jj = 0; jj < n_cand; ++jj) rank += sm.cand[jj] > mine;
+          if (rank < (uint32_t)k) {
+            out_ids[rank] = row_ids[0xffffffffu - (uint32_t)(mine & 0xffffffffull)];
+            if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+          }
+        }
+        return;
+      }
       bitonic_sort_desc<THREADS>(sm.cand, P2);
       write_topk<THREADS>(sm.cand, take, k, row_ids, out_ids, out_scores);
       return;
@@ -380,25 +446,24 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams
 
 // Scoring + top-k in ONE launch for segments of at most kFusedMaxRows rows: grid = (row groups, nq).
 // The CTA that finishes a query's scores last (a wait-free ticket) selects and sorts that query's top-k from
-// keys held in shared memory.  Dynamic shared memory: emb_dim floats (query) + keys_capacity uint32 keys.
+// keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
+// of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
-                                                                         uint32_t* tickets, int keys_capacity) {
-  extern __shared__ float s_q[];
+                                                                         uint32_t* tickets, int keys_capacity, int n_host) {
+  extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ int s_last;
-  uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_q + p.emb_dim);
   const int q = blockIdx.y;
-  const int user = p.query_users ? p.query_users[q] : 0;
-  const bool user_ok = user >= 0 && user < p.n_users;
-  const int n = user_ok ? min(p.user_count[user], keys_capacity) : 0;
-  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
-  if (row0 < n) {
-    const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * p.emb_dim;
-    for (int d = threadIdx.x; d < p.emb_dim; d += kScoreThreads) s_q[d] = (float)qv[d];
-    __syncthreads();
-    score_rows<T>(p, s_q, q, user, n, row0, rows_per_cta);
+  int user = 0, n = n_host;
+  bool user_ok = true;
+  if (n_host < 0) {
+    user = p.query_users ? p.query_users[q] : 0;
+    user_ok = user >= 0 && user < p.n_users;
+    n = user_ok ? min(p.user_count[user], keys_capacity) : 0;
   }
+  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+  if (row0 < n) score_rows_direct<T>(p, q, user, n, row0, rows_per_cta);
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();  // this CTA's scores are visible before its ticket is
@@ -410,10 +475,17 @@ __global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const R
   if (!s_last) return;
   __threadfence();
   const float* sc = p.scores + (int64_t)q * p.score_stride;
-  for (int i = threadIdx.x; i < n; i += kScoreThreads) s_keys[i] = order_key(__ldcg(sc + i));
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for (int i = threadIdx.x; i < n; i += kScoreThreads) {
+    const uint32_t kx = order_key(__ldcg(sc + i));
+    s_keys[i] = kx;
+    lo = min(lo, kx);
+    hi = max(hi, kx);
+  }
   __syncthreads();
   topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity,
-                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
+                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
+                            hi);
 }
 
 }  // namespace ms
