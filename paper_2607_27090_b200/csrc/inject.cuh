@@ -228,10 +228,10 @@ constexpr int kUnitsPerThread = 2;
 constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a token row served by one CTA
 
 // ------------------------------------------------------------------------------------------------
-// Copy kernel (I4 + I5): ONE CTA per work item = (tile of 8 tokens, layer, row part), no loop, no shared memory.
-// The grid is an upper bound computed on the host (the real tile count is only known on the device); CTAs beyond
-// it return at once.  The hardware CTA scheduler keeps every SM full and balances SMs that get unequal memory
-// service, and with ~1000 resident threads per SM each holding eight 16-byte loads, about 128 KB per SM are in
+// Copy kernel (I4 + I5): ONE CTA per work item = (tile of 8 tokens, layer, row part), no shared memory.
+// The grid is the host's estimate of the item count (the real tile count is only known on the device); CTAs
+// beyond the real count return at once and a low estimate makes some CTAs take a second item.  The hardware CTA scheduler keeps every SM full and balances SMs that get unequal memory
+// service, and with 768 resident threads per SM each holding eight 16-byte loads, about 96 KB per SM are in
 // flight: measured on B200 this plain structure sustains the copy rate of the device, and a persistent
 // shared-memory ring fed by bulk copies does not (see inject_tma.cuh).
 //
@@ -240,7 +240,7 @@ constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a
 // both units of a thread share the frequency octet: its 8 cos/sin pairs are computed once, while the loads fly.
 // ------------------------------------------------------------------------------------------------
 template <int STYLE>
-__global__ void __launch_bounds__(kCopyThreads, 4) inject_copy_kernel(const InjectParams p) {
+__global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const InjectParams p) {
   const int tid = threadIdx.x;
   const int tk = tid >> 5;  // token of the tile
   const int l = tid & 31;
@@ -257,51 +257,53 @@ __global__ void __launch_bounds__(kCopyThreads, 4) inject_copy_kernel(const Inje
   grid_dependency_wait();  // tile descriptors come from the plan kernel
 
   const uint32_t n_tiles = min(p.ctrl->n_tiles, p.tiles_capacity);
-  // items in (layer, tile) order: CTAs that run together stream neighbouring rows of one layer
-  if (n_tiles == 0) return;
-  const uint32_t item = blockIdx.x;
-  const uint32_t layer = item / n_tiles;
-  if (layer >= (uint32_t)p.n_layers) return;
-  const uint32_t tile = item - layer * n_tiles;
-  const TileDesc* d = p.tiles + tile;
-  const int32_t src = d->src_tok[tk];
-  if (src < 0) return;
-  const int64_t dst = d->dst_off[tk];
-  const int32_t pos = d->pos0 + tk;
+  const uint32_t n_items = n_tiles * (uint32_t)p.n_layers;
+  // items in (layer, tile) order: CTAs that run together stream neighbouring rows of one layer.  The grid is the
+  // host's ESTIMATE of the item count: CTAs beyond the real count leave at once, and if the estimate was low the
+  // first CTAs take a second item.
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t layer = item / n_tiles;
+    const uint32_t tile = item - layer * n_tiles;
+    const TileDesc* d = p.tiles + tile;
+    const int32_t src = d->src_tok[tk];
+    if (src < 0) continue;
+    const int64_t dst = d->dst_off[tk];
+    const int32_t pos = d->pos0 + tk;
 
-  const int64_t src_row = ((int64_t)layer * p.arena_tokens + src) * (int64_t)(p.n_heads * D);
-  const __nv_bfloat16* ks = p.k_arena + src_row;
-  const __nv_bfloat16* vs = p.v_arena + src_row;
-  const int64_t dbase = (int64_t)layer * p.layer_stride + dst;
-  uint4 ka[kUnitsPerThread], kb[kUnitsPerThread], va[kUnitsPerThread], vb[kUnitsPerThread];
+    const int64_t src_row = ((int64_t)layer * p.arena_tokens + src) * (int64_t)(p.n_heads * D);
+    const __nv_bfloat16* ks = p.k_arena + src_row;
+    const __nv_bfloat16* vs = p.v_arena + src_row;
+    const int64_t dbase = (int64_t)layer * p.layer_stride + dst;
+    uint4 ka[kUnitsPerThread], kb[kUnitsPerThread], va[kUnitsPerThread], vb[kUnitsPerThread];
 #pragma unroll
-  for (int u = 0; u < kUnitsPerThread; ++u) {
-    const int unit = u0 + u * kThreadsPerToken;
-    if (unit < n_units) {
-      const int h = unit >> g_shift;
-      ka[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offA));
-      kb[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offB));
-      va[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offA));
-      vb[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offB));
+    for (int u = 0; u < kUnitsPerThread; ++u) {
+      const int unit = u0 + u * kThreadsPerToken;
+      if (unit < n_units) {
+        const int h = unit >> g_shift;
+        ka[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offA));
+        kb[u] = ld_stream(reinterpret_cast<const uint4*>(ks + h * D + offB));
+        va[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offA));
+        vb[u] = ld_stream(reinterpret_cast<const uint4*>(vs + h * D + offB));
+      }
     }
-  }
-  // cos/sin of (pos, 8 frequencies), evaluated while the loads are in flight
-  float sn[8], cs[8];
-  const float posf = (float)pos;
+    // cos/sin of (pos, 8 frequencies), evaluated while the loads are in flight
+    float sn[8], cs[8];
+    const float posf = (float)pos;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
+    for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
 #pragma unroll
-  for (int u = 0; u < kUnitsPerThread; ++u) {
-    const int unit = u0 + u * kThreadsPerToken;
-    if (unit < n_units) {
-      const int h = unit >> g_shift;
-      rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
-      __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
-      st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
-      st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
-      __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
-      st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
-      st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
+    for (int u = 0; u < kUnitsPerThread; ++u) {
+      const int unit = u0 + u * kThreadsPerToken;
+      if (unit < n_units) {
+        const int h = unit >> g_shift;
+        rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+        __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
+        st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
+        st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
+        __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
+        st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
+        st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
+      }
     }
   }
 }

@@ -613,9 +613,14 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     else
       e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<1>, p, ts, v_rows);
   } else {
-    // direct kernel: one CTA per (tile, layer, row part); the grid covers the largest request the ids could name
+    // direct kernel: one CTA per (tile, layer, row part).  The ids are on the device, so the host sizes the grid
+    // from the mean length of the resident facts (plus a ragged tile per request and 3 %); the kernel's
+    // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
     const int units = c.n_kv_heads * (c.head_dim / 16);
-    const int64_t items = tiles_needed * c.n_layers;
+    const double mean_len = s->n_resident > 0 ? (double)s->kv_tokens_used / (double)s->n_resident : 0.0;
+    int64_t est_tiles_grid = (int64_t)(((double)k * mean_len / kTileTokens + 2.0) * nreq * 1.03) + 1;
+    est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
+    const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
     if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
     lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
     lc.blockDim = dim3(kCopyThreads);
