@@ -407,8 +407,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per launch of the copy kernel from an ncu capture; see profiles/.  None until measured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {}
+# DRAM bytes (read + write) per launch of the copy kernel from the ncu capture summarised in
+# profiles/inject_copy_kernel_llama8b_k50.md (mean of the two captured launches; the capture starts from a flushed L2, so
+# about 50 MB of the written bytes are still in L2 when the kernel ends and are not in this figure).
+NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {("llama8b", 50): 468.2e6}
 
 
 if __name__ == "__main__":
