@@ -132,6 +132,10 @@ ms_status memstore_add_facts(memstore_t* store, int32_t user, int64_t n, const v
  *                padded with -1 when the user has fewer than k facts
  *   out_scores   device fp32 [nq][k] or NULL (0 where the id is -1)
  * Products of the stored values are accumulated in fp32.  1 <= k <= 2048.
+ * Kernel choice: segments of at most 8192 rows are scored and selected in one launch; larger segments use a
+ * scoring launch and a selection launch; with 8 or more fp16 queries (emb_dim a multiple of 64, at most 1024,
+ * k <= 256, no per-query users) on a large segment the scoring runs on the tensor cores (tcgen05) as a filter
+ * that is followed by an exact fp32 rescoring of the surviving rows, so results do not depend on the path.
  */
 ms_status memstore_retrieve(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                             int32_t* out_ids, float* out_scores, ms_stream stream);
@@ -197,12 +201,14 @@ ms_status memstore_inject(memstore_t* store, const int32_t* fact_ids, int32_t nr
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
                           uint32_t flags, ms_stream stream);
 
-/* Counters since creation (host side; bytes are the algorithmic ones, not measured traffic). */
+/* Counters since creation (host side; bytes are the algorithmic ones, not measured traffic).  Reading
+ * kernel_timeouts synchronises the device. */
 typedef struct {
   int64_t n_facts, n_resident_facts, kv_tokens_used;
   int64_t retrieve_calls, inject_calls;
   int64_t kernels_launched; /* kernels of this library enqueued so far */
   int64_t arena_bytes, embedding_bytes;
+  int64_t kernel_timeouts; /* 1 if a bounded wait inside the tensor-core scoring kernel ever ran out (results of that call are invalid) */
 } memstore_stats_t;
 ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
 

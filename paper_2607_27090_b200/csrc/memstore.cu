@@ -16,6 +16,7 @@
 #include "inject.cuh"
 #include "inject_tma.cuh"
 #include "retrieve.cuh"
+#include "score_gemm.cuh"
 
 using namespace ms;
 
@@ -34,6 +35,15 @@ struct memstore {
   // scratch shared by all calls (ordered on the device through `last_done`)
   float* scores = nullptr;
   uint32_t* tickets = nullptr;  // one wait-free counter per query of the fused retrieve kernel
+  // tensor-core retrieve path (allocated on first use): group maxima, selected groups, candidate scores / rows
+  float* tc_gmax = nullptr;
+  int64_t tc_gmax_stride = 0;
+  int32_t* tc_sel = nullptr;
+  float* tc_cand_scores = nullptr;
+  int32_t* tc_cand_rows = nullptr;
+  uint32_t* tc_tickets = nullptr;
+  int* tc_error = nullptr;
+  bool tc_ready = false;
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
   uint32_t tiles_capacity = 0;
@@ -131,6 +141,78 @@ cudaError_t ensure_fused_smem(int device, size_t bytes) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) set_bytes[d] = bytes;
   return e;
+}
+
+// ---- tensor-core retrieve path -------------------------------------------------------------------------------
+constexpr int kTcMinQueries = 8;     // below this the CUDA-core kernels re-reading the segment per query are cheaper
+constexpr int kTcMaxK = 256;
+constexpr int kTcGroupMargin = 28;   // groups selected beyond k: slack for tensor-core vs CUDA-core rounding at the k-th score
+constexpr int kTcMaxK2 = kTcMaxK + kTcGroupMargin;
+
+bool tc_path_applies(const memstore* s, const int32_t* query_users, int nq, int k, int64_t n_max) {
+  const memstore_config& c = s->cfg;
+  return c.emb_dtype == MS_DTYPE_F16 && c.emb_dim % kGemmKChunk == 0 && c.emb_dim <= kGemmMaxE && !query_users &&
+         nq >= kTcMinQueries && k <= kTcMaxK && n_max > kFusedMaxRows;
+}
+
+ms_status tc_prepare(memstore* s) {
+  if (s->tc_ready) return MS_OK;
+  const memstore_config& c = s->cfg;
+  const int64_t tiles = (c.max_facts_per_user + kGemmTileRows - 1) / kGemmTileRows;
+  s->tc_gmax_stride = tiles * kGemmGroupsPerTile;
+  MS_CUDA(s, cudaDeviceSynchronize());
+  MS_CUDA(s, cudaMalloc(&s->tc_gmax, (size_t)kGemmMaxQ * s->tc_gmax_stride * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_sel, (size_t)kGemmMaxQ * kTcMaxK2 * sizeof(int32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_cand_scores, (size_t)kGemmMaxQ * kTcMaxK2 * 8 * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_cand_rows, (size_t)kGemmMaxQ * kTcMaxK2 * 8 * sizeof(int32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_tickets, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_error, sizeof(int)));
+  MS_CUDA(s, cudaMemset(s->tc_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tc_error, 0, sizeof(int)));
+  MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)gemm_smem_bytes(kGemmMaxE)));
+  const size_t rs = (size_t)kTcMaxK2 * 8 * sizeof(uint32_t);
+  MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
+  s->tc_ready = true;
+  return MS_OK;
+}
+
+// Many queries on the one segment of user 0: (1) tcgen05 GEMM that keeps only the maximum score of every group of 8
+// rows, (2) per query the k + margin best groups, (3) exact CUDA-core rescoring of their rows and top-k.
+ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t n_rows, cudaStream_t st) {
+  const memstore_config& c = s->cfg;
+  ms_status rc = tc_prepare(s);
+  if (rc != MS_OK) return rc;
+  const int n_groups = (int)((n_rows + kGemmGroupRows - 1) / kGemmGroupRows);
+  const int k2 = std::min(kTcMaxK2, base.k + kTcGroupMargin);
+  const int n_tiles = (int)((n_rows + kGemmTileRows - 1) / kGemmTileRows);
+  CUtensorMap tmap_emb;
+  if (!make_tmap_rows_f16(&tmap_emb, s->emb, (uint64_t)n_rows, (uint64_t)c.emb_dim, kGemmTileRows))
+    return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the embedding matrix");
+  const size_t esz = 2;
+  for (int q0 = 0; q0 < base.nq; q0 += kGemmMaxQ) {
+    const int nqb = std::min(kGemmMaxQ, base.nq - q0);
+    const char* qptr = (const char*)base.queries + (size_t)q0 * c.emb_dim * esz;
+    CUtensorMap tmap_q;
+    if (!make_tmap_rows_f16(&tmap_q, qptr, (uint64_t)nqb, (uint64_t)c.emb_dim, kGemmMaxQ))
+      return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the query batch");
+    GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error};
+    score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, gemm_smem_bytes(c.emb_dim), st>>>(tmap_emb, tmap_q, gp);
+    MS_CUDA(s, cudaGetLastError());
+    select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel);
+    MS_CUDA(s, cudaGetLastError());
+    RetrieveParams p = base;
+    p.queries = qptr;
+    p.nq = nqb;
+    p.out_ids = base.out_ids + (int64_t)q0 * base.k;
+    p.out_scores = base.out_scores ? base.out_scores + (int64_t)q0 * base.k : nullptr;
+    dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
+    rescore_topk_kernel<__half><<<grid, kScoreThreads, (size_t)k2 * 8 * sizeof(uint32_t), st>>>(
+        p, s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched += 3;
+  }
+  return MS_OK;
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -246,6 +328,12 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->ctrl);
     cudaFree(s->scores);
     cudaFree(s->tickets);
+    cudaFree(s->tc_gmax);
+    cudaFree(s->tc_sel);
+    cudaFree(s->tc_cand_scores);
+    cudaFree(s->tc_cand_rows);
+    cudaFree(s->tc_tickets);
+    cudaFree(s->tc_error);
     cudaFree(s->tiles);
     if (s->last_done) cudaEventDestroy(s->last_done);
     cudaGetLastError();
@@ -340,7 +428,8 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
-  if (nq > s->scores_nq) {  // grow the score scratch (first call, or a larger batch than ever before)
+  const bool tc = tc_path_applies(s, query_users, nq, k, query_users ? s->max_user_count : s->user_count[0]);
+  if (!tc && nq > s->scores_nq) {  // grow the score scratch (first call, or a larger batch than ever before)
     MS_CUDA(s, cudaDeviceSynchronize());
     cudaFree(s->scores);
     cudaFree(s->tickets);
@@ -372,6 +461,12 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   p.out_scores = out_scores;
 
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
+  if (tc) {
+    rc = retrieve_tensor_core(s, p, n_max, st);
+    if (rc != MS_OK) return rc;
+    s->retrieve_calls++;
+    return mark_last(s, st);
+  }
   // enough CTAs to fill the GPU, at least one row per warp
   const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
   int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
@@ -652,6 +747,13 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->kernels_launched = s->kernels_launched;
   out->arena_bytes = (int64_t)memstore_arena_bytes(&s->cfg);
   out->embedding_bytes = (int64_t)s->cfg.n_users * s->cfg.max_facts_per_user * s->cfg.emb_dim * (int64_t)emb_elem_size(s->cfg.emb_dtype);
+  out->kernel_timeouts = 0;
+  if (s->tc_error) {
+    DeviceGuard g(s->cfg.device);
+    int flag = 0;
+    MS_CUDA(s, cudaMemcpy(&flag, s->tc_error, sizeof(int), cudaMemcpyDeviceToHost));
+    out->kernel_timeouts = flag;
+  }
   return MS_OK;
 }
 

@@ -166,9 +166,20 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long* cand, int 
   }
 }
 
+// What a selected index stands for: the index itself, a row taken from an index->row map (candidate lists), and/or
+// the fact id of that row.  Both maps are optional.
+struct IdMap {
+  const int32_t* idx_to_row;  // or nullptr: the index is the row
+  const int32_t* row_ids;     // or nullptr: the row is the id
+  __device__ __forceinline__ int32_t operator()(uint32_t idx) const {
+    int32_t row = idx_to_row ? idx_to_row[idx] : (int32_t)idx;
+    return (row >= 0 && row_ids) ? row_ids[row] : row;
+  }
+};
+
 // Ranks 0..k-1: fact id and fp32 score of the sorted candidates, -1 / 0 beyond `take`.
 template <int THREADS>
-__device__ __forceinline__ void write_topk(const unsigned long long* cand, int take, int k, const int32_t* row_ids,
+__device__ __forceinline__ void write_topk(const unsigned long long* cand, int take, int k, const IdMap ids,
                                            int32_t* out_ids, float* out_scores) {
   for (int r = threadIdx.x; r < k; r += THREADS) {
     int32_t id = -1;
@@ -176,7 +187,7 @@ __device__ __forceinline__ void write_topk(const unsigned long long* cand, int t
     if (r < take) {
       const unsigned long long c = cand[r];
       const uint32_t row = 0xffffffffu - (uint32_t)(c & 0xffffffffull);
-      id = row_ids[row];
+      id = ids(row);
       s = key_score((uint32_t)(c >> 32));
     }
     out_ids[r] = id;
@@ -201,7 +212,7 @@ struct TopkShared {
 // without it they are recomputed from the scores in global memory on every pass.
 // ------------------------------------------------------------------------------------------------
 template <int THREADS>
-__device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const int32_t* row_ids,
+__device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const IdMap ids,
                            int32_t* out_ids, float* out_scores, bool have_minmax = false, uint32_t my_lo = 0xffffffffu,
                            uint32_t my_hi = 0u) {
   const int tid = threadIdx.x;
@@ -301,14 +312,14 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
           uint32_t rank = 0;
           for (uint32_t jj = 0; jj < n_cand; ++jj) rank += sm.cand[jj] > mine;
           if (rank < (uint32_t)k) {
-            out_ids[rank] = row_ids[0xffffffffu - (uint32_t)(mine & 0xffffffffull)];
+            out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
             if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
           }
         }
         return;
       }
       bitonic_sort_desc<THREADS>(sm.cand, P2);
-      write_topk<THREADS>(sm.cand, take, k, row_ids, out_ids, out_scores);
+      write_topk<THREADS>(sm.cand, take, k, ids, out_ids, out_scores);
       return;
     }
   }
@@ -413,7 +424,7 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   __syncthreads();
 
   bitonic_sort_desc<THREADS>(sm.cand, P);
-  write_topk<THREADS>(sm.cand, take, k, row_ids, out_ids, out_scores);
+  write_topk<THREADS>(sm.cand, take, k, ids, out_ids, out_scores);
 }
 
 // Scoring only (large segments): grid = (row groups, nq); dynamic shared memory holds the query as fp32.
@@ -440,8 +451,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams
   const bool user_ok = user >= 0 && user < p.n_users;
   const int n = user_ok ? p.user_count[user] : 0;
   topk_block<kTopkThreads>(sm, p.scores + (int64_t)q * p.score_stride, nullptr, n, p.k,
-                           p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity, p.out_ids + (int64_t)q * p.k,
-                           p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
+                           IdMap{nullptr, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
+                           p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
 }
 
 // Scoring + top-k in ONE launch for segments of at most kFusedMaxRows rows: grid = (row groups, nq).
@@ -483,9 +494,151 @@ __global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const R
     hi = max(hi, kx);
   }
   __syncthreads();
-  topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity,
+  topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k,
+                            IdMap{nullptr, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
+}
+
+// ---- tensor-core path, steps 2 and 3 (step 1 is score_gemm_groupmax_kernel) -------------------------------------
+
+// Step 2: per query, the k2 groups with the largest group maximum, written in ASCENDING group order (so that the
+// candidate rows of step 3 are in row order and "lower index first" among equal scores means "lower fact id first").
+__global__ void __launch_bounds__(kTopkThreads) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
+                                                                    int32_t* sel /*[nq][k2]*/) {
+  __shared__ TopkShared sm;
+  __shared__ int32_t s_sel[512];
+  const int q = blockIdx.x;
+  int32_t* out = sel + (int64_t)q * k2;
+  topk_block<kTopkThreads>(sm, gmax + (int64_t)q * gmax_stride, nullptr, n_groups, k2, IdMap{nullptr, nullptr}, out, nullptr);
+  __syncthreads();
+  // sort the chosen group indices ascending (k2 <= 512; -1 padding becomes the largest key and stays last)
+  for (int i = threadIdx.x; i < 512; i += kTopkThreads) s_sel[i] = i < k2 ? out[i] : -1;
+  __syncthreads();
+  for (int size = 2; size <= 512; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < 256; t += kTopkThreads) {
+        const int lo = 2 * t - (t & (stride - 1));
+        const int hi = lo + stride;
+        const bool asc = (lo & size) == 0;
+        const uint32_t a = (uint32_t)s_sel[lo], b = (uint32_t)s_sel[hi];
+        if ((a > b) == asc) {
+          s_sel[lo] = (int32_t)b;
+          s_sel[hi] = (int32_t)a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  for (int i = threadIdx.x; i < k2; i += kTopkThreads) out[i] = s_sel[i];
+}
+
+// One row's score with the lane layout and summation order of score_rows (all lanes return the sum).
+template <typename T>
+__device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, const T* seg, int64_t row) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int E = p.emb_dim;
+  const int lane = threadIdx.x & 31;
+  const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
+  const uint4* rp = reinterpret_cast<const uint4*>(seg + row * E);
+  const int nvec = E / VEC;
+  float acc = 0.f;
+  for (int v0 = 0; v0 < nvec; v0 += 128) {
+    uint4 x[4], y[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        x[u] = __ldg(rp + v);
+        y[u] = __ldg(qp + v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        if (sizeof(T) == 2) {
+          float f[8], g[8];
+          unpack8(x[u], f);
+          unpack8(y[u], g);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc = fmaf(f[i], g[i], acc);
+        } else {
+          const float* f = reinterpret_cast<const float*>(&x[u]);
+          const float* g = reinterpret_cast<const float*>(&y[u]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc = fmaf(f[i], g[i], acc);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  return acc;
+}
+
+// Step 3: rescore the rows of the selected groups exactly (fp32 CUDA-core sums, the same arithmetic as the other
+// retrieve kernels) and take the top-k of these candidates.  grid = (candidate groups of 8 rows per warp..., nq);
+// candidate c of query q is row sel[q][c / 8] * 8 + c % 8.  The last CTA of a query (wait-free ticket) selects.
+// Dynamic shared memory: n_cand uint32 keys.
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const RetrieveParams p, const int32_t* sel, int k2, int n_rows,
+                                                                     float* cand_scores, int32_t* cand_rows, uint32_t* tickets) {
+  extern __shared__ uint32_t s_keys[];
+  __shared__ TopkShared sm;
+  __shared__ int s_last;
+  const int q = blockIdx.y;
+  const int n_cand = k2 * 8;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const T* seg = reinterpret_cast<const T*>(p.emb);  // user 0
+  float* cs = cand_scores + (int64_t)q * n_cand;
+  int32_t* cr = cand_rows + (int64_t)q * n_cand;
+  const int c0 = blockIdx.x * kScoreWarps * 8;  // one group of 8 candidate rows per warp
+  {
+    const int g_idx = c0 / 8 + warp;
+    if (g_idx < k2) {
+      const int32_t g = sel[(int64_t)q * k2 + g_idx];
+      for (int r = 0; r < 8; ++r) {
+        const int64_t row = (int64_t)g * 8 + r;
+        const bool ok = g >= 0 && row < n_rows;
+        float s = -INFINITY;
+        if (ok) s = score_one_row<T>(p, q, seg, row) + 0.0f;
+        if (lane == 0) {
+          cs[g_idx * 8 + r] = s;
+          cr[g_idx * 8 + r] = ok ? (int32_t)row : -1;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const uint32_t t = atomicAdd(&tickets[q], 1u);
+    s_last = t == gridDim.x - 1;
+    if (s_last) tickets[q] = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // Candidates are in ascending row order with every absent one (padding group, row beyond the segment) at the
+  // end, so the valid candidates are a prefix: count them and select among those only.
+  int mine = 0;
+  for (int i = threadIdx.x; i < n_cand; i += kScoreThreads) mine += __ldcg(cr + i) >= 0;
+  mine = __reduce_add_sync(0xffffffffu, mine);
+  if (lane == 0) sm.warp_cnt[warp] = (uint32_t)mine;
+  __syncthreads();
+  int n_valid = 0;
+  for (int w = 0; w < kScoreThreads / 32; ++w) n_valid += (int)sm.warp_cnt[w];
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for (int i = threadIdx.x; i < n_valid; i += kScoreThreads) {
+    const uint32_t kx = order_key(__ldcg(cs + i));
+    s_keys[i] = kx;
+    lo = min(lo, kx);
+    hi = max(hi, kx);
+  }
+  __syncthreads();
+  topk_block<kScoreThreads>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
+                            p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo, hi);
 }
 
 }  // namespace ms

@@ -53,7 +53,7 @@ class _PagedCache(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "kernel_timeouts")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares

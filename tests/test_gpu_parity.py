@@ -96,6 +96,32 @@ def test_retrieve_empty_store_and_per_user_segments():
         check_ids(ids[i], sc[i], hs.emb[rows], q[i], 60, row_ids=rows.astype(np.int32))
 
 
+@pytest.mark.parametrize("n,E,nq", [(20000, 1024, 64), (9001, 256, 37), (12345, 64, 100)])
+def test_retrieve_many_queries_tensor_core_path(n, E, nq):
+    """8+ fp16 queries on one large segment: tcgen05 group-max filter, group selection, exact rescoring."""
+    hs = HostStore(30, n, 1, 1, 16, 1, 1, E, "float16")
+    hs.emb[n - 1] = hs.emb[17]  # duplicates in different groups, one in the ragged last tile
+    hs.emb[5000] = hs.emb[17]
+    ms = hs.to_memstore(1e4, batch=4096)
+    q = synth.queries(30, nq, E, "float16")
+    q[0] = hs.emb[17]  # a query equal to a stored row: the three copies tie for rank 0..2
+    for k in (1, 100, 256):
+        ids, sc = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+        assert ms.stats()["kernel_timeouts"] == 0
+        if k >= 3:
+            assert ids[0, :3].tolist() == [17, 5000, n - 1] and sc[0, 0] == sc[0, 1] == sc[0, 2]
+        for i in list(range(0, nq, 9)) + [nq - 1]:
+            check_ids(ids[i], sc[i], hs.emb, q[i], k)
+    # the same queries one by one go through the CUDA-core kernels: identical ids and bit-identical scores
+    ids_tc, sc_tc = ms.retrieve(to_dev(q), 50)
+    for i in (0, 1, nq - 1):
+        ids_1, sc_1 = ms.retrieve(to_dev(q[i : i + 1]), 50)
+        assert torch.equal(ids_1[0], ids_tc[i]) and torch.equal(sc_1[0], sc_tc[i])
+    ms.close()
+
+
 # ------------------------------------------------------------------------------------------------ injection
 PATHS = [0, 1]  # 0: direct copy kernel (default), 1: MS_STORE_TMA_COPY_PATH (bulk-async staged kernel)
 
