@@ -76,13 +76,27 @@ def fact_lengths(seed: int, n: int, lo: int, hi: int) -> np.ndarray:
 
 
 def unit_rows(seed: int, stream: int, n: int, dim: int, dtype: str, chunk: int = 65536) -> np.ndarray:
-    """i.i.d. Gaussian rows, normalised to unit length in float32, then rounded to ``dtype`` (not re-normalised)."""
+    """i.i.d. Gaussian rows, normalised to unit length in float32, then rounded to ``dtype`` (not re-normalised).
+    Every chunk of rows has its own generator, so chunks are drawn in parallel threads with identical results."""
     out = np.empty((n, dim), dtype=np.dtype(dtype))
-    for c, a in enumerate(range(0, n, chunk)):
+
+    def draw(c: int) -> None:
+        a = c * chunk
         b = min(n, a + chunk)
         x = _rng(seed, stream, c).standard_normal((b - a, dim), dtype=np.float32)
         x /= np.linalg.norm(x, axis=1, keepdims=True)
         out[a:b] = x.astype(out.dtype)
+
+    n_chunks = (n + chunk - 1) // chunk
+    if n_chunks <= 1:
+        for c in range(n_chunks):
+            draw(c)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+
+        with ThreadPoolExecutor(max_workers=min(n_chunks, os.cpu_count() or 1, 16)) as pool:
+            list(pool.map(draw, range(n_chunks)))
     return out
 
 

@@ -56,13 +56,15 @@ class Workload:
 
 def build(name: str, seed: int = 0, device="cuda", n_query_pool: int | None = None, num_blocks: int | None = None,
           resident_ids=None, hot_per_user: int | None = None, scale_facts: float = 1.0, add_batch_tokens: int = 4096,
-          want_cache: bool = True) -> Workload:  # fmt: skip
+          want_cache: bool = True, emb: np.ndarray | None = None, queries: np.ndarray | None = None) -> Workload:  # fmt: skip
     """Create the store of configuration ``name`` and fill it.
 
     ``resident_ids``: for configurations with a hot subset, the global fact ids that must have K/V (the
     harness passes the ids its requests will inject); random filler ids complete the subset up to
     ``hot_per_user`` facts per user (default: the configuration's figure).
-    ``scale_facts`` < 1 shrinks the number of facts per user (tests on smaller boxes)."""
+    ``scale_facts`` < 1 shrinks the number of facts per user (tests on smaller boxes).
+    ``emb`` / ``queries``: arrays already drawn with ``synth.embeddings`` / ``synth.queries`` for the same seed
+    (saves drawing a million rows twice)."""
     s = synth.CONFIGS[name]
     dev = torch.device(device)
     n_per_user = max(1, int(round(s.n_facts * scale_facts)))
@@ -81,9 +83,12 @@ def build(name: str, seed: int = 0, device="cuda", n_query_pool: int | None = No
                 cold = seg[~hot[seg]]
                 hot[rng.choice(cold, size=min(missing, cold.size), replace=False)] = True
         lens = np.where(hot, lens, 0).astype(np.int32)
-    emb = synth.embeddings(seed, total, s.emb_dim, s.emb_dtype)
+    if emb is None:
+        emb = synth.embeddings(seed, total, s.emb_dim, s.emb_dtype)
     nq_pool = n_query_pool or max(s.nq, 16)
-    queries = synth.queries(seed, nq_pool, s.emb_dim, s.emb_dtype)
+    if queries is None:
+        queries = synth.queries(seed, nq_pool, s.emb_dim, s.emb_dtype)
+    assert emb.shape == (total, s.emb_dim) and queries.shape[1] == s.emb_dim
     tdt = torch.float32 if s.emb_dtype == "float32" else torch.float16
     store = MemStore(device=dev.index or 0, n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim,
                      emb_dim=s.emb_dim, emb_dtype=tdt, rope_theta=s.rope_theta, n_users=s.n_users,

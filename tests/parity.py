@@ -72,10 +72,9 @@ class HostStore:
         return ms
 
 
-def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None, oracle_scores=None):
+def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None):
     """Near-tie rule for one query. ``emb``: the rows visible to the query; row_ids: their fact ids."""
     n = emb.shape[0]
-    s = oracle.scores(emb, query) if oracle_scores is None else oracle_scores
     ids_o, sc_o = oracle.retrieve(emb, query, k, row_ids=row_ids)
     ids_o, sc_o = ids_o[0], sc_o[0]
     gpu_ids = np.asarray(gpu_ids)
@@ -84,13 +83,14 @@ def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None, oracle_scores=No
     g = gpu_ids[:take]
     assert len(set(g.tolist())) == take, "duplicate ids"
     if row_ids is None:
-        rows = g
+        rows = g.astype(np.int64)
         assert np.all((g >= 0) & (g < n)), "invalid id"
     else:
         lookup = {int(f): i for i, f in enumerate(row_ids)}
         assert all(int(x) in lookup for x in g), "id outside the user's segment"
         rows = np.array([lookup[int(x)] for x in g], dtype=np.int64)
-    s_gpu_choice = s[rows].astype(np.float32)
+    # the oracle's exact score of every row the GPU chose
+    s_gpu_choice = oracle.scores(emb[rows], query).astype(np.float32) if take else np.zeros(0, np.float32)
     diff = np.abs(s_gpu_choice - sc_o[:take])
     assert np.all(diff < SCORE_TIE), f"rank-wise score gap {diff.max()} (not a near-tie)"
     exact = g == ids_o[:take]  # ranks where the lists differ are swaps inside a near-tie group

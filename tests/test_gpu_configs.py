@@ -135,8 +135,7 @@ def test_users100_batched_retrieve_and_shared_cache():
     pool_blocks = 65536
     while pool_blocks * c.block_size * c.token_bytes / 2**30 > free_gib() - 40 and pool_blocks > 8192:
         pool_blocks //= 2
-    wl = workload.build("users100", seed=2, num_blocks=pool_blocks, resident_ids=want, n_query_pool=n_users)
-    assert np.array_equal(wl.emb, emb) and np.array_equal(wl.queries, queries)
+    wl = workload.build("users100", seed=2, num_blocks=pool_blocks, resident_ids=want, n_query_pool=n_users, emb=emb, queries=queries)
     cache = wl.cache
     fill_sentinel(cache)
     users = torch.arange(n_users, dtype=torch.int32, device="cuda")
@@ -181,7 +180,8 @@ def test_stress1m_64_queries_top100_inject_top50():
     for i in range(c.nq):
         hot.update(np.argpartition(-cand_scores[i], 64)[:64].tolist())
     del cand_scores
-    wl = workload.build("stress1m", seed=3, num_blocks=16384, resident_ids=sorted(hot), n_query_pool=c.nq, hot_per_user=len(hot))
+    wl = workload.build("stress1m", seed=3, num_blocks=16384, resident_ids=sorted(hot), n_query_pool=c.nq, hot_per_user=len(hot),
+                        emb=emb, queries=queries)
     ids, sc = wl.store.retrieve(torch.from_numpy(queries).cuda(), c.k)
     torch.cuda.synchronize()
     ids_np, sc_np = ids.cpu().numpy(), sc.cpu().numpy()
