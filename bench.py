@@ -310,24 +310,13 @@ def run_ours(args):
     n_e2e = min(args.steps, 500)
     q_host = torch.from_numpy(wl.queries).pin_memory()
     t_host = torch.from_numpy(synth.block_tables(args.seed + rank, cache.num_blocks, per_req_blocks, n_pool)).pin_memory()
-    s_host = torch.full((1,), shape.start_pos, dtype=torch.int32).pin_memory()
     out_host = torch.empty((k + 2,), dtype=torch.int32).pin_memory()
-    q_dev = torch.empty_like(queries[:1])
-    t_dev = torch.empty_like(tables[:1])
-    s_dev = torch.empty_like(start)
-    res_dev = torch.empty((k + 2,), dtype=torch.int32, device=dev)
-    ids_v = res_dev[:k].view(1, k)
 
     def e2e_step(i):
+        # the public host-buffer call: one H2D transfer (query, start position, block table), retrieve, inject,
+        # one D2H transfer (ids, token count, status) and a stream synchronise, all inside the library
         j = i % n_pool
-        q_dev.copy_(q_host[j : j + 1], non_blocking=True)
-        t_dev.copy_(t_host[j : j + 1], non_blocking=True)
-        s_dev.copy_(s_host, non_blocking=True)
-        store.retrieve(q_dev, k, out_ids=ids_v, want_scores=False, stream=stream)
-        store.inject(ids_v, s_dev, t_dev, cache, out_n_tokens=res_dev[k : k + 1], out_status=res_dev[k + 1 : k + 2],
-                     flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
-        out_host.copy_(res_dev, non_blocking=True)
-        stream.synchronize()  # the caller needs ids / token count / status before it can schedule the request
+        store.serve_host(q_host[j], k, shape.start_pos, t_host[j], cache, out_host, flags=M.INJECT_REVERSE, stream=stream)
 
     for i in range(5):
         e2e_step(i)
@@ -343,7 +332,7 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t[0])
     e2e_us = e2e_ms * 1e3 / (n_e2e * world)
-    h2d = q_host[0:1].numel() * q_host.element_size() + t_host[0:1].numel() * 4 + 4
+    h2d = ((q_host[0].numel() * q_host.element_size() + 15) // 16) * 16 + 16 + ((t_host[0].numel() * 4 + 15) // 16) * 16
     d2h = (k + 2) * 4
 
     line = {

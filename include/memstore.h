@@ -201,6 +201,20 @@ ms_status memstore_inject(memstore_t* store, const int32_t* fact_ids, int32_t nr
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
                           uint32_t flags, ms_stream stream);
 
+/*
+ * One request end to end from HOST buffers, for a caller that holds its query and block table in host memory
+ * (Sec. 3.3 and 3.4 in one call: search, compose, scatter).  Copies the query, the start position and the block table
+ * to the device in one transfer (through a pinned staging buffer owned by the store, allocated on first use),
+ * retrieves the k best facts of `user`, injects them (flags: MS_INJECT_*), copies ids, token count and status
+ * back in one transfer and waits for the stream.
+ *   query        host, [emb_dim] in emb_dtype          block_table  host int32 [max_blocks]
+ *   out_ids      host int32 [k] (best first, -1 padded) out_n_tokens, out_status  host, optional
+ * The paged cache itself stays on the device.  Not thread-safe against other calls on the same store.
+ */
+ms_status memstore_serve_host(memstore_t* store, const void* query, int32_t user, int32_t k, int32_t start_pos,
+                              const int32_t* block_table, int32_t max_blocks, const ms_paged_cache* cache, uint32_t flags,
+                              int32_t* out_ids, int32_t* out_n_tokens, int32_t* out_status, ms_stream stream);
+
 /* Counters since creation (host side; bytes are the algorithmic ones, not measured traffic).  Reading
  * kernel_timeouts synchronises the device. */
 typedef struct {

@@ -50,6 +50,10 @@ struct memstore {
   InjectCtrl* ctrl = nullptr;
   cudaEvent_t last_done = nullptr;
   cudaEvent_t prof_before = nullptr, prof_after = nullptr;  // caller-owned, optional
+  // memstore_serve_host staging: one pinned host buffer and one device buffer, inputs first, outputs after
+  unsigned char* host_stage = nullptr;
+  unsigned char* dev_stage = nullptr;
+  size_t stage_bytes = 0;
   cudaStream_t last_stream = nullptr;
   bool have_last = false;
   // host mirrors
@@ -60,7 +64,7 @@ struct memstore {
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
   int copy_ctas_per_sm = 1;
   bool tma_path = false;  // MS_STORE_TMA_COPY_PATH
-  std::mutex mu;
+  std::recursive_mutex mu;  // recursive: memstore_serve_host holds it across retrieve and inject
   std::string err;
 };
 
@@ -335,6 +339,8 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_tickets);
     cudaFree(s->tc_error);
     cudaFree(s->tiles);
+    cudaFree(s->dev_stage);
+    if (s->host_stage) cudaFreeHost(s->host_stage);
     if (s->last_done) cudaEventDestroy(s->last_done);
     cudaGetLastError();
   }
@@ -345,7 +351,7 @@ ms_status memstore_destroy(memstore_t* s) {
 ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
                              const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
   if (n < 0 || (n > 0 && (!embs || !n_tokens))) return fail(s, MS_ERR_INVALID_ARG, "null embeddings or lengths");
@@ -420,7 +426,7 @@ ms_status memstore_add_fact(memstore_t* s, int32_t user, const void* emb, const 
 ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                             int32_t* out_ids, float* out_scores, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (nq < 0 || k < 1 || k > kTopkMaxK) return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d (1 <= k <= %d)", nq, k, kTopkMaxK);
   if (nq == 0) return MS_OK;
@@ -526,7 +532,7 @@ cudaError_t static_scratch_address(int device, unsigned char** out) {
 ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                                    int32_t* out_ids, float* out_scores, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (nq < 0 || k < 1 || k > kTopkMaxK) return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d (1 <= k <= %d)", nq, k, kTopkMaxK);
   if (nq == 0) return MS_OK;
@@ -600,7 +606,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
                           uint32_t flags, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (nreq < 0 || k < 0 || k > kPlanMaxK) return fail(s, MS_ERR_INVALID_ARG, "nreq=%d k=%d (k <= %d)", nreq, k, kPlanMaxK);
   if (flags & ~(uint32_t)MS_INJECT_REVERSE) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
@@ -736,9 +742,60 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   return mark_last(s, st);
 }
 
+ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, int32_t k, int32_t start_pos,
+                              const int32_t* block_table, int32_t max_blocks, const ms_paged_cache* cache, uint32_t flags,
+                              int32_t* out_ids, int32_t* out_n_tokens, int32_t* out_status, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (!query || !block_table || !out_ids || max_blocks <= 0 || k < 1 || k > kTopkMaxK)
+    return fail(s, MS_ERR_INVALID_ARG, "memstore_serve_host: null buffer, max_blocks=%d or k=%d out of range", max_blocks, k);
+  if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  // layout of both staging buffers: [query | start_pos, user, pad, pad | block table] then [ids | n_tokens, status]
+  const size_t q_bytes = ((size_t)c.emb_dim * emb_elem_size(c.emb_dtype) + 15) & ~(size_t)15;
+  const size_t in_bytes = q_bytes + 16 + (((size_t)max_blocks * 4 + 15) & ~(size_t)15);
+  const size_t out_bytes = (((size_t)k + 2) * 4 + 15) & ~(size_t)15;
+  if (in_bytes + out_bytes > s->stage_bytes) {
+    MS_CUDA(s, cudaDeviceSynchronize());
+    cudaFree(s->dev_stage);
+    if (s->host_stage) cudaFreeHost(s->host_stage);
+    s->dev_stage = nullptr;
+    s->host_stage = nullptr;
+    s->stage_bytes = 0;
+    const size_t want = (in_bytes + out_bytes) * 2;
+    MS_CUDA(s, cudaMalloc(&s->dev_stage, want));
+    MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocDefault));
+    s->stage_bytes = want;
+  }
+  unsigned char* h = s->host_stage;
+  unsigned char* d = s->dev_stage;
+  memcpy(h, query, (size_t)c.emb_dim * emb_elem_size(c.emb_dtype));
+  int32_t* hdr = reinterpret_cast<int32_t*>(h + q_bytes);
+  hdr[0] = start_pos;
+  hdr[1] = user;
+  memcpy(h + q_bytes + 16, block_table, (size_t)max_blocks * 4);
+  MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, st));
+  int32_t* d_hdr = reinterpret_cast<int32_t*>(d + q_bytes);
+  int32_t* d_ids = reinterpret_cast<int32_t*>(d + in_bytes);
+  ms_status rc = memstore_retrieve(s, d, c.n_users > 1 ? d_hdr + 1 : nullptr, 1, k, d_ids, nullptr, stream);
+  if (rc != MS_OK) return rc;
+  rc = memstore_inject(s, d_ids, 1, k, d_hdr, reinterpret_cast<const int32_t*>(d + q_bytes + 16), max_blocks, cache, d_ids + k,
+                       d_ids + k + 1, nullptr, 0, flags, stream);
+  if (rc != MS_OK) return rc;
+  MS_CUDA(s, cudaMemcpyAsync(h + in_bytes, d_ids, ((size_t)k + 2) * 4, cudaMemcpyDeviceToHost, st));
+  MS_CUDA(s, cudaStreamSynchronize(st));
+  const int32_t* res = reinterpret_cast<const int32_t*>(h + in_bytes);
+  memcpy(out_ids, res, (size_t)k * 4);
+  if (out_n_tokens) *out_n_tokens = res[k];
+  if (out_status) *out_status = res[k + 1];
+  return MS_OK;
+}
+
 ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   if (!s || !out) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   out->n_facts = s->n_facts;
   out->n_resident_facts = s->n_resident;
   out->kv_tokens_used = s->kv_tokens_used;
@@ -759,7 +816,7 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
 
 ms_status memstore_set_profile_events(memstore_t* s, void* before_copy, void* after_copy) {
   if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(s->mu);
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
   if ((before_copy == nullptr) != (after_copy == nullptr)) return fail(s, MS_ERR_INVALID_ARG, "give both events or neither");
   s->prof_before = (cudaEvent_t)before_copy;
   s->prof_after = (cudaEvent_t)after_copy;

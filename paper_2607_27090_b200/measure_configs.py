@@ -1,0 +1,126 @@
+"""Timing of the batched workload configurations (many queries / many requests per call) on one GPU.
+
+    python -m paper_2607_27090_b200.measure_configs --config users100|stress1m|gqa14b|llama8b [--iters 20]
+
+``bench.py`` times the headline configuration (one request at k = 50).  This module times the others the same
+way (CUDA events on one stream, warm-up first, inputs already in HBM) and prints one JSON line per
+configuration: microseconds of the batched retrieve call and of the batched inject call, bytes scanned / moved,
+and the rates they imply.  No step of the method runs here; the hot set of a configuration with partial
+residency is picked by the harness from a plain numpy product (a store-construction input).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import memstore as M
+from . import synth, workload
+
+
+def candidate_hot_ids(emb: np.ndarray, queries: np.ndarray, per_query: int, users: np.ndarray | None = None, per_user: int = 0):
+    """Ids that a request may name: per query the ``per_query`` rows with the largest fp32 numpy scores (inside the
+    query's user segment when ``users`` is given).  A superset of every exact top-k list with k < per_query."""
+    hot: set[int] = set()
+    qf = queries.astype(np.float32)
+    if users is None:
+        n = emb.shape[0]
+        best = np.full((qf.shape[0], per_query), -np.inf, np.float32)
+        best_id = np.zeros((qf.shape[0], per_query), np.int64)
+        for a in range(0, n, 131072):
+            sc = qf @ emb[a : a + 131072].astype(np.float32).T
+            allsc = np.concatenate([best, sc], axis=1)
+            allid = np.concatenate([best_id, np.broadcast_to(np.arange(a, a + sc.shape[1]), sc.shape)], axis=1)
+            part = np.argpartition(-allsc, per_query - 1, axis=1)[:, :per_query]
+            best = np.take_along_axis(allsc, part, axis=1)
+            best_id = np.take_along_axis(allid, part, axis=1)
+        hot.update(best_id.reshape(-1).tolist())
+    else:
+        for i, u in enumerate(users):
+            rows = np.arange(u * per_user, (u + 1) * per_user)
+            sc = emb[rows].astype(np.float32) @ qf[i]
+            hot.update(rows[np.argpartition(-sc, per_query - 1)[:per_query]].tolist())
+    return sorted(hot)
+
+
+def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
+    s = synth.CONFIGS[name]
+    dev = torch.device("cuda")
+    total = s.n_facts * s.n_users
+    emb = synth.embeddings(seed, total, s.emb_dim, s.emb_dtype)
+    nq = s.nq
+    queries = synth.queries(seed, nq, s.emb_dim, s.emb_dtype)
+    k_inj = 50 if name == "stress1m" else s.k
+    users = np.arange(s.n_users, dtype=np.int32) if s.n_users > 1 else None
+    hot = None
+    if s.resident_per_user is not None:
+        hot = candidate_hot_ids(emb, queries, k_inj + 14, users, s.n_facts)
+        if hot_per_user is None:
+            hot_per_user = max(s.resident_per_user // 5, (len(hot) + s.n_users - 1) // s.n_users) if name == "stress1m" else s.resident_per_user
+    per_req = workload.blocks_per_request(s, k_inj)
+    nb = pool_blocks or max(1024, 1 << int(np.ceil(np.log2(per_req * nq * 2))))
+    wl = workload.build(name, seed=seed, device=dev, n_query_pool=nq, num_blocks=nb, resident_ids=hot, hot_per_user=hot_per_user,
+                        emb=emb, queries=queries)  # fmt: skip
+    store, cache = wl.store, wl.cache
+    q_dev = torch.from_numpy(queries).to(dev)
+    u_dev = torch.from_numpy(users).to(dev) if users is not None else None
+    n_sets = 2
+    tables = [torch.from_numpy(synth.block_tables(seed + t, cache.num_blocks, per_req, nq)).to(dev) for t in range(n_sets)]
+    starts = torch.full((nq,), s.start_pos, dtype=torch.int32, device=dev)
+    ids = torch.empty((nq, s.k), dtype=torch.int32, device=dev)
+    n_tok = torch.zeros(nq, dtype=torch.int32, device=dev)
+    status = torch.zeros(nq, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def retrieve():
+        store.retrieve(q_dev, s.k, query_users=u_dev, out_ids=ids, want_scores=False, stream=stream)
+
+    def inject(i):
+        top = ids if k_inj == s.k else ids[:, :k_inj].contiguous()
+        store.inject(top, starts, tables[i % n_sets], cache, out_n_tokens=n_tok, out_status=status, flags=M.INJECT_REVERSE, stream=stream)
+
+    for i in range(3):
+        retrieve()
+        inject(i)
+    torch.cuda.synchronize()
+    assert int(status.abs().sum()) == 0, "a request named a fact without K/V: the hot set was chosen too small"
+    m_total = int(n_tok.sum())
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    t_r, t_i = [], []
+    for i in range(iters):
+        ev[0].record(stream)
+        retrieve()
+        ev[1].record(stream)
+        inject(i)
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        t_r.append(ev[0].elapsed_time(ev[1]) * 1e3)
+        t_i.append(ev[1].elapsed_time(ev[2]) * 1e3)
+    r_us, i_us = float(np.median(t_r)), float(np.median(t_i))
+    emb_bytes = workload.emb_bytes_scanned(s, total)
+    kv_bytes = workload.kv_bytes_moved(s, m_total)
+    flops = 2.0 * total * s.emb_dim * nq if s.n_users == 1 else 2.0 * total * s.emb_dim
+    line = {
+        "config": name, "queries_per_call": nq, "k": s.k, "k_injected": k_inj, "requests_per_call": nq,
+        "facts_scanned": total, "tokens_injected": m_total, "pool_blocks": cache.num_blocks,
+        "resident_facts": int((wl.lens > 0).sum()),
+        "retrieve_us": r_us, "retrieve_emb_gbs": emb_bytes / (r_us * 1e-6) / 1e9, "retrieve_tflops": flops / (r_us * 1e-6) / 1e12,
+        "inject_us": i_us, "inject_gbs": kv_bytes / (i_us * 1e-6) / 1e9,
+        "us_per_request": (r_us + i_us) / nq,
+        "kernel_timeouts": store.stats()["kernel_timeouts"],
+    }  # fmt: skip
+    store.close()
+    return line
+
+
+if __name__ == "__main__":
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="users100")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--hot-per-user", type=int, default=None)
+    ap.add_argument("--pool-blocks", type=int, default=None)
+    a = ap.parse_args()
+    print(json.dumps(measure(a.config, a.iters, a.seed, a.hot_per_user, a.pool_blocks)))

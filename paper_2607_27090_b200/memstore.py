@@ -60,7 +60,7 @@ class _Stats(C.Structure):
 EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
-    "memstore_set_profile_events", "memstore_retrieve_static",
+    "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
 )  # fmt: skip
 
 _lib = None
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.memstore_retrieve_static.restype = i32
     L.memstore_retrieve_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    L.memstore_serve_host.restype = i32
+    L.memstore_serve_host.argtypes = [vp, vp, i32, i32, i32, vp, i32, C.POINTER(_PagedCache), u32, vp, vp, vp, vp]
     L.memstore_inject.restype = i32
     L.memstore_inject.argtypes = [vp, vp, i32, i32, vp, vp, i32, C.POINTER(_PagedCache), vp, vp, vp, i64, u32, vp]
     L.memstore_stats.restype = i32
@@ -295,6 +297,27 @@ class MemStore:
                                        flags, _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out_n_tokens, out_status
+
+    def serve_host(self, query, k, start_pos, block_table, cache: PagedCache, out, user=0, flags=0, stream=None):
+        """One request from HOST buffers (numpy arrays or CPU tensors): ``query`` [emb_dim], ``block_table`` int32
+        [max_blocks]; ``out`` int32 [k + 2] receives ids, then the token count, then the status word."""
+        import numpy as np
+
+        def host_ptr(a, dtype):
+            if isinstance(a, torch.Tensor):
+                assert not a.is_cuda and a.is_contiguous() and a.dtype == dtype
+                return C.c_void_p(a.data_ptr())
+            assert isinstance(a, np.ndarray) and a.flags.c_contiguous
+            return C.c_void_p(a.ctypes.data)
+
+        cs = cache._struct()
+        o = host_ptr(out, torch.int32)
+        rc = self._lib.memstore_serve_host(self._h, host_ptr(query, self.emb_torch_dtype), user, k, int(start_pos),
+                                           host_ptr(block_table, torch.int32), int(block_table.shape[-1]), C.byref(cs), flags,
+                                           o, C.c_void_p(o.value + 4 * k), C.c_void_p(o.value + 4 * k + 4),
+                                           _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out
 
     def set_profile_events(self, before_copy=None, after_copy=None):
         """torch.cuda.Event pair (created with enable_timing=True and already recorded once so that they own a

@@ -229,6 +229,28 @@ def test_inject_empty_and_degenerate_requests():
     assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
 
 
+def test_serve_host_matches_the_device_calls():
+    """memstore_serve_host (host buffers in, host results out) against retrieve + inject on device buffers."""
+    hs = HostStore(19, 120, 2, 8, 128, 8, 40, 256, "float16", n_users=2)
+    ms = hs.to_memstore(5e5)
+    bs, nb, k, start = 16, 64, 7, 21
+    table = synth.block_tables(20, nb, 40, 1)[0]
+    for user in (0, 1):
+        q = synth.queries(19 + user, 1, 256, "float16")
+        ca, cb = make_cache(hs, nb, bs), make_cache(hs, nb, bs)
+        users = to_dev(np.array([user], np.int32))
+        ids, _ = ms.retrieve(to_dev(q), k, query_users=users)
+        n_tok, status = ms.inject(ids, to_dev(np.array([start], np.int32)), to_dev(table[None]), ca, flags=M.INJECT_REVERSE)
+        out = np.full(k + 2, -5, np.int32)
+        ms.serve_host(q[0], k, start, table, cb, out, user=user, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        assert out[:k].tolist() == ids[0].cpu().tolist() and out[k] == int(n_tok[0]) and out[k + 1] == int(status[0]) == 0
+        assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+        rows = np.arange(user * 120, (user + 1) * 120)
+        check_ids(out[:k], None, hs.emb[rows], q[0], k, row_ids=rows.astype(np.int32))
+    ms.close()
+
+
 # ------------------------------------------------------------------------------------------------ safety
 def test_inject_data_errors_set_status_and_skip():
     lens = [4, 6, 0, 5]
