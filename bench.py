@@ -241,10 +241,10 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     def step(i):
+        # one request through the whole path: the library's retrieve+inject call (two kernel launches)
         j = i % n_pool
-        store.retrieve(queries[j : j + 1], k, out_ids=ids, want_scores=False, stream=stream)
-        store.inject(ids, start, tables[j : j + 1], cache, out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1],
-                     flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+        store.retrieve_inject(queries[j : j + 1], k, start, tables[j : j + 1], cache, out_ids=ids, out_n_tokens=n_tok[j : j + 1],
+                              out_status=status[j : j + 1], flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
 
     def barrier():
         if world > 1:
@@ -365,16 +365,18 @@ def run_ours(args):
         sweep = {}
         for kk in (5, 10, 20):
             ids_k = torch.empty((1, kk), dtype=torch.int32, device=dev)
+            def step_k(i):
+                j = i % n_pool
+                store.retrieve_inject(queries[j : j + 1], kk, start, tables[j : j + 1], cache, out_ids=ids_k,
+                                      out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1], flags=M.INJECT_REVERSE,
+                                      stream=stream)  # fmt: skip
+
             for i in range(10):
-                store.retrieve(queries[i % n_pool : i % n_pool + 1], kk, out_ids=ids_k, want_scores=False, stream=stream)
-                store.inject(ids_k, start, tables[i % n_pool : i % n_pool + 1], cache, flags=M.INJECT_REVERSE, stream=stream)
+                step_k(i)
             torch.cuda.synchronize()
             e0.record(stream)
             for i in range(args.steps):
-                j = i % n_pool
-                store.retrieve(queries[j : j + 1], kk, out_ids=ids_k, want_scores=False, stream=stream)
-                store.inject(ids_k, start, tables[j : j + 1], cache, out_n_tokens=n_tok[j : j + 1],
-                             out_status=status[j : j + 1], flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
+                step_k(i)
             e1.record(stream)
             torch.cuda.synchronize()
             sweep[f"k{kk}_us"] = e0.elapsed_time(e1) * 1e3 / args.steps

@@ -202,6 +202,18 @@ ms_status memstore_inject(memstore_t* store, const int32_t* fact_ids, int32_t nr
                           uint32_t flags, ms_stream stream);
 
 /*
+ * memstore_retrieve immediately followed by memstore_inject of every query's id list (query q = request q), with
+ * the ids handed over on the device and, for segments of at most 8192 rows, the requests planned inside the
+ * retrieval kernel, so that the whole path is two launches (Sec. 3.3: search, compose and scatter per request).
+ * Arguments as in the two calls; out_ids [nq][k] is both the retrieval output and the injection input.
+ */
+ms_status memstore_retrieve_inject(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                                   const int32_t* start_pos, const int32_t* block_tables, int32_t max_blocks,
+                                   const ms_paged_cache* cache, int32_t* out_ids, float* out_scores, int32_t* out_n_tokens,
+                                   int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags,
+                                   ms_stream stream);
+
+/*
  * One request end to end from HOST buffers, for a caller that holds its query and block table in host memory
  * (Sec. 3.3 and 3.4 in one call: search, compose, scatter).  Copies the query, the start position and the block table
  * to the device in one transfer (through a pinned staging buffer owned by the store, allocated on first use),

@@ -49,17 +49,21 @@ constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by t
 //   I1 fact resolution (id -> arena offset, length), I2 exclusive scan of lengths (b_i, m),
 //   I3 slot = block_table[pos / bs] * bs + pos % bs, validation, tile descriptors.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectParams p) {
-  __shared__ int32_t s_begin[kPlanMaxK];  // b_i: first composed token of placed fact i
-  __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
-  __shared__ int32_t s_scan[kPlanThreads / 32];
-  __shared__ int32_t s_carry, s_status;
-  __shared__ uint32_t s_tile_base;
+// Shared memory of one planning CTA: s_begin / s_src hold one entry per fact of the request (the caller sizes them).
+struct PlanShared {
+  int32_t scan[kPlanThreads / 32];
+  int32_t carry, status;
+  uint32_t tile_base;
+};
 
-  const int r = blockIdx.x;
+// Plans request r with the kPlanThreads threads of the calling CTA (all of them must call).
+__device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps) {
+  int32_t* const s_scan = ps.scan;
+  int32_t& s_carry = ps.carry;
+  int32_t& s_status = ps.status;
+  uint32_t& s_tile_base = ps.tile_base;
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
-  grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
   if (tid == 0) {
     *p.ctrl_next = InjectCtrl{0u, 0u, 0u, 0u};  // the counters the NEXT inject call will use
     s_carry = 0;
@@ -165,6 +169,14 @@ __global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectP
     if (p.out_n_tokens) p.out_n_tokens[r] = m;
     if (p.out_status) p.out_status[r] = s_status;
   }
+}
+
+__global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectParams p) {
+  __shared__ int32_t s_begin[kPlanMaxK];  // b_i: first composed token of placed fact i
+  __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
+  __shared__ PlanShared ps;
+  grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
+  plan_request(p, blockIdx.x, s_begin, s_src, ps);
 }
 
 // ------------------------------------------------------------------------------------------------

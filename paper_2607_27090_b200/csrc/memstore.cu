@@ -143,6 +143,8 @@ cudaError_t ensure_fused_smem(int device, size_t bytes) {
   if (bytes <= set_bytes[d]) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(score_topk_fused_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_plan_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_plan_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) set_bytes[d] = bytes;
   return e;
 }
@@ -601,16 +603,16 @@ ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int
   return mark_last(s, st);
 }
 
-ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
-                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
-                          int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
-                          uint32_t flags, ms_stream stream) {
-  if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::recursive_mutex> lock(s->mu);
+namespace {
+
+// Validation, scratch sizing and parameter block shared by memstore_inject and memstore_retrieve_inject.
+ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
+                         const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache, int32_t* out_n_tokens,
+                         int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags, InjectParams* out,
+                         int64_t* out_tiles_needed) {
   const memstore_config& c = s->cfg;
   if (nreq < 0 || k < 0 || k > kPlanMaxK) return fail(s, MS_ERR_INVALID_ARG, "nreq=%d k=%d (k <= %d)", nreq, k, kPlanMaxK);
   if (flags & ~(uint32_t)MS_INJECT_REVERSE) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
-  if (nreq == 0) return MS_OK;
   if (!start_pos || !block_tables || !cache || (k > 0 && !fact_ids) || max_blocks < 0)
     return fail(s, MS_ERR_INVALID_ARG, "null request arrays");
   if (!cache->k_base || !cache->v_base || cache->block_size <= 0 || cache->num_blocks <= 0)
@@ -621,8 +623,6 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     return fail(s, MS_ERR_INVALID_ARG, "cache bases must be 16-byte aligned and strides non-negative multiples of 8");
   if (out_slot_mapping && slot_stride < 0) return fail(s, MS_ERR_INVALID_ARG, "negative slot_stride");
   if (c.max_kv_tokens == 0 || !s->k_arena) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
-  DeviceGuard g(c.device);
-  cudaStream_t st = (cudaStream_t)stream;
 
   // upper bound on tiles: each request composes at most k * (longest fact) tokens, plus a ragged first tile
   const int64_t max_m = (int64_t)k * s->max_fact_len;
@@ -637,8 +637,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     MS_CUDA(s, cudaMalloc(&s->tiles, (size_t)tiles_needed * sizeof(TileDesc)));
     s->tiles_capacity = (uint32_t)tiles_needed;
   }
-  ms_status rc = order_after_last(s, st);
-  if (rc != MS_OK) return rc;
+  *out_tiles_needed = tiles_needed;
 
   InjectParams p{};
   p.facts = s->facts_d;
@@ -676,7 +675,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   p.ctrl = s->ctrl + (s->inject_calls & 1);
   p.ctrl_next = s->ctrl + ((s->inject_calls + 1) & 1);
 
-  // layers per work item: the largest power of two that still leaves every resident CTA about 16 items
+  // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
   const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
   const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
@@ -684,10 +683,15 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   int lpi = 1;
   while (lpi * 2 <= c.n_layers && c.n_layers % (lpi * 2) == 0 && est_tiles * (c.n_layers / (lpi * 2)) >= 16ll * resident_ctas) lpi *= 2;
   p.layers_per_item = lpi;
+  *out = p;
+  return MS_OK;
+}
 
-  inject_plan_kernel<<<nreq, kPlanThreads, 0, st>>>(p);
-  MS_CUDA(s, cudaGetLastError());
-
+// Launches the copy kernel as a programmatic dependent of the kernel that planned the request(s).
+ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* cache, int64_t tiles_needed, cudaStream_t st) {
+  const memstore_config& c = s->cfg;
+  const int row_bytes = c.n_kv_heads * c.head_dim * 2;
+  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
   cudaLaunchConfig_t lc{};
   lc.stream = st;
   cudaLaunchAttribute attr[1];
@@ -719,7 +723,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
     const int units = c.n_kv_heads * (c.head_dim / 16);
     const double mean_len = s->n_resident > 0 ? (double)s->kv_tokens_used / (double)s->n_resident : 0.0;
-    int64_t est_tiles_grid = (int64_t)(((double)k * mean_len / kTileTokens + 2.0) * nreq * 1.03) + 1;
+    int64_t est_tiles_grid = (int64_t)(((double)p.k * mean_len / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
     est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
     const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
     if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
@@ -732,13 +736,104 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
       e = cudaLaunchKernelEx(&lc, inject_copy_kernel<1>, p);
   }
   if (e != cudaSuccess) {
-    // the plan kernel has already counted tiles that no copy kernel will clear
+    // the plan has already counted tiles that no copy kernel will consume
     cudaMemsetAsync(s->ctrl, 0, 2 * sizeof(InjectCtrl), st);
     return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
   }
   if (prof) MS_CUDA(s, cudaEventRecord(s->prof_after, st));
-  s->kernels_launched += 2;
+  s->kernels_launched++;
   s->inject_calls++;
+  return MS_OK;
+}
+
+}  // namespace
+
+ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
+                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
+                          int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
+                          uint32_t flags, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  if (nreq == 0) return MS_OK;
+  DeviceGuard g(s->cfg.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  InjectParams p;
+  int64_t tiles_needed = 0;
+  ms_status rc = prepare_inject(s, fact_ids, nreq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
+                                out_slot_mapping, slot_stride, flags, &p, &tiles_needed);
+  if (rc != MS_OK) return rc;
+  rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+  inject_plan_kernel<<<nreq, kPlanThreads, 0, st>>>(p);
+  MS_CUDA(s, cudaGetLastError());
+  s->kernels_launched++;
+  rc = launch_copy(s, p, cache, tiles_needed, st);
+  if (rc != MS_OK) return rc;
+  return mark_last(s, st);
+}
+
+ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                                   const int32_t* start_pos, const int32_t* block_tables, int32_t max_blocks,
+                                   const ms_paged_cache* cache, int32_t* out_ids, float* out_scores, int32_t* out_n_tokens,
+                                   int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags,
+                                   ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (nq < 0 || k < 1 || k > kTopkMaxK) return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d (1 <= k <= %d)", nq, k, kTopkMaxK);
+  if (nq == 0) return MS_OK;
+  if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
+  if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
+  const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
+  if (n_max > kFusedMaxRows || nq > s->scores_nq) {
+    // large segments (or a first call that still has to size its scratch): the two calls one after the other
+    ms_status rc = memstore_retrieve(s, queries, query_users, nq, k, out_ids, out_scores, stream);
+    if (rc != MS_OK) return rc;
+    return memstore_inject(s, out_ids, nq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
+                           out_slot_mapping, slot_stride, flags, stream);
+  }
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  InjectParams ip;
+  int64_t tiles_needed = 0;
+  ms_status rc = prepare_inject(s, out_ids, nq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
+                                out_slot_mapping, slot_stride, flags, &ip, &tiles_needed);
+  if (rc != MS_OK) return rc;
+  rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+
+  RetrieveParams p{};
+  p.emb = s->emb;
+  p.emb_fact_id = s->emb_fact_id;
+  p.user_count = s->user_count_d;
+  p.seg_capacity = c.max_facts_per_user;
+  p.n_users = c.n_users;
+  p.emb_dim = c.emb_dim;
+  p.queries = queries;
+  p.query_users = query_users;
+  p.nq = nq;
+  p.k = k;
+  p.scores = s->scores;
+  p.score_stride = c.max_facts_per_user;
+  p.out_ids = out_ids;
+  p.out_scores = out_scores;
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
+  int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
+  rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
+  dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+  const int keys_cap = (int)std::max<int64_t>(n_max, 1);
+  const size_t smem = (size_t)keys_cap * sizeof(uint32_t);
+  const int n_host = query_users ? -1 : (int)n_max;
+  MS_CUDA(s, ensure_fused_smem(c.device, smem));
+  if (c.emb_dtype == MS_DTYPE_F16)
+    score_topk_plan_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host, ip);
+  else
+    score_topk_plan_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host, ip);
+  MS_CUDA(s, cudaGetLastError());
+  s->kernels_launched++;
+  s->retrieve_calls++;
+  rc = launch_copy(s, ip, cache, tiles_needed, st);
+  if (rc != MS_OK) return rc;
   return mark_last(s, st);
 }
 
@@ -779,10 +874,9 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
   MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, st));
   int32_t* d_hdr = reinterpret_cast<int32_t*>(d + q_bytes);
   int32_t* d_ids = reinterpret_cast<int32_t*>(d + in_bytes);
-  ms_status rc = memstore_retrieve(s, d, c.n_users > 1 ? d_hdr + 1 : nullptr, 1, k, d_ids, nullptr, stream);
-  if (rc != MS_OK) return rc;
-  rc = memstore_inject(s, d_ids, 1, k, d_hdr, reinterpret_cast<const int32_t*>(d + q_bytes + 16), max_blocks, cache, d_ids + k,
-                       d_ids + k + 1, nullptr, 0, flags, stream);
+  ms_status rc = memstore_retrieve_inject(s, d, c.n_users > 1 ? d_hdr + 1 : nullptr, 1, k, d_hdr,
+                                          reinterpret_cast<const int32_t*>(d + q_bytes + 16), max_blocks, cache, d_ids, nullptr,
+                                          d_ids + k, d_ids + k + 1, nullptr, 0, flags, stream);
   if (rc != MS_OK) return rc;
   MS_CUDA(s, cudaMemcpyAsync(h + in_bytes, d_ids, ((size_t)k + 2) * 4, cudaMemcpyDeviceToHost, st));
   MS_CUDA(s, cudaStreamSynchronize(st));

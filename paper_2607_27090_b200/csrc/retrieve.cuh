@@ -3,6 +3,7 @@
 // Paper: Sec. 3.2 (top-k search by embedding similarity returning fact ids; inner product, Sec. 6.1).
 #pragma once
 #include "common.cuh"
+#include "inject.cuh"
 
 namespace ms {
 
@@ -26,6 +27,8 @@ constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkMaxK = 2048;
 constexpr int kFusedMaxRows = 8192;  // largest segment whose top-k runs inside the scoring kernel
+static_assert(kScoreThreads == kPlanThreads, "the fused kernel plans with its own threads");
+static_assert(2 * kTopkMaxK * sizeof(int32_t) <= kTopkMaxK * sizeof(unsigned long long), "plan arrays reuse the candidate buffer");
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   const __half2* h = reinterpret_cast<const __half2*>(&v);
@@ -455,15 +458,13 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams
                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
 }
 
-// Scoring + top-k in ONE launch for segments of at most kFusedMaxRows rows: grid = (row groups, nq).
-// The CTA that finishes a query's scores last (a wait-free ticket) selects and sorts that query's top-k from
-// keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
-// of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
-template <typename T>
-__global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
-                                                                         uint32_t* tickets, int keys_capacity, int n_host) {
+// Body of the fused scoring + top-k kernels below (PLAN: the last CTA of a query also plans its injection).
+template <typename T, bool PLAN>
+__device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int rows_per_cta, uint32_t* tickets, int keys_capacity,
+                                                int n_host, const InjectParams* ip) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
+  __shared__ PlanShared ps;
   __shared__ int s_last;
   const int q = blockIdx.y;
   int user = 0, n = n_host;
@@ -498,6 +499,32 @@ __global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const R
                             IdMap{nullptr, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
+  if (PLAN) {
+    // the ids of query q are request q's fact list: plan it right here (steps I1-I3), in the shared memory the
+    // selection no longer needs, so that the copy kernel can follow without a separate planning launch
+    __syncthreads();
+    int32_t* s_begin = reinterpret_cast<int32_t*>(sm.cand);
+    plan_request(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
+  }
+}
+
+// Scoring + top-k in ONE launch for segments of at most kFusedMaxRows rows: grid = (row groups, nq).
+// The CTA that finishes a query's scores last (a wait-free ticket) selects and sorts that query's top-k from
+// keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
+// of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
+                                                                         uint32_t* tickets, int keys_capacity, int n_host) {
+  score_topk_body<T, false>(p, rows_per_cta, tickets, keys_capacity, n_host, nullptr);
+}
+
+// The same, and the last CTA of a query goes on to plan that query's injection request (memstore_retrieve_inject).
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
+                                                                        uint32_t* tickets, int keys_capacity, int n_host,
+                                                                        const __grid_constant__ InjectParams ip) {
+  grid_launch_dependents();  // the copy kernel may be scheduled early; it waits for this grid before reading the plan
+  score_topk_body<T, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip);
 }
 
 // ---- tensor-core path, steps 2 and 3 (step 1 is score_gemm_groupmax_kernel) -------------------------------------

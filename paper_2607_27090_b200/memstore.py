@@ -61,6 +61,7 @@ EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
+    "memstore_retrieve_inject",
 )  # fmt: skip
 
 _lib = None
@@ -94,6 +95,8 @@ def load_library() -> C.CDLL:
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.memstore_retrieve_static.restype = i32
     L.memstore_retrieve_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    L.memstore_retrieve_inject.restype = i32
+    L.memstore_retrieve_inject.argtypes = [vp, vp, vp, i32, i32, vp, vp, i32, C.POINTER(_PagedCache), vp, vp, vp, vp, vp, i64, u32, vp]
     L.memstore_serve_host.restype = i32
     L.memstore_serve_host.argtypes = [vp, vp, i32, i32, i32, vp, i32, C.POINTER(_PagedCache), u32, vp, vp, vp, vp]
     L.memstore_inject.restype = i32
@@ -297,6 +300,28 @@ class MemStore:
                                        flags, _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out_n_tokens, out_status
+
+    def retrieve_inject(self, queries, k, start_pos, block_tables, cache: PagedCache, query_users=None, out_ids=None,
+                        out_scores=None, out_n_tokens=None, out_status=None, out_slot_mapping=None, flags=0, stream=None):  # fmt: skip
+        """``retrieve`` then ``inject`` of every query's ids (query q = request q) in one call."""
+        nq = queries.shape[0]
+        dev = queries.device
+        if out_ids is None:
+            out_ids = torch.empty((nq, k), dtype=torch.int32, device=dev)
+        if out_n_tokens is None:
+            out_n_tokens = torch.empty(nq, dtype=torch.int32, device=dev)
+        if out_status is None:
+            out_status = torch.empty(nq, dtype=torch.int32, device=dev)
+        cs = cache._struct()
+        rc = self._lib.memstore_retrieve_inject(
+            self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"), _dev_ptr(query_users, torch.int32, "query_users"), nq,
+            k, _dev_ptr(start_pos, torch.int32, "start_pos"), _dev_ptr(block_tables, torch.int32, "block_tables"),
+            block_tables.shape[1], C.byref(cs), _dev_ptr(out_ids, torch.int32, "out_ids"),
+            _dev_ptr(out_scores, torch.float32, "out_scores"), _dev_ptr(out_n_tokens, torch.int32, "out_n_tokens"),
+            _dev_ptr(out_status, torch.int32, "out_status"), _dev_ptr(out_slot_mapping, torch.int64, "out_slot_mapping"),
+            out_slot_mapping.shape[1] if out_slot_mapping is not None else 0, flags, _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out_ids, out_n_tokens, out_status
 
     def serve_host(self, query, k, start_pos, block_table, cache: PagedCache, out, user=0, flags=0, stream=None):
         """One request from HOST buffers (numpy arrays or CPU tensors): ``query`` [emb_dim], ``block_table`` int32

@@ -229,6 +229,31 @@ def test_inject_empty_and_degenerate_requests():
     assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
 
 
+@pytest.mark.parametrize("n_users,nq", [(1, 1), (1, 5), (3, 7)])
+def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq):
+    """memstore_retrieve_inject (requests planned inside the retrieval kernel) against retrieve followed by inject."""
+    hs = HostStore(40, 90, 2, 8, 128, 8, 40, 256, "float16", n_users=n_users)
+    ms = hs.to_memstore(5e5)
+    bs, nb, k = 16, 256, 6
+    q = to_dev(synth.queries(41, nq, 256, "float16"))
+    users = to_dev((np.arange(nq) % n_users).astype(np.int32)) if n_users > 1 else None
+    starts = to_dev((np.arange(nq) * 5 + 3).astype(np.int32))
+    tables = to_dev(synth.block_tables(42, nb, (3 + 5 * nq + k * 40) // bs + 1, nq))
+    ca, cb = make_cache(hs, nb, bs), make_cache(hs, nb, bs)
+    for rep in range(2):  # the second round runs with the scratch already sized: the fused kernel path
+        ids_a, sc_a = ms.retrieve(q, k, query_users=users)
+        n_a, st_a = ms.inject(ids_a, starts, tables, ca, flags=M.INJECT_REVERSE)
+        sm = torch.full((nq, 300), -3, dtype=torch.int64, device=DEV)
+        sc_b = torch.empty((nq, k), dtype=torch.float32, device=DEV)
+        ids_b, n_b, st_b = ms.retrieve_inject(q, k, starts, tables, cb, query_users=users, out_scores=sc_b, out_slot_mapping=sm,
+                                              flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        assert torch.equal(ids_a, ids_b) and torch.equal(sc_a, sc_b) and torch.equal(n_a, n_b) and torch.equal(st_a, st_b)
+        assert int(st_b.abs().sum()) == 0 and bool((sm[:, 0] >= 0).all())
+        assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+    ms.close()
+
+
 def test_serve_host_matches_the_device_calls():
     """memstore_serve_host (host buffers in, host results out) against retrieve + inject on device buffers."""
     hs = HostStore(19, 120, 2, 8, 128, 8, 40, 256, "float16", n_users=2)
