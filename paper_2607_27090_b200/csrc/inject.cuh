@@ -50,7 +50,9 @@ constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by t
 //   I3 slot = block_table[pos / bs] * bs + pos % bs, validation, tile descriptors.
 // ------------------------------------------------------------------------------------------------
 // Shared memory of one planning CTA: s_begin / s_src hold one entry per fact of the request (the caller sizes them).
+constexpr int kPlanTableCache = 2048;  // block-table entries of a request kept in shared memory
 struct PlanShared {
+  int32_t table[kPlanTableCache];
   int32_t scan[kPlanThreads / 32];
   int32_t carry, status;
   uint32_t tile_base;
@@ -69,6 +71,11 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     s_carry = 0;
     s_status = 0;
   }
+  // the request's block-table row goes to shared memory in one coalesced sweep: the per-token lookups below would
+  // otherwise be a chain of dependent global loads
+  const int32_t* table_row = p.block_tables + (int64_t)r * p.max_blocks;
+  const int n_cached = min(p.max_blocks, kPlanTableCache);
+  for (int i = tid; i < n_cached; i += kPlanThreads) ps.table[i] = table_row[i];
   __syncthreads();
 
   // lengths of the facts in placement order, exclusive scan in chunks of kPlanThreads
@@ -144,7 +151,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
         if (bi >= p.max_blocks) {
           st = 4;  // MS_REQ_BLOCK_TABLE_SHORT
         } else {
-          int32_t blk = p.block_tables[(int64_t)r * p.max_blocks + bi];
+          const int32_t blk = bi < n_cached ? ps.table[bi] : table_row[bi];
           if (blk < 0 || blk >= p.num_blocks) {
             st = 8;  // MS_REQ_BAD_BLOCK_ID
           } else {

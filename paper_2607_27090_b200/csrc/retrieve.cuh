@@ -263,9 +263,13 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
       }
     }
     __syncthreads();
-    const uint32_t kmin = sm.kmin, range = sm.kmax - kmin;
-    const int sh = max(0, 24 - __clz(range));  // (range >> sh) < 256
-    for (int i = tid; i < n; i += THREADS) atomicAdd(&sm.hist[(key_at(i) - kmin) >> sh], 1u);
+    const uint32_t range = sm.kmax - sm.kmin;
+    // bucket of a score: linear in the VALUE between the smallest and the largest score (linear in the key would
+    // be logarithmic in the value and put a whole octave of top scores into one bucket); monotone in the score
+    const float smin = key_score(sm.kmin);
+    const float bscale = 255.5f / fmaxf(key_score(sm.kmax) - smin, 1e-30f);
+    auto bucket_of = [&](uint32_t kx) -> uint32_t { return min(255u, (uint32_t)((key_score(kx) - smin) * bscale)); };
+    for (int i = tid; i < n; i += THREADS) atomicAdd(&sm.hist[bucket_of(key_at(i))], 1u);
     __syncthreads();
     if (warp == 0) {
       uint32_t c[8], sum = 0;
@@ -302,14 +306,28 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
       __syncthreads();
       for (int i = tid; i < n; i += THREADS) {
         const uint32_t kx = key_at(i);
-        if (((kx - kmin) >> sh) >= B) {
+        if (bucket_of(kx) >= B) {
           const uint32_t slot = atomicAdd(&sm.ngt, 1u);
           sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
         }
       }
       __syncthreads();
+      if (n_cand * 4 <= (uint32_t)THREADS) {
+        // few candidates: the rank of a candidate is the number of larger ones (keys are distinct); no sorting
+        // network.  Four lanes share a candidate and split the comparisons.
+        const uint32_t ci = (uint32_t)tid >> 2, part = (uint32_t)tid & 3u;
+        const unsigned long long mine = ci < n_cand ? sm.cand[ci] : 0ull;
+        uint32_t rank = 0;
+        for (uint32_t jj = part; jj < n_cand; jj += 4) rank += sm.cand[jj] > mine;
+        rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+        rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+        if (ci < n_cand && part == 0 && rank < (uint32_t)k) {
+          out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+          if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+        }
+        return;
+      }
       if (n_cand <= (uint32_t)THREADS) {
-        // few candidates: the rank of a candidate is the number of larger ones (keys are distinct); no sorting network
         if (tid < (int)n_cand) {
           const unsigned long long mine = sm.cand[tid];
           uint32_t rank = 0;
