@@ -66,6 +66,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   uint32_t& s_tile_base = ps.tile_base;
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
+  const int32_t start = p.start_pos[r];  // issued first: its latency hides behind the scan
   if (tid == 0) {
     *p.ctrl_next = InjectCtrl{0u, 0u, 0u, 0u};  // the counters the NEXT inject call will use
     s_carry = 0;
@@ -120,12 +121,16 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     __syncthreads();
   }
   const int32_t m = s_carry;
-  const int32_t start = p.start_pos[r];
   const int32_t first_tile_pos = (start / kTileTokens) * kTileTokens;
   const uint32_t n_tiles = m > 0 ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
-  if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->n_tiles, n_tiles) : 0u;
-  __syncthreads();
-  const uint32_t tile_base = s_tile_base;
+  uint32_t tile_base = 0;
+  if (p.nreq == 1) {
+    if (tid == 0) p.ctrl->n_tiles = n_tiles;  // a single request owns the whole tile list: no ticket needed
+  } else {
+    if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->n_tiles, n_tiles) : 0u;
+    __syncthreads();
+    tile_base = s_tile_base;
+  }
 
   const int bs = p.block_size;
   for (uint32_t e = tid; e < n_tiles * kTileTokens; e += kPlanThreads) {

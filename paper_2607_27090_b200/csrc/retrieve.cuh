@@ -513,8 +513,9 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     hi = max(hi, kx);
   }
   __syncthreads();
+  // with a single user segment facts are numbered in row order: the row is the fact id
   topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k,
-                            IdMap{nullptr, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
+                            IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
   if (PLAN) {
