@@ -214,6 +214,26 @@ struct TopkShared {
 // the 64-bit key (score key << 32) | ~row.  `keys` (shared memory, optional) holds the n order keys;
 // without it they are recomputed from the scores in global memory on every pass.
 // ------------------------------------------------------------------------------------------------
+// Visits keys i = tid, tid + THREADS, ... < n, eight at a time: the eight loads are issued before any is used, so
+// that a pass over keys in global memory is not a chain of dependent round trips.
+template <int THREADS, class KeyAt, class Visit>
+__device__ __forceinline__ void for_each_key(int n, KeyAt key_at, Visit visit) {
+  const int tid = threadIdx.x;
+  for (int base = tid; base < n; base += THREADS * 8) {
+    uint32_t kx[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = base + u * THREADS;
+      if (i < n) kx[u] = key_at(i);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = base + u * THREADS;
+      if (i < n) visit(i, kx[u]);
+    }
+  }
+}
+
 template <int THREADS>
 __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const IdMap ids,
                            int32_t* out_ids, float* out_scores, bool have_minmax = false, uint32_t my_lo = 0xffffffffu,
@@ -232,11 +252,10 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   if (n > k) {
     uint32_t lo = my_lo, hi = my_hi;
     if (!have_minmax) {
-      for (int i = tid; i < n; i += THREADS) {
-        const uint32_t kx = key_at(i);
+      for_each_key<THREADS>(n, key_at, [&](int, uint32_t kx) {
         lo = min(lo, kx);
         hi = max(hi, kx);
-      }
+      });
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -264,38 +283,56 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
     }
     __syncthreads();
     const uint32_t range = sm.kmax - sm.kmin;
-    // bucket of a score: linear in the VALUE between the smallest and the largest score (linear in the key would
-    // be logarithmic in the value and put a whole octave of top scores into one bucket); monotone in the score
-    const float smin = key_score(sm.kmin);
-    const float bscale = 255.5f / fmaxf(key_score(sm.kmax) - smin, 1e-30f);
-    auto bucket_of = [&](uint32_t kx) -> uint32_t { return min(255u, (uint32_t)((key_score(kx) - smin) * bscale)); };
-    for (int i = tid; i < n; i += THREADS) atomicAdd(&sm.hist[bucket_of(key_at(i))], 1u);
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t c[8], sum = 0;
-#pragma unroll
-      for (int b = 0; b < 8; ++b) {
-        c[b] = sm.hist[8 * lane + b];
-        sum += c[b];
+    // bucket of a score: linear in the VALUE (linear in the key would be logarithmic in the value and put a whole
+    // octave of top scores into one bucket); monotone in the score.  With k much smaller than n only the upper part
+    // of the value range can hold the k-th largest, so the first attempt histograms the upper half alone (twice the
+    // resolution and a fraction of the shared-memory atomics); if fewer than k keys live there the whole range is used.
+    const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
+    float s_lo = 0.f, bscale = 0.f;
+    auto bucket_of = [&](uint32_t kx) -> uint32_t {  // 256 = below the histogrammed range
+      const float sv = key_score(kx);
+      return sv < s_lo ? 256u : min(255u, (uint32_t)((sv - s_lo) * bscale));
+    };
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      s_lo = attempt == 0 ? smin + 0.5f * (smax - smin) : smin;
+      bscale = 255.5f / fmaxf(smax - s_lo, 1e-30f);
+      if (attempt) {
+        for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
       }
-      uint32_t incl = sum;
+      if (tid == 0) sm.n_cand = 0xffffffffu;
+      __syncthreads();
+      for_each_key<THREADS>(n, key_at, [&](int, uint32_t kx) {
+        const uint32_t b = bucket_of(kx);
+        if (b < 256u) atomicAdd(&sm.hist[b], 1u);
+      });
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t c[8], sum = 0;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
-        if (lane + o < 32) incl += y;
-      }
-      uint32_t above = incl - sum;
-      if (above < (uint32_t)k && incl >= (uint32_t)k) {
-        int b = 7;
-        for (; b > 0; --b) {
-          if (above + c[b] >= (uint32_t)k) break;
-          above += c[b];
+        for (int b = 0; b < 8; ++b) {
+          c[b] = sm.hist[8 * lane + b];
+          sum += c[b];
         }
-        sm.bucket = 8 * lane + b;
-        sm.n_cand = above + c[b];
+        uint32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += y;
+        }
+        uint32_t above = incl - sum;
+        if (above < (uint32_t)k && incl >= (uint32_t)k) {
+          int b = 7;
+          for (; b > 0; --b) {
+            if (above + c[b] >= (uint32_t)k) break;
+            above += c[b];
+          }
+          sm.bucket = 8 * lane + b;
+          sm.n_cand = above + c[b];
+        }
       }
+      __syncthreads();
+      if (sm.n_cand != 0xffffffffu) break;  // the k-th largest lies in the histogrammed range
     }
-    __syncthreads();
     fast = range != 0 && sm.n_cand <= (uint32_t)kTopkMaxK;
     if (fast) {
       const uint32_t B = sm.bucket, n_cand = sm.n_cand;
@@ -304,13 +341,13 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
       if (tid == 0) sm.ngt = 0;
       for (int i = tid; i < P2; i += THREADS) sm.cand[i] = 0ull;
       __syncthreads();
-      for (int i = tid; i < n; i += THREADS) {
-        const uint32_t kx = key_at(i);
-        if (bucket_of(kx) >= B) {
+      for_each_key<THREADS>(n, key_at, [&](int i, uint32_t kx) {
+        const uint32_t b = bucket_of(kx);
+        if (b < 256u && b >= B) {  // 256 marks a key below the histogrammed range: never a candidate
           const uint32_t slot = atomicAdd(&sm.ngt, 1u);
-          sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+          if (slot < (uint32_t)kTopkMaxK) sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
         }
-      }
+      });
       __syncthreads();
       if (n_cand * 4 <= (uint32_t)THREADS) {
         // few candidates: the rank of a candidate is the number of larger ones (keys are distinct); no sorting
@@ -558,25 +595,19 @@ __global__ void __launch_bounds__(kTopkThreads) select_groups_kernel(const float
   int32_t* out = sel + (int64_t)q * k2;
   topk_block<kTopkThreads>(sm, gmax + (int64_t)q * gmax_stride, nullptr, n_groups, k2, IdMap{nullptr, nullptr}, out, nullptr);
   __syncthreads();
-  // sort the chosen group indices ascending (k2 <= 512; -1 padding becomes the largest key and stays last)
-  for (int i = threadIdx.x; i < 512; i += kTopkThreads) s_sel[i] = i < k2 ? out[i] : -1;
+  // order the chosen group indices ascending by counting (k2 <= 512 distinct indices; -1 padding, present only when
+  // the segment has fewer than k2 groups, counts as the largest value and keeps its relative order)
+  for (int i = threadIdx.x; i < k2; i += kTopkThreads) s_sel[i] = out[i];
   __syncthreads();
-  for (int size = 2; size <= 512; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int t = threadIdx.x; t < 256; t += kTopkThreads) {
-        const int lo = 2 * t - (t & (stride - 1));
-        const int hi = lo + stride;
-        const bool asc = (lo & size) == 0;
-        const uint32_t a = (uint32_t)s_sel[lo], b = (uint32_t)s_sel[hi];
-        if ((a > b) == asc) {
-          s_sel[lo] = (int32_t)b;
-          s_sel[hi] = (int32_t)a;
-        }
-      }
-      __syncthreads();
+  for (int i = threadIdx.x; i < k2; i += kTopkThreads) {
+    const uint32_t mine = (uint32_t)s_sel[i];
+    int rank = 0;
+    for (int j = 0; j < k2; ++j) {
+      const uint32_t other = (uint32_t)s_sel[j];
+      rank += (other < mine) || (other == mine && j < i);
     }
+    out[rank] = (int32_t)mine;
   }
-  for (int i = threadIdx.x; i < k2; i += kTopkThreads) out[i] = s_sel[i];
 }
 
 // One row's score with the lane layout and summation order of score_rows (all lanes return the sum).

@@ -45,6 +45,41 @@ def candidate_hot_ids(emb: np.ndarray, queries: np.ndarray, per_query: int, user
     return sorted(hot)
 
 
+def measure_retrieve_only(name: str, iters: int, seed: int = 0):
+    """Batched retrieval alone on an embedding-only store (no K/V, no cache): a few GB at most, for profiler captures."""
+    s = synth.CONFIGS[name]
+    dev = torch.device("cuda")
+    total = s.n_facts * s.n_users
+    emb = synth.embeddings(seed, total, s.emb_dim, s.emb_dtype)
+    queries = synth.queries(seed, s.nq, s.emb_dim, s.emb_dtype)
+    tdt = torch.float32 if s.emb_dtype == "float32" else torch.float16
+    store = M.MemStore(n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, emb_dim=s.emb_dim, emb_dtype=tdt,
+                       rope_theta=s.rope_theta, n_users=s.n_users, max_facts_per_user=s.n_facts, max_kv_tokens=0)  # fmt: skip
+    for u in range(s.n_users):
+        for a in range(u * s.n_facts, (u + 1) * s.n_facts, 65536):
+            b = min((u + 1) * s.n_facts, a + 65536)
+            store.add_facts(torch.from_numpy(emb[a:b]).to(dev), [0] * (b - a), user=u)
+    q_dev = torch.from_numpy(queries).to(dev)
+    u_dev = torch.arange(s.n_users, dtype=torch.int32, device=dev) if s.n_users > 1 else None
+    ids = torch.empty((s.nq, s.k), dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(2):
+        store.retrieve(q_dev, s.k, query_users=u_dev, out_ids=ids, want_scores=False, stream=stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(iters):
+        store.retrieve(q_dev, s.k, query_users=u_dev, out_ids=ids, want_scores=False, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / iters
+    line = {"config": name, "mode": "retrieve only", "queries_per_call": s.nq, "k": s.k, "facts_scanned": total,
+            "retrieve_us": us, "retrieve_emb_gbs": workload.emb_bytes_scanned(s, total) / (us * 1e-6) / 1e9,
+            "kernel_timeouts": store.stats()["kernel_timeouts"]}  # fmt: skip
+    store.close()
+    return line
+
+
 def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
     s = synth.CONFIGS[name]
     dev = torch.device("cuda")
@@ -122,5 +157,9 @@ if __name__ == "__main__":
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--hot-per-user", type=int, default=None)
     ap.add_argument("--pool-blocks", type=int, default=None)
+    ap.add_argument("--retrieve-only", action="store_true", help="embedding-only store, time the batched retrieval alone")
     a = ap.parse_args()
-    print(json.dumps(measure(a.config, a.iters, a.seed, a.hot_per_user, a.pool_blocks)))
+    if a.retrieve_only:
+        print(json.dumps(measure_retrieve_only(a.config, a.iters, a.seed)))
+    else:
+        print(json.dumps(measure(a.config, a.iters, a.seed, a.hot_per_user, a.pool_blocks)))
