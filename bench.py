@@ -108,6 +108,21 @@ class ClockSampler:
                 "samples": len(s)}  # fmt: skip
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """The slowest rank's figure (every multi-GPU time is the max over ranks).  Works on any initialised backend."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+THERMAL_REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
+
+
 # ---------------------------------------------------------------------------------------------- CPU oracle arm
 class OracleArm:
     """Times the CPU oracle, as it stands, on a bounded sample of one request of the workload and scales the
@@ -262,21 +277,26 @@ def run_ours(args):
         barrier()
         m_pool = n_tok.cpu().numpy().astype(np.int64)
 
-    launches0 = store.stats()["kernels_launched"]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clk:
-        barrier()
-        e0.record(stream)
-        for i in range(args.steps):
-            step(i)
-        e1.record(stream)
-        barrier()
-    ms_total = e0.elapsed_time(e1)
-    launches = store.stats()["kernels_launched"] - launches0
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t[0])
+    remeasured = False
+    while True:
+        launches0 = store.stats()["kernels_launched"]
+        with ClockSampler(local) as clk:
+            barrier()
+            e0.record(stream)
+            for i in range(args.steps):
+                step(i)
+            e1.record(stream)
+            barrier()
+        ms_total = e0.elapsed_time(e1)
+        launches = store.stats()["kernels_launched"] - launches0
+        throttled = max_over_ranks(float(any(r in clk.reasons for r in THERMAL_REASONS)), world, dev) > 0
+        if throttled and not remeasured:  # a thermally throttled run is rejected and measured once more
+            remeasured = True
+            time.sleep(2.0)
+            continue
+        break
+    ms_total = max_over_ranks(ms_total, world, dev)
     us_per_request = ms_total * 1e3 / (args.steps * world)
 
     # ---- per-part timing and the roofline of the dominant kernel (the copy kernel of inject) --------------
@@ -326,11 +346,7 @@ def run_ours(args):
         e2e_step(i)
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     e2e_us = e2e_ms * 1e3 / (n_e2e * world)
     h2d = ((q_host[0].numel() * q_host.element_size() + 15) // 16) * 16 + 16 + ((t_host[0].numel() * 4 + 15) // 16) * 16
     d2h = (k + 2) * 4
@@ -338,7 +354,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": us_per_request, "unit": "us", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 data, f32 arithmetic", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"{args.config}: {wl.lens.size} facts of {shape.len_lo}-{shape.len_hi} tokens, L={shape.n_layers} "
                         f"h={shape.n_kv_heads} d={shape.head_dim}, {shape.emb_dim}-d {shape.emb_dtype} embeddings, k={k}, "
@@ -346,7 +362,7 @@ def run_ours(args):
             "mean_tokens_per_request": mean_m, "bytes_per_request": bytes_step,
             "l2_policy": "inputs larger than L2: each request moves ~%.0f MB and rotates over %d queries / block tables"
                          % (bytes_step / 1e6, n_pool),
-            "replicas": world,
+            "replicas": world, "storage_dtype": "bf16 K/V, fp16 embeddings", "remeasured_after_throttle": remeasured,
         },
         "retrieve_us": float(np.median(retr_us)), "inject_copy_kernel_us": float(np.median(copy_us)),
         "path_gbs": bytes_step / (us_per_request * world * 1e-6) / 1e9,

@@ -1,0 +1,68 @@
+"""CPU-only checks of the benchmark's contract: the reference arm prints one JSON line with the agreed keys, under a
+two-rank launch only rank 0 works, and the max-over-ranks reduction used for every multi-GPU time works over gloo."""
+import json
+import os
+import subprocess
+import sys
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent.parent
+REQUIRED = {"metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+            "vs_baseline", "dtype", "data", "config", "impl", "cpu_baseline", "e2e"}  # fmt: skip
+
+
+def run(cmd, env=None):
+    e = dict(os.environ)
+    e.update(env or {})
+    e["OMP_NUM_THREADS"] = "2"
+    return subprocess.run(cmd, cwd=ROOT, env=e, capture_output=True, text=True, timeout=600)
+
+
+def test_reference_arm_prints_one_contract_line():
+    r = run([sys.executable, "bench.py", "--impl", "reference", "--steps", "2", "--warmup", "1", "--k", "5"])
+    assert r.returncode == 0, r.stderr
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert REQUIRED <= set(d) and d["impl"] == "reference" and d["higher_is_better"] is False and d["unit"] == "us"
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["value"] > 0
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["vs_baseline"] is None and "workload" in d["config"]
+
+
+def test_reference_arm_under_two_ranks_only_rank_zero_works():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", "29631", "bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--k", "5"]  # fmt: skip
+    r = run(cmd)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2
+
+
+def test_max_over_ranks_with_gloo_world_size_two():
+    code = (
+        "import os, sys, torch.distributed as dist\n"
+        "sys.path.insert(0, os.getcwd())\n"
+        "import bench\n"
+        "dist.init_process_group('gloo')\n"
+        "r = dist.get_rank()\n"
+        "v = bench.max_over_ranks(10.0 + 5.0 * r, dist.get_world_size())\n"
+        "assert v == 15.0, v\n"
+        "assert bench.max_over_ranks(float(r == 1), 2) == 1.0\n"
+        "dist.barrier(); dist.destroy_process_group()\n"
+        "print('rank', r, 'ok')\n"
+    )
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", "29632", "-c", code]  # fmt: skip
+    # torch.distributed.run needs a script path: write the snippet next to the test's temp dir
+    import tempfile
+
+    with tempfile.NamedTemporaryFile("w", suffix=".py", delete=False) as f:
+        f.write(code)
+        path = f.name
+    try:
+        cmd = cmd[:-2] + [path]
+        r = run(cmd)
+        assert r.returncode == 0, r.stderr[-2000:]
+        assert r.stdout.count("ok") == 2
+    finally:
+        os.unlink(path)
