@@ -53,12 +53,13 @@ constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by t
 constexpr int kPlanTableCache = 2048;  // block-table entries of a request kept in shared memory
 struct PlanShared {
   int32_t table[kPlanTableCache];
-  int32_t scan[kPlanThreads / 32];
+  int32_t scan[32];  // one partial sum per warp (up to 1024 threads)
   int32_t carry, status;
   uint32_t tile_base;
 };
 
-// Plans request r with the kPlanThreads threads of the calling CTA (all of them must call).
+// Plans request r with the THREADS threads of the calling CTA (all of them must call).
+template <int THREADS>
 __device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps) {
   int32_t* const s_scan = ps.scan;
   int32_t& s_carry = ps.carry;
@@ -76,12 +77,12 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   // otherwise be a chain of dependent global loads
   const int32_t* table_row = p.block_tables + (int64_t)r * p.max_blocks;
   const int n_cached = min(p.max_blocks, kPlanTableCache);
-  for (int i = tid; i < n_cached; i += kPlanThreads) ps.table[i] = table_row[i];
+  for (int i = tid; i < n_cached; i += THREADS) ps.table[i] = table_row[i];
   __syncthreads();
 
-  // lengths of the facts in placement order, exclusive scan in chunks of kPlanThreads
+  // lengths of the facts in placement order, exclusive scan in chunks of THREADS
   const int32_t* ids = p.fact_ids + (int64_t)r * p.k;
-  for (int base = 0; base < p.k; base += kPlanThreads) {
+  for (int base = 0; base < p.k; base += THREADS) {
     int j = base + tid;
     int32_t len = 0, src = 0;
     if (j < p.k) {
@@ -117,7 +118,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       s_src[j] = src;
     }
     __syncthreads();
-    if (tid == kPlanThreads - 1) s_carry = carry + warp_off + x;
+    if (tid == THREADS - 1) s_carry = carry + warp_off + x;
     __syncthreads();
   }
   const int32_t m = s_carry;
@@ -133,7 +134,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   }
 
   const int bs = p.block_size;
-  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += kPlanThreads) {
+  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += THREADS) {
     const uint32_t t = e / kTileTokens, ln = e % kTileTokens;
     const int32_t pos = first_tile_pos + (int32_t)e;
     const int32_t q = pos - start;  // index in the composed segment
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectP
   __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
   __shared__ PlanShared ps;
   grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
-  plan_request(p, blockIdx.x, s_begin, s_src, ps);
+  plan_request<kPlanThreads>(p, blockIdx.x, s_begin, s_src, ps);
 }
 
 // ------------------------------------------------------------------------------------------------

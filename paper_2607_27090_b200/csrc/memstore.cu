@@ -141,10 +141,13 @@ cudaError_t ensure_fused_smem(int device, size_t bytes) {
   std::lock_guard<std::mutex> lock(mu);
   const int d = device & 63;
   if (bytes <= set_bytes[d]) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(score_topk_fused_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_plan_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_plan_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  cudaError_t e = cudaSuccess;
+  const void* fns[] = {(const void*)score_topk_fused_kernel<__half, kFusedThreadsFew>, (const void*)score_topk_fused_kernel<float, kFusedThreadsFew>,
+                       (const void*)score_topk_fused_kernel<__half, kFusedThreadsMany>, (const void*)score_topk_fused_kernel<float, kFusedThreadsMany>,
+                       (const void*)score_topk_plan_kernel<__half, kFusedThreadsFew>, (const void*)score_topk_plan_kernel<float, kFusedThreadsFew>,
+                       (const void*)score_topk_plan_kernel<__half, kFusedThreadsMany>, (const void*)score_topk_plan_kernel<float, kFusedThreadsMany>};
+  for (const void* fn : fns)
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) set_bytes[d] = bytes;
   return e;
 }
@@ -219,6 +222,32 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     s->kernels_launched += 3;
   }
   return MS_OK;
+}
+
+// Launch of the one-launch scoring + top-k (+ plan) kernels: 1024-thread CTAs when few queries are served (the last
+// CTA of a query selects and plans alone, which wants many threads), 256-thread CTAs otherwise.
+template <typename T, int THREADS, bool PLAN>
+void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,
+                               const InjectParams* ip, size_t smem, cudaStream_t st) {
+  // enough CTAs to fill the GPU, at least one row per warp
+  constexpr int64_t kWarps = THREADS / 32;
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * 8 / nq);
+  int64_t rows = std::max<int64_t>(kWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
+  rows = (rows + kWarps - 1) / kWarps * kWarps;
+  const int rows_per_cta = (int)rows;
+  const dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
+  if constexpr (PLAN)
+    score_topk_plan_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host, *ip);
+  else
+    score_topk_fused_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host);
+}
+template <typename T, bool PLAN>
+void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,
+                       const InjectParams* ip, size_t smem, cudaStream_t st) {
+  if (nq <= kFusedFewQueries)
+    launch_score_topk_threads<T, kFusedThreadsFew, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st);
+  else
+    launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st);
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -487,9 +516,9 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
     const int n_host = query_users ? -1 : (int)n_max;
     MS_CUDA(s, ensure_fused_smem(c.device, smem));
     if (c.emb_dtype == MS_DTYPE_F16)
-      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host);
+      launch_score_topk<__half, false>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, nullptr, smem, st);
     else
-      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host);
+      launch_score_topk<float, false>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, nullptr, smem, st);
     MS_CUDA(s, cudaGetLastError());
     s->kernels_launched++;
   } else {
@@ -583,9 +612,9 @@ ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int
     const int n_host = query_users ? -1 : (int)n_max;
     MS_CUDA(s, ensure_fused_smem(c.device, smem));  // a function attribute, not an allocation
     if (c.emb_dtype == MS_DTYPE_F16)
-      score_topk_fused_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap, n_host);
+      launch_score_topk<__half, false>(s->sm_count, nq, n_max, p, tickets, keys_cap, n_host, nullptr, smem, st);
     else
-      score_topk_fused_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, tickets, keys_cap, n_host);
+      launch_score_topk<float, false>(s->sm_count, nq, n_max, p, tickets, keys_cap, n_host, nullptr, smem, st);
     MS_CUDA(s, cudaGetLastError());
     s->kernels_launched++;
   } else {
@@ -817,18 +846,14 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   p.score_stride = c.max_facts_per_user;
   p.out_ids = out_ids;
   p.out_scores = out_scores;
-  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
-  int64_t rows_per_cta = std::max<int64_t>(kScoreWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
-  rows_per_cta = (rows_per_cta + kScoreWarps - 1) / kScoreWarps * kScoreWarps;
-  dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
   const int keys_cap = (int)std::max<int64_t>(n_max, 1);
   const size_t smem = (size_t)keys_cap * sizeof(uint32_t);
   const int n_host = query_users ? -1 : (int)n_max;
   MS_CUDA(s, ensure_fused_smem(c.device, smem));
   if (c.emb_dtype == MS_DTYPE_F16)
-    score_topk_plan_kernel<__half><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host, ip);
+    launch_score_topk<__half, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st);
   else
-    score_topk_plan_kernel<float><<<grid, kScoreThreads, smem, st>>>(p, (int)rows_per_cta, s->tickets, keys_cap, n_host, ip);
+    launch_score_topk<float, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st);
   MS_CUDA(s, cudaGetLastError());
   s->kernels_launched++;
   s->retrieve_calls++;

@@ -27,7 +27,9 @@ constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkMaxK = 2048;
 constexpr int kFusedMaxRows = 8192;  // largest segment whose top-k runs inside the scoring kernel
-static_assert(kScoreThreads == kPlanThreads, "the fused kernel plans with its own threads");
+// CTA size of the one-launch scoring + top-k (+ plan) kernels: the last CTA of a query does the selection and the
+// planning alone, which want many threads when there are few queries; with many queries smaller CTAs fill the GPU better
+constexpr int kFusedThreadsFew = 1024, kFusedThreadsMany = 256, kFusedFewQueries = 8;
 static_assert(2 * kTopkMaxK * sizeof(int32_t) <= kTopkMaxK * sizeof(unsigned long long), "plan arrays reuse the candidate buffer");
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
@@ -101,7 +103,7 @@ __device__ __forceinline__ void score_rows(const RetrieveParams& p, const float*
 // The same scoring with the query read straight from global memory (through L1) next to the row, so that one
 // memory round trip serves both and no shared-memory staging or barrier is needed.  Same lane layout and
 // summation order as score_rows.
-template <typename T>
+template <typename T, int WARPS>
 __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q, int user, int n, int64_t row0, int rows_per_cta) {
   constexpr int VEC = 16 / sizeof(T);
   const int E = p.emb_dim;
@@ -110,7 +112,7 @@ __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q
   const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
   const int64_t row_end = min(row0 + rows_per_cta, (int64_t)n);
   const int nvec = E / VEC;
-  for (int64_t row = row0 + warp; row < row_end; row += kScoreWarps) {
+  for (int64_t row = row0 + warp; row < row_end; row += WARPS) {
     const uint4* rp = reinterpret_cast<const uint4*>(seg + row * E);
     float acc = 0.f;
     for (int v0 = 0; v0 < nvec; v0 += 128) {
@@ -514,7 +516,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams
 }
 
 // Body of the fused scoring + top-k kernels below (PLAN: the last CTA of a query also plans its injection).
-template <typename T, bool PLAN>
+template <typename T, int THREADS, bool PLAN>
 __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int rows_per_cta, uint32_t* tickets, int keys_capacity,
                                                 int n_host, const InjectParams* ip) {
   extern __shared__ uint32_t s_keys[];
@@ -530,7 +532,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     n = user_ok ? min(p.user_count[user], keys_capacity) : 0;
   }
   const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
-  if (row0 < n) score_rows_direct<T>(p, q, user, n, row0, rows_per_cta);
+  if (row0 < n) score_rows_direct<T, THREADS / 32>(p, q, user, n, row0, rows_per_cta);
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();  // this CTA's scores are visible before its ticket is
@@ -543,7 +545,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   __threadfence();
   const float* sc = p.scores + (int64_t)q * p.score_stride;
   uint32_t lo = 0xffffffffu, hi = 0u;
-  for (int i = threadIdx.x; i < n; i += kScoreThreads) {
+  for (int i = threadIdx.x; i < n; i += THREADS) {
     const uint32_t kx = order_key(__ldcg(sc + i));
     s_keys[i] = kx;
     lo = min(lo, kx);
@@ -551,7 +553,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   }
   __syncthreads();
   // with a single user segment facts are numbered in row order: the row is the fact id
-  topk_block<kScoreThreads>(sm, sc, s_keys, n, p.k,
+  topk_block<THREADS>(sm, sc, s_keys, n, p.k,
                             IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
@@ -560,7 +562,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     // selection no longer needs, so that the copy kernel can follow without a separate planning launch
     __syncthreads();
     int32_t* s_begin = reinterpret_cast<int32_t*>(sm.cand);
-    plan_request(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
+    plan_request<THREADS>(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
   }
 }
 
@@ -568,19 +570,19 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
 // The CTA that finishes a query's scores last (a wait-free ticket) selects and sorts that query's top-k from
 // keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
 // of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
-template <typename T>
-__global__ void __launch_bounds__(kScoreThreads) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
                                                                          uint32_t* tickets, int keys_capacity, int n_host) {
-  score_topk_body<T, false>(p, rows_per_cta, tickets, keys_capacity, n_host, nullptr);
+  score_topk_body<T, THREADS, false>(p, rows_per_cta, tickets, keys_capacity, n_host, nullptr);
 }
 
 // The same, and the last CTA of a query goes on to plan that query's injection request (memstore_retrieve_inject).
-template <typename T>
-__global__ void __launch_bounds__(kScoreThreads) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
                                                                         uint32_t* tickets, int keys_capacity, int n_host,
                                                                         const __grid_constant__ InjectParams ip) {
   grid_launch_dependents();  // the copy kernel may be scheduled early; it waits for this grid before reading the plan
-  score_topk_body<T, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip);
+  score_topk_body<T, THREADS, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip);
 }
 
 // ---- tensor-core path, steps 2 and 3 (step 1 is score_gemm_groupmax_kernel) -------------------------------------
