@@ -88,6 +88,7 @@ typedef struct {
   int64_t max_kv_tokens;  /* capacity of the K/V arena in tokens (0: embedding-only store) */
   void* kv_arena;         /* optional caller-provided DEVICE buffer for the arena, else NULL */
   size_t kv_arena_bytes;  /* its size; must be >= memstore_arena_bytes(config) */
+  int64_t max_host_kv_tokens; /* capacity in tokens of the second K/V arena in pinned HOST memory (0: none), < 2^30 */
 } memstore_config;
 
 /* Bytes of the K/V arena for this configuration: 2 * L * max_kv_tokens * h * d * 2
@@ -122,6 +123,16 @@ ms_status memstore_add_fact(memstore_t* store, int32_t user, const void* emb, co
  */
 ms_status memstore_add_facts(memstore_t* store, int32_t user, int64_t n, const void* embs, const void* k_pre,
                              const void* v, const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream);
+
+/*
+ * Append n facts whose K/V stay in HOST memory (the paper's CPU-offloaded store, Sec. 6.8: the KV store moves to
+ * pinned host DRAM and retrieved facts are streamed over PCIe).  Same arguments as memstore_add_facts except that
+ * k_pre and v are HOST pointers; embs is still a device pointer (retrieval always runs from HBM).  The rows are copied
+ * into the store's pinned host arena (capacity max_host_kv_tokens) before the call returns.  memstore_inject reads the
+ * rows of such facts directly over PCIe inside the same copy kernel; a request may mix facts of both tiers.
+ */
+ms_status memstore_add_facts_host(memstore_t* store, int32_t user, int64_t n, const void* embs, const void* k_pre_host,
+                                  const void* v_host, const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream);
 
 /*
  * Score each query against every fact of its user by inner product and select the k best
@@ -234,6 +245,7 @@ typedef struct {
   int64_t retrieve_calls, inject_calls;
   int64_t kernels_launched; /* kernels of this library enqueued so far */
   int64_t arena_bytes, embedding_bytes;
+  int64_t host_kv_tokens_used;
   int64_t kernel_timeouts; /* 1 if a bounded wait inside the tensor-core scoring kernel ever ran out (results of that call are invalid) */
 } memstore_stats_t;
 ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);

@@ -13,12 +13,16 @@ struct FactRec {
   int32_t tok_off;   // first token of the fact in the K/V arena
   int32_t n_tokens;  // length of the fact in tokens
   int32_t user;      // owner segment
-  int32_t resident;  // 1: K/V present in the arena, 0: embedding only
+  int32_t resident;  // 0: embedding only, 1: K/V in the HBM arena, 2: K/V in the pinned host arena
 };
 
 // Tokens per injection tile: 8 consecutive positions aligned to a multiple of 8, so a tile never
 // straddles a cache block whose size is a multiple of 8 (and covers whole smaller power-of-two blocks).
 constexpr int kTileTokens = 8;
+
+// A source token index with this bit set lives in the pinned host arena (the paper's CPU-offloaded store, Sec. 6.8)
+// and is read over PCIe by the copy kernel; both arenas hold fewer than 2^30 tokens.
+constexpr int32_t kHostTierBit = 0x40000000;
 
 // Work description of one tile, written by the plan kernel and read by the copy kernel.
 struct __align__(16) TileDesc {

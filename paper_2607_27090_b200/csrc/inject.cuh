@@ -13,6 +13,9 @@ struct InjectParams {
   const __nv_bfloat16* k_arena;  // [L][arena_tokens][H][D]
   const __nv_bfloat16* v_arena;
   int64_t arena_tokens;
+  const __nv_bfloat16* k_host;  // pinned host arena as seen from the device, [L][host_tokens][H][D], or nullptr
+  const __nv_bfloat16* v_host;
+  int64_t host_tokens;
   const float* inv_freq;  // [D/2]
   int32_t n_layers, n_heads, head_dim, rope_style;
   int32_t max_position;
@@ -96,7 +99,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
             atomicOr(&s_status, 2 /*MS_REQ_NOT_RESIDENT*/);
           } else {
             len = f.n_tokens;
-            src = f.tok_off;
+            src = f.resident == 2 ? (f.tok_off | kHostTierBit) : f.tok_off;
           }
         }
       }
@@ -295,9 +298,11 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
     const int64_t dst = d->dst_off[tk];
     const int32_t pos = d->pos0 + tk;
 
-    const int64_t src_row = ((int64_t)layer * p.arena_tokens + src) * (int64_t)(p.n_heads * D);
-    const __nv_bfloat16* ks = p.k_arena + src_row;
-    const __nv_bfloat16* vs = p.v_arena + src_row;
+    // source rows: the HBM arena, or (host tier) the pinned host arena read straight over PCIe
+    const bool host = (src & kHostTierBit) != 0;
+    const int64_t src_row = ((int64_t)layer * (host ? p.host_tokens : p.arena_tokens) + (src & ~kHostTierBit)) * (int64_t)(p.n_heads * D);
+    const __nv_bfloat16* ks = (host ? p.k_host : p.k_arena) + src_row;
+    const __nv_bfloat16* vs = (host ? p.v_host : p.v_arena) + src_row;
     const int64_t dbase = (int64_t)layer * p.layer_stride + dst;
     uint4 ka[kUnitsPerThread], kb[kUnitsPerThread], va[kUnitsPerThread], vb[kUnitsPerThread];
 #pragma unroll

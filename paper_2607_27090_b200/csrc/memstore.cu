@@ -27,6 +27,12 @@ struct memstore {
   __nv_bfloat16* k_arena = nullptr;  // [L][max_kv_tokens][h][d]
   __nv_bfloat16* v_arena = nullptr;
   void* arena_alloc = nullptr;       // non-null when the store owns the arena
+  __nv_bfloat16* k_host = nullptr;   // pinned host arena [L][max_host_kv_tokens][h][d] (K then V), host address
+  __nv_bfloat16* v_host = nullptr;
+  __nv_bfloat16* k_host_dev = nullptr;  // the same memory as the device sees it
+  __nv_bfloat16* v_host_dev = nullptr;
+  void* host_arena_alloc = nullptr;
+  int64_t host_tokens_used = 0;
   void* emb = nullptr;               // [n_users][max_facts_per_user][emb_dim]
   int32_t* emb_fact_id = nullptr;    // [n_users][max_facts_per_user]
   int32_t* user_count_d = nullptr;   // [n_users]
@@ -116,7 +122,7 @@ ms_status check_config(const memstore_config* c) {
   // the copy kernels give 32 or more threads to a token and one frequency octet to a thread: d/16 must divide 32
   const int d = c->head_dim;
   if (!(d == 16 || d == 32 || d == 64 || d == 128 || d == 256)) return MS_ERR_UNSUPPORTED;
-  if (c->max_kv_tokens >= (1ll << 31) || (int64_t)c->n_users * c->max_facts_per_user >= (1ll << 31))
+  if (c->max_host_kv_tokens < 0 || c->max_host_kv_tokens >= (1ll << 30) || c->max_kv_tokens >= (1ll << 30) || (int64_t)c->n_users * c->max_facts_per_user >= (1ll << 31))
     return MS_ERR_UNSUPPORTED;
   return MS_OK;
 }
@@ -309,6 +315,19 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
     s->k_arena = (__nv_bfloat16*)s->arena_alloc;
   }
   s->v_arena = s->k_arena ? (__nv_bfloat16*)((char*)s->k_arena + arena_bytes / 2) : nullptr;
+  if (config->max_host_kv_tokens > 0) {
+    const size_t half = (size_t)config->n_layers * (size_t)config->max_host_kv_tokens * config->n_kv_heads * config->head_dim * sizeof(__nv_bfloat16);
+    void* dptr = nullptr;
+    if (cudaHostAlloc(&s->host_arena_alloc, 2 * half, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess ||
+        cudaHostGetDevicePointer(&dptr, s->host_arena_alloc, 0) != cudaSuccess) {
+      cudaGetLastError();
+      return bail(MS_ERR_OOM);
+    }
+    s->k_host = (__nv_bfloat16*)s->host_arena_alloc;
+    s->v_host = (__nv_bfloat16*)((char*)s->host_arena_alloc + half);
+    s->k_host_dev = (__nv_bfloat16*)dptr;
+    s->v_host_dev = (__nv_bfloat16*)((char*)dptr + half);
+  }
 
   const int64_t rows = (int64_t)config->n_users * config->max_facts_per_user;
   const size_t esz = emb_elem_size(config->emb_dtype);
@@ -336,7 +355,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
     return bail(MS_ERR_CUDA);
   }
   s->user_count.assign(config->n_users, 0);
-  s->tma_path = (config->flags & MS_STORE_TMA_COPY_PATH) != 0;
+  s->tma_path = (config->flags & MS_STORE_TMA_COPY_PATH) != 0 && config->max_host_kv_tokens == 0;  // HBM arena only
   int occ = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0>, kCopyThreads, 0) == cudaSuccess && occ > 0)
     s->copy_ctas_per_sm = occ;
@@ -355,6 +374,7 @@ ms_status memstore_destroy(memstore_t* s) {
     DeviceGuard g(s->cfg.device);
     cudaDeviceSynchronize();
     cudaFree(s->arena_alloc);
+    if (s->host_arena_alloc) cudaFreeHost(s->host_arena_alloc);
     cudaFree(s->emb);
     cudaFree(s->emb_fact_id);
     cudaFree(s->facts_d);
@@ -379,8 +399,9 @@ ms_status memstore_destroy(memstore_t* s) {
   return MS_OK;
 }
 
-ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
-                             const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+// tier 1: k_pre / v are device buffers appended to the HBM arena; tier 2: host buffers copied into the pinned host arena
+static ms_status add_facts_tier(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
+                                const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream, int tier) {
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -396,14 +417,17 @@ ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void*
     T += n_tokens[i];
   }
   if (T > 0 && (!k_pre || !v)) return fail(s, MS_ERR_INVALID_ARG, "null K/V for %lld tokens", (long long)T);
-  if (((uintptr_t)embs & 15) || ((uintptr_t)k_pre & 15) || ((uintptr_t)v & 15))
+  if (((uintptr_t)embs & 15) || (tier == 1 && (((uintptr_t)k_pre & 15) || ((uintptr_t)v & 15))))
     return fail(s, MS_ERR_INVALID_ARG, "device buffers must be 16-byte aligned");
   if (s->user_count[user] + n > c.max_facts_per_user)
     return fail(s, MS_ERR_CAPACITY, "user %d segment full (%lld + %lld > %lld)", user, (long long)s->user_count[user],
                 (long long)n, (long long)c.max_facts_per_user);
-  if (s->kv_tokens_used + T > c.max_kv_tokens)
+  if (tier == 1 && s->kv_tokens_used + T > c.max_kv_tokens)
     return fail(s, MS_ERR_CAPACITY, "K/V arena full (%lld + %lld > %lld tokens)", (long long)s->kv_tokens_used,
                 (long long)T, (long long)c.max_kv_tokens);
+  if (tier == 2 && s->host_tokens_used + T > c.max_host_kv_tokens)
+    return fail(s, MS_ERR_CAPACITY, "host K/V arena full (%lld + %lld > %lld tokens)", (long long)s->host_tokens_used,
+                (long long)T, (long long)c.max_host_kv_tokens);
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
   const int64_t slot0 = s->user_count[user];
@@ -412,11 +436,11 @@ ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void*
 
   std::vector<FactRec> recs(n);
   std::vector<int32_t> ids(n);
-  int64_t off = s->kv_tokens_used;
+  int64_t off = tier == 1 ? s->kv_tokens_used : s->host_tokens_used;
   int64_t resident = 0;
   int32_t max_len = s->max_fact_len;
   for (int64_t i = 0; i < n; ++i) {
-    recs[i] = FactRec{(int32_t)off, n_tokens[i], user, n_tokens[i] > 0 ? 1 : 0};
+    recs[i] = FactRec{(int32_t)off, n_tokens[i], user, n_tokens[i] > 0 ? tier : 0};
     ids[i] = (int32_t)(s->n_facts + i);
     off += n_tokens[i];
     resident += n_tokens[i] > 0;
@@ -429,7 +453,15 @@ ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void*
   MS_CUDA(s, cudaMemcpyAsync(s->facts_d + s->n_facts, recs.data(), (size_t)n * sizeof(FactRec), cudaMemcpyHostToDevice, st));
   MS_CUDA(s, cudaMemcpyAsync(s->emb_fact_id + row0, ids.data(), (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
   MS_CUDA(s, cudaMemcpyAsync(s->user_count_d + user, &new_count, sizeof(int32_t), cudaMemcpyHostToDevice, st));
-  if (T > 0) {
+  if (T > 0 && tier == 2) {
+    // host tier: plain host copies, layer by layer, into the pinned arena (visible to later kernels as is)
+    const size_t row = (size_t)c.n_kv_heads * c.head_dim * sizeof(__nv_bfloat16);
+    for (int l = 0; l < c.n_layers; ++l) {
+      const size_t dst = ((size_t)l * c.max_host_kv_tokens + s->host_tokens_used) * row;
+      memcpy((char*)s->k_host + dst, (const char*)k_pre + (size_t)l * T * row, (size_t)T * row);
+      memcpy((char*)s->v_host + dst, (const char*)v + (size_t)l * T * row, (size_t)T * row);
+    }
+  } else if (T > 0) {
     const int64_t row_vec = (int64_t)c.n_kv_heads * c.head_dim * 2 / 16;
     const int64_t src_vec = T * row_vec;
     int gx = (int)std::min<int64_t>((src_vec + 255) / 256, 4 * s->sm_count);
@@ -444,9 +476,20 @@ ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void*
   if (s->user_count[user] > s->max_user_count) s->max_user_count = s->user_count[user];
   s->n_facts += n;
   s->n_resident += resident;
-  s->kv_tokens_used += T;
+  if (tier == 1) s->kv_tokens_used += T; else s->host_tokens_used += T;
   s->max_fact_len = max_len;
   return MS_OK;
+}
+
+ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
+                             const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+  return add_facts_tier(s, user, n, embs, k_pre, v, n_tokens, out_first_id, stream, 1);
+}
+
+ms_status memstore_add_facts_host(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre_host,
+                                  const void* v_host, const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+  if (s && s->cfg.max_host_kv_tokens == 0) return fail(s, MS_ERR_INVALID_ARG, "store was created without a host K/V arena");
+  return add_facts_tier(s, user, n, embs, k_pre_host, v_host, n_tokens, out_first_id, stream, 2);
 }
 
 ms_status memstore_add_fact(memstore_t* s, int32_t user, const void* emb, const void* k_pre, const void* v,
@@ -651,7 +694,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
       cache->block_stride < 0 || cache->token_stride < 0 || cache->head_stride < 0)
     return fail(s, MS_ERR_INVALID_ARG, "cache bases must be 16-byte aligned and strides non-negative multiples of 8");
   if (out_slot_mapping && slot_stride < 0) return fail(s, MS_ERR_INVALID_ARG, "negative slot_stride");
-  if (c.max_kv_tokens == 0 || !s->k_arena) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
+  if ((c.max_kv_tokens == 0 || !s->k_arena) && !s->k_host) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
 
   // upper bound on tiles: each request composes at most k * (longest fact) tokens, plus a ragged first tile
   const int64_t max_m = (int64_t)k * s->max_fact_len;
@@ -674,6 +717,9 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.k_arena = s->k_arena;
   p.v_arena = s->v_arena;
   p.arena_tokens = c.max_kv_tokens;
+  p.k_host = s->k_host_dev;
+  p.v_host = s->v_host_dev;
+  p.host_tokens = c.max_host_kv_tokens;
   p.inv_freq = s->inv_freq_d;
   p.n_layers = c.n_layers;
   p.n_heads = c.n_kv_heads;
@@ -751,7 +797,7 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
     // from the mean length of the resident facts (plus a ragged tile per request and 3 %); the kernel's
     // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
     const int units = c.n_kv_heads * (c.head_dim / 16);
-    const double mean_len = s->n_resident > 0 ? (double)s->kv_tokens_used / (double)s->n_resident : 0.0;
+    const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used + s->host_tokens_used) / (double)s->n_resident : 0.0;
     int64_t est_tiles_grid = (int64_t)(((double)p.k * mean_len / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
     est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
     const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
@@ -918,6 +964,7 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->n_facts = s->n_facts;
   out->n_resident_facts = s->n_resident;
   out->kv_tokens_used = s->kv_tokens_used;
+  out->host_kv_tokens_used = s->host_tokens_used;
   out->retrieve_calls = s->retrieve_calls;
   out->inject_calls = s->inject_calls;
   out->kernels_launched = s->kernels_launched;

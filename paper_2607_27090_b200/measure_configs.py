@@ -80,6 +80,53 @@ def measure_retrieve_only(name: str, iters: int, seed: int = 0):
     return line
 
 
+def measure_host_tier(iters: int, seed: int = 0, n_facts: int = 400, ks=(5, 10, 20, 50)):
+    """The Llama-3.1-8B KV shape with every fact's K/V in the pinned host arena (the CPU-offloaded store): injection
+    of k facts read over PCIe by the copy kernel.  A shrunken store (n_facts) keeps the pinned allocation near 2 GB."""
+    s = synth.CONFIGS["llama8b"]
+    dev = torch.device("cuda")
+    lens = synth.fact_lengths(seed, n_facts, s.len_lo, s.len_hi)
+    emb = synth.embeddings(seed, n_facts, s.emb_dim, s.emb_dtype)
+    T = int(lens.sum())
+    store = M.MemStore(n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, emb_dim=s.emb_dim,
+                       rope_theta=s.rope_theta, max_facts_per_user=n_facts, max_kv_tokens=0, max_host_kv_tokens=T)  # fmt: skip
+    g = torch.Generator().manual_seed(seed)
+    for a in range(0, n_facts, 50):
+        b = min(n_facts, a + 50)
+        t = int(lens[a:b].sum())
+        kv = torch.randn((2, s.n_layers, t, s.n_kv_heads, s.head_dim), generator=g, dtype=torch.float32).to(torch.bfloat16)
+        store.add_facts_host(torch.from_numpy(emb[a:b]).to(dev), lens[a:b], kv[0].contiguous(), kv[1].contiguous())
+    lines = []
+    rng = np.random.default_rng(seed)
+    for k in ks:
+        per_req = workload.blocks_per_request(s, k)
+        cache = M.PagedCache.allocate(s.n_layers, max(1024, per_req * 4), s.block_size, s.n_kv_heads, s.head_dim, dev)
+        tables = torch.from_numpy(synth.block_tables(seed, cache.num_blocks, per_req, 4)).to(dev)
+        ids = torch.from_numpy(np.stack([rng.choice(n_facts, k, replace=False) for _ in range(4)]).astype(np.int32)).to(dev)
+        start = torch.full((1,), s.start_pos, dtype=torch.int32, device=dev)
+        n_tok = torch.zeros(1, dtype=torch.int32, device=dev)
+        stream = torch.cuda.current_stream()
+        for i in range(3):
+            store.inject(ids[i % 4 : i % 4 + 1], start, tables[i % 4 : i % 4 + 1], cache, out_n_tokens=n_tok, stream=stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m_sum = 0
+        e0.record(stream)
+        for i in range(iters):
+            store.inject(ids[i % 4 : i % 4 + 1], start, tables[i % 4 : i % 4 + 1], cache, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        for i in range(4):
+            m_sum += int(lens[ids[i].cpu().numpy()].sum())
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        m = m_sum / 4
+        lines.append({"config": "llama8b host tier", "k": k, "tokens": m, "inject_us": us,
+                      "pcie_read_gbs": m * s.token_bytes / (us * 1e-6) / 1e9})  # fmt: skip
+        del cache
+    store.close()
+    return lines
+
+
 def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
     s = synth.CONFIGS[name]
     dev = torch.device("cuda")
@@ -158,8 +205,12 @@ if __name__ == "__main__":
     ap.add_argument("--hot-per-user", type=int, default=None)
     ap.add_argument("--pool-blocks", type=int, default=None)
     ap.add_argument("--retrieve-only", action="store_true", help="embedding-only store, time the batched retrieval alone")
+    ap.add_argument("--host-tier", action="store_true", help="Llama shape with all K/V in the pinned host arena: inject over PCIe")
     a = ap.parse_args()
-    if a.retrieve_only:
+    if a.host_tier:
+        for ln in measure_host_tier(a.iters, a.seed):
+            print(json.dumps(ln))
+    elif a.retrieve_only:
         print(json.dumps(measure_retrieve_only(a.config, a.iters, a.seed)))
     else:
         print(json.dumps(measure(a.config, a.iters, a.seed, a.hot_per_user, a.pool_blocks)))

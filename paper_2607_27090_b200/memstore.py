@@ -39,6 +39,7 @@ class _Config(C.Structure):
         ("rope_theta", C.c_double), ("inv_freq_override", C.POINTER(C.c_float)), ("max_position", C.c_int64),
         ("n_users", C.c_int32), ("flags", C.c_uint32), ("max_facts_per_user", C.c_int64),
         ("max_kv_tokens", C.c_int64), ("kv_arena", C.c_void_p), ("kv_arena_bytes", C.c_size_t),
+        ("max_host_kv_tokens", C.c_int64),
     ]  # fmt: skip
 
 
@@ -53,7 +54,7 @@ class _PagedCache(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes", "kernel_timeouts")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares
@@ -61,7 +62,7 @@ EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
-    "memstore_retrieve_inject",
+    "memstore_retrieve_inject", "memstore_add_facts_host",
 )  # fmt: skip
 
 _lib = None
@@ -91,6 +92,8 @@ def load_library() -> C.CDLL:
     L.memstore_add_fact.argtypes = [vp, i32, vp, vp, vp, i32, C.POINTER(i32), vp]
     L.memstore_add_facts.restype = i32
     L.memstore_add_facts.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
+    L.memstore_add_facts_host.restype = i32
+    L.memstore_add_facts_host.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
     L.memstore_retrieve.restype = i32
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.memstore_retrieve_static.restype = i32
@@ -181,7 +184,7 @@ class MemStore:
 
     def __init__(self, *, device=0, n_layers, n_kv_heads, head_dim, emb_dim, emb_dtype=torch.float16, rope_theta=1.0e4,
                  rope_style=ROPE_HALF_SPLIT, inv_freq_override=None, max_position=1 << 24, n_users=1,
-                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None, flags=0):  # fmt: skip
+                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None, flags=0, max_host_kv_tokens=0):  # fmt: skip
         self._lib = load_library()
         self._h = C.c_void_p()
         self.device = torch.device("cuda", device if isinstance(device, int) else torch.device(device).index or 0)
@@ -199,7 +202,7 @@ class MemStore:
         cfg = _Config(self.device.index, n_layers, n_kv_heads, head_dim, DTYPE_BF16, emb_dim, emb_code, rope_style,
                       float(rope_theta), ov, max_position, n_users, flags, max_facts_per_user, max_kv_tokens,
                       kv_arena.data_ptr() if kv_arena is not None else None,
-                      kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0)  # fmt: skip
+                      kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0, max_host_kv_tokens)  # fmt: skip
         self.n_layers, self.n_kv_heads, self.head_dim, self.emb_dim = n_layers, n_kv_heads, head_dim, emb_dim
         rc = self._lib.memstore_create(C.byref(cfg), C.byref(self._h))
         if rc != MS_OK:
@@ -246,6 +249,26 @@ class MemStore:
         rc = self._lib.memstore_add_facts(self._h, user, n, _dev_ptr(embs, self.emb_torch_dtype, "embs"),
                                           _dev_ptr(k_pre, torch.bfloat16, "k_pre"), _dev_ptr(v, torch.bfloat16, "v"),
                                           lens, C.byref(out), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return out.value
+
+    def add_facts_host(self, embs, n_tokens, k_pre_host, v_host, user=0, stream=None) -> int:
+        """Like ``add_facts`` but K/V are HOST arrays (numpy uint16 bf16 bits or CPU bf16 tensors, [L, sum(n_tokens), h, d])
+        that go to the store's pinned host arena; injection reads them over PCIe."""
+        import numpy as np
+
+        def host_ptr(a):
+            if isinstance(a, torch.Tensor):
+                assert not a.is_cuda and a.is_contiguous() and a.element_size() == 2
+                return C.c_void_p(a.data_ptr())
+            assert isinstance(a, np.ndarray) and a.flags.c_contiguous and a.itemsize == 2
+            return C.c_void_p(a.ctypes.data)
+
+        n = embs.shape[0]
+        lens = (C.c_int32 * n)(*[int(x) for x in n_tokens])
+        out = C.c_int32(-1)
+        rc = self._lib.memstore_add_facts_host(self._h, user, n, _dev_ptr(embs, self.emb_torch_dtype, "embs"), host_ptr(k_pre_host),
+                                               host_ptr(v_host), lens, C.byref(out), _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out.value
 

@@ -27,12 +27,12 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header_sizes():
-    # the ctypes mirrors must have the C sizes (x86-64 / LP64): config 96 bytes, cache 64, stats 72
+    # the ctypes mirrors must have the C sizes (x86-64 / LP64): config 104 bytes, cache 64, stats 80
     from paper_2607_27090_b200 import memstore
 
-    assert ctypes.sizeof(memstore._Config) == 96
+    assert ctypes.sizeof(memstore._Config) == 104
     assert ctypes.sizeof(memstore._PagedCache) == 64
-    assert ctypes.sizeof(memstore._Stats) == 72
+    assert ctypes.sizeof(memstore._Stats) == 80
 
 
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):

@@ -254,6 +254,44 @@ def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq):
     ms.close()
 
 
+def test_host_tier_facts_are_injected_over_pcie_and_mix_with_hbm_facts():
+    """Facts whose K/V live in the pinned host arena (the CPU-offloaded store) give the same cache contents as the
+    same facts in HBM; one request may name facts of both tiers."""
+    hs = HostStore(50, 24, 3, 8, 128, 5, 40, 128, "float16")
+    T = int(hs.lens.sum())
+    ms = MemStore(n_layers=hs.L, n_kv_heads=hs.H, head_dim=hs.D, emb_dim=128, rope_theta=5e5, max_facts_per_user=24,
+                  max_kv_tokens=T, max_host_kv_tokens=T)
+    # even facts go to HBM, odd facts to the host arena; ids stay dense in insertion order
+    for f in range(24):
+        t0, t1 = int(hs.offs[f]), int(hs.offs[f] + hs.lens[f])
+        kf, vf = np.ascontiguousarray(hs.k[:, t0:t1]), np.ascontiguousarray(hs.v[:, t0:t1])
+        if f % 2 == 0:
+            fid = ms.add_facts(to_dev(hs.emb[f : f + 1]), [hs.lens[f]], to_dev(kf), to_dev(vf))
+        else:
+            fid = ms.add_facts_host(to_dev(hs.emb[f : f + 1]), [hs.lens[f]], kf, vf)
+        assert fid == f
+    st = ms.stats()
+    assert st["host_kv_tokens_used"] == int(hs.lens[1::2].sum()) and st["kv_tokens_used"] == int(hs.lens[0::2].sum())
+    table = synth.block_tables(51, 64, 30, 1)[0]
+    for ids in ([1, 3, 5, 7], [0, 1, 2, 3, 10, 11], [23, 22, -1, 9, 9]):
+        cache = make_cache(hs, 64, 16)
+        out = run_inject_and_check(ms, hs, ids, 19, table, cache, 5e5, flags=M.INJECT_REVERSE)
+        assert out["exact_frac"] > 0.995
+    # retrieval is tier-blind and the one-call path works on host-tier facts too
+    q = to_dev(synth.queries(50, 1, 128, "float16"))
+    ca, cb = make_cache(hs, 64, 16), make_cache(hs, 64, 16)
+    start, tb = to_dev(np.array([3], np.int32)), to_dev(table[None])
+    ids_a, _ = ms.retrieve(q, 6)
+    ms.inject(ids_a, start, tb, ca)
+    ids_b, n_b, st_b = ms.retrieve_inject(q, 6, start, tb, cb)
+    torch.cuda.synchronize()
+    assert torch.equal(ids_a, ids_b) and int(st_b[0]) == 0
+    assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+    with pytest.raises(M.MemStoreError):
+        ms.add_facts_host(to_dev(hs.emb[:1]), [T], np.zeros((3, T, 8, 128), np.uint16), np.zeros((3, T, 8, 128), np.uint16))
+    ms.close()
+
+
 def test_serve_host_matches_the_device_calls():
     """memstore_serve_host (host buffers in, host results out) against retrieve + inject on device buffers."""
     hs = HostStore(19, 120, 2, 8, 128, 8, 40, 256, "float16", n_users=2)
