@@ -377,6 +377,47 @@ def run_ours(args):
         "clocks": clk.summary(),
     }  # fmt: skip
 
+    # ---- per-request latency distribution (separate pass: an event after every step) and CUDA-graph replay ---------
+    n_lat = min(args.steps, 500)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat + 1)]
+    torch.cuda.synchronize()
+    marks[0].record(stream)
+    for i in range(n_lat):
+        step(i)
+        marks[i + 1].record(stream)
+    torch.cuda.synchronize()
+    lat = np.sort(np.array([marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(n_lat)]))
+    line["latency_us"] = {"p10": float(lat[n_lat // 10]), "p50": float(lat[n_lat // 2]), "p90": float(lat[(n_lat * 9) // 10]),
+                          "n": n_lat, "note": "one CUDA event per step on the stream, steady state"}  # fmt: skip
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for i in range(2):  # make sure nothing is allocated lazily on this stream inside the capture
+                store.retrieve_inject(queries[0:1], k, start, tables[0:1], cache, out_ids=ids, out_n_tokens=n_tok[0:1],
+                                      out_status=status[0:1], flags=M.INJECT_REVERSE, stream=side)  # fmt: skip
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                for j in range(n_pool):
+                    store.retrieve_inject(queries[j : j + 1], k, start, tables[j : j + 1], cache, out_ids=ids,
+                                          out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1], flags=M.INJECT_REVERSE,
+                                          stream=side)  # fmt: skip
+        torch.cuda.synchronize()
+        reps = max(1, min(args.steps, 800) // n_pool)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        line["graph_replay_us"] = e0.elapsed_time(e1) * 1e3 / (reps * n_pool)
+    except Exception as ex:  # graph capture is optional evidence, never a reason to lose the bench line
+        line["graph_replay_us"] = None
+        line["graph_replay_error"] = str(ex)[:200]
+        torch.cuda.synchronize()
+
     if args.sweep_k:
         sweep = {}
         for kk in (5, 10, 20):
@@ -405,8 +446,10 @@ def run_ours(args):
         while not vals or (time.perf_counter() - t_begin < args.cpu_baseline_seconds and len(vals) < 100):
             v, sample = arm.time_step(n_take)
             vals.append(v)
+        one = OracleArm(shape, k, args.seed, n_threads=1)
+        v1, _ = one.time_step(one.facts_for_budget(3.0))
         line["cpu_baseline"] = {"value": sum(vals) / len(vals), "unit": "us", "cores": arm.cores, "kind": "oracle",
-                                "sample": f"mean of {len(vals)} repeats of: {sample}"}  # fmt: skip
+                                "sample": f"mean of {len(vals)} repeats of: {sample}", "single_thread_value": v1}  # fmt: skip
     if rank == 0:
         print(json.dumps(line))
     store.close()
