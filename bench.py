@@ -457,8 +457,8 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per launch of the copy kernel from the ncu capture summarised in
-# profiles/inject_copy_kernel_llama8b_k50.md (mean of the two captured launches; the capture starts from a flushed L2, so
+# DRAM bytes (read + write) per launch of the copy kernel from the committed ncu capture summary of that kernel
+# (mean of the two captured launches; the capture starts from a flushed L2, so
 # about 50 MB of the written bytes are still in L2 when the kernel ends and are not in this figure).
 NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {("llama8b", 50): 468.2e6}
 
