@@ -200,6 +200,11 @@ __device__ __forceinline__ void write_topk(const unsigned long long* cand, int t
   }
 }
 
+// Sampled bucket choice of topk_block: sample size and shape, and the shortest list it is used for.
+constexpr int kSampleSize = 4096;
+constexpr int kSampleChunks = 64;
+constexpr int kSampleMinN = 65536;
+
 struct TopkShared {
   uint32_t hist[256];
   unsigned long long cand[kTopkMaxK];
@@ -222,7 +227,7 @@ template <int THREADS, class KeyAt, class Visit>
 __device__ __forceinline__ void for_each_key(int n, KeyAt key_at, Visit visit) {
   const int tid = threadIdx.x;
   for (int base = tid; base < n; base += THREADS * 8) {
-    uint32_t kx[8];
+    decltype(key_at(0)) kx[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int i = base + u * THREADS;
@@ -236,6 +241,263 @@ __device__ __forceinline__ void for_each_key(int n, KeyAt key_at, Visit visit) {
   }
 }
 
+// 256 buckets linear in the score VALUE over [s_lo, s_hi] (linear in the key would be logarithmic in the value and
+// put a whole octave of top scores into one bucket); monotone in the score; scores above s_hi land in bucket 255.
+struct LinearBuckets {
+  float s_lo, scale;
+  __device__ __forceinline__ static LinearBuckets over(float lo, float hi) { return {lo, 255.5f / fmaxf(hi - lo, 1e-30f)}; }
+  __device__ __forceinline__ uint32_t of(float sv) const {  // of a score sv >= s_lo
+    return min(255u, (uint32_t)((sv - s_lo) * scale));
+  }
+};
+
+// Block-wide minimum and maximum of per-thread keys -> sm.kmin, sm.kmax (visible to all threads on return);
+// also clears the histogram.
+template <int THREADS>
+__device__ __forceinline__ void block_min_max(TopkShared& sm, uint32_t lo, uint32_t hi) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  if (lane == 0) {
+    sm.warp_min[warp] = lo;
+    sm.warp_max[warp] = hi;
+  }
+  for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
+  __syncthreads();
+  if (warp == 0) {
+    lo = lane < THREADS / 32 ? sm.warp_min[lane] : 0xffffffffu;
+    hi = lane < THREADS / 32 ? sm.warp_max[lane] : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+      sm.kmin = lo;
+      sm.kmax = hi;
+    }
+  }
+  __syncthreads();
+}
+
+// Warp 0: the highest bucket B with at least `target` histogram entries in buckets >= B -> sm.bucket, and that
+// count -> sm.n_cand.  Nothing is written when the whole histogram holds fewer than `target` entries.
+__device__ __forceinline__ void find_rank_bucket(TopkShared& sm, uint32_t target) {
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x >= 32) return;
+  uint32_t c[8], sum = 0;
+#pragma unroll
+  for (int b = 0; b < 8; ++b) {
+    c[b] = sm.hist[8 * lane + b];
+    sum += c[b];
+  }
+  uint32_t incl = sum;  // buckets of this lane and of all higher lanes
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += y;
+  }
+  uint32_t above = incl - sum;
+  if (above < target && incl >= target) {
+    int b = 7;
+    for (; b > 0; --b) {
+      if (above + c[b] >= target) break;
+      above += c[b];
+    }
+    sm.bucket = 8 * lane + b;
+    sm.n_cand = above + c[b];
+  }
+}
+
+// The n_cand (>= min(n, k), <= kTopkMaxK) candidates in `cand` (shared memory), distinct 64-bit keys, are ranked and the best k
+// written out.  Few candidates: the rank of a candidate is the number of larger ones, no sorting network.
+template <int THREADS>
+__device__ __forceinline__ void rank_candidates(unsigned long long* cand, uint32_t n_cand, int k, int take, const IdMap ids,
+                                                int32_t* out_ids, float* out_scores) {
+  const int tid = threadIdx.x;
+  if (n_cand * 4 <= (uint32_t)THREADS) {
+    // four lanes share a candidate and split the comparisons
+    const uint32_t ci = (uint32_t)tid >> 2, part = (uint32_t)tid & 3u;
+    const unsigned long long mine = ci < n_cand ? cand[ci] : 0ull;
+    uint32_t rank = 0;
+    for (uint32_t jj = part; jj < n_cand; jj += 4) rank += cand[jj] > mine;
+    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+    if (ci < n_cand && part == 0 && rank < (uint32_t)k) {
+      out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+      if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+    }
+    return;
+  }
+  if (n_cand <= (uint32_t)THREADS) {
+    if (tid < (int)n_cand) {
+      const unsigned long long mine = cand[tid];
+      uint32_t rank = 0;
+      for (uint32_t jj = 0; jj < n_cand; ++jj) rank += cand[jj] > mine;
+      if (rank < (uint32_t)k) {
+        out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+        if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+      }
+    }
+    return;
+  }
+  int P2 = 1;
+  while (P2 < (int)n_cand) P2 <<= 1;
+  for (int i = (int)n_cand + tid; i < P2; i += THREADS) cand[i] = 0ull;
+  __syncthreads();
+  bitonic_sort_desc<THREADS>(cand, P2);
+  write_topk<THREADS>(cand, take, k, ids, out_ids, out_scores);
+}
+
+// A visit of (index, score) over fp32 scores in global memory, read as 16-byte vectors, UNROLL vectors per thread in flight: a
+// long score list (a hundred thousand group maxima per query) is swept by ONE CTA, whose speed is set by the bytes
+// it keeps in flight.  `sc` must be 16-byte aligned.  The visiting order differs from for_each_key; callers depend
+// on the set of (index, key) pairs only.
+template <int THREADS, int UNROLL, class Visit>
+__device__ __forceinline__ void for_each_score_vec4(const float* sc, int n, Visit visit) {
+  const int tid = threadIdx.x;
+  const int n4 = n >> 2;
+  const float4* v = reinterpret_cast<const float4*>(sc);
+  for (int base = tid; base < n4; base += THREADS * UNROLL) {
+    float4 x[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int i = base + u * THREADS;
+      if (i < n4) x[u] = __ldcg(v + i);
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int i = base + u * THREADS;
+      if (i < n4) {
+        visit(4 * i + 0, x[u].x);
+        visit(4 * i + 1, x[u].y);
+        visit(4 * i + 2, x[u].z);
+        visit(4 * i + 3, x[u].w);
+      }
+    }
+  }
+  const int i = 4 * n4 + tid;
+  if (i < n) visit(i, __ldcg(sc + i));
+}
+
+// Second selection level for a candidate set that is several times larger than k (ranking by counting is
+// quadratic): the same bucket search over the candidates' own score range keeps those in or above the bucket of
+// the k-th largest.  n_cand <= kTopkMaxK / 2 candidates in sm.cand[0..n_cand); the survivors (at least k) go to
+// sm.cand[kTopkMaxK / 2 ...) and their number is returned (0: the candidates' scores are all equal, nothing moved).
+template <int THREADS>
+__device__ __forceinline__ uint32_t refine_candidates(TopkShared& sm, uint32_t n_cand, int k) {
+  const int tid = threadIdx.x;
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for (uint32_t j = tid; j < n_cand; j += THREADS) {
+    const uint32_t kx = (uint32_t)(sm.cand[j] >> 32);
+    lo = min(lo, kx);
+    hi = max(hi, kx);
+  }
+  block_min_max<THREADS>(sm, lo, hi);
+  const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
+  if (!(smax > smin)) return 0u;
+  LinearBuckets bk{0.f, 0.f};
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    bk = LinearBuckets::over(attempt == 0 ? smin + 0.5f * (smax - smin) : smin, smax);
+    if (attempt) {
+      for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
+    }
+    if (tid == 0) sm.n_cand = 0xffffffffu;
+    __syncthreads();
+    for (uint32_t j = tid; j < n_cand; j += THREADS) {
+      const float sv = key_score((uint32_t)(sm.cand[j] >> 32));
+      if (sv >= bk.s_lo) atomicAdd(&sm.hist[bk.of(sv)], 1u);
+    }
+    __syncthreads();
+    find_rank_bucket(sm, (uint32_t)k);
+    __syncthreads();
+    if (sm.n_cand != 0xffffffffu) break;
+  }
+  const uint32_t B = sm.bucket, n2 = sm.n_cand;
+  if (tid == 0) sm.ngt = 0;
+  __syncthreads();
+  for (uint32_t j = tid; j < n_cand; j += THREADS) {
+    const unsigned long long c = sm.cand[j];
+    const float sv = key_score((uint32_t)(c >> 32));
+    if (sv >= bk.s_lo && bk.of(sv) >= B) sm.cand[kTopkMaxK / 2 + atomicAdd(&sm.ngt, 1u)] = c;
+  }
+  __syncthreads();
+  return n2;
+}
+
+// Top-k of a LONG fp32 score list in global memory (n >= kSampleMinN, 16-byte aligned) with one sweep of the list:
+// the buckets and the candidate threshold come from kSampleSize scores taken in kSampleChunks evenly spaced runs,
+// aiming at about 4.5 k candidates; the sweep gathers every score in or above the threshold bucket and counts
+// them.  Returns true (the same value in every thread) when the gathered set held at least k and at most
+// kTopkMaxK candidates and the result has been written; false when the sample was unrepresentative or unlucky (or
+// the list too long for the candidate array), in which case nothing has been written and the caller runs the exact
+// selection: a bad sample costs time, never correctness.
+template <int THREADS>
+__device__ bool topk_sampled(TopkShared& sm, const float* sc, int n, int k, const IdMap ids, int32_t* out_ids,
+                             float* out_scores) {
+  static_assert(kSampleSize * sizeof(float) <= sizeof(sm.cand), "the sample lives in the candidate array");
+  const int tid = threadIdx.x;
+  const uint32_t sample_rank = max(12u, (uint32_t)((4.5f * (float)k * (float)kSampleSize) / (float)n) + 1u);
+  if ((float)sample_rank * (float)n / (float)kSampleSize > 0.5f * (float)kTopkMaxK) return false;
+  float* samp = reinterpret_cast<float*>(sm.cand);
+  constexpr int kRun = kSampleSize / kSampleChunks;
+  const int64_t stride = n / kSampleChunks;
+  float flo = INFINITY, fhi = -INFINITY;
+  for (int j = tid; j < kSampleSize; j += THREADS) {
+    const float sv = __ldcg(sc + (int64_t)(j / kRun) * stride + (j % kRun));
+    samp[j] = sv;
+    flo = fminf(flo, sv);
+    fhi = fmaxf(fhi, sv);
+  }
+  block_min_max<THREADS>(sm, order_key(flo), order_key(fhi));
+  const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
+  if (!(smax > smin)) return false;
+  LinearBuckets bk{0.f, 0.f};
+  for (int attempt = 0; attempt < 2; ++attempt) {  // upper half of the sample's range first, as in topk_block
+    bk = LinearBuckets::over(attempt == 0 ? smin + 0.5f * (smax - smin) : smin, smax);
+    if (attempt) {
+      for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
+    }
+    if (tid == 0) sm.n_cand = 0xffffffffu;
+    __syncthreads();
+    for (int j = tid; j < kSampleSize; j += THREADS) {
+      const float sv = samp[j];
+      if (sv >= bk.s_lo) atomicAdd(&sm.hist[bk.of(sv)], 1u);
+    }
+    __syncthreads();
+    find_rank_bucket(sm, sample_rank);
+    __syncthreads();
+    if (sm.n_cand != 0xffffffffu) break;
+  }
+  if (sm.n_cand == 0xffffffffu) return false;
+  const uint32_t B = sm.bucket;
+  if (tid == 0) sm.ngt = 0;
+  __syncthreads();  // the sample has been read by everyone: the candidates may overwrite it
+  for_each_score_vec4<THREADS, 8>(sc, n, [&](int i, float sv) {
+    if (sv >= bk.s_lo && bk.of(sv) >= B) {
+      const uint32_t slot = atomicAdd(&sm.ngt, 1u);
+      if (slot < (uint32_t)kTopkMaxK)
+        sm.cand[slot] = ((unsigned long long)order_key(sv) << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+    }
+  });
+  __syncthreads();
+  const uint32_t n_cand = sm.ngt;
+  __syncthreads();  // everyone has read the count before a later selection resets it
+  if (n_cand < (uint32_t)k || n_cand > (uint32_t)kTopkMaxK) return false;
+  if (n_cand > 2u * (uint32_t)k && n_cand <= (uint32_t)kTopkMaxK / 2) {
+    const uint32_t n2 = refine_candidates<THREADS>(sm, n_cand, k);
+    if (n2) {
+      rank_candidates<THREADS>(sm.cand + kTopkMaxK / 2, n2, k, k, ids, out_ids, out_scores);
+      return true;
+    }
+  }
+  rank_candidates<THREADS>(sm.cand, n_cand, k, k, ids, out_ids, out_scores);
+  return true;
+}
+
 template <int THREADS>
 __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const IdMap ids,
                            int32_t* out_ids, float* out_scores, bool have_minmax = false, uint32_t my_lo = 0xffffffffu,
@@ -244,142 +506,75 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   const int lane = tid & 31, warp = tid >> 5;
   const int take = min(n, k);
   auto key_at = [&](int i) -> uint32_t { return keys ? keys[i] : order_key(__ldcg(sc + i)); };
+  // The fast path below works on the SCORES (a key converts back without loss): most elements then cost one
+  // comparison per pass.  Long lists in global memory are swept with vector loads.
+  auto score_at = [&](int i) -> float { return keys ? key_score(keys[i]) : __ldcg(sc + i); };
+  const bool vec = keys == nullptr && n >= THREADS * 16 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0;
+  auto sweep = [&](auto visit) {
+    if (vec)
+      for_each_score_vec4<THREADS, 4>(sc, n, visit);
+    else
+      for_each_key<THREADS>(n, score_at, visit);
+  };
 
-  // ---- fast path: one histogram over 256 LINEAR buckets of [min key, max key] ---------------------------
+  // ---- sampled path: long lists in global memory, bucket choice from a sample, ONE sweep of the list ------
+  if (n > k && vec && !have_minmax && n >= kSampleMinN) {
+    if (topk_sampled<THREADS>(sm, sc, n, k, ids, out_ids, out_scores)) return;
+  }
+
+  // ---- fast path: one histogram over 256 LINEAR buckets of the score range -------------------------------
   // Scores of unit-norm embeddings share sign and exponent, so the leading radix digits of almost all keys
-  // coincide; buckets that are linear in the key spread them.  Every key in or above the bucket B that holds
-  // the k-th largest becomes a candidate (their number is k plus part of one bucket); the 64-bit sort below
-  // orders them exactly, ties by row.  If the candidates do not fit (massive ties) the radix path runs instead.
-  bool fast = false;
+  // coincide; buckets that are linear in the score value spread them.  Every score in or above the bucket B
+  // that holds the k-th largest becomes a candidate (their number is k plus part of one bucket); the 64-bit
+  // keys order them exactly, ties by row.  If the candidates do not fit (massive ties) the radix path runs.
   if (n > k) {
     uint32_t lo = my_lo, hi = my_hi;
     if (!have_minmax) {
-      for_each_key<THREADS>(n, key_at, [&](int, uint32_t kx) {
-        lo = min(lo, kx);
-        hi = max(hi, kx);
+      float flo = INFINITY, fhi = -INFINITY;
+      sweep([&](int, float sv) {
+        flo = fminf(flo, sv);
+        fhi = fmaxf(fhi, sv);
       });
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
-    }
-    if (lane == 0) {
-      sm.warp_min[warp] = lo;
-      sm.warp_max[warp] = hi;
-    }
-    for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
-    __syncthreads();
-    if (warp == 0) {
-      lo = lane < THREADS / 32 ? sm.warp_min[lane] : 0xffffffffu;
-      hi = lane < THREADS / 32 ? sm.warp_max[lane] : 0u;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-        hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
-      }
-      if (lane == 0) {
-        sm.kmin = lo;
-        sm.kmax = hi;
+      if (flo <= fhi) {  // this thread saw at least one score
+        lo = order_key(flo);
+        hi = order_key(fhi);
       }
     }
-    __syncthreads();
+    block_min_max<THREADS>(sm, lo, hi);  // -> sm.kmin, sm.kmax; clears sm.hist
     const uint32_t range = sm.kmax - sm.kmin;
-    // bucket of a score: linear in the VALUE (linear in the key would be logarithmic in the value and put a whole
-    // octave of top scores into one bucket); monotone in the score.  With k much smaller than n only the upper part
-    // of the value range can hold the k-th largest, so the first attempt histograms the upper half alone (twice the
-    // resolution and a fraction of the shared-memory atomics); if fewer than k keys live there the whole range is used.
     const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
-    float s_lo = 0.f, bscale = 0.f;
-    auto bucket_of = [&](uint32_t kx) -> uint32_t {  // 256 = below the histogrammed range
-      const float sv = key_score(kx);
-      return sv < s_lo ? 256u : min(255u, (uint32_t)((sv - s_lo) * bscale));
-    };
+    // With k much smaller than n only the upper part of the value range can hold the k-th largest, so the first
+    // attempt histograms the upper half alone (twice the resolution and a fraction of the shared-memory atomics);
+    // if fewer than k scores live there the whole range is used.
+    LinearBuckets bk{0.f, 0.f};
     for (int attempt = 0; attempt < 2; ++attempt) {
-      s_lo = attempt == 0 ? smin + 0.5f * (smax - smin) : smin;
-      bscale = 255.5f / fmaxf(smax - s_lo, 1e-30f);
+      bk = LinearBuckets::over(attempt == 0 ? smin + 0.5f * (smax - smin) : smin, smax);
       if (attempt) {
         for (int b = tid; b < 256; b += THREADS) sm.hist[b] = 0;
       }
       if (tid == 0) sm.n_cand = 0xffffffffu;
       __syncthreads();
-      for_each_key<THREADS>(n, key_at, [&](int, uint32_t kx) {
-        const uint32_t b = bucket_of(kx);
-        if (b < 256u) atomicAdd(&sm.hist[b], 1u);
+      sweep([&](int, float sv) {
+        if (sv >= bk.s_lo) atomicAdd(&sm.hist[bk.of(sv)], 1u);
       });
       __syncthreads();
-      if (warp == 0) {
-        uint32_t c[8], sum = 0;
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          c[b] = sm.hist[8 * lane + b];
-          sum += c[b];
-        }
-        uint32_t incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
-          if (lane + o < 32) incl += y;
-        }
-        uint32_t above = incl - sum;
-        if (above < (uint32_t)k && incl >= (uint32_t)k) {
-          int b = 7;
-          for (; b > 0; --b) {
-            if (above + c[b] >= (uint32_t)k) break;
-            above += c[b];
-          }
-          sm.bucket = 8 * lane + b;
-          sm.n_cand = above + c[b];
-        }
-      }
+      find_rank_bucket(sm, (uint32_t)k);
       __syncthreads();
       if (sm.n_cand != 0xffffffffu) break;  // the k-th largest lies in the histogrammed range
     }
-    fast = range != 0 && sm.n_cand <= (uint32_t)kTopkMaxK;
-    if (fast) {
+    if (range != 0 && sm.n_cand <= (uint32_t)kTopkMaxK) {
       const uint32_t B = sm.bucket, n_cand = sm.n_cand;
-      int P2 = 1;
-      while (P2 < (int)n_cand) P2 <<= 1;
       if (tid == 0) sm.ngt = 0;
-      for (int i = tid; i < P2; i += THREADS) sm.cand[i] = 0ull;
       __syncthreads();
-      for_each_key<THREADS>(n, key_at, [&](int i, uint32_t kx) {
-        const uint32_t b = bucket_of(kx);
-        if (b < 256u && b >= B) {  // 256 marks a key below the histogrammed range: never a candidate
+      sweep([&](int i, float sv) {
+        if (sv >= bk.s_lo && bk.of(sv) >= B) {  // a score below the histogrammed range is never a candidate
           const uint32_t slot = atomicAdd(&sm.ngt, 1u);
-          if (slot < (uint32_t)kTopkMaxK) sm.cand[slot] = ((unsigned long long)kx << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
+          if (slot < (uint32_t)kTopkMaxK)
+            sm.cand[slot] = ((unsigned long long)order_key(sv) << 32) | (uint32_t)(0xffffffffu - (uint32_t)i);
         }
       });
       __syncthreads();
-      if (n_cand * 4 <= (uint32_t)THREADS) {
-        // few candidates: the rank of a candidate is the number of larger ones (keys are distinct); no sorting
-        // network.  Four lanes share a candidate and split the comparisons.
-        const uint32_t ci = (uint32_t)tid >> 2, part = (uint32_t)tid & 3u;
-        const unsigned long long mine = ci < n_cand ? sm.cand[ci] : 0ull;
-        uint32_t rank = 0;
-        for (uint32_t jj = part; jj < n_cand; jj += 4) rank += sm.cand[jj] > mine;
-        rank += __shfl_xor_sync(0xffffffffu, rank, 1);
-        rank += __shfl_xor_sync(0xffffffffu, rank, 2);
-        if (ci < n_cand && part == 0 && rank < (uint32_t)k) {
-          out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
-          if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
-        }
-        return;
-      }
-      if (n_cand <= (uint32_t)THREADS) {
-        if (tid < (int)n_cand) {
-          const unsigned long long mine = sm.cand[tid];
-          uint32_t rank = 0;
-          for (uint32_t jj = 0; jj < n_cand; ++jj) rank += sm.cand[jj] > mine;
-          if (rank < (uint32_t)k) {
-            out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
-            if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
-          }
-        }
-        return;
-      }
-      bitonic_sort_desc<THREADS>(sm.cand, P2);
-      write_topk<THREADS>(sm.cand, take, k, ids, out_ids, out_scores);
+      rank_candidates<THREADS>(sm.cand, n_cand, k, take, ids, out_ids, out_scores);
       return;
     }
   }
@@ -504,7 +699,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const Retriev
 }
 
 // Top-k only (large segments): one CTA per query, keys recomputed from global scores.
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const RetrieveParams p) {
+__global__ void __launch_bounds__(kTopkThreads, 1) topk_kernel(const RetrieveParams p) {
   __shared__ TopkShared sm;
   const int q = blockIdx.x;
   const int user = p.query_users ? p.query_users[q] : 0;
@@ -589,7 +784,7 @@ __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const Retrieve
 
 // Step 2: per query, the k2 groups with the largest group maximum, written in ASCENDING group order (so that the
 // candidate rows of step 3 are in row order and "lower index first" among equal scores means "lower fact id first").
-__global__ void __launch_bounds__(kTopkThreads) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
+__global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
                                                                     int32_t* sel /*[nq][k2]*/) {
   __shared__ TopkShared sm;
   __shared__ int32_t s_sel[512];

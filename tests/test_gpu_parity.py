@@ -122,6 +122,39 @@ def test_retrieve_many_queries_tensor_core_path(n, E, nq):
     ms.close()
 
 
+@pytest.mark.parametrize("case", ["plain", "too_many_candidates", "biased_sample"])
+def test_retrieve_long_segment_group_selection_from_a_sample(case):
+    """600,000 rows: the group selection of the tensor-core path picks its buckets from a sample of the group
+    maxima and must fall back to exact statistics when the sample misleads it (results identical either way)."""
+    n, E, nq, k = 600_000, 64, 8, 100
+    emb = synth.embeddings(41, n, E, "float16")
+    q = synth.queries(41, nq, E, "float16")
+    rng = np.random.default_rng(41)
+    if case == "too_many_candidates":
+        # 3000 rows close to query 0 in 3000 different groups: more candidates above any sampled threshold than fit
+        rows = rng.choice(n // 8, 3000, replace=False) * 8 + 3
+        noise = rng.standard_normal((3000, E)).astype(np.float32) * 0.02
+        emb[rows] = (q[0].astype(np.float32)[None, :] + noise).astype(np.float16)
+    if case == "biased_sample":
+        # 40 rows equal or close to query 1 sitting exactly where the sample looks (64 runs of 64 groups, evenly
+        # spaced over the 75,000 groups): the sample then promises far more high scores than the list holds
+        stride = (n // 8) // 64
+        groups = np.array([c * stride + o for c in range(0, 64, 8) for o in range(0, 10, 2)])
+        noise = rng.standard_normal((len(groups), E)).astype(np.float32) * 0.01
+        emb[groups * 8 + 5] = (q[1].astype(np.float32)[None, :] + noise).astype(np.float16)
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float16, rope_theta=1e4,
+                  max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+    for a in range(0, n, 100_000):
+        ms.add_facts(to_dev(emb[a : a + 100_000]), np.zeros(100_000, np.int32))
+    ids, sc = ms.retrieve(to_dev(q), k)
+    torch.cuda.synchronize()
+    assert ms.stats()["kernel_timeouts"] == 0
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    for i in range(nq):
+        check_ids(ids[i], sc[i], emb, q[i], k)
+    ms.close()
+
+
 # ------------------------------------------------------------------------------------------------ injection
 PATHS = [0, 1]  # 0: direct copy kernel (default), 1: MS_STORE_TMA_COPY_PATH (bulk-async staged kernel)
 
