@@ -65,7 +65,10 @@ enum {
 
 enum { MS_DTYPE_F32 = 0, MS_DTYPE_F16 = 1, MS_DTYPE_BF16 = 2 };
 enum { MS_ROPE_HALF_SPLIT = 0, MS_ROPE_INTERLEAVED = 1 };
-enum { MS_INJECT_REVERSE = 1u }; /* place ids[k-1] first, so that ids[0] ends next to the query */
+enum {
+  MS_INJECT_REVERSE = 1u, /* place ids[k-1] first, so that ids[0] ends next to the query */
+  MS_INJECT_PREFIX = 2u   /* place the store's instruction prefix (memstore_set_prefix) before the facts */
+};
 /* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
  * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */
 enum { MS_STORE_TMA_COPY_PATH = 1u };
@@ -205,12 +208,29 @@ typedef struct {
  *   out_slot_mapping  device int64 [nreq][slot_stride] or NULL: slot of each composed token
  *                 (-1 for a skipped token; entries beyond min(m, slot_stride) are not written)
  *   flags         MS_INJECT_REVERSE: place ids in reverse order (the paper's policy for a best-first list)
+ *                 MS_INJECT_PREFIX: the composed segment of every request starts with the stored instruction
+ *                 prefix (positions start_pos .. start_pos + n_prefix - 1), the facts follow; m counts its tokens,
+ *                 the slot mapping lists them first; k is then at most 4095 (2047 in memstore_retrieve_inject's
+ *                 two-launch form).  MS_ERR_INVALID_ARG when no prefix is stored.
  * Two requests that map to the same cache slot race (last writer wins, undetected).
  */
 ms_status memstore_inject(memstore_t* store, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
                           const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
                           uint32_t flags, ms_stream stream);
+
+/*
+ * The fixed instruction prefix of the composed segment (Sec. 3.3: the retrieved facts are gathered, a fixed
+ * instruction prefix is prepended, and the whole is given contiguous positions).  It is kept like a fact - keys
+ * BEFORE RoPE and raw values, appended to the device K/V arena (n_tokens of max_kv_tokens) - but has no embedding
+ * and no fact id, so retrieval never returns it; injections with MS_INJECT_PREFIX rotate it at its serving-time
+ * positions together with the facts.
+ *   k_pre, v   device bf16 [n_layers][n_tokens][n_kv_heads][head_dim], 16-byte aligned; copied on `stream`
+ *   n_tokens   0 removes the prefix.  A second call replaces the prefix; the arena tokens of the old one are not
+ *              reclaimed (the arena is append-only).
+ * MS_ERR_CAPACITY when the arena cannot take n_tokens more.
+ */
+ms_status memstore_set_prefix(memstore_t* store, const void* k_pre, const void* v, int32_t n_tokens, ms_stream stream);
 
 /*
  * memstore_retrieve immediately followed by memstore_inject of every query's id list (query q = request q), with

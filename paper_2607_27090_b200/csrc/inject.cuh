@@ -22,6 +22,7 @@ struct InjectParams {
   // request
   const int32_t* fact_ids;  // [nreq][k]
   int32_t nreq, k;
+  int32_t prefix_src, prefix_len;  // instruction prefix placed before the facts (arena token, length); length 0 = none
   const int32_t* start_pos;
   const int32_t* block_tables;
   int32_t max_blocks;
@@ -52,7 +53,8 @@ constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by t
 //   I1 fact resolution (id -> arena offset, length), I2 exclusive scan of lengths (b_i, m),
 //   I3 slot = block_table[pos / bs] * bs + pos % bs, validation, tile descriptors.
 // ------------------------------------------------------------------------------------------------
-// Shared memory of one planning CTA: s_begin / s_src hold one entry per fact of the request (the caller sizes them).
+// Shared memory of one planning CTA: s_begin / s_src hold one entry per fact of the request plus one for the
+// instruction prefix (the caller sizes them).
 constexpr int kPlanTableCache = 2048;  // block-table entries of a request kept in shared memory
 struct PlanShared {
   int32_t table[kPlanTableCache];
@@ -83,13 +85,20 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   for (int i = tid; i < n_cached; i += THREADS) ps.table[i] = table_row[i];
   __syncthreads();
 
-  // lengths of the facts in placement order, exclusive scan in chunks of THREADS
+  // lengths of the entries in placement order (the instruction prefix, if any, then the facts), exclusive scan in
+  // chunks of THREADS
   const int32_t* ids = p.fact_ids + (int64_t)r * p.k;
-  for (int base = 0; base < p.k; base += THREADS) {
+  const int has_prefix = p.prefix_len > 0;
+  const int n_entries = p.k + has_prefix;
+  for (int base = 0; base < n_entries; base += THREADS) {
     int j = base + tid;
     int32_t len = 0, src = 0;
-    if (j < p.k) {
-      int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - j) : j];
+    if (j < has_prefix) {
+      len = p.prefix_len;
+      src = p.prefix_src;
+    } else if (j < n_entries) {
+      const int jf = j - has_prefix;
+      int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - jf) : jf];
       if (id >= 0) {
         if (id >= p.n_facts) {
           atomicOr(&s_status, 1 /*MS_REQ_BAD_FACT_ID*/);
@@ -116,7 +125,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     int32_t warp_off = 0;
     for (int w = 0; w < warp; ++w) warp_off += s_scan[w];
     int32_t carry = s_carry;
-    if (j < p.k) {
+    if (j < n_entries) {
       s_begin[j] = carry + warp_off + x - len;
       s_src[j] = src;
     }
@@ -146,7 +155,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     if (q >= 0 && q < m) {
       // the fact that owns composed token q is the LAST i with b_i <= q: entries of length zero (skipped,
       // unknown or non-resident ids) share their b_i with the next placed fact, and trailing ones have b_i = m > q
-      int lo = 0, hi = p.k - 1;
+      int lo = 0, hi = n_entries - 1;
       while (lo < hi) {
         int mid = (lo + hi + 1) >> 1;
         if (s_begin[mid] <= q) lo = mid; else hi = mid - 1;

@@ -66,6 +66,9 @@ struct memstore {
   std::vector<int64_t> user_count;
   int64_t n_facts = 0, n_resident = 0, kv_tokens_used = 0;
   int32_t max_fact_len = 0;
+  int64_t prefix_off = 0;   // instruction prefix (memstore_set_prefix): first arena token and length (0 = none)
+  int32_t prefix_len = 0;
+  int64_t prefix_tokens_total = 0;  // arena tokens taken by this and earlier prefixes (not facts)
   int64_t max_user_count = 0;
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
   int copy_ctas_per_sm = 1;
@@ -497,6 +500,37 @@ ms_status memstore_add_fact(memstore_t* s, int32_t user, const void* emb, const 
   return memstore_add_facts(s, user, 1, emb, k_pre, v, &n_tokens, out_fact_id, stream);
 }
 
+ms_status memstore_set_prefix(memstore_t* s, const void* k_pre, const void* v, int32_t n_tokens, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (n_tokens < 0) return fail(s, MS_ERR_INVALID_ARG, "negative token count");
+  if (n_tokens == 0) {
+    s->prefix_len = 0;
+    return MS_OK;
+  }
+  if (!k_pre || !v) return fail(s, MS_ERR_INVALID_ARG, "null K/V for the prefix");
+  if (((uintptr_t)k_pre & 15) || ((uintptr_t)v & 15)) return fail(s, MS_ERR_INVALID_ARG, "device buffers must be 16-byte aligned");
+  if (!s->k_arena || s->kv_tokens_used + n_tokens > c.max_kv_tokens)
+    return fail(s, MS_ERR_CAPACITY, "K/V arena full (%lld + %d > %lld tokens)", (long long)s->kv_tokens_used, n_tokens,
+                (long long)c.max_kv_tokens);
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t row_vec = (int64_t)c.n_kv_heads * c.head_dim * 2 / 16;
+  const int64_t src_vec = (int64_t)n_tokens * row_vec;
+  const int gx = (int)std::min<int64_t>((src_vec + 255) / 256, 4 * s->sm_count);
+  dim3 grid(gx > 0 ? gx : 1, c.n_layers, 2);
+  arena_append_kernel<<<grid, 256, 0, st>>>((const uint4*)k_pre, (const uint4*)v, (uint4*)s->k_arena, (uint4*)s->v_arena, src_vec,
+                                            c.max_kv_tokens * row_vec, s->kv_tokens_used * row_vec);
+  MS_CUDA(s, cudaGetLastError());
+  s->kernels_launched++;
+  s->prefix_off = s->kv_tokens_used;
+  s->prefix_len = n_tokens;
+  s->kv_tokens_used += n_tokens;
+  s->prefix_tokens_total += n_tokens;
+  return MS_OK;
+}
+
 ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                             int32_t* out_ids, float* out_scores, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
@@ -683,8 +717,12 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
                          int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags, InjectParams* out,
                          int64_t* out_tiles_needed) {
   const memstore_config& c = s->cfg;
-  if (nreq < 0 || k < 0 || k > kPlanMaxK) return fail(s, MS_ERR_INVALID_ARG, "nreq=%d k=%d (k <= %d)", nreq, k, kPlanMaxK);
-  if (flags & ~(uint32_t)MS_INJECT_REVERSE) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  if (flags & ~(uint32_t)(MS_INJECT_REVERSE | MS_INJECT_PREFIX)) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  const bool with_prefix = (flags & MS_INJECT_PREFIX) != 0;
+  if (with_prefix && s->prefix_len == 0) return fail(s, MS_ERR_INVALID_ARG, "MS_INJECT_PREFIX without a stored prefix (memstore_set_prefix)");
+  // the planning code keeps one entry per fact, plus one for the prefix, in shared memory
+  if (nreq < 0 || k < 0 || k + (with_prefix ? 1 : 0) > kPlanMaxK)
+    return fail(s, MS_ERR_INVALID_ARG, "nreq=%d k=%d (k <= %d, one less with a prefix)", nreq, k, kPlanMaxK);
   if (!start_pos || !block_tables || !cache || (k > 0 && !fact_ids) || max_blocks < 0)
     return fail(s, MS_ERR_INVALID_ARG, "null request arrays");
   if (!cache->k_base || !cache->v_base || cache->block_size <= 0 || cache->num_blocks <= 0)
@@ -697,7 +735,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   if ((c.max_kv_tokens == 0 || !s->k_arena) && !s->k_host) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
 
   // upper bound on tiles: each request composes at most k * (longest fact) tokens, plus a ragged first tile
-  const int64_t max_m = (int64_t)k * s->max_fact_len;
+  const int64_t max_m = (int64_t)k * s->max_fact_len + (with_prefix ? s->prefix_len : 0);
   const int64_t tiles_per_req = (max_m + kTileTokens - 1) / kTileTokens + 1;
   const int64_t tiles_needed = std::max<int64_t>(1, tiles_per_req * nreq);
   if (tiles_needed > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
@@ -729,6 +767,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.fact_ids = fact_ids;
   p.nreq = nreq;
   p.k = k;
+  p.prefix_src = with_prefix ? (int32_t)s->prefix_off : 0;
+  p.prefix_len = with_prefix ? s->prefix_len : 0;
   p.start_pos = start_pos;
   p.block_tables = block_tables;
   p.max_blocks = max_blocks;
@@ -754,7 +794,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
   const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
   const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
-  const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + kTileTokens - 1) / kTileTokens * nreq);
+  const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + p.prefix_len + kTileTokens - 1) / kTileTokens * nreq);
   int lpi = 1;
   while (lpi * 2 <= c.n_layers && c.n_layers % (lpi * 2) == 0 && est_tiles * (c.n_layers / (lpi * 2)) >= 16ll * resident_ctas) lpi *= 2;
   p.layers_per_item = lpi;
@@ -797,8 +837,8 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
     // from the mean length of the resident facts (plus a ragged tile per request and 3 %); the kernel's
     // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
     const int units = c.n_kv_heads * (c.head_dim / 16);
-    const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used + s->host_tokens_used) / (double)s->n_resident : 0.0;
-    int64_t est_tiles_grid = (int64_t)(((double)p.k * mean_len / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
+    const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used - s->prefix_tokens_total + s->host_tokens_used) / (double)s->n_resident : 0.0;
+    int64_t est_tiles_grid = (int64_t)((((double)p.k * mean_len + p.prefix_len) / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
     est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
     const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
     if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
@@ -860,7 +900,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
   if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
-  if (n_max > kFusedMaxRows || nq > s->scores_nq) {
+  if (n_max > kFusedMaxRows || nq > s->scores_nq || ((flags & MS_INJECT_PREFIX) && k + 1 > kTopkMaxK)) {
     // large segments (or a first call that still has to size its scratch): the two calls one after the other
     ms_status rc = memstore_retrieve(s, queries, query_users, nq, k, out_ids, out_scores, stream);
     if (rc != MS_OK) return rc;

@@ -22,6 +22,7 @@ REQ_BAD_FACT_ID, REQ_NOT_RESIDENT, REQ_BLOCK_TABLE_SHORT, REQ_BAD_BLOCK_ID, REQ_
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
 ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
 INJECT_REVERSE = 1
+INJECT_PREFIX = 2
 STORE_TMA_COPY_PATH = 1
 REQ_KERNEL_TIMEOUT = 32
 
@@ -62,7 +63,7 @@ EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
-    "memstore_retrieve_inject", "memstore_add_facts_host",
+    "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix",
 )  # fmt: skip
 
 _lib = None
@@ -95,6 +96,8 @@ def load_library() -> C.CDLL:
     L.memstore_add_facts_host.restype = i32
     L.memstore_add_facts_host.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
     L.memstore_retrieve.restype = i32
+    L.memstore_set_prefix.restype = i32
+    L.memstore_set_prefix.argtypes = [vp, vp, vp, i32, vp]
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
     L.memstore_retrieve_static.restype = i32
     L.memstore_retrieve_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
@@ -240,6 +243,14 @@ class MemStore:
                                          n_tokens, C.byref(out), _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out.value
+
+    def set_prefix(self, k_pre=None, v=None, stream=None) -> None:
+        """The fixed instruction prefix placed before the facts by injections with ``INJECT_PREFIX``:
+        ``k_pre``/``v`` [L, n, h, d] bf16 on the device (keys before RoPE); ``None`` removes it."""
+        n_tokens = 0 if k_pre is None else k_pre.shape[1]
+        rc = self._lib.memstore_set_prefix(self._h, _dev_ptr(k_pre, torch.bfloat16, "k_pre"), _dev_ptr(v, torch.bfloat16, "v"),
+                                           n_tokens, _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
 
     def add_facts(self, embs, n_tokens, k_pre=None, v=None, user=0, stream=None) -> int:
         """``n_tokens``: host sequence of ints; ``k_pre``/``v``: [L, sum(n_tokens), h, d] bf16 on the device."""

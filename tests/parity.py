@@ -55,13 +55,13 @@ class HostStore:
         self.emb = synth.embeddings(seed, total, emb_dim, emb_dtype)
         self.emb_dim, self.emb_dtype = emb_dim, emb_dtype
 
-    def to_memstore(self, theta, batch=64, **kw) -> MemStore:
+    def to_memstore(self, theta, batch=64, extra_kv_tokens=0, **kw) -> MemStore:
         """Facts are added user by user in id order (ids are global and dense in insertion order)."""
         tdt = torch.float32 if self.emb_dtype == "float32" else torch.float16
         T = int(self.lens.sum())
         ms = MemStore(n_layers=self.L, n_kv_heads=self.H, head_dim=self.D, emb_dim=self.emb_dim, emb_dtype=tdt,
                       rope_theta=theta, n_users=self.n_users, max_facts_per_user=max(self.per_user, 1),
-                      max_kv_tokens=max(T, 1), **kw)  # fmt: skip
+                      max_kv_tokens=max(T + extra_kv_tokens, 1), **kw)  # fmt: skip
         for u in range(self.n_users):
             for a in range(u * self.per_user, (u + 1) * self.per_user, batch):
                 b = min((u + 1) * self.per_user, a + batch)
@@ -170,9 +170,22 @@ def untouched_mask_ok(cache: PagedCache, written_slots: np.ndarray, sentinel_bit
     return True
 
 
+def with_prefix(hs: HostStore, placed, prefix):
+    """The oracle's view of an injection that starts with the instruction prefix: the prefix (k, v uint16
+    [L, n, H, D]) becomes one more fact after the store's own and leads the placement list."""
+    pk, pv = prefix
+    n = len(hs.lens)
+    offs = np.concatenate([hs.offs, [int(hs.lens.sum())]]).astype(np.int64)
+    lens = np.concatenate([hs.lens, [pk.shape[1]]]).astype(np.int32)
+    k = np.concatenate([hs.k, pk], axis=1)
+    v = np.concatenate([hs.v, pv], axis=1)
+    return np.concatenate([[n], np.asarray(placed, np.int32)]).astype(np.int32), offs, lens, k, v
+
+
 def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, cache: PagedCache, theta, style=0,
-                         inv_freq=None, flags=0, sentinel=synth.SENTINEL_BF16, check_untouched=True):  # fmt: skip
-    """One request: inject on the GPU, run the oracle on the same ids, compare. Returns stats dict."""
+                         inv_freq=None, flags=0, sentinel=synth.SENTINEL_BF16, check_untouched=True, prefix=None):  # fmt: skip
+    """One request: inject on the GPU, run the oracle on the same ids, compare. Returns stats dict.
+    ``prefix``: (k, v) of the instruction prefix the store holds, when ``flags`` asks for it."""
     dev = cache.k.device
     ids = torch.from_numpy(np.asarray(ids_np, np.int32).reshape(1, -1)).to(dev)
     sp = torch.tensor([start], dtype=torch.int32, device=dev)
@@ -180,7 +193,10 @@ def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, c
     placed = np.asarray(ids_np, np.int32).reshape(-1)
     if flags & 1:
         placed = placed[::-1]
-    res = oracle.inject(placed, hs.offs, hs.lens, hs.k, hs.v, theta, start, table_np, cache.block_size,
+    offs, lens, hk, hv = hs.offs, hs.lens, hs.k, hs.v
+    if flags & 2:
+        placed, offs, lens, hk, hv = with_prefix(hs, placed, prefix)
+    res = oracle.inject(placed, offs, lens, hk, hv, theta, start, table_np, cache.block_size,
                         cache.num_blocks, style=style, inv_freq_override=inv_freq)  # fmt: skip
     slot_map = torch.full((1, max(res.m, 1) + 3), -7, dtype=torch.int64, device=dev)
     n_tok, status = ms.inject(ids, sp, bt, cache, out_slot_mapping=slot_map, flags=flags)

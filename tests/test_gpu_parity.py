@@ -10,7 +10,7 @@ pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
     import oracle
-    from parity import (HostStore, check_ids, run_inject_and_check, to_dev, untouched_mask_ok)  # noqa: F401
+    from parity import (HostStore, check_ids, run_inject_and_check, to_dev, untouched_mask_ok, with_prefix)  # noqa: F401
     from paper_2607_27090_b200 import memstore as M
     from paper_2607_27090_b200.memstore import MemStore, PagedCache
 
@@ -284,6 +284,85 @@ def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq):
         assert torch.equal(ids_a, ids_b) and torch.equal(sc_a, sc_b) and torch.equal(n_a, n_b) and torch.equal(st_a, st_b)
         assert int(st_b.abs().sum()) == 0 and bool((sm[:, 0] >= 0).all())
         assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+    ms.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_inject_with_instruction_prefix(path):
+    """The stored instruction prefix leads the composed segment (pre-RoPE keys rotated at the positions it gets), in
+    plain and reverse fact order; it has no fact id, retrieval never sees it, and it can be replaced or removed."""
+    hs = HostStore(60, 40, 3, 4, 64, 3, 30, 64, "float32")
+    ms = hs.to_memstore(1e4, extra_kv_tokens=13 + 21, flags=path)
+    table = synth.block_tables(61, 64, 40, 1)[0]
+    ids0 = torch.tensor([[1, 2]], dtype=torch.int32, device=DEV)
+    with pytest.raises(RuntimeError):  # no prefix stored yet
+        ms.inject(ids0, torch.zeros(1, dtype=torch.int32, device=DEV), to_dev(table.reshape(1, -1)), make_cache(hs, 64, 16), flags=M.INJECT_PREFIX)
+    pre = synth.kv_fact(60, 10_000, hs.L, 13, hs.H, hs.D)
+    ms.set_prefix(to_dev(pre[0]), to_dev(pre[1]))
+    assert ms.stats()["n_facts"] == 40 and ms.stats()["kv_tokens_used"] == int(hs.lens.sum()) + 13
+    for ids, start, flags in (([5, 6, 7], 0, M.INJECT_PREFIX), ([30, 2, -1, 11, 11], 7, M.INJECT_PREFIX | M.INJECT_REVERSE),
+                              ([], 3, M.INJECT_PREFIX), ([9, 8], 16, 0)):  # fmt: skip
+        cache = make_cache(hs, 64, 16)
+        if len(ids) == 0:  # the prefix alone: k = 0 needs no id array
+            placed, offs, lens, hk, hv = with_prefix(hs, [], pre)
+            res = oracle.inject(placed, offs, lens, hk, hv, 1e4, start, table, 16, 64)
+            n_tok, status = ms.inject(torch.empty((1, 0), dtype=torch.int32, device=DEV), torch.tensor([start], dtype=torch.int32, device=DEV),
+                                      to_dev(table.reshape(1, -1)), cache, flags=flags)  # fmt: skip
+            torch.cuda.synchronize()
+            assert int(n_tok[0]) == res.m == 13 and int(status[0]) == 0
+            continue
+        out = run_inject_and_check(ms, hs, ids, start, table, cache, 1e4, flags=flags, prefix=pre)
+        assert out["worst"] <= 1.0
+    # a second prefix replaces the first; removing it makes the flag an error again
+    pre2 = synth.kv_fact(60, 10_001, hs.L, 21, hs.H, hs.D)
+    ms.set_prefix(to_dev(pre2[0]), to_dev(pre2[1]))
+    run_inject_and_check(ms, hs, [4, 0], 5, table, make_cache(hs, 64, 16), 1e4, flags=M.INJECT_PREFIX | M.INJECT_REVERSE, prefix=pre2)
+    q = to_dev(synth.queries(62, 1, 64, "float32"))
+    ids, _ = ms.retrieve(q, 40)
+    assert sorted(ids[0].tolist()) == list(range(40))  # every fact, and nothing else
+    ms.set_prefix(None, None)
+    with pytest.raises(RuntimeError):
+        ms.inject(ids0, torch.zeros(1, dtype=torch.int32, device=DEV), to_dev(table.reshape(1, -1)), make_cache(hs, 64, 16), flags=M.INJECT_PREFIX)
+    with pytest.raises(RuntimeError):  # the arena is append-only and now full
+        ms.set_prefix(to_dev(pre[0]), to_dev(pre[1]))
+    ms.close()
+
+
+def test_retrieve_inject_and_serve_host_with_instruction_prefix():
+    """The one-call forms place the prefix too (planned inside the retrieval kernel)."""
+    from parity import check_k, gather_cache_rows
+
+    hs = HostStore(63, 120, 2, 8, 128, 8, 40, 256, "float16")
+    ms = hs.to_memstore(5e5, extra_kv_tokens=17)
+    pre = synth.kv_fact(63, 10_000, hs.L, 17, hs.H, hs.D)
+    ms.set_prefix(to_dev(pre[0]), to_dev(pre[1]))
+    bs, nb, k = 16, 128, 7
+    qh = synth.queries(64, 2, 256, "float16")
+    table = synth.block_tables(65, nb, 40, 2)
+    flags = M.INJECT_PREFIX | M.INJECT_REVERSE
+    for rep in range(2):  # the second round takes the two-launch path
+        cache = make_cache(hs, nb, bs)
+        starts = to_dev(np.array([0, 0], np.int32))
+        ids, n_tok, status = ms.retrieve_inject(to_dev(qh), k, starts, to_dev(table), cache, flags=flags)
+        torch.cuda.synchronize()
+        assert int(status.abs().sum()) == 0
+        for r in range(2):
+            placed, offs, lens, hk, hv = with_prefix(hs, ids[r].cpu().numpy()[::-1], pre)
+            res = oracle.inject(placed, offs, lens, hk, hv, 5e5, 0, table[r], bs, nb)
+            assert int(n_tok[r]) == res.m
+            kb, vb = gather_cache_rows(cache, res.slots)
+            assert np.array_equal(vb, res.v)
+            check_k(kb, res.k_ref)
+    cache = make_cache(hs, nb, bs)
+    out = np.full(k + 2, -5, np.int32)
+    ms.serve_host(qh[0], k, 4, table[0], cache, out, flags=flags)
+    placed, offs, lens, hk, hv = with_prefix(hs, out[:k][::-1], pre)
+    res = oracle.inject(placed, offs, lens, hk, hv, 5e5, 4, table[0], bs, nb)
+    assert out[k] == res.m and out[k + 1] == 0
+    kb, vb = gather_cache_rows(cache, res.slots)
+    assert np.array_equal(vb, res.v)
+    check_k(kb, res.k_ref)
+    assert untouched_mask_ok(cache, res.slots, SENT)
     ms.close()
 
 
