@@ -70,7 +70,14 @@ def lib() -> C.CDLL:
             + [i64] * 4
             + [i32]
         )
-        for name in ("oracle_bf16_from_double", "oracle_bf16_to_double", "oracle_f16_to_double"):
+        L.oracle_inject_ex.restype = i32
+        L.oracle_inject_ex.argtypes = L.oracle_inject.argtypes + [i32, C.c_float, C.c_float, p, p]
+        L.oracle_rope_rows_partial.restype = i32
+        L.oracle_rope_rows_partial.argtypes = [p, i64, i32, i32, p, dbl, i32, p, p]
+        L.oracle_inv_freq_llama3.restype = i32
+        L.oracle_inv_freq_llama3.argtypes = [i32, dbl, dbl, dbl, dbl, dbl, p]
+        for name in ("oracle_bf16_from_double", "oracle_bf16_to_double", "oracle_f16_to_double", "oracle_e4m3_from_double",
+                     "oracle_e4m3_to_double"):  # fmt: skip
             getattr(L, name).restype = None
             getattr(L, name).argtypes = [p, i64, p]
         _lib = L
@@ -118,6 +125,21 @@ def f16_to_double(x: np.ndarray) -> np.ndarray:
     return out
 
 
+def e4m3_from_double(x: np.ndarray) -> np.ndarray:
+    """Round to the 8-bit e4m3 format (nearest even, one step, saturating at +-448)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(x.shape, dtype=np.uint8)
+    lib().oracle_e4m3_from_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def e4m3_to_double(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.uint8)
+    out = np.empty(x.shape, dtype=np.float64)
+    lib().oracle_e4m3_to_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
 def scores(emb: np.ndarray, query: np.ndarray, n_threads: int = 0) -> np.ndarray:
     """Double-precision inner product of one query with every row of ``emb``."""
     emb = np.ascontiguousarray(emb)
@@ -159,16 +181,30 @@ def inv_freq(D: int, theta: float) -> np.ndarray:
     return out
 
 
-def rope_rows(x: np.ndarray, pos: np.ndarray, theta: float, style: int = 0, inv_freq_override=None) -> np.ndarray:
-    """Rotate rows of ``x`` ([n, D] float64), row r at position ``pos[r]``."""
+def inv_freq_llama3(R: int, theta: float, factor=8.0, low_freq_factor=1.0, high_freq_factor=4.0, original_max=8192.0) -> np.ndarray:
+    """The rescaled frequency table of the Llama-3.1 family for a rotary dimension ``R``."""
+    out = np.empty(R // 2, dtype=np.float32)
+    rc = lib().oracle_inv_freq_llama3(R, float(theta), float(factor), float(low_freq_factor), float(high_freq_factor),
+                                      float(original_max), _ptr(out))  # fmt: skip
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def rope_rows(x: np.ndarray, pos: np.ndarray, theta: float, style: int = 0, inv_freq_override=None, rotary_dim: int = 0) -> np.ndarray:
+    """Rotate rows of ``x`` ([n, D] float64), row r at position ``pos[r]``; ``rotary_dim``: only the first
+    so many coordinates rotate (0 = all)."""
     x = np.ascontiguousarray(x, dtype=np.float64)
     n, D = x.shape
     pos = np.ascontiguousarray(np.broadcast_to(np.asarray(pos, dtype=np.int64), (n,)))
     if inv_freq_override is not None:
         inv_freq_override = np.ascontiguousarray(inv_freq_override, dtype=np.float32)
-        assert inv_freq_override.size == D // 2
+        assert inv_freq_override.size == (rotary_dim or D) // 2
     y = np.empty_like(x)
-    rc = lib().oracle_rope_rows(_ptr(x), n, D, _ptr(pos), float(theta), style, _ptr(inv_freq_override), _ptr(y))
+    if rotary_dim:
+        rc = lib().oracle_rope_rows_partial(_ptr(x), n, D, rotary_dim, _ptr(pos), float(theta), style, _ptr(inv_freq_override), _ptr(y))
+    else:
+        rc = lib().oracle_rope_rows(_ptr(x), n, D, _ptr(pos), float(theta), style, _ptr(inv_freq_override), _ptr(y))
     if rc:
         raise OracleError(rc)
     return y
@@ -197,8 +233,9 @@ def slots(ids, fact_len, start_pos, block_table, bs, num_blocks):
 class InjectResult:
     """m, slots [m], k_ref float64 / k_bf16 uint16 / v uint16, each [nl, m, H, D]."""
 
-    def __init__(self, m, slots, k_ref, k_bf16, v):
+    def __init__(self, m, slots, k_ref, k_bf16, v, k_fp8=None, v_fp8=None):
         self.m, self.slots, self.k_ref, self.k_bf16, self.v = m, slots, k_ref, k_bf16, v
+        self.k_fp8, self.v_fp8 = k_fp8, v_fp8  # uint8 e4m3 codes of K / k_scale and V / v_scale, when scales were given
 
 
 def inject(
@@ -220,12 +257,17 @@ def inject(
     v_cache=None,
     cache_strides=None,
     n_threads=0,
+    rotary_dim=0,
+    k_scale=None,
+    v_scale=None,
 ) -> InjectResult:
     """Compose facts ``ids`` (placement order) at ``start_pos`` and place them through ``block_table``.
 
     ``k_pre`` / ``v``: uint16 (bf16 bits) arrays [n_layers, store_tokens, H, D] on the host.
     ``k_cache`` / ``v_cache``: optional uint16 host images of the paged cache, written in place using
     ``cache_strides = (layer, block, token, head)`` in elements.
+    ``rotary_dim``: only the first so many coordinates of a head rotate (0 = all).  ``k_scale`` / ``v_scale``:
+    also return the e4m3 codes of an 8-bit cache that holds K / k_scale and V / v_scale.
     """
     ids = np.ascontiguousarray(ids, dtype=np.int32).reshape(-1)
     fact_offset = np.ascontiguousarray(fact_offset, dtype=np.int64)
@@ -253,13 +295,16 @@ def inject(
         strides = tuple(int(s) for s in cache_strides)
         for c_ in (k_cache, v_cache):
             assert c_ is None or (c_.dtype == np.uint16 and c_.flags.c_contiguous)
-    rc = lib().oracle_inject(
+    k_fp8 = np.empty(shape, dtype=np.uint8) if k_scale is not None else None
+    v_fp8 = np.empty(shape, dtype=np.uint8) if v_scale is not None else None
+    rc = lib().oracle_inject_ex(
         _ptr(ids), ids.size, fact_len.size, _ptr(fact_offset), _ptr(fact_len), _ptr(k_pre), _ptr(v), store_tokens,
         n_layers, H, D, float(theta), style, _ptr(inv_freq_override), int(start_pos), _ptr(block_table),
         block_table.size, bs, num_blocks, l0, l1, C.byref(m), _ptr(slots), _ptr(k_ref), _ptr(k_bf16), _ptr(v_out),
-        _ptr(k_cache), _ptr(v_cache), *strides, n_threads,
+        _ptr(k_cache), _ptr(v_cache), *strides, n_threads, int(rotary_dim), float(k_scale or 0.0), float(v_scale or 0.0),
+        _ptr(k_fp8), _ptr(v_fp8),
     )  # fmt: skip
     if rc:
         raise OracleError(rc)
     assert m.value == m_guess
-    return InjectResult(m.value, slots, k_ref, k_bf16, v_out)
+    return InjectResult(m.value, slots, k_ref, k_bf16, v_out, k_fp8, v_fp8)

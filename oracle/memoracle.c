@@ -26,9 +26,13 @@
  *   - V is stored raw and copied unchanged (Sec. 5.1, closing paragraph).
  *   - bytes per fact:   "Storage cost" (Sec. 3.5): 2 * L * c * h * d * b.
  *
+ *   - variants beyond the paper's text (its evaluation spans "RoPE parameterizations", Sec. 6.1): the
+ *     Llama-3.1 rescaled frequency table, rotation of only the first R coordinates of a head, and an
+ *     8-bit e4m3 cache image with per-tensor scales.
+ *
  * Parity pins: every exported function is pinned by the CPU tests
  * (closed forms, group law, brute-force joint rotation, numpy float64
- * cross-checks, full-sort comparison); none is "parity unpinned".
+ * cross-checks, full-sort comparison, exhaustive e4m3 code tables); none is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -92,6 +96,48 @@ static uint16_t double_to_bf16_rne(double x) {
   uint32_t u;
   memcpy(&u, &f, 4);
   return sign | (uint16_t)(u >> 16);
+}
+
+/*
+ * 8-bit float "e4m3" as used for quantised KV caches: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits, no
+ * infinities, exponent 15 with mantissa 7 is NaN, so the largest finite value is 1.75 * 2^8 = 448; subnormals are
+ * multiples of 2^-9.  Decoding is exact.
+ */
+static double e4m3_to_double(uint8_t c) {
+  int e = (c >> 3) & 15, m = c & 7;
+  double v;
+  if (e == 15 && m == 7) return NAN;
+  v = e == 0 ? ldexp((double)m, -9) : ldexp(1.0 + (double)m / 8.0, e - 7);
+  return (c & 0x80) ? -v : v;
+}
+
+/* double -> e4m3, round to nearest even in ONE step, saturating to +-448 (no NaN is produced from a finite input). */
+static uint8_t double_to_e4m3_rne_sat(double x) {
+  uint8_t sign = signbit(x) ? 0x80 : 0;
+  double a = fabs(x);
+  int e;
+  double q;
+  if (isnan(x)) return 0x7f;
+  if (a >= 448.0) return (uint8_t)(sign | 0x7e);
+  if (a < ldexp(1.0, -6)) {            /* subnormal range: spacing 2^-9 */
+    q = rint(ldexp(a, 9));             /* 0..8, ties to even */
+    return (uint8_t)(sign | (uint8_t)q); /* q == 8 is the code of the smallest normal, 2^-6 */
+  }
+  (void)frexp(a, &e);                  /* a = f * 2^e, f in [0.5, 1)  ->  a in [2^(e-1), 2^e) */
+  e -= 1;
+  q = rint((ldexp(a, -e) - 1.0) * 8.0); /* 0..8 */
+  if (q == 8.0) {
+    q = 0.0;
+    e += 1;
+  }
+  return (uint8_t)(sign | (uint8_t)(((e + 7) << 3) | (int)q));
+}
+
+void oracle_e4m3_from_double(const double* x, int64_t n, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = double_to_e4m3_rne_sat(x[i]);
+}
+void oracle_e4m3_to_double(const uint8_t* x, int64_t n, double* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = e4m3_to_double(x[i]);
 }
 
 void oracle_bf16_from_double(const double* x, int64_t n, uint16_t* out) {
@@ -214,12 +260,13 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
 /* ---------------------------------------------------------------- RoPE */
 
 /*
- * Frequency of pair i: theta^(-2i/D), evaluated in double and rounded ONCE to
- * binary32 (models keep this vector in fp32).  An override vector replaces it.
+ * Frequency of pair i: theta^(-2i/R) for a rotary dimension R (the whole head unless the model rotates only the
+ * first R coordinates), evaluated in double and rounded ONCE to binary32 (models keep this vector in fp32).  An
+ * override vector replaces it.
  */
-static double pair_freq(int i, int D, double theta, const float* inv_freq_override) {
+static double pair_freq(int i, int R, double theta, const float* inv_freq_override) {
   if (inv_freq_override) return (double)inv_freq_override[i];
-  return (double)(float)pow(theta, -(double)(2 * i) / (double)D);
+  return (double)(float)pow(theta, -(double)(2 * i) / (double)R);
 }
 
 void oracle_inv_freq(int D, double theta, float* out) {
@@ -227,30 +274,67 @@ void oracle_inv_freq(int D, double theta, float* out) {
 }
 
 /*
- * Rotate one head vector x[0..D) at position pos into y.
- * style 0 (half-split): pair i is (x[i], x[i + D/2]);  style 1 (interleaved): (x[2i], x[2i+1]).
+ * The rescaled frequency table of the Llama-3.1 family ("the model's own rotary tables", Sec. 3.3; the primary
+ * model of the evaluation, Sec. 6.1): a pair whose wavelength 2*pi/f exceeds original_max / low_freq_factor is
+ * slowed down by `factor`, one whose wavelength is below original_max / high_freq_factor is kept, and in between
+ * the two are blended linearly in  s = (original_max / wavelength - low_freq_factor) / (high - low).
+ * Computed in double from the unrounded theta^(-2i/R) and rounded once to binary32.
+ */
+int oracle_inv_freq_llama3(int R, double theta, double factor, double low_freq_factor, double high_freq_factor,
+                           double original_max, float* out) {
+  const double two_pi = 6.283185307179586476925286766559;
+  if (R <= 0 || (R & 1) || !out || !(factor > 0) || !(high_freq_factor > low_freq_factor) || !(original_max > 0))
+    return ORACLE_ERR_ARG;
+  for (int i = 0; i < R / 2; ++i) {
+    double f = pow(theta, -(double)(2 * i) / (double)R);
+    double wavelen = two_pi / f;
+    double g;
+    if (wavelen > original_max / low_freq_factor) {
+      g = f / factor;
+    } else if (wavelen < original_max / high_freq_factor) {
+      g = f;
+    } else {
+      double sm = (original_max / wavelen - low_freq_factor) / (high_freq_factor - low_freq_factor);
+      g = (1.0 - sm) * f / factor + sm * f;
+    }
+    out[i] = (float)g;
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Rotate one head vector x[0..D) at position pos into y.  Only the first R coordinates rotate (R = D for the
+ * models of the paper; R < D is the "partial rotary" parameterisation); the rest is copied.
+ * style 0 (half-split): pair i is (x[i], x[i + R/2]);  style 1 (interleaved): (x[2i], x[2i+1]);  i < R/2.
  * (x1, x2) -> (x1 cos a - x2 sin a,  x2 cos a + x1 sin a),  a = pos * freq_i.
  */
-static void rope_head(const double* x, double* y, int D, int64_t pos, double theta, int style,
+static void rope_head(const double* x, double* y, int D, int R, int64_t pos, double theta, int style,
                       const float* inv_freq_override) {
-  int half = D / 2;
+  int half = R / 2;
   for (int i = 0; i < half; ++i) {
     int i1 = style == 0 ? i : 2 * i;
     int i2 = style == 0 ? i + half : 2 * i + 1;
-    double angle = (double)pos * pair_freq(i, D, theta, inv_freq_override);
+    double angle = (double)pos * pair_freq(i, R, theta, inv_freq_override);
     double c = cos(angle), s = sin(angle);
     double x1 = x[i1], x2 = x[i2];
     y[i1] = x1 * c - x2 * s;
     y[i2] = x2 * c + x1 * s;
   }
+  for (int d = R; d < D; ++d) y[d] = x[d];
 }
 
-/* Rotate n_rows independent head vectors (row r at position pos[r]). */
+/* Rotate n_rows independent head vectors (row r at position pos[r]); rotary_dim = 0 means the whole head. */
+int oracle_rope_rows_partial(const double* x, int64_t n_rows, int D, int rotary_dim, const int64_t* pos, double theta,
+                             int style, const float* inv_freq_override, double* y) {
+  int R = rotary_dim ? rotary_dim : D;
+  if (!x || !y || !pos || D <= 0 || R <= 0 || R > D || (R & 1) || (style != 0 && style != 1)) return ORACLE_ERR_ARG;
+  for (int64_t r = 0; r < n_rows; ++r) rope_head(x + r * D, y + r * D, D, R, pos[r], theta, style, inv_freq_override);
+  return ORACLE_OK;
+}
 int oracle_rope_rows(const double* x, int64_t n_rows, int D, const int64_t* pos, double theta, int style,
                      const float* inv_freq_override, double* y) {
-  if (!x || !y || !pos || D <= 0 || (D & 1) || (style != 0 && style != 1)) return ORACLE_ERR_ARG;
-  for (int64_t r = 0; r < n_rows; ++r) rope_head(x + r * D, y + r * D, D, pos[r], theta, style, inv_freq_override);
-  return ORACLE_OK;
+  if (D & 1) return ORACLE_ERR_ARG;
+  return oracle_rope_rows_partial(x, n_rows, D, 0, pos, theta, style, inv_freq_override, y);
 }
 
 /* ---------------------------------------------------------------- injection */
@@ -271,18 +355,30 @@ int oracle_rope_rows(const double* x, int64_t n_rows, int D, const int64_t* pos,
  *   k_cache / v_cache            a host image of the paged cache (bf16), written in place at
  *                                layer*layer_stride + block*block_stride + (slot % bs)*token_stride
  *                                + head*head_stride + d   (strides in elements; layer = absolute index)
+ *
+ * Variants of the model / cache parameterisation (defaults reproduce the plain path):
+ *   rotary_dim       0 = the whole head, else only the first rotary_dim coordinates of a head rotate
+ *   k_scale, v_scale quantised (e4m3) cache: the cache holds x / scale.  Used only for out_k_fp8 / out_v_fp8
+ *                    [nl][m][H][D] bytes, both optional:
+ *                      K: the rotated key in double times inv, inv = (double)(1.0f / k_scale), rounded once to e4m3;
+ *                      V: the stored bf16 value times 1.0f / v_scale as a binary32 product (the arithmetic type
+ *                         of the path), then rounded once to e4m3.
  * Returns ORACLE_OK or a negative error; on error the outputs are unspecified.
  */
-int oracle_inject(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
-                  const uint16_t* k_pre, const uint16_t* v, int64_t store_tokens, int n_layers, int H, int D,
-                  double theta, int style, const float* inv_freq_override, int64_t start_pos,
-                  const int32_t* block_table, int64_t n_table, int bs, int64_t num_blocks, int layer_begin,
-                  int layer_end, int64_t* out_m, int64_t* out_slots, double* out_k_ref, uint16_t* out_k_bf16,
-                  uint16_t* out_v, uint16_t* k_cache, uint16_t* v_cache, int64_t layer_stride, int64_t block_stride,
-                  int64_t token_stride, int64_t head_stride, int n_threads) {
+int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
+                     const uint16_t* k_pre, const uint16_t* v, int64_t store_tokens, int n_layers, int H, int D,
+                     double theta, int style, const float* inv_freq_override, int64_t start_pos,
+                     const int32_t* block_table, int64_t n_table, int bs, int64_t num_blocks, int layer_begin,
+                     int layer_end, int64_t* out_m, int64_t* out_slots, double* out_k_ref, uint16_t* out_k_bf16,
+                     uint16_t* out_v, uint16_t* k_cache, uint16_t* v_cache, int64_t layer_stride, int64_t block_stride,
+                     int64_t token_stride, int64_t head_stride, int n_threads, int rotary_dim, float k_scale,
+                     float v_scale, uint8_t* out_k_fp8, uint8_t* out_v_fp8) {
+  const int R = rotary_dim ? rotary_dim : D;
   if (!out_m || k < 0 || (k > 0 && !ids) || !fact_offset || !fact_len || H <= 0 || D <= 0 || (D & 1) || D > 1024 ||
-      bs <= 0)
+      bs <= 0 || R <= 0 || R > D || (R & 1))
     return ORACLE_ERR_ARG;
+  if ((out_k_fp8 && !(k_scale > 0.0f)) || (out_v_fp8 && !(v_scale > 0.0f))) return ORACLE_ERR_ARG;
+  const float k_inv = out_k_fp8 ? 1.0f / k_scale : 0.0f, v_inv = out_v_fp8 ? 1.0f / v_scale : 0.0f;
   if (layer_begin < 0 || layer_end > n_layers || layer_begin > layer_end) return ORACLE_ERR_ARG;
   if (start_pos < 0) return ORACLE_ERR_ARG;
 
@@ -348,13 +444,15 @@ int oracle_inject(const int32_t* ids, int k, int64_t n_facts, const int64_t* fac
       int64_t cbase = (int64_t)l * layer_stride + blk * block_stride + inb * token_stride;
       for (int h = 0; h < H; ++h) {
         for (int d = 0; d < D; ++d) xin[d] = bf16_to_double(ksrc[h * D + d]);
-        rope_head(xin, yout, D, pos, theta, style, inv_freq_override);
+        rope_head(xin, yout, D, R, pos, theta, style, inv_freq_override);
         for (int d = 0; d < D; ++d) {
           uint16_t kb = double_to_bf16_rne(yout[d]);
           uint16_t vb = vsrc[h * D + d];
           if (out_k_ref) out_k_ref[o + h * D + d] = yout[d];
           if (out_k_bf16) out_k_bf16[o + h * D + d] = kb;
           if (out_v) out_v[o + h * D + d] = vb;
+          if (out_k_fp8) out_k_fp8[o + h * D + d] = double_to_e4m3_rne_sat(yout[d] * (double)k_inv);
+          if (out_v_fp8) out_v_fp8[o + h * D + d] = double_to_e4m3_rne_sat((double)(float)(bf16_to_double(vb) * (double)v_inv));
           if (k_cache) k_cache[cbase + h * head_stride + d] = kb;
           if (v_cache) v_cache[cbase + h * head_stride + d] = vb;
         }
@@ -364,4 +462,18 @@ int oracle_inject(const int32_t* ids, int k, int64_t n_facts, const int64_t* fac
   free(src);
   free(slots);
   return ORACLE_OK;
+}
+
+/* The plain path: every coordinate rotates, bf16 cache. */
+int oracle_inject(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
+                  const uint16_t* k_pre, const uint16_t* v, int64_t store_tokens, int n_layers, int H, int D,
+                  double theta, int style, const float* inv_freq_override, int64_t start_pos,
+                  const int32_t* block_table, int64_t n_table, int bs, int64_t num_blocks, int layer_begin,
+                  int layer_end, int64_t* out_m, int64_t* out_slots, double* out_k_ref, uint16_t* out_k_bf16,
+                  uint16_t* out_v, uint16_t* k_cache, uint16_t* v_cache, int64_t layer_stride, int64_t block_stride,
+                  int64_t token_stride, int64_t head_stride, int n_threads) {
+  return oracle_inject_ex(ids, k, n_facts, fact_offset, fact_len, k_pre, v, store_tokens, n_layers, H, D, theta, style,
+                          inv_freq_override, start_pos, block_table, n_table, bs, num_blocks, layer_begin, layer_end, out_m,
+                          out_slots, out_k_ref, out_k_bf16, out_v, k_cache, v_cache, layer_stride, block_stride,
+                          token_stride, head_stride, n_threads, 0, 0.0f, 0.0f, NULL, NULL);
 }
