@@ -92,7 +92,23 @@ typedef struct {
   void* kv_arena;         /* optional caller-provided DEVICE buffer for the arena, else NULL */
   size_t kv_arena_bytes;  /* its size; must be >= memstore_arena_bytes(config) */
   int64_t max_host_kv_tokens; /* capacity in tokens of the second K/V arena in pinned HOST memory (0: none), < 2^30 */
+  int32_t rotary_dim;     /* R: only the first R coordinates of a head rotate (pairs (i, i+R/2) or (2i, 2i+1), i < R/2,
+                             frequencies theta^(-2i/R); the rest is copied).  0 = head_dim, the paper's models; else a
+                             multiple of 16, <= head_dim.  inv_freq_override then holds R/2 floats. */
+  int32_t reserved1;      /* 0 */
 } memstore_config;
+
+/*
+ * The rescaled frequency table of the Llama-3.1 family, the paper's primary model ("the model's own rotary
+ * tables", Sec. 3.3; Sec. 6.1): pair i of an R-dimensional rotation starts from f = theta^(-2i/R); a wavelength
+ * 2*pi/f above original_max_position / low_freq_factor is slowed down by `factor`, one below
+ * original_max_position / high_freq_factor is kept, and in between the two are blended linearly in
+ * (original_max_position / wavelength - low_freq_factor) / (high_freq_factor - low_freq_factor).  Evaluated in
+ * double, rounded once to fp32.  Pure host arithmetic: out (host, R/2 floats) is meant for inv_freq_override.
+ * Llama-3.1: factor 8, low 1, high 4, original_max_position 8192.
+ */
+ms_status memstore_rope_table_llama3(int32_t rotary_dim, double rope_theta, double factor, double low_freq_factor,
+                                     double high_freq_factor, double original_max_position, float* out);
 
 /* Bytes of the K/V arena for this configuration: 2 * L * max_kv_tokens * h * d * 2
  * (the paper's storage formula, Sec. 3.5, with c = max_kv_tokens and bf16). */
@@ -178,10 +194,17 @@ ms_status memstore_retrieve(memstore_t* store, const void* queries, const int32_
 ms_status memstore_retrieve_static(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq,
                                    int32_t k, int32_t* out_ids, float* out_scores, ms_stream stream);
 
-/* A caller-owned paged KV cache, bf16, described by strides in ELEMENTS:
+/* element type of the paged cache */
+enum {
+  MS_CACHE_BF16 = 0,    /* the paper's cache */
+  MS_CACHE_FP8_E4M3 = 1 /* one byte per element: sign, 4 exponent bits (bias 7), 3 mantissa bits, finite maximum 448 */
+};
+
+/* A caller-owned paged KV cache, bf16 unless dtype says otherwise, described by strides in ELEMENTS:
  *   element (layer, block, token-in-block, head, d) of K is at
  *   k_base[layer*layer_stride + block*block_stride + token*token_stride + head*head_stride + d]
  * and the same for V from v_base.  All strides must be multiples of 8 and the bases 16-byte aligned.
+ * An 8-bit cache takes half the write traffic; its strides are still counted in elements (= bytes).
  * This covers separate K/V planes, stacked planes, token-major and head-major blocks. */
 typedef struct {
   void* k_base;
@@ -189,7 +212,10 @@ typedef struct {
   int64_t layer_stride, block_stride, token_stride, head_stride;
   int64_t num_blocks;
   int32_t block_size;
-  int32_t reserved0;
+  int32_t dtype;            /* MS_CACHE_BF16 (0) or MS_CACHE_FP8_E4M3 */
+  float k_scale, v_scale;   /* MS_CACHE_FP8_E4M3 only, both > 0: the cache holds K / k_scale and V / v_scale (per-tensor
+                               scales).  The rotated key (fp32) and the stored value are multiplied by 1.0f / scale in
+                               fp32 and rounded once, to nearest even, saturating at +-448. */
 } ms_paged_cache;
 
 /*

@@ -360,9 +360,12 @@ int oracle_rope_rows(const double* x, int64_t n_rows, int D, const int64_t* pos,
  *   rotary_dim       0 = the whole head, else only the first rotary_dim coordinates of a head rotate
  *   k_scale, v_scale quantised (e4m3) cache: the cache holds x / scale.  Used only for out_k_fp8 / out_v_fp8
  *                    [nl][m][H][D] bytes, both optional:
- *                      K: the rotated key in double times inv, inv = (double)(1.0f / k_scale), rounded once to e4m3;
- *                      V: the stored bf16 value times 1.0f / v_scale as a binary32 product (the arithmetic type
- *                         of the path), then rounded once to e4m3.
+ *                      the value (rotated key in double, or stored bf16 value) times 1.0f / scale is first
+ *                      rounded to binary32, the arithmetic type of the path in which the code is decided, and that
+ *                      binary32 number is rounded once to e4m3.  (For V and for unrotated key coordinates the
+ *                      operands are bf16 and binary32, so the binary32 product is fully determined; short bf16
+ *                      mantissas make exact e4m3 ties common there, and deciding them in another precision would
+ *                      flip a sizeable share of codes.)
  * Returns ORACLE_OK or a negative error; on error the outputs are unspecified.
  */
 int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
@@ -451,7 +454,7 @@ int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* 
           if (out_k_ref) out_k_ref[o + h * D + d] = yout[d];
           if (out_k_bf16) out_k_bf16[o + h * D + d] = kb;
           if (out_v) out_v[o + h * D + d] = vb;
-          if (out_k_fp8) out_k_fp8[o + h * D + d] = double_to_e4m3_rne_sat(yout[d] * (double)k_inv);
+          if (out_k_fp8) out_k_fp8[o + h * D + d] = double_to_e4m3_rne_sat((double)(float)(yout[d] * (double)k_inv));
           if (out_v_fp8) out_v_fp8[o + h * D + d] = double_to_e4m3_rne_sat((double)(float)(bf16_to_double(vb) * (double)v_inv));
           if (k_cache) k_cache[cbase + h * head_stride + d] = kb;
           if (v_cache) v_cache[cbase + h * head_stride + d] = vb;

@@ -18,6 +18,7 @@ struct InjectParams {
   int64_t host_tokens;
   const float* inv_freq;  // [D/2]
   int32_t n_layers, n_heads, head_dim, rope_style;
+  int32_t rotary_dim;  // first coordinates of a head that rotate (a multiple of 16, <= head_dim)
   int32_t max_position;
   // request
   const int32_t* fact_ids;  // [nreq][k]
@@ -32,6 +33,7 @@ struct InjectParams {
   __nv_bfloat16* v_cache;
   int64_t layer_stride, block_stride, token_stride, head_stride, num_blocks;
   int32_t block_size;
+  float k_inv_scale, v_inv_scale;  // 8-bit cache: 1.0f / scale of K and V
   // outputs
   int32_t* out_n_tokens;
   int32_t* out_status;
@@ -259,6 +261,57 @@ __device__ __forceinline__ void rotate_unit(uint4& a, uint4& b, const float* sn,
   }
 }
 
+// Eight fp32 values -> eight e4m3 bytes (round to nearest even, saturating), lowest address first.
+__device__ __forceinline__ uint2 pack_e4m3x8(const float* f) {
+  uint32_t w[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(f[4 * h], f[4 * h + 1]), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(f[4 * h + 2], f[4 * h + 3]), __NV_SATFINITE, __NV_E4M3);
+    w[h] = lo | (hi << 16);
+  }
+  return make_uint2(w[0], w[1]);
+}
+
+// The 8 bf16 values of a 16-byte vector times `scale` (one fp32 rounding each).
+__device__ __forceinline__ void scaled_floats(const uint4& a, float scale, float* f) {
+  const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    f[2 * w] = __fmul_rn(bf16lo(aw[w]), scale);
+    f[2 * w + 1] = __fmul_rn(bf16hi(aw[w]), scale);
+  }
+}
+
+// rotate_unit with fp32 results (times `scale`) instead of packed bf16: fa = the 8 elements of vector a, fb of b.
+template <int STYLE>
+__device__ __forceinline__ void rotate_unit_f32(const uint4& a, const uint4& b, const float* sn, const float* cs, float scale,
+                                                float* fa, float* fb) {
+  const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
+  const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b);
+  if (STYLE == 0) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float x1l = bf16lo(aw[w]), x1h = bf16hi(aw[w]);
+      const float x2l = bf16lo(bw[w]), x2h = bf16hi(bw[w]);
+      fa[2 * w] = (x1l * cs[2 * w] - x2l * sn[2 * w]) * scale;
+      fb[2 * w] = (x2l * cs[2 * w] + x1l * sn[2 * w]) * scale;
+      fa[2 * w + 1] = (x1h * cs[2 * w + 1] - x2h * sn[2 * w + 1]) * scale;
+      fb[2 * w + 1] = (x2h * cs[2 * w + 1] + x1h * sn[2 * w + 1]) * scale;
+    }
+  } else {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float x1 = bf16lo(aw[w]), x2 = bf16hi(aw[w]);
+      fa[2 * w] = (x1 * cs[w] - x2 * sn[w]) * scale;
+      fa[2 * w + 1] = (x2 * cs[w] + x1 * sn[w]) * scale;
+      const float z1 = bf16lo(bw[w]), z2 = bf16hi(bw[w]);
+      fb[2 * w] = (z1 * cs[4 + w] - z2 * sn[4 + w]) * scale;
+      fb[2 * w + 1] = (z2 * cs[4 + w] + z1 * sn[4 + w]) * scale;
+    }
+  }
+}
+
 constexpr int kCopyThreads = 256;
 constexpr int kThreadsPerToken = kCopyThreads / kTileTokens;  // 32
 constexpr int kUnitsPerThread = 2;
@@ -276,7 +329,11 @@ constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a
 // octet): two 16-byte vectors of K (rotated) and the same two of V (copied).  32 and 64 are multiples of D/16, so
 // both units of a thread share the frequency octet: its 8 cos/sin pairs are computed once, while the loads fly.
 // ------------------------------------------------------------------------------------------------
-template <int STYLE>
+//
+// Variants: when only the first R < D coordinates rotate, octets j >= R/16 of a head are plain copies (for both pair
+// styles their two vectors are the 32 contiguous bytes at element 16 j).  FP8 = true writes an 8-bit e4m3 cache:
+// rotated keys and values are scaled in fp32 and rounded once; a thread then stores two 8-byte vectors per row.
+template <int STYLE, bool FP8>
 __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const InjectParams p) {
   const int tid = threadIdx.x;
   const int tk = tid >> 5;  // token of the tile
@@ -285,9 +342,11 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
   const int G = D >> 4, g_shift = 31 - __clz(G);  // frequency octets per head (a power of two, at most 16)
   const int n_units = p.n_heads << g_shift;
   const int j = l & (G - 1);
+  const int R = p.rotary_dim;
+  const bool rotates = 16 * j < R;
   // element offsets of this thread's two vectors inside a head
-  const int offA = STYLE == 0 ? 8 * j : 16 * j;
-  const int offB = STYLE == 0 ? D / 2 + 8 * j : 16 * j + 8;
+  const int offA = (STYLE == 0 && rotates) ? 8 * j : 16 * j;
+  const int offB = (STYLE == 0 && rotates) ? R / 2 + 8 * j : 16 * j + 8;
   const int u0 = blockIdx.y * kUnitsPerPart + l;
   if (u0 >= n_units) return;
 
@@ -328,20 +387,40 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
     // cos/sin of (pos, 8 frequencies), evaluated while the loads are in flight
     float sn[8], cs[8];
     const float posf = (float)pos;
+    if (rotates) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
+      for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
+    }
 #pragma unroll
     for (int u = 0; u < kUnitsPerThread; ++u) {
       const int unit = u0 + u * kThreadsPerToken;
       if (unit < n_units) {
         const int h = unit >> g_shift;
-        rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
-        __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
-        st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
-        st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
-        __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
-        st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
-        st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
+        if (!FP8) {
+          if (rotates) rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+          __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
+          st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
+          st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
+          __nv_bfloat16* vd = p.v_cache + dbase + (int64_t)h * p.head_stride;
+          st_stream(reinterpret_cast<uint4*>(vd + offA), va[u]);
+          st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
+        } else {
+          float fa[8], fb[8];
+          if (rotates) {
+            rotate_unit_f32<STYLE>(ka[u], kb[u], sn, cs, p.k_inv_scale, fa, fb);
+          } else {
+            scaled_floats(ka[u], p.k_inv_scale, fa);
+            scaled_floats(kb[u], p.k_inv_scale, fb);
+          }
+          uint8_t* kd = reinterpret_cast<uint8_t*>(p.k_cache) + dbase + (int64_t)h * p.head_stride;
+          st_stream8(reinterpret_cast<uint2*>(kd + offA), pack_e4m3x8(fa));
+          st_stream8(reinterpret_cast<uint2*>(kd + offB), pack_e4m3x8(fb));
+          scaled_floats(va[u], p.v_inv_scale, fa);
+          scaled_floats(vb[u], p.v_inv_scale, fb);
+          uint8_t* vd = reinterpret_cast<uint8_t*>(p.v_cache) + dbase + (int64_t)h * p.head_stride;
+          st_stream8(reinterpret_cast<uint2*>(vd + offA), pack_e4m3x8(fa));
+          st_stream8(reinterpret_cast<uint2*>(vd + offB), pack_e4m3x8(fb));
+        }
       }
     }
   }

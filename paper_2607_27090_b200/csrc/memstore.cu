@@ -125,6 +125,7 @@ ms_status check_config(const memstore_config* c) {
   // the copy kernels give 32 or more threads to a token and one frequency octet to a thread: d/16 must divide 32
   const int d = c->head_dim;
   if (!(d == 16 || d == 32 || d == 64 || d == 128 || d == 256)) return MS_ERR_UNSUPPORTED;
+  if (c->rotary_dim < 0 || c->rotary_dim > d || (c->rotary_dim % 16) || c->reserved1 != 0) return MS_ERR_INVALID_ARG;
   if (c->max_host_kv_tokens < 0 || c->max_host_kv_tokens >= (1ll << 30) || c->max_kv_tokens >= (1ll << 30) || (int64_t)c->n_users * c->max_facts_per_user >= (1ll << 31))
     return MS_ERR_UNSUPPORTED;
   return MS_OK;
@@ -285,6 +286,28 @@ size_t memstore_arena_bytes(const memstore_config* c) {
   return (size_t)2 * c->n_layers * (size_t)c->max_kv_tokens * c->n_kv_heads * c->head_dim * sizeof(__nv_bfloat16);
 }
 
+ms_status memstore_rope_table_llama3(int32_t rotary_dim, double rope_theta, double factor, double low_freq_factor,
+                                     double high_freq_factor, double original_max_position, float* out) {
+  if (rotary_dim <= 0 || (rotary_dim & 1) || !out || !(rope_theta > 0.0) || !(factor > 0.0) ||
+      !(high_freq_factor > low_freq_factor) || !(low_freq_factor > 0.0) || !(original_max_position > 0.0))
+    return MS_ERR_INVALID_ARG;
+  const double kTwoPi = 6.283185307179586476925286766559;
+  const double long_wave = original_max_position / low_freq_factor, short_wave = original_max_position / high_freq_factor;
+  for (int i = 0; i < rotary_dim / 2; ++i) {
+    const double f = std::pow(rope_theta, -(double)(2 * i) / (double)rotary_dim);
+    const double wave = kTwoPi / f;
+    double g = f;
+    if (wave > long_wave) {
+      g = f / factor;
+    } else if (!(wave < short_wave)) {
+      const double t = (original_max_position / wave - low_freq_factor) / (high_freq_factor - low_freq_factor);
+      g = (1.0 - t) * f / factor + t * f;
+    }
+    out[i] = (float)g;
+  }
+  return MS_OK;
+}
+
 ms_status memstore_create(const memstore_config* config, memstore_t** out) {
   if (out) *out = nullptr;
   if (!out) return MS_ERR_INVALID_ARG;
@@ -344,11 +367,13 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
     cudaGetLastError();
     return bail(MS_ERR_OOM);
   }
-  // RoPE frequencies: theta^(-2i/d) in double, rounded once to fp32 (Sec. 2.4; models keep this vector in fp32)
-  std::vector<float> f(config->head_dim / 2);
-  for (int i = 0; i < config->head_dim / 2; ++i)
-    f[i] = config->inv_freq_override ? config->inv_freq_override[i]
-                                     : (float)std::pow(config->rope_theta, -(double)(2 * i) / (double)config->head_dim);
+  // RoPE frequencies: theta^(-2i/R) in double, rounded once to fp32 (Sec. 2.4; models keep this vector in fp32);
+  // R = the rotary dimension, the whole head unless the configuration says otherwise.  Entries beyond R/2 are unused.
+  if (s->cfg.rotary_dim == 0) s->cfg.rotary_dim = config->head_dim;
+  const int R = s->cfg.rotary_dim;
+  std::vector<float> f(config->head_dim / 2, 0.f);
+  for (int i = 0; i < R / 2; ++i)
+    f[i] = config->inv_freq_override ? config->inv_freq_override[i] : (float)std::pow(config->rope_theta, -(double)(2 * i) / (double)R);
   ok = cudaMemcpy(s->inv_freq_d, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
        cudaMemset(s->user_count_d, 0, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
        cudaMemset(s->ctrl, 0, 2 * sizeof(InjectCtrl)) == cudaSuccess &&
@@ -360,7 +385,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
   s->user_count.assign(config->n_users, 0);
   s->tma_path = (config->flags & MS_STORE_TMA_COPY_PATH) != 0 && config->max_host_kv_tokens == 0;  // HBM arena only
   int occ = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0>, kCopyThreads, 0) == cudaSuccess && occ > 0)
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0, false>, kCopyThreads, 0) == cudaSuccess && occ > 0)
     s->copy_ctas_per_sm = occ;
   if (cudaFuncSetAttribute(inject_copy_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(inject_copy_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess) {
@@ -731,6 +756,9 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
       (cache->block_stride % 8) || (cache->token_stride % 8) || (cache->head_stride % 8) || cache->layer_stride < 0 ||
       cache->block_stride < 0 || cache->token_stride < 0 || cache->head_stride < 0)
     return fail(s, MS_ERR_INVALID_ARG, "cache bases must be 16-byte aligned and strides non-negative multiples of 8");
+  if (cache->dtype != MS_CACHE_BF16 && cache->dtype != MS_CACHE_FP8_E4M3) return fail(s, MS_ERR_INVALID_ARG, "unknown cache dtype %d", cache->dtype);
+  if (cache->dtype == MS_CACHE_FP8_E4M3 && !(cache->k_scale > 0.f && cache->v_scale > 0.f && std::isfinite(cache->k_scale) && std::isfinite(cache->v_scale)))
+    return fail(s, MS_ERR_INVALID_ARG, "an 8-bit cache needs finite positive k_scale and v_scale");
   if (out_slot_mapping && slot_stride < 0) return fail(s, MS_ERR_INVALID_ARG, "negative slot_stride");
   if ((c.max_kv_tokens == 0 || !s->k_arena) && !s->k_host) return fail(s, MS_ERR_INVALID_ARG, "store has no K/V arena");
 
@@ -763,6 +791,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.n_heads = c.n_kv_heads;
   p.head_dim = c.head_dim;
   p.rope_style = c.rope_style;
+  p.rotary_dim = c.rotary_dim;
   p.max_position = (int32_t)c.max_position;
   p.fact_ids = fact_ids;
   p.nreq = nreq;
@@ -781,6 +810,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.head_stride = cache->head_stride;
   p.num_blocks = cache->num_blocks;
   p.block_size = cache->block_size;
+  p.k_inv_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? 1.0f / cache->k_scale : 1.0f;
+  p.v_inv_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? 1.0f / cache->v_scale : 1.0f;
   p.out_n_tokens = out_n_tokens;
   p.out_status = out_status;
   p.out_slot_mapping = out_slot_mapping;
@@ -792,7 +823,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
 
   // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
-  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
+  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
   const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
   const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + p.prefix_len + kTileTokens - 1) / kTileTokens * nreq);
   int lpi = 1;
@@ -806,7 +837,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
 ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* cache, int64_t tiles_needed, cudaStream_t st) {
   const memstore_config& c = s->cfg;
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
-  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes;
+  // the staged kernel serves the plain parameterisation only (whole-head rotation, bf16 cache)
+  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
   cudaLaunchConfig_t lc{};
   lc.stream = st;
   cudaLaunchAttribute attr[1];
@@ -845,10 +877,11 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
     lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
     lc.blockDim = dim3(kCopyThreads);
     lc.dynamicSmemBytes = 0;
+    const bool fp8 = cache->dtype == MS_CACHE_FP8_E4M3;
     if (c.rope_style == MS_ROPE_HALF_SPLIT)
-      e = cudaLaunchKernelEx(&lc, inject_copy_kernel<0>, p);
+      e = fp8 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, true>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<0, false>, p);
     else
-      e = cudaLaunchKernelEx(&lc, inject_copy_kernel<1>, p);
+      e = fp8 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, true>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, false>, p);
   }
   if (e != cudaSuccess) {
     // the plan has already counted tiles that no copy kernel will consume

@@ -23,6 +23,7 @@ DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
 ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
 INJECT_REVERSE = 1
 INJECT_PREFIX = 2
+CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 STORE_TMA_COPY_PATH = 1
 REQ_KERNEL_TIMEOUT = 32
 
@@ -40,7 +41,7 @@ class _Config(C.Structure):
         ("rope_theta", C.c_double), ("inv_freq_override", C.POINTER(C.c_float)), ("max_position", C.c_int64),
         ("n_users", C.c_int32), ("flags", C.c_uint32), ("max_facts_per_user", C.c_int64),
         ("max_kv_tokens", C.c_int64), ("kv_arena", C.c_void_p), ("kv_arena_bytes", C.c_size_t),
-        ("max_host_kv_tokens", C.c_int64),
+        ("max_host_kv_tokens", C.c_int64), ("rotary_dim", C.c_int32), ("reserved1", C.c_int32),
     ]  # fmt: skip
 
 
@@ -48,7 +49,7 @@ class _PagedCache(C.Structure):
     _fields_ = [
         ("k_base", C.c_void_p), ("v_base", C.c_void_p), ("layer_stride", C.c_int64), ("block_stride", C.c_int64),
         ("token_stride", C.c_int64), ("head_stride", C.c_int64), ("num_blocks", C.c_int64),
-        ("block_size", C.c_int32), ("reserved0", C.c_int32),
+        ("block_size", C.c_int32), ("dtype", C.c_int32), ("k_scale", C.c_float), ("v_scale", C.c_float),
     ]  # fmt: skip
 
 
@@ -63,7 +64,7 @@ EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
-    "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix",
+    "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
 )  # fmt: skip
 
 _lib = None
@@ -96,6 +97,8 @@ def load_library() -> C.CDLL:
     L.memstore_add_facts_host.restype = i32
     L.memstore_add_facts_host.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
     L.memstore_retrieve.restype = i32
+    L.memstore_rope_table_llama3.restype = i32
+    L.memstore_rope_table_llama3.argtypes = [i32, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_float)]
     L.memstore_set_prefix.restype = i32
     L.memstore_set_prefix.argtypes = [vp, vp, vp, i32, vp]
     L.memstore_retrieve.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
@@ -135,6 +138,17 @@ def _stream_ptr(stream) -> C.c_void_p:
     return C.c_void_p(stream.cuda_stream)
 
 
+def rope_table_llama3(rotary_dim, rope_theta, factor=8.0, low_freq_factor=1.0, high_freq_factor=4.0, original_max_position=8192):
+    """The Llama-3.1 family's rescaled frequency table (computed by the library) as a list of floats for
+    ``MemStore(inv_freq_override=...)``."""
+    out = (C.c_float * (rotary_dim // 2))()
+    rc = load_library().memstore_rope_table_llama3(rotary_dim, float(rope_theta), float(factor), float(low_freq_factor),
+                                                   float(high_freq_factor), float(original_max_position), out)  # fmt: skip
+    if rc != MS_OK:
+        raise MemStoreError(rc, "memstore_rope_table_llama3")
+    return list(out)
+
+
 @dataclass
 class PagedCache:
     """A caller-owned paged KV cache: two bf16 tensors and strides in elements (see ``ms_paged_cache``)."""
@@ -148,38 +162,53 @@ class PagedCache:
     num_blocks: int
     block_size: int
     layout: str = "NHD"  # informational: how `allocate` shaped the tensors
+    k_scale: float = 1.0  # 8-bit (uint8, e4m3 codes) caches only: the cache holds K / k_scale and V / v_scale
+    v_scale: float = 1.0
 
     @classmethod
-    def allocate(cls, n_layers, num_blocks, block_size, n_kv_heads, head_dim, device, layout="NHD", stacked=False, fill_bits=None):
+    def allocate(cls, n_layers, num_blocks, block_size, n_kv_heads, head_dim, device, layout="NHD", stacked=False, fill_bits=None,
+                 fp8=False, k_scale=1.0, v_scale=1.0):  # fmt: skip
         """Allocate a cache. ``layout`` "NHD": [L][blocks][bs][h][d]; "HND": [L][blocks][h][bs][d].
-        ``stacked``: K and V are planes 0 and 1 of one buffer [L][2][blocks]..., else separate buffers."""
+        ``stacked``: K and V are planes 0 and 1 of one buffer [L][2][blocks]..., else separate buffers.
+        ``fp8``: one byte per element (uint8 tensors of e4m3 codes) with the given per-tensor scales;
+        ``fill_bits`` is then a byte."""
         shape = (num_blocks, block_size, n_kv_heads, head_dim) if layout == "NHD" else (num_blocks, n_kv_heads, block_size, head_dim)
         blk = block_size * n_kv_heads * head_dim
+        dt = torch.uint8 if fp8 else torch.bfloat16
         if stacked:
-            buf = torch.empty((n_layers, 2, *shape), dtype=torch.bfloat16, device=device)
+            buf = torch.empty((n_layers, 2, *shape), dtype=dt, device=device)
             k, v = buf[:, 0], buf[:, 1]
             layer_stride = 2 * num_blocks * blk
             keep = buf
         else:
-            k = torch.empty((n_layers, *shape), dtype=torch.bfloat16, device=device)
-            v = torch.empty((n_layers, *shape), dtype=torch.bfloat16, device=device)
+            k = torch.empty((n_layers, *shape), dtype=dt, device=device)
+            v = torch.empty((n_layers, *shape), dtype=dt, device=device)
             layer_stride = num_blocks * blk
             keep = None
         if fill_bits is not None:
             for t in ((keep,) if stacked else (k, v)):
-                t.view(torch.int16).fill_(fill_bits - 0x10000 if fill_bits >= 0x8000 else fill_bits)
+                if fp8:
+                    t.fill_(fill_bits)
+                else:
+                    t.view(torch.int16).fill_(fill_bits - 0x10000 if fill_bits >= 0x8000 else fill_bits)
         token_stride, head_stride = (n_kv_heads * head_dim, head_dim) if layout == "NHD" else (head_dim, block_size * head_dim)
         c = cls(k, v, layer_stride, blk, token_stride, head_stride, num_blocks, block_size)
         c._keep = keep
         c.layout = layout
+        c.k_scale, c.v_scale = float(k_scale), float(v_scale)
         return c
+
+    @property
+    def fp8(self) -> bool:
+        return self.k.dtype == torch.uint8
 
     def _struct(self) -> _PagedCache:
         for t, n in ((self.k, "k"), (self.v, "v")):
-            if not t.is_cuda or t.dtype != torch.bfloat16:
-                raise TypeError(f"cache.{n} must be a CUDA bfloat16 tensor")
+            if not t.is_cuda or t.dtype not in (torch.bfloat16, torch.uint8) or t.dtype != self.k.dtype:
+                raise TypeError(f"cache.{n} must be a CUDA bfloat16 (or, for an 8-bit cache, uint8) tensor")
         return _PagedCache(self.k.data_ptr(), self.v.data_ptr(), self.layer_stride, self.block_stride,
-                           self.token_stride, self.head_stride, self.num_blocks, self.block_size, 0)  # fmt: skip
+                           self.token_stride, self.head_stride, self.num_blocks, self.block_size,
+                           CACHE_FP8_E4M3 if self.fp8 else CACHE_BF16, self.k_scale, self.v_scale)  # fmt: skip
 
 
 class MemStore:
@@ -187,7 +216,8 @@ class MemStore:
 
     def __init__(self, *, device=0, n_layers, n_kv_heads, head_dim, emb_dim, emb_dtype=torch.float16, rope_theta=1.0e4,
                  rope_style=ROPE_HALF_SPLIT, inv_freq_override=None, max_position=1 << 24, n_users=1,
-                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None, flags=0, max_host_kv_tokens=0):  # fmt: skip
+                 max_facts_per_user, max_kv_tokens, kv_arena: torch.Tensor | None = None, flags=0, max_host_kv_tokens=0,
+                 rotary_dim=0):  # fmt: skip
         self._lib = load_library()
         self._h = C.c_void_p()
         self.device = torch.device("cuda", device if isinstance(device, int) else torch.device(device).index or 0)
@@ -199,13 +229,14 @@ class MemStore:
         if inv_freq_override is not None:
             vals = [float(x) for x in inv_freq_override]
             ov = (C.c_float * len(vals))(*vals)
-            if len(vals) != head_dim // 2:
-                raise ValueError("inv_freq_override needs head_dim/2 entries")
+            if len(vals) != (rotary_dim or head_dim) // 2:
+                raise ValueError("inv_freq_override needs rotary_dim/2 (head_dim/2) entries")
         self._arena = kv_arena
         cfg = _Config(self.device.index, n_layers, n_kv_heads, head_dim, DTYPE_BF16, emb_dim, emb_code, rope_style,
                       float(rope_theta), ov, max_position, n_users, flags, max_facts_per_user, max_kv_tokens,
                       kv_arena.data_ptr() if kv_arena is not None else None,
-                      kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0, max_host_kv_tokens)  # fmt: skip
+                      kv_arena.numel() * kv_arena.element_size() if kv_arena is not None else 0, max_host_kv_tokens,
+                      rotary_dim, 0)  # fmt: skip
         self.n_layers, self.n_kv_heads, self.head_dim, self.emb_dim = n_layers, n_kv_heads, head_dim, emb_dim
         rc = self._lib.memstore_create(C.byref(cfg), C.byref(self._h))
         if rc != MS_OK:

@@ -32,7 +32,9 @@ def to_dev(a: np.ndarray, device="cuda"):
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> uint16 numpy bit patterns (host)."""
+    """bf16 tensor -> uint16 numpy bit patterns (host); a uint8 tensor (8-bit cache) -> its bytes."""
+    if t.dtype == torch.uint8:
+        return t.contiguous().cpu().numpy()
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
@@ -101,24 +103,53 @@ def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None):
     return int((~exact).sum())
 
 
-def k_tolerance(k_ref: np.ndarray, style: int) -> np.ndarray:
-    """Per-element tolerance 2^-7 * max(|ref|, 2^-10 * ||pair||); rotation preserves the pair norm."""
+def k_tolerance(k_ref: np.ndarray, style: int, rotary_dim: int = 0) -> np.ndarray:
+    """Per-element tolerance 2^-7 * max(|ref|, 2^-10 * ||pair||); rotation preserves the pair norm.
+    Coordinates beyond ``rotary_dim`` are copies: their "pair" is the element itself."""
     D = k_ref.shape[-1]
+    R = rotary_dim or D
+    lead = k_ref[..., :R]
     if style == 0:
-        a, b = k_ref[..., : D // 2], k_ref[..., D // 2 :]
+        a, b = lead[..., : R // 2], lead[..., R // 2 :]
         nrm = np.sqrt(a * a + b * b)
         pair = np.concatenate([nrm, nrm], axis=-1)
     else:
-        a, b = k_ref[..., 0::2], k_ref[..., 1::2]
+        a, b = lead[..., 0::2], lead[..., 1::2]
         nrm = np.sqrt(a * a + b * b)
         pair = np.repeat(nrm, 2, axis=-1)
+    pair = np.concatenate([pair, np.abs(k_ref[..., R:])], axis=-1)
     return K_REL_TOL * np.maximum(np.abs(k_ref), K_FLOOR * pair), pair
 
 
-def check_k(gpu_bits: np.ndarray, k_ref: np.ndarray, style: int = 0):
+def check_k_fp8(gpu_codes: np.ndarray, want: np.ndarray, k_ref: np.ndarray, k_scale: float, style: int = 0, rotary_dim: int = 0):
+    """Keys of an 8-bit (e4m3) cache against the oracle's codes ``want`` and its unrounded rotated keys ``k_ref``.
+    Coordinates beyond ``rotary_dim`` are copies, decided by a binary32 product on both sides: bit-exact.  A rotated
+    coordinate is decided by the kernel's fp32 rotation here and by a double there, so a value within fp32
+    evaluation error of a rounding tie may round the other way: the decoded code must lie within half an e4m3
+    step of ref / scale plus 4e-6 of the pair norm / scale, and must be the oracle's code everywhere else.
+    Returns the fraction of codes equal to the oracle's."""
+    inv = float(np.float32(1.0) / np.float32(k_scale))
+    target = k_ref * inv
+    _, pair = k_tolerance(k_ref, style, rotary_dim)
+    slack = 4e-6 * pair * inv
+    dec = oracle.e4m3_to_double(gpu_codes)
+    assert not np.isnan(dec).any(), "NaN code in the cache"
+    clipped = np.clip(target, -448.0, 448.0)
+    step = np.maximum(2.0 ** (np.floor(np.log2(np.maximum(np.abs(clipped), 2.0**-6))) - 3), 2.0**-9)
+    assert np.all(np.abs(dec - clipped) <= step / 2 + slack), "key further than half an e4m3 step from the exact value"
+    eq = gpu_codes == want
+    if rotary_dim:
+        assert np.all(eq[..., rotary_dim:]), "unrotated coordinates must carry exactly the oracle's code"
+    # where the exact value is not within `slack` of a rounding tie the code must be the oracle's
+    lo, hi = oracle.e4m3_from_double(target - slack), oracle.e4m3_from_double(target + slack)
+    assert np.all(eq | (lo != hi)), "wrong e4m3 code away from a tie"
+    return float(eq.mean()) if eq.size else 1.0
+
+
+def check_k(gpu_bits: np.ndarray, k_ref: np.ndarray, style: int = 0, rotary_dim: int = 0):
     """Returns (fraction bit-equal to the correctly rounded value, worst error / tolerance)."""
     got = oracle.bf16_to_double(gpu_bits)
-    tol, pair = k_tolerance(k_ref, style)
+    tol, pair = k_tolerance(k_ref, style, rotary_dim)
     err = np.abs(got - k_ref)
     ratio = err / np.maximum(tol, 1e-300)
     worst = float(ratio.max()) if ratio.size else 0.0
@@ -158,10 +189,11 @@ def untouched_mask_ok(cache: PagedCache, written_slots: np.ndarray, sentinel_bit
         keep[torch.from_numpy(np.asarray(written_slots, dtype=np.int64)).to(dev)] = False
     keep = keep.view(cache.num_blocks, bs)
     nhd = cache.layout == "NHD"
-    sent = sentinel_bits - 0x10000 if sentinel_bits >= 0x8000 else sentinel_bits
+    fp8 = cache.k.dtype == torch.uint8  # then the sentinel is a byte
+    sent = sentinel_bits if fp8 else (sentinel_bits - 0x10000 if sentinel_bits >= 0x8000 else sentinel_bits)
     for t in (cache.k, cache.v):
         for l in range(t.shape[0]):
-            xl = t[l].view(torch.int16) if t[l].is_contiguous() else t[l].contiguous().view(torch.int16)
+            xl = t[l] if fp8 else (t[l].view(torch.int16) if t[l].is_contiguous() else t[l].contiguous().view(torch.int16))
             ok = xl == sent  # [blocks, bs, H, D] or [blocks, H, bs, D]
             ok = ok.all(dim=-1)
             ok = ok.all(dim=2) if nhd else ok.all(dim=1)  # -> [blocks, bs]
@@ -183,7 +215,8 @@ def with_prefix(hs: HostStore, placed, prefix):
 
 
 def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, cache: PagedCache, theta, style=0,
-                         inv_freq=None, flags=0, sentinel=synth.SENTINEL_BF16, check_untouched=True, prefix=None):  # fmt: skip
+                         inv_freq=None, flags=0, sentinel=synth.SENTINEL_BF16, check_untouched=True, prefix=None,
+                         rotary_dim=0):  # fmt: skip
     """One request: inject on the GPU, run the oracle on the same ids, compare. Returns stats dict.
     ``prefix``: (k, v) of the instruction prefix the store holds, when ``flags`` asks for it."""
     dev = cache.k.device
@@ -196,8 +229,10 @@ def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, c
     offs, lens, hk, hv = hs.offs, hs.lens, hs.k, hs.v
     if flags & 2:
         placed, offs, lens, hk, hv = with_prefix(hs, placed, prefix)
+    fp8 = cache.k.dtype == torch.uint8
     res = oracle.inject(placed, offs, lens, hk, hv, theta, start, table_np, cache.block_size,
-                        cache.num_blocks, style=style, inv_freq_override=inv_freq)  # fmt: skip
+                        cache.num_blocks, style=style, inv_freq_override=inv_freq, rotary_dim=rotary_dim,
+                        k_scale=cache.k_scale if fp8 else None, v_scale=cache.v_scale if fp8 else None)  # fmt: skip
     slot_map = torch.full((1, max(res.m, 1) + 3), -7, dtype=torch.int64, device=dev)
     n_tok, status = ms.inject(ids, sp, bt, cache, out_slot_mapping=slot_map, flags=flags)
     torch.cuda.synchronize()
@@ -206,10 +241,16 @@ def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, c
     sm = slot_map[0].cpu().numpy()
     assert np.array_equal(sm[: res.m], res.slots) and np.all(sm[res.m :] == -7)
     out = {"m": res.m, "exact_frac": 1.0, "worst": 0.0}
-    if res.m:
+    if res.m and fp8:
+        kb, vb = gather_cache_rows(cache, res.slots)
+        assert np.array_equal(vb, res.v_fp8), "V codes must be bit-exact (fp32 product, one rounding)"
+        out["exact_frac"] = check_k_fp8(kb, res.k_fp8, res.k_ref, cache.k_scale, style, rotary_dim)
+    elif res.m:
         kb, vb = gather_cache_rows(cache, res.slots)
         assert np.array_equal(vb, res.v), "V must be bit-exact"
-        out["exact_frac"], out["worst"] = check_k(kb, res.k_ref, style)
+        out["exact_frac"], out["worst"] = check_k(kb, res.k_ref, style, rotary_dim)
+        if rotary_dim:
+            assert np.array_equal(kb[..., rotary_dim:], res.k_bf16[..., rotary_dim:]), "coordinates beyond rotary_dim are copies"
     if check_untouched:
         assert untouched_mask_ok(cache, res.slots, sentinel), "a slot outside the request was modified"
     return out

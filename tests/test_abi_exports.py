@@ -10,7 +10,7 @@ ROOT = Path(__file__).resolve().parent.parent
 def declared_functions():
     text = (ROOT / "include" / "memstore.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(memstore_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(memstore_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
@@ -27,11 +27,11 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header_sizes():
-    # the ctypes mirrors must have the C sizes (x86-64 / LP64): config 104 bytes, cache 64, stats 80
+    # the ctypes mirrors must have the C sizes (x86-64 / LP64): config 112 bytes, cache 72, stats 80
     from paper_2607_27090_b200 import memstore
 
-    assert ctypes.sizeof(memstore._Config) == 104
-    assert ctypes.sizeof(memstore._PagedCache) == 64
+    assert ctypes.sizeof(memstore._Config) == 112
+    assert ctypes.sizeof(memstore._PagedCache) == 72
     assert ctypes.sizeof(memstore._Stats) == 80
 
 
@@ -51,3 +51,22 @@ def test_product_path_does_not_import_the_oracle():
         if f.suffix in (".py", ".cu", ".cuh", ".h"):
             src = f.read_text()
             assert "import oracle" not in src and "from oracle" not in src and "memoracle" not in src, f
+
+
+def test_llama3_frequency_table_of_the_library_equals_the_oracles():
+    """Host arithmetic inside the library (no GPU needed): the rescaled table must agree bit for bit with the
+    oracle's independent evaluation, because a one-ulp difference in a frequency is visible at large positions."""
+    import numpy as np
+
+    import oracle
+    from paper_2607_27090_b200 import memstore
+
+    for R, theta, args in ((128, 5e5, (8.0, 1.0, 4.0, 8192)), (64, 1e4, (4.0, 1.0, 4.0, 4096)), (96, 1e6, (32.0, 1.0, 4.0, 8192)),
+                           (128, 5e5, (1.0, 1.0, 4.0, 8192))):  # fmt: skip
+        got = np.array(memstore.rope_table_llama3(R, theta, *args), np.float32)
+        want = oracle.inv_freq_llama3(R, theta, *args)
+        assert np.array_equal(got, want)
+    import pytest
+
+    with pytest.raises(memstore.MemStoreError):
+        memstore.rope_table_llama3(127, 5e5)

@@ -209,6 +209,54 @@ def test_inject_head_shapes_and_rope_styles(style, H, D, path):
     assert out["exact_frac"] > 0.995
 
 
+@pytest.mark.parametrize("style", [0, 1])
+@pytest.mark.parametrize("D,R", [(128, 64), (128, 16), (64, 32), (256, 64), (32, 32)])
+def test_inject_partial_rotary(style, D, R):
+    """Only the first R coordinates of a head rotate (frequencies theta^(-2i/R)); the rest is copied bit for bit."""
+    hs = HostStore(70 + R, 10, 2, 3, D, 5, 40, 64, "float16")
+    ms = hs.to_memstore(1e6, rope_style=style, rotary_dim=R)
+    table = synth.block_tables(71, 32, 20, 1)[0]
+    cache = make_cache(hs, 32, 16)
+    out = run_inject_and_check(ms, hs, [3, 9, 0, 4], 11, table, cache, 1e6, style=style, rotary_dim=R, flags=M.INJECT_REVERSE)
+    assert out["exact_frac"] > 0.995
+    ms.close()
+
+
+def test_inject_llama3_rescaled_table():
+    """The library's Llama-3.1 frequency table is bit-identical to the oracle's and drives the rotation."""
+    tab = M.rope_table_llama3(128, 5e5)
+    assert np.array_equal(np.array(tab, np.float32), oracle.inv_freq_llama3(128, 5e5))
+    hs = HostStore(72, 8, 2, 8, 128, 20, 60, 64, "float16")
+    ms = hs.to_memstore(5e5, inv_freq_override=tab)
+    table = synth.block_tables(73, 2100, 2080, 1)[0]  # positions around 33,000: the slowed pairs turn visibly
+    cache = make_cache(hs, 2100, 16)
+    out = run_inject_and_check(ms, hs, [1, 5, 2], 33000, table, cache, 5e5, inv_freq=np.array(tab, np.float32))
+    assert out["exact_frac"] > 0.995
+    plain = oracle.inject([1], hs.offs, hs.lens, hs.k, hs.v, 5e5, 33000, table, 16, 2100)
+    scaled = oracle.inject([1], hs.offs, hs.lens, hs.k, hs.v, 5e5, 33000, table, 16, 2100, inv_freq_override=np.array(tab, np.float32))
+    assert not np.array_equal(plain.k_bf16, scaled.k_bf16)  # the table matters at this position
+    ms.close()
+
+
+@pytest.mark.parametrize("layout", ["NHD", "HND"])
+@pytest.mark.parametrize("style,R", [(0, 0), (1, 0), (0, 64)])
+def test_inject_into_an_8_bit_e4m3_cache(layout, style, R):
+    """K / k_scale and V / v_scale as e4m3 codes: V bit-exact, K the correctly rounded code except next to a tie;
+    slots outside the request keep their bytes."""
+    hs = HostStore(74, 12, 3, 4, 128, 5, 40, 64, "float16")
+    ms = hs.to_memstore(5e5, rope_style=style, rotary_dim=R)
+    table = synth.block_tables(75, 48, 20, 1)[0]
+    for k_scale, v_scale in ((1.0, 1.0), (0.037, 0.11), (3.0, 0.004)):  # the last pair saturates many values
+        cache = PagedCache.allocate(hs.L, 48, 16, hs.H, hs.D, DEV, layout=layout, fill_bits=0x5A, fp8=True, k_scale=k_scale, v_scale=v_scale)
+        out = run_inject_and_check(ms, hs, [7, 0, 11, 3], 9, table, cache, 5e5, style=style, rotary_dim=R, sentinel=0x5A)
+        assert out["exact_frac"] > 0.999
+    bad = PagedCache.allocate(hs.L, 48, 16, hs.H, hs.D, DEV, fp8=True, k_scale=0.0)
+    with pytest.raises(RuntimeError):
+        ms.inject(torch.zeros((1, 1), dtype=torch.int32, device=DEV), torch.zeros(1, dtype=torch.int32, device=DEV),
+                  to_dev(table.reshape(1, -1)), bad)  # fmt: skip
+    ms.close()
+
+
 def test_inject_inv_freq_override_and_reverse_flag():
     D = 64
     f = (np.linspace(1.0, 0.001, D // 2)).astype(np.float32)

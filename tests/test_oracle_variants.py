@@ -145,13 +145,13 @@ def test_inject_with_partial_rotation_and_e4m3_cache_images(oracle_mod):
     pos = 5 + np.arange(part.m)
     lead = oracle_mod.rope_rows(x[..., :16].reshape(-1, 16), np.tile(np.repeat(pos, 2), 2), 1e4)
     assert np.array_equal(part.k_ref[..., :16].reshape(-1, 16), lead)
-    # quantised images: within half an e4m3 step of value / scale, and exactly the one-step rounding of it
+    # quantised images: within half an e4m3 step of value / scale, and exactly the rounding of its binary32 value
     for codes, ref, scale in ((part.k_fp8, part.k_ref, 0.5), (part.v_fp8, oracle_mod.bf16_to_double(part.v), 0.25)):
         target = ref / scale  # 1 / 0.5 and 1 / 0.25 are exact in binary32, so this is the value both paths quantise
         dec = oracle_mod.e4m3_to_double(codes)
         step = np.maximum(2.0 ** (np.floor(np.log2(np.maximum(np.abs(target), 2.0**-6))) - 3), 2.0**-9)
         assert np.all(np.abs(dec - np.clip(target, -448, 448)) <= step / 2)
-        assert np.array_equal(codes, oracle_mod.e4m3_from_double(target))
+        assert np.array_equal(codes, oracle_mod.e4m3_from_double(target.astype(np.float32).astype(np.float64)))
     # a value that e4m3 represents exactly survives quantisation with scale 1
     exact = np.array([[[[0.5, -1.75, 448.0, 2.0**-9] * 8]]], np.float32)  # [1, 1, 1, 32]
     eb = torch.from_numpy(exact).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
