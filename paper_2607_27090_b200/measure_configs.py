@@ -127,6 +127,52 @@ def measure_host_tier(iters: int, seed: int = 0, n_facts: int = 400, ks=(5, 10, 
     return lines
 
 
+def measure_variants(iters: int, seed: int = 0, n_facts: int = 400, k: int = 50):
+    """Injection of k facts on the Llama-3.1-8B KV shape (a shrunken store: the traffic of a request does not depend on
+    the store size) in the parameterisation variants: bf16 cache (the headline path), 8-bit e4m3 cache (half the
+    write traffic), and rotation of the first 64 coordinates only."""
+    s = synth.CONFIGS["llama8b"]
+    dev = torch.device("cuda")
+    lens = synth.fact_lengths(seed, n_facts, s.len_lo, s.len_hi)
+    T = int(lens.sum())
+    emb = synth.embeddings(seed, n_facts, s.emb_dim, s.emb_dtype)
+    rng = np.random.default_rng(seed)
+    per_req = workload.blocks_per_request(s, k)
+    ids = torch.from_numpy(np.stack([rng.choice(n_facts, k, replace=False) for _ in range(4)]).astype(np.int32)).to(dev)
+    m = float(np.mean([lens[ids[i].cpu().numpy()].sum() for i in range(4)]))
+    lines = []
+    for variant, rotary_dim, fp8 in (("bf16 cache", 0, False), ("e4m3 cache", 0, True), ("rotary_dim 64, bf16 cache", 64, False)):
+        store = M.MemStore(n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, emb_dim=s.emb_dim, rope_theta=s.rope_theta,
+                           max_facts_per_user=n_facts, max_kv_tokens=T, rotary_dim=rotary_dim)  # fmt: skip
+        g = torch.Generator(device=dev).manual_seed(seed)
+        for a in range(0, n_facts, 50):
+            b = min(n_facts, a + 50)
+            t = int(lens[a:b].sum())
+            kv = torch.randn((2, s.n_layers, t, s.n_kv_heads, s.head_dim), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            store.add_facts(torch.from_numpy(emb[a:b]).to(dev), lens[a:b], kv[0].contiguous(), kv[1].contiguous())
+        cache = M.PagedCache.allocate(s.n_layers, max(1024, per_req * 4), s.block_size, s.n_kv_heads, s.head_dim, dev, fp8=fp8,
+                                      k_scale=0.05, v_scale=0.05)  # fmt: skip
+        tables = torch.from_numpy(synth.block_tables(seed, cache.num_blocks, per_req, 4)).to(dev)
+        start = torch.full((1,), s.start_pos, dtype=torch.int32, device=dev)
+        stream = torch.cuda.current_stream()
+        for i in range(3):
+            store.inject(ids[i % 4 : i % 4 + 1], start, tables[i % 4 : i % 4 + 1], cache, stream=stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(iters):
+            store.inject(ids[i % 4 : i % 4 + 1], start, tables[i % 4 : i % 4 + 1], cache, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        moved = m * s.token_bytes * (1.5 if fp8 else 2.0)  # read K and V (bf16), write both (one or two bytes per element)
+        lines.append({"config": "llama8b " + variant, "k": k, "tokens": m, "inject_us": us, "bytes_moved": moved,
+                      "inject_gbs": moved / (us * 1e-6) / 1e9})  # fmt: skip
+        store.close()
+        del cache
+    return lines
+
+
 def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
     s = synth.CONFIGS[name]
     dev = torch.device("cuda")
@@ -206,8 +252,12 @@ if __name__ == "__main__":
     ap.add_argument("--pool-blocks", type=int, default=None)
     ap.add_argument("--retrieve-only", action="store_true", help="embedding-only store, time the batched retrieval alone")
     ap.add_argument("--host-tier", action="store_true", help="Llama shape with all K/V in the pinned host arena: inject over PCIe")
+    ap.add_argument("--variants", action="store_true", help="Llama shape: bf16 cache, e4m3 cache, partial rotary (inject only)")
     a = ap.parse_args()
-    if a.host_tier:
+    if a.variants:
+        for ln in measure_variants(a.iters, a.seed):
+            print(json.dumps(ln))
+    elif a.host_tier:
         for ln in measure_host_tier(a.iters, a.seed):
             print(json.dumps(ln))
     elif a.retrieve_only:
