@@ -70,6 +70,12 @@ def lib() -> C.CDLL:
             + [i64] * 4
             + [i32]
         )
+        L.oracle_scores_f32.restype = i32
+        L.oracle_scores_f32.argtypes = [p, i32, i64, i32, p, p]
+        L.oracle_knn_graph.restype = i32
+        L.oracle_knn_graph.argtypes = [p, i32, i64, i32, i32, p, i32]
+        L.oracle_ann_search.restype = i32
+        L.oracle_ann_search.argtypes = [p, i32, i64, i32, p, i32, p, i32, i32, i32, i32, i32, p, p, p, p]
         L.oracle_inject_ex.restype = i32
         L.oracle_inject_ex.argtypes = L.oracle_inject.argtypes + [i32, C.c_float, C.c_float, p, p]
         L.oracle_rope_rows_partial.restype = i32
@@ -173,6 +179,54 @@ def retrieve(emb: np.ndarray, queries: np.ndarray, k: int, row_ids: np.ndarray |
     if rc:
         raise OracleError(rc)
     return ids, sc
+
+
+def scores_f32(emb: np.ndarray, query: np.ndarray) -> np.ndarray:
+    """Inner products in binary32 with the fixed lane order that the graph search compares scores in."""
+    emb = np.ascontiguousarray(emb)
+    query = np.ascontiguousarray(query, dtype=emb.dtype).reshape(-1)
+    out = np.empty(emb.shape[0], dtype=np.float32)
+    rc = lib().oracle_scores_f32(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(query), _ptr(out))
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def knn_graph(emb: np.ndarray, deg: int, n_threads: int = 0) -> np.ndarray:
+    """Exact k-nearest-neighbour graph by inner product: int32 [n, deg], best first, -1 padded."""
+    emb = np.ascontiguousarray(emb)
+    out = np.empty((emb.shape[0], deg), dtype=np.int32)
+    rc = lib().oracle_knn_graph(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], deg, _ptr(out), n_threads)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+class AnnResult:
+    def __init__(self, ids, scores, iters, scored):
+        self.ids, self.scores, self.iters, self.scored = ids, scores, iters, scored
+
+
+def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, beam: int = 64, parents: int = 4,
+               n_entry: int = 64, max_iters: int = 32) -> AnnResult:  # fmt: skip
+    """Beam search over ``graph`` for each query: ids / scores [nq, k], steps taken and rows scored per query."""
+    emb = np.ascontiguousarray(emb)
+    graph = np.ascontiguousarray(graph, dtype=np.int32)
+    queries = np.ascontiguousarray(queries, dtype=emb.dtype).reshape(-1, emb.shape[1])
+    nq = queries.shape[0]
+    ids = np.empty((nq, k), dtype=np.int32)
+    sc = np.empty((nq, k), dtype=np.float32)
+    iters = np.zeros(nq, dtype=np.int32)
+    scored = np.zeros(nq, dtype=np.int64)
+    for q in range(nq):
+        it, ns = C.c_int32(0), C.c_int64(0)
+        rc = lib().oracle_ann_search(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(graph), graph.shape[1],
+                                     _ptr(queries[q]), k, beam, parents, n_entry, max_iters, _ptr(ids[q]), _ptr(sc[q]),
+                                     C.byref(it), C.byref(ns))  # fmt: skip
+        if rc:
+            raise OracleError(rc)
+        iters[q], scored[q] = it.value, ns.value
+    return AnnResult(ids, sc, iters, scored)
 
 
 def inv_freq(D: int, theta: float) -> np.ndarray:

@@ -26,6 +26,9 @@
  *   - V is stored raw and copied unchanged (Sec. 5.1, closing paragraph).
  *   - bytes per fact:   "Storage cost" (Sec. 3.5): 2 * L * c * h * d * b.
  *
+ *   - graph index:      "Jasper: a GPU-native vector index" (Sec. 2.5) and the index parameters of the
+ *     evaluation setup (Sec. 6.1): a proximity graph searched by a beam search; the concrete algorithm is
+ *     fixed in the comment above oracle_ann_search.
  *   - variants beyond the paper's text (its evaluation spans "RoPE parameterizations", Sec. 6.1): the
  *     Llama-3.1 rescaled frequency table, rotation of only the first R coordinates of a head, and an
  *     8-bit e4m3 cache image with per-tensor scales.
@@ -254,6 +257,181 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
   }
   free(s);
   free(all);
+  return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------- graph index (approximate retrieval) */
+
+/*
+ * The paper retrieves with a GPU-resident proximity-graph index searched by a beam search (Sec. 2.5; Sec. 6.1:
+ * inner-product distance, 64 graph neighbours, beam width 64) and does not print the index's algorithm.  The
+ * algorithm fixed here, step by step, is the one this oracle and the library both follow:
+ *
+ *   graph    G[n][deg]: row r lists the deg rows with the largest inner product with row r, r itself
+ *            excluded, best first, ties to the lower row (an exact k-nearest-neighbour graph); -1 pads.
+ *   scores   a search compares scores, so they are formed in the arithmetic of the path that takes the
+ *            decisions: binary32, the fixed summation order below (score_f32_lanes).
+ *   list     at most L = max(beam, k) entries (score, row, expanded?), ordered by score descending, ties to
+ *            the lower row; V = the set of rows ever scored.
+ *   start    rows e_i = ((i + 1) * 2654435761) mod n, i < n_entry (duplicates dropped), scored and listed.
+ *   step     take the first `parents` unexpanded entries of the list in list order (stop when there is none, or
+ *            after max_iters steps), mark them expanded; collect their neighbours that are valid rows and
+ *            not in V, add them to V, score them, and keep the best L of list + new.
+ *   result   the first k entries of the list; -1 / 0 pads.
+ */
+
+/*
+ * Inner product in binary32 with a fixed order: the row is cut into vectors of 16 bytes (8 halves or 4
+ * floats); vector v belongs to "lane" v mod 32; a lane adds its products one fused multiply-add at a time in
+ * increasing element order; the 32 lane sums are then combined by a butterfly (lane l adds lane l xor 16,
+ * then xor 8, 4, 2, 1).  Every lane ends with the same value.
+ */
+static float score_f32_lanes(const void* emb, int dtype, int64_t row, int dim, const void* query) {
+  int vec = dtype == ORACLE_F32 ? 4 : 8;
+  int nvec = dim / vec;
+  float acc[32], tmp[32];
+  for (int l = 0; l < 32; ++l) acc[l] = 0.0f;
+  for (int v0 = 0; v0 < nvec; v0 += 128)
+    for (int l = 0; l < 32; ++l)
+      for (int u = 0; u < 4; ++u) {
+        int v = v0 + u * 32 + l;
+        if (v >= nvec) continue;
+        for (int i = 0; i < vec; ++i) {
+          float a = (float)emb_at(emb, dtype, row * dim + (int64_t)v * vec + i);
+          float b = (float)emb_at(query, dtype, (int64_t)v * vec + i);
+          acc[l] = fmaf(a, b, acc[l]);
+        }
+      }
+  for (int o = 16; o > 0; o >>= 1) {
+    for (int l = 0; l < 32; ++l) tmp[l] = acc[l] + acc[l ^ o];
+    for (int l = 0; l < 32; ++l) acc[l] = tmp[l];
+  }
+  return acc[0] + 0.0f; /* -0 becomes +0 */
+}
+
+int oracle_scores_f32(const void* emb, int emb_dtype, int64_t n_rows, int emb_dim, const void* query, float* out) {
+  if (!emb || !query || !out || emb_dim <= 0 || emb_dim % 8) return ORACLE_ERR_ARG;
+  for (int64_t r = 0; r < n_rows; ++r) out[r] = score_f32_lanes(emb, emb_dtype, r, emb_dim, query);
+  return ORACLE_OK;
+}
+
+/* Exact k-nearest-neighbour graph by inner product (double scores, full sort per row). */
+int oracle_knn_graph(const void* emb, int emb_dtype, int64_t n, int emb_dim, int deg, int32_t* out_graph, int n_threads) {
+  if (!emb || !out_graph || n < 0 || deg <= 0 || emb_dim <= 0) return ORACLE_ERR_ARG;
+  size_t esz = emb_dtype == ORACLE_F32 ? 4 : 2;
+  int rc_all = ORACLE_OK;
+  set_threads(n_threads);
+#pragma omp parallel for schedule(dynamic, 8)
+  for (int64_t r = 0; r < n; ++r) {
+    scored_t* all = (scored_t*)malloc(sizeof(scored_t) * (size_t)n);
+    if (!all) {
+      rc_all = ORACLE_ERR_NOMEM;
+      continue;
+    }
+    const char* q = (const char*)emb + (size_t)r * emb_dim * esz;
+    int64_t m = 0;
+    for (int64_t f = 0; f < n; ++f) {
+      if (f == r) continue;
+      double sc = 0.0;
+      for (int d = 0; d < emb_dim; ++d) sc += emb_at(q, emb_dtype, d) * emb_at(emb, emb_dtype, f * emb_dim + d);
+      all[m].s = sc;
+      all[m].id = (int32_t)f;
+      ++m;
+    }
+    qsort(all, (size_t)m, sizeof(scored_t), cmp_scored);
+    for (int j = 0; j < deg; ++j) out_graph[r * deg + j] = j < m ? all[j].id : -1;
+    free(all);
+  }
+  return rc_all;
+}
+
+typedef struct {
+  float s;
+  int32_t row;
+  int32_t expanded;
+} beam_t;
+
+static int cmp_beam(const void* a, const void* b) {
+  const beam_t* x = (const beam_t*)a;
+  const beam_t* y = (const beam_t*)b;
+  if (x->s > y->s) return -1;
+  if (x->s < y->s) return 1;
+  if (x->row < y->row) return -1;
+  if (x->row > y->row) return 1;
+  return 0;
+}
+
+/*
+ * Beam search of one query over the graph, as defined above.  out_ids / out_scores [k]; out_iters (optional):
+ * steps taken; out_scored (optional): |V|, the number of rows scored.
+ */
+int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
+                      const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
+                      float* out_scores, int32_t* out_iters, int64_t* out_scored) {
+  if (!out_ids || k <= 0 || beam <= 0 || parents <= 0 || n_entry <= 0 || max_iters < 0 || deg <= 0 || n < 0 ||
+      emb_dim <= 0 || emb_dim % 8)
+    return ORACLE_ERR_ARG;
+  if (n > 0 && (!emb || !graph || !query)) return ORACLE_ERR_ARG;
+  int L = beam > k ? beam : k;
+  int cap = L + (parents * deg > n_entry ? parents * deg : n_entry);
+  beam_t* list = (beam_t*)malloc(sizeof(beam_t) * (size_t)cap);
+  unsigned char* seen = (unsigned char*)calloc((size_t)(n > 0 ? n : 1), 1);
+  int32_t* chosen = (int32_t*)malloc(sizeof(int32_t) * (size_t)parents);
+  if (!list || !seen || !chosen) {
+    free(list);
+    free(seen);
+    free(chosen);
+    return ORACLE_ERR_NOMEM;
+  }
+  int len = 0, iters = 0;
+  int64_t scored = 0;
+  if (n > 0) {
+    for (int i = 0; i < n_entry; ++i) {
+      int64_t e = (int64_t)(((uint64_t)(i + 1) * 2654435761ull) % (uint64_t)n);
+      if (seen[e]) continue;
+      seen[e] = 1;
+      list[len].s = score_f32_lanes(emb, emb_dtype, e, emb_dim, query);
+      list[len].row = (int32_t)e;
+      list[len].expanded = 0;
+      ++len;
+      ++scored;
+    }
+    qsort(list, (size_t)len, sizeof(beam_t), cmp_beam);
+    if (len > L) len = L;
+    for (; iters < max_iters; ++iters) {
+      int np = 0;
+      for (int i = 0; i < len && np < parents; ++i)
+        if (!list[i].expanded) {
+          list[i].expanded = 1;
+          chosen[np++] = list[i].row;
+        }
+      if (np == 0) break;
+      int added = 0;
+      for (int p = 0; p < np; ++p)
+        for (int j = 0; j < deg; ++j) {
+          int32_t nb = graph[(int64_t)chosen[p] * deg + j];
+          if (nb < 0 || nb >= n || seen[nb]) continue;
+          seen[nb] = 1;
+          list[len + added].s = score_f32_lanes(emb, emb_dtype, nb, emb_dim, query);
+          list[len + added].row = nb;
+          list[len + added].expanded = 0;
+          ++added;
+          ++scored;
+        }
+      len += added;
+      qsort(list, (size_t)len, sizeof(beam_t), cmp_beam);
+      if (len > L) len = L;
+    }
+  }
+  for (int r = 0; r < k; ++r) {
+    out_ids[r] = r < len ? list[r].row : -1;
+    if (out_scores) out_scores[r] = r < len ? list[r].s : 0.0f;
+  }
+  if (out_iters) *out_iters = iters;
+  if (out_scored) *out_scored = scored;
+  free(list);
+  free(seen);
+  free(chosen);
   return ORACLE_OK;
 }
 

@@ -108,6 +108,43 @@ def queries(seed: int, nq: int, dim: int, dtype: str) -> np.ndarray:
     return unit_rows(seed, 3, nq, dim, dtype)
 
 
+def embeddings_low_rank(seed: int, n: int, dim: int, dtype: str, intrinsic_dim: int = 32, noise: float = 0.05,
+                        chunk: int = 65536) -> np.ndarray:  # fmt: skip
+    """Unit-norm rows with low intrinsic dimension, the structure that text embeddings have and isotropic Gaussian
+    rows lack (on which no proximity graph can beat a full scan): a Gaussian latent vector of ``intrinsic_dim``
+    coordinates goes through a fixed random linear map to ``dim`` coordinates, a little isotropic noise is added,
+    and the row is normalised in float32 and rounded to ``dtype``."""
+    proj = _rng(seed, 4).standard_normal((intrinsic_dim, dim)).astype(np.float32) / np.sqrt(intrinsic_dim)
+    out = np.empty((n, dim), dtype=np.float32 if dtype == "float32" else np.float16)
+    for a in range(0, n, chunk):
+        b = min(n, a + chunk)
+        g = _rng(seed, 5, a)
+        z = g.standard_normal((b - a, intrinsic_dim)).astype(np.float32)
+        x = z @ proj + noise * g.standard_normal((b - a, dim)).astype(np.float32)
+        x /= np.linalg.norm(x, axis=1, keepdims=True)
+        out[a:b] = x
+    return out
+
+
+def queries_near_rows(seed: int, emb: np.ndarray, nq: int, noise: float = 0.3) -> np.ndarray:
+    """Queries that resemble stored rows: a random row plus isotropic noise of relative norm ``noise``, normalised."""
+    g = _rng(seed, 6)
+    rows = g.integers(0, emb.shape[0], nq)
+    x = emb[rows].astype(np.float32)
+    x += noise * g.standard_normal(x.shape).astype(np.float32) / np.sqrt(emb.shape[1])
+    x /= np.linalg.norm(x, axis=1, keepdims=True)
+    return x.astype(emb.dtype)
+
+
+def random_graph(seed: int, n: int, deg: int, holes: float = 0.05) -> np.ndarray:
+    """A seeded directed graph as search input: ``deg`` random neighbours per row (repeats and self-loops
+    allowed), a share ``holes`` of the entries set to -1, int32 [n, deg]."""
+    g = _rng(seed, 7)
+    out = g.integers(0, max(n, 1), (n, deg)).astype(np.int32)
+    out[g.random((n, deg)) < holes] = -1
+    return out
+
+
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float32 values to bfloat16 (nearest even) and return the 16-bit patterns."""
     u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)

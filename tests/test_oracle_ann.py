@@ -1,0 +1,140 @@
+"""Pins for the oracle's graph index (CPU only): the fixed-order binary32 scores, the exact neighbour graph and the
+beam search.  Each check is against something other than the oracle's own code: exact sums with a rounding
+behaviour known by construction, numpy's float64 matmul and argsort, brute force over all rows where the search
+must degenerate to it, and walks on a path graph that can be followed by hand."""
+import numpy as np
+
+from paper_2607_27090_b200 import synth
+
+
+def test_f32_scores_follow_the_stated_lane_order(oracle_mod):
+    # dim 512 in halves: 64 vectors of 8, vector v in lane v mod 32, two vectors per lane.
+    # element 0 carries a product of 2^24; a further 1.0 added to 2^24 in binary32 is lost (ties to even).
+    dim = 512
+    row = np.zeros((1, dim), np.float16)
+    q = np.ones(dim, np.float16)
+    row[0, 0], q[0] = 4096.0, 4096.0
+    row[0, 1:8] = 1.0  # same vector, same lane, added after the big product: all seven are lost
+    assert oracle_mod.scores_f32(row, q)[0] == 2.0**24
+    row[0, 256:264] = 1.0  # vector 32 is lane 0 again: lost as well
+    assert oracle_mod.scores_f32(row, q)[0] == 2.0**24
+    row[0, 8:16] = 1.0  # vector 1 is lane 1: its 8 is kept and joins in the butterfly
+    assert oracle_mod.scores_f32(row, q)[0] == 2.0**24 + 8
+    row[0, 1:8] = 0
+    row[0, 256:264] = 0
+    row[0, 8:16] = 0
+    row[0, 504:512] = 0.5  # last vector (63) is lane 31: 8 * 0.5 = 4 survives
+    assert oracle_mod.scores_f32(row, q)[0] == 2.0**24 + 4
+    # float32 rows: vectors of 4 elements
+    r32 = np.zeros((1, 256), np.float32)
+    q32 = np.ones(256, np.float32)
+    r32[0, 0] = 2.0**24
+    r32[0, 1:4] = 1.0  # same vector as element 0
+    r32[0, 128:132] = 1.0  # vector 32: lane 0 again
+    r32[0, 4:8] = 1.0  # vector 1, lane 1
+    assert oracle_mod.scores_f32(r32, q32)[0] == 2.0**24 + 4
+
+
+def test_f32_scores_are_close_to_the_double_scores(oracle_mod):
+    for dtype, dim in (("float16", 1024), ("float32", 64), ("float16", 136)):
+        emb = synth.embeddings(1, 300, dim, dtype)
+        q = synth.queries(1, 1, dim, dtype)[0]
+        exact = oracle_mod.scores(emb, q)
+        assert np.abs(oracle_mod.scores_f32(emb, q) - exact).max() < 3e-7
+
+
+def test_knn_graph_against_numpy_argsort(oracle_mod):
+    emb = synth.embeddings_low_rank(2, 400, 64, "float32", intrinsic_dim=8)
+    emb[37] = emb[5]  # duplicate rows: equal scores against every third row, lower row first
+    g = oracle_mod.knn_graph(emb, 10)
+    s = emb.astype(np.float64) @ emb.astype(np.float64).T
+    np.fill_diagonal(s, -np.inf)
+    for r in (0, 5, 37, 399, 123):
+        order = np.lexsort((np.arange(400), -s[r]))[:10]
+        # numpy's pairwise summation differs from a left-to-right sum in the last bits: compare scores, not ids
+        assert np.allclose(s[r][g[r]], s[r][order], rtol=0, atol=1e-12) and len(set(g[r].tolist())) == 10 and r not in g[r]
+    assert g[5][0] == 37 and g[37][0] == 5
+    both = [r for r in range(400) if 5 in g[r] and 37 in g[r]]
+    assert both and all(list(g[r]).index(5) + 1 == list(g[r]).index(37) for r in both)  # tie: row 5 right before row 37
+    tiny = oracle_mod.knn_graph(emb[:4], 6)
+    assert np.all(tiny[:, 3:] == -1) and np.all(tiny[:, :3] >= 0)  # fewer rows than neighbours: padded
+
+
+def test_search_on_a_complete_graph_is_brute_force(oracle_mod):
+    n, dim, k = 150, 64, 12
+    emb = synth.embeddings(3, n, dim, "float32")
+    complete = np.array([[c for c in range(n) if c != r] for r in range(n)], np.int32)
+    q = synth.queries(3, 4, dim, "float32")
+    res = oracle_mod.ann_search(emb, complete, q, k, beam=4, parents=1, n_entry=1, max_iters=3)
+    want, _ = oracle_mod.retrieve(emb, q, k)
+    assert np.array_equal(res.ids, want)
+    assert np.all(res.scored == n) and np.all(res.iters >= 1)
+    for i in range(4):
+        assert np.array_equal(res.scores[i], oracle_mod.scores_f32(emb, q[i])[res.ids[i]])
+
+
+def test_search_with_a_beam_as_large_as_the_store_visits_the_whole_component(oracle_mod):
+    n, dim = 300, 64
+    emb = synth.embeddings_low_rank(4, n, dim, "float32", intrinsic_dim=6)
+    g = oracle_mod.knn_graph(emb, 8)
+    q = synth.queries_near_rows(4, emb, 3)
+    res = oracle_mod.ann_search(emb, g, q, 10, beam=n, parents=3, n_entry=n, max_iters=1000)
+    want, _ = oracle_mod.retrieve(emb, q, 10)
+    assert np.array_equal(res.ids, want) and np.all(res.scored == n)  # every row is an entry point here
+
+
+def arc(n):
+    a = np.linspace(0.0, 1.0, n)
+    return np.stack([np.cos(a), np.sin(a)] + [np.zeros(n)] * 6, axis=1).astype(np.float32)  # dim 8
+
+
+def test_greedy_walk_on_a_path_graph_can_be_followed_by_hand(oracle_mod):
+    # 100 points on an arc, row i linked to i-1 and i+1; the only entry point is (1 * 2654435761) mod 100 = 61.
+    n = 100
+    emb = arc(n)
+    path = np.array([[i - 1 if i > 0 else -1, i + 1 if i + 1 < n else -1] for i in range(n)], np.int32)
+    q = emb[70:71].copy()
+    # beam 1: each step expands the single listed row and moves one row towards 70; 9 moves, then the step that
+    # expands 70 itself finds nothing better; the next look finds no unexpanded entry
+    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=50)
+    # rows scored: the entry, 60 and 62 in step 1, then one new row per step (the other neighbour was seen): 63..70, 71
+    assert res.ids[0, 0] == 70 and res.iters[0] == 10 and res.scored[0] == 1 + 2 + 8 + 1
+    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=5)
+    assert res.ids[0, 0] == 66 and res.iters[0] == 5
+    # beam 3 keeps the trail: after 4 steps the list is 65, 64, 63 (closest to 70 first)
+    res = oracle_mod.ann_search(emb, path, q, 3, beam=3, parents=1, n_entry=1, max_iters=4)
+    assert res.ids[0].tolist() == [65, 64, 63]
+    # two entry points, 61 and (2 * 2654435761) mod 100 = 22: the walk from 61 still wins, 22 is never expanded first
+    res = oracle_mod.ann_search(emb, path, q, 2, beam=2, parents=1, n_entry=2, max_iters=50)
+    assert res.ids[0].tolist() == [70, 71] or res.ids[0].tolist() == [70, 69]
+    assert abs(float(res.scores[0, 0]) - 1.0) < 1e-6
+
+
+def test_holes_bad_rows_padding_and_duplicate_entry_points(oracle_mod):
+    emb = arc(10)
+    g = np.array([[-1, 11], [0, 2], [1, 1], [2, 2], [-5, 3], [4, 4], [5, 5], [6, 6], [7, 7], [8, 8]], np.int32)
+    # entry (2654435761 mod 10) = 1; from 1 the walk reaches 0 and 2 only; rows 3.. point backwards
+    res = oracle_mod.ann_search(emb, g, emb[9:10], 5, beam=5, parents=2, n_entry=1, max_iters=20)
+    assert sorted(res.ids[0, :3].tolist()) == [0, 1, 2] and res.ids[0, 3:].tolist() == [-1, -1] and res.scored[0] == 3
+    assert res.scores[0, 3:].tolist() == [0.0, 0.0]
+    # 30 entry points on 10 rows: duplicates dropped, at most 10 rows scored
+    res = oracle_mod.ann_search(emb, g, emb[9:10], 3, beam=3, parents=1, n_entry=30, max_iters=0)
+    assert res.scored[0] <= 10 and res.iters[0] == 0 and res.ids[0, 0] >= 0
+    # empty store
+    res = oracle_mod.ann_search(emb[:0], g[:0], emb[9:10], 2)
+    assert res.ids[0].tolist() == [-1, -1]
+
+
+def test_recall_grows_with_the_beam_on_structured_rows(oracle_mod):
+    n, dim, k = 3000, 64, 10
+    emb = synth.embeddings_low_rank(5, n, dim, "float32", intrinsic_dim=8)
+    g = oracle_mod.knn_graph(emb, 16)
+    q = synth.queries_near_rows(5, emb, 20)
+    want, _ = oracle_mod.retrieve(emb, q, k)
+
+    def recall(beam):
+        got = oracle_mod.ann_search(emb, g, q, k, beam=beam, parents=2, n_entry=16, max_iters=200).ids
+        return np.mean([len(set(got[i]) & set(want[i])) / k for i in range(len(q))])
+
+    r_small, r_large = recall(10), recall(96)
+    assert r_large >= r_small and r_large > 0.9
