@@ -194,6 +194,47 @@ ms_status memstore_retrieve(memstore_t* store, const void* queries, const int32_
 ms_status memstore_retrieve_static(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq,
                                    int32_t k, int32_t* out_ids, float* out_scores, ms_stream stream);
 
+/*
+ * Approximate retrieval over a proximity graph (Sec. 2.5: the paper retrieves with a GPU-resident graph index
+ * searched by a beam search; Sec. 6.1: inner-product distance, 64 graph neighbours, beam width 64).  The paper
+ * does not print the index's algorithm; this library's is:
+ *   graph   G[n][degree], row r = the `degree` rows with the largest inner product with row r (r excluded), best
+ *           first, -1 padded: an exact neighbour graph, built on the device by the exact retrieval kernels with
+ *           the rows themselves as queries (n / 64 retrieval calls: an offline step, as in the paper);
+ *   search  a list of at most max(beam, k) rows ordered by score (ties to the lower row) starts from the rows
+ *           ((i + 1) * 2654435761) mod n, i < n_entry; each step marks the first `parents` unexpanded rows of the
+ *           list expanded, scores their neighbours that were never scored before, and keeps the best; it ends
+ *           when no unexpanded row is left or after max_iters steps.  Scores are the fp32 sums of
+ *           memstore_retrieve, so a result differs from the exact one only in which rows were looked at.
+ * Single-segment stores (n_users = 1) only; rows are fact ids there.  The graph covers the facts present when it
+ * was built or set: facts added later are not found until it is rebuilt.
+ */
+typedef struct {
+  int32_t beam;      /* list length (the result needs max(beam, k) <= 256); 0 = 64 */
+  int32_t parents;   /* rows expanded per step, <= 32 and parents * degree <= 512; 0 = 4 */
+  int32_t n_entry;   /* starting rows, <= 512; 0 = 64 */
+  int32_t max_iters; /* step limit; max_iters * parents * degree + n_entry rows must fit the visited table
+                        (about 25,000); 0 = 32 */
+} ms_ann_params;
+
+/* Build the graph of all facts present (degree <= 255); replaces an earlier graph.  Synchronises the device once
+ * (allocation), then enqueues the retrieval calls on `stream`. */
+ms_status memstore_build_graph(memstore_t* store, int32_t degree, ms_stream stream);
+/* Install a caller-made graph: device int32 [n_rows][degree], entries are rows of the segment (others are ignored
+ * by the search), n_rows <= number of facts.  Copied on `stream`. */
+ms_status memstore_set_graph(memstore_t* store, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream);
+/* Copy the graph out: out = device int32 buffer of out_capacity entries or NULL; *out_rows, *out_degree (host,
+ * optional) receive its shape.  MS_ERR_CAPACITY when the buffer is too small. */
+ms_status memstore_get_graph(memstore_t* store, int32_t* out, int64_t out_capacity, int64_t* out_rows, int32_t* out_degree,
+                             ms_stream stream);
+/*
+ * The search.  queries: device [nq][emb_dim]; params NULL = defaults; out_ids device int32 [nq][k] (best first, -1
+ * padded), out_scores device fp32 [nq][k] or NULL, out_counters device int32 [nq][2] or NULL: steps taken and rows
+ * scored per query.  One CTA per query; asynchronous on `stream`.
+ */
+ms_status memstore_retrieve_ann(memstore_t* store, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
+                                int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream);
+
 /* element type of the paged cache */
 enum {
   MS_CACHE_BF16 = 0,    /* the paper's cache */

@@ -1,0 +1,256 @@
+// Approximate retrieval: beam search over a fixed-degree proximity graph held in HBM next to the embeddings
+// (Sec. 2.5 of the paper: a GPU-resident graph index searched by a beam search on the device; Sec. 6.1:
+// inner-product distance, 64 graph neighbours, beam width 64).  The paper does not print the index's algorithm;
+// the one implemented here, step by step:
+//
+//   graph    G[n][deg]: row r lists the deg rows with the largest inner product with row r (r excluded), best
+//            first; -1 pads.  Built by the exact retrieval kernels with the rows themselves as queries.
+//   list     at most L = max(beam, k) entries (score, row, expanded?), ordered by score descending, ties to the
+//            lower row; V = the set of rows ever scored (exact: an open-addressing table in shared memory).
+//   start    rows e_i = ((i + 1) * 2654435761) mod n, i < n_entry (duplicates dropped), scored and listed.
+//   step     the first `parents` unexpanded entries of the list are marked expanded (none left, or max_iters
+//            steps done: stop); their neighbours that are valid rows and not in V join V and are scored;
+//            the best L of list + new form the next list.
+//   result   the first k entries of the list; -1 / 0 pads.
+//
+// Scores are the fp32 sums of the exact retrieval kernels (same lane layout and summation order), so an approximate
+// result differs from the exact one only in WHICH rows were looked at.  Every decision (membership in V, the order
+// of the list) is independent of the order in which threads work, so the result is deterministic.
+#pragma once
+#include "retrieve.cuh"
+
+namespace ms {
+
+constexpr int kAnnThreads = 1024;
+constexpr int kAnnMaxList = 256;   // L = max(beam, k)
+constexpr int kAnnMaxCand = 512;   // rows scored in one step: parents * degree, and n_entry
+constexpr uint32_t kAnnEmpty = 0xffffffffu;
+
+struct AnnParams {
+  const void* emb;      // [n][E] rows of user 0
+  const int32_t* graph; // [n][deg]
+  const void* queries;  // [nq][E]
+  int32_t n, emb_dim, deg;
+  int32_t k, list_len, parents, n_entry, max_iters;
+  uint32_t table_mask;  // visited table: table_mask + 1 slots (a power of two, at least twice the rows ever scored)
+  int32_t* out_ids;     // [nq][k]
+  float* out_scores;    // [nq][k] or nullptr
+  int32_t* out_counters;  // [nq][2] or nullptr: steps taken, rows scored
+};
+
+// key of a list entry: order key of the score, then lower row first, lowest bit = not yet expanded
+__device__ __forceinline__ unsigned long long ann_key(float score, int32_t row, bool unexpanded) {
+  return ((unsigned long long)order_key(score) << 32) | ((unsigned long long)(0x7fffffffu - (uint32_t)row) << 1) |
+         (unexpanded ? 1ull : 0ull);
+}
+__device__ __forceinline__ int32_t ann_key_row(unsigned long long key) {
+  return (int32_t)(0x7fffffffu - (uint32_t)((key & 0xffffffffull) >> 1));
+}
+
+// Scores of two rows at once (two rows' loads in flight per warp) against the query held in shared memory as
+// fp32; lane layout and summation order of score_rows.  All lanes return both sums.
+template <typename T>
+__device__ __forceinline__ void ann_score_pair(const T* seg, int E, const float* s_q, int64_t r0, int64_t r1, bool has1, float& s0,
+                                               float& s1) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int lane = threadIdx.x & 31;
+  const int nvec = E / VEC;
+  const uint4* p0 = reinterpret_cast<const uint4*>(seg + r0 * E);
+  const uint4* p1 = reinterpret_cast<const uint4*>(seg + (has1 ? r1 : r0) * E);
+  float a0 = 0.f, a1 = 0.f;
+  for (int v0 = 0; v0 < nvec; v0 += 128) {
+    uint4 x[4], y[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        x[u] = __ldg(p0 + v);
+        y[u] = __ldg(p1 + v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        const float* qs = s_q + v * VEC;
+        if (sizeof(T) == 2) {
+          float f[8], g[8];
+          unpack8(x[u], f);
+          unpack8(y[u], g);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            a0 = fmaf(f[i], qs[i], a0);
+            a1 = fmaf(g[i], qs[i], a1);
+          }
+        } else {
+          const float* f = reinterpret_cast<const float*>(&x[u]);
+          const float* g = reinterpret_cast<const float*>(&y[u]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            a0 = fmaf(f[i], qs[i], a0);
+            a1 = fmaf(g[i], qs[i], a1);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+  }
+  s0 = a0 + 0.0f;  // -0 -> +0
+  s1 = a1 + 0.0f;
+}
+
+struct AnnShared {
+  unsigned long long list[kAnnMaxList];
+  unsigned long long merged[kAnnMaxList + kAnnMaxCand];
+  int32_t cand[kAnnMaxCand];
+  int32_t parent[32];
+  uint32_t warp_cnt[32];
+  uint32_t n_cand, n_parent, len, n_scored;
+};
+
+// One CTA per query.  Dynamic shared memory: the query as fp32 (emb_dim floats), then the visited table.
+template <typename T>
+__global__ void __launch_bounds__(kAnnThreads, 1) ann_search_kernel(const AnnParams p) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  __shared__ AnnShared sm;
+  float* s_q = reinterpret_cast<float*>(dyn);
+  uint32_t* table = reinterpret_cast<uint32_t*>(dyn + (size_t)p.emb_dim * sizeof(float));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int q = blockIdx.x;
+  const int E = p.emb_dim, n = p.n, L = p.list_len;
+  const T* seg = reinterpret_cast<const T*>(p.emb);
+  const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * E;
+
+  for (int i = tid; i < E; i += kAnnThreads) s_q[i] = (float)qv[i];
+  for (uint32_t i = tid; i <= p.table_mask; i += kAnnThreads) table[i] = kAnnEmpty;
+  if (tid == 0) {
+    sm.n_cand = 0;
+    sm.len = 0;
+    sm.n_scored = 0;
+  }
+  __syncthreads();
+
+  // a row joins V at most once: the thread that claims its slot lists it as a candidate
+  auto visit = [&](int32_t row) {
+    uint32_t slot = ((uint32_t)row * 2654435761u) & p.table_mask;
+    for (uint32_t probe = 0; probe <= p.table_mask; ++probe) {
+      const uint32_t old = atomicCAS(&table[slot], kAnnEmpty, (uint32_t)row);
+      if (old == kAnnEmpty) {
+        const uint32_t c = atomicAdd(&sm.n_cand, 1u);
+        if (c < (uint32_t)kAnnMaxCand) sm.cand[c] = row;
+        return;
+      }
+      if (old == (uint32_t)row) return;
+      slot = (slot + 1) & p.table_mask;
+    }
+  };
+
+  // scores the candidates and merges them into the list (all threads)
+  auto score_and_merge = [&]() {
+    const int n_cand = min((int)sm.n_cand, kAnnMaxCand);
+    const int len = (int)sm.len;
+    for (int i = tid; i < len; i += kAnnThreads) sm.merged[i] = sm.list[i];
+    for (int c = 2 * warp; c < n_cand; c += 2 * (kAnnThreads / 32)) {
+      const bool has1 = c + 1 < n_cand;
+      const int32_t r0 = sm.cand[c], r1 = has1 ? sm.cand[c + 1] : r0;
+      float s0, s1;
+      ann_score_pair<T>(seg, E, s_q, r0, r1, has1, s0, s1);
+      if (lane == 0) {
+        sm.merged[len + c] = ann_key(s0, r0, true);
+        if (has1) sm.merged[len + c + 1] = ann_key(s1, r1, true);
+      }
+    }
+    __syncthreads();
+    // rank by counting (keys are distinct: a row is listed once); the best L stay
+    const int total = len + n_cand;
+    if (tid < total) {
+      const unsigned long long mine = sm.merged[tid];
+      int rank = 0;
+      for (int j = 0; j < total; ++j) rank += sm.merged[j] > mine;
+      if (rank < L) sm.list[rank] = mine;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      sm.len = (uint32_t)min(total, L);
+      sm.n_scored += (uint32_t)n_cand;
+      sm.n_cand = 0;
+    }
+    __syncthreads();
+  };
+
+  int steps = 0;
+  if (n > 0) {
+    if (tid < p.n_entry) visit((int32_t)(((unsigned long long)(tid + 1) * 2654435761ull) % (unsigned long long)n));
+    __syncthreads();
+    score_and_merge();
+    for (; steps < p.max_iters; ++steps) {
+      // the first `parents` unexpanded entries, in list order
+      const int len = (int)sm.len;
+      const bool mine = tid < len && (sm.list[tid] & 1ull);
+      const uint32_t ballot = __ballot_sync(0xffffffffu, mine);
+      if (lane == 0) sm.warp_cnt[warp] = __popc(ballot);
+      __syncthreads();
+      uint32_t before = 0, all = 0;
+      for (int w = 0; w < kAnnMaxList / 32; ++w) {
+        const uint32_t c = sm.warp_cnt[w];
+        before += w < warp ? c : 0u;
+        all += c;
+      }
+      if (all == 0) break;  // uniform: every thread read the same counts
+      const uint32_t rank = before + __popc(ballot & ((1u << lane) - 1u));
+      if (mine && rank < (uint32_t)p.parents) {
+        sm.parent[rank] = ann_key_row(sm.list[tid]);
+        sm.list[tid] &= ~1ull;
+      }
+      if (tid == 0) sm.n_parent = min(all, (uint32_t)p.parents);
+      __syncthreads();
+      const int n_slots = (int)sm.n_parent * p.deg;
+      if (tid < n_slots) {
+        const int32_t nb = __ldg(p.graph + (int64_t)sm.parent[tid / p.deg] * p.deg + tid % p.deg);
+        if (nb >= 0 && nb < n) visit(nb);
+      }
+      __syncthreads();
+      score_and_merge();
+    }
+  }
+  const int len = (int)sm.len;
+  for (int r = tid; r < p.k; r += kAnnThreads) {
+    const bool ok = r < len;
+    const unsigned long long key = ok ? sm.list[r] : 0ull;
+    p.out_ids[(int64_t)q * p.k + r] = ok ? ann_key_row(key) : -1;
+    if (p.out_scores) p.out_scores[(int64_t)q * p.k + r] = ok ? key_score((uint32_t)(key >> 32)) : 0.f;
+  }
+  if (p.out_counters && tid == 0) {
+    p.out_counters[2 * q] = steps;
+    p.out_counters[2 * q + 1] = (int32_t)sm.n_scored;
+  }
+}
+
+// Graph rows of a batch of `nb` consecutive rows starting at `row0` from their top-(deg + 1) lists (exact retrieval
+// with the rows as queries): the row itself is dropped wherever it ranks (rows with duplicates need not rank first),
+// the first deg others stay, -1 pads.
+__global__ void graph_rows_kernel(const int32_t* topk, int k1, int32_t* graph, int deg, int64_t row0, int nb) {
+  const int r = blockIdx.x * blockDim.y + threadIdx.y;  // one warp per row
+  if (r >= nb) return;
+  const int lane = threadIdx.x;
+  const int32_t self = (int32_t)(row0 + r);
+  const int32_t* src = topk + (int64_t)r * k1;
+  int32_t* dst = graph + (row0 + r) * deg;
+  int written = 0;
+  for (int base = 0; base < k1; base += 32) {
+    const int j = base + lane;
+    const int32_t id = j < k1 ? src[j] : -1;
+    const bool keep = id >= 0 && id != self;
+    const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+    const int pos = written + __popc(ballot & ((1u << lane) - 1u));
+    if (keep && pos < deg) dst[pos] = id;
+    written += __popc(ballot);
+  }
+  for (int j = min(written, deg) + lane; j < deg; j += 32) dst[j] = -1;
+}
+
+}  // namespace ms

@@ -17,6 +17,7 @@
 #include "inject_tma.cuh"
 #include "retrieve.cuh"
 #include "score_gemm.cuh"
+#include "ann.cuh"
 
 using namespace ms;
 
@@ -66,6 +67,11 @@ struct memstore {
   std::vector<int64_t> user_count;
   int64_t n_facts = 0, n_resident = 0, kv_tokens_used = 0;
   int32_t max_fact_len = 0;
+  // proximity graph of user 0's rows (memstore_build_graph / memstore_set_graph): [graph_rows][graph_deg]
+  int32_t* graph = nullptr;
+  int64_t graph_rows = 0;
+  int32_t graph_deg = 0;
+  int32_t* graph_topk = nullptr;  // build scratch: [64][deg + 1] ids
   int64_t prefix_off = 0;   // instruction prefix (memstore_set_prefix): first arena token and length (0 = none)
   int32_t prefix_len = 0;
   int64_t prefix_tokens_total = 0;  // arena tokens taken by this and earlier prefixes (not facts)
@@ -418,6 +424,8 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_tickets);
     cudaFree(s->tc_error);
     cudaFree(s->tiles);
+    cudaFree(s->graph);
+    cudaFree(s->graph_topk);
     cudaFree(s->dev_stage);
     if (s->host_stage) cudaFreeHost(s->host_stage);
     if (s->last_done) cudaEventDestroy(s->last_done);
@@ -634,6 +642,139 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
     MS_CUDA(s, cudaGetLastError());
     s->kernels_launched += 2;
   }
+  s->retrieve_calls++;
+  return mark_last(s, st);
+}
+
+// ---- graph index -------------------------------------------------------------------------------------------------
+static ms_status graph_alloc(memstore* s, int64_t n_rows, int32_t degree) {
+  MS_CUDA(s, cudaDeviceSynchronize());
+  cudaFree(s->graph);
+  s->graph = nullptr;
+  s->graph_rows = 0;
+  s->graph_deg = 0;
+  if (n_rows > 0) MS_CUDA(s, cudaMalloc(&s->graph, (size_t)n_rows * degree * sizeof(int32_t)));
+  s->graph_rows = n_rows;
+  s->graph_deg = degree;
+  return MS_OK;
+}
+
+static ms_status graph_check_store(memstore* s, int32_t degree) {
+  if (s->cfg.n_users != 1) return fail(s, MS_ERR_UNSUPPORTED, "the graph index serves single-segment stores (n_users = 1)");
+  if (degree < 1 || degree > kAnnMaxCand || degree + 1 > kTcMaxK)
+    return fail(s, MS_ERR_INVALID_ARG, "degree %d out of range (1..%d)", degree, kTcMaxK - 1);
+  return MS_OK;
+}
+
+ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  ms_status rc = graph_check_store(s, degree);
+  if (rc != MS_OK) return rc;
+  const memstore_config& c = s->cfg;
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t n = s->user_count[0];
+  rc = graph_alloc(s, n, degree);
+  if (rc != MS_OK || n == 0) return rc;
+  constexpr int kBatch = 64;
+  const int k1 = degree + 1;
+  cudaFree(s->graph_topk);
+  s->graph_topk = nullptr;
+  MS_CUDA(s, cudaMalloc(&s->graph_topk, (size_t)kBatch * k1 * sizeof(int32_t)));
+  const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
+  for (int64_t row0 = 0; row0 < n; row0 += kBatch) {
+    const int nb = (int)std::min<int64_t>(kBatch, n - row0);
+    // the rows themselves are the queries: exact top-(degree + 1) of each, the row itself among them
+    rc = memstore_retrieve(s, (const char*)s->emb + (size_t)row0 * row_bytes, nullptr, nb, k1, s->graph_topk, nullptr, stream);
+    if (rc != MS_OK) return rc;
+    graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, degree, row0, nb);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched++;
+  }
+  return MS_OK;
+}
+
+ms_status memstore_set_graph(memstore_t* s, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  ms_status rc = graph_check_store(s, degree);
+  if (rc != MS_OK) return rc;
+  if (n_rows < 0 || n_rows > s->user_count[0] || (n_rows > 0 && !graph))
+    return fail(s, MS_ERR_INVALID_ARG, "graph of %lld rows for a segment of %lld", (long long)n_rows, (long long)s->user_count[0]);
+  DeviceGuard g(s->cfg.device);
+  rc = graph_alloc(s, n_rows, degree);
+  if (rc != MS_OK || n_rows == 0) return rc;
+  MS_CUDA(s, cudaMemcpyAsync(s->graph, graph, (size_t)n_rows * degree * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return MS_OK;
+}
+
+ms_status memstore_get_graph(memstore_t* s, int32_t* out, int64_t out_capacity, int64_t* out_rows, int32_t* out_degree, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  if (out_rows) *out_rows = s->graph_rows;
+  if (out_degree) *out_degree = s->graph_deg;
+  if (!out) return MS_OK;
+  const int64_t need = s->graph_rows * s->graph_deg;
+  if (out_capacity < need) return fail(s, MS_ERR_CAPACITY, "graph holds %lld entries, the buffer %lld", (long long)need, (long long)out_capacity);
+  DeviceGuard g(s->cfg.device);
+  if (need) MS_CUDA(s, cudaMemcpyAsync(out, s->graph, (size_t)need * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return MS_OK;
+}
+
+ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
+                                int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (!s->graph_deg) return fail(s, MS_ERR_INVALID_ARG, "no graph: call memstore_build_graph or memstore_set_graph first");
+  const int beam = params && params->beam > 0 ? params->beam : 64;
+  const int parents = params && params->parents > 0 ? params->parents : 4;
+  const int n_entry = params && params->n_entry > 0 ? params->n_entry : 64;
+  const int max_iters = params && params->max_iters > 0 ? params->max_iters : 32;
+  if (nq < 0 || k < 1 || k > kAnnMaxList || beam > kAnnMaxList)
+    return fail(s, MS_ERR_INVALID_ARG, "nq=%d k=%d beam=%d (k, beam <= %d)", nq, k, beam, kAnnMaxList);
+  if (parents > 32 || (int64_t)parents * s->graph_deg > kAnnMaxCand || n_entry > kAnnMaxCand)
+    return fail(s, MS_ERR_INVALID_ARG, "parents=%d (<= 32, parents * degree <= %d), n_entry=%d (<= %d)", parents, kAnnMaxCand, n_entry, kAnnMaxCand);
+  if (nq == 0) return MS_OK;
+  if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
+  // visited table: a power of two of at least twice the rows that can ever be scored
+  const int64_t max_scored = (int64_t)n_entry + (int64_t)max_iters * parents * s->graph_deg;
+  uint32_t slots = 1024;
+  while ((int64_t)slots < 2 * max_scored && slots < (1u << 20)) slots <<= 1;
+  const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)slots * sizeof(uint32_t);
+  if ((int64_t)slots < 2 * max_scored || smem > 200 * 1024)
+    return fail(s, MS_ERR_UNSUPPORTED, "max_iters * parents * degree = %lld rows do not fit the visited table in shared memory",
+                (long long)max_scored);
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  AnnParams p{};
+  p.emb = s->emb;
+  p.graph = s->graph;
+  p.queries = queries;
+  p.n = (int32_t)s->graph_rows;
+  p.emb_dim = c.emb_dim;
+  p.deg = s->graph_deg;
+  p.k = k;
+  p.list_len = std::max(beam, k);
+  p.parents = parents;
+  p.n_entry = n_entry;
+  p.max_iters = max_iters;
+  p.table_mask = slots - 1;
+  p.out_ids = out_ids;
+  p.out_scores = out_scores;
+  p.out_counters = out_counters;
+  ms_status rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+  if (c.emb_dtype == MS_DTYPE_F16) {
+    MS_CUDA(s, cudaFuncSetAttribute(ann_search_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    ann_search_kernel<__half><<<nq, kAnnThreads, smem, st>>>(p);
+  } else {
+    MS_CUDA(s, cudaFuncSetAttribute(ann_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    ann_search_kernel<float><<<nq, kAnnThreads, smem, st>>>(p);
+  }
+  MS_CUDA(s, cudaGetLastError());
+  s->kernels_launched++;
   s->retrieve_calls++;
   return mark_last(s, st);
 }

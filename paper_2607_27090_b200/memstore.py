@@ -53,6 +53,10 @@ class _PagedCache(C.Structure):
     ]  # fmt: skip
 
 
+class _AnnParams(C.Structure):
+    _fields_ = [("beam", C.c_int32), ("parents", C.c_int32), ("n_entry", C.c_int32), ("max_iters", C.c_int32)]
+
+
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
@@ -65,6 +69,7 @@ EXPORTS = (
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
+    "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann",
 )  # fmt: skip
 
 _lib = None
@@ -97,6 +102,14 @@ def load_library() -> C.CDLL:
     L.memstore_add_facts_host.restype = i32
     L.memstore_add_facts_host.argtypes = [vp, i32, i64, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), vp]
     L.memstore_retrieve.restype = i32
+    L.memstore_build_graph.restype = i32
+    L.memstore_build_graph.argtypes = [vp, i32, vp]
+    L.memstore_set_graph.restype = i32
+    L.memstore_set_graph.argtypes = [vp, vp, i64, i32, vp]
+    L.memstore_get_graph.restype = i32
+    L.memstore_get_graph.argtypes = [vp, vp, i64, C.POINTER(i64), C.POINTER(i32), vp]
+    L.memstore_retrieve_ann.restype = i32
+    L.memstore_retrieve_ann.argtypes = [vp, vp, i32, i32, C.POINTER(_AnnParams), vp, vp, vp, vp]
     L.memstore_rope_table_llama3.restype = i32
     L.memstore_rope_table_llama3.argtypes = [i32, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_float)]
     L.memstore_set_prefix.restype = i32
@@ -326,6 +339,40 @@ class MemStore:
                                          _dev_ptr(out_scores, torch.float32, "out_scores"), _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return out_ids, out_scores
+
+    # -- graph index ------------------------------------------------------------------------------
+    def build_graph(self, degree=64, stream=None) -> None:
+        """Exact neighbour graph of all facts present (single-segment stores), built on the device."""
+        self._check(self._lib.memstore_build_graph(self._h, degree, _stream_ptr(stream)))
+
+    def set_graph(self, graph: torch.Tensor, stream=None) -> None:
+        """Install a graph: int32 device tensor [n_rows, degree] of row numbers."""
+        self._check(self._lib.memstore_set_graph(self._h, _dev_ptr(graph, torch.int32, "graph"), graph.shape[0], graph.shape[1],
+                                                 _stream_ptr(stream)))  # fmt: skip
+
+    def get_graph(self, stream=None) -> torch.Tensor:
+        rows, deg = C.c_int64(0), C.c_int32(0)
+        self._check(self._lib.memstore_get_graph(self._h, None, 0, C.byref(rows), C.byref(deg), _stream_ptr(stream)))
+        out = torch.empty((rows.value, deg.value), dtype=torch.int32, device=self.device)
+        self._check(self._lib.memstore_get_graph(self._h, _dev_ptr(out, torch.int32, "out"), out.numel(), None, None, _stream_ptr(stream)))
+        return out
+
+    def retrieve_ann(self, queries, k, beam=0, parents=0, n_entry=0, max_iters=0, out_ids=None, out_scores=None, want_scores=True,
+                     want_counters=False, stream=None):  # fmt: skip
+        """Beam search over the graph (0 = the library's default for that parameter).  Returns (ids, scores) or, with
+        ``want_counters``, (ids, scores, counters [nq, 2] = steps taken and rows scored)."""
+        nq = queries.shape[0]
+        if out_ids is None:
+            out_ids = torch.empty((nq, k), dtype=torch.int32, device=queries.device)
+        if out_scores is None and want_scores:
+            out_scores = torch.empty((nq, k), dtype=torch.float32, device=queries.device)
+        counters = torch.zeros((nq, 2), dtype=torch.int32, device=queries.device) if want_counters else None
+        prm = _AnnParams(beam, parents, n_entry, max_iters)
+        rc = self._lib.memstore_retrieve_ann(self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"), nq, k, C.byref(prm),
+                                             _dev_ptr(out_ids, torch.int32, "out_ids"), _dev_ptr(out_scores, torch.float32, "out_scores"),
+                                             _dev_ptr(counters, torch.int32, "counters"), _stream_ptr(stream))  # fmt: skip
+        self._check(rc)
+        return (out_ids, out_scores, counters) if want_counters else (out_ids, out_scores)
 
     def retrieve_static(self, queries, k, query_users=None, out_ids=None, out_scores=None, want_scores=True, stream=None):
         """``retrieve`` through the entry point that never allocates device memory, for callers that cannot let the

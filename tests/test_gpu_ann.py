@@ -1,0 +1,141 @@
+"""GPU parity tests of the graph index: the beam search against the oracle's (bit for bit: both compare fp32 scores
+formed in the same order), the graph build against the oracle's exact neighbour graph (near-tie rule of the exact
+retrieval), recall against exact retrieval on structured rows, and the error paths."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_27090_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    import oracle
+    from parity import to_dev
+    from paper_2607_27090_b200.memstore import MemStore, MemStoreError
+
+DEV = "cuda"
+
+
+def emb_store(emb, n_users=1):
+    n, E = emb.shape
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float32 if emb.dtype == np.float32 else torch.float16,
+                  rope_theta=1e4, n_users=n_users, max_facts_per_user=max(n, 1), max_kv_tokens=0)  # fmt: skip
+    for a in range(0, n, 50_000):
+        b = min(n, a + 50_000)
+        ms.add_facts(to_dev(emb[a:b]), np.zeros(b - a, np.int32))
+    return ms
+
+
+@pytest.mark.parametrize("dtype,dim,n,deg,kind", [
+    ("float32", 64, 3000, 16, "knn"), ("float16", 1024, 2000, 64, "random"), ("float16", 136, 5000, 8, "random"),
+    ("float16", 256, 700, 32, "knn"), ("float32", 8, 40, 4, "random"),
+])  # fmt: skip
+def test_search_equals_the_oracle_bit_for_bit(dtype, dim, n, deg, kind):
+    emb = synth.embeddings_low_rank(80, n, dim, dtype, intrinsic_dim=min(8, dim))
+    emb[n // 2] = emb[3]  # equal scores: the lower row goes first
+    graph = oracle.knn_graph(emb, deg) if kind == "knn" else synth.random_graph(81, n, deg)
+    if kind == "random":
+        graph[5, 0] = n + 7  # a row outside the segment is ignored
+    q = synth.queries_near_rows(82, emb, 9)
+    q[0] = emb[3]
+    ms = emb_store(emb)
+    ms.set_graph(to_dev(graph))
+    assert torch.equal(ms.get_graph().cpu(), torch.from_numpy(graph))
+    for k, beam, parents, n_entry, max_iters in ((10, 64, 4, 64, 32), (1, 1, 1, 1, 50), (50, 16, 2, 7, 5), (100, 128, 8, 200, 12),
+                                                  (256, 256, 1, 512, 3)):  # fmt: skip
+        if parents * deg > 512:
+            continue
+        want = oracle.ann_search(emb, graph, q, k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters)
+        ids, sc, cnt = ms.retrieve_ann(to_dev(q), k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters, want_counters=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(ids.cpu().numpy(), want.ids), (k, beam, parents, n_entry, max_iters)
+        assert np.array_equal(sc.cpu().numpy().view(np.uint32), want.scores.view(np.uint32))
+        assert np.array_equal(cnt[:, 0].cpu().numpy(), want.iters) and np.array_equal(cnt[:, 1].cpu().numpy(), want.scored)
+    # the scores are those of the exact path
+    ids, sc = ms.retrieve_ann(to_dev(q), 5)
+    ex_ids, ex_sc = ms.retrieve(to_dev(q), n if n < 100 else 100)
+    for i in range(len(q)):
+        lookup = dict(zip(ex_ids[i].tolist(), ex_sc[i].tolist()))
+        assert all(lookup.get(a, b) == b for a, b in zip(ids[i].tolist(), sc[i].tolist()))
+    ms.close()
+
+
+@pytest.mark.parametrize("dtype,dim,n,deg", [("float32", 64, 2500, 16), ("float16", 128, 9000, 64), ("float16", 64, 30, 40)])
+def test_graph_build_matches_the_exact_neighbour_graph(dtype, dim, n, deg):
+    """Rows as queries through the exact retrieval kernels (CUDA-core path below 8193 rows, tensor-core filter
+    above); compared with the oracle's graph under the near-tie rule of exact retrieval."""
+    emb = synth.embeddings_low_rank(83, n, dim, dtype, intrinsic_dim=min(8, dim))
+    for r in (7, 11, 19):
+        emb[r] = emb[2]  # four identical rows
+    ms = emb_store(emb)
+    ms.build_graph(deg)
+    g = ms.get_graph().cpu().numpy()
+    assert g.shape == (n, deg)
+    want = oracle.knn_graph(emb, deg)
+    rows = list(range(0, n, max(1, n // 40))) + [2, 7, 11, 19, n - 1]
+    exact_same = 0
+    for r in rows:
+        got = g[r]
+        valid = got[got >= 0]
+        assert len(valid) == min(deg, n - 1) and np.all(got[len(valid):] == -1)
+        assert r not in valid and len(set(valid.tolist())) == len(valid) and np.all(valid < n)
+        s_got = oracle.scores(emb[valid], emb[r])
+        s_want = oracle.scores(emb[want[r][: len(valid)]], emb[r])
+        assert np.all(np.abs(s_got.astype(np.float32) - s_want.astype(np.float32)) < 1e-5)
+        exact_same += int(np.array_equal(valid, want[r][: len(valid)]))
+    assert exact_same >= len(rows) * 0.8
+    assert set(g[2][:3].tolist()) == {7, 11, 19} and g[7][0] == 2
+    ms.close()
+
+
+def test_recall_against_exact_retrieval_on_structured_rows():
+    n, dim, k = 60_000, 128, 10
+    emb = synth.embeddings_low_rank(84, n, dim, "float16", intrinsic_dim=16)
+    q = synth.queries_near_rows(85, emb, 48)
+    ms = emb_store(emb)
+    ms.build_graph(32)
+    ex_ids, _ = ms.retrieve(to_dev(q), k)
+    recalls = {}
+    for beam in (16, 64, 128):
+        ids, _, cnt = ms.retrieve_ann(to_dev(q), k, beam=beam, want_counters=True)
+        a, b = ids.cpu().numpy(), ex_ids.cpu().numpy()
+        recalls[beam] = float(np.mean([len(set(a[i]) & set(b[i])) / k for i in range(len(q))]))
+        assert int(cnt[:, 1].max()) < n // 4  # far fewer rows scored than a scan
+    assert recalls[64] >= 0.9 and recalls[128] >= recalls[16]
+    # the library's graph, handed to the oracle, gives the oracle the same answers (search parity at this size)
+    g = ms.get_graph().cpu().numpy()
+    want = oracle.ann_search(emb, g, q[:6], k)
+    ids, sc = ms.retrieve_ann(to_dev(q[:6]), k)
+    assert np.array_equal(ids.cpu().numpy(), want.ids)
+    ms.close()
+
+
+def test_graph_index_errors_and_empty_cases():
+    emb = synth.embeddings(86, 100, 64, "float16")
+    ms = emb_store(emb)
+    q = to_dev(synth.queries(86, 2, 64, "float16"))
+    with pytest.raises(MemStoreError):  # no graph yet
+        ms.retrieve_ann(q, 5)
+    ms.build_graph(8)
+    for bad in (dict(beam=300), dict(parents=33), dict(parents=8, n_entry=513), dict(max_iters=100000)):
+        with pytest.raises(MemStoreError):
+            ms.retrieve_ann(q, 5, **bad)
+    with pytest.raises(MemStoreError):
+        ms.retrieve_ann(q, 300)
+    with pytest.raises(MemStoreError):
+        ms.build_graph(0)
+    with pytest.raises(MemStoreError):
+        ms.set_graph(torch.zeros((101, 4), dtype=torch.int32, device=DEV))  # more rows than facts
+    ids, _ = ms.retrieve_ann(q, 5)  # still usable after the refused calls
+    assert bool((ids >= 0).all())
+    ms.close()
+    two = emb_store(emb[:50], n_users=2)
+    with pytest.raises(MemStoreError):
+        two.build_graph(8)
+    two.close()
+    empty = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=64, rope_theta=1e4, max_facts_per_user=10, max_kv_tokens=0)
+    empty.build_graph(4)
+    ids, sc = empty.retrieve_ann(q, 3)
+    assert ids.cpu().tolist() == [[-1] * 3] * 2 and sc.cpu().tolist() == [[0.0] * 3] * 2
+    empty.close()
