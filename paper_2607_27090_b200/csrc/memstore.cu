@@ -169,7 +169,10 @@ cudaError_t ensure_fused_smem(int device, size_t bytes) {
 }
 
 // ---- tensor-core retrieve path -------------------------------------------------------------------------------
-constexpr int kTcMinQueries = 8;     // below this the CUDA-core kernels re-reading the segment per query are cheaper
+constexpr int kTcMinQueries = 8;     // below this the CUDA-core kernels re-reading the segment per query are cheaper ...
+constexpr int64_t kTcFewQueriesRows = 131072;  // ... unless the segment is long: the filter reads it once whatever the number
+                                               // of queries and leaves 1/8 of the scores to select from, while the CUDA-core
+                                               // path ends in one CTA selecting among ALL scores at one SM's bandwidth
 constexpr int kTcMaxK = 256;
 constexpr int kTcGroupMargin = 28;   // groups selected beyond k: slack for tensor-core vs CUDA-core rounding at the k-th score
 constexpr int kTcMaxK2 = kTcMaxK + kTcGroupMargin;
@@ -177,7 +180,7 @@ constexpr int kTcMaxK2 = kTcMaxK + kTcGroupMargin;
 bool tc_path_applies(const memstore* s, const int32_t* query_users, int nq, int k, int64_t n_max) {
   const memstore_config& c = s->cfg;
   return c.emb_dtype == MS_DTYPE_F16 && c.emb_dim % kGemmKChunk == 0 && c.emb_dim <= kGemmMaxE && !query_users &&
-         nq >= kTcMinQueries && k <= kTcMaxK && n_max > kFusedMaxRows;
+         (nq >= kTcMinQueries || n_max >= kTcFewQueriesRows) && k <= kTcMaxK && n_max > kFusedMaxRows;
 }
 
 ms_status tc_prepare(memstore* s) {

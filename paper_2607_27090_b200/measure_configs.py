@@ -173,6 +173,61 @@ def measure_variants(iters: int, seed: int = 0, n_facts: int = 400, k: int = 50)
     return lines
 
 
+def measure_ann(n: int, iters: int, seed: int = 0, dim: int = 1024, degree: int = 64, k: int = 50, intrinsic_dim: int = 32):
+    """Graph index on an embedding-only store of ``n`` structured rows (low intrinsic dimension, queries near stored
+    rows): build time, search time for 1 and for 64 queries, rows scored, recall against the exact retrieval of the
+    same store, and the exact retrieval times beside them."""
+    import time
+
+    dev = torch.device("cuda")
+    emb = synth.embeddings_low_rank(seed, n, dim, "float16", intrinsic_dim=intrinsic_dim)
+    q = synth.queries_near_rows(seed, emb, 64)
+    store = M.MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=dim, rope_theta=1e4, max_facts_per_user=n, max_kv_tokens=0)
+    for a in range(0, n, 65536):
+        b = min(n, a + 65536)
+        store.add_facts(torch.from_numpy(emb[a:b]).to(dev), [0] * (b - a))
+    q_dev = torch.from_numpy(q).to(dev)
+    stream = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    store.build_graph(degree, stream=stream)
+    torch.cuda.synchronize()
+    build_s = time.perf_counter() - t0
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / iters
+
+    ids_e = torch.empty((64, k), dtype=torch.int32, device=dev)
+    ids_a = torch.empty((64, k), dtype=torch.int32, device=dev)
+    exact_64 = timed(lambda: store.retrieve(q_dev, k, out_ids=ids_e, want_scores=False, stream=stream))
+    exact_1 = timed(lambda: store.retrieve(q_dev[:1], k, out_ids=ids_e[:1], want_scores=False, stream=stream))
+    store.retrieve(q_dev, k, out_ids=ids_e, want_scores=False, stream=stream)
+    lines = []
+    for beam in (64, 128, 256):
+        L = max(beam, k)
+        ann_64 = timed(lambda: store.retrieve_ann(q_dev, k, beam=L, out_ids=ids_a, want_scores=False, stream=stream))
+        ann_1 = timed(lambda: store.retrieve_ann(q_dev[:1], k, beam=L, out_ids=ids_a[:1], want_scores=False, stream=stream))
+        _, _, cnt = store.retrieve_ann(q_dev, k, beam=L, out_ids=ids_a, want_scores=False, want_counters=True, stream=stream)
+        torch.cuda.synchronize()
+        a, b = ids_a.cpu().numpy(), ids_e.cpu().numpy()
+        recall = float(np.mean([len(set(a[i]) & set(b[i])) / k for i in range(64)]))
+        lines.append({"config": f"graph index, {n} rows x {dim} fp16, degree {degree}", "k": k, "beam": L, "build_s": build_s,
+                      "recall_at_k": recall, "ann_us_1_query": ann_1, "ann_us_64_queries": ann_64,
+                      "exact_us_1_query": exact_1, "exact_us_64_queries": exact_64,
+                      "mean_steps": float(cnt[:, 0].float().mean()), "mean_rows_scored": float(cnt[:, 1].float().mean())})  # fmt: skip
+    store.close()
+    return lines
+
+
 def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
     s = synth.CONFIGS[name]
     dev = torch.device("cuda")
@@ -253,8 +308,12 @@ if __name__ == "__main__":
     ap.add_argument("--retrieve-only", action="store_true", help="embedding-only store, time the batched retrieval alone")
     ap.add_argument("--host-tier", action="store_true", help="Llama shape with all K/V in the pinned host arena: inject over PCIe")
     ap.add_argument("--variants", action="store_true", help="Llama shape: bf16 cache, e4m3 cache, partial rotary (inject only)")
+    ap.add_argument("--ann", type=int, default=0, metavar="ROWS", help="graph index on ROWS structured embedding rows")
     a = ap.parse_args()
-    if a.variants:
+    if a.ann:
+        for ln in measure_ann(a.ann, a.iters, a.seed):
+            print(json.dumps(ln))
+    elif a.variants:
         for ln in measure_variants(a.iters, a.seed):
             print(json.dumps(ln))
     elif a.host_tier:

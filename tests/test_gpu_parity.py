@@ -152,6 +152,12 @@ def test_retrieve_long_segment_group_selection_from_a_sample(case):
     ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
     for i in range(nq):
         check_ids(ids[i], sc[i], emb, q[i], k)
+    # on a segment this long one query, or three, take the same filter path: identical results
+    ids1, sc1 = ms.retrieve(to_dev(q[:1]), k)
+    ids3, sc3 = ms.retrieve(to_dev(q[2:5]), k)
+    torch.cuda.synchronize()
+    assert np.array_equal(ids1.cpu().numpy()[0], ids[0]) and np.array_equal(sc1.cpu().numpy()[0], sc[0])
+    assert np.array_equal(ids3.cpu().numpy(), ids[2:5]) and np.array_equal(sc3.cpu().numpy(), sc[2:5])
     ms.close()
 
 
