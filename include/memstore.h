@@ -211,10 +211,10 @@ ms_status memstore_retrieve_static(memstore_t* store, const void* queries, const
  */
 typedef struct {
   int32_t beam;      /* list length (the result needs max(beam, k) <= 256); 0 = 64 */
-  int32_t parents;   /* rows expanded per step, <= 32 and parents * degree <= 512; 0 = 4 */
+  int32_t parents;   /* rows expanded per step, <= 32 and parents * degree <= 512; 0 = min(8, 512 / degree) */
   int32_t n_entry;   /* starting rows, <= 512; 0 = 64 */
   int32_t max_iters; /* step limit; max_iters * parents * degree + n_entry rows must fit the visited table
-                        (about 25,000); 0 = 32 */
+                        (about 39,000 rows for 1024-d embeddings); 0 = 32 */
 } ms_ann_params;
 
 /* Build the graph of all facts present (degree <= 255); replaces an earlier graph.  Synchronises the device once

@@ -207,7 +207,7 @@ class AnnResult:
         self.ids, self.scores, self.iters, self.scored = ids, scores, iters, scored
 
 
-def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, beam: int = 64, parents: int = 4,
+def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, beam: int = 64, parents: int = 8,
                n_entry: int = 64, max_iters: int = 32) -> AnnResult:  # fmt: skip
     """Beam search over ``graph`` for each query: ids / scores [nq, k], steps taken and rows scored per query."""
     emb = np.ascontiguousarray(emb)

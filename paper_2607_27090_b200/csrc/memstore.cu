@@ -732,7 +732,7 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
   const memstore_config& c = s->cfg;
   if (!s->graph_deg) return fail(s, MS_ERR_INVALID_ARG, "no graph: call memstore_build_graph or memstore_set_graph first");
   const int beam = params && params->beam > 0 ? params->beam : 64;
-  const int parents = params && params->parents > 0 ? params->parents : 4;
+  const int parents = params && params->parents > 0 ? params->parents : std::max(1, std::min(8, kAnnMaxCand / s->graph_deg));
   const int n_entry = params && params->n_entry > 0 ? params->n_entry : 64;
   const int max_iters = params && params->max_iters > 0 ? params->max_iters : 32;
   if (nq < 0 || k < 1 || k > kAnnMaxList || beam > kAnnMaxList)
@@ -741,12 +741,14 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
     return fail(s, MS_ERR_INVALID_ARG, "parents=%d (<= 32, parents * degree <= %d), n_entry=%d (<= %d)", parents, kAnnMaxCand, n_entry, kAnnMaxCand);
   if (nq == 0) return MS_OK;
   if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
-  // visited table: a power of two of at least twice the rows that can ever be scored
+  // visited table: a power of two that the rows that can ever be scored fill to 80 % at most (a search that
+  // converges, as searches do, scores a fraction of that bound)
   const int64_t max_scored = (int64_t)n_entry + (int64_t)max_iters * parents * s->graph_deg;
+  const int64_t want_slots = max_scored + max_scored / 4;
   uint32_t slots = 1024;
-  while ((int64_t)slots < 2 * max_scored && slots < (1u << 20)) slots <<= 1;
+  while ((int64_t)slots < want_slots && slots < (1u << 20)) slots <<= 1;
   const size_t smem = (size_t)c.emb_dim * sizeof(float) + (size_t)slots * sizeof(uint32_t);
-  if ((int64_t)slots < 2 * max_scored || smem > 200 * 1024)
+  if ((int64_t)slots < want_slots || smem > 200 * 1024)
     return fail(s, MS_ERR_UNSUPPORTED, "max_iters * parents * degree = %lld rows do not fit the visited table in shared memory",
                 (long long)max_scored);
   DeviceGuard g(c.device);
@@ -769,14 +771,31 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
   p.out_counters = out_counters;
   ms_status rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
-  if (c.emb_dtype == MS_DTYPE_F16) {
-    MS_CUDA(s, cudaFuncSetAttribute(ann_search_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    ann_search_kernel<__half><<<nq, kAnnThreads, smem, st>>>(p);
-  } else {
-    MS_CUDA(s, cudaFuncSetAttribute(ann_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    ann_search_kernel<float><<<nq, kAnnThreads, smem, st>>>(p);
+  // one cluster per query; its size spreads a small batch over the GPU (a single SM cannot pull the candidate rows
+  // fast enough), shrinking as the batch grows so that all clusters still run at once
+  int cluster = 8;
+  while (cluster > 1 && (int64_t)nq * cluster > s->sm_count) cluster >>= 1;
+  const void* fn = c.emb_dtype == MS_DTYPE_F16 ? (const void*)ann_search_kernel<__half> : (const void*)ann_search_kernel<float>;
+  MS_CUDA(s, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  cudaLaunchConfig_t lc{};
+  cudaLaunchAttribute attr[1];
+  lc.blockDim = dim3(kAnnThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  for (;; cluster >>= 1) {  // a cluster that the device cannot co-schedule with this much shared memory: halve it
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.gridDim = dim3((unsigned)nq * (unsigned)cluster);
+    int n_clusters = 0;
+    if (cluster == 1 || (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess && n_clusters > 0)) break;
+    cudaGetLastError();
   }
-  MS_CUDA(s, cudaGetLastError());
+  void* args[] = {(void*)&p};
+  MS_CUDA(s, cudaLaunchKernelExC(&lc, fn, args));
   s->kernels_launched++;
   s->retrieve_calls++;
   return mark_last(s, st);

@@ -105,7 +105,7 @@ def test_recall_against_exact_retrieval_on_structured_rows():
     assert recalls[64] >= 0.9 and recalls[128] >= recalls[16]
     # the library's graph, handed to the oracle, gives the oracle the same answers (search parity at this size)
     g = ms.get_graph().cpu().numpy()
-    want = oracle.ann_search(emb, g, q[:6], k)
+    want = oracle.ann_search(emb, g, q[:6], k, beam=64, parents=8, n_entry=64, max_iters=32)  # the library's defaults at degree 32
     ids, sc = ms.retrieve_ann(to_dev(q[:6]), k)
     assert np.array_equal(ids.cpu().numpy(), want.ids)
     ms.close()
