@@ -498,7 +498,9 @@ __device__ bool topk_sampled(TopkShared& sm, const float* sc, int n, int k, cons
   return true;
 }
 
-template <int THREADS>
+// LONG = false leaves out the code for long lists in global memory (vector sweeps, sampled bucket choice): the fused
+// kernels, whose keys sit in shared memory, stay small.
+template <int THREADS, bool LONG = true>
 __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys, int n, int k, const IdMap ids,
                            int32_t* out_ids, float* out_scores, bool have_minmax = false, uint32_t my_lo = 0xffffffffu,
                            uint32_t my_hi = 0u) {
@@ -509,17 +511,22 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   // The fast path below works on the SCORES (a key converts back without loss): most elements then cost one
   // comparison per pass.  Long lists in global memory are swept with vector loads.
   auto score_at = [&](int i) -> float { return keys ? key_score(keys[i]) : __ldcg(sc + i); };
-  const bool vec = keys == nullptr && n >= THREADS * 16 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0;
+  const bool vec = LONG && keys == nullptr && n >= THREADS * 16 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0;
   auto sweep = [&](auto visit) {
-    if (vec)
-      for_each_score_vec4<THREADS, 4>(sc, n, visit);
-    else
-      for_each_key<THREADS>(n, score_at, visit);
+    if constexpr (LONG) {
+      if (vec) {
+        for_each_score_vec4<THREADS, 4>(sc, n, visit);
+        return;
+      }
+    }
+    for_each_key<THREADS>(n, score_at, visit);
   };
 
   // ---- sampled path: long lists in global memory, bucket choice from a sample, ONE sweep of the list ------
-  if (n > k && vec && !have_minmax && n >= kSampleMinN) {
-    if (topk_sampled<THREADS>(sm, sc, n, k, ids, out_ids, out_scores)) return;
+  if constexpr (LONG) {
+    if (n > k && vec && !have_minmax && n >= kSampleMinN) {
+      if (topk_sampled<THREADS>(sm, sc, n, k, ids, out_ids, out_scores)) return;
+    }
   }
 
   // ---- fast path: one histogram over 256 LINEAR buckets of the score range -------------------------------
@@ -748,7 +755,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   }
   __syncthreads();
   // with a single user segment facts are numbered in row order: the row is the fact id
-  topk_block<THREADS>(sm, sc, s_keys, n, p.k,
+  topk_block<THREADS, false>(sm, sc, s_keys, n, p.k,
                             IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
@@ -911,7 +918,7 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
     hi = max(hi, kx);
   }
   __syncthreads();
-  topk_block<kScoreThreads>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
+  topk_block<kScoreThreads, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
                             p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo, hi);
 }
 
