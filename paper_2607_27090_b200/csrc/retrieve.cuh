@@ -858,6 +858,66 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
   return acc;
 }
 
+// Two rows at once (both rows' loads in flight together), each with the lane layout and summation order of
+// score_rows; all lanes return both sums.
+template <typename T>
+__device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, const T* seg, int64_t row0, int64_t row1, float& s0,
+                                               float& s1) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int E = p.emb_dim;
+  const int lane = threadIdx.x & 31;
+  const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
+  const uint4* r0 = reinterpret_cast<const uint4*>(seg + row0 * E);
+  const uint4* r1 = reinterpret_cast<const uint4*>(seg + row1 * E);
+  const int nvec = E / VEC;
+  float a0 = 0.f, a1 = 0.f;
+  for (int v0 = 0; v0 < nvec; v0 += 128) {
+    uint4 x[4], z[4], y[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        x[u] = __ldg(r0 + v);
+        z[u] = __ldg(r1 + v);
+        y[u] = __ldg(qp + v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        if (sizeof(T) == 2) {
+          float f[8], h[8], g[8];
+          unpack8(x[u], f);
+          unpack8(z[u], h);
+          unpack8(y[u], g);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            a0 = fmaf(f[i], g[i], a0);
+            a1 = fmaf(h[i], g[i], a1);
+          }
+        } else {
+          const float* f = reinterpret_cast<const float*>(&x[u]);
+          const float* h = reinterpret_cast<const float*>(&z[u]);
+          const float* g = reinterpret_cast<const float*>(&y[u]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            a0 = fmaf(f[i], g[i], a0);
+            a1 = fmaf(h[i], g[i], a1);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+  }
+  s0 = a0;
+  s1 = a1;
+}
+
 // Step 3: rescore the rows of the selected groups exactly (fp32 CUDA-core sums, the same arithmetic as the other
 // retrieve kernels) and take the top-k of these candidates.  grid = (candidate groups of 8 rows per warp..., nq);
 // candidate c of query q is row sel[q][c / 8] * 8 + c % 8.  The last CTA of a query (wait-free ticket) selects.
@@ -879,14 +939,22 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
     const int g_idx = c0 / 8 + warp;
     if (g_idx < k2) {
       const int32_t g = sel[(int64_t)q * k2 + g_idx];
-      for (int r = 0; r < 8; ++r) {
+      for (int r = 0; r < 8; r += 2) {  // two rows of the group in flight at a time
         const int64_t row = (int64_t)g * 8 + r;
-        const bool ok = g >= 0 && row < n_rows;
-        float s = -INFINITY;
-        if (ok) s = score_one_row<T>(p, q, seg, row) + 0.0f;
+        const bool ok0 = g >= 0 && row < n_rows, ok1 = g >= 0 && row + 1 < n_rows;
+        float s0 = -INFINITY, s1 = -INFINITY;
+        if (ok1) {
+          score_two_rows<T>(p, q, seg, row, row + 1, s0, s1);
+          s0 += 0.0f;
+          s1 += 0.0f;
+        } else if (ok0) {
+          s0 = score_one_row<T>(p, q, seg, row) + 0.0f;
+        }
         if (lane == 0) {
-          cs[g_idx * 8 + r] = s;
-          cr[g_idx * 8 + r] = ok ? (int32_t)row : -1;
+          cs[g_idx * 8 + r] = s0;
+          cr[g_idx * 8 + r] = ok0 ? (int32_t)row : -1;
+          cs[g_idx * 8 + r + 1] = s1;
+          cr[g_idx * 8 + r + 1] = ok1 ? (int32_t)(row + 1) : -1;
         }
       }
     }
