@@ -100,6 +100,66 @@ __device__ __forceinline__ void score_rows(const RetrieveParams& p, const float*
   }
 }
 
+// Two rows at once (both rows' loads in flight together), each with the lane layout and summation order of
+// score_rows; all lanes return both sums.
+template <typename T>
+__device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, const T* seg, int64_t row0, int64_t row1, float& s0,
+                                               float& s1) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int E = p.emb_dim;
+  const int lane = threadIdx.x & 31;
+  const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
+  const uint4* r0 = reinterpret_cast<const uint4*>(seg + row0 * E);
+  const uint4* r1 = reinterpret_cast<const uint4*>(seg + row1 * E);
+  const int nvec = E / VEC;
+  float a0 = 0.f, a1 = 0.f;
+  for (int v0 = 0; v0 < nvec; v0 += 128) {
+    uint4 x[4], z[4], y[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        x[u] = __ldg(r0 + v);
+        z[u] = __ldg(r1 + v);
+        y[u] = __ldg(qp + v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        if (sizeof(T) == 2) {
+          float f[8], h[8], g[8];
+          unpack8(x[u], f);
+          unpack8(z[u], h);
+          unpack8(y[u], g);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            a0 = fmaf(f[i], g[i], a0);
+            a1 = fmaf(h[i], g[i], a1);
+          }
+        } else {
+          const float* f = reinterpret_cast<const float*>(&x[u]);
+          const float* h = reinterpret_cast<const float*>(&z[u]);
+          const float* g = reinterpret_cast<const float*>(&y[u]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            a0 = fmaf(f[i], g[i], a0);
+            a1 = fmaf(h[i], g[i], a1);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+  }
+  s0 = a0;
+  s1 = a1;
+}
+
 // The same scoring with the query read straight from global memory (through L1) next to the row, so that one
 // memory round trip serves both and no shared-memory staging or barrier is needed.  Same lane layout and
 // summation order as score_rows.
@@ -112,7 +172,20 @@ __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q
   const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
   const int64_t row_end = min(row0 + rows_per_cta, (int64_t)n);
   const int nvec = E / VEC;
-  for (int64_t row = row0 + warp; row < row_end; row += WARPS) {
+  int64_t row = row0 + warp;
+  if constexpr (WARPS <= 8) {
+    // small CTAs (many queries in flight): two rows per warp at a time, which keeps about 128 KB of loads in flight
+    // per SM; the 1024-thread CTAs of the few-query case have no registers for that
+    for (; row + WARPS < row_end; row += 2 * WARPS) {
+      float s0, s1;
+      score_two_rows<T>(p, q, seg, row, row + WARPS, s0, s1);
+      if (lane == 0) {
+        p.scores[(int64_t)q * p.score_stride + row] = s0 + 0.0f;
+        p.scores[(int64_t)q * p.score_stride + row + WARPS] = s1 + 0.0f;
+      }
+    }
+  }
+  for (; row < row_end; row += WARPS) {
     const uint4* rp = reinterpret_cast<const uint4*>(seg + row * E);
     float acc = 0.f;
     for (int v0 = 0; v0 < nvec; v0 += 128) {
@@ -856,66 +929,6 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   return acc;
-}
-
-// Two rows at once (both rows' loads in flight together), each with the lane layout and summation order of
-// score_rows; all lanes return both sums.
-template <typename T>
-__device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, const T* seg, int64_t row0, int64_t row1, float& s0,
-                                               float& s1) {
-  constexpr int VEC = 16 / sizeof(T);
-  const int E = p.emb_dim;
-  const int lane = threadIdx.x & 31;
-  const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.queries) + (int64_t)q * E);
-  const uint4* r0 = reinterpret_cast<const uint4*>(seg + row0 * E);
-  const uint4* r1 = reinterpret_cast<const uint4*>(seg + row1 * E);
-  const int nvec = E / VEC;
-  float a0 = 0.f, a1 = 0.f;
-  for (int v0 = 0; v0 < nvec; v0 += 128) {
-    uint4 x[4], z[4], y[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int v = v0 + u * 32 + lane;
-      if (v < nvec) {
-        x[u] = __ldg(r0 + v);
-        z[u] = __ldg(r1 + v);
-        y[u] = __ldg(qp + v);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int v = v0 + u * 32 + lane;
-      if (v < nvec) {
-        if (sizeof(T) == 2) {
-          float f[8], h[8], g[8];
-          unpack8(x[u], f);
-          unpack8(z[u], h);
-          unpack8(y[u], g);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            a0 = fmaf(f[i], g[i], a0);
-            a1 = fmaf(h[i], g[i], a1);
-          }
-        } else {
-          const float* f = reinterpret_cast<const float*>(&x[u]);
-          const float* h = reinterpret_cast<const float*>(&z[u]);
-          const float* g = reinterpret_cast<const float*>(&y[u]);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            a0 = fmaf(f[i], g[i], a0);
-            a1 = fmaf(h[i], g[i], a1);
-          }
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
-    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-  }
-  s0 = a0;
-  s1 = a1;
 }
 
 // Step 3: rescore the rows of the selected groups exactly (fp32 CUDA-core sums, the same arithmetic as the other
