@@ -29,6 +29,12 @@
  *   - Calls on one store may be issued from several streams; the store orders them on the device
  *     (they share scratch memory).  add_fact(s) must not run concurrently with other calls from
  *     another host thread.
+ *   - CUDA graphs: memstore_retrieve, memstore_inject and memstore_retrieve_inject may be recorded on a stream
+ *     that is being captured, once a call of the same shape has run eagerly (scratch is sized, and grown with
+ *     cudaMalloc, on first use, which a capture does not allow).  A call depends on no earlier call (its kernels
+ *     leave the store's control state clean), so a graph may hold any number of calls and be replayed any number
+ *     of times, also between eager calls.  The store cannot see replays: the caller orders a replay against every other use of
+ *     the same store (same stream, or events), as the store does for eager calls.
  *   - There is no CPU fallback: every step runs in CUDA kernels of this library.
  */
 #ifndef MEMSTORE_H

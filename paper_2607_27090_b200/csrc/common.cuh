@@ -35,11 +35,15 @@ struct __align__(16) TileDesc {
 
 // Counters shared by the plan and copy kernels of one inject call.  A store keeps two of them and alternates:
 // the plan kernel of a call clears the pair the next call will use (calls on a store are ordered on the device).
+// Control block of the injection calls of one store.  The planning CTAs of a call (one per request) leave it ready
+// for the copy kernel and clean for the next call by themselves - the last one to finish publishes the tile count
+// and zeroes the rest - so a call depends on no earlier call, memset or host-side bookkeeping, and a call recorded
+// in a CUDA graph can be replayed at any time.
 struct InjectCtrl {
-  uint32_t n_tiles;
-  uint32_t work_next;
-  uint32_t done_ctas;
-  uint32_t pad;
+  uint32_t n_tiles;    // tiles of this call: written by the last planning CTA, read by the copy kernel
+  uint32_t work_next;  // work ticket of the staged copy kernel (zeroed by the last planning CTA)
+  uint32_t acc;        // tiles claimed so far by the planning CTAs of the running call (zero between calls)
+  uint32_t planned;    // planning CTAs that have finished (zero between calls)
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {

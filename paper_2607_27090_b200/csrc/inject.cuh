@@ -42,8 +42,7 @@ struct InjectParams {
   // scratch
   TileDesc* tiles;
   uint32_t tiles_capacity;
-  InjectCtrl* ctrl;       // counters of this call (zero when its plan kernel starts)
-  InjectCtrl* ctrl_next;  // counters of the next call, cleared by this call's plan kernel
+  InjectCtrl* ctrl;  // control block of the store (see InjectCtrl)
   int32_t layers_per_item;
 };
 
@@ -76,7 +75,6 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   const int lane = tid & 31, warp = tid >> 5;
   const int32_t start = p.start_pos[r];  // issued first: its latency hides behind the scan
   if (tid == 0) {
-    *p.ctrl_next = InjectCtrl{0u, 0u, 0u, 0u};  // the counters the NEXT inject call will use
     s_carry = 0;
     s_status = 0;
   }
@@ -139,10 +137,8 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   const int32_t first_tile_pos = (start / kTileTokens) * kTileTokens;
   const uint32_t n_tiles = m > 0 ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
   uint32_t tile_base = 0;
-  if (p.nreq == 1) {
-    if (tid == 0) p.ctrl->n_tiles = n_tiles;  // a single request owns the whole tile list: no ticket needed
-  } else {
-    if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->n_tiles, n_tiles) : 0u;
+  if (p.nreq > 1) {  // (a single request owns the whole tile list: no ticket needed)
+    if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->acc, n_tiles) : 0u;
     __syncthreads();
     tile_base = s_tile_base;
   }
@@ -195,6 +191,19 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   if (tid == 0) {
     if (p.out_n_tokens) p.out_n_tokens[r] = m;
     if (p.out_status) p.out_status[r] = s_status;
+    // the last planning CTA of the call hands the control block to the copy kernel and leaves it clean
+    if (p.nreq == 1) {
+      p.ctrl->n_tiles = n_tiles;
+      p.ctrl->work_next = 0;
+    } else {
+      __threadfence();  // this CTA's claim on `acc` is visible before its arrival is
+      if (atomicAdd(&p.ctrl->planned, 1u) == (uint32_t)p.nreq - 1u) {
+        __threadfence();
+        p.ctrl->n_tiles = atomicExch(&p.ctrl->acc, 0u);
+        p.ctrl->work_next = 0;
+        p.ctrl->planned = 0;
+      }
+    }
   }
 }
 

@@ -54,7 +54,7 @@ struct memstore {
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
   uint32_t tiles_capacity = 0;
-  InjectCtrl* ctrl = nullptr;
+  InjectCtrl* ctrl = nullptr;  // one control block, kept clean by the planning kernels themselves
   cudaEvent_t last_done = nullptr;
   cudaEvent_t prof_before = nullptr, prof_after = nullptr;  // caller-owned, optional
   // memstore_serve_host staging: one pinned host buffer and one device buffer, inputs first, outputs after
@@ -271,7 +271,19 @@ void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
 // stream than the previous one, an event recorded at the tail of the previous stream is waited for.
+// A stream that is being captured into a CUDA graph: the calls recorded on it run later, at every replay, and cannot
+// wait on other streams' work.
+bool stream_is_capturing(cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return cs != cudaStreamCaptureStatusNone;
+}
+
 ms_status order_after_last(memstore* s, cudaStream_t st) {
+  if (stream_is_capturing(st)) return MS_OK;  // ordering a replay against other uses of the store is the caller's job
   if (s->have_last && s->last_stream != st) {
     MS_CUDA(s, cudaEventRecord(s->last_done, s->last_stream));
     MS_CUDA(s, cudaStreamWaitEvent(st, s->last_done, 0));
@@ -279,6 +291,7 @@ ms_status order_after_last(memstore* s, cudaStream_t st) {
   return MS_OK;
 }
 ms_status mark_last(memstore* s, cudaStream_t st) {
+  if (stream_is_capturing(st)) return MS_OK;
   s->last_stream = st;
   s->have_last = true;
   return MS_OK;
@@ -371,7 +384,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
             cudaMalloc(&s->facts_d, (size_t)rows * sizeof(FactRec)) == cudaSuccess &&
             cudaMalloc(&s->user_count_d, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
             cudaMalloc(&s->inv_freq_d, (size_t)(config->head_dim / 2) * sizeof(float)) == cudaSuccess &&
-            cudaMalloc(&s->ctrl, 2 * sizeof(InjectCtrl)) == cudaSuccess;
+            cudaMalloc(&s->ctrl, sizeof(InjectCtrl)) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return bail(MS_ERR_OOM);
@@ -385,7 +398,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
     f[i] = config->inv_freq_override ? config->inv_freq_override[i] : (float)std::pow(config->rope_theta, -(double)(2 * i) / (double)R);
   ok = cudaMemcpy(s->inv_freq_d, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
        cudaMemset(s->user_count_d, 0, (size_t)config->n_users * sizeof(int32_t)) == cudaSuccess &&
-       cudaMemset(s->ctrl, 0, 2 * sizeof(InjectCtrl)) == cudaSuccess &&
+       cudaMemset(s->ctrl, 0, sizeof(InjectCtrl)) == cudaSuccess &&
        cudaEventCreateWithFlags(&s->last_done, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -902,8 +915,8 @@ namespace {
 // Validation, scratch sizing and parameter block shared by memstore_inject and memstore_retrieve_inject.
 ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache, int32_t* out_n_tokens,
-                         int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags, InjectParams* out,
-                         int64_t* out_tiles_needed) {
+                         int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags, cudaStream_t st,
+                         InjectParams* out, int64_t* out_tiles_needed) {
   const memstore_config& c = s->cfg;
   if (flags & ~(uint32_t)(MS_INJECT_REVERSE | MS_INJECT_PREFIX)) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
   const bool with_prefix = (flags & MS_INJECT_PREFIX) != 0;
@@ -981,8 +994,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.slot_stride = slot_stride;
   p.tiles = s->tiles;
   p.tiles_capacity = s->tiles_capacity;
-  p.ctrl = s->ctrl + (s->inject_calls & 1);
-  p.ctrl_next = s->ctrl + ((s->inject_calls + 1) & 1);
+  p.ctrl = s->ctrl;
 
   // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
@@ -1047,8 +1059,7 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
       e = fp8 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, true>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, false>, p);
   }
   if (e != cudaSuccess) {
-    // the plan has already counted tiles that no copy kernel will consume
-    cudaMemsetAsync(s->ctrl, 0, 2 * sizeof(InjectCtrl), st);
+    // (the planning kernel has left the control block clean: nothing to undo)
     return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
   }
   if (prof) MS_CUDA(s, cudaEventRecord(s->prof_after, st));
@@ -1071,7 +1082,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   InjectParams p;
   int64_t tiles_needed = 0;
   ms_status rc = prepare_inject(s, fact_ids, nreq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
-                                out_slot_mapping, slot_stride, flags, &p, &tiles_needed);
+                                out_slot_mapping, slot_stride, flags, st, &p, &tiles_needed);
   if (rc != MS_OK) return rc;
   rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
@@ -1108,7 +1119,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   InjectParams ip;
   int64_t tiles_needed = 0;
   ms_status rc = prepare_inject(s, out_ids, nq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
-                                out_slot_mapping, slot_stride, flags, &ip, &tiles_needed);
+                                out_slot_mapping, slot_stride, flags, st, &ip, &tiles_needed);
   if (rc != MS_OK) return rc;
   rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;

@@ -420,6 +420,55 @@ def test_retrieve_inject_and_serve_host_with_instruction_prefix():
     ms.close()
 
 
+@pytest.mark.parametrize("n_calls", [1, 2, 3])
+def test_calls_captured_in_a_cuda_graph_replay_correctly(n_calls):
+    """inject, retrieve_inject and retrieve captured into a CUDA graph (any number of calls, several requests each)
+    give the eager results on every replay, also when eager calls run between replays."""
+    hs = HostStore(90, 60, 2, 4, 64, 4, 30, 64, "float16")
+    ms = hs.to_memstore(1e4)
+    bs, nb, k, nq = 16, 256, 5, 3
+    q = to_dev(synth.queries(91, nq * n_calls, 64, "float16"))
+    starts = to_dev((np.arange(nq) * 3 + 2).astype(np.int32))
+    tables = [to_dev(synth.block_tables(92 + c, nb, 16, nq)) for c in range(n_calls)]
+    eager, graphed = [make_cache(hs, nb, bs) for _ in range(n_calls)], [make_cache(hs, nb, bs) for _ in range(n_calls)]
+    ids_e = [None] * n_calls
+    for rep in range(2):  # scratch is sized by the first round
+        for c in range(n_calls):
+            ids_e[c], n_e, st_e = ms.retrieve_inject(q[c * nq : (c + 1) * nq], k, starts, tables[c], eager[c], flags=M.INJECT_REVERSE)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    ids_g = [torch.empty((nq, k), dtype=torch.int32, device=DEV) for _ in range(n_calls)]
+    n_g = torch.zeros((n_calls, nq), dtype=torch.int32, device=DEV)
+    st_g = torch.zeros((n_calls, nq), dtype=torch.int32, device=DEV)
+    with torch.cuda.stream(side):
+        ms.retrieve_inject(q[:nq], k, starts, tables[0], graphed[0], out_ids=ids_g[0], out_n_tokens=n_g[0], out_status=st_g[0], stream=side)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for c in range(n_calls):
+                ms.retrieve_inject(q[c * nq : (c + 1) * nq], k, starts, tables[c], graphed[c], out_ids=ids_g[c], out_n_tokens=n_g[c],
+                                   out_status=st_g[c], flags=M.INJECT_REVERSE, stream=side)  # fmt: skip
+                ms.inject(ids_g[c], starts, tables[c], graphed[c], flags=M.INJECT_REVERSE, stream=side)  # the same again, as a plain inject
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for c in range(n_calls):
+            graphed[c].k.view(torch.int16).fill_(SENT - 0x10000)
+            graphed[c].v.view(torch.int16).fill_(SENT - 0x10000)
+        g.replay()
+        torch.cuda.synchronize()
+        assert int(st_g.abs().sum()) == 0
+        for c in range(n_calls):
+            assert torch.equal(ids_g[c], ids_e[c])
+            assert torch.equal(graphed[c].k.view(torch.int16), eager[c].k.view(torch.int16))
+            assert torch.equal(graphed[c].v.view(torch.int16), eager[c].v.view(torch.int16))
+        # an eager call between replays must neither disturb nor be disturbed
+        scratch = make_cache(hs, nb, bs)
+        ids_x, n_x, st_x = ms.retrieve_inject(q[:nq], k, starts, tables[0], scratch, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        assert torch.equal(scratch.k.view(torch.int16), eager[0].k.view(torch.int16)) and int(st_x.abs().sum()) == 0
+    ms.close()
+
+
 def test_host_tier_facts_are_injected_over_pcie_and_mix_with_hbm_facts():
     """Facts whose K/V live in the pinned host arena (the CPU-offloaded store) give the same cache contents as the
     same facts in HBM; one request may name facts of both tiers."""
