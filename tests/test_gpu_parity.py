@@ -469,6 +469,32 @@ def test_calls_captured_in_a_cuda_graph_replay_correctly(n_calls):
     ms.close()
 
 
+def test_head_sharded_stores_reproduce_the_unsharded_cache():
+    """Tensor-parallel serving: each shard holds a slice of the KV heads (and all embeddings), retrieves the same ids and
+    fills its own cache; together the shard caches are the unsharded cache, bit for bit.  (Shards run one after the
+    other on this one GPU; they never wait for one another.)"""
+    hs = HostStore(95, 40, 2, 8, 128, 6, 30, 128, "float16")
+    full = hs.to_memstore(5e5)
+    bs, nb, k = 16, 96, 6
+    q = to_dev(synth.queries(96, 2, 128, "float16"))
+    starts = to_dev(np.array([3, 40], np.int32))
+    tables = to_dev(synth.block_tables(97, nb, 20, 2))
+    c_full = make_cache(hs, nb, bs)
+    ids_f, n_f, st_f = full.retrieve_inject(q, k, starts, tables, c_full, flags=M.INJECT_REVERSE)
+    T = int(hs.lens.sum())
+    for h0, h1 in ((0, 3), (3, 8)):  # unequal shards
+        sh = MemStore(n_layers=hs.L, n_kv_heads=h1 - h0, head_dim=hs.D, emb_dim=128, rope_theta=5e5, max_facts_per_user=40, max_kv_tokens=T)
+        sh.add_facts(to_dev(hs.emb), hs.lens, to_dev(np.ascontiguousarray(hs.k[:, :, h0:h1])), to_dev(np.ascontiguousarray(hs.v[:, :, h0:h1])))
+        c_sh = PagedCache.allocate(hs.L, nb, bs, h1 - h0, hs.D, DEV, fill_bits=SENT)
+        ids_s, n_s, st_s = sh.retrieve_inject(q, k, starts, tables, c_sh, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        assert torch.equal(ids_s, ids_f) and torch.equal(n_s, n_f) and int(st_s.abs().sum()) == 0
+        assert torch.equal(c_sh.k.view(torch.int16), c_full.k[..., h0:h1, :].contiguous().view(torch.int16))
+        assert torch.equal(c_sh.v.view(torch.int16), c_full.v[..., h0:h1, :].contiguous().view(torch.int16))
+        sh.close()
+    full.close()
+
+
 def test_host_tier_facts_are_injected_over_pcie_and_mix_with_hbm_facts():
     """Facts whose K/V live in the pinned host arena (the CPU-offloaded store) give the same cache contents as the
     same facts in HBM; one request may name facts of both tiers."""
