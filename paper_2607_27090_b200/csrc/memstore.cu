@@ -6,11 +6,14 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
 #include <string>
 #include <vector>
+
+#include <nvtx3/nvToolsExt.h>  // header-only: ranges cost nothing unless a profiler is attached
 
 #include "common.cuh"
 #include "inject.cuh"
@@ -85,6 +88,15 @@ struct memstore {
 
 namespace {
 
+// MEMSTORE_LOG=1 in the environment makes every refused call print its reason to stderr (read once).
+bool log_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("MEMSTORE_LOG");
+    return e && e[0] && e[0] != '0';
+  }();
+  return on;
+}
+
 ms_status fail(memstore* s, ms_status code, const char* fmt, ...) {
   char buf[512];
   va_list ap;
@@ -92,8 +104,15 @@ ms_status fail(memstore* s, ms_status code, const char* fmt, ...) {
   vsnprintf(buf, sizeof buf, fmt, ap);
   va_end(ap);
   if (s) s->err = buf;
+  if (log_enabled()) fprintf(stderr, "[memstore] status %d: %s\n", (int)code, buf);
   return code;
 }
+
+// A named range around a public call, visible in profilers' timelines.
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
 
 #define MS_CUDA(s, call)                                                                         \
   do {                                                                                           \
@@ -535,11 +554,13 @@ static ms_status add_facts_tier(memstore_t* s, int32_t user, int64_t n, const vo
 
 ms_status memstore_add_facts(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre, const void* v,
                              const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+  Range range("memstore_add_facts");
   return add_facts_tier(s, user, n, embs, k_pre, v, n_tokens, out_first_id, stream, 1);
 }
 
 ms_status memstore_add_facts_host(memstore_t* s, int32_t user, int64_t n, const void* embs, const void* k_pre_host,
                                   const void* v_host, const int32_t* n_tokens, int32_t* out_first_id, ms_stream stream) {
+  Range range("memstore_add_facts_host");
   if (s && s->cfg.max_host_kv_tokens == 0) return fail(s, MS_ERR_INVALID_ARG, "store was created without a host K/V arena");
   return add_facts_tier(s, user, n, embs, k_pre_host, v_host, n_tokens, out_first_id, stream, 2);
 }
@@ -582,6 +603,7 @@ ms_status memstore_set_prefix(memstore_t* s, const void* k_pre, const void* v, i
 
 ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                             int32_t* out_ids, float* out_scores, ms_stream stream) {
+  Range range("memstore_retrieve");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -683,6 +705,7 @@ static ms_status graph_check_store(memstore* s, int32_t degree) {
 }
 
 ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) {
+  Range range("memstore_build_graph");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   ms_status rc = graph_check_store(s, degree);
@@ -740,6 +763,7 @@ ms_status memstore_get_graph(memstore_t* s, int32_t* out, int64_t out_capacity, 
 
 ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
                                 int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream) {
+  Range range("memstore_retrieve_ann");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -840,6 +864,7 @@ cudaError_t static_scratch_address(int device, unsigned char** out) {
 
 ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                                    int32_t* out_ids, float* out_scores, ms_stream stream) {
+  Range range("memstore_retrieve_static");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -1074,6 +1099,7 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
                           const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache,
                           int32_t* out_n_tokens, int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride,
                           uint32_t flags, ms_stream stream) {
+  Range range("memstore_inject");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   if (nreq == 0) return MS_OK;
@@ -1099,6 +1125,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
                                    const ms_paged_cache* cache, int32_t* out_ids, float* out_scores, int32_t* out_n_tokens,
                                    int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags,
                                    ms_stream stream) {
+  Range range("memstore_retrieve_inject");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -1158,6 +1185,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
 ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, int32_t k, int32_t start_pos,
                               const int32_t* block_table, int32_t max_blocks, const ms_paged_cache* cache, uint32_t flags,
                               int32_t* out_ids, int32_t* out_n_tokens, int32_t* out_status, ms_stream stream) {
+  Range range("memstore_serve_host");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;

@@ -598,6 +598,40 @@ def test_inject_data_errors_set_status_and_skip():
     assert untouched_mask_ok(cache, np.arange(3 * bs + 10, 4 * bs), SENT)
 
 
+@pytest.mark.parametrize("path", PATHS)
+def test_canaries_around_the_arena_and_the_cache_survive(path):
+    """The K/V arena and the cache planes are slices of larger buffers whose margins hold a canary pattern: store
+    construction, good requests and requests full of data errors leave every margin byte alone."""
+    lens = [5, 17, 33, 8, 1, 64]
+    hs = HostStore(98, len(lens), 2, 4, 64, 0, 0, 64, "float16", lens=lens)
+    T = int(sum(lens))
+    arena_bytes = 2 * hs.L * T * hs.H * hs.D * 2
+    margin = 4096
+    big = torch.full((arena_bytes + 2 * margin,), 0xA5, dtype=torch.uint8, device=DEV)
+    ms = MemStore(n_layers=hs.L, n_kv_heads=hs.H, head_dim=hs.D, emb_dim=64, rope_theta=1e4, max_facts_per_user=len(lens),
+                  max_kv_tokens=T, kv_arena=big[margin : margin + arena_bytes], max_position=200, flags=path)  # fmt: skip
+    ms.add_facts(to_dev(hs.emb), hs.lens, to_dev(hs.k), to_dev(hs.v))
+    bs, nb = 16, 12
+    planes = [torch.full((hs.L + 2, nb, bs, hs.H, hs.D), -121.0, dtype=torch.bfloat16, device=DEV) for _ in range(2)]
+    blk = bs * hs.H * hs.D
+    cache = PagedCache(planes[0][1 : hs.L + 1], planes[1][1 : hs.L + 1], nb * blk, blk, hs.H * hs.D, hs.D, nb, bs)
+    table = synth.block_tables(99, nb, nb, 1)[0]
+    out = run_inject_and_check(ms, hs, [1, 5, 0, 2], 7, table, cache, 1e4, flags=M.INJECT_REVERSE)
+    assert out["m"] == 17 + 64 + 5 + 33
+    bad_requests = [([0, 99, -3, 5], 150, table),  # unknown id, position overflow at 200
+                    ([1, 2, 3], 0, np.array([nb, -1, 5, nb + 7], np.int32)),  # bad block ids, short table
+                    ([5, 5, 5, 5], 190, table[:3])]  # fmt: skip
+    for ids, start, tb in bad_requests:
+        n, st = ms.inject(to_dev(np.array([ids], np.int32)), to_dev(np.array([start], np.int32)), to_dev(np.asarray(tb, np.int32)[None]), cache)
+        torch.cuda.synchronize()
+        assert int(st[0]) != 0
+    assert bool((big[:margin] == 0xA5).all()) and bool((big[margin + arena_bytes :] == 0xA5).all())
+    for p_ in planes:
+        canary = p_[[0, hs.L + 1]].view(torch.int16)
+        assert bool((canary == SENT - 0x10000).all())
+    ms.close()
+
+
 def test_host_errors_return_codes_and_enqueue_nothing():
     with pytest.raises(M.MemStoreError) as e:
         MemStore(n_layers=1, n_kv_heads=1, head_dim=48, emb_dim=64, max_facts_per_user=4, max_kv_tokens=4)
