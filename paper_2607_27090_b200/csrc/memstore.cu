@@ -216,8 +216,7 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_error, sizeof(int)));
   MS_CUDA(s, cudaMemset(s->tc_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
   MS_CUDA(s, cudaMemset(s->tc_error, 0, sizeof(int)));
-  MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)gemm_smem_bytes(kGemmMaxE)));
+  MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
   const size_t rs = (size_t)kTcMaxK2 * 8 * sizeof(uint32_t);
   MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
   s->tc_ready = true;
@@ -243,8 +242,8 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     CUtensorMap tmap_q;
     if (!make_tmap_rows_f16(&tmap_q, qptr, (uint64_t)nqb, (uint64_t)c.emb_dim, kGemmMaxQ))
       return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the query batch");
-    GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error};
-    score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, gemm_smem_bytes(c.emb_dim), st>>>(tmap_emb, tmap_q, gp);
+    GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes};
+    score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
     MS_CUDA(s, cudaGetLastError());
     select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel);
     MS_CUDA(s, cudaGetLastError());

@@ -24,7 +24,8 @@ namespace ms {
 
 constexpr int kGemmTileRows = 128;
 constexpr int kGemmKChunk = 64;       // fp16 elements per swizzle row (128 bytes)
-constexpr int kGemmStages = 4;
+constexpr int kGemmMaxStages = 8;   // the ring holds as many 16 KiB tiles as fit beside the queries, at most this many
+constexpr size_t kGemmSmemBytes = 232448;  // all the dynamic shared memory a CTA can have: always requested
 constexpr int kGemmMaxQ = 64;
 constexpr int kGemmGroupRows = 8;
 constexpr int kGemmGroupsPerTile = kGemmTileRows / kGemmGroupRows;  // 16
@@ -41,11 +42,17 @@ struct GemmParams {
   float* gmax;  // [nq][gmax_stride]: entry [q][g] = max over rows 8g..8g+7 of the score of query q
   int64_t gmax_stride;  // multiple of 16, >= 16 * ceil(n_rows / 128)
   int* error_flag;
+  uint32_t smem_bytes;  // dynamic shared memory of the launch
 };
 
-constexpr size_t gemm_smem_bytes(int emb_dim) {
-  return 1024 /*alignment slack*/ + (size_t)(emb_dim / kGemmKChunk) * kGemmQBytes + (size_t)kGemmStages * kGemmABytes +
-         4 * kGemmGroupsPerTile / 4 * kGemmMaxQ * sizeof(float) /*epilogue staging*/ + 256 /*barriers*/;
+// Shared memory after the 1 KiB alignment of the base: queries, ring, epilogue staging (4 warps x [4 groups][32
+// queries] floats), barriers.
+constexpr uint32_t kGemmStagingBytes = 4 * 4 * 32 * sizeof(float);
+constexpr uint32_t kGemmBarrierBytes = 256;
+__host__ __device__ constexpr int gemm_stages(uint32_t usable_bytes, int emb_dim) {
+  const int64_t left = (int64_t)usable_bytes - (int64_t)(emb_dim / kGemmKChunk) * kGemmQBytes - kGemmStagingBytes - kGemmBarrierBytes;
+  const int64_t n = left / kGemmABytes;
+  return n > kGemmMaxStages ? kGemmMaxStages : (int)n;
 }
 
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -107,21 +114,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int nkc = p.emb_dim / kGemmKChunk;
   uint8_t* q_smem = smem;                                   // nkc chunks of [64 queries][128 B]
-  uint8_t* a_smem = q_smem + (size_t)nkc * kGemmQBytes;     // kGemmStages tiles of [128 rows][128 B]
-  float* stage_f = reinterpret_cast<float*>(a_smem + (size_t)kGemmStages * kGemmABytes);  // [4 warps][4 groups][64 q]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stage_f + 4 * 4 * kGemmMaxQ);
+  // the ring takes what the alignment of the base and the queries leave: 6 tiles for 1024-d embeddings, 8 below
+  const int n_stages = gemm_stages(p.smem_bytes - (uint32_t)(smem - smem_raw), p.emb_dim);
+  uint8_t* a_smem = q_smem + (size_t)nkc * kGemmQBytes;     // n_stages tiles of [128 rows][128 B]
+  float* stage_f = reinterpret_cast<float*>(a_smem + (size_t)n_stages * kGemmABytes);  // [4 warps][4 groups][32 q]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(stage_f) + kGemmStagingBytes);
   uint64_t* q_full = bars;
   uint64_t* full = bars + 1;
-  uint64_t* empty = full + kGemmStages;
-  uint64_t* acc_full = empty + kGemmStages;
+  uint64_t* empty = full + kGemmMaxStages;
+  uint64_t* acc_full = empty + kGemmMaxStages;
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (n_stages < 2) {  // cannot happen with the launch this library makes; nothing has been set up yet
+    if (threadIdx.x == 0) atomicExch(p.error_flag, 1);
+    return;
+  }
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < kGemmStages; ++s) {
+    for (int s = 0; s < n_stages; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
@@ -159,7 +172,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           if (!ok) break;
           mbar_arrive_expect_tx(&full[s], kGemmABytes);
           tma_load_2d(a_smem + (size_t)s * kGemmABytes, &tmap_emb, kc * kGemmKChunk, tile * kGemmTileRows, &full[s]);
-          if (++s == kGemmStages) {
+          if (++s == n_stages) {
             s = 0;
             ph ^= 1u;
           }
@@ -189,7 +202,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           for (int k4 = 0; k4 < kGemmKChunk / 16; ++k4)  // 16 fp16 = 32 bytes per MMA along K: +2 in the address field
             umma_f16(d_tmem, a_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), kGemmIdesc, (kc | k4) != 0 ? 1u : 0u);
           umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
-          if (++s == kGemmStages) {
+          if (++s == n_stages) {
             s = 0;
             ph ^= 1u;
           }
@@ -201,7 +214,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
-    float* my_stage = stage_f + (size_t)(warp - 2) * 4 * kGemmMaxQ;
+    float* my_stage = stage_f + (size_t)(warp - 2) * 4 * 32;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int b = it & 1;
@@ -228,22 +241,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
         x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
         v[q] = x;
       }
-      if ((lane & 7) == 0) {
-        float4* dst = reinterpret_cast<float4*>(my_stage + (lane >> 3) * kGemmMaxQ);
-#pragma unroll
-        for (int q4 = 0; q4 < kGemmMaxQ / 4; ++q4) dst[q4] = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
-      }
-      __syncwarp();
+      // transpose through shared memory, 32 queries at a time: lane q then owns the four group maxima of query q
       const int64_t col = (int64_t)tile * kGemmGroupsPerTile + quarter * 4;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
+        if ((lane & 7) == 0) {
+          float4* dst = reinterpret_cast<float4*>(my_stage + (lane >> 3) * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            dst[q4] = make_float4(v[32 * h + 4 * q4], v[32 * h + 4 * q4 + 1], v[32 * h + 4 * q4 + 2], v[32 * h + 4 * q4 + 3]);
+        }
+        __syncwarp();
         const int q = lane + 32 * h;
         if (q < p.nq) {
-          const float4 g = make_float4(my_stage[q], my_stage[kGemmMaxQ + q], my_stage[2 * kGemmMaxQ + q], my_stage[3 * kGemmMaxQ + q]);
+          const float4 g = make_float4(my_stage[lane], my_stage[32 + lane], my_stage[64 + lane], my_stage[96 + lane]);
           *reinterpret_cast<float4*>(p.gmax + (int64_t)q * p.gmax_stride + col) = g;
         }
+        __syncwarp();
       }
-      __syncwarp();
     }
   }
 
