@@ -234,7 +234,7 @@ def test_inject_llama3_rescaled_table():
     assert np.array_equal(np.array(tab, np.float32), oracle.inv_freq_llama3(128, 5e5))
     hs = HostStore(72, 8, 2, 8, 128, 20, 60, 64, "float16")
     ms = hs.to_memstore(5e5, inv_freq_override=tab)
-    table = synth.block_tables(73, 2100, 2080, 1)[0]  # positions around 33,000: the slowed pairs turn visibly
+    table = synth.block_tables(73, 2100, 2080, 1)[0]  # positions near 33,000: the slowed pairs turn visibly
     cache = make_cache(hs, 2100, 16)
     out = run_inject_and_check(ms, hs, [1, 5, 2], 33000, table, cache, 5e5, inv_freq=np.array(tab, np.float32))
     assert out["exact_frac"] > 0.995
