@@ -360,6 +360,9 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
   if (u0 >= n_units) return;
 
   grid_dependency_wait();  // tile descriptors come from the plan kernel
+  // A kernel launched after this one as a programmatic dependent (the next request's retrieval) may be placed on the
+  // SMs once every CTA of this grid has got this far; it waits for this grid's completion before it does anything.
+  grid_launch_dependents();
 
   const uint32_t n_tiles = min(p.ctrl->n_tiles, p.tiles_capacity);
   const uint32_t n_items = n_tiles * (uint32_t)p.n_layers;

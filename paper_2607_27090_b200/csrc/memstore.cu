@@ -273,9 +273,23 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
   rows = (rows + kWarps - 1) / kWarps * kWarps;
   const int rows_per_cta = (int)rows;
   const dim3 grid((unsigned)((std::max<int64_t>(n_max, 1) + rows_per_cta - 1) / rows_per_cta), (unsigned)nq);
-  if constexpr (PLAN)
-    score_topk_plan_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host, *ip);
-  else
+  if constexpr (PLAN) {
+    // A programmatic dependent of whatever precedes it in the stream: when that is this library's copy kernel (which
+    // lets its dependents go as soon as all its CTAs have started) the CTAs of this kernel are placed on the SMs while
+    // the copy kernel drains, and the launch latency between two requests disappears.  The kernel waits for the
+    // preceding grid before it touches anything, so ordering is that of an ordinary launch.
+    cudaLaunchConfig_t lc{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.gridDim = grid;
+    lc.blockDim = dim3(THREADS);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaLaunchKernelEx(&lc, score_topk_plan_kernel<T, THREADS>, p, rows_per_cta, tickets, keys_cap, n_host, *ip);
+  } else
     score_topk_fused_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host);
 }
 template <typename T, bool PLAN>

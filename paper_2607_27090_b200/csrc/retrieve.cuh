@@ -856,6 +856,7 @@ template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
                                                                         uint32_t* tickets, int keys_capacity, int n_host,
                                                                         const __grid_constant__ InjectParams ip) {
+  grid_dependency_wait();    // launched as a programmatic dependent: nothing is touched before the preceding grid is done
   grid_launch_dependents();  // the copy kernel may be scheduled early; it waits for this grid before reading the plan
   score_topk_body<T, THREADS, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip);
 }
