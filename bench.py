@@ -460,7 +460,7 @@ def run_ours(args):
 # DRAM bytes (read + write) per launch of the copy kernel from the committed ncu capture summary of that kernel
 # (mean of the two captured launches; the capture starts from a flushed L2, so
 # about 50 MB of the written bytes are still in L2 when the kernel ends and are not in this figure).
-NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {("llama8b", 50): 468.2e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {("llama8b", 50): 467.5e6}
 
 
 if __name__ == "__main__":
