@@ -139,3 +139,17 @@ def test_graph_index_errors_and_empty_cases():
     ids, sc = empty.retrieve_ann(q, 3)
     assert ids.cpu().tolist() == [[-1] * 3] * 2 and sc.cpu().tolist() == [[0.0] * 3] * 2
     empty.close()
+
+
+def test_measurement_modes_of_the_package_run_at_small_sizes():
+    """The committed measurement entry points (graph index, cache variants, retrieval alone) keep working: run them
+    at toy sizes and check that their lines are sane."""
+    from paper_2607_27090_b200 import measure_configs as mc
+
+    lines = mc.measure_ann(20_000, 2, dim=128, degree=16, k=10, intrinsic_dim=8)
+    assert len(lines) == 3 and all(ln["recall_at_k"] > 0.8 and ln["ann_us_1_query"] > 0 for ln in lines)
+    lines = mc.measure_variants(2, n_facts=60, k=10)
+    assert [ln["config"].split()[1] for ln in lines] == ["bf16", "e4m3", "rotary_dim"]
+    assert lines[1]["bytes_moved"] == 0.75 * lines[0]["bytes_moved"] and all(ln["inject_us"] > 0 for ln in lines)
+    line = mc.measure_retrieve_only("tiny", 2)
+    assert line["kernel_timeouts"] == 0 and line["retrieve_us"] > 0
