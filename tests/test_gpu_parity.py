@@ -300,6 +300,56 @@ def test_inject_batch_of_requests_shares_one_cache():
     assert untouched_mask_ok(cache, np.concatenate(all_slots), SENT)
 
 
+def test_inject_at_the_largest_sizes():
+    """The longest id list (4096 entries, repeats allowed), one entry too many, and the last representable positions
+    (2^24 - 1 is the largest position that is exact in fp32; tokens beyond max_position are refused)."""
+    lens = [1, 2, 3, 1, 2]
+    hs = HostStore(33, len(lens), 2, 2, 64, 0, 0, 64, "float16", lens=lens)
+    ms = hs.to_memstore(1e4)
+    rng = np.random.default_rng(34)
+    ids = rng.integers(0, len(lens), 4096).astype(np.int32)
+    ids[rng.random(4096) < 0.1] = -1
+    m = int(sum(lens[i] for i in ids if i >= 0))
+    bs = 16
+    nb = (7 + m + bs - 1) // bs + 3
+    table = synth.block_tables(35, nb, nb - 2, 1)[0]
+    cache = make_cache(hs, nb, bs)
+    out = run_inject_and_check(ms, hs, ids, 7, table, cache, 1e4, flags=M.INJECT_REVERSE)
+    assert out["m"] == m and out["exact_frac"] > 0.99
+    with pytest.raises(RuntimeError):
+        ms.inject(to_dev(np.zeros((1, 4097), np.int32)), to_dev(np.array([0], np.int32)), to_dev(table[None]), cache)
+    # the end of the position range: 31 tokens placed from 2^24 - 20; the last 11 are refused
+    top = 1 << 24
+    start = top - 20
+    n_blocks_needed = (top + bs - 1) // bs
+    big_table = np.zeros(n_blocks_needed + 1, np.int32)
+    big_table[start // bs :] = np.arange(1, n_blocks_needed + 2 - start // bs, dtype=np.int32)  # real blocks only where needed
+    nb2 = int(big_table.max()) + 1
+    cache2 = make_cache(hs, nb2, bs)
+    req = [2, 1, 2, 2, 1, 2, 2, 0, 2, 2, 3, 1, 4]  # 20 tokens that fit, then 11 that do not
+    total = sum(lens[i] for i in req)
+    assert sum(lens[i] for i in req[:8]) == 20 and total == 31
+    n_tok, status = ms.inject(to_dev(np.array([req], np.int32)), to_dev(np.array([start], np.int32)), to_dev(big_table[None]), cache2)
+    torch.cuda.synchronize()
+    assert int(n_tok[0]) == total and int(status[0]) == M.REQ_POSITION_OVERFLOW
+    # the 20 tokens that fit are exactly the oracle's first 20 (the oracle is asked for a prefix of the request)
+    fit, acc = [], 0
+    for i in req:
+        if acc + lens[i] <= 20:
+            fit.append(i)
+            acc += lens[i]
+        else:
+            break
+    res = oracle.inject(fit, hs.offs, hs.lens, hs.k, hs.v, 1e4, start, big_table, bs, nb2)
+    from parity import check_k, gather_cache_rows
+
+    kb, vb = gather_cache_rows(cache2, res.slots)
+    assert np.array_equal(vb, res.v)
+    frac, worst = check_k(kb, res.k_ref)
+    assert worst <= 1.0 and frac > 0.98
+    ms.close()
+
+
 def test_inject_empty_and_degenerate_requests():
     hs = HostStore(15, 4, 1, 2, 64, 3, 9, 64, "float16")
     ms = hs.to_memstore(1e4)
