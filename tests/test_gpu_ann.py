@@ -61,7 +61,7 @@ def test_search_equals_the_oracle_bit_for_bit(dtype, dim, n, deg, kind):
     ms.close()
 
 
-@pytest.mark.parametrize("dtype,dim,n,deg", [("float32", 64, 2500, 16), ("float16", 128, 9000, 64), ("float16", 64, 30, 40)])
+@pytest.mark.parametrize("dtype,dim,n,deg", [("float32", 64, 2500, 16), ("float16", 128, 9000, 64), ("float16", 64, 30, 40), ("float32", 32, 8500, 12)])
 def test_graph_build_matches_the_exact_neighbour_graph(dtype, dim, n, deg):
     """Rows as queries through the exact retrieval kernels (CUDA-core path below 8193 rows, tensor-core filter
     above); compared with the oracle's graph under the near-tie rule of exact retrieval."""
