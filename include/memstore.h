@@ -84,12 +84,12 @@ typedef struct {
   int32_t n_layers;       /* L */
   int32_t n_kv_heads;     /* h */
   int32_t head_dim;       /* d: 16, 32, 64, 128 or 256 */
-  int32_t kv_dtype;       /* MS_DTYPE_BF16 only (the paper's cache is bf16) */
+  int32_t kv_dtype;       /* dtype of the STORED K/V: MS_DTYPE_BF16 only (Sec. 3.5 counts bfloat16 bytes) */
   int32_t emb_dim;        /* a multiple of 8 */
   int32_t emb_dtype;      /* MS_DTYPE_F32 or MS_DTYPE_F16 */
   int32_t rope_style;     /* MS_ROPE_HALF_SPLIT pairs (i, i+d/2); MS_ROPE_INTERLEAVED pairs (2i, 2i+1) */
-  double rope_theta;      /* frequency of pair i is theta^(-2i/d), rounded once to fp32 */
-  const float* inv_freq_override; /* host, d/2 floats, or NULL; replaces the formula above (copied) */
+  double rope_theta;      /* frequency of pair i is theta^(-2i/R), R = rotary_dim (d by default), rounded once to fp32 */
+  const float* inv_freq_override; /* host, R/2 floats, or NULL; replaces the formula above (copied) */
   int64_t max_position;   /* tokens at pos >= max_position are refused; 0 < max_position <= 2^24 */
   int32_t n_users;        /* number of private embedding segments (>= 1) */
   uint32_t flags;         /* MS_STORE_* bits, normally 0 */
