@@ -127,6 +127,49 @@ def measure_host_tier(iters: int, seed: int = 0, n_facts: int = 400, ks=(5, 10, 
     return lines
 
 
+def measure_permuted_chunks(iters: int, seed: int = 0, sizes=(1024, 2048, 4096, 8192, 16384, 32768), chunk: int = 64):
+    """The shape of the paper's chunk-order experiment (appendix "Position independence and rotation fidelity") on the
+    Llama-3.1-8B KV shape: fixed 64-token chunks injected
+    in a fresh random order every time, 1K to 32K tokens per request (512 chunks = 4.3 GB of stored K/V)."""
+    s = synth.CONFIGS["llama8b"]
+    dev = torch.device("cuda")
+    n_chunks = max(sizes) // chunk
+    T = n_chunks * chunk
+    store = M.MemStore(n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, emb_dim=s.emb_dim, rope_theta=s.rope_theta,
+                       max_facts_per_user=n_chunks, max_kv_tokens=T)  # fmt: skip
+    emb = synth.embeddings(seed, n_chunks, s.emb_dim, s.emb_dtype)
+    g = torch.Generator(device=dev).manual_seed(seed)
+    for a in range(0, n_chunks, 32):
+        b = min(n_chunks, a + 32)
+        kv = torch.randn((2, s.n_layers, (b - a) * chunk, s.n_kv_heads, s.head_dim), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        store.add_facts(torch.from_numpy(emb[a:b]).to(dev), [chunk] * (b - a), kv[0].contiguous(), kv[1].contiguous())
+    bs = s.block_size
+    nb = max(sizes) // bs + 8
+    cache = M.PagedCache.allocate(s.n_layers, nb, bs, s.n_kv_heads, s.head_dim, dev)
+    rng = np.random.default_rng(seed)
+    table = torch.from_numpy(synth.block_tables(seed, nb, nb - 1, 1)).to(dev)
+    start = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    lines = []
+    for m in sizes:
+        k = m // chunk
+        orders = torch.from_numpy(np.stack([rng.permutation(n_chunks)[:k] for _ in range(4)]).astype(np.int32)).to(dev)
+        for i in range(2):
+            store.inject(orders[i : i + 1], start, table, cache, stream=stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(iters):
+            store.inject(orders[i % 4 : i % 4 + 1], start, table, cache, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        lines.append({"config": "llama8b permuted 64-token chunks", "tokens": m, "chunks": k, "inject_us": us,
+                      "inject_gbs": 2.0 * m * s.token_bytes / (us * 1e-6) / 1e9})  # fmt: skip
+    store.close()
+    return lines
+
+
 def measure_variants(iters: int, seed: int = 0, n_facts: int = 400, k: int = 50):
     """Injection of k facts on the Llama-3.1-8B KV shape (a shrunken store: the traffic of a request does not depend on
     the store size) in the parameterisation variants: bf16 cache (the headline path), 8-bit e4m3 cache (half the
@@ -309,8 +352,12 @@ if __name__ == "__main__":
     ap.add_argument("--host-tier", action="store_true", help="Llama shape with all K/V in the pinned host arena: inject over PCIe")
     ap.add_argument("--variants", action="store_true", help="Llama shape: bf16 cache, e4m3 cache, partial rotary (inject only)")
     ap.add_argument("--ann", type=int, default=0, metavar="ROWS", help="graph index on ROWS structured embedding rows")
+    ap.add_argument("--permuted-chunks", action="store_true", help="Llama shape: 64-token chunks in random order, 1K-32K tokens")
     a = ap.parse_args()
-    if a.ann:
+    if a.permuted_chunks:
+        for ln in measure_permuted_chunks(a.iters, a.seed):
+            print(json.dumps(ln))
+    elif a.ann:
         for ln in measure_ann(a.ann, a.iters, a.seed):
             print(json.dumps(ln))
     elif a.variants:

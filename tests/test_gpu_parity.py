@@ -350,6 +350,39 @@ def test_inject_at_the_largest_sizes():
     ms.close()
 
 
+def test_inject_permuted_chunks_up_to_32k_positions():
+    """The shape of the paper's chunk-order experiment (appendix "Position independence and rotation fidelity":
+    fixed 64-token chunks, permuted order, 1K to 32K injected tokens): every order gives the oracle's cache, and a chunk's values land bit-identical
+    wherever the permutation puts it."""
+    n_chunks, clen = 512, 64
+    hs = HostStore(36, n_chunks, 1, 2, 64, 0, 0, 64, "float16", lens=[clen] * n_chunks)
+    ms = hs.to_memstore(5e5)
+    bs = 16
+    rng = np.random.default_rng(37)
+    for n_use in (16, 512):  # 1K and 32K tokens
+        m = n_use * clen
+        nb = m // bs + 4
+        table = synth.block_tables(38, nb, nb - 1, 1)[0]
+        orders = [np.arange(n_use, dtype=np.int32), rng.permutation(n_use).astype(np.int32)]
+        slots_of = []
+        for order in orders:
+            cache = make_cache(hs, nb, bs)
+            out = run_inject_and_check(ms, hs, order, 0, table, cache, 5e5)
+            assert out["m"] == m and out["exact_frac"] > 0.995
+            from parity import gather_cache_rows
+
+            res = oracle.slots(order, hs.lens, 0, table, bs, nb)[1]
+            _, vb = gather_cache_rows(cache, res)
+            slots_of.append((order, vb))
+        # values of chunk c: the same bits in both runs, at the positions each order gives it
+        (o0, v0), (o1, v1) = slots_of
+        pos1 = {int(c): i for i, c in enumerate(o1)}
+        for c in (0, 3, n_use - 1):
+            i0, i1 = int(np.where(o0 == c)[0][0]), pos1[c]
+            assert np.array_equal(v0[:, i0 * clen : (i0 + 1) * clen], v1[:, i1 * clen : (i1 + 1) * clen])
+    ms.close()
+
+
 def test_inject_empty_and_degenerate_requests():
     hs = HostStore(15, 4, 1, 2, 64, 3, 9, 64, "float16")
     ms = hs.to_memstore(1e4)
