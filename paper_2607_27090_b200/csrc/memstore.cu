@@ -739,9 +739,15 @@ ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) 
     const int nb = (int)std::min<int64_t>(kBatch, n - row0);
     // the rows themselves are the queries: exact top-(degree + 1) of each, the row itself among them
     rc = memstore_retrieve(s, (const char*)s->emb + (size_t)row0 * row_bytes, nullptr, nb, k1, s->graph_topk, nullptr, stream);
-    if (rc != MS_OK) return rc;
-    graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, degree, row0, nb);
-    MS_CUDA(s, cudaGetLastError());
+    if (rc == MS_OK) {
+      graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, degree, row0, nb);
+      if (cudaGetLastError() != cudaSuccess) rc = fail(s, MS_ERR_CUDA, "graph_rows_kernel launch failed");
+    }
+    if (rc != MS_OK) {  // a half-built graph must not be searched
+      s->graph_rows = 0;
+      s->graph_deg = 0;
+      return rc;
+    }
     s->kernels_launched++;
   }
   return MS_OK;
