@@ -64,8 +64,26 @@ struct PlanShared {
   uint32_t tile_base;
 };
 
-// Plans request r with the THREADS threads of the calling CTA (all of them must call).
+// What planning request r needs and what does not depend on the request's ids, fetched ahead of time (all THREADS
+// threads call; plan_request<THREADS, true> completes it): the block-table row goes to shared memory with asynchronous
+// copies, and the head of the fact table is pulled towards the SM, so that a caller with other work to do first (the
+// retrieval kernel selects the ids in the meantime) finds both at hand.
 template <int THREADS>
+__device__ __forceinline__ void plan_prefetch(const InjectParams& p, const int r, PlanShared& ps) {
+  const int tid = threadIdx.x;
+  const int32_t* table_row = p.block_tables + (int64_t)r * p.max_blocks;
+  const int n_cached = min(p.max_blocks, kPlanTableCache);
+  for (int i = tid; i < n_cached; i += THREADS)
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(&ps.table[i])), "l"(table_row + i)
+                 : "memory");
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  const int n_lines = min((p.n_facts * (int)sizeof(FactRec) + 127) / 128, THREADS);
+  if (tid < n_lines) asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(p.facts) + (size_t)tid * 128));
+}
+
+// Plans request r with the THREADS threads of the calling CTA (all of them must call).  PREFETCHED: plan_prefetch has
+// been called for this request by the same threads.
+template <int THREADS, bool PREFETCHED = false>
 __device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps) {
   int32_t* const s_scan = ps.scan;
   int32_t& s_carry = ps.carry;
@@ -82,7 +100,11 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   // otherwise be a chain of dependent global loads
   const int32_t* table_row = p.block_tables + (int64_t)r * p.max_blocks;
   const int n_cached = min(p.max_blocks, kPlanTableCache);
-  for (int i = tid; i < n_cached; i += THREADS) ps.table[i] = table_row[i];
+  if constexpr (PREFETCHED) {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+    for (int i = tid; i < n_cached; i += THREADS) ps.table[i] = table_row[i];
+  }
   __syncthreads();
 
   // lengths of the entries in placement order (the instruction prefix, if any, then the facts), exclusive scan in

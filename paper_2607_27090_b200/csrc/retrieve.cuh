@@ -818,6 +818,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   __syncthreads();
   if (!s_last) return;
   __threadfence();
+  if (PLAN) plan_prefetch<THREADS>(*ip, q, ps);  // in flight while the ids are being selected
   const float* sc = p.scores + (int64_t)q * p.score_stride;
   uint32_t lo = 0xffffffffu, hi = 0u;
   for (int i = threadIdx.x; i < n; i += THREADS) {
@@ -837,7 +838,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     // selection no longer needs, so that the copy kernel can follow without a separate planning launch
     __syncthreads();
     int32_t* s_begin = reinterpret_cast<int32_t*>(sm.cand);
-    plan_request<THREADS>(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
+    plan_request<THREADS, true>(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
   }
 }
 
