@@ -84,7 +84,8 @@ __device__ __forceinline__ void plan_prefetch(const InjectParams& p, const int r
 // Plans request r with the THREADS threads of the calling CTA (all of them must call).  PREFETCHED: plan_prefetch has
 // been called for this request by the same threads.
 template <int THREADS, bool PREFETCHED = false>
-__device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps) {
+__device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps,
+                                             const int32_t* ids_smem = nullptr) {
   int32_t* const s_scan = ps.scan;
   int32_t& s_carry = ps.carry;
   int32_t& s_status = ps.status;
@@ -109,7 +110,9 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
 
   // lengths of the entries in placement order (the instruction prefix, if any, then the facts), exclusive scan in
   // chunks of THREADS
-  const int32_t* ids = p.fact_ids + (int64_t)r * p.k;
+  // ids_smem: the request's id list in shared memory, when its producer ran in this CTA (the same values as in
+  // p.fact_ids; it saves a round trip to global memory)
+  const int32_t* ids = ids_smem ? ids_smem : p.fact_ids + (int64_t)r * p.k;
   const int has_prefix = p.prefix_len > 0;
   const int n_entries = p.k + has_prefix;
   for (int base = 0; base < n_entries; base += THREADS) {

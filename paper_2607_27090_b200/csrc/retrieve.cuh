@@ -249,6 +249,7 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long* cand, int 
 struct IdMap {
   const int32_t* idx_to_row;  // or nullptr: the index is the row
   const int32_t* row_ids;     // or nullptr: the row is the id
+  int32_t* mirror = nullptr;  // optional copy of the result ids (by rank) in shared memory, for a consumer in the same CTA
   __device__ __forceinline__ int32_t operator()(uint32_t idx) const {
     int32_t row = idx_to_row ? idx_to_row[idx] : (int32_t)idx;
     return (row >= 0 && row_ids) ? row_ids[row] : row;
@@ -269,6 +270,7 @@ __device__ __forceinline__ void write_topk(const unsigned long long* cand, int t
       s = key_score((uint32_t)(c >> 32));
     }
     out_ids[r] = id;
+    if (ids.mirror) ids.mirror[r] = id;
     if (out_scores) out_scores[r] = s;
   }
 }
@@ -400,7 +402,9 @@ __device__ __forceinline__ void rank_candidates(unsigned long long* cand, uint32
     rank += __shfl_xor_sync(0xffffffffu, rank, 1);
     rank += __shfl_xor_sync(0xffffffffu, rank, 2);
     if (ci < n_cand && part == 0 && rank < (uint32_t)k) {
-      out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+      const int32_t id = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+      out_ids[rank] = id;
+      if (ids.mirror) ids.mirror[rank] = id;
       if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
     }
     return;
@@ -411,7 +415,9 @@ __device__ __forceinline__ void rank_candidates(unsigned long long* cand, uint32
       uint32_t rank = 0;
       for (uint32_t jj = 0; jj < n_cand; ++jj) rank += cand[jj] > mine;
       if (rank < (uint32_t)k) {
-        out_ids[rank] = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+        const int32_t id = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+        out_ids[rank] = id;
+        if (ids.mirror) ids.mirror[rank] = id;
         if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
       }
     }
@@ -797,6 +803,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ PlanShared ps;
+  __shared__ int32_t s_ids[PLAN ? kTopkMaxK : 1];  // the selected ids by rank, for the planning that follows in this CTA
   __shared__ int s_last;
   const int q = blockIdx.y;
   int user = 0, n = n_host;
@@ -830,7 +837,8 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   __syncthreads();
   // with a single user segment facts are numbered in row order: the row is the fact id
   topk_block<THREADS, false>(sm, sc, s_keys, n, p.k,
-                            IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
+                            IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity,
+                                  PLAN ? s_ids : nullptr},
                             p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
                             hi);
   if (PLAN) {
@@ -838,7 +846,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     // selection no longer needs, so that the copy kernel can follow without a separate planning launch
     __syncthreads();
     int32_t* s_begin = reinterpret_cast<int32_t*>(sm.cand);
-    plan_request<THREADS, true>(*ip, q, s_begin, s_begin + kTopkMaxK, ps);
+    plan_request<THREADS, true>(*ip, q, s_begin, s_begin + kTopkMaxK, ps, s_ids);
   }
 }
 
