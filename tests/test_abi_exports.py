@@ -70,3 +70,22 @@ def test_llama3_frequency_table_of_the_library_equals_the_oracles():
 
     with pytest.raises(memstore.MemStoreError):
         memstore.rope_table_llama3(127, 5e5)
+
+
+def test_header_is_plain_c_and_cpp_and_matches_the_struct_sizes(tmp_path):
+    """include/memstore.h compiles as C99 and as C++11 with warnings as errors, and the C compiler's struct sizes are
+    the ones the ctypes mirrors assume."""
+    import subprocess
+
+    src = tmp_path / "hdr.c"
+    src.write_text(
+        '#include "memstore.h"\n#include <stdio.h>\n'
+        "int main(void) { printf(\"%zu %zu %zu %zu\\n\", sizeof(memstore_config), sizeof(ms_paged_cache), sizeof(memstore_stats_t),"
+        " sizeof(ms_ann_params)); return 0; }\n"
+    )
+    inc = str(ROOT / "include")
+    exe = tmp_path / "hdr"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", inc, str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert [int(x) for x in out] == [112, 72, 80, 16]
+    subprocess.run(["g++", "-std=c++11", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
