@@ -73,7 +73,9 @@ enum { MS_DTYPE_F32 = 0, MS_DTYPE_F16 = 1, MS_DTYPE_BF16 = 2 };
 enum { MS_ROPE_HALF_SPLIT = 0, MS_ROPE_INTERLEAVED = 1 };
 enum {
   MS_INJECT_REVERSE = 1u, /* place ids[k-1] first, so that ids[0] ends next to the query */
-  MS_INJECT_PREFIX = 2u   /* place the store's instruction prefix (memstore_set_prefix) before the facts */
+  MS_INJECT_PREFIX = 2u,  /* place the store's instruction prefix (memstore_set_prefix) before the facts */
+  MS_RETRIEVE_ANN = 4u    /* memstore_retrieve_inject / memstore_serve_host only: retrieve through the graph index
+                             (memstore_retrieve_ann with its default parameters) instead of the exact scan */
 };
 /* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
  * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */
@@ -310,6 +312,8 @@ ms_status memstore_set_prefix(memstore_t* store, const void* k_pre, const void* 
  * the ids handed over on the device and, for segments of at most 8192 rows, the requests planned inside the
  * retrieval kernel, so that the whole path is two launches (Sec. 3.3: search, compose and scatter per request).
  * Arguments as in the two calls; out_ids [nq][k] is both the retrieval output and the injection input.
+ * With MS_RETRIEVE_ANN in flags the ids come from the graph search (the paper's own pipeline: index search, compose,
+ * scatter), followed by the planning and copy kernels; query_users must then be NULL and k <= 256.
  */
 ms_status memstore_retrieve_inject(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                                    const int32_t* start_pos, const int32_t* block_tables, int32_t max_blocks,

@@ -1152,6 +1152,13 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   if (nq == 0) return MS_OK;
   if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
   if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
+  if (flags & MS_RETRIEVE_ANN) {
+    if (query_users) return fail(s, MS_ERR_INVALID_ARG, "MS_RETRIEVE_ANN serves single-segment stores: query_users must be NULL");
+    ms_status rc = memstore_retrieve_ann(s, queries, nq, k, nullptr, out_ids, out_scores, nullptr, stream);
+    if (rc != MS_OK) return rc;
+    return memstore_inject(s, out_ids, nq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
+                           out_slot_mapping, slot_stride, flags & ~(uint32_t)MS_RETRIEVE_ANN, stream);
+  }
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
   if (n_max > kFusedMaxRows || nq > s->scores_nq || ((flags & MS_INJECT_PREFIX) && k + 1 > kTopkMaxK)) {
     // large segments (or a first call that still has to size its scratch): the two calls one after the other

@@ -153,3 +153,37 @@ def test_measurement_modes_of_the_package_run_at_small_sizes():
     assert lines[1]["bytes_moved"] == 0.75 * lines[0]["bytes_moved"] and all(ln["inject_us"] > 0 for ln in lines)
     line = mc.measure_retrieve_only("tiny", 2)
     assert line["kernel_timeouts"] == 0 and line["retrieve_us"] > 0
+
+
+def test_retrieve_inject_through_the_graph_index():
+    """MS_RETRIEVE_ANN: index search, then planning and the copy kernel, in one call and from host buffers; the cache
+    is the one that retrieve_ann followed by inject gives, and memstore_inject itself refuses the flag."""
+    from parity import HostStore
+    from paper_2607_27090_b200 import memstore as M
+    from paper_2607_27090_b200.memstore import PagedCache
+
+    hs = HostStore(87, 300, 2, 4, 64, 4, 20, 64, "float16")
+    hs.emb = synth.embeddings_low_rank(87, 300, 64, "float16", intrinsic_dim=6)
+    ms = hs.to_memstore(1e4)
+    ms.build_graph(16)
+    bs, nb, k = 16, 128, 8
+    q = synth.queries_near_rows(88, hs.emb, 3)
+    starts = to_dev(np.array([0, 5, 17], np.int32))
+    tables = to_dev(synth.block_tables(89, nb, 16, 3))
+    ca = PagedCache.allocate(hs.L, nb, bs, hs.H, hs.D, DEV, fill_bits=synth.SENTINEL_BF16)
+    cb = PagedCache.allocate(hs.L, nb, bs, hs.H, hs.D, DEV, fill_bits=synth.SENTINEL_BF16)
+    ids_a, _ = ms.retrieve_ann(to_dev(q), k)
+    n_a, st_a = ms.inject(ids_a, starts, tables, ca, flags=M.INJECT_REVERSE)
+    ids_b, n_b, st_b = ms.retrieve_inject(to_dev(q), k, starts, tables, cb, flags=M.INJECT_REVERSE | M.RETRIEVE_ANN)
+    torch.cuda.synchronize()
+    assert torch.equal(ids_a, ids_b) and torch.equal(n_a, n_b) and int(st_b.abs().sum()) == 0
+    assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+    want = oracle.ann_search(hs.emb, ms.get_graph().cpu().numpy(), q, k, parents=8)
+    assert np.array_equal(ids_b.cpu().numpy(), want.ids)
+    out = np.full(k + 2, -5, np.int32)
+    cc = PagedCache.allocate(hs.L, nb, bs, hs.H, hs.D, DEV, fill_bits=synth.SENTINEL_BF16)
+    ms.serve_host(q[1], k, 5, tables[1].cpu().numpy(), cc, out, flags=M.INJECT_REVERSE | M.RETRIEVE_ANN)
+    assert out[:k].tolist() == ids_b[1].cpu().tolist() and out[k] == int(n_b[1]) and out[k + 1] == 0
+    with pytest.raises(MemStoreError):
+        ms.inject(ids_a, starts, tables, ca, flags=M.RETRIEVE_ANN)
+    ms.close()
