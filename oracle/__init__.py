@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
         L.oracle_scores_f32.argtypes = [p, i32, i64, i32, p, p]
         L.oracle_knn_graph.restype = i32
         L.oracle_knn_graph.argtypes = [p, i32, i64, i32, i32, p, i32]
+        L.oracle_graph_append.restype = i32
+        L.oracle_graph_append.argtypes = [p, i32, i64, i64, i32, p, i32, p, i32]
         L.oracle_ann_search.restype = i32
         L.oracle_ann_search.argtypes = [p, i32, i64, i32, p, i32, p, i32, i32, i32, i32, i32, p, p, p, p]
         L.oracle_inject_ex.restype = i32
@@ -197,6 +199,19 @@ def knn_graph(emb: np.ndarray, deg: int, n_threads: int = 0) -> np.ndarray:
     emb = np.ascontiguousarray(emb)
     out = np.empty((emb.shape[0], deg), dtype=np.int32)
     rc = lib().oracle_knn_graph(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], deg, _ptr(out), n_threads)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def graph_append(emb: np.ndarray, old_graph: np.ndarray, n_threads: int = 0) -> np.ndarray:
+    """The graph after rows ``old_graph.shape[0]`` .. ``emb.shape[0] - 1`` have been appended: exact lists for the new
+    rows; an old row is offered the new rows that list it and keeps the best ``deg`` of old list + offers."""
+    emb = np.ascontiguousarray(emb)
+    old_graph = np.ascontiguousarray(old_graph, dtype=np.int32)
+    n_old, deg = old_graph.shape
+    out = np.empty((emb.shape[0], deg), dtype=np.int32)
+    rc = lib().oracle_graph_append(_ptr(emb), _emb_dtype(emb), n_old, emb.shape[0], emb.shape[1], _ptr(old_graph), deg, _ptr(out), n_threads)
     if rc:
         raise OracleError(rc)
     return out

@@ -345,6 +345,80 @@ int oracle_knn_graph(const void* emb, int emb_dtype, int64_t n, int emb_dim, int
   return rc_all;
 }
 
+/*
+ * Growing the graph when rows n_old .. n-1 have been appended to the store (the paper lists online insertion as future
+ * work; the rule fixed here is the usual one for incremental neighbour graphs):
+ *   - a new row gets its exact list over all n rows, like any row of a fresh graph;
+ *   - an old row nb is offered every new row that lists nb among its own neighbours; its list becomes the best deg
+ *     of (old list + offers) by inner product with nb, best first, ties to the lower row.  Old rows that nobody
+ *     offers anything keep their list.  (A fresh build could differ: it would also give nb a new row that does
+ *     not list nb back.)
+ * Scores in double, full sorts.  old_graph [n_old][deg], out_graph [n][deg].
+ */
+int oracle_graph_append(const void* emb, int emb_dtype, int64_t n_old, int64_t n, int emb_dim, const int32_t* old_graph,
+                        int deg, int32_t* out_graph, int n_threads) {
+  if (!emb || !out_graph || n_old < 0 || n < n_old || deg <= 0 || emb_dim <= 0 || (n_old > 0 && !old_graph)) return ORACLE_ERR_ARG;
+  size_t esz = emb_dtype == ORACLE_F32 ? 4 : 2;
+  int rc_all = ORACLE_OK;
+  set_threads(n_threads);
+  /* new rows: exact lists over everything */
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t r = n_old; r < n; ++r) {
+    scored_t* all = (scored_t*)malloc(sizeof(scored_t) * (size_t)n);
+    if (!all) {
+      rc_all = ORACLE_ERR_NOMEM;
+      continue;
+    }
+    const char* q = (const char*)emb + (size_t)r * emb_dim * esz;
+    int64_t m = 0;
+    for (int64_t f = 0; f < n; ++f) {
+      if (f == r) continue;
+      double sc = 0.0;
+      for (int d = 0; d < emb_dim; ++d) sc += emb_at(q, emb_dtype, d) * emb_at(emb, emb_dtype, f * emb_dim + d);
+      all[m].s = sc;
+      all[m].id = (int32_t)f;
+      ++m;
+    }
+    qsort(all, (size_t)m, sizeof(scored_t), cmp_scored);
+    for (int j = 0; j < deg; ++j) out_graph[r * deg + j] = j < m ? all[j].id : -1;
+    free(all);
+  }
+  if (rc_all != ORACLE_OK) return rc_all;
+  /* old rows: old list plus the new rows that list them */
+  int64_t n_add = n - n_old;
+  scored_t* cand = (scored_t*)malloc(sizeof(scored_t) * (size_t)(deg + n_add + 1));
+  if (!cand) return ORACLE_ERR_NOMEM;
+  for (int64_t nb = 0; nb < n_old; ++nb) {
+    const char* q = (const char*)emb + (size_t)nb * emb_dim * esz;
+    int64_t m = 0, offers = 0;
+    for (int j = 0; j < deg; ++j) {
+      int32_t f = old_graph[nb * deg + j];
+      if (f < 0 || f >= n_old) continue;
+      cand[m++].id = f;
+    }
+    for (int64_t r = n_old; r < n; ++r)
+      for (int j = 0; j < deg; ++j)
+        if (out_graph[r * deg + j] == nb) {
+          cand[m++].id = (int32_t)r;
+          ++offers;
+          break;
+        }
+    if (offers == 0) {
+      for (int j = 0; j < deg; ++j) out_graph[nb * deg + j] = old_graph[nb * deg + j];
+      continue;
+    }
+    for (int64_t i = 0; i < m; ++i) {
+      double sc = 0.0;
+      for (int d = 0; d < emb_dim; ++d) sc += emb_at(q, emb_dtype, d) * emb_at(emb, emb_dtype, (int64_t)cand[i].id * emb_dim + d);
+      cand[i].s = sc;
+    }
+    qsort(cand, (size_t)m, sizeof(scored_t), cmp_scored);
+    for (int j = 0; j < deg; ++j) out_graph[nb * deg + j] = j < m ? cand[j].id : -1;
+  }
+  free(cand);
+  return ORACLE_OK;
+}
+
 typedef struct {
   float s;
   int32_t row;

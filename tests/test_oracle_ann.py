@@ -138,3 +138,40 @@ def test_recall_grows_with_the_beam_on_structured_rows(oracle_mod):
 
     r_small, r_large = recall(10), recall(96)
     assert r_large >= r_small and r_large > 0.9
+
+
+def test_graph_append_rule(oracle_mod):
+    n_old, n, dim, deg = 300, 360, 32, 8
+    emb = synth.embeddings_low_rank(6, n, dim, "float32", intrinsic_dim=5)
+    old = oracle_mod.knn_graph(emb[:n_old], deg)
+    new = oracle_mod.graph_append(emb, old)
+    full = oracle_mod.knn_graph(emb, deg)
+    # new rows: the exact lists of a fresh graph
+    assert np.array_equal(new[n_old:], full[n_old:])
+    s = emb.astype(np.float64) @ emb.astype(np.float64).T
+    touched = 0
+    for nb in range(n_old):
+        offers = [r for r in range(n_old, n) if nb in new[r]]
+        if not offers:
+            assert np.array_equal(new[nb], old[nb])  # nobody offered anything
+            continue
+        touched += 1
+        pool = np.array(list(old[nb]) + offers)
+        order = pool[np.lexsort((pool, -s[nb][pool]))][:deg]  # brute force with numpy: best deg of old list + offers
+        assert np.allclose(s[nb][new[nb]], s[nb][order], rtol=0, atol=1e-12)
+        assert np.all(s[nb][new[nb]] >= s[nb][old[nb]] - 1e-12)  # a list only improves, entry by entry
+        assert len(set(new[nb].tolist())) == deg and nb not in new[nb]
+    assert touched > 20
+    # appending in two steps is appending at once when the first step's rows are fixed... for the OLD rows' lists:
+    half = oracle_mod.graph_append(emb[: n_old + 30], old)
+    both = oracle_mod.graph_append(emb, half)
+    # rows of the first step were given lists over 330 rows only, so compare the old rows offered by second-step rows
+    for nb in range(n_old):
+        offers_all = {r for r in range(n_old, n) if nb in new[r]}
+        offers_two = {r for r in range(n_old, n_old + 30) if nb in half[r]} | {r for r in range(n_old + 30, n) if nb in both[r]}
+        if offers_all == offers_two:
+            assert np.array_equal(both[nb], new[nb])
+    # nothing appended: nothing changes
+    assert np.array_equal(oracle_mod.graph_append(emb[:n_old], old), old)
+    # a store that starts empty: append equals build
+    assert np.array_equal(oracle_mod.graph_append(emb[:50], np.zeros((0, deg), np.int32)), oracle_mod.knn_graph(emb[:50], deg))
