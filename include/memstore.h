@@ -228,6 +228,15 @@ typedef struct {
 /* Build the graph of all facts present (degree <= 255); replaces an earlier graph.  Synchronises the device once
  * (allocation), then enqueues the retrieval calls on `stream`. */
 ms_status memstore_build_graph(memstore_t* store, int32_t degree, ms_stream stream);
+/*
+ * Grow the graph for the facts added since it was built, set or last grown (the paper names online insertion as future
+ * work; the rule is this library's): a new row gets its exact neighbour list over all rows; an old row is offered
+ * every new row that lists it and keeps the best `degree` of its old list plus those offers, best first.  One exact
+ * retrieval call and two small kernels per 64 new rows (fewer when degree > 64), instead of a rebuild.  Old rows that
+ * no new row lists keep their lists, so the result can differ from a fresh build.  Synchronises the device once
+ * (allocation of the larger graph).  No-op when nothing was added; MS_ERR_INVALID_ARG when there is no graph.
+ */
+ms_status memstore_graph_append(memstore_t* store, ms_stream stream);
 /* Install a caller-made graph: device int32 [n_rows][degree], entries are rows of the segment (others are ignored
  * by the search), n_rows <= number of facts.  Copied on `stream`. */
 ms_status memstore_set_graph(memstore_t* store, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream);

@@ -306,4 +306,80 @@ __global__ void graph_rows_kernel(const int32_t* topk, int k1, int32_t* graph, i
   for (int j = min(written, deg) + lane; j < deg; j += 32) dst[j] = -1;
 }
 
+// ---- growing the graph for appended rows ------------------------------------------------------------------------
+// Rule (the oracle states it the same way): a new row gets its exact list over all rows, like any row of a fresh
+// graph (the build code above does that); an OLD row nb is offered every new row that lists nb among its own
+// neighbours, and keeps the best `deg` of (old list + offers) by inner product with nb, best first, ties to the
+// lower row.  Rows are processed in batches; after each batch two kernels apply the batch's offers.
+constexpr int kAppendMaxPairs = 4096;   // (old row, new row) offers of one batch: batch rows * degree
+constexpr int kAppendMaxOffers = 64;    // new rows of one batch (each offers itself to an old row at most once)
+constexpr int kAppendWarps = 8;
+
+// One CTA: the batch's offers as keys (old row << 32 | new row), sorted ascending, so that the offers to one old row
+// form a run; *n_pairs = their number.  Neighbours that are new rows themselves get no offer (their lists are exact).
+__global__ void __launch_bounds__(1024) append_pairs_kernel(const int32_t* graph, int deg, int64_t row0, int nb_rows, int64_t n_old,
+                                                            unsigned long long* pairs, int* n_pairs) {
+  __shared__ unsigned long long keys[kAppendMaxPairs];
+  __shared__ int s_count;
+  const int tid = threadIdx.x;
+  if (tid == 0) s_count = 0;
+  __syncthreads();
+  const int total = nb_rows * deg;
+  int mine = 0;
+  for (int t = tid; t < kAppendMaxPairs; t += 1024) {
+    unsigned long long key = 0ull;  // sorts last in a descending sort of inverted keys
+    if (t < total) {
+      const int64_t r = row0 + t / deg;
+      const int32_t nbr = graph[r * deg + t % deg];
+      if (nbr >= 0 && nbr < n_old) {
+        key = ~(((unsigned long long)(uint32_t)nbr << 32) | (unsigned long long)(uint32_t)r);
+        ++mine;
+      }
+    }
+    keys[t] = key;
+  }
+  if (mine) atomicAdd(&s_count, mine);
+  __syncthreads();
+  bitonic_sort_desc<1024>(keys, kAppendMaxPairs);  // descending in the inverted keys = ascending in (old row, new row)
+  for (int t = tid; t < kAppendMaxPairs; t += 1024) pairs[t] = ~keys[t];
+  if (tid == 0) *n_pairs = s_count;
+}
+
+// One warp per run of offers to the same old row nb: scores of the old list and of the offers against row nb (the
+// fp32 sums of the retrieval kernels), ranking by counting, best `deg` written back.
+template <typename T>
+__global__ void __launch_bounds__(kAppendWarps * 32) append_update_kernel(const RetrieveParams p, int32_t* graph, int deg, int64_t n_rows,
+                                                                          const unsigned long long* pairs, const int* n_pairs) {
+  __shared__ unsigned long long s_key[kAppendWarps][256 + kAppendMaxOffers];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int i = blockIdx.x * kAppendWarps + warp;
+  const int n = *n_pairs;
+  if (i >= n) return;
+  const unsigned long long first = pairs[i];
+  const int32_t nb = (int32_t)(first >> 32);
+  if (i > 0 && (int32_t)(pairs[i - 1] >> 32) == nb) return;  // not the start of a run
+  int run = 1;
+  while (i + run < n && (int32_t)(pairs[i + run] >> 32) == nb && run < kAppendMaxOffers) ++run;
+  const T* seg = reinterpret_cast<const T*>(p.emb);
+  unsigned long long* key = s_key[warp];
+  int32_t* list = graph + (int64_t)nb * deg;
+  // candidates: the valid old entries, then the offers
+  int n_cand = 0;
+  for (int j = 0; j < deg + run; ++j) {
+    const int32_t c = j < deg ? list[j] : (int32_t)(pairs[i + j - deg] & 0xffffffffull);
+    if (j < deg && (c < 0 || c >= n_rows)) continue;  // (the list may hold new rows accepted from earlier batches)
+    const float sc = score_one_row<T>(p, nb, seg, c) + 0.0f;  // "query" = row nb (p.queries is the embedding matrix)
+    if (lane == 0) key[n_cand] = ((unsigned long long)order_key(sc) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)c);
+    ++n_cand;
+  }
+  __syncwarp();
+  for (int c = lane; c < n_cand; c += 32) {
+    const unsigned long long mine = key[c];
+    int rank = 0;
+    for (int j = 0; j < n_cand; ++j) rank += key[j] > mine;
+    if (rank < deg) list[rank] = (int32_t)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+  }
+  for (int j = n_cand + lane; j < deg; j += 32) list[j] = -1;
+}
+
 }  // namespace ms

@@ -75,6 +75,7 @@ struct memstore {
   int64_t graph_rows = 0;
   int32_t graph_deg = 0;
   int32_t* graph_topk = nullptr;  // build scratch: [64][deg + 1] ids
+  unsigned long long* append_pairs = nullptr;  // graph_append scratch: sorted (old row, new row) offers, then their count
   int64_t prefix_off = 0;   // instruction prefix (memstore_set_prefix): first arena token and length (0 = none)
   int32_t prefix_len = 0;
   int64_t prefix_tokens_total = 0;  // arena tokens taken by this and earlier prefixes (not facts)
@@ -474,6 +475,7 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tiles);
     cudaFree(s->graph);
     cudaFree(s->graph_topk);
+    cudaFree(s->append_pairs);
     cudaFree(s->dev_stage);
     if (s->host_stage) cudaFreeHost(s->host_stage);
     if (s->last_done) cudaEventDestroy(s->last_done);
@@ -751,6 +753,65 @@ ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) 
     s->kernels_launched++;
   }
   return MS_OK;
+}
+
+ms_status memstore_graph_append(memstore_t* s, ms_stream stream) {
+  Range range("memstore_graph_append");
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  if (!s->graph_deg) return fail(s, MS_ERR_INVALID_ARG, "no graph to grow: call memstore_build_graph or memstore_set_graph first");
+  const memstore_config& c = s->cfg;
+  const int deg = s->graph_deg;
+  const int64_t n_old = s->graph_rows, n = s->user_count[0];
+  if (n == n_old) return MS_OK;
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  // a larger graph array: the old rows are carried over, the new rows are filled below
+  MS_CUDA(s, cudaDeviceSynchronize());
+  int32_t* grown = nullptr;
+  MS_CUDA(s, cudaMalloc(&grown, (size_t)n * deg * sizeof(int32_t)));
+  if (n_old) cudaMemcpy(grown, s->graph, (size_t)n_old * deg * sizeof(int32_t), cudaMemcpyDeviceToDevice);
+  cudaFree(s->graph);
+  s->graph = grown;
+  s->graph_rows = n;  // searches after this call see all rows (a failure below clears the graph)
+  const int k1 = deg + 1;
+  const int batch = std::max(1, std::min(kAppendMaxOffers, kAppendMaxPairs / deg));
+  cudaFree(s->graph_topk);
+  s->graph_topk = nullptr;
+  cudaFree(s->append_pairs);
+  s->append_pairs = nullptr;
+  ms_status rc = MS_OK;
+  if (cudaMalloc(&s->graph_topk, (size_t)kAppendMaxOffers * k1 * sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&s->append_pairs, (size_t)kAppendMaxPairs * sizeof(unsigned long long) + 16) != cudaSuccess)
+    rc = fail(s, MS_ERR_OOM, "scratch for growing the graph");
+  const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
+  RetrieveParams p{};
+  p.emb = s->emb;
+  p.queries = s->emb;  // the rows are scored against one another
+  p.emb_dim = c.emb_dim;
+  int* n_pairs = s->append_pairs ? reinterpret_cast<int*>(s->append_pairs + kAppendMaxPairs) : nullptr;
+  for (int64_t row0 = n_old; rc == MS_OK && row0 < n; row0 += batch) {
+    const int nb = (int)std::min<int64_t>(batch, n - row0);
+    rc = memstore_retrieve(s, (const char*)s->emb + (size_t)row0 * row_bytes, nullptr, nb, k1, s->graph_topk, nullptr, stream);
+    if (rc != MS_OK) break;
+    graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, deg, row0, nb);
+    if (n_old > 0) {
+      append_pairs_kernel<<<1, 1024, 0, st>>>(s->graph, deg, row0, nb, n_old, s->append_pairs, n_pairs);
+      const int grid = kAppendMaxPairs / kAppendWarps;
+      if (c.emb_dtype == MS_DTYPE_F16)
+        append_update_kernel<__half><<<grid, kAppendWarps * 32, 0, st>>>(p, s->graph, deg, n, s->append_pairs, n_pairs);
+      else
+        append_update_kernel<float><<<grid, kAppendWarps * 32, 0, st>>>(p, s->graph, deg, n, s->append_pairs, n_pairs);
+      s->kernels_launched += 2;
+    }
+    if (cudaGetLastError() != cudaSuccess) rc = fail(s, MS_ERR_CUDA, "graph append kernels failed to launch");
+    s->kernels_launched++;
+  }
+  if (rc != MS_OK) {  // a half-grown graph must not be searched
+    s->graph_rows = 0;
+    s->graph_deg = 0;
+  }
+  return rc;
 }
 
 ms_status memstore_set_graph(memstore_t* s, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream) {

@@ -226,8 +226,9 @@ def measure_ann(n: int, iters: int, seed: int = 0, dim: int = 1024, degree: int 
     emb = synth.embeddings_low_rank(seed, n, dim, "float16", intrinsic_dim=intrinsic_dim)
     q = synth.queries_near_rows(seed, emb, 64)
     store = M.MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=dim, rope_theta=1e4, max_facts_per_user=n, max_kv_tokens=0)
-    for a in range(0, n, 65536):
-        b = min(n, a + 65536)
+    n_late = min(640, n // 10)  # these rows arrive after the build and are linked by graph_append
+    for a in range(0, n - n_late, 65536):
+        b = min(n - n_late, a + 65536)
         store.add_facts(torch.from_numpy(emb[a:b]).to(dev), [0] * (b - a))
     q_dev = torch.from_numpy(q).to(dev)
     stream = torch.cuda.current_stream()
@@ -236,6 +237,12 @@ def measure_ann(n: int, iters: int, seed: int = 0, dim: int = 1024, degree: int 
     store.build_graph(degree, stream=stream)
     torch.cuda.synchronize()
     build_s = time.perf_counter() - t0
+    store.add_facts(torch.from_numpy(emb[n - n_late :]).to(dev), [0] * n_late)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    store.graph_append(stream=stream)
+    torch.cuda.synchronize()
+    append_s = time.perf_counter() - t0
 
     def timed(fn):
         for _ in range(3):
@@ -264,6 +271,7 @@ def measure_ann(n: int, iters: int, seed: int = 0, dim: int = 1024, degree: int 
         a, b = ids_a.cpu().numpy(), ids_e.cpu().numpy()
         recall = float(np.mean([len(set(a[i]) & set(b[i])) / k for i in range(64)]))
         lines.append({"config": f"graph index, {n} rows x {dim} fp16, degree {degree}", "k": k, "beam": L, "build_s": build_s,
+                      "append_rows": n_late, "append_ms": append_s * 1e3,
                       "recall_at_k": recall, "ann_us_1_query": ann_1, "ann_us_64_queries": ann_64,
                       "exact_us_1_query": exact_1, "exact_us_64_queries": exact_64,
                       "mean_steps": float(cnt[:, 0].float().mean()), "mean_rows_scored": float(cnt[:, 1].float().mean())})  # fmt: skip

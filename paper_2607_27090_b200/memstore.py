@@ -70,7 +70,7 @@ EXPORTS = (
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
-    "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann",
+    "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
 )  # fmt: skip
 
 _lib = None
@@ -105,6 +105,8 @@ def load_library() -> C.CDLL:
     L.memstore_retrieve.restype = i32
     L.memstore_build_graph.restype = i32
     L.memstore_build_graph.argtypes = [vp, i32, vp]
+    L.memstore_graph_append.restype = i32
+    L.memstore_graph_append.argtypes = [vp, vp]
     L.memstore_set_graph.restype = i32
     L.memstore_set_graph.argtypes = [vp, vp, i64, i32, vp]
     L.memstore_get_graph.restype = i32
@@ -345,6 +347,10 @@ class MemStore:
     def build_graph(self, degree=64, stream=None) -> None:
         """Exact neighbour graph of all facts present (single-segment stores), built on the device."""
         self._check(self._lib.memstore_build_graph(self._h, degree, _stream_ptr(stream)))
+
+    def graph_append(self, stream=None) -> None:
+        """Grow the graph for the facts added since it was built, set or last grown."""
+        self._check(self._lib.memstore_graph_append(self._h, _stream_ptr(stream)))
 
     def set_graph(self, graph: torch.Tensor, stream=None) -> None:
         """Install a graph: int32 device tensor [n_rows, degree] of row numbers."""

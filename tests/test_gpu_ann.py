@@ -187,3 +187,47 @@ def test_retrieve_inject_through_the_graph_index():
     with pytest.raises(MemStoreError):
         ms.inject(ids_a, starts, tables, ca, flags=M.RETRIEVE_ANN)
     ms.close()
+
+
+@pytest.mark.parametrize("dtype,dim,n_old,n_add,deg", [("float32", 32, 900, 150, 8), ("float16", 128, 9000, 200, 64), ("float16", 64, 0, 90, 16),
+                                                       ("float16", 64, 500, 70, 100)])  # fmt: skip
+def test_graph_append_matches_the_oracle_rule(dtype, dim, n_old, n_add, deg):
+    """Rows added after the build are linked by memstore_graph_append: their own lists are exact, and an old row keeps
+    the best of its list plus the new rows that list it.  Compared row by row with the oracle's graph (its own build,
+    its own append) under the near-tie rule; then the grown graph is searched."""
+    n = n_old + n_add
+    emb = synth.embeddings_low_rank(93, n, dim, dtype, intrinsic_dim=min(6, dim))
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=dim, emb_dtype=torch.float32 if dtype == "float32" else torch.float16,
+                  rope_theta=1e4, max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+    if n_old:
+        ms.add_facts(to_dev(emb[:n_old]), np.zeros(n_old, np.int32))
+    ms.build_graph(deg)
+    ms.graph_append()  # nothing added yet: a no-op
+    assert ms.get_graph().shape == (n_old, deg)
+    for a in range(n_old, n, 64):  # facts arrive in several calls
+        b = min(n, a + 64)
+        ms.add_facts(to_dev(emb[a:b]), np.zeros(b - a, np.int32))
+    ms.graph_append()
+    g = ms.get_graph().cpu().numpy()
+    assert g.shape == (n, deg)
+    want = oracle.graph_append(emb, oracle.knn_graph(emb[:n_old], deg) if n_old else np.zeros((0, deg), np.int32))
+    rows = list(range(0, n, max(1, n // 60))) + list(range(n_old, n, 7)) + [n - 1]
+    changed = [r for r in range(n_old) if not np.array_equal(want[r], oracle.knn_graph(emb[:n_old], deg)[r])] if n_old and n_old <= 1000 else []
+    rows += changed[:40]
+    same = 0
+    for r in rows:
+        got = g[r][g[r] >= 0]
+        exp = want[r][want[r] >= 0]
+        assert len(got) == len(exp) == min(deg, n - 1) and r not in got and len(set(got.tolist())) == len(got)
+        s_got = oracle.scores(emb[got], emb[r]).astype(np.float32)
+        s_exp = oracle.scores(emb[exp], emb[r]).astype(np.float32)
+        assert np.all(np.abs(s_got - s_exp) < 1e-5), r
+        same += int(np.array_equal(got, exp))
+    assert same >= 0.8 * len(rows)
+    if n_old and n_old <= 1000:
+        assert len(changed) > 10  # the append did change old rows' lists
+    # the grown graph is searched like any other; new rows are found
+    q = emb[n - 3 : n].copy()
+    ids, _ = ms.retrieve_ann(to_dev(q), 5, beam=64)
+    assert ids[:, 0].cpu().tolist() == [n - 3, n - 2, n - 1]
+    ms.close()
