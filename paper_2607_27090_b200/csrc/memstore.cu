@@ -1294,7 +1294,7 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
     s->stage_bytes = 0;
     const size_t want = (in_bytes + out_bytes) * 2;
     MS_CUDA(s, cudaMalloc(&s->dev_stage, want));
-    MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocDefault));
+    MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocMapped));
     s->stage_bytes = want;
   }
   unsigned char* h = s->host_stage;
@@ -1306,12 +1306,15 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
   memcpy(h + q_bytes + 16, block_table, (size_t)max_blocks * 4);
   MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, st));
   int32_t* d_hdr = reinterpret_cast<int32_t*>(d + q_bytes);
-  int32_t* d_ids = reinterpret_cast<int32_t*>(d + in_bytes);
+  // The results (k ids, token count, status: a few hundred bytes) are written by the kernels straight into the pinned
+  // host buffer through its device address, so that no copy back has to be queued behind the copy kernel.
+  void* res_dev = nullptr;
+  MS_CUDA(s, cudaHostGetDevicePointer(&res_dev, h + in_bytes, 0));
+  int32_t* d_ids = static_cast<int32_t*>(res_dev);
   ms_status rc = memstore_retrieve_inject(s, d, c.n_users > 1 ? d_hdr + 1 : nullptr, 1, k, d_hdr,
                                           reinterpret_cast<const int32_t*>(d + q_bytes + 16), max_blocks, cache, d_ids, nullptr,
                                           d_ids + k, d_ids + k + 1, nullptr, 0, flags, stream);
   if (rc != MS_OK) return rc;
-  MS_CUDA(s, cudaMemcpyAsync(h + in_bytes, d_ids, ((size_t)k + 2) * 4, cudaMemcpyDeviceToHost, st));
   MS_CUDA(s, cudaStreamSynchronize(st));
   const int32_t* res = reinterpret_cast<const int32_t*>(h + in_bytes);
   memcpy(out_ids, res, (size_t)k * 4);
