@@ -269,7 +269,8 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
                                const InjectParams* ip, size_t smem, cudaStream_t st) {
   // enough CTAs to fill the GPU, at least one row per warp
   constexpr int64_t kWarps = THREADS / 32;
-  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * 8 / nq);
+  // (a 1024-thread CTA fills an SM: more CTAs than SMs would only queue behind the first wave)
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * (THREADS >= 1024 ? 1 : 8) / nq);
   int64_t rows = std::max<int64_t>(kWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
   rows = (rows + kWarps - 1) / kWarps * kWarps;
   const int rows_per_cta = (int)rows;
