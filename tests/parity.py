@@ -216,7 +216,7 @@ def with_prefix(hs: HostStore, placed, prefix):
 
 def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, cache: PagedCache, theta, style=0,
                          inv_freq=None, flags=0, sentinel=synth.SENTINEL_BF16, check_untouched=True, prefix=None,
-                         rotary_dim=0):  # fmt: skip
+                         rotary_dim=0, expect_status=0):  # fmt: skip
     """One request: inject on the GPU, run the oracle on the same ids, compare. Returns stats dict.
     ``prefix``: (k, v) of the instruction prefix the store holds, when ``flags`` asks for it."""
     dev = cache.k.device
@@ -236,7 +236,7 @@ def run_inject_and_check(ms: MemStore, hs: HostStore, ids_np, start, table_np, c
     slot_map = torch.full((1, max(res.m, 1) + 3), -7, dtype=torch.int64, device=dev)
     n_tok, status = ms.inject(ids, sp, bt, cache, out_slot_mapping=slot_map, flags=flags)
     torch.cuda.synchronize()
-    assert int(status[0]) == 0, f"status {int(status[0])}"
+    assert int(status[0]) == expect_status, f"status {int(status[0])}"
     assert int(n_tok[0]) == res.m
     sm = slot_map[0].cpu().numpy()
     assert np.array_equal(sm[: res.m], res.slots) and np.all(sm[res.m :] == -7)

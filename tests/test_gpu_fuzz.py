@@ -1,0 +1,94 @@
+"""Seeded random differential tests: many small random stores, requests and cache shapes through the C ABI against
+the oracle.  Every case is reproducible from its number."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_27090_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from parity import HostStore, check_ids, run_inject_and_check, to_dev
+    from paper_2607_27090_b200 import memstore as M
+    from paper_2607_27090_b200.memstore import PagedCache
+
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("block", range(10))
+def test_random_injections(block):
+    rng = np.random.default_rng(1000 + block)
+    for case in range(6):
+        H = int(rng.choice([1, 2, 3, 4, 8]))
+        D = int(rng.choice([16, 32, 64, 128, 256]))
+        L = int(rng.integers(1, 4))
+        n_facts = int(rng.integers(1, 24))
+        lens = rng.integers(0, 40, n_facts).astype(np.int32)
+        lens[rng.integers(0, n_facts)] = int(rng.integers(1, 70))  # at least one fact with tokens
+        style = int(rng.integers(0, 2))
+        R = int(rng.choice([0, 16, D // 2 if D >= 32 else 0, D]))
+        theta = float(rng.choice([1e4, 5e5, 1e6]))
+        hs = HostStore(2000 + 10 * block + case, n_facts, L, H, D, 0, 0, 64, "float16", lens=lens)
+        extra = int(rng.integers(0, 20))
+        ms = hs.to_memstore(theta, rope_style=style, rotary_dim=R, extra_kv_tokens=extra, flags=int(rng.integers(0, 2)))
+        prefix = None
+        if extra:
+            prefix = synth.kv_fact(7, 999, L, extra, H, D)
+            ms.set_prefix(to_dev(prefix[0]), to_dev(prefix[1]))
+        k = int(rng.integers(1, 30))
+        ids = rng.integers(-1, n_facts, k).astype(np.int32)
+        flags = int(rng.integers(0, 2)) | (2 if extra and rng.random() < 0.7 else 0)
+        m = int(lens[ids[ids >= 0]].sum()) + (extra if flags & 2 else 0)
+        bs = int(rng.choice([4, 8, 16, 32]))
+        start = int(rng.choice([0, 1, 7, 100, 4095, 65536 + 3]))
+        n_table = (start + m + bs - 1) // bs + 1
+        used = np.arange(start // bs, n_table)
+        nb = len(used) + 3
+        table = np.zeros(n_table, np.int32)
+        table[used] = synth.block_tables(3000 + block, nb, len(used), 1)[0]
+        fp8 = bool(rng.random() < 0.3)
+        layout = str(rng.choice(["NHD", "HND"]))
+        cache = PagedCache.allocate(L, nb, bs, H, D, DEV, layout=layout, stacked=bool(rng.random() < 0.5), fp8=fp8,
+                                    fill_bits=0x5A if fp8 else synth.SENTINEL_BF16, k_scale=float(rng.choice([1.0, 0.05, 2.5])),
+                                    v_scale=float(rng.choice([1.0, 0.02])))  # fmt: skip
+        # a fact without tokens is embedding-only: asking for its K/V adds nothing and raises the status bit
+        expect = M.REQ_NOT_RESIDENT if np.any(lens[ids[ids >= 0]] == 0) else 0
+        out = run_inject_and_check(ms, hs, ids, start, table, cache, theta, style=style, flags=flags, prefix=prefix, rotary_dim=R,
+                                   sentinel=0x5A if fp8 else synth.SENTINEL_BF16, expect_status=expect)  # fmt: skip
+        assert out["m"] == m, (block, case)
+        ms.close()
+
+
+@pytest.mark.parametrize("block", range(6))
+def test_random_retrievals(block):
+    rng = np.random.default_rng(4000 + block)
+    for case in range(5):
+        dtype = str(rng.choice(["float16", "float32"]))
+        E = int(rng.choice([8, 64, 136, 256, 1024]))
+        n_users = int(rng.choice([1, 1, 3]))
+        per_user = int(rng.integers(1, 1500))
+        hs = HostStore(5000 + 10 * block + case, per_user, 1, 1, 16, 0, 0, E, dtype, n_users=n_users, lens=[0] * (per_user * n_users))
+        if per_user > 4:  # duplicates: ties go to the lower id
+            hs.emb[per_user - 1] = hs.emb[1]
+            hs.emb[per_user // 2] = hs.emb[1]
+        ms = hs.to_memstore(1e4, batch=512)
+        nq = int(rng.choice([1, 2, 9, 40]))
+        q = synth.queries(6000 + block * 10 + case, nq, E, dtype)
+        if per_user > 4:
+            q[0] = hs.emb[1]
+        users = (rng.integers(0, n_users, nq)).astype(np.int32) if n_users > 1 else None
+        if users is not None:
+            users[0] = 0
+        k = int(rng.choice([1, 3, 20, 100, per_user, per_user + 5]))
+        k = max(1, min(k, 2048))
+        ids, sc = ms.retrieve(to_dev(q), k, query_users=to_dev(users) if users is not None else None)
+        torch.cuda.synchronize()
+        ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+        for i in range(nq):
+            u = int(users[i]) if users is not None else 0
+            rows = np.arange(u * per_user, (u + 1) * per_user)
+            check_ids(ids[i], sc[i], hs.emb[rows], q[i], k, row_ids=rows.astype(np.int32) if n_users > 1 else None)
+        if per_user > 4 and k >= 3:
+            assert ids[0, :3].tolist() == sorted({1, per_user // 2, per_user - 1})[:3] or len({1, per_user // 2, per_user - 1}) < 3
+        ms.close()
