@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 if torch.cuda.is_available():
     from parity import HostStore, check_ids, run_inject_and_check, to_dev
     from paper_2607_27090_b200 import memstore as M
-    from paper_2607_27090_b200.memstore import PagedCache
+    from paper_2607_27090_b200.memstore import MemStore, PagedCache
 
 DEV = "cuda"
 
@@ -91,4 +91,41 @@ def test_random_retrievals(block):
             check_ids(ids[i], sc[i], hs.emb[rows], q[i], k, row_ids=rows.astype(np.int32) if n_users > 1 else None)
         if per_user > 4 and k >= 3:
             assert ids[0, :3].tolist() == sorted({1, per_user // 2, per_user - 1})[:3] or len({1, per_user // 2, per_user - 1}) < 3
+        ms.close()
+
+
+@pytest.mark.parametrize("block", range(6))
+def test_random_graph_searches(block):
+    """Random segments, graphs (holes, repeats, rows outside the segment) and search parameters: ids, scores, step and
+    row counts equal the oracle's, bit for bit."""
+    import oracle
+
+    rng = np.random.default_rng(7000 + block)
+    for case in range(4):
+        dtype = str(rng.choice(["float16", "float32"]))
+        dim = int(rng.choice([8, 64, 136, 512]))
+        n = int(rng.integers(1, 2500))
+        deg = int(rng.choice([1, 2, 5, 16, 32, 64]))
+        emb = synth.embeddings_low_rank(7100 + 10 * block + case, n, dim, dtype, intrinsic_dim=min(6, dim))
+        graph = synth.random_graph(7200 + 10 * block + case, n, deg, holes=float(rng.choice([0.0, 0.05, 0.5])))
+        if n > 3:
+            graph[rng.integers(0, n), 0] = n + int(rng.integers(0, 5))  # outside the segment: ignored
+        ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=dim, emb_dtype=torch.float32 if dtype == "float32" else torch.float16,
+                      rope_theta=1e4, max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+        ms.add_facts(to_dev(emb), np.zeros(n, np.int32))
+        ms.set_graph(to_dev(graph))
+        nq = int(rng.choice([1, 3, 20]))
+        q = synth.queries_near_rows(7300 + 10 * block + case, emb, nq)
+        k = int(rng.choice([1, 7, 64, 256]))
+        beam = int(rng.choice([1, 16, 64, 200]))
+        parents = int(rng.integers(1, min(32, 512 // deg) + 1))
+        n_entry = int(rng.choice([1, 5, 64, 300]))
+        max_iters = int(rng.choice([1, 4, 20]))
+        want = oracle.ann_search(emb, graph, q, k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters)
+        ids, sc, cnt = ms.retrieve_ann(to_dev(q), k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters, want_counters=True)
+        torch.cuda.synchronize()
+        tag = (block, case, n, deg, k, beam, parents, n_entry, max_iters)
+        assert np.array_equal(ids.cpu().numpy(), want.ids), tag
+        assert np.array_equal(sc.cpu().numpy().view(np.uint32), want.scores.view(np.uint32)), tag
+        assert np.array_equal(cnt[:, 0].cpu().numpy(), want.iters) and np.array_equal(cnt[:, 1].cpu().numpy(), want.scored), tag
         ms.close()
