@@ -129,3 +129,33 @@ def test_random_graph_searches(block):
         assert np.array_equal(sc.cpu().numpy().view(np.uint32), want.scores.view(np.uint32)), tag
         assert np.array_equal(cnt[:, 0].cpu().numpy(), want.iters) and np.array_equal(cnt[:, 1].cpu().numpy(), want.scored), tag
         ms.close()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_retrievals_on_long_segments(block):
+    """Segments above 8192 rows: the tensor-core filter path (fp16, dimension a multiple of 64, k <= 256, 8+ queries) and
+    the unfused CUDA-core path (everything else), by the near-tie rule."""
+    rng = np.random.default_rng(8000 + block)
+    for case in range(2):
+        dtype = str(rng.choice(["float16", "float16", "float32"]))
+        E = int(rng.choice([64, 136, 256, 1024]))
+        n = int(rng.integers(8193, 30000))
+        emb = synth.embeddings(8100 + 10 * block + case, n, E, dtype)
+        emb[n - 1] = emb[5]
+        emb[n // 2] = emb[5]
+        ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float32 if dtype == "float32" else torch.float16,
+                      rope_theta=1e4, max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+        for a in range(0, n, 8192):
+            ms.add_facts(to_dev(emb[a : a + 8192]), np.zeros(min(8192, n - a), np.int32))
+        nq = int(rng.choice([1, 8, 33, 70]))
+        q = synth.queries(8200 + 10 * block + case, nq, E, dtype)
+        q[0] = emb[5]
+        k = int(rng.choice([1, 100, 256, 300]))
+        ids, sc = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+        if k >= 3:
+            assert ids[0, :3].tolist() == [5, n // 2, n - 1], (block, case)
+        for i in sorted({0, nq // 2, nq - 1}):
+            check_ids(ids[i], sc[i], emb, q[i], k)
+        ms.close()
