@@ -236,6 +236,7 @@ __global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectP
   __shared__ int32_t s_begin[kPlanMaxK];  // b_i: first composed token of placed fact i
   __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
   __shared__ PlanShared ps;
+  grid_dependency_wait();    // launched as a programmatic dependent (of the previous call's copy kernel, typically)
   grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
   plan_request<kPlanThreads>(p, blockIdx.x, s_begin, s_src, ps);
 }

@@ -1193,8 +1193,20 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
   if (rc != MS_OK) return rc;
   rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
-  inject_plan_kernel<<<nreq, kPlanThreads, 0, st>>>(p);
-  MS_CUDA(s, cudaGetLastError());
+  {
+    // a programmatic dependent of what precedes it (see launch_score_topk_threads): placed on the SMs while the
+    // previous call's copy kernel drains; the kernel waits for that grid before it does anything
+    cudaLaunchConfig_t lc{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.gridDim = dim3((unsigned)nreq);
+    lc.blockDim = dim3(kPlanThreads);
+    lc.stream = st;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    MS_CUDA(s, cudaLaunchKernelEx(&lc, inject_plan_kernel, p));
+  }
   s->kernels_launched++;
   rc = launch_copy(s, p, cache, tiles_needed, st);
   if (rc != MS_OK) return rc;
