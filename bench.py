@@ -437,6 +437,17 @@ def run_ours(args):
             e1.record(stream)
             torch.cuda.synchronize()
             sweep[f"k{kk}_us"] = e0.elapsed_time(e1) * 1e3 / args.steps
+            # the same request every time: at k = 5 and 10 its source rows and cache blocks (52 / 105 MB) stay in the
+            # 126 MB L2, the "warm" figure next to the rotating ("cold") one above
+            for i in range(10):
+                step_k(0)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(args.steps):
+                step_k(0)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            sweep[f"k{kk}_same_request_us"] = e0.elapsed_time(e1) * 1e3 / args.steps
         line["sweep"] = sweep
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
