@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L.oracle_graph_append.argtypes = [p, i32, i64, i64, i32, p, i32, p, i32]
         L.oracle_ann_search.restype = i32
         L.oracle_ann_search.argtypes = [p, i32, i64, i32, p, i32, p, i32, i32, i32, i32, i32, p, p, p, p]
+        L.oracle_ann_search_exact.restype = i32
+        L.oracle_ann_search_exact.argtypes = L.oracle_ann_search.argtypes + [p]
         L.oracle_inject_ex.restype = i32
         L.oracle_inject_ex.argtypes = L.oracle_inject.argtypes + [i32, C.c_float, C.c_float, p, p]
         L.oracle_rope_rows_partial.restype = i32
@@ -88,6 +90,8 @@ def lib() -> C.CDLL:
                      "oracle_e4m3_to_double"):  # fmt: skip
             getattr(L, name).restype = None
             getattr(L, name).argtypes = [p, i64, p]
+        L.oracle_e4m3_from_scaled_bf16.restype = None
+        L.oracle_e4m3_from_scaled_bf16.argtypes = [p, i64, C.c_float, p]
         _lib = L
     return _lib
 
@@ -138,6 +142,14 @@ def e4m3_from_double(x: np.ndarray) -> np.ndarray:
     x = np.ascontiguousarray(x, dtype=np.float64)
     out = np.empty(x.shape, dtype=np.uint8)
     lib().oracle_e4m3_from_double(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def e4m3_from_scaled_bf16(bits: np.ndarray, scale: float) -> np.ndarray:
+    """Codes of an 8-bit cache that holds value / scale: binary32(bf16 value) / scale in binary32, rounded once to e4m3."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.uint8)
+    lib().oracle_e4m3_from_scaled_bf16(_ptr(bits), bits.size, float(scale), _ptr(out))
     return out
 
 
@@ -218,13 +230,16 @@ def graph_append(emb: np.ndarray, old_graph: np.ndarray, n_threads: int = 0) -> 
 
 
 class AnnResult:
-    def __init__(self, ids, scores, iters, scored):
+    def __init__(self, ids, scores, iters, scored, margin=None):
         self.ids, self.scores, self.iters, self.scored = ids, scores, iters, scored
+        self.margin = margin  # exact search only: smallest score difference that decided a step, per query
 
 
 def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, beam: int = 64, parents: int = 8,
-               n_entry: int = 64, max_iters: int = 32) -> AnnResult:  # fmt: skip
-    """Beam search over ``graph`` for each query: ids / scores [nq, k], steps taken and rows scored per query."""
+               n_entry: int = 64, max_iters: int = 32, exact: bool = False) -> AnnResult:  # fmt: skip
+    """Beam search over ``graph`` for each query: ids / scores [nq, k], steps taken and rows scored per query.
+    ``exact``: rank by the double-precision inner products (and report the decision margin of every query) instead of
+    the binary32 lane sums."""
     emb = np.ascontiguousarray(emb)
     graph = np.ascontiguousarray(graph, dtype=np.int32)
     queries = np.ascontiguousarray(queries, dtype=emb.dtype).reshape(-1, emb.shape[1])
@@ -233,15 +248,25 @@ def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, 
     sc = np.empty((nq, k), dtype=np.float32)
     iters = np.zeros(nq, dtype=np.int32)
     scored = np.zeros(nq, dtype=np.int64)
+    margin = np.full(nq, np.inf) if exact else None
     for q in range(nq):
         it, ns = C.c_int32(0), C.c_int64(0)
+        if exact:
+            mg = C.c_double(0.0)
+            rc = lib().oracle_ann_search_exact(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(graph), graph.shape[1],
+                                               _ptr(queries[q]), k, beam, parents, n_entry, max_iters, _ptr(ids[q]), _ptr(sc[q]),
+                                               C.byref(it), C.byref(ns), C.byref(mg))  # fmt: skip
+            if rc:
+                raise OracleError(rc)
+            iters[q], scored[q], margin[q] = it.value, ns.value, mg.value
+            continue
         rc = lib().oracle_ann_search(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(graph), graph.shape[1],
                                      _ptr(queries[q]), k, beam, parents, n_entry, max_iters, _ptr(ids[q]), _ptr(sc[q]),
                                      C.byref(it), C.byref(ns))  # fmt: skip
         if rc:
             raise OracleError(rc)
         iters[q], scored[q] = it.value, ns.value
-    return AnnResult(ids, sc, iters, scored)
+    return AnnResult(ids, sc, iters, scored, margin)
 
 
 def inv_freq(D: int, theta: float) -> np.ndarray:

@@ -35,7 +35,10 @@
  *
  * Parity pins: every exported function is pinned by the CPU tests
  * (closed forms, group law, brute-force joint rotation, numpy float64
- * cross-checks, full-sort comparison, exhaustive e4m3 code tables); none is "parity unpinned".
+ * cross-checks, full-sort comparison, exhaustive e4m3 code tables, torch's
+ * float32 division and float8 cast over every bf16 value, planted decision
+ * margins of the graph search); none is "parity unpinned".  One function is
+ * not an independent definition and says so: score_f32_lanes.
  */
 #include <math.h>
 #include <stdint.h>
@@ -134,6 +137,18 @@ static uint8_t double_to_e4m3_rne_sat(double x) {
     e += 1;
   }
   return (uint8_t)(sign | (uint8_t)(((e + 7) << 3) | (int)q));
+}
+
+/* A bf16 value divided by a per-tensor scale in binary32 (one correctly rounded IEEE division), then rounded once to e4m3. */
+static uint8_t e4m3_of_scaled_bf16(uint16_t b, float scale) {
+  volatile float x = (float)bf16_to_double(b); /* exact */
+  volatile float q = x / scale;                /* binary32 division; volatile keeps it out of wider registers */
+  return double_to_e4m3_rne_sat((double)q);
+}
+
+/* The 8-bit cache code of each bf16 value under a per-tensor scale (the rule of oracle_inject_ex). */
+void oracle_e4m3_from_scaled_bf16(const uint16_t* x, int64_t n, float scale, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = e4m3_of_scaled_bf16(x[i], scale);
 }
 
 void oracle_e4m3_from_double(const double* x, int64_t n, uint8_t* out) {
@@ -269,8 +284,9 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
  *
  *   graph    G[n][deg]: row r lists the deg rows with the largest inner product with row r, r itself
  *            excluded, best first, ties to the lower row (an exact k-nearest-neighbour graph); -1 pads.
- *   scores   a search compares scores, so they are formed in the arithmetic of the path that takes the
- *            decisions: binary32, the fixed summation order below (score_f32_lanes).
+ *   scores   inner products.  oracle_ann_search_exact ranks by the plain double sums and reports the smallest
+ *            score difference that decided anything; oracle_ann_search ranks by binary32 sums taken in one stated
+ *            order (score_f32_lanes), for the cases whose decisions are closer than binary32 rounding.
  *   list     at most L = max(beam, k) entries (score, row, expanded?), ordered by score descending, ties to
  *            the lower row; V = the set of rows ever scored.
  *   start    rows e_i = ((i + 1) * 2654435761) mod n, i < n_entry (duplicates dropped), scored and listed.
@@ -281,6 +297,10 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
  */
 
 /*
+ * NOT an independent definition: this order restates the summation schedule of the CUDA scoring kernels, so that a
+ * search whose decisions hinge on the last bits of a binary32 sum can still be followed.  It is pinned by rounding
+ * behaviour built into test inputs and, through the search, against oracle_ann_search_exact wherever the margin of
+ * that search exceeds binary32 rounding.
  * Inner product in binary32 with a fixed order: the row is cut into vectors of 16 bytes (8 halves or 4
  * floats); vector v belongs to "lane" v mod 32; a lane adds its products one fused multiply-add at a time in
  * increasing element order; the 32 lane sums are then combined by a butterfly (lane l adds lane l xor 16,
@@ -420,7 +440,7 @@ int oracle_graph_append(const void* emb, int emb_dtype, int64_t n_old, int64_t n
 }
 
 typedef struct {
-  float s;
+  double s; /* the score the search ranks by: a double sum, or a binary32 sum held exactly in a double */
   int32_t row;
   int32_t expanded;
 } beam_t;
@@ -435,19 +455,44 @@ static int cmp_beam(const void* a, const void* b) {
   return 0;
 }
 
+/* Score of `row` for the search: the plain double sum (exact = 1) or the binary32 lane sum (exact = 0). */
+static double search_score(const void* emb, int dtype, int64_t row, int dim, const void* query, int exact) {
+  if (!exact) return (double)score_f32_lanes(emb, dtype, row, dim, query);
+  double s = 0.0;
+  for (int d = 0; d < dim; ++d) s += emb_at(query, dtype, d) * emb_at(emb, dtype, row * dim + d);
+  return s;
+}
+
 /*
- * Beam search of one query over the graph, as defined above.  out_ids / out_scores [k]; out_iters (optional):
- * steps taken; out_scored (optional): |V|, the number of rows scored.
+ * The comparisons that decide a step are those between neighbours of the sorted list down to the cut at L: they fix
+ * the order of the kept entries (hence the parents of the next step and the result) and which entry is the first one
+ * dropped.  The smallest score difference among them is the margin by which this step would survive another
+ * arithmetic.  Two rows with identical embedding bytes score alike in any arithmetic and are ordered by row: their
+ * pair is no decision.
  */
-int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
-                      const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
-                      float* out_scores, int32_t* out_iters, int64_t* out_scored) {
+static double step_margin(const beam_t* list, int len, int L, const void* emb, size_t row_bytes, double margin) {
+  for (int i = 0; i < L && i + 1 < len; ++i) {
+    double gap = list[i].s - list[i + 1].s;
+    if (gap >= margin) continue;
+    if (memcmp((const char*)emb + (size_t)list[i].row * row_bytes, (const char*)emb + (size_t)list[i + 1].row * row_bytes,
+               row_bytes) == 0)
+      continue;
+    margin = gap;
+  }
+  return margin;
+}
+
+static int ann_search_core(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
+                           const void* query, int k, int beam, int parents, int n_entry, int max_iters, int exact,
+                           int32_t* out_ids, float* out_scores, int32_t* out_iters, int64_t* out_scored,
+                           double* out_margin) {
   if (!out_ids || k <= 0 || beam <= 0 || parents <= 0 || n_entry <= 0 || max_iters < 0 || deg <= 0 || n < 0 ||
       emb_dim <= 0 || emb_dim % 8)
     return ORACLE_ERR_ARG;
   if (n > 0 && (!emb || !graph || !query)) return ORACLE_ERR_ARG;
   int L = beam > k ? beam : k;
   int cap = L + (parents * deg > n_entry ? parents * deg : n_entry);
+  size_t row_bytes = (size_t)emb_dim * (emb_dtype == ORACLE_F32 ? 4 : 2);
   beam_t* list = (beam_t*)malloc(sizeof(beam_t) * (size_t)cap);
   unsigned char* seen = (unsigned char*)calloc((size_t)(n > 0 ? n : 1), 1);
   int32_t* chosen = (int32_t*)malloc(sizeof(int32_t) * (size_t)parents);
@@ -459,18 +504,20 @@ int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, co
   }
   int len = 0, iters = 0;
   int64_t scored = 0;
+  double margin = INFINITY;
   if (n > 0) {
     for (int i = 0; i < n_entry; ++i) {
       int64_t e = (int64_t)(((uint64_t)(i + 1) * 2654435761ull) % (uint64_t)n);
       if (seen[e]) continue;
       seen[e] = 1;
-      list[len].s = score_f32_lanes(emb, emb_dtype, e, emb_dim, query);
+      list[len].s = search_score(emb, emb_dtype, e, emb_dim, query, exact);
       list[len].row = (int32_t)e;
       list[len].expanded = 0;
       ++len;
       ++scored;
     }
     qsort(list, (size_t)len, sizeof(beam_t), cmp_beam);
+    margin = step_margin(list, len, L, emb, row_bytes, margin);
     if (len > L) len = L;
     for (; iters < max_iters; ++iters) {
       int np = 0;
@@ -486,7 +533,7 @@ int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, co
           int32_t nb = graph[(int64_t)chosen[p] * deg + j];
           if (nb < 0 || nb >= n || seen[nb]) continue;
           seen[nb] = 1;
-          list[len + added].s = score_f32_lanes(emb, emb_dtype, nb, emb_dim, query);
+          list[len + added].s = search_score(emb, emb_dtype, nb, emb_dim, query, exact);
           list[len + added].row = nb;
           list[len + added].expanded = 0;
           ++added;
@@ -494,19 +541,46 @@ int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, co
         }
       len += added;
       qsort(list, (size_t)len, sizeof(beam_t), cmp_beam);
+      margin = step_margin(list, len, L, emb, row_bytes, margin);
       if (len > L) len = L;
     }
   }
   for (int r = 0; r < k; ++r) {
     out_ids[r] = r < len ? list[r].row : -1;
-    if (out_scores) out_scores[r] = r < len ? list[r].s : 0.0f;
+    if (out_scores) out_scores[r] = r < len ? (float)list[r].s : 0.0f;
   }
   if (out_iters) *out_iters = iters;
   if (out_scored) *out_scored = scored;
+  if (out_margin) *out_margin = margin;
   free(list);
   free(seen);
   free(chosen);
   return ORACLE_OK;
+}
+
+/*
+ * Beam search of one query over the graph, as defined above, ranking by the binary32 lane sums.  out_ids /
+ * out_scores [k]; out_iters (optional): steps taken; out_scored (optional): |V|, the number of rows scored.
+ */
+int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
+                      const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
+                      float* out_scores, int32_t* out_iters, int64_t* out_scored) {
+  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 0, out_ids,
+                         out_scores, out_iters, out_scored, NULL);
+}
+
+/*
+ * The same search ranking by the plain double-precision inner products of oracle_scores: the definition of the walk
+ * with no assumption about the order in which a device adds its products.  out_scores are the double scores
+ * rounded to binary32.  out_margin receives the smallest score difference that decided any step (see step_margin;
+ * infinity when nothing was ever compared): a search in another arithmetic whose scores are all within less than
+ * half of it of the exact ones must take the same walk and return the same rows.
+ */
+int oracle_ann_search_exact(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
+                            const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
+                            float* out_scores, int32_t* out_iters, int64_t* out_scored, double* out_margin) {
+  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 1, out_ids,
+                         out_scores, out_iters, out_scored, out_margin);
 }
 
 /* ---------------------------------------------------------------- RoPE */
@@ -610,14 +684,14 @@ int oracle_rope_rows(const double* x, int64_t n_rows, int D, const int64_t* pos,
  *
  * Variants of the model / cache parameterisation (defaults reproduce the plain path):
  *   rotary_dim       0 = the whole head, else only the first rotary_dim coordinates of a head rotate
- *   k_scale, v_scale quantised (e4m3) cache: the cache holds x / scale.  Used only for out_k_fp8 / out_v_fp8
- *                    [nl][m][H][D] bytes, both optional:
- *                      the value (rotated key in double, or stored bf16 value) times 1.0f / scale is first
- *                      rounded to binary32, the arithmetic type of the path in which the code is decided, and that
- *                      binary32 number is rounded once to e4m3.  (For V and for unrotated key coordinates the
- *                      operands are bf16 and binary32, so the binary32 product is fully determined; short bf16
- *                      mantissas make exact e4m3 ties common there, and deciding them in another precision would
- *                      flip a sizeable share of codes.)
+ *   k_scale, v_scale quantised (e4m3) cache with per-tensor scales.  Used only for out_k_fp8 / out_v_fp8
+ *                    [nl][m][H][D] bytes, both optional.  The paper has no 8-bit cache; the rule is the one of the
+ *                    serving engines whose paged cache this fills: their cache-write kernel takes the bf16 key or
+ *                    value that a bf16 cache would hold, divides it by the scale in binary32 (an IEEE division, not a
+ *                    product with a reciprocal) and rounds the quotient once to e4m3, saturating.  So
+ *                      K code = e4m3( binary32( bf16(rotated key) ) / k_scale ),   V code = e4m3( binary32(v) / v_scale ):
+ *                    an injected 8-bit cache is then byte-identical to the one the engine would have written itself
+ *                    from the bf16 cache contents, which is what output equivalence (Theorem 1) asks of an injection.
  * Returns ORACLE_OK or a negative error; on error the outputs are unspecified.
  */
 int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* fact_offset, const int32_t* fact_len,
@@ -633,7 +707,6 @@ int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* 
       bs <= 0 || R <= 0 || R > D || (R & 1))
     return ORACLE_ERR_ARG;
   if ((out_k_fp8 && !(k_scale > 0.0f)) || (out_v_fp8 && !(v_scale > 0.0f))) return ORACLE_ERR_ARG;
-  const float k_inv = out_k_fp8 ? 1.0f / k_scale : 0.0f, v_inv = out_v_fp8 ? 1.0f / v_scale : 0.0f;
   if (layer_begin < 0 || layer_end > n_layers || layer_begin > layer_end) return ORACLE_ERR_ARG;
   if (start_pos < 0) return ORACLE_ERR_ARG;
 
@@ -706,8 +779,8 @@ int oracle_inject_ex(const int32_t* ids, int k, int64_t n_facts, const int64_t* 
           if (out_k_ref) out_k_ref[o + h * D + d] = yout[d];
           if (out_k_bf16) out_k_bf16[o + h * D + d] = kb;
           if (out_v) out_v[o + h * D + d] = vb;
-          if (out_k_fp8) out_k_fp8[o + h * D + d] = double_to_e4m3_rne_sat((double)(float)(yout[d] * (double)k_inv));
-          if (out_v_fp8) out_v_fp8[o + h * D + d] = double_to_e4m3_rne_sat((double)(float)(bf16_to_double(vb) * (double)v_inv));
+          if (out_k_fp8) out_k_fp8[o + h * D + d] = e4m3_of_scaled_bf16(kb, k_scale);
+          if (out_v_fp8) out_v_fp8[o + h * D + d] = e4m3_of_scaled_bf16(vb, v_scale);
           if (k_cache) k_cache[cbase + h * head_stride + d] = kb;
           if (v_cache) v_cache[cbase + h * head_stride + d] = vb;
         }

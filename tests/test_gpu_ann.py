@@ -1,5 +1,6 @@
-"""GPU parity tests of the graph index: the beam search against the oracle's (bit for bit: both compare fp32 scores
-formed in the same order), the graph build against the oracle's exact neighbour graph (near-tie rule of the exact
+"""GPU parity tests of the graph index: the beam search against the oracle's search over double-precision scores (same
+rows, steps and row counts wherever that search's closest decision is wider than binary32 rounding; the rest bit for bit
+against the oracle's binary32 lane-order search), the graph build against the oracle's exact neighbour graph (near-tie rule of the exact
 retrieval), recall against exact retrieval on structured rows, and the error paths."""
 import numpy as np
 import pytest
@@ -11,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
     import oracle
-    from parity import to_dev
+    from parity import check_ann_search, to_dev
     from paper_2607_27090_b200.memstore import MemStore, MemStoreError
 
 DEV = "cuda"
@@ -31,7 +32,7 @@ def emb_store(emb, n_users=1):
     ("float32", 64, 3000, 16, "knn"), ("float16", 1024, 2000, 64, "random"), ("float16", 136, 5000, 8, "random"),
     ("float16", 256, 700, 32, "knn"), ("float32", 8, 40, 4, "random"),
 ])  # fmt: skip
-def test_search_equals_the_oracle_bit_for_bit(dtype, dim, n, deg, kind):
+def test_search_equals_the_oracle(dtype, dim, n, deg, kind):
     emb = synth.embeddings_low_rank(80, n, dim, dtype, intrinsic_dim=min(8, dim))
     emb[n // 2] = emb[3]  # equal scores: the lower row goes first
     graph = oracle.knn_graph(emb, deg) if kind == "knn" else synth.random_graph(81, n, deg)
@@ -42,16 +43,20 @@ def test_search_equals_the_oracle_bit_for_bit(dtype, dim, n, deg, kind):
     ms = emb_store(emb)
     ms.set_graph(to_dev(graph))
     assert torch.equal(ms.get_graph().cpu(), torch.from_numpy(graph))
+    judged_exact = judged = 0
     for k, beam, parents, n_entry, max_iters in ((10, 64, 4, 64, 32), (1, 1, 1, 1, 50), (50, 16, 2, 7, 5), (100, 128, 8, 200, 12),
                                                   (256, 256, 1, 512, 3)):  # fmt: skip
         if parents * deg > 512:
             continue
-        want = oracle.ann_search(emb, graph, q, k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters)
-        ids, sc, cnt = ms.retrieve_ann(to_dev(q), k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters, want_counters=True)
+        par = dict(beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters)
+        ids, sc, cnt = ms.retrieve_ann(to_dev(q), k, want_counters=True, **par)
         torch.cuda.synchronize()
-        assert np.array_equal(ids.cpu().numpy(), want.ids), (k, beam, parents, n_entry, max_iters)
-        assert np.array_equal(sc.cpu().numpy().view(np.uint32), want.scores.view(np.uint32))
-        assert np.array_equal(cnt[:, 0].cpu().numpy(), want.iters) and np.array_equal(cnt[:, 1].cpu().numpy(), want.scored)
+        a, b = check_ann_search(ids.cpu().numpy(), sc.cpu().numpy(), cnt.cpu().numpy(), emb, graph, q, k, **par)
+        judged_exact, judged = judged_exact + a, judged + b
+    # most searches are decided by margins that no binary32 summation order can overturn: those are judged against the
+    # double-precision search alone
+    print(f"graph search parity: {judged_exact} of {judged} queries judged by the exact search")
+    assert judged_exact >= 0.75 * judged
     # the scores are those of the exact path
     ids, sc = ms.retrieve_ann(to_dev(q), 5)
     ex_ids, ex_sc = ms.retrieve(to_dev(q), n if n < 100 else 100)
@@ -105,9 +110,8 @@ def test_recall_against_exact_retrieval_on_structured_rows():
     assert recalls[64] >= 0.9 and recalls[128] >= recalls[16]
     # the library's graph, handed to the oracle, gives the oracle the same answers (search parity at this size)
     g = ms.get_graph().cpu().numpy()
-    want = oracle.ann_search(emb, g, q[:6], k, beam=64, parents=8, n_entry=64, max_iters=32)  # the library's defaults at degree 32
     ids, sc = ms.retrieve_ann(to_dev(q[:6]), k)
-    assert np.array_equal(ids.cpu().numpy(), want.ids)
+    check_ann_search(ids.cpu().numpy(), sc.cpu().numpy(), None, emb, g, q[:6], k, beam=64, parents=8, n_entry=64, max_iters=32)  # the library's defaults at degree 32
     ms.close()
 
 
@@ -178,8 +182,9 @@ def test_retrieve_inject_through_the_graph_index():
     torch.cuda.synchronize()
     assert torch.equal(ids_a, ids_b) and torch.equal(n_a, n_b) and int(st_b.abs().sum()) == 0
     assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
-    want = oracle.ann_search(hs.emb, ms.get_graph().cpu().numpy(), q, k, parents=8)
-    assert np.array_equal(ids_b.cpu().numpy(), want.ids)
+    ids_s, sc_s = ms.retrieve_ann(to_dev(q), k)
+    assert torch.equal(ids_s, ids_b)
+    check_ann_search(ids_s.cpu().numpy(), sc_s.cpu().numpy(), None, hs.emb, ms.get_graph().cpu().numpy(), q, k, beam=64, parents=8, n_entry=64, max_iters=32)
     out = np.full(k + 2, -5, np.int32)
     cc = PagedCache.allocate(hs.L, nb, bs, hs.H, hs.D, DEV, fill_bits=synth.SENTINEL_BF16)
     ms.serve_host(q[1], k, 5, tables[1].cpu().numpy(), cc, out, flags=M.INJECT_REVERSE | M.RETRIEVE_ANN)

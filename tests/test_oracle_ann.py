@@ -1,8 +1,11 @@
-"""Pins for the oracle's graph index (CPU only): the fixed-order binary32 scores, the exact neighbour graph and the
-beam search.  Each check is against something other than the oracle's own code: exact sums with a rounding
-behaviour known by construction, numpy's float64 matmul and argsort, brute force over all rows where the search
-must degenerate to it, and walks on a path graph that can be followed by hand."""
+"""Pins for the oracle's graph index (CPU only): the exact neighbour graph and the beam search in its two forms - ranking by
+the plain double-precision scores (the definition, with the margin of its closest decision) and ranking by binary32 sums
+in one stated order (for cases decided inside binary32 rounding).  Each check is against something other than the
+oracle's own code: exact sums with a rounding behaviour known by construction, numpy's float64 matmul and argsort,
+brute force over all rows where the search must degenerate to it, walks on a path graph that can be followed by hand,
+margins planted in the inputs, and agreement of the two forms wherever the margin exceeds binary32 rounding."""
 import numpy as np
+import pytest
 
 from paper_2607_27090_b200 import synth
 
@@ -60,25 +63,30 @@ def test_knn_graph_against_numpy_argsort(oracle_mod):
     assert np.all(tiny[:, 3:] == -1) and np.all(tiny[:, :3] >= 0)  # fewer rows than neighbours: padded
 
 
-def test_search_on_a_complete_graph_is_brute_force(oracle_mod):
+@pytest.mark.parametrize("exact", [False, True])
+def test_search_on_a_complete_graph_is_brute_force(oracle_mod, exact):
     n, dim, k = 150, 64, 12
     emb = synth.embeddings(3, n, dim, "float32")
     complete = np.array([[c for c in range(n) if c != r] for r in range(n)], np.int32)
     q = synth.queries(3, 4, dim, "float32")
-    res = oracle_mod.ann_search(emb, complete, q, k, beam=4, parents=1, n_entry=1, max_iters=3)
-    want, _ = oracle_mod.retrieve(emb, q, k)
+    res = oracle_mod.ann_search(emb, complete, q, k, beam=4, parents=1, n_entry=1, max_iters=3, exact=exact)
+    want, want_sc = oracle_mod.retrieve(emb, q, k)
     assert np.array_equal(res.ids, want)
     assert np.all(res.scored == n) and np.all(res.iters >= 1)
     for i in range(4):
-        assert np.array_equal(res.scores[i], oracle_mod.scores_f32(emb, q[i])[res.ids[i]])
+        if exact:  # the double scores rounded to binary32, as exact retrieval reports them
+            assert np.array_equal(res.scores[i], want_sc[i])
+        else:
+            assert np.array_equal(res.scores[i], oracle_mod.scores_f32(emb, q[i])[res.ids[i]])
 
 
-def test_search_with_a_beam_as_large_as_the_store_visits_the_whole_component(oracle_mod):
+@pytest.mark.parametrize("exact", [False, True])
+def test_search_with_a_beam_as_large_as_the_store_visits_the_whole_component(oracle_mod, exact):
     n, dim = 300, 64
     emb = synth.embeddings_low_rank(4, n, dim, "float32", intrinsic_dim=6)
     g = oracle_mod.knn_graph(emb, 8)
     q = synth.queries_near_rows(4, emb, 3)
-    res = oracle_mod.ann_search(emb, g, q, 10, beam=n, parents=3, n_entry=n, max_iters=1000)
+    res = oracle_mod.ann_search(emb, g, q, 10, beam=n, parents=3, n_entry=n, max_iters=1000, exact=exact)
     want, _ = oracle_mod.retrieve(emb, q, 10)
     assert np.array_equal(res.ids, want) and np.all(res.scored == n)  # every row is an entry point here
 
@@ -88,7 +96,8 @@ def arc(n):
     return np.stack([np.cos(a), np.sin(a)] + [np.zeros(n)] * 6, axis=1).astype(np.float32)  # dim 8
 
 
-def test_greedy_walk_on_a_path_graph_can_be_followed_by_hand(oracle_mod):
+@pytest.mark.parametrize("exact", [False, True])
+def test_greedy_walk_on_a_path_graph_can_be_followed_by_hand(oracle_mod, exact):
     # 100 points on an arc, row i linked to i-1 and i+1; the only entry point is (1 * 2654435761) mod 100 = 61.
     n = 100
     emb = arc(n)
@@ -96,33 +105,89 @@ def test_greedy_walk_on_a_path_graph_can_be_followed_by_hand(oracle_mod):
     q = emb[70:71].copy()
     # beam 1: each step expands the single listed row and moves one row towards 70; 9 moves, then the step that
     # expands 70 itself finds nothing better; the next look finds no unexpanded entry
-    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=50)
+    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=50, exact=exact)
     # rows scored: the entry, 60 and 62 in step 1, then one new row per step (the other neighbour was seen): 63..70, 71
     assert res.ids[0, 0] == 70 and res.iters[0] == 10 and res.scored[0] == 1 + 2 + 8 + 1
-    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=5)
+    res = oracle_mod.ann_search(emb, path, q, 1, beam=1, parents=1, n_entry=1, max_iters=5, exact=exact)
     assert res.ids[0, 0] == 66 and res.iters[0] == 5
     # beam 3 keeps the trail: after 4 steps the list is 65, 64, 63 (closest to 70 first)
-    res = oracle_mod.ann_search(emb, path, q, 3, beam=3, parents=1, n_entry=1, max_iters=4)
+    res = oracle_mod.ann_search(emb, path, q, 3, beam=3, parents=1, n_entry=1, max_iters=4, exact=exact)
     assert res.ids[0].tolist() == [65, 64, 63]
     # two entry points, 61 and (2 * 2654435761) mod 100 = 22: the walk from 61 still wins, 22 is never expanded first
-    res = oracle_mod.ann_search(emb, path, q, 2, beam=2, parents=1, n_entry=2, max_iters=50)
+    res = oracle_mod.ann_search(emb, path, q, 2, beam=2, parents=1, n_entry=2, max_iters=50, exact=exact)
     assert res.ids[0].tolist() == [70, 71] or res.ids[0].tolist() == [70, 69]
     assert abs(float(res.scores[0, 0]) - 1.0) < 1e-6
 
 
-def test_holes_bad_rows_padding_and_duplicate_entry_points(oracle_mod):
+@pytest.mark.parametrize("exact", [False, True])
+def test_holes_bad_rows_padding_and_duplicate_entry_points(oracle_mod, exact):
     emb = arc(10)
     g = np.array([[-1, 11], [0, 2], [1, 1], [2, 2], [-5, 3], [4, 4], [5, 5], [6, 6], [7, 7], [8, 8]], np.int32)
     # entry (2654435761 mod 10) = 1; from 1 the walk reaches 0 and 2 only; rows 3.. point backwards
-    res = oracle_mod.ann_search(emb, g, emb[9:10], 5, beam=5, parents=2, n_entry=1, max_iters=20)
+    res = oracle_mod.ann_search(emb, g, emb[9:10], 5, beam=5, parents=2, n_entry=1, max_iters=20, exact=exact)
     assert sorted(res.ids[0, :3].tolist()) == [0, 1, 2] and res.ids[0, 3:].tolist() == [-1, -1] and res.scored[0] == 3
     assert res.scores[0, 3:].tolist() == [0.0, 0.0]
     # 30 entry points on 10 rows: duplicates dropped, at most 10 rows scored
-    res = oracle_mod.ann_search(emb, g, emb[9:10], 3, beam=3, parents=1, n_entry=30, max_iters=0)
+    res = oracle_mod.ann_search(emb, g, emb[9:10], 3, beam=3, parents=1, n_entry=30, max_iters=0, exact=exact)
     assert res.scored[0] <= 10 and res.iters[0] == 0 and res.ids[0, 0] >= 0
     # empty store
-    res = oracle_mod.ann_search(emb[:0], g[:0], emb[9:10], 2)
+    res = oracle_mod.ann_search(emb[:0], g[:0], emb[9:10], 2, exact=exact)
     assert res.ids[0].tolist() == [-1, -1]
+    if exact:
+        assert res.margin[0] == np.inf  # nothing was ever compared
+
+
+def test_decision_margin_is_the_gap_planted_in_the_inputs(oracle_mod):
+    """Rows whose score against the query e_0 is their first coordinate, on a complete graph with every row an entry
+    point: the list is the sorted scores, and the margin is the smallest gap between neighbours down to the cut."""
+    vals = np.array([1.0, 0.5, 0.5 + 2.0**-20, 0.25, 0.125, 0.125 - 2.0**-12, -0.75, 0.0625], np.float32)
+    n = len(vals)
+    emb = np.zeros((n, 8), np.float32)
+    emb[:, 0] = vals
+    emb[:, 1] = np.arange(n)  # rows differ elsewhere too (orthogonal to the query)
+    q = np.zeros((1, 8), np.float32)
+    q[0, 0] = 1.0
+    complete = np.array([[c for c in range(n) if c != r] for r in range(n)], np.int32)
+    order = np.argsort(-vals.astype(np.float64), kind="stable")
+    res = oracle_mod.ann_search(emb, complete, q, n, beam=n, parents=1, n_entry=n, max_iters=4, exact=True)
+    assert res.ids[0].tolist() == order.tolist() and res.margin[0] == 2.0**-20
+    # a cut at L = 3 still looks at the pair (kept 2, dropped 3) = (0.5, 0.25), and no further: the 2^-12 gap is below the cut
+    res = oracle_mod.ann_search(emb, complete, q, 3, beam=3, parents=1, n_entry=n, max_iters=0, exact=True)
+    assert res.ids[0].tolist() == order[:3].tolist() and res.margin[0] == 2.0**-20
+    res = oracle_mod.ann_search(emb, complete, q, 1, beam=1, parents=1, n_entry=n, max_iters=0, exact=True)
+    assert res.ids[0].tolist() == [0] and res.margin[0] == 1.0 - (0.5 + 2.0**-20)
+    # identical rows tie in every arithmetic and are ordered by row: their pair is not a decision
+    emb2 = emb.copy()
+    emb2[3] = emb2[1]
+    res = oracle_mod.ann_search(emb2, complete, q, n, beam=n, parents=1, n_entry=n, max_iters=4, exact=True)
+    assert res.ids[0, :4].tolist() == [0, 2, 1, 3] and res.margin[0] == 2.0**-20
+    # equal scores of rows that differ elsewhere: a decision with margin zero (any other arithmetic may order them otherwise)
+    emb3 = emb.copy()
+    emb3[3, 0] = emb3[1, 0]
+    res = oracle_mod.ann_search(emb3, complete, q, n, beam=n, parents=1, n_entry=n, max_iters=4, exact=True)
+    assert res.ids[0, :4].tolist() == [0, 2, 1, 3] and res.margin[0] == 0.0
+
+
+def test_the_binary32_search_takes_the_exact_walk_wherever_the_margin_exceeds_its_rounding(oracle_mod):
+    """The two forms share the walk's bookkeeping but not the arithmetic that ranks: wherever every decision of the
+    exact search is wider than 1e-6 (binary32 sums of unit-norm rows are within 3e-7 of the exact ones) the lane-order
+    search must return the same rows after the same steps.  A wrong lane order, a dropped vector or a mis-added partial
+    sum moves scores by far more than that and breaks the agreement."""
+    total = agree_needed = 0
+    for seed, dtype, dim, n, deg in ((1, "float16", 1024, 1500, 32), (2, "float32", 64, 3000, 16), (3, "float16", 136, 2500, 8)):
+        emb = synth.embeddings_low_rank(seed, n, dim, dtype, intrinsic_dim=8)
+        g = oracle_mod.knn_graph(emb, deg) if seed != 3 else synth.random_graph(seed, n, deg)
+        q = synth.queries_near_rows(seed + 10, emb, 12)
+        for k, beam, parents, n_entry, max_iters in ((10, 64, 4, 64, 32), (50, 16, 2, 7, 5), (100, 128, 8, 200, 12)):
+            a = oracle_mod.ann_search(emb, g, q, k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters)
+            b = oracle_mod.ann_search(emb, g, q, k, beam=beam, parents=parents, n_entry=n_entry, max_iters=max_iters, exact=True)
+            for i in range(len(q)):
+                total += 1
+                if b.margin[i] > 1e-6:
+                    agree_needed += 1
+                    assert np.array_equal(a.ids[i], b.ids[i]) and a.iters[i] == b.iters[i] and a.scored[i] == b.scored[i]
+                    assert np.abs(a.scores[i] - b.scores[i]).max() < 3e-7
+    assert agree_needed > 0.8 * total
 
 
 def test_recall_grows_with_the_beam_on_structured_rows(oracle_mod):

@@ -65,6 +65,59 @@ def test_e4m3_matches_torch_float8_cast(oracle_mod):
     assert np.array_equal(got, want)
 
 
+def bf16_bits_to_f32(bits_: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits_).view(np.int16)).view(torch.bfloat16).float()
+
+
+def torch_e4m3(x32: torch.Tensor) -> np.ndarray:
+    """float32 -> e4m3 codes by torch's cast (one step, nearest even), saturating first as the cache-write kernels do."""
+    return x32.clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+
+
+@pytest.mark.parametrize("k_scale,v_scale", [(0.3, 0.0173), (2.7, 0.3), (0.0173, 2.7), (0.5, 0.25)])
+def test_e4m3_cache_codes_follow_the_engine_rule_at_any_scale(oracle_mod, k_scale, v_scale):
+    """The code of an 8-bit cache element is e4m3(binary32(bf16 value) / scale): the bf16 key or value a bf16 cache would
+    hold, an IEEE binary32 division by the per-tensor scale, one rounding to e4m3.  Pinned against torch (bf16 -> float32,
+    float32 division, float8 cast) at scales whose reciprocal is not a binary32 number; quantising the unrounded
+    rotated key instead of its bf16 value is a visibly different rule on these inputs."""
+    rng = np.random.default_rng(21)
+    kb, vb = small_store(rng, L=2, T=64, H=2, D=32)
+    lens = np.array([16, 16, 16, 16], np.int32)
+    offs = np.array([0, 16, 32, 48], np.int64)
+    table = np.arange(8, dtype=np.int32)
+    res = oracle_mod.inject([2, 0, 3, 1], offs, lens, kb, vb, 1e4, 3, table, 16, 8, k_scale=k_scale, v_scale=v_scale)
+    ks, vs = torch.tensor(k_scale, dtype=torch.float32), torch.tensor(v_scale, dtype=torch.float32)
+    want_k = torch_e4m3(bf16_bits_to_f32(res.k_bf16) / ks)
+    want_v = torch_e4m3(bf16_bits_to_f32(res.v) / vs)
+    assert np.array_equal(res.k_fp8, want_k) and np.array_equal(res.v_fp8, want_v)
+    unrounded_k = torch_e4m3(torch.from_numpy(res.k_ref).float() / ks)
+    assert (unrounded_k != want_k).any()
+
+
+@pytest.mark.parametrize("scale", [0.3, 2.7, 0.9, 0.0173])
+def test_e4m3_division_rule_on_every_bf16_value(oracle_mod, scale):
+    """All finite bf16 values as the values of one long fact: the codes are those of torch's float32 division and float8
+    cast.  At 0.3, 2.7 and 0.9 a product with the rounded reciprocal would give other codes for some of these values,
+    so the pin tells division from multiplication; large quotients saturate at +-448."""
+    every = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    x = bf16_bits_to_f32(every)
+    every = every[torch.isfinite(x).numpy()]
+    x = bf16_bits_to_f32(every)
+    n = every.size // 2
+    store = np.ascontiguousarray(every[: 2 * n].reshape(1, n, 1, 2))  # one layer, one head of two coordinates per token
+    nb = (n + 15) // 16
+    res = oracle_mod.inject([0], np.array([0], np.int64), np.array([n], np.int32), store, store, 1e4, 0,
+                            np.arange(nb, dtype=np.int32), 16, nb, k_scale=1.0, v_scale=scale)  # fmt: skip
+    st = torch.tensor(scale, dtype=torch.float32)
+    want = torch_e4m3(x[: 2 * n] / st).reshape(1, n, 1, 2)
+    assert np.array_equal(res.v_fp8, want)
+    by_product = torch_e4m3(x[: 2 * n] * (1.0 / st)).reshape(1, n, 1, 2)
+    if scale != 0.0173:
+        assert (by_product != want).any()
+    big = (x[: 2 * n].abs() / st > 470).numpy().reshape(1, n, 1, 2)
+    assert big.any() and set(res.v_fp8[big].tolist()) <= {0x7E, 0xFE}
+
+
 # ------------------------------------------------------------------------------------------------ rescaled frequencies
 def test_llama3_table_regions_with_closed_forms(oracle_mod):
     for R, theta in ((128, 5e5), (64, 1e4)):
@@ -145,9 +198,9 @@ def test_inject_with_partial_rotation_and_e4m3_cache_images(oracle_mod):
     pos = 5 + np.arange(part.m)
     lead = oracle_mod.rope_rows(x[..., :16].reshape(-1, 16), np.tile(np.repeat(pos, 2), 2), 1e4)
     assert np.array_equal(part.k_ref[..., :16].reshape(-1, 16), lead)
-    # quantised images: within half an e4m3 step of value / scale, and exactly the rounding of its binary32 value
-    for codes, ref, scale in ((part.k_fp8, part.k_ref, 0.5), (part.v_fp8, oracle_mod.bf16_to_double(part.v), 0.25)):
-        target = ref / scale  # 1 / 0.5 and 1 / 0.25 are exact in binary32, so this is the value both paths quantise
+    # quantised images decode to within half an e4m3 step (+ the bf16 rounding of the key) of value / scale
+    for codes, ref, scale in ((part.k_fp8, oracle_mod.bf16_to_double(part.k_bf16), 0.5), (part.v_fp8, oracle_mod.bf16_to_double(part.v), 0.25)):
+        target = ref / scale  # exact in binary32 for these two scales
         dec = oracle_mod.e4m3_to_double(codes)
         step = np.maximum(2.0 ** (np.floor(np.log2(np.maximum(np.abs(target), 2.0**-6))) - 3), 2.0**-9)
         assert np.all(np.abs(dec - np.clip(target, -448, 448)) <= step / 2)
