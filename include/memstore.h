@@ -66,7 +66,8 @@ enum {
   MS_REQ_BLOCK_TABLE_SHORT = 4, /* pos / block_size >= max_blocks: token skipped */
   MS_REQ_BAD_BLOCK_ID = 8,      /* table entry < 0 or >= num_blocks: token skipped */
   MS_REQ_POSITION_OVERFLOW = 16, /* pos >= max_position: token skipped */
-  MS_REQ_KERNEL_TIMEOUT = 32     /* a bounded wait inside the copy kernel ran out: the cache contents of this call are incomplete */
+  MS_REQ_KERNEL_TIMEOUT = 32,    /* a bounded wait inside the copy kernel ran out: the cache contents of this call are incomplete */
+  MS_REQ_BAD_START = 64          /* start_pos < 0: no token of the request is placed */
 };
 
 enum { MS_DTYPE_F32 = 0, MS_DTYPE_F16 = 1, MS_DTYPE_BF16 = 2 };
@@ -272,8 +273,9 @@ typedef struct {
   int32_t block_size;
   int32_t dtype;            /* MS_CACHE_BF16 (0) or MS_CACHE_FP8_E4M3 */
   float k_scale, v_scale;   /* MS_CACHE_FP8_E4M3 only, both > 0: the cache holds K / k_scale and V / v_scale (per-tensor
-                               scales).  The rotated key (fp32) and the stored value are multiplied by 1.0f / scale in
-                               fp32 and rounded once, to nearest even, saturating at +-448. */
+                               scales), formed as a serving engine's own cache write forms them: the bf16 key (rotated
+                               and rounded as for a bf16 cache) or bf16 value is divided by the scale in fp32 (IEEE
+                               division) and the quotient rounded once to e4m3, to nearest even, saturating at +-448. */
 } ms_paged_cache;
 
 /*
@@ -285,7 +287,9 @@ typedef struct {
  *   on the fly, one round-to-nearest-even to bf16), V rows are copied bit for bit.
  *
  *   fact_ids      device int32 [nreq][k], placement order; entries < 0 are skipped
- *   start_pos     device int32 [nreq]
+ *   start_pos     device int32 [nreq]; the position of the first composed token (Sec. 3.3 / 5.2: positions are
+ *                 contiguous from there).  A negative value places nothing and sets MS_REQ_BAD_START; a value at or
+ *                 beyond max_position places nothing and sets MS_REQ_POSITION_OVERFLOW
  *   block_tables  device int32 [nreq][max_blocks]
  *   out_n_tokens  device int32 [nreq] or NULL: m = number of tokens composed (including skipped ones)
  *   out_status    device int32 [nreq] or NULL: MS_REQ_* bits

@@ -33,7 +33,7 @@ struct InjectParams {
   __nv_bfloat16* v_cache;
   int64_t layer_stride, block_stride, token_stride, head_stride, num_blocks;
   int32_t block_size;
-  float k_inv_scale, v_inv_scale;  // 8-bit cache: 1.0f / scale of K and V
+  float k_scale, v_scale;  // 8-bit cache: per-tensor scales of K and V (the cache holds value / scale)
   // outputs
   int32_t* out_n_tokens;
   int32_t* out_status;
@@ -159,8 +159,17 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     __syncthreads();
   }
   const int32_t m = s_carry;
-  const int32_t first_tile_pos = (start / kTileTokens) * kTileTokens;
-  const uint32_t n_tiles = m > 0 ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
+  // A start position that is negative, or at or beyond the position bound, places no token at all: no tile is made
+  // (the divisions and the block-table lookups below assume 0 <= pos), the request gets a status bit, and the slot
+  // mapping lists every composed token as skipped.
+  const bool bad_start = start < 0 || start >= p.max_position;
+  if (bad_start && m > 0) {
+    if (tid == 0) atomicOr(&s_status, start < 0 ? 64 /*MS_REQ_BAD_START*/ : 16 /*MS_REQ_POSITION_OVERFLOW*/);
+    if (p.out_slot_mapping)
+      for (int64_t q = tid; q < min((int64_t)m, p.slot_stride); q += THREADS) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = -1;
+  }
+  const int32_t first_tile_pos = bad_start ? 0 : (start / kTileTokens) * kTileTokens;
+  const uint32_t n_tiles = (m > 0 && !bad_start) ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
   uint32_t tile_base = 0;
   if (p.nreq > 1) {  // (a single request owns the whole tile list: no ticket needed)
     if (tid == 0) s_tile_base = n_tiles ? atomicAdd(&p.ctrl->acc, n_tiles) : 0u;
@@ -308,42 +317,14 @@ __device__ __forceinline__ uint2 pack_e4m3x8(const float* f) {
   return make_uint2(w[0], w[1]);
 }
 
-// The 8 bf16 values of a 16-byte vector times `scale` (one fp32 rounding each).
+// The 8 bf16 values of a 16-byte vector divided by `scale`: IEEE fp32 division, the arithmetic of the serving engines'
+// own 8-bit cache write (they divide the bf16 key or value by the per-tensor scale in fp32 and round once to e4m3).
 __device__ __forceinline__ void scaled_floats(const uint4& a, float scale, float* f) {
   const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    f[2 * w] = __fmul_rn(bf16lo(aw[w]), scale);
-    f[2 * w + 1] = __fmul_rn(bf16hi(aw[w]), scale);
-  }
-}
-
-// rotate_unit with fp32 results (times `scale`) instead of packed bf16: fa = the 8 elements of vector a, fb of b.
-template <int STYLE>
-__device__ __forceinline__ void rotate_unit_f32(const uint4& a, const uint4& b, const float* sn, const float* cs, float scale,
-                                                float* fa, float* fb) {
-  const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
-  const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b);
-  if (STYLE == 0) {
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float x1l = bf16lo(aw[w]), x1h = bf16hi(aw[w]);
-      const float x2l = bf16lo(bw[w]), x2h = bf16hi(bw[w]);
-      fa[2 * w] = (x1l * cs[2 * w] - x2l * sn[2 * w]) * scale;
-      fb[2 * w] = (x2l * cs[2 * w] + x1l * sn[2 * w]) * scale;
-      fa[2 * w + 1] = (x1h * cs[2 * w + 1] - x2h * sn[2 * w + 1]) * scale;
-      fb[2 * w + 1] = (x2h * cs[2 * w + 1] + x1h * sn[2 * w + 1]) * scale;
-    }
-  } else {
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float x1 = bf16lo(aw[w]), x2 = bf16hi(aw[w]);
-      fa[2 * w] = (x1 * cs[w] - x2 * sn[w]) * scale;
-      fa[2 * w + 1] = (x2 * cs[w] + x1 * sn[w]) * scale;
-      const float z1 = bf16lo(bw[w]), z2 = bf16hi(bw[w]);
-      fb[2 * w] = (z1 * cs[4 + w] - z2 * sn[4 + w]) * scale;
-      fb[2 * w + 1] = (z2 * cs[4 + w] + z1 * sn[4 + w]) * scale;
-    }
+    f[2 * w] = __fdiv_rn(bf16lo(aw[w]), scale);
+    f[2 * w + 1] = __fdiv_rn(bf16hi(aw[w]), scale);
   }
 }
 
@@ -366,8 +347,10 @@ constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a
 // ------------------------------------------------------------------------------------------------
 //
 // Variants: when only the first R < D coordinates rotate, octets j >= R/16 of a head are plain copies (for both pair
-// styles their two vectors are the 32 contiguous bytes at element 16 j).  FP8 = true writes an 8-bit e4m3 cache:
-// rotated keys and values are scaled in fp32 and rounded once; a thread then stores two 8-byte vectors per row.
+// styles their two vectors are the 32 contiguous bytes at element 16 j).  FP8 = true writes an 8-bit e4m3 cache: the
+// bf16 key (rotated and rounded exactly as for a bf16 cache) and the bf16 value are divided by the per-tensor scale in
+// fp32 and rounded once to e4m3, so the cache is byte for byte what an engine's own cache write would make of the
+// bf16 cache contents; a thread then stores two 8-byte vectors per row.
 template <int STYLE, bool FP8>
 __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const InjectParams p) {
   const int tid = threadIdx.x;
@@ -444,17 +427,14 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
           st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
         } else {
           float fa[8], fb[8];
-          if (rotates) {
-            rotate_unit_f32<STYLE>(ka[u], kb[u], sn, cs, p.k_inv_scale, fa, fb);
-          } else {
-            scaled_floats(ka[u], p.k_inv_scale, fa);
-            scaled_floats(kb[u], p.k_inv_scale, fb);
-          }
+          if (rotates) rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+          scaled_floats(ka[u], p.k_scale, fa);
+          scaled_floats(kb[u], p.k_scale, fb);
           uint8_t* kd = reinterpret_cast<uint8_t*>(p.k_cache) + dbase + (int64_t)h * p.head_stride;
           st_stream8(reinterpret_cast<uint2*>(kd + offA), pack_e4m3x8(fa));
           st_stream8(reinterpret_cast<uint2*>(kd + offB), pack_e4m3x8(fb));
-          scaled_floats(va[u], p.v_inv_scale, fa);
-          scaled_floats(vb[u], p.v_inv_scale, fb);
+          scaled_floats(va[u], p.v_scale, fa);
+          scaled_floats(vb[u], p.v_scale, fb);
           uint8_t* vd = reinterpret_cast<uint8_t*>(p.v_cache) + dbase + (int64_t)h * p.head_stride;
           st_stream8(reinterpret_cast<uint2*>(vd + offA), pack_e4m3x8(fa));
           st_stream8(reinterpret_cast<uint2*>(vd + offB), pack_e4m3x8(fb));

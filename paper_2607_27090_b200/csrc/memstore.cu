@@ -73,8 +73,10 @@ struct memstore {
   // proximity graph of user 0's rows (memstore_build_graph / memstore_set_graph): [graph_rows][graph_deg]
   int32_t* graph = nullptr;
   int64_t graph_rows = 0;
+  int64_t graph_cap_rows = 0;  // rows the graph array has room for (memstore_graph_append grows it geometrically)
   int32_t graph_deg = 0;
   int32_t* graph_topk = nullptr;  // build scratch: [64][deg + 1] ids
+  size_t graph_topk_cap = 0;      // its size in entries
   unsigned long long* append_pairs = nullptr;  // graph_append scratch: sorted (old row, new row) offers, then their count
   int64_t prefix_off = 0;   // instruction prefix (memstore_set_prefix): first arena token and length (0 = none)
   int32_t prefix_len = 0;
@@ -706,9 +708,11 @@ static ms_status graph_alloc(memstore* s, int64_t n_rows, int32_t degree) {
   cudaFree(s->graph);
   s->graph = nullptr;
   s->graph_rows = 0;
+  s->graph_cap_rows = 0;
   s->graph_deg = 0;
   if (n_rows > 0) MS_CUDA(s, cudaMalloc(&s->graph, (size_t)n_rows * degree * sizeof(int32_t)));
   s->graph_rows = n_rows;
+  s->graph_cap_rows = n_rows;
   s->graph_deg = degree;
   return MS_OK;
 }
@@ -736,7 +740,9 @@ ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) 
   const int k1 = degree + 1;
   cudaFree(s->graph_topk);
   s->graph_topk = nullptr;
+  s->graph_topk_cap = 0;
   MS_CUDA(s, cudaMalloc(&s->graph_topk, (size_t)kBatch * k1 * sizeof(int32_t)));
+  s->graph_topk_cap = (size_t)kBatch * k1;
   const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
   for (int64_t row0 = 0; row0 < n; row0 += kBatch) {
     const int nb = (int)std::min<int64_t>(kBatch, n - row0);
@@ -767,23 +773,39 @@ ms_status memstore_graph_append(memstore_t* s, ms_stream stream) {
   if (n == n_old) return MS_OK;
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
-  // a larger graph array: the old rows are carried over, the new rows are filled below
-  MS_CUDA(s, cudaDeviceSynchronize());
-  int32_t* grown = nullptr;
-  MS_CUDA(s, cudaMalloc(&grown, (size_t)n * deg * sizeof(int32_t)));
-  if (n_old) cudaMemcpy(grown, s->graph, (size_t)n_old * deg * sizeof(int32_t), cudaMemcpyDeviceToDevice);
-  cudaFree(s->graph);
-  s->graph = grown;
+  // room for the new rows: the array grows geometrically (to at least 1.5 times its size, at most the segment's
+  // capacity), so that a stream of small appends does not reallocate and copy the whole graph each time
+  if (n > s->graph_cap_rows) {
+    const int64_t cap = std::min<int64_t>(c.max_facts_per_user, std::max<int64_t>(n, s->graph_cap_rows + s->graph_cap_rows / 2 + 1024));
+    MS_CUDA(s, cudaDeviceSynchronize());
+    int32_t* grown = nullptr;
+    MS_CUDA(s, cudaMalloc(&grown, (size_t)cap * deg * sizeof(int32_t)));
+    if (n_old) {
+      const cudaError_t e = cudaMemcpy(grown, s->graph, (size_t)n_old * deg * sizeof(int32_t), cudaMemcpyDeviceToDevice);
+      if (e != cudaSuccess) {  // the old graph stays in place and usable
+        cudaFree(grown);
+        return fail(s, MS_ERR_CUDA, "copying the graph into its larger array: %s", cudaGetErrorString(e));
+      }
+    }
+    cudaFree(s->graph);
+    s->graph = grown;
+    s->graph_cap_rows = cap;
+  }
   s->graph_rows = n;  // searches after this call see all rows (a failure below clears the graph)
   const int k1 = deg + 1;
   const int batch = std::max(1, std::min(kAppendMaxOffers, kAppendMaxPairs / deg));
-  cudaFree(s->graph_topk);
-  s->graph_topk = nullptr;
-  cudaFree(s->append_pairs);
-  s->append_pairs = nullptr;
   ms_status rc = MS_OK;
-  if (cudaMalloc(&s->graph_topk, (size_t)kAppendMaxOffers * k1 * sizeof(int32_t)) != cudaSuccess ||
-      cudaMalloc(&s->append_pairs, (size_t)kAppendMaxPairs * sizeof(unsigned long long) + 16) != cudaSuccess)
+  if (s->graph_topk_cap < (size_t)kAppendMaxOffers * k1) {
+    MS_CUDA(s, cudaDeviceSynchronize());
+    cudaFree(s->graph_topk);
+    s->graph_topk = nullptr;
+    s->graph_topk_cap = 0;
+    if (cudaMalloc(&s->graph_topk, (size_t)kAppendMaxOffers * k1 * sizeof(int32_t)) != cudaSuccess)
+      rc = fail(s, MS_ERR_OOM, "scratch for growing the graph");
+    else
+      s->graph_topk_cap = (size_t)kAppendMaxOffers * k1;
+  }
+  if (rc == MS_OK && !s->append_pairs && cudaMalloc(&s->append_pairs, (size_t)kAppendMaxPairs * sizeof(unsigned long long) + 16) != cudaSuccess)
     rc = fail(s, MS_ERR_OOM, "scratch for growing the graph");
   const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
   RetrieveParams p{};
@@ -1046,6 +1068,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
 
   // upper bound on tiles: each request composes at most k * (longest fact) tokens, plus a ragged first tile
   const int64_t max_m = (int64_t)k * s->max_fact_len + (with_prefix ? s->prefix_len : 0);
+  if (max_m > 0x3fffffff) return fail(s, MS_ERR_UNSUPPORTED, "a request could compose %lld tokens (k x longest fact): more than 2^30", (long long)max_m);
   const int64_t tiles_per_req = (max_m + kTileTokens - 1) / kTileTokens + 1;
   const int64_t tiles_needed = std::max<int64_t>(1, tiles_per_req * nreq);
   if (tiles_needed > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
@@ -1092,8 +1115,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.head_stride = cache->head_stride;
   p.num_blocks = cache->num_blocks;
   p.block_size = cache->block_size;
-  p.k_inv_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? 1.0f / cache->k_scale : 1.0f;
-  p.v_inv_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? 1.0f / cache->v_scale : 1.0f;
+  p.k_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? cache->k_scale : 1.0f;
+  p.v_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? cache->v_scale : 1.0f;
   p.out_n_tokens = out_n_tokens;
   p.out_status = out_status;
   p.out_slot_mapping = out_slot_mapping;
@@ -1292,6 +1315,7 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
   if (!query || !block_table || !out_ids || max_blocks <= 0 || k < 1 || k > kTopkMaxK)
     return fail(s, MS_ERR_INVALID_ARG, "memstore_serve_host: null buffer, max_blocks=%d or k=%d out of range", max_blocks, k);
   if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
+  if (start_pos < 0) return fail(s, MS_ERR_INVALID_ARG, "negative start position %d", start_pos);
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
   // layout of both staging buffers: [query | start_pos, user, pad, pad | block table] then [ids | n_tokens, status]

@@ -27,6 +27,7 @@ RETRIEVE_ANN = 4
 CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 STORE_TMA_COPY_PATH = 1
 REQ_KERNEL_TIMEOUT = 32
+REQ_BAD_START = 64
 
 
 class MemStoreError(RuntimeError):

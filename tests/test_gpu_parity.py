@@ -679,6 +679,25 @@ def test_inject_data_errors_set_status_and_skip():
     n, s = run([1, 3], 58, [0, 1, 2, 3, 4])
     assert n == 11 and s == M.REQ_POSITION_OVERFLOW
     assert untouched_mask_ok(cache, np.arange(3 * bs + 10, 4 * bs), SENT)
+    # a negative start position (the oracle refuses it as an argument error): nothing is placed, also not the tokens
+    # whose position would be >= 0; a start at or beyond the position bound places nothing either
+    for start, bit in ((-1, M.REQ_BAD_START), (-16, M.REQ_BAD_START), (-(2**31), M.REQ_BAD_START), (64, M.REQ_POSITION_OVERFLOW),
+                       (2**31 - 1, M.REQ_POSITION_OVERFLOW)):  # fmt: skip
+        cache = make_cache(hs, nb, bs)
+        slot_map = torch.full((1, 20), -7, dtype=torch.int64, device=DEV)
+        n, s = ms.inject(to_dev(np.array([[0, 1, 3]], np.int32)), to_dev(np.array([start], np.int32)),
+                         to_dev(np.array([[0, 1, 2, 3, 4]], np.int32)), cache, out_slot_mapping=slot_map)  # fmt: skip
+        torch.cuda.synchronize()
+        assert int(n[0]) == 15 and int(s[0]) == bit, (start, int(s[0]))
+        assert slot_map[0].cpu().tolist() == [-1] * 15 + [-7] * 5
+        assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
+    # the next ordinary request on the same store is unaffected
+    cache = make_cache(hs, nb, bs)
+    n, s = run([0, 3], 2, ok_table)
+    kb, vb = gather_cache_rows(cache, res.slots)
+    assert n == 9 and s == 0 and np.array_equal(vb, res.v)
+    with pytest.raises(RuntimeError):
+        ms.serve_host(hs.emb[0], 2, -1, np.array(ok_table, np.int32), cache, np.zeros(4, np.int32))
 
 
 @pytest.mark.parametrize("path", PATHS)
