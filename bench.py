@@ -43,7 +43,8 @@ def parse_args():
     ap.add_argument("--scale-facts", type=float, default=1.0, help="shrink the store (profiling captures); the request keeps its shape")
     ap.add_argument("--pool-blocks", type=int, default=0, help="cache pool size in blocks (default: at least 4096)")
     ap.add_argument("--query-pool", type=int, default=16)
-    ap.add_argument("--sweep-k", action="store_true", help="also report k = 5, 10, 20 (extra keys, same JSON line)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the extra keys: k = 5, 10, 20 and the batched configurations")
+    ap.add_argument("--configs-budget-seconds", type=float, default=90.0, help="time budget of the batched configurations")
     return ap.parse_args()
 
 
@@ -57,10 +58,15 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+    """Polls SM clock and throttle reasons through NVML (read-only).  One sampler thread lives for the whole run and
+    keeps a sample only while a GPU pass is marked with ``under_load()``: the timed region, the per-kernel and
+    end-to-end passes, a sustained run of the same step, and the batched configurations - so that a short timed
+    region (a few milliseconds at 20 steps) still comes with a clock record of the same work."""
 
     def __init__(self, index: int, period_s: float = 0.005):
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.timed_samples, self.timed_reasons = 0, set()
+        self._load = self._timed = False
         self._stop = threading.Event()
         self._thr = None
         self.period = period_s
@@ -81,15 +87,33 @@ class ClockSampler:
             "hw_power_brake": 0x80, "sync_boost": 0x10, "applications_clocks": 0x2,
         }  # fmt: skip
         while not self._stop.is_set():
-            try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
-                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-                for n, bit in names.items():
-                    if r & bit:
-                        self.reasons.add(n)
-            except Exception:
-                pass
+            if self._load:
+                try:
+                    mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    if self._load:  # still inside the pass when the readings came back
+                        self.samples.append(mhz)
+                        self.timed_samples += self._timed
+                        for n, bit in names.items():
+                            if r & bit:
+                                self.reasons.add(n)
+                                if self._timed:
+                                    self.timed_reasons.add(n)
+                except Exception:
+                    pass
             time.sleep(self.period)
+
+    def under_load(self, timed: bool = False):
+        sampler = self
+
+        class _Pass:
+            def __enter__(self):
+                sampler._timed, sampler._load = timed, True
+
+            def __exit__(self, *a):
+                sampler._load = sampler._timed = False
+
+        return _Pass()
 
     def __enter__(self):
         if self.nv is not None:
@@ -105,7 +129,9 @@ class ClockSampler:
     def summary(self):
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(s)}  # fmt: skip
+                "samples": len(s), "samples_in_timed_region": self.timed_samples,
+                "note": "samples are taken only while GPU passes run: the timed region, the per-kernel / end-to-end / latency "
+                        "passes, a sustained run of the same step and the batched configurations"}  # fmt: skip
 
 
 def max_over_ranks(value: float, world: int, device=None) -> float:
@@ -118,6 +144,32 @@ def max_over_ranks(value: float, world: int, device=None) -> float:
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t[0])
+
+
+def workload_string(name: str, shape, n_facts: int, k: int) -> str:
+    """The one description of the benchmarked workload, printed by both arms."""
+    return (f"{name}: {n_facts} facts of {shape.len_lo}-{shape.len_hi} tokens, L={shape.n_layers} h={shape.n_kv_heads} "
+            f"d={shape.head_dim}, {shape.emb_dim}-d {shape.emb_dtype} embeddings, k={k}, start {shape.start_pos}, "
+            f"block {shape.block_size}")  # fmt: skip
+
+
+def captured_traffic(config: str, k: int):
+    """DRAM bytes (read + write) per launch of the copy kernel from the committed ncu capture of that kernel: the data
+    file next to the summary in profiles/ (one 'key = value' pair per line).  None when there is no capture of this
+    workload."""
+    path = os.path.join(ROOT, "profiles", f"inject_copy_kernel_{config}_k{k}.traffic.txt")
+    if not os.path.exists(path):
+        return None, None
+    kv = {}
+    with open(path) as f:
+        for ln in f:
+            if "=" in ln and not ln.lstrip().startswith("#"):
+                a, b = ln.split("=", 1)
+                kv[a.strip()] = b.strip()
+    try:
+        return float(kv["dram_bytes_per_launch"]), kv.get("captured_at_commit")
+    except (KeyError, ValueError):
+        return None, None
 
 
 THERMAL_REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
@@ -213,7 +265,7 @@ def run_reference(args):
         "metric": METRIC, "value": v, "unit": "us", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": v / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "impl": "reference",
-        "config": {"workload": f"{args.config} k={args.k}", "n_facts": shape.n_facts, "emb_dim": shape.emb_dim},
+        "config": {"workload": workload_string(args.config, shape, shape.n_facts, args.k)},
         "cpu_baseline": {"value": v, "unit": "us", "cores": arm.cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -279,10 +331,12 @@ def run_ours(args):
 
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     remeasured = False
+    clk = ClockSampler(local)
+    clk.__enter__()
     while True:
         launches0 = store.stats()["kernels_launched"]
-        with ClockSampler(local) as clk:
-            barrier()
+        barrier()
+        with clk.under_load(timed=True):
             e0.record(stream)
             for i in range(args.steps):
                 step(i)
@@ -290,9 +344,18 @@ def run_ours(args):
             barrier()
         ms_total = e0.elapsed_time(e1)
         launches = store.stats()["kernels_launched"] - launches0
+        # the same step, sustained for about 0.4 s: the clock record of this work under load (not part of `value`)
+        with clk.under_load():
+            for i in range(max(200, int(0.4e3 / max(ms_total / args.steps, 1e-3)))):
+                step(i)
+            torch.cuda.synchronize()
         throttled = max_over_ranks(float(any(r in clk.reasons for r in THERMAL_REASONS)), world, dev) > 0
         if throttled and not remeasured:  # a thermally throttled run is rejected and measured once more
             remeasured = True
+            clk.samples.clear()
+            clk.reasons.clear()
+            clk.timed_reasons.clear()
+            clk.timed_samples = 0
             time.sleep(2.0)
             continue
         break
@@ -308,6 +371,8 @@ def run_ours(args):
     r0 = [torch.cuda.Event(enable_timing=True) for _ in range(n_prof)]
     r1 = [torch.cuda.Event(enable_timing=True) for _ in range(n_prof)]
     torch.cuda.synchronize()
+    load = clk.under_load()
+    load.__enter__()
     for i in range(n_prof):
         j = i % n_pool
         r0[i].record(stream)
@@ -318,6 +383,7 @@ def run_ours(args):
                      flags=M.INJECT_REVERSE, stream=stream)  # fmt: skip
     store.set_profile_events(None, None)
     torch.cuda.synchronize()
+    load.__exit__()
     copy_us = np.array([a.elapsed_time(b) * 1e3 for a, b in evs])
     retr_us = np.array([a.elapsed_time(b) * 1e3 for a, b in zip(r0, r1)])
     bytes_prof = np.array([workload.kv_bytes_moved(shape, int(m_pool[i % n_pool])) for i in range(n_prof)], dtype=np.float64)
@@ -341,24 +407,24 @@ def run_ours(args):
     for i in range(5):
         e2e_step(i)
     barrier()
-    e0.record(stream)
-    for i in range(n_e2e):
-        e2e_step(i)
-    e1.record(stream)
-    barrier()
+    with clk.under_load():
+        e0.record(stream)
+        for i in range(n_e2e):
+            e2e_step(i)
+        e1.record(stream)
+        barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     e2e_us = e2e_ms * 1e3 / (n_e2e * world)
     h2d = ((q_host[0].numel() * q_host.element_size() + 15) // 16) * 16 + 16 + ((t_host[0].numel() * 4 + 15) // 16) * 16
     d2h = (k + 2) * 4
 
+    traffic, traffic_commit = captured_traffic(args.config, k)
     line = {
         "metric": METRIC, "value": us_per_request, "unit": "us", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": f"{args.config}: {wl.lens.size} facts of {shape.len_lo}-{shape.len_hi} tokens, L={shape.n_layers} "
-                        f"h={shape.n_kv_heads} d={shape.head_dim}, {shape.emb_dim}-d {shape.emb_dtype} embeddings, k={k}, "
-                        f"start {shape.start_pos}, block {shape.block_size}",
+            "workload": workload_string(args.config, shape, int(wl.lens.size), k),
             "mean_tokens_per_request": mean_m, "bytes_per_request": bytes_step,
             "l2_policy": "inputs larger than L2: each request moves ~%.0f MB and rotates over %d queries / block tables"
                          % (bytes_step / 1e6, n_pool),
@@ -369,23 +435,23 @@ def run_ours(args):
         "roofline": {
             "bound": "hbm", "kernel": "inject_copy_kernel", "achieved": copy_gbs, "peak": peak, "unit": "GB/s",
             "frac": copy_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": copy_gbs / NOMINAL_HBM_GBS,
-            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.config, k)),
+            "traffic": traffic, "traffic_captured_at_commit": traffic_commit,
             "algorithmic_bytes_per_launch": float(bytes_prof.mean()),
         },
         "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
-        "clocks": clk.summary(),
     }  # fmt: skip
 
     # ---- per-request latency distribution (separate pass: an event after every step) and CUDA-graph replay ---------
     n_lat = min(args.steps, 500)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat + 1)]
     torch.cuda.synchronize()
-    marks[0].record(stream)
-    for i in range(n_lat):
-        step(i)
-        marks[i + 1].record(stream)
-    torch.cuda.synchronize()
+    with clk.under_load():
+        marks[0].record(stream)
+        for i in range(n_lat):
+            step(i)
+            marks[i + 1].record(stream)
+        torch.cuda.synchronize()
     lat = np.sort(np.array([marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(n_lat)]))
     line["latency_us"] = {"p10": float(lat[n_lat // 10]), "p50": float(lat[n_lat // 2]), "p90": float(lat[(n_lat * 9) // 10]),
                           "n": n_lat, "note": "one CUDA event per step on the stream, steady state"}  # fmt: skip
@@ -418,36 +484,44 @@ def run_ours(args):
         line["graph_replay_error"] = str(ex)[:200]
         torch.cuda.synchronize()
 
-    if args.sweep_k:
-        sweep = {}
+    if not args.no_configs:
+        # the other values of k of this configuration (extra keys; at least 200 steps each whatever --steps says)
+        sweep, n_sweep = {}, max(args.steps, 200)
         for kk in (5, 10, 20):
             ids_k = torch.empty((1, kk), dtype=torch.int32, device=dev)
+
             def step_k(i):
                 j = i % n_pool
                 store.retrieve_inject(queries[j : j + 1], kk, start, tables[j : j + 1], cache, out_ids=ids_k,
                                       out_n_tokens=n_tok[j : j + 1], out_status=status[j : j + 1], flags=M.INJECT_REVERSE,
                                       stream=stream)  # fmt: skip
 
-            for i in range(10):
+            for i in range(n_pool):
                 step_k(i)
             torch.cuda.synchronize()
-            e0.record(stream)
-            for i in range(args.steps):
-                step_k(i)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            sweep[f"k{kk}_us"] = e0.elapsed_time(e1) * 1e3 / args.steps
+            m_k = float(n_tok.cpu().numpy().astype(np.float64).mean())
+            with clk.under_load():
+                e0.record(stream)
+                for i in range(n_sweep):
+                    step_k(i)
+                e1.record(stream)
+                torch.cuda.synchronize()
+            us_k = e0.elapsed_time(e1) * 1e3 / n_sweep
             # the same request every time: at k = 5 and 10 its source rows and cache blocks (52 / 105 MB) stay in the
             # 126 MB L2, the "warm" figure next to the rotating ("cold") one above
             for i in range(10):
                 step_k(0)
             torch.cuda.synchronize()
-            e0.record(stream)
-            for i in range(args.steps):
-                step_k(0)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            sweep[f"k{kk}_same_request_us"] = e0.elapsed_time(e1) * 1e3 / args.steps
+            with clk.under_load():
+                e0.record(stream)
+                for i in range(n_sweep):
+                    step_k(0)
+                e1.record(stream)
+                torch.cuda.synchronize()
+            bytes_k = workload.kv_bytes_moved(shape, 1) * m_k + workload.emb_bytes_scanned(shape, int(wl.lens.size))
+            sweep[f"k{kk}"] = {"us_per_request": us_k, "same_request_us": e0.elapsed_time(e1) * 1e3 / n_sweep, "tokens": m_k,
+                               "path_gbs": bytes_k / (us_k * 1e-6) / 1e9, "frac_of_measured": bytes_k / (us_k * 1e-6) / 1e9 / peak,
+                               "hbm_floor_us": bytes_k / (peak * 1e9) * 1e6}  # fmt: skip
         line["sweep"] = sweep
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -461,17 +535,22 @@ def run_ours(args):
         v1, _ = one.time_step(one.facts_for_budget(3.0))
         line["cpu_baseline"] = {"value": sum(vals) / len(vals), "unit": "us", "cores": arm.cores, "kind": "oracle",
                                 "sample": f"mean of {len(vals)} repeats of: {sample}", "single_thread_value": v1}  # fmt: skip
+    store.close()
+    if rank == 0 and world == 1 and not args.no_configs:
+        # the batched configurations of the workload list (100 users, the 14B-class shape, 1M facts), each with its own
+        # store: the headline store and pool are released first
+        from paper_2607_27090_b200 import measure_configs
+
+        del wl, cache, tables, queries
+        torch.cuda.empty_cache()
+        with clk.under_load():
+            line["configs"] = measure_configs.measure_all(peak, budget_s=args.configs_budget_seconds, seed=args.seed)
+    clk.__exit__()
+    line["clocks"] = clk.summary()
     if rank == 0:
         print(json.dumps(line))
-    store.close()
     if world > 1:
         dist.destroy_process_group()
-
-
-# DRAM bytes (read + write) per launch of the copy kernel from the committed ncu capture summary of that kernel
-# (mean of the two captured launches; the capture starts from a flushed L2, so
-# about 50 MB of the written bytes are still in L2 when the kernel ends and are not in this figure).
-NCU_TRAFFIC_BYTES_PER_LAUNCH: dict = {("llama8b", 50): 467.5e6}
 
 
 if __name__ == "__main__":

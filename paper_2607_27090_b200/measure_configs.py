@@ -6,7 +6,7 @@
 way (CUDA events on one stream, warm-up first, inputs already in HBM) and prints one JSON line per
 configuration: microseconds of the batched retrieve call and of the batched inject call, bytes scanned / moved,
 and the rates they imply.  No step of the method runs here; the hot set of a configuration with partial
-residency is picked by the harness from a plain numpy product (a store-construction input).
+residency (a store-construction input) comes from the library's own retrieval on an embedding-only store.
 """
 from __future__ import annotations
 
@@ -20,29 +20,34 @@ from . import memstore as M
 from . import synth, workload
 
 
-def candidate_hot_ids(emb: np.ndarray, queries: np.ndarray, per_query: int, users: np.ndarray | None = None, per_user: int = 0):
-    """Ids that a request may name: per query the ``per_query`` rows with the largest fp32 numpy scores (inside the
-    query's user segment when ``users`` is given).  A superset of every exact top-k list with k < per_query."""
-    hot: set[int] = set()
-    qf = queries.astype(np.float32)
-    if users is None:
-        n = emb.shape[0]
-        best = np.full((qf.shape[0], per_query), -np.inf, np.float32)
-        best_id = np.zeros((qf.shape[0], per_query), np.int64)
-        for a in range(0, n, 131072):
-            sc = qf @ emb[a : a + 131072].astype(np.float32).T
-            allsc = np.concatenate([best, sc], axis=1)
-            allid = np.concatenate([best_id, np.broadcast_to(np.arange(a, a + sc.shape[1]), sc.shape)], axis=1)
-            part = np.argpartition(-allsc, per_query - 1, axis=1)[:, :per_query]
-            best = np.take_along_axis(allsc, part, axis=1)
-            best_id = np.take_along_axis(allid, part, axis=1)
-        hot.update(best_id.reshape(-1).tolist())
-    else:
-        for i, u in enumerate(users):
-            rows = np.arange(u * per_user, (u + 1) * per_user)
-            sc = emb[rows].astype(np.float32) @ qf[i]
-            hot.update(rows[np.argpartition(-sc, per_query - 1)[:per_query]].tolist())
-    return sorted(hot)
+def free_gib(device) -> float:
+    free, _ = torch.cuda.mem_get_info(device)
+    return free / 2**30
+
+
+def candidate_hot_ids(emb: np.ndarray, queries: np.ndarray, per_query: int, users: np.ndarray | None = None, per_user: int = 0,
+                      device="cuda"):  # fmt: skip
+    """Ids that a request may name (a store-construction input: facts outside this set get no K/V): per query the
+    ``per_query`` best facts of its user's segment, taken from the LIBRARY's own exact retrieval on a temporary
+    embedding-only store, so that no scoring or selection is restated here.  A superset of every top-k list with
+    k <= per_query."""
+    dev = torch.device(device)
+    n_users = 1 if users is None else int(per_user and emb.shape[0] // per_user)
+    seg = emb.shape[0] // n_users
+    tdt = torch.float32 if emb.dtype == np.float32 else torch.float16
+    store = M.MemStore(device=dev.index or 0, n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=emb.shape[1], emb_dtype=tdt,
+                       rope_theta=1e4, n_users=n_users, max_facts_per_user=seg, max_kv_tokens=0)  # fmt: skip
+    for u in range(n_users):
+        for a in range(u * seg, (u + 1) * seg, 65536):
+            b = min((u + 1) * seg, a + 65536)
+            store.add_facts(torch.from_numpy(emb[a:b]).to(dev), [0] * (b - a), user=u)
+    q_dev = torch.from_numpy(queries).to(dev)
+    u_dev = torch.from_numpy(np.asarray(users, np.int32)).to(dev) if users is not None else None
+    ids, _ = store.retrieve(q_dev, per_query, query_users=u_dev)
+    torch.cuda.synchronize(dev)
+    hot = sorted({int(i) for i in ids.cpu().numpy().reshape(-1) if i >= 0})
+    store.close()
+    return hot
 
 
 def measure_retrieve_only(name: str, iters: int, seed: int = 0):
@@ -279,7 +284,11 @@ def measure_ann(n: int, iters: int, seed: int = 0, dim: int = 1024, degree: int 
     return lines
 
 
-def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None):
+def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = None, pool_blocks: int | None = None,
+            want_pool_blocks: int | None = None, headroom_gib: float = 6.0):  # fmt: skip
+    """One batched configuration: the store is built as the configuration states it when the free device memory allows
+    (hot subset of ``resident_per_user`` facts, ``want_pool_blocks`` cache blocks), else the hot subset and then the
+    pool are halved until they fit; the sizes used are in the line."""
     s = synth.CONFIGS[name]
     dev = torch.device("cuda")
     total = s.n_facts * s.n_users
@@ -288,13 +297,27 @@ def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = Non
     queries = synth.queries(seed, nq, s.emb_dim, s.emb_dtype)
     k_inj = 50 if name == "stress1m" else s.k
     users = np.arange(s.n_users, dtype=np.int32) if s.n_users > 1 else None
-    hot = None
-    if s.resident_per_user is not None:
-        hot = candidate_hot_ids(emb, queries, k_inj + 14, users, s.n_facts)
-        if hot_per_user is None:
-            hot_per_user = max(s.resident_per_user // 5, (len(hot) + s.n_users - 1) // s.n_users) if name == "stress1m" else s.resident_per_user
     per_req = workload.blocks_per_request(s, k_inj)
-    nb = pool_blocks or max(1024, 1 << int(np.ceil(np.log2(per_req * nq * 2))))
+    nb_min = max(1024, 1 << int(np.ceil(np.log2(per_req * nq))))  # every request of a call has its own blocks
+    nb = pool_blocks or max(nb_min, want_pool_blocks or 0)
+    mean_len = (s.len_lo + s.len_hi) / 2
+    hot, note = None, "as configured"
+    if s.resident_per_user is not None:
+        hot = candidate_hot_ids(emb, queries, k_inj + 14, users, s.n_facts, dev)
+        need_per_user = (len(hot) + s.n_users - 1) // s.n_users
+        if hot_per_user is None:
+            hot_per_user = max(s.resident_per_user, need_per_user)
+        # what fits: store (hot facts) + pool + the embeddings, with some headroom for scratch
+        emb_gib = workload.emb_bytes_scanned(s, total) / 2**30
+        avail = free_gib(dev) - headroom_gib - emb_gib
+        store_gib = lambda h: h * s.n_users * mean_len * 1.03 * s.token_bytes / 2**30  # noqa: E731
+        pool_gib = lambda n: n * s.block_size * s.token_bytes / 2**30  # noqa: E731
+        while pool_blocks is None and nb > nb_min and store_gib(hot_per_user) + pool_gib(nb) > avail:
+            nb //= 2
+            note = "pool halved to fit the free device memory"
+        while hot_per_user > need_per_user and store_gib(hot_per_user) + pool_gib(nb) > avail:
+            hot_per_user = max(need_per_user, hot_per_user // 2)
+            note = "hot subset (and pool) reduced to fit the free device memory"
     wl = workload.build(name, seed=seed, device=dev, n_query_pool=nq, num_blocks=nb, resident_ids=hot, hot_per_user=hot_per_user,
                         emb=emb, queries=queries)  # fmt: skip
     store, cache = wl.store, wl.cache
@@ -332,6 +355,13 @@ def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = Non
         torch.cuda.synchronize()
         t_r.append(ev[0].elapsed_time(ev[1]) * 1e3)
         t_i.append(ev[1].elapsed_time(ev[2]) * 1e3)
+    # the retrieval call alone, back to back (no injection between two calls)
+    ev[0].record(stream)
+    for i in range(iters):
+        retrieve()
+    ev[1].record(stream)
+    torch.cuda.synchronize()
+    r_b2b = ev[0].elapsed_time(ev[1]) * 1e3 / iters
     r_us, i_us = float(np.median(t_r)), float(np.median(t_i))
     emb_bytes = workload.emb_bytes_scanned(s, total)
     kv_bytes = workload.kv_bytes_moved(s, m_total)
@@ -339,14 +369,52 @@ def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = Non
     line = {
         "config": name, "queries_per_call": nq, "k": s.k, "k_injected": k_inj, "requests_per_call": nq,
         "facts_scanned": total, "tokens_injected": m_total, "pool_blocks": cache.num_blocks,
-        "resident_facts": int((wl.lens > 0).sum()),
-        "retrieve_us": r_us, "retrieve_emb_gbs": emb_bytes / (r_us * 1e-6) / 1e9, "retrieve_tflops": flops / (r_us * 1e-6) / 1e12,
+        "resident_facts": int((wl.lens > 0).sum()), "sizes_note": note,
+        "store_gib": float(wl.lens.sum()) * s.token_bytes / 2**30, "pool_gib": cache.num_blocks * s.block_size * s.token_bytes / 2**30,
+        "retrieve_us": r_us, "retrieve_back_to_back_us": r_b2b, "retrieve_emb_gbs": emb_bytes / (r_us * 1e-6) / 1e9,
+        "retrieve_tflops": flops / (r_us * 1e-6) / 1e12,
         "inject_us": i_us, "inject_gbs": kv_bytes / (i_us * 1e-6) / 1e9,
         "us_per_request": (r_us + i_us) / nq,
         "kernel_timeouts": store.stats()["kernel_timeouts"],
     }  # fmt: skip
     store.close()
+    del wl, cache, tables
+    torch.cuda.empty_cache()
     return line
+
+
+# the pool sizes the configurations state (blocks); others derive theirs from the requests
+CONFIGURED_POOL_BLOCKS = {"users100": 65536, "stress1m": 16384}
+
+
+def measure_all(peak_gbs: float, budget_s: float = 90.0, iters: int = 10, seed: int = 0, names=("gqa14b", "users100", "stress1m")):
+    """The batched configurations one after the other for the benchmark line: per configuration retrieve and inject
+    microseconds, the injection's rate and its fraction of ``peak_gbs``, tokens injected and the sizes used.  A
+    configuration that would start after ``budget_s`` seconds is reported as skipped."""
+    import time
+
+    out, t0 = {}, time.perf_counter()
+    for name in names:
+        if time.perf_counter() - t0 > budget_s:
+            out[name] = {"skipped": f"time budget of {budget_s:.0f} s used up by the configurations before it"}
+            continue
+        t1 = time.perf_counter()
+        try:
+            ln = measure(name, iters, seed, want_pool_blocks=CONFIGURED_POOL_BLOCKS.get(name))
+        except Exception as ex:  # a configuration that does not fit this box must not lose the whole line
+            out[name] = {"error": str(ex)[:300]}
+            torch.cuda.empty_cache()
+            continue
+        out[name] = {
+            "retrieve_us": ln["retrieve_us"], "retrieve_back_to_back_us": ln["retrieve_back_to_back_us"],
+            "retrieve_emb_gbs": ln["retrieve_emb_gbs"], "inject_us": ln["inject_us"], "inject_gbs": ln["inject_gbs"],
+            "frac_of_measured": ln["inject_gbs"] / peak_gbs, "tokens": ln["tokens_injected"], "us_per_request": ln["us_per_request"],
+            "sizes_used": {"facts": ln["facts_scanned"], "resident_facts": ln["resident_facts"], "store_gib": round(ln["store_gib"], 2),
+                           "pool_blocks": ln["pool_blocks"], "pool_gib": round(ln["pool_gib"], 2), "queries": ln["queries_per_call"],
+                           "k": ln["k"], "k_injected": ln["k_injected"], "note": ln["sizes_note"]},
+            "kernel_timeouts": ln["kernel_timeouts"], "wall_s": round(time.perf_counter() - t1, 1),
+        }  # fmt: skip
+    return out
 
 
 if __name__ == "__main__":

@@ -29,6 +29,22 @@ def test_reference_arm_prints_one_contract_line():
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["vs_baseline"] is None and "workload" in d["config"]
 
 
+def test_both_arms_name_the_workload_alike_and_traffic_comes_from_the_profile_data_file():
+    sys.path.insert(0, str(ROOT))
+    import bench
+    from paper_2607_27090_b200 import synth
+
+    r = run([sys.executable, "bench.py", "--impl", "reference", "--steps", "1", "--warmup", "0", "--k", "5"])
+    assert r.returncode == 0, r.stderr
+    d = json.loads([ln for ln in r.stdout.splitlines() if ln.startswith("{")][0])
+    shape = synth.CONFIGS["llama8b"]
+    # the CUDA arm builds its line's workload string with the same function and the same arguments (the full store)
+    assert d["config"]["workload"] == bench.workload_string("llama8b", shape, shape.n_facts, 5)
+    traffic, commit = bench.captured_traffic("llama8b", 50)
+    assert traffic and 3e8 < traffic < 7e8 and commit
+    assert bench.captured_traffic("llama8b", 7) == (None, None)
+
+
 def test_reference_arm_under_two_ranks_only_rank_zero_works():
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
            "--master-port", "29631", "bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--k", "5"]  # fmt: skip
