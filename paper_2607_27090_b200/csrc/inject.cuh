@@ -82,8 +82,10 @@ __device__ __forceinline__ void plan_prefetch(const InjectParams& p, const int r
 }
 
 // Plans request r with the THREADS threads of the calling CTA (all of them must call).  PREFETCHED: plan_prefetch has
-// been called for this request by the same threads.
-template <int THREADS, bool PREFETCHED = false>
+// been called for this request by the same threads.  PREFILLED: the caller has resolved the facts already - s_begin[j]
+// holds the LENGTH and s_src[j] the source token of entry j (placement order, entry 0 left for the prefix when there
+// is one), data errors of the lookup are in ps.status, and a block barrier separates those writes from this call.
+template <int THREADS, bool PREFETCHED = false, bool PREFILLED = false>
 __device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps,
                                              const int32_t* ids_smem = nullptr) {
   int32_t* const s_scan = ps.scan;
@@ -95,7 +97,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   const int32_t start = p.start_pos[r];  // issued first: its latency hides behind the scan
   if (tid == 0) {
     s_carry = 0;
-    s_status = 0;
+    if (!PREFILLED) s_status = 0;
   }
   // the request's block-table row goes to shared memory in one coalesced sweep: the per-token lookups below would
   // otherwise be a chain of dependent global loads
@@ -121,6 +123,11 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     if (j < has_prefix) {
       len = p.prefix_len;
       src = p.prefix_src;
+    } else if (PREFILLED) {
+      if (j < n_entries) {
+        len = s_begin[j];
+        src = s_src[j];
+      }
     } else if (j < n_entries) {
       const int jf = j - has_prefix;
       int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - jf) : jf];

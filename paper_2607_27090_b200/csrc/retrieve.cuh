@@ -768,6 +768,142 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
   write_topk<THREADS>(sm.cand, take, k, ids, out_ids, out_scores);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Selection for the fused kernels (short segments, moderate k): a threshold from the warps' own best keys instead of
+// a block-wide histogram.  The n keys sit in registers, key i with thread i mod THREADS.  Every warp pulls out the
+// VALUES of its t = ceil(k / warps) + 1 best keys (a warp-wide maximum per key: one redux instruction, no shared
+// memory, no block barrier).  The k-th largest of those warps * t values is a lower bound of the k-th largest key
+// of the whole segment (the k-th largest of a subset never exceeds the k-th largest of the set), and a tight one:
+// for rows spread evenly over the warps, about 1.1 k keys reach it.  Every key at or above the bound becomes a
+// candidate, and the candidates are ranked exactly by counting on the 64-bit keys (score, then lower row).  Three
+// block barriers; nothing depends on the distribution of the scores.  More candidates than threads (massive ties,
+// or the best rows all in a few warps) is the caller's cue to run topk_block instead.
+// ------------------------------------------------------------------------------------------------
+constexpr int kExtractMaxK = 256;   // largest k served this way
+constexpr int kExtractMaxKpl = 8;   // keys per thread held in registers
+struct ExtractShared {
+  uint32_t sub[32 * 32];               // [warp][t]: the values of the warp's t best keys (0: the warp has fewer)
+  int32_t plan_len[kExtractMaxK + 1];  // planning entries (placement order): length and source token of each
+  int32_t plan_src[kExtractMaxK + 1];
+  uint32_t bound;                      // the lower bound of the k-th largest key
+  uint32_t n_cand;
+};
+
+__host__ __device__ __forceinline__ int extract_rounds(int k, int n_warps) { return (k + n_warps - 1) / n_warps + 1; }
+
+// All THREADS threads call.  Returns true (the same in every thread) when the candidates fit one per thread: then every
+// rank < min(n, k) is held by exactly one thread, which gets it in my_rank together with the key in my_key (score key
+// in the upper half, 0xffffffff - row in the lower); the other threads get my_rank = -1.  When n < k the ranks from n
+// on have no key.  Returns false otherwise; s_keys holds the n order keys for the fallback either way.
+// `cand` is shared memory for THREADS 64-bit keys.
+template <int THREADS, int KPL>
+__device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long long* cand, const float* __restrict__ sc, uint32_t* s_keys,
+                                             int n, int k, int& my_rank, unsigned long long& my_key) {
+  constexpr int NW = THREADS / 32;
+  constexpr unsigned kFull = 0xffffffffu;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t = extract_rounds(k, NW);
+  uint32_t key[KPL], live[KPL];
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) {
+    const int i = j * THREADS + tid;
+    key[j] = i < n ? order_key(__ldcg(sc + i)) : 0u;  // 0 marks an empty place (no finite score has key 0)
+    live[j] = key[j];
+  }
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) {
+    const int i = j * THREADS + tid;
+    if (i < n) s_keys[i] = key[j];
+  }
+  if (tid == 0) {
+    es.bound = 0u;
+    es.n_cand = 0u;
+  }
+  // the values of this warp's t best keys: lane r ends up with the r-th
+  uint32_t mine = 0u;
+  for (int r = 0; r < t; ++r) {
+    uint32_t hb = live[0];
+#pragma unroll
+    for (int j = 1; j < KPL; ++j) hb = max(hb, live[j]);
+    const uint32_t wmax = __reduce_max_sync(kFull, hb);
+    if (wmax == 0u) break;  // the warp has nothing left (uniform)
+    // one holder of that value gives it up: the lowest lane, its first place
+    const unsigned holders = __ballot_sync(kFull, hb == wmax);
+    if (lane == __ffs(holders) - 1) {
+      bool gone = false;
+#pragma unroll
+      for (int j = 0; j < KPL; ++j)
+        if (!gone && live[j] == wmax) {
+          live[j] = 0u;
+          gone = true;
+        }
+    }
+    if (lane == r) mine = wmax;
+  }
+  if (lane < t) es.sub[warp * t + lane] = mine;
+  __syncwarp();
+  __syncthreads();
+
+  // the k-th largest of the warps' values (rank by counting; equal values are told apart by their place)
+  const int S = NW * t;
+  if (tid < S) {
+    const uint32_t v = es.sub[tid];
+    uint32_t rank = 0;
+    for (int j = 0; j < S; ++j) {
+      const uint32_t o = es.sub[j];
+      rank += (o > v) || (o == v && j < tid);
+    }
+    if (rank == (uint32_t)k - 1u) es.bound = v;  // 0 when fewer than k values exist: then every key is a candidate
+  }
+  __syncwarp();
+  __syncthreads();
+
+  // candidates: every key at or above the bound, as 64-bit keys (score key, then lower row first)
+  const uint32_t bound = es.bound;
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) {
+    const bool in = key[j] != 0u && key[j] >= bound;
+    const unsigned votes = __ballot_sync(kFull, in);
+    if (votes) {
+      uint32_t base = 0;
+      if (lane == 0) base = atomicAdd(&es.n_cand, (uint32_t)__popc(votes));
+      base = __shfl_sync(kFull, base, 0);
+      const uint32_t slot = base + (uint32_t)__popc(votes & ((1u << lane) - 1u));
+      if (in && slot < (uint32_t)THREADS)
+        cand[slot] = ((unsigned long long)key[j] << 32) | (uint32_t)(0xffffffffu - (uint32_t)(j * THREADS + tid));
+    }
+  }
+  __syncwarp();
+  __syncthreads();
+  const uint32_t C = es.n_cand;
+  my_rank = -1;
+  my_key = 0ull;
+  if (C > (uint32_t)THREADS) return false;
+  if (C * 4u <= (uint32_t)THREADS) {
+    // four lanes share a candidate and split the comparisons
+    const uint32_t ci = (uint32_t)tid >> 2, part = (uint32_t)tid & 3u;
+    const unsigned long long me = ci < C ? cand[ci] : 0ull;
+    uint32_t rank = 0;
+    for (uint32_t jj = part; jj < C; jj += 4) rank += cand[jj] > me;
+    rank += __shfl_xor_sync(kFull, rank, 1);
+    rank += __shfl_xor_sync(kFull, rank, 2);
+    if (ci < C && part == 0 && rank < (uint32_t)k) {
+      my_rank = (int)rank;
+      my_key = me;
+    }
+  } else if (tid < (int)C) {
+    const unsigned long long me = cand[tid];
+    uint32_t rank = 0;
+    for (uint32_t jj = 0; jj < C; ++jj) rank += cand[jj] > me;
+    if (rank < (uint32_t)k) {
+      my_rank = (int)rank;
+      my_key = me;
+    }
+  }
+  __syncwarp();
+  return true;
+}
+
 // Scoring only (large segments): grid = (row groups, nq); dynamic shared memory holds the query as fp32.
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads) score_rows_kernel(const RetrieveParams p, int rows_per_cta) {
@@ -802,6 +938,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
                                                 int n_host, const InjectParams* ip) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
+  __shared__ ExtractShared es;
   __shared__ PlanShared ps;
   __shared__ int32_t s_ids[PLAN ? kTopkMaxK : 1];  // the selected ids by rank, for the planning that follows in this CTA
   __shared__ int s_last;
@@ -827,20 +964,68 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   __threadfence();
   if (PLAN) plan_prefetch<THREADS>(*ip, q, ps);  // in flight while the ids are being selected
   const float* sc = p.scores + (int64_t)q * p.score_stride;
-  uint32_t lo = 0xffffffffu, hi = 0u;
-  for (int i = threadIdx.x; i < n; i += THREADS) {
-    const uint32_t kx = order_key(__ldcg(sc + i));
-    s_keys[i] = kx;
-    lo = min(lo, kx);
-    hi = max(hi, kx);
+  // with a single user segment facts are numbered in row order: the row is the fact id
+  const int32_t* row_ids = p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity;
+  int32_t* out_ids = p.out_ids + (int64_t)q * p.k;
+  float* out_scores = p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr;
+  const int k = p.k;
+
+  // ---- fast selection: a threshold from the warps' own best keys (see topk_extract) -------------------------
+  bool done = false;
+  const bool plan_fast = PLAN && k + (ip->prefix_len > 0 ? 1 : 0) <= kExtractMaxK + 1;
+  if (k <= kExtractMaxK && n <= THREADS * kExtractMaxKpl && extract_rounds(k, THREADS / 32) <= 32 && (!PLAN || plan_fast)) {
+    const int has_prefix = PLAN ? (ip->prefix_len > 0) : 0;
+    if (PLAN) {
+      // planning entries default to "nothing" (ranks beyond the segment); a fact's entry is filled in the moment
+      // its rank is known, so the fact-table reads overlap one another and nothing waits for the id list
+      for (int j = threadIdx.x; j < k + has_prefix; j += THREADS) {
+        es.plan_len[j] = 0;
+        es.plan_src[j] = 0;
+      }
+      if (threadIdx.x == 0) ps.status = 0;
+    }
+    auto emit = [&](int rank, uint32_t row, uint32_t score_key) {
+      const int32_t id = row_ids ? row_ids[row] : (int32_t)row;
+      out_ids[rank] = id;
+      if (out_scores) out_scores[rank] = key_score(score_key);
+      if (PLAN) {
+        const int j = has_prefix + ((ip->flags & 1u) ? (k - 1 - rank) : rank);
+        const FactRec f = ip->facts[id];
+        if (!f.resident) {
+          atomicOr(&ps.status, 2 /*MS_REQ_NOT_RESIDENT*/);
+        } else {
+          es.plan_len[j] = f.n_tokens;
+          es.plan_src[j] = f.resident == 2 ? (f.tok_off | kHostTierBit) : f.tok_off;
+        }
+      }
+    };
+    auto pad = [&](int rank) {
+      out_ids[rank] = -1;
+      if (out_scores) out_scores[rank] = 0.f;
+    };
+    int my_rank = -1;
+    unsigned long long my_key = 0ull;
+    if (n <= THREADS) done = topk_extract<THREADS, 1>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
+    else if (n <= 2 * THREADS) done = topk_extract<THREADS, 2>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
+    else if (n <= 4 * THREADS) done = topk_extract<THREADS, 4>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
+    else done = topk_extract<THREADS, 8>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
+    if (done) {
+      if (my_rank >= 0) emit(my_rank, 0xffffffffu - (uint32_t)my_key, (uint32_t)(my_key >> 32));
+      for (int r = n + (int)threadIdx.x; r < k; r += THREADS) pad(r);  // a segment shorter than k: the other ranks are empty
+      if (PLAN) {
+        __syncwarp();  // only some lanes resolved a fact: together again before the barrier
+        __syncthreads();
+        plan_request<THREADS, true, true>(*ip, q, es.plan_len, es.plan_src, ps, nullptr);
+      }
+      return;
+    }
+  } else {
+    for (int i = threadIdx.x; i < n; i += THREADS) s_keys[i] = order_key(__ldcg(sc + i));
   }
   __syncthreads();
-  // with a single user segment facts are numbered in row order: the row is the fact id
-  topk_block<THREADS, false>(sm, sc, s_keys, n, p.k,
-                            IdMap{nullptr, p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity,
-                                  PLAN ? s_ids : nullptr},
-                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo,
-                            hi);
+
+  // ---- general selection (large k, long segments, or the extraction's check failed) -------------------------
+  topk_block<THREADS, false>(sm, sc, s_keys, n, k, IdMap{nullptr, row_ids, PLAN ? s_ids : nullptr}, out_ids, out_scores);
   if (PLAN) {
     // the ids of query q are request q's fact list: plan it right here (steps I1-I3), in the shared memory the
     // selection no longer needs, so that the copy kernel can follow without a separate planning launch

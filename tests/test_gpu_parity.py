@@ -399,21 +399,27 @@ def test_inject_empty_and_degenerate_requests():
     assert untouched_mask_ok(cache, np.array([], np.int64), SENT)
 
 
-@pytest.mark.parametrize("n_users,nq", [(1, 1), (1, 5), (3, 7)])
-def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq):
-    """memstore_retrieve_inject (requests planned inside the retrieval kernel) against retrieve followed by inject."""
-    hs = HostStore(40, 90, 2, 8, 128, 8, 40, 256, "float16", n_users=n_users)
+@pytest.mark.parametrize("n_users,nq,n_facts,k", [(1, 1, 90, 6), (1, 5, 90, 6), (3, 7, 90, 6), (1, 1, 2000, 50), (1, 3, 2500, 100), (4, 9, 500, 20),
+                                                   (1, 2, 1100, 256), (1, 1, 40, 300)])  # fmt: skip
+def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq, n_facts, k):
+    """memstore_retrieve_inject (requests planned inside the retrieval kernel) against retrieve followed by inject, on
+    segments that take one, two and four keys per thread of the selecting CTA, with small and large k, and with k larger
+    than the segment."""
+    hs = HostStore(40, n_facts, 2, 2 if n_facts > 100 else 8, 128, 1 if n_facts > 100 else 8, 3 if n_facts > 100 else 40, 256, "float16",
+                   n_users=n_users)  # fmt: skip
     ms = hs.to_memstore(5e5)
-    bs, nb, k = 16, 256, 6
+    bs, nb = 16, 256
     q = to_dev(synth.queries(41, nq, 256, "float16"))
     users = to_dev((np.arange(nq) % n_users).astype(np.int32)) if n_users > 1 else None
     starts = to_dev((np.arange(nq) * 5 + 3).astype(np.int32))
-    tables = to_dev(synth.block_tables(42, nb, (3 + 5 * nq + k * 40) // bs + 1, nq))
+    per_req = (3 + 5 * nq + k * int(hs.lens.max())) // bs + 1
+    nb = max(nb, per_req * nq)
+    tables = to_dev(synth.block_tables(42, nb, per_req, nq))
     ca, cb = make_cache(hs, nb, bs), make_cache(hs, nb, bs)
     for rep in range(2):  # the second round runs with the scratch already sized: the fused kernel path
         ids_a, sc_a = ms.retrieve(q, k, query_users=users)
         n_a, st_a = ms.inject(ids_a, starts, tables, ca, flags=M.INJECT_REVERSE)
-        sm = torch.full((nq, 300), -3, dtype=torch.int64, device=DEV)
+        sm = torch.full((nq, 1000), -3, dtype=torch.int64, device=DEV)
         sc_b = torch.empty((nq, k), dtype=torch.float32, device=DEV)
         ids_b, n_b, st_b = ms.retrieve_inject(q, k, starts, tables, cb, query_users=users, out_scores=sc_b, out_slot_mapping=sm,
                                               flags=M.INJECT_REVERSE)
@@ -421,6 +427,12 @@ def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq):
         assert torch.equal(ids_a, ids_b) and torch.equal(sc_a, sc_b) and torch.equal(n_a, n_b) and torch.equal(st_a, st_b)
         assert int(st_b.abs().sum()) == 0 and bool((sm[:, 0] >= 0).all())
         assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+        ids_np, lens = ids_b.cpu().numpy(), hs.lens
+        assert n_b.cpu().tolist() == [int(lens[r[r >= 0]].sum()) for r in ids_np]
+        for i in sorted({0, nq - 1}):
+            u = i % n_users
+            rows = np.arange(u * n_facts, (u + 1) * n_facts)
+            check_ids(ids_np[i], sc_b[i].cpu().numpy(), hs.emb[rows], q[i].cpu().numpy(), k, row_ids=rows.astype(np.int32) if n_users > 1 else None)
     ms.close()
 
 
