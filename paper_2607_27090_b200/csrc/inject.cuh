@@ -117,9 +117,10 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   const int32_t* ids = ids_smem ? ids_smem : p.fact_ids + (int64_t)r * p.k;
   const int has_prefix = p.prefix_len > 0;
   const int n_entries = p.k + has_prefix;
-  for (int base = 0; base < n_entries; base += THREADS) {
-    int j = base + tid;
-    int32_t len = 0, src = 0;
+  // length and source token of entry j of the placement list (nothing for an absent, unknown or non-resident fact)
+  auto entry = [&](int j, int32_t& len, int32_t& src) {
+    len = 0;
+    src = 0;
     if (j < has_prefix) {
       len = p.prefix_len;
       src = p.prefix_src;
@@ -130,12 +131,12 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       }
     } else if (j < n_entries) {
       const int jf = j - has_prefix;
-      int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - jf) : jf];
+      const int32_t id = ids[(p.flags & 1u) ? (p.k - 1 - jf) : jf];
       if (id >= 0) {
         if (id >= p.n_facts) {
           atomicOr(&s_status, 1 /*MS_REQ_BAD_FACT_ID*/);
         } else {
-          FactRec f = p.facts[id];
+          const FactRec f = p.facts[id];
           if (!f.resident) {
             atomicOr(&s_status, 2 /*MS_REQ_NOT_RESIDENT*/);
           } else {
@@ -145,27 +146,65 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
         }
       }
     }
-    // block-wide exclusive scan of len
+  };
+  int32_t m;
+  if (n_entries <= THREADS) {
+    // at most one entry per thread: one barrier, then every warp combines the warps' totals by a shuffle scan
+    const int j = tid;
+    int32_t len, src;
+    entry(j, len, src);
     int32_t x = len;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      const int32_t y = __shfl_up_sync(0xffffffffu, x, o);
       if (lane >= o) x += y;
     }
     if (lane == 31) s_scan[warp] = x;
+    __syncwarp();
     __syncthreads();
-    int32_t warp_off = 0;
-    for (int w = 0; w < warp; ++w) warp_off += s_scan[w];
-    int32_t carry = s_carry;
+    int32_t tot = lane < THREADS / 32 ? s_scan[lane] : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int32_t y = __shfl_up_sync(0xffffffffu, tot, o);
+      if (lane >= o) tot += y;
+    }
+    const int32_t below = __shfl_sync(0xffffffffu, tot, warp > 0 ? warp - 1 : 0);
+    m = __shfl_sync(0xffffffffu, tot, 31);
     if (j < n_entries) {
-      s_begin[j] = carry + warp_off + x - len;
+      s_begin[j] = (warp > 0 ? below : 0) + x - len;
       s_src[j] = src;
     }
+    __syncwarp();
     __syncthreads();
-    if (tid == THREADS - 1) s_carry = carry + warp_off + x;
-    __syncthreads();
+  } else {
+    // longer lists: chunks of THREADS entries with a running carry
+    for (int base = 0; base < n_entries; base += THREADS) {
+      const int j = base + tid;
+      int32_t len, src;
+      entry(j, len, src);
+      int32_t x = len;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+      }
+      if (lane == 31) s_scan[warp] = x;
+      __syncwarp();
+      __syncthreads();
+      int32_t warp_off = 0;
+      for (int w = 0; w < warp; ++w) warp_off += s_scan[w];
+      const int32_t carry = s_carry;
+      if (j < n_entries) {
+        s_begin[j] = carry + warp_off + x - len;
+        s_src[j] = src;
+      }
+      __syncthreads();
+      if (tid == THREADS - 1) s_carry = carry + warp_off + x;
+      __syncwarp();
+      __syncthreads();
+    }
+    m = s_carry;
   }
-  const int32_t m = s_carry;
   // A start position that is negative, or at or beyond the position bound, places no token at all: no tile is made
   // (the divisions and the block-table lookups below assume 0 <= pos), the request gets a status bit, and the slot
   // mapping lists every composed token as skipped.
@@ -185,7 +224,78 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   }
 
   const int bs = p.block_size;
-  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += THREADS) {
+  // A block size that is a multiple of the tile keeps a tile inside one cache block (tiles start at multiples of 8):
+  // then one thread plans a whole tile - one block lookup, one search for the fact that owns the tile's first token,
+  // a walk along the facts for the other seven, and the descriptor written with 16-byte stores.
+  const bool tile_in_block = (bs % kTileTokens) == 0;
+  for (uint32_t t = tid; tile_in_block && t < n_tiles; t += THREADS) {
+    const int32_t pos0 = first_tile_pos + (int32_t)(t * kTileTokens);
+    int32_t src_tok[kTileTokens];
+    int64_t dst[kTileTokens];
+#pragma unroll
+    for (int ln = 0; ln < kTileTokens; ++ln) {
+      src_tok[ln] = -1;
+      dst[ln] = 0;
+    }
+    const int32_t q_lo = max(pos0 - start, 0), q_hi = min(pos0 + kTileTokens - start, m);  // composed tokens of this tile
+    if (q_lo < q_hi) {
+      const int32_t bi = pos0 / bs;
+      const int32_t in0 = pos0 - bi * bs;
+      int32_t blk = -1;
+      if (bi < p.max_blocks) blk = bi < n_cached ? ps.table[bi] : table_row[bi];
+      const bool blk_ok = blk >= 0 && blk < p.num_blocks;
+      const int64_t dst0 = (int64_t)blk * p.block_stride + (int64_t)in0 * p.token_stride;
+      // the fact that owns composed token q is the LAST i with b_i <= q (see the per-token loop below)
+      int lo = 0, hi = n_entries - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_begin[mid] <= q_lo) lo = mid; else hi = mid - 1;
+      }
+      int i = lo;
+      int32_t b_i = s_begin[i], src_i = s_src[i];
+      int32_t b_next = i + 1 < n_entries ? s_begin[i + 1] : 0x7fffffff;
+      int32_t st = 0;
+#pragma unroll
+      for (int ln = 0; ln < kTileTokens; ++ln) {
+        const int32_t pos = pos0 + ln;
+        const int32_t q = pos - start;
+        if (q >= q_lo && q < q_hi) {
+          while (b_next <= q) {  // next placed fact (entries of length zero are stepped over)
+            ++i;
+            b_i = b_next;
+            src_i = s_src[i];
+            b_next = i + 1 < n_entries ? s_begin[i + 1] : 0x7fffffff;
+          }
+          int64_t slot = -1;
+          if (pos >= p.max_position) {
+            st |= 16;  // MS_REQ_POSITION_OVERFLOW
+          } else if (bi >= p.max_blocks) {
+            st |= 4;  // MS_REQ_BLOCK_TABLE_SHORT
+          } else if (!blk_ok) {
+            st |= 8;  // MS_REQ_BAD_BLOCK_ID
+          } else {
+            src_tok[ln] = src_i + (q - b_i);
+            dst[ln] = dst0 + (int64_t)ln * p.token_stride;
+            slot = (int64_t)blk * bs + in0 + ln;
+          }
+          if (p.out_slot_mapping && q < p.slot_stride) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = slot;
+        }
+      }
+      if (st) atomicOr(&s_status, st);
+    }
+    if (tile_base + t < p.tiles_capacity) {
+      TileDesc* d = p.tiles + tile_base + t;
+      *reinterpret_cast<int4*>(d) = make_int4(pos0, 0, 0, 0);
+      int4* ds = reinterpret_cast<int4*>(d->src_tok);
+      ds[0] = make_int4(src_tok[0], src_tok[1], src_tok[2], src_tok[3]);
+      ds[1] = make_int4(src_tok[4], src_tok[5], src_tok[6], src_tok[7]);
+      longlong2* dd = reinterpret_cast<longlong2*>(d->dst_off);
+#pragma unroll
+      for (int h = 0; h < kTileTokens / 2; ++h) dd[h] = make_longlong2(dst[2 * h], dst[2 * h + 1]);
+    }
+  }
+  // any other block size: one thread per token
+  for (uint32_t e = tid; !tile_in_block && e < n_tiles * kTileTokens; e += THREADS) {
     const uint32_t t = e / kTileTokens, ln = e % kTileTokens;
     const int32_t pos = first_tile_pos + (int32_t)e;
     const int32_t q = pos - start;  // index in the composed segment
@@ -228,6 +338,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       d->dst_off[ln] = dst;
     }
   }
+  __syncwarp();
   __syncthreads();
   if (tid == 0) {
     if (p.out_n_tokens) p.out_n_tokens[r] = m;

@@ -803,12 +803,11 @@ __device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long lo
   constexpr unsigned kFull = 0xffffffffu;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t = extract_rounds(k, NW);
-  uint32_t key[KPL], live[KPL];
+  uint32_t key[KPL];
 #pragma unroll
   for (int j = 0; j < KPL; ++j) {
     const int i = j * THREADS + tid;
     key[j] = i < n ? order_key(__ldcg(sc + i)) : 0u;  // 0 marks an empty place (no finite score has key 0)
-    live[j] = key[j];
   }
 #pragma unroll
   for (int j = 0; j < KPL; ++j) {
@@ -819,41 +818,37 @@ __device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long lo
     es.bound = 0u;
     es.n_cand = 0u;
   }
-  // the values of this warp's t best keys: lane r ends up with the r-th
-  uint32_t mine = 0u;
+  // the t largest DISTINCT values of this warp, largest first: lane r ends up with the r-th.  (Equal keys count once
+  // here; a bound taken from distinct values, each held by at least one key, is still a lower bound.)
+  uint32_t mine = 0u, prev = 0xffffffffu;
   for (int r = 0; r < t; ++r) {
-    uint32_t hb = live[0];
+    uint32_t hb = 0u;
 #pragma unroll
-    for (int j = 1; j < KPL; ++j) hb = max(hb, live[j]);
-    const uint32_t wmax = __reduce_max_sync(kFull, hb);
-    if (wmax == 0u) break;  // the warp has nothing left (uniform)
-    // one holder of that value gives it up: the lowest lane, its first place
-    const unsigned holders = __ballot_sync(kFull, hb == wmax);
-    if (lane == __ffs(holders) - 1) {
-      bool gone = false;
-#pragma unroll
-      for (int j = 0; j < KPL; ++j)
-        if (!gone && live[j] == wmax) {
-          live[j] = 0u;
-          gone = true;
-        }
-    }
-    if (lane == r) mine = wmax;
+    for (int j = 0; j < KPL; ++j) hb = max(hb, key[j] < prev ? key[j] : 0u);
+    prev = __reduce_max_sync(kFull, hb);
+    if (prev == 0u) break;  // the warp has no smaller value left (uniform)
+    if (lane == r) mine = prev;
   }
   if (lane < t) es.sub[warp * t + lane] = mine;
   __syncwarp();
   __syncthreads();
 
-  // the k-th largest of the warps' values (rank by counting; equal values are told apart by their place)
+  // the k-th largest of the warps' values: rank by counting, G lanes per value (equal values of different warps are
+  // told apart by their place, so ranks are distinct)
   const int S = NW * t;
-  if (tid < S) {
-    const uint32_t v = es.sub[tid];
+  int g_shift = 3;
+  while (g_shift > 0 && (S << g_shift) > THREADS) --g_shift;
+  {
+    const int vi = tid >> g_shift, part = tid & ((1 << g_shift) - 1);
+    const uint32_t v = vi < S ? es.sub[vi] : 0u;
     uint32_t rank = 0;
-    for (int j = 0; j < S; ++j) {
-      const uint32_t o = es.sub[j];
-      rank += (o > v) || (o == v && j < tid);
-    }
-    if (rank == (uint32_t)k - 1u) es.bound = v;  // 0 when fewer than k values exist: then every key is a candidate
+    if (vi < S)
+      for (int j = part; j < S; j += 1 << g_shift) {
+        const uint32_t o = es.sub[j];
+        rank += (o > v) || (o == v && j < vi);
+      }
+    for (int o = 1; o < (1 << g_shift); o <<= 1) rank += __shfl_xor_sync(kFull, rank, o);
+    if (vi < S && part == 0 && rank == (uint32_t)k - 1u) es.bound = v;  // stays 0 when fewer than k values exist: every key is a candidate
   }
   __syncwarp();
   __syncthreads();
