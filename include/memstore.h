@@ -75,8 +75,15 @@ enum { MS_ROPE_HALF_SPLIT = 0, MS_ROPE_INTERLEAVED = 1 };
 enum {
   MS_INJECT_REVERSE = 1u, /* place ids[k-1] first, so that ids[0] ends next to the query */
   MS_INJECT_PREFIX = 2u,  /* place the store's instruction prefix (memstore_set_prefix) before the facts */
-  MS_RETRIEVE_ANN = 4u    /* memstore_retrieve_inject / memstore_serve_host only: retrieve through the graph index
+  MS_RETRIEVE_ANN = 4u,   /* memstore_retrieve_inject / memstore_serve_host only: retrieve through the graph index
                              (memstore_retrieve_ann with its default parameters) instead of the exact scan */
+  MS_INPUTS_STABLE = 8u   /* memstore_retrieve_inject only: the caller vouches that queries, query_users, start_pos and
+                             block_tables were completely written before the work that precedes this call in the stream
+                             began (a serving loop whose next query is ready before the previous injection is enqueued).
+                             The scoring and selection of this call may then overlap the tail of the preceding kernel -
+                             typically the previous request's copy kernel, whose draining SMs they use; ids, plan and
+                             cache are still written strictly after it.  Without the flag the call orders itself after
+                             all preceding work, as any launch does.  Results are the same either way. */
 };
 /* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
  * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */

@@ -224,78 +224,8 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   }
 
   const int bs = p.block_size;
-  // A block size that is a multiple of the tile keeps a tile inside one cache block (tiles start at multiples of 8):
-  // then one thread plans a whole tile - one block lookup, one search for the fact that owns the tile's first token,
-  // a walk along the facts for the other seven, and the descriptor written with 16-byte stores.
-  const bool tile_in_block = (bs % kTileTokens) == 0;
-  for (uint32_t t = tid; tile_in_block && t < n_tiles; t += THREADS) {
-    const int32_t pos0 = first_tile_pos + (int32_t)(t * kTileTokens);
-    int32_t src_tok[kTileTokens];
-    int64_t dst[kTileTokens];
-#pragma unroll
-    for (int ln = 0; ln < kTileTokens; ++ln) {
-      src_tok[ln] = -1;
-      dst[ln] = 0;
-    }
-    const int32_t q_lo = max(pos0 - start, 0), q_hi = min(pos0 + kTileTokens - start, m);  // composed tokens of this tile
-    if (q_lo < q_hi) {
-      const int32_t bi = pos0 / bs;
-      const int32_t in0 = pos0 - bi * bs;
-      int32_t blk = -1;
-      if (bi < p.max_blocks) blk = bi < n_cached ? ps.table[bi] : table_row[bi];
-      const bool blk_ok = blk >= 0 && blk < p.num_blocks;
-      const int64_t dst0 = (int64_t)blk * p.block_stride + (int64_t)in0 * p.token_stride;
-      // the fact that owns composed token q is the LAST i with b_i <= q (see the per-token loop below)
-      int lo = 0, hi = n_entries - 1;
-      while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (s_begin[mid] <= q_lo) lo = mid; else hi = mid - 1;
-      }
-      int i = lo;
-      int32_t b_i = s_begin[i], src_i = s_src[i];
-      int32_t b_next = i + 1 < n_entries ? s_begin[i + 1] : 0x7fffffff;
-      int32_t st = 0;
-#pragma unroll
-      for (int ln = 0; ln < kTileTokens; ++ln) {
-        const int32_t pos = pos0 + ln;
-        const int32_t q = pos - start;
-        if (q >= q_lo && q < q_hi) {
-          while (b_next <= q) {  // next placed fact (entries of length zero are stepped over)
-            ++i;
-            b_i = b_next;
-            src_i = s_src[i];
-            b_next = i + 1 < n_entries ? s_begin[i + 1] : 0x7fffffff;
-          }
-          int64_t slot = -1;
-          if (pos >= p.max_position) {
-            st |= 16;  // MS_REQ_POSITION_OVERFLOW
-          } else if (bi >= p.max_blocks) {
-            st |= 4;  // MS_REQ_BLOCK_TABLE_SHORT
-          } else if (!blk_ok) {
-            st |= 8;  // MS_REQ_BAD_BLOCK_ID
-          } else {
-            src_tok[ln] = src_i + (q - b_i);
-            dst[ln] = dst0 + (int64_t)ln * p.token_stride;
-            slot = (int64_t)blk * bs + in0 + ln;
-          }
-          if (p.out_slot_mapping && q < p.slot_stride) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = slot;
-        }
-      }
-      if (st) atomicOr(&s_status, st);
-    }
-    if (tile_base + t < p.tiles_capacity) {
-      TileDesc* d = p.tiles + tile_base + t;
-      *reinterpret_cast<int4*>(d) = make_int4(pos0, 0, 0, 0);
-      int4* ds = reinterpret_cast<int4*>(d->src_tok);
-      ds[0] = make_int4(src_tok[0], src_tok[1], src_tok[2], src_tok[3]);
-      ds[1] = make_int4(src_tok[4], src_tok[5], src_tok[6], src_tok[7]);
-      longlong2* dd = reinterpret_cast<longlong2*>(d->dst_off);
-#pragma unroll
-      for (int h = 0; h < kTileTokens / 2; ++h) dd[h] = make_longlong2(dst[2 * h], dst[2 * h + 1]);
-    }
-  }
-  // any other block size: one thread per token
-  for (uint32_t e = tid; !tile_in_block && e < n_tiles * kTileTokens; e += THREADS) {
+  const int bs_shift = (bs & (bs - 1)) == 0 ? 31 - __clz(bs) : -1;  // block sizes are powers of two in practice
+  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += THREADS) {
     const uint32_t t = e / kTileTokens, ln = e % kTileTokens;
     const int32_t pos = first_tile_pos + (int32_t)e;
     const int32_t q = pos - start;  // index in the composed segment
@@ -314,7 +244,8 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       if (pos >= p.max_position) {
         st = 16;  // MS_REQ_POSITION_OVERFLOW
       } else {
-        int32_t bi = pos / bs;
+        const int32_t bi = bs_shift >= 0 ? pos >> bs_shift : pos / bs;
+        const int32_t in_block = bs_shift >= 0 ? (pos & (bs - 1)) : pos - bi * bs;
         if (bi >= p.max_blocks) {
           st = 4;  // MS_REQ_BLOCK_TABLE_SHORT
         } else {
@@ -323,8 +254,8 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
             st = 8;  // MS_REQ_BAD_BLOCK_ID
           } else {
             src_tok = s_src[i] + (q - s_begin[i]);
-            dst = (int64_t)blk * p.block_stride + (int64_t)(pos % bs) * p.token_stride;
-            slot = (int64_t)blk * bs + pos % bs;
+            dst = (int64_t)blk * p.block_stride + (int64_t)in_block * p.token_stride;
+            slot = (int64_t)blk * bs + in_block;
           }
         }
       }

@@ -268,7 +268,7 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
 // CTA of a query selects and plans alone, which wants many threads), 256-thread CTAs otherwise.
 template <typename T, int THREADS, bool PLAN>
 void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,
-                               const InjectParams* ip, size_t smem, cudaStream_t st) {
+                               const InjectParams* ip, size_t smem, cudaStream_t st, int early) {
   // enough CTAs to fill the GPU, at least one row per warp
   constexpr int64_t kWarps = THREADS / 32;
   // (a 1024-thread CTA fills an SM: more CTAs than SMs would only queue behind the first wave)
@@ -292,17 +292,17 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
     lc.stream = st;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    cudaLaunchKernelEx(&lc, score_topk_plan_kernel<T, THREADS>, p, rows_per_cta, tickets, keys_cap, n_host, *ip);
+    cudaLaunchKernelEx(&lc, score_topk_plan_kernel<T, THREADS>, p, rows_per_cta, tickets, keys_cap, n_host, *ip, early);
   } else
     score_topk_fused_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host);
 }
 template <typename T, bool PLAN>
 void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,
-                       const InjectParams* ip, size_t smem, cudaStream_t st) {
+                       const InjectParams* ip, size_t smem, cudaStream_t st, int early = 0) {
   if (nq <= kFusedFewQueries)
-    launch_score_topk_threads<T, kFusedThreadsFew, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st);
+    launch_score_topk_threads<T, kFusedThreadsFew, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
   else
-    launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st);
+    launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -1249,6 +1249,10 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   if (nq == 0) return MS_OK;
   if (!queries || !out_ids) return fail(s, MS_ERR_INVALID_ARG, "null queries or out_ids");
   if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
+  // MS_INPUTS_STABLE only matters to the one-launch retrieval + planning kernel below; every other route orders itself
+  // after the preceding work of the stream as an ordinary launch does
+  const int early = (flags & MS_INPUTS_STABLE) ? 1 : 0;
+  flags &= ~(uint32_t)MS_INPUTS_STABLE;
   if (flags & MS_RETRIEVE_ANN) {
     if (query_users) return fail(s, MS_ERR_INVALID_ARG, "MS_RETRIEVE_ANN serves single-segment stores: query_users must be NULL");
     ms_status rc = memstore_retrieve_ann(s, queries, nq, k, nullptr, out_ids, out_scores, nullptr, stream);
@@ -1294,9 +1298,9 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   const int n_host = query_users ? -1 : (int)n_max;
   MS_CUDA(s, ensure_fused_smem(c.device, smem));
   if (c.emb_dtype == MS_DTYPE_F16)
-    launch_score_topk<__half, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st);
+    launch_score_topk<__half, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st, early);
   else
-    launch_score_topk<float, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st);
+    launch_score_topk<float, true>(s->sm_count, nq, n_max, p, s->tickets, keys_cap, n_host, &ip, smem, st, early);
   MS_CUDA(s, cudaGetLastError());
   s->kernels_launched++;
   s->retrieve_calls++;

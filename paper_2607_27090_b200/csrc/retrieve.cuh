@@ -928,9 +928,12 @@ __global__ void __launch_bounds__(kTopkThreads, 1) topk_kernel(const RetrievePar
 }
 
 // Body of the fused scoring + top-k kernels below (PLAN: the last CTA of a query also plans its injection).
+// early (PLAN only): the kernel was launched as a programmatic dependent and has NOT yet waited for the preceding grid;
+// everything up to the selection reads only the store and the caller's inputs and writes only this library's scratch,
+// and the wait comes right before the first write that a preceding kernel could still be concerned with.
 template <typename T, int THREADS, bool PLAN>
 __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int rows_per_cta, uint32_t* tickets, int keys_capacity,
-                                                int n_host, const InjectParams* ip) {
+                                                int n_host, const InjectParams* ip, bool early = false) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ ExtractShared es;
@@ -979,21 +982,6 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
       }
       if (threadIdx.x == 0) ps.status = 0;
     }
-    auto emit = [&](int rank, uint32_t row, uint32_t score_key) {
-      const int32_t id = row_ids ? row_ids[row] : (int32_t)row;
-      out_ids[rank] = id;
-      if (out_scores) out_scores[rank] = key_score(score_key);
-      if (PLAN) {
-        const int j = has_prefix + ((ip->flags & 1u) ? (k - 1 - rank) : rank);
-        const FactRec f = ip->facts[id];
-        if (!f.resident) {
-          atomicOr(&ps.status, 2 /*MS_REQ_NOT_RESIDENT*/);
-        } else {
-          es.plan_len[j] = f.n_tokens;
-          es.plan_src[j] = f.resident == 2 ? (f.tok_off | kHostTierBit) : f.tok_off;
-        }
-      }
-    };
     auto pad = [&](int rank) {
       out_ids[rank] = -1;
       if (out_scores) out_scores[rank] = 0.f;
@@ -1005,7 +993,28 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     else if (n <= 4 * THREADS) done = topk_extract<THREADS, 4>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
     else done = topk_extract<THREADS, 8>(es, sm.cand, sc, s_keys, n, k, my_rank, my_key);
     if (done) {
-      if (my_rank >= 0) emit(my_rank, 0xffffffffu - (uint32_t)my_key, (uint32_t)(my_key >> 32));
+      // the thread that holds a rank resolves the fact (store data only) ...
+      int32_t id = -1;
+      if (my_rank >= 0) {
+        const uint32_t row = 0xffffffffu - (uint32_t)my_key;
+        id = row_ids ? row_ids[row] : (int32_t)row;
+        if (PLAN) {
+          const int j = has_prefix + ((ip->flags & 1u) ? (k - 1 - my_rank) : my_rank);
+          const FactRec f = ip->facts[id];
+          if (!f.resident) {
+            atomicOr(&ps.status, 2 /*MS_REQ_NOT_RESIDENT*/);
+          } else {
+            es.plan_len[j] = f.n_tokens;
+            es.plan_src[j] = f.resident == 2 ? (f.tok_off | kHostTierBit) : f.tok_off;
+          }
+        }
+      }
+      // ... and only then come the first writes outside this library's scratch
+      if (PLAN && early) grid_dependency_wait();
+      if (my_rank >= 0) {
+        out_ids[my_rank] = id;
+        if (out_scores) out_scores[my_rank] = key_score((uint32_t)(my_key >> 32));
+      }
       for (int r = n + (int)threadIdx.x; r < k; r += THREADS) pad(r);  // a segment shorter than k: the other ranks are empty
       if (PLAN) {
         __syncwarp();  // only some lanes resolved a fact: together again before the barrier
@@ -1018,8 +1027,9 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     for (int i = threadIdx.x; i < n; i += THREADS) s_keys[i] = order_key(__ldcg(sc + i));
   }
   __syncthreads();
+  if (PLAN && early) grid_dependency_wait();
 
-  // ---- general selection (large k, long segments, or the extraction's check failed) -------------------------
+  // ---- general selection (large k, long segments, or more candidates than threads) --------------------------
   topk_block<THREADS, false>(sm, sc, s_keys, n, k, IdMap{nullptr, row_ids, PLAN ? s_ids : nullptr}, out_ids, out_scores);
   if (PLAN) {
     // the ids of query q are request q's fact list: plan it right here (steps I1-I3), in the shared memory the
@@ -1041,13 +1051,17 @@ __global__ void __launch_bounds__(THREADS) score_topk_fused_kernel(const Retriev
 }
 
 // The same, and the last CTA of a query goes on to plan that query's injection request (memstore_retrieve_inject).
+// early != 0 (the caller vouches that the queries, users, start positions and block tables were complete before the
+// preceding work of the stream began): the scoring and the selection do not wait for the preceding grid - when that is
+// this library's copy kernel, they run on the SMs it vacates while it drains - and only the last CTA of a query waits,
+// right before it writes the ids and the plan.
 template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
                                                                         uint32_t* tickets, int keys_capacity, int n_host,
-                                                                        const __grid_constant__ InjectParams ip) {
-  grid_dependency_wait();    // launched as a programmatic dependent: nothing is touched before the preceding grid is done
+                                                                        const __grid_constant__ InjectParams ip, int early) {
+  if (!early) grid_dependency_wait();  // launched as a programmatic dependent: nothing is touched before the preceding grid is done
   grid_launch_dependents();  // the copy kernel may be scheduled early; it waits for this grid before reading the plan
-  score_topk_body<T, THREADS, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip);
+  score_topk_body<T, THREADS, true>(p, rows_per_cta, tickets, keys_capacity, n_host, &ip, early != 0);
 }
 
 // ---- tensor-core path, steps 2 and 3 (step 1 is score_gemm_groupmax_kernel) -------------------------------------

@@ -24,6 +24,7 @@ ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
 INJECT_REVERSE = 1
 INJECT_PREFIX = 2
 RETRIEVE_ANN = 4
+INPUTS_STABLE = 8
 CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 STORE_TMA_COPY_PATH = 1
 REQ_KERNEL_TIMEOUT = 32

@@ -436,6 +436,39 @@ def test_retrieve_inject_one_call_equals_the_two_calls(n_users, nq, n_facts, k):
     ms.close()
 
 
+def test_inputs_stable_flag_overlaps_requests_without_changing_results():
+    """MS_INPUTS_STABLE lets the scoring of a request start while the previous request's copy kernel drains.  Requests
+    issued back to back (no host synchronisation) with the flag must leave ids, token counts, status words and the cache
+    exactly as the same requests without the flag do - including when consecutive requests share blocks, so that a
+    plan written too early would corrupt the copy kernel still running."""
+    hs = HostStore(43, 1500, 4, 8, 128, 8, 40, 256, "float16")
+    ms = hs.to_memstore(5e5)
+    bs, k, nreq = 16, 24, 12
+    q = to_dev(synth.queries(44, nreq, 256, "float16"))
+    per_req = (7 + k * int(hs.lens.max())) // bs + 1
+    nb = per_req * 4
+    # request i uses table i mod 4: every fourth request overwrites the same blocks
+    tables = to_dev(synth.block_tables(45, nb, per_req, 4))
+    start = to_dev(np.array([7], np.int32))
+    outs = {}
+    for flags in (M.INJECT_REVERSE, M.INJECT_REVERSE | M.INPUTS_STABLE):
+        cache = make_cache(hs, nb, bs)
+        ids = torch.empty((nreq, k), dtype=torch.int32, device=DEV)
+        n_tok = torch.zeros(nreq, dtype=torch.int32, device=DEV)
+        status = torch.zeros(nreq, dtype=torch.int32, device=DEV)
+        ms.retrieve_inject(q[:1], k, start, tables[:1], cache, out_ids=ids[:1], flags=M.INJECT_REVERSE)  # sizes the scratch
+        for rep in range(3):
+            for i in range(nreq):
+                ms.retrieve_inject(q[i : i + 1], k, start, tables[i % 4 : i % 4 + 1], cache, out_ids=ids[i : i + 1],
+                                   out_n_tokens=n_tok[i : i + 1], out_status=status[i : i + 1], flags=flags)  # fmt: skip
+        torch.cuda.synchronize()
+        outs[flags] = (ids.cpu(), n_tok.cpu(), status.cpu(), cache.k.view(torch.int16).cpu(), cache.v.view(torch.int16).cpu())
+    a, b = outs[M.INJECT_REVERSE], outs[M.INJECT_REVERSE | M.INPUTS_STABLE]
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+    assert int(a[2].abs().sum()) == 0 and a[1].tolist() == [int(hs.lens[r].sum()) for r in a[0].numpy()]
+    ms.close()
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_inject_with_instruction_prefix(path):
     """The stored instruction prefix leads the composed segment (pre-RoPE keys rotated at the positions it gets), in
