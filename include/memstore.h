@@ -364,6 +364,10 @@ typedef struct {
   int64_t arena_bytes, embedding_bytes;
   int64_t host_kv_tokens_used;
   int64_t kernel_timeouts; /* 1 if a bounded wait inside the tensor-core scoring kernel ever ran out (results of that call are invalid) */
+  int64_t filter_fixups;   /* queries of the tensor-core retrieve path that were re-scanned exactly because the filter's margin
+                              check failed (more groups within rounding of the k-th score than the margin keeps) */
+  int64_t filter_fixup_overflows; /* 1 if such a re-scan ever met more than 4096 rows within rounding of the k-th score: that
+                                     query kept the filter's answer (ids inside the 1e-5 near-tie rule, exact ties unordered) */
 } memstore_stats_t;
 ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
 
@@ -375,6 +379,18 @@ ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
  * (NULL, NULL) when timing whole calls.  The caller owns the events.
  */
 ms_status memstore_set_profile_events(memstore_t* store, void* before_copy, void* after_copy);
+
+/*
+ * Test aid (no counterpart in the paper).  The kernels of this library that wait on a barrier (the bulk-async staged
+ * copy kernel, the tensor-core scoring kernel) bound every wait and report a time-out - MS_REQ_KERNEL_TIMEOUT in the
+ * requests' status words, kernel_timeouts in the statistics - instead of hanging.  That path cannot be reached by
+ * valid inputs, so this call lets a test reach it without any fault: with mute_producers != 0 the producer role of
+ * those kernels issues nothing at all (no copy is ever in flight), and with wait_poll_limit != 0 every wait gives up
+ * after that many polls (a few thousand polls are a fraction of a millisecond).  The kernels then return normally
+ * with the time-out reported; the call's outputs are unspecified but stay inside the caller's buffers.  (0, 0)
+ * restores normal behaviour and clears the recorded kernel_timeouts.
+ */
+ms_status memstore_test_hooks(memstore_t* store, uint32_t wait_poll_limit, int32_t mute_producers);
 
 /* Text of the last error on this store (never NULL; valid until the next call on the store). */
 const char* memstore_last_error(memstore_t* store);

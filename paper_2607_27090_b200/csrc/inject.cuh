@@ -44,6 +44,8 @@ struct InjectParams {
   uint32_t tiles_capacity;
   InjectCtrl* ctrl;  // control block of the store (see InjectCtrl)
   int32_t layers_per_item;
+  uint32_t spin_limit;    // 0: the default bound of the staged kernel's waits; else a test's shorter bound
+  int32_t mute_producer;  // test aid: the staged kernel's producer role issues nothing
 };
 
 constexpr int kPlanThreads = 256;

@@ -44,9 +44,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
                : "memory");
 }
 // Bounded wait for the phase with the given parity.  Returns false on time-out or when another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = kSpinLimit) {
   const uint32_t addr = smem_u32(bar);
-  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+  for (uint32_t spin = 0; spin < limit; ++spin) {
     uint32_t ok;
     asm volatile(
         "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int D = p.head_dim, H = p.n_heads, L = p.n_layers;
   const int row_bytes = H * D * 2;
+  const uint32_t limit = p.spin_limit ? p.spin_limit : kSpinLimit;  // (a test shortens the waits, see memstore_test_hooks)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kTmaStages; ++s) {
@@ -124,7 +125,9 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
   const uint32_t n_lg = (uint32_t)((L + lg - 1) / lg);
   const uint32_t n_chunks = n_ts * n_lg;
 
-  if (warp == 0) {
+  if (warp == 0 && p.mute_producer) {
+    // test aid: this role issues nothing at all (no copy is ever in flight), so the other roles' waits run out
+  } else if (warp == 0) {
     // ---------------------------------------------------------------- producer
     // Lanes 0..7 hold token t of the stage for K, lanes 8..15 the same tokens for V.  Rows that follow one
     // another in the arena (tokens of one fact) are fetched by ONE bulk copy issued by the first lane of the run.
@@ -176,7 +179,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
       const int to_next = stop ? __ffs((int)stop) : (8 - t);
       const uint32_t run_rows = (start && (is_k || is_v)) ? (uint32_t)min(to_next, 8 - t) : 0u;
       for (int layer = l0; layer < l1; ++layer) {
-        ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag);
+        ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, limit);
         if (!ok) break;
         if (is_k) meta[s].dst_off[t] = dst;
         if (lane == 0) {
@@ -201,7 +204,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
       c0 = c1;
     }
     // end marker: a stage with layer = -1 tells the other roles that no more work will come
-    if (ok && mbar_wait(&empty[s], ph ^ 1u, abort_flag)) {
+    if (ok && mbar_wait(&empty[s], ph ^ 1u, abort_flag, limit)) {
       if (lane == 0) {
         meta[s].layer = -1;
         meta[s].valid = 0;
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
     uint32_t ph = 0;
     const int t = lane & 7;
     for (;;) {
-      if (!mbar_wait(&full[s], ph, abort_flag)) break;
+      if (!mbar_wait(&full[s], ph, abort_flag, limit)) break;
       const int layer = meta[s].layer;
       if (layer < 0) break;
       const uint32_t valid = meta[s].valid;
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) inject_copy_tma_kernel(const I
     int s = 0;
     uint32_t ph = 0;
     for (;;) {
-      if (!mbar_wait(&full[s], ph, abort_flag)) break;
+      if (!mbar_wait(&full[s], ph, abort_flag, limit)) break;
       const StageMeta& mt = meta[s];
       if (mt.layer < 0) break;
       if (mt.tsub != cur) {

@@ -52,6 +52,14 @@ struct memstore {
   float* tc_cand_scores = nullptr;
   int32_t* tc_cand_rows = nullptr;
   uint32_t* tc_tickets = nullptr;
+  float* tc_next_best = nullptr;  // per query: the filter's best score among the rows that are not rescored
+  float* tc_kth = nullptr;        // per query: the k-th exact score after rescoring
+  int* tc_redo = nullptr;         // per query: the margin check failed, the fix-up kernel rescans the segment
+  float* tc_scores_out = nullptr; // [64][kTcMaxK] exact scores by rank when the caller asks for none
+  uint32_t* tc_fix_counts = nullptr;
+  unsigned long long* tc_fix_keys = nullptr;  // [64][kFixupCap]
+  uint32_t* tc_fix_tickets = nullptr;
+  uint32_t* tc_n_fixups = nullptr;  // queries the fix-up kernel has redone since creation
   int* tc_error = nullptr;
   bool tc_ready = false;
   int64_t scores_nq = 0;
@@ -83,6 +91,8 @@ struct memstore {
   int64_t prefix_tokens_total = 0;  // arena tokens taken by this and earlier prefixes (not facts)
   int64_t max_user_count = 0;
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
+  uint32_t test_spin_limit = 0;  // memstore_test_hooks
+  int test_mute_producers = 0;
   int copy_ctas_per_sm = 1;
   bool tma_path = false;  // MS_STORE_TMA_COPY_PATH
   std::recursive_mutex mu;  // recursive: memstore_serve_host holds it across retrieve and inject
@@ -216,9 +226,22 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_cand_scores, (size_t)kGemmMaxQ * kTcMaxK2 * 8 * sizeof(float)));
   MS_CUDA(s, cudaMalloc(&s->tc_cand_rows, (size_t)kGemmMaxQ * kTcMaxK2 * 8 * sizeof(int32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_tickets, (size_t)kGemmMaxQ * sizeof(uint32_t)));
-  MS_CUDA(s, cudaMalloc(&s->tc_error, sizeof(int)));
+  MS_CUDA(s, cudaMalloc(&s->tc_next_best, (size_t)kGemmMaxQ * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_kth, (size_t)kGemmMaxQ * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_redo, (size_t)kGemmMaxQ * sizeof(int)));
+  MS_CUDA(s, cudaMalloc(&s->tc_scores_out, (size_t)kGemmMaxQ * kTcMaxK * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_fix_counts, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_fix_keys, (size_t)kGemmMaxQ * kFixupCap * sizeof(unsigned long long)));
+  MS_CUDA(s, cudaMalloc(&s->tc_fix_tickets, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_n_fixups, 2 * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_error, 2 * sizeof(int)));
   MS_CUDA(s, cudaMemset(s->tc_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
-  MS_CUDA(s, cudaMemset(s->tc_error, 0, sizeof(int)));
+  MS_CUDA(s, cudaMemset(s->tc_redo, 0, (size_t)kGemmMaxQ * sizeof(int)));
+  MS_CUDA(s, cudaMemset(s->tc_fix_counts, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tc_fix_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tc_n_fixups, 0, 2 * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tc_error, 0, 2 * sizeof(int)));
+  MS_CUDA(s, cudaFuncSetAttribute(tc_fixup_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kFixupCap * sizeof(unsigned long long))));
   MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
   const size_t rs = (size_t)kTcMaxK2 * 8 * sizeof(uint32_t);
   MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
@@ -245,10 +268,11 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     CUtensorMap tmap_q;
     if (!make_tmap_rows_f16(&tmap_q, qptr, (uint64_t)nqb, (uint64_t)c.emb_dim, kGemmMaxQ))
       return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the query batch");
-    GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes};
+    GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes,
+                  s->test_spin_limit, s->test_mute_producers};
     score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
     MS_CUDA(s, cudaGetLastError());
-    select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel);
+    select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best);
     MS_CUDA(s, cudaGetLastError());
     RetrieveParams p = base;
     p.queries = qptr;
@@ -256,10 +280,21 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     p.out_ids = base.out_ids + (int64_t)q0 * base.k;
     p.out_scores = base.out_scores ? base.out_scores + (int64_t)q0 * base.k : nullptr;
     dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
+    float* scores_out = p.out_scores ? p.out_scores : s->tc_scores_out;
     rescore_topk_kernel<__half><<<grid, kScoreThreads, (size_t)k2 * 8 * sizeof(uint32_t), st>>>(
-        p, s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets);
+        p, s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets, scores_out, s->tc_next_best, s->tc_redo,
+        s->tc_kth);
     MS_CUDA(s, cudaGetLastError());
-    s->kernels_launched += 3;
+    // the fix-up of the queries whose margin check failed (its CTAs leave at once for all the others, so the grid is
+    // kept small: a few CTAs per query, each taking a slice of the segment)
+    const int fix_ctas = std::max(1, std::min(8 * s->sm_count / nqb, (int)((n_rows + 2047) / 2048)));
+    const int fix_rows = (int)(((n_rows + fix_ctas - 1) / fix_ctas + 1) & ~(int64_t)1);
+    dim3 fgrid((unsigned)((n_rows + fix_rows - 1) / fix_rows), (unsigned)nqb);
+    tc_fixup_kernel<__half><<<fgrid, kScoreThreads, kFixupCap * sizeof(unsigned long long), st>>>(
+        p, (int)n_rows, fix_rows, s->tc_redo, s->tc_kth, s->tc_fix_counts, s->tc_fix_keys, s->tc_fix_tickets, scores_out, s->tc_error + 1,
+        s->tc_n_fixups);
+    MS_CUDA(s, cudaGetLastError());
+    s->kernels_launched += 4;
   }
   return MS_OK;
 }
@@ -474,6 +509,14 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_cand_scores);
     cudaFree(s->tc_cand_rows);
     cudaFree(s->tc_tickets);
+    cudaFree(s->tc_next_best);
+    cudaFree(s->tc_kth);
+    cudaFree(s->tc_redo);
+    cudaFree(s->tc_scores_out);
+    cudaFree(s->tc_fix_counts);
+    cudaFree(s->tc_fix_keys);
+    cudaFree(s->tc_fix_tickets);
+    cudaFree(s->tc_n_fixups);
     cudaFree(s->tc_error);
     cudaFree(s->tiles);
     cudaFree(s->graph);
@@ -1124,6 +1167,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.tiles = s->tiles;
   p.tiles_capacity = s->tiles_capacity;
   p.ctrl = s->ctrl;
+  p.spin_limit = s->test_spin_limit;
+  p.mute_producer = s->test_mute_producers;
 
   // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
@@ -1377,11 +1422,29 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->arena_bytes = (int64_t)memstore_arena_bytes(&s->cfg);
   out->embedding_bytes = (int64_t)s->cfg.n_users * s->cfg.max_facts_per_user * s->cfg.emb_dim * (int64_t)emb_elem_size(s->cfg.emb_dtype);
   out->kernel_timeouts = 0;
+  out->filter_fixups = 0;
+  out->filter_fixup_overflows = 0;
   if (s->tc_error) {
     DeviceGuard g(s->cfg.device);
-    int flag = 0;
-    MS_CUDA(s, cudaMemcpy(&flag, s->tc_error, sizeof(int), cudaMemcpyDeviceToHost));
-    out->kernel_timeouts = flag;
+    int flags[2] = {0, 0};
+    uint32_t fix = 0;
+    MS_CUDA(s, cudaMemcpy(flags, s->tc_error, sizeof flags, cudaMemcpyDeviceToHost));
+    MS_CUDA(s, cudaMemcpy(&fix, s->tc_n_fixups, sizeof fix, cudaMemcpyDeviceToHost));
+    out->kernel_timeouts = flags[0];
+    out->filter_fixup_overflows = flags[1];
+    out->filter_fixups = fix;
+  }
+  return MS_OK;
+}
+
+ms_status memstore_test_hooks(memstore_t* s, uint32_t wait_poll_limit, int32_t mute_producers) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  s->test_spin_limit = wait_poll_limit;
+  s->test_mute_producers = mute_producers ? 1 : 0;
+  if (!wait_poll_limit && !mute_producers && s->tc_error) {  // back to normal: forget a time-out that a test provoked
+    DeviceGuard g(s->cfg.device);
+    MS_CUDA(s, cudaMemset(s->tc_error, 0, sizeof(int)));
   }
   return MS_OK;
 }

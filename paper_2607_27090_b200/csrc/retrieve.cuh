@@ -1069,17 +1069,19 @@ __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const Retrieve
 // Step 2: per query, the k2 groups with the largest group maximum, written in ASCENDING group order (so that the
 // candidate rows of step 3 are in row order and "lower index first" among equal scores means "lower fact id first").
 __global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
-                                                                    int32_t* sel /*[nq][k2]*/) {
+                                                                    int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/) {
   __shared__ TopkShared sm;
   __shared__ int32_t s_sel[512];
+  __shared__ float s_val[512];
   const int q = blockIdx.x;
   int32_t* out = sel + (int64_t)q * k2;
-  topk_block<kTopkThreads>(sm, gmax + (int64_t)q * gmax_stride, nullptr, n_groups, k2, IdMap{nullptr, nullptr}, out, nullptr);
+  // one group more than asked for: its maximum is the best score the filter saw among the rows that will NOT be
+  // rescored, which the rescoring step compares with the k-th exact score it finds
+  topk_block<kTopkThreads>(sm, gmax + (int64_t)q * gmax_stride, nullptr, n_groups, k2 + 1, IdMap{nullptr, nullptr}, s_sel, s_val);
   __syncthreads();
+  if (threadIdx.x == 0) next_best[q] = n_groups > k2 ? s_val[k2] : -INFINITY;
   // order the chosen group indices ascending by counting (k2 <= 512 distinct indices; -1 padding, present only when
   // the segment has fewer than k2 groups, counts as the largest value and keeps its relative order)
-  for (int i = threadIdx.x; i < k2; i += kTopkThreads) s_sel[i] = out[i];
-  __syncthreads();
   for (int i = threadIdx.x; i < k2; i += kTopkThreads) {
     const uint32_t mine = (uint32_t)s_sel[i];
     int rank = 0;
@@ -1139,9 +1141,15 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
 // retrieve kernels) and take the top-k of these candidates.  grid = (candidate groups of 8 rows per warp..., nq);
 // candidate c of query q is row sel[q][c / 8] * 8 + c % 8.  The last CTA of a query (wait-free ticket) selects.
 // Dynamic shared memory: n_cand uint32 keys.
+// The margin check: `scores_out` ([nq][k], never NULL) receives the exact scores by rank; when the k-th of them does not
+// beat next_best[q] (the filter's best score among the rows that were not rescored) by more than the filter's rounding,
+// a row outside the selected groups may belong to the top-k: redo[q] is raised and kth[q] tells the fix-up kernel which
+// exact score a row must reach.
+constexpr float kTcFilterRounding = 1e-5f;  // tensor-core fp32 accumulation against the fixed-order CUDA-core sum, times max(1, |score|)
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const RetrieveParams p, const int32_t* sel, int k2, int n_rows,
-                                                                     float* cand_scores, int32_t* cand_rows, uint32_t* tickets) {
+                                                                     float* cand_scores, int32_t* cand_rows, uint32_t* tickets,
+                                                                     float* scores_out, const float* next_best, int* redo, float* kth) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ int s_last;
@@ -1204,7 +1212,86 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
   }
   __syncthreads();
   topk_block<kScoreThreads, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
-                            p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr, true, lo, hi);
+                            scores_out + (int64_t)q * p.k, true, lo, hi);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int again = 0;
+    float need = 0.f;
+    if (n_valid >= p.k) {
+      need = __ldcg(scores_out + (int64_t)q * p.k + p.k - 1);
+      again = next_best[q] >= need - kTcFilterRounding * fmaxf(1.f, fabsf(need));
+    }
+    redo[q] = again;
+    kth[q] = need;
+  }
+}
+
+// Fix-up of the tensor-core path for the queries whose margin check failed (rare: more groups than the margin within
+// rounding of the k-th score - near-duplicate rows spread over many groups).  Launched after every rescoring; CTAs of
+// queries that passed leave at once.  For a flagged query every row of the segment is scored exactly (the CUDA-core
+// routine of the other kernels) and the rows that reach kth[q] - every row of the true top-k does - are collected as
+// 64-bit keys; the last CTA of the query sorts them and writes the top-k.  More collected rows than `cap` (thousands
+// of rows within rounding of one another) leave the filter's answer in place and raise *overflow.
+constexpr int kFixupCap = 4096;
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads) tc_fixup_kernel(const RetrieveParams p, int n_rows, int rows_per_cta, int* redo, const float* kth,
+                                                                 uint32_t* counts, unsigned long long* keys /*[nq][kFixupCap]*/,
+                                                                 uint32_t* tickets, float* scores_out, int* overflow, uint32_t* n_fixups) {
+  extern __shared__ unsigned long long s_fix[];  // kFixupCap keys
+  __shared__ int s_last;
+  const int q = blockIdx.y;
+  if (!redo[q]) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const T* seg = reinterpret_cast<const T*>(p.emb);  // user 0
+  const float need = kth[q];
+  const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta, row_end = min(row0 + rows_per_cta, (int64_t)n_rows);
+  unsigned long long* mine = keys + (int64_t)q * kFixupCap;
+  for (int64_t row = row0 + 2 * warp; row < row_end; row += 2 * kScoreWarps) {
+    float s0, s1 = -INFINITY;
+    if (row + 1 < row_end) {
+      score_two_rows<T>(p, q, seg, row, row + 1, s0, s1);
+      s1 += 0.0f;
+    } else {
+      s0 = score_one_row<T>(p, q, seg, row);
+    }
+    s0 += 0.0f;
+    if (lane == 0) {
+      if (s0 >= need) {
+        const uint32_t slot = atomicAdd(&counts[q], 1u);
+        if (slot < (uint32_t)kFixupCap) mine[slot] = ((unsigned long long)order_key(s0) << 32) | (uint32_t)(0xffffffffu - (uint32_t)row);
+      }
+      if (s1 >= need) {
+        const uint32_t slot = atomicAdd(&counts[q], 1u);
+        if (slot < (uint32_t)kFixupCap) mine[slot] = ((unsigned long long)order_key(s1) << 32) | (uint32_t)(0xffffffffu - (uint32_t)(row + 1));
+      }
+    }
+  }
+  __syncwarp();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const uint32_t t = atomicAdd(&tickets[q], 1u);
+    s_last = t == gridDim.x - 1;
+    if (s_last) tickets[q] = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const uint32_t n = __ldcg(&counts[q]);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    counts[q] = 0;
+    redo[q] = 0;
+    atomicAdd(n_fixups, 1u);
+    if (n > (uint32_t)kFixupCap) atomicExch(overflow, 1);
+  }
+  if (n > (uint32_t)kFixupCap || n < (uint32_t)p.k) return;  // (fewer than k cannot happen: the k rescored rows reach kth)
+  int P2 = 1;
+  while (P2 < (int)n) P2 <<= 1;
+  for (int i = threadIdx.x; i < P2; i += kScoreThreads) s_fix[i] = i < (int)n ? __ldcg(mine + i) : 0ull;
+  __syncthreads();
+  bitonic_sort_desc<kScoreThreads>(s_fix, P2);
+  write_topk<kScoreThreads>(s_fix, p.k, p.k, IdMap{nullptr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k, scores_out + (int64_t)q * p.k);
 }
 
 }  // namespace ms

@@ -43,6 +43,8 @@ struct GemmParams {
   int64_t gmax_stride;  // multiple of 16, >= 16 * ceil(n_rows / 128)
   int* error_flag;
   uint32_t smem_bytes;  // dynamic shared memory of the launch
+  uint32_t spin_limit;  // 0: the default bound of every wait; else a test's shorter bound
+  int mute_producer;    // test aid: the producer role issues nothing, so the other roles' waits run out
 };
 
 // Shared memory after the 1 KiB alignment of the base: queries, ring, epilogue staging (4 warps x [4 groups][32
@@ -157,10 +159,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   const uint32_t tmem_base = *tmem_slot;
 
   const int n_tiles = (p.n_rows + kGemmTileRows - 1) / kGemmTileRows;
+  const uint32_t limit = p.spin_limit ? p.spin_limit : kSpinLimit;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && !p.mute_producer) {
       mbar_arrive_expect_tx(q_full, (uint32_t)nkc * kGemmQBytes);
       for (int kc = 0; kc < nkc; ++kc) tma_load_2d(q_smem + (size_t)kc * kGemmQBytes, &tmap_q, kc * kGemmKChunk, 0, q_full);
       int s = 0;
@@ -168,7 +171,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
         for (int kc = 0; kc < nkc; ++kc) {
-          ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag);
+          ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, limit);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[s], kGemmABytes);
           tma_load_2d(a_smem + (size_t)s * kGemmABytes, &tmap_emb, kc * kGemmKChunk, tile * kGemmTileRows, &full[s]);
@@ -182,18 +185,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      bool ok = mbar_wait(q_full, 0, abort_flag);
+      bool ok = mbar_wait(q_full, 0, abort_flag, limit);
       int s = 0;
       uint32_t ph = 0;
       int it = 0;
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
         const int b = it & 1;
-        ok = mbar_wait(&acc_empty[b], (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag);
+        ok = mbar_wait(&acc_empty[b], (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag, limit);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * kGemmMaxQ);
         for (int kc = 0; kc < nkc; ++kc) {
-          ok = mbar_wait(&full[s], ph, abort_flag);
+          ok = mbar_wait(&full[s], ph, abort_flag, limit);
           if (!ok) break;
           tc_fence_after();
           const uint64_t a_desc = umma_desc_k_sw128(smem_u32(a_smem + (size_t)s * kGemmABytes));
@@ -218,7 +221,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int b = it & 1;
-      if (!mbar_wait(&acc_full[b], (uint32_t)((it >> 1) & 1), abort_flag)) break;
+      if (!mbar_wait(&acc_full[b], (uint32_t)((it >> 1) & 1), abort_flag, limit)) break;
       tc_fence_after();
       float v[kGemmMaxQ];
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * kGemmMaxQ);

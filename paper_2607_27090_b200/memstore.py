@@ -63,7 +63,7 @@ class _AnnParams(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "filter_fixup_overflows")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares
@@ -73,6 +73,7 @@ EXPORTS = (
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
     "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
+    "memstore_test_hooks",
 )  # fmt: skip
 
 _lib = None
@@ -109,6 +110,8 @@ def load_library() -> C.CDLL:
     L.memstore_build_graph.argtypes = [vp, i32, vp]
     L.memstore_graph_append.restype = i32
     L.memstore_graph_append.argtypes = [vp, vp]
+    L.memstore_test_hooks.restype = i32
+    L.memstore_test_hooks.argtypes = [vp, C.c_uint32, C.c_int32]
     L.memstore_set_graph.restype = i32
     L.memstore_set_graph.argtypes = [vp, vp, i64, i32, vp]
     L.memstore_get_graph.restype = i32
@@ -349,6 +352,11 @@ class MemStore:
     def build_graph(self, degree=64, stream=None) -> None:
         """Exact neighbour graph of all facts present (single-segment stores), built on the device."""
         self._check(self._lib.memstore_build_graph(self._h, degree, _stream_ptr(stream)))
+
+    def test_hooks(self, wait_poll_limit: int = 0, mute_producers: bool = False) -> None:
+        """Test aid: shorten every bounded wait of the staged kernels and silence their producer roles, so that the
+        time-out reporting can be exercised; ``test_hooks()`` restores normal behaviour."""
+        self._check(self._lib.memstore_test_hooks(self._h, int(wait_poll_limit), int(bool(mute_producers))))
 
     def graph_append(self, stream=None) -> None:
         """Grow the graph for the facts added since it was built, set or last grown."""
