@@ -381,6 +381,22 @@ ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
 ms_status memstore_set_profile_events(memstore_t* store, void* before_copy, void* after_copy);
 
 /*
+ * Size every scratch buffer ahead of serving (no counterpart in the paper; Sec. 3.3 / 3.4 only ask that the serving
+ * path be search, compose, scatter).  memstore_retrieve, memstore_inject, memstore_retrieve_inject and
+ * memstore_serve_host allocate their scratch (scores, tickets, tile descriptors, staging buffers, the tensor-core
+ * path's buffers) the first time a call needs more than there is, which synchronises the device once; after this
+ * call, calls within the stated sizes allocate nothing and never synchronise with the host (memstore_serve_host still
+ * waits for its own stream at its end):
+ *   nq                      queries per retrieve / retrieve_inject call (0: leave the retrieval scratch alone)
+ *   k                       ids per query or request (sizes memstore_serve_host's buffers together with max_blocks)
+ *   nreq                    requests per inject call (0: leave the injection scratch alone)
+ *   max_tokens_per_request  most tokens one request composes (k x longest fact + prefix)
+ *   max_blocks              block-table length given to memstore_serve_host (0: leave its staging buffers alone)
+ * Larger calls later still work: they grow the scratch as before.  Call it with no work of this store in flight.
+ */
+ms_status memstore_reserve(memstore_t* store, int32_t nq, int32_t k, int32_t nreq, int64_t max_tokens_per_request, int32_t max_blocks);
+
+/*
  * Test aid (no counterpart in the paper).  The kernels of this library that wait on a barrier (the bulk-async staged
  * copy kernel, the tensor-core scoring kernel) bound every wait and report a time-out - MS_REQ_KERNEL_TIMEOUT in the
  * requests' status words, kernel_timeouts in the statistics - instead of hanging.  That path cannot be reached by

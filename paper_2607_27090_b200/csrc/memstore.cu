@@ -340,6 +340,57 @@ void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams
     launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
 }
 
+// Scratch that grows on first use.  Each helper synchronises the device only when it really has to allocate;
+// memstore_reserve calls them ahead of serving so that no later call does.
+ms_status ensure_scores(memstore* s, int64_t nq) {
+  if (nq <= s->scores_nq) return MS_OK;
+  MS_CUDA(s, cudaDeviceSynchronize());
+  cudaFree(s->scores);
+  cudaFree(s->tickets);
+  s->scores = nullptr;
+  s->tickets = nullptr;
+  s->scores_nq = 0;
+  MS_CUDA(s, cudaMalloc(&s->scores, (size_t)nq * s->cfg.max_facts_per_user * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tickets, (size_t)nq * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tickets, 0, (size_t)nq * sizeof(uint32_t)));
+  s->scores_nq = nq;
+  return MS_OK;
+}
+
+ms_status ensure_tiles(memstore* s, int64_t tiles_needed) {
+  if (tiles_needed <= s->tiles_capacity) return MS_OK;
+  if (tiles_needed > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
+  MS_CUDA(s, cudaDeviceSynchronize());
+  cudaFree(s->tiles);
+  s->tiles = nullptr;
+  s->tiles_capacity = 0;
+  MS_CUDA(s, cudaMalloc(&s->tiles, (size_t)tiles_needed * sizeof(TileDesc)));
+  s->tiles_capacity = (uint32_t)tiles_needed;
+  return MS_OK;
+}
+
+ms_status ensure_stage(memstore* s, size_t bytes) {
+  if (bytes <= s->stage_bytes) return MS_OK;
+  MS_CUDA(s, cudaDeviceSynchronize());
+  cudaFree(s->dev_stage);
+  if (s->host_stage) cudaFreeHost(s->host_stage);
+  s->dev_stage = nullptr;
+  s->host_stage = nullptr;
+  s->stage_bytes = 0;
+  const size_t want = bytes * 2;
+  MS_CUDA(s, cudaMalloc(&s->dev_stage, want));
+  MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocMapped));
+  s->stage_bytes = want;
+  return MS_OK;
+}
+
+// staging bytes of one memstore_serve_host request: [query | header | block table] and [ids | n_tokens, status]
+void serve_host_layout(const memstore_config& c, int32_t max_blocks, int32_t k, size_t* q_bytes, size_t* in_bytes, size_t* out_bytes) {
+  *q_bytes = ((size_t)c.emb_dim * emb_elem_size(c.emb_dtype) + 15) & ~(size_t)15;
+  *in_bytes = *q_bytes + 16 + (((size_t)max_blocks * 4 + 15) & ~(size_t)15);
+  *out_bytes = (((size_t)k + 2) * 4 + 15) & ~(size_t)15;
+}
+
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
 // stream than the previous one, an event recorded at the tail of the previous stream is waited for.
 // A stream that is being captured into a CUDA graph: the calls recorded on it run later, at every replay, and cannot
@@ -675,19 +726,12 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
   const bool tc = tc_path_applies(s, query_users, nq, k, query_users ? s->max_user_count : s->user_count[0]);
-  if (!tc && nq > s->scores_nq) {  // grow the score scratch (first call, or a larger batch than ever before)
-    MS_CUDA(s, cudaDeviceSynchronize());
-    cudaFree(s->scores);
-    cudaFree(s->tickets);
-    s->scores = nullptr;
-    s->tickets = nullptr;
-    s->scores_nq = 0;
-    MS_CUDA(s, cudaMalloc(&s->scores, (size_t)nq * c.max_facts_per_user * sizeof(float)));
-    MS_CUDA(s, cudaMalloc(&s->tickets, (size_t)nq * sizeof(uint32_t)));
-    MS_CUDA(s, cudaMemset(s->tickets, 0, (size_t)nq * sizeof(uint32_t)));
-    s->scores_nq = nq;
+  ms_status rc = MS_OK;
+  if (!tc) {  // grow the score scratch (first call, or a larger batch than ever before)
+    rc = ensure_scores(s, nq);
+    if (rc != MS_OK) return rc;
   }
-  ms_status rc = order_after_last(s, st);
+  rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
 
   RetrieveParams p{};
@@ -1114,14 +1158,9 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   if (max_m > 0x3fffffff) return fail(s, MS_ERR_UNSUPPORTED, "a request could compose %lld tokens (k x longest fact): more than 2^30", (long long)max_m);
   const int64_t tiles_per_req = (max_m + kTileTokens - 1) / kTileTokens + 1;
   const int64_t tiles_needed = std::max<int64_t>(1, tiles_per_req * nreq);
-  if (tiles_needed > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
-  if (tiles_needed > s->tiles_capacity) {
-    MS_CUDA(s, cudaDeviceSynchronize());
-    cudaFree(s->tiles);
-    s->tiles = nullptr;
-    s->tiles_capacity = 0;
-    MS_CUDA(s, cudaMalloc(&s->tiles, (size_t)tiles_needed * sizeof(TileDesc)));
-    s->tiles_capacity = (uint32_t)tiles_needed;
+  {
+    const ms_status rc = ensure_tiles(s, tiles_needed);
+    if (rc != MS_OK) return rc;
   }
   *out_tiles_needed = tiles_needed;
 
@@ -1368,20 +1407,11 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
   DeviceGuard g(c.device);
   cudaStream_t st = (cudaStream_t)stream;
   // layout of both staging buffers: [query | start_pos, user, pad, pad | block table] then [ids | n_tokens, status]
-  const size_t q_bytes = ((size_t)c.emb_dim * emb_elem_size(c.emb_dtype) + 15) & ~(size_t)15;
-  const size_t in_bytes = q_bytes + 16 + (((size_t)max_blocks * 4 + 15) & ~(size_t)15);
-  const size_t out_bytes = (((size_t)k + 2) * 4 + 15) & ~(size_t)15;
-  if (in_bytes + out_bytes > s->stage_bytes) {
-    MS_CUDA(s, cudaDeviceSynchronize());
-    cudaFree(s->dev_stage);
-    if (s->host_stage) cudaFreeHost(s->host_stage);
-    s->dev_stage = nullptr;
-    s->host_stage = nullptr;
-    s->stage_bytes = 0;
-    const size_t want = (in_bytes + out_bytes) * 2;
-    MS_CUDA(s, cudaMalloc(&s->dev_stage, want));
-    MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocMapped));
-    s->stage_bytes = want;
+  size_t q_bytes, in_bytes, out_bytes;
+  serve_host_layout(c, max_blocks, k, &q_bytes, &in_bytes, &out_bytes);
+  {
+    const ms_status rc = ensure_stage(s, in_bytes + out_bytes);
+    if (rc != MS_OK) return rc;
   }
   unsigned char* h = s->host_stage;
   unsigned char* d = s->dev_stage;
@@ -1433,6 +1463,40 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
     out->kernel_timeouts = flags[0];
     out->filter_fixup_overflows = flags[1];
     out->filter_fixups = fix;
+  }
+  return MS_OK;
+}
+
+ms_status memstore_reserve(memstore_t* s, int32_t nq, int32_t k, int32_t nreq, int64_t max_tokens_per_request, int32_t max_blocks) {
+  Range range("memstore_reserve");
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (nq < 0 || nreq < 0 || k < 0 || k > kTopkMaxK || max_tokens_per_request < 0 || max_blocks < 0)
+    return fail(s, MS_ERR_INVALID_ARG, "memstore_reserve: negative size or k > %d", kTopkMaxK);
+  DeviceGuard g(c.device);
+  ms_status rc = MS_OK;
+  if (nq > 0) {
+    rc = ensure_scores(s, nq);
+    if (rc != MS_OK) return rc;
+    const size_t smem = (size_t)std::min<int64_t>(c.max_facts_per_user, kFusedMaxRows) * sizeof(uint32_t);
+    MS_CUDA(s, ensure_fused_smem(c.device, smem));
+    // the tensor-core filter path serves long fp16 segments: its scratch as well, when this store can take that path
+    if (c.emb_dtype == MS_DTYPE_F16 && c.emb_dim % kGemmKChunk == 0 && c.emb_dim <= kGemmMaxE && c.max_facts_per_user > kFusedMaxRows) {
+      rc = tc_prepare(s);
+      if (rc != MS_OK) return rc;
+    }
+  }
+  if (nreq > 0) {
+    const int64_t tiles_per_req = (max_tokens_per_request + kTileTokens - 1) / kTileTokens + 1;
+    rc = ensure_tiles(s, std::max<int64_t>(1, tiles_per_req * nreq));
+    if (rc != MS_OK) return rc;
+  }
+  if (max_blocks > 0 && k > 0) {
+    size_t q_bytes, in_bytes, out_bytes;
+    serve_host_layout(c, max_blocks, k, &q_bytes, &in_bytes, &out_bytes);
+    rc = ensure_stage(s, in_bytes + out_bytes);
+    if (rc != MS_OK) return rc;
   }
   return MS_OK;
 }

@@ -73,7 +73,7 @@ EXPORTS = (
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
     "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
-    "memstore_test_hooks",
+    "memstore_test_hooks", "memstore_reserve",
 )  # fmt: skip
 
 _lib = None
@@ -110,6 +110,8 @@ def load_library() -> C.CDLL:
     L.memstore_build_graph.argtypes = [vp, i32, vp]
     L.memstore_graph_append.restype = i32
     L.memstore_graph_append.argtypes = [vp, vp]
+    L.memstore_reserve.restype = i32
+    L.memstore_reserve.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int32]
     L.memstore_test_hooks.restype = i32
     L.memstore_test_hooks.argtypes = [vp, C.c_uint32, C.c_int32]
     L.memstore_set_graph.restype = i32
@@ -352,6 +354,10 @@ class MemStore:
     def build_graph(self, degree=64, stream=None) -> None:
         """Exact neighbour graph of all facts present (single-segment stores), built on the device."""
         self._check(self._lib.memstore_build_graph(self._h, degree, _stream_ptr(stream)))
+
+    def reserve(self, nq: int = 0, k: int = 0, nreq: int = 0, max_tokens_per_request: int = 0, max_blocks: int = 0) -> None:
+        """Allocate every scratch buffer that calls of these sizes need, so that they allocate nothing later."""
+        self._check(self._lib.memstore_reserve(self._h, nq, k, nreq, max_tokens_per_request, max_blocks))
 
     def test_hooks(self, wait_poll_limit: int = 0, mute_producers: bool = False) -> None:
         """Test aid: shorten every bounded wait of the staged kernels and silence their producer roles, so that the

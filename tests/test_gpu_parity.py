@@ -911,6 +911,43 @@ def test_host_errors_return_codes_and_enqueue_nothing():
 
 
 # ------------------------------------------------------------------------------------------------ determinism
+def test_reserve_sizes_all_scratch_ahead_of_serving():
+    """After memstore_reserve the serving calls within the stated sizes allocate no device memory (the free-memory
+    figure of the device does not move) and give the results of an unreserved store."""
+    hs = HostStore(60, 300, 2, 4, 64, 4, 20, 64, "float16")
+    k, nreq, bs, nb = 12, 5, 16, 256
+    per_req = (3 + k * int(hs.lens.max())) // bs + 1
+    q = to_dev(synth.queries(61, nreq, 64, "float16"))
+    starts = to_dev(np.full(nreq, 3, np.int32))
+    tables = to_dev(synth.block_tables(62, nb, per_req, nreq))
+    results = []
+    for reserve in (True, False):
+        ms = hs.to_memstore(1e4)
+        cache = make_cache(hs, nb, bs)
+        out = np.full(k + 2, -5, np.int32)
+        if reserve:
+            ms.reserve(nq=nreq, k=k, nreq=nreq, max_tokens_per_request=k * int(hs.lens.max()), max_blocks=per_req)
+        warm = [torch.empty(1 << 14, device=DEV) for _ in range(16)]  # torch's own small-block pool is in place
+        del warm
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        ids, sc = ms.retrieve(q, k)
+        n_tok, st = ms.inject(ids, starts, tables, cache, flags=M.INJECT_REVERSE)
+        ids2, n2, st2 = ms.retrieve_inject(q, k, starts, tables, cache, flags=M.INJECT_REVERSE)
+        ms.serve_host(hs.emb[7], k, 3, tables[0].cpu().numpy(), cache, out, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        free1 = torch.cuda.mem_get_info()[0]
+        if reserve:
+            assert free1 == free0, f"{free0 - free1} bytes were allocated after memstore_reserve"
+        results.append((ids.cpu(), n_tok.cpu(), ids2.cpu(), n2.cpu(), out.copy(), cache.k.view(torch.int16).cpu()))
+        assert int(st.abs().sum()) == 0 and int(st2.abs().sum()) == 0
+        ms.close()
+    for a, b in zip(*results):
+        assert (torch.equal(a, b) if isinstance(a, torch.Tensor) else np.array_equal(a, b))
+    with pytest.raises(RuntimeError):
+        hs.to_memstore(1e4).reserve(nq=-1)
+
+
 def test_same_call_twice_and_on_two_streams_is_bit_identical():
     hs = HostStore(17, 30, 4, 8, 128, 16, 64, 256, "float16")
     ms = hs.to_memstore(5e5)
