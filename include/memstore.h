@@ -366,6 +366,8 @@ typedef struct {
   int64_t kernel_timeouts; /* 1 if a bounded wait inside the tensor-core scoring kernel ever ran out (results of that call are invalid) */
   int64_t filter_fixups;   /* queries of the tensor-core retrieve path that were re-scanned exactly because the filter's margin
                               check failed (more groups within rounding of the k-th score than the margin keeps) */
+  int64_t compose_cache_hits, compose_cache_fills; /* requests served from / recorded into the composition cache */
+  int64_t compose_cache_segments;                  /* segments the composition cache can hold (0: none) */
   int64_t filter_fixup_overflows; /* 1 if such a re-scan ever met more than 4096 rows within rounding of the k-th score: that
                                      query kept the filter's answer (ids inside the 1e-5 near-tie rule, exact ties unordered) */
 } memstore_stats_t;
@@ -379,6 +381,27 @@ ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
  * (NULL, NULL) when timing whole calls.  The caller owns the events.
  */
 ms_status memstore_set_profile_events(memstore_t* store, void* before_copy, void* after_copy);
+
+/*
+ * The composition cache (appendix "Position independence and rotation fidelity", closing remark: the one-time
+ * composition is cached across queries that reuse the same memory).  In this library composing IS the scatter, so for
+ * facts in HBM a cached segment saves nothing; it pays for facts of the host tier (Sec. 6.8), whose rows cross PCIe
+ * every time they are composed: a request that repeats an earlier one is served by an HBM-rate copy instead.
+ *   budget_bytes            device memory for cached segments (0: switch the cache off and free it)
+ *   max_tokens_per_segment  longest composed segment that is kept; the cache holds budget / (that many tokens' K and V
+ *                           over all layers) segments, at most 64
+ *   flags                   0: only requests that name at least one host-tier fact are recorded;
+ *                           MS_COMPOSE_CACHE_ALL: every eligible request
+ * A segment is the composed K (rotated, rounded to bf16) and V of one request.  Its key is the request's id list as
+ * given (at most 256 ids), its start position, MS_INJECT_REVERSE / MS_INJECT_PREFIX and the stored prefix: a request
+ * with the same key is a hit and is served by copying the segment through its own block table - byte for byte what
+ * composing again would write, into a bf16 or an 8-bit cache alike; anything else (another start position, another
+ * order) is a miss.  Requests are looked up by memstore_inject, memstore_retrieve_inject and memstore_serve_host on
+ * the device (the ids never reach the host); a miss is recorded, the least recently used segment making room, when the
+ * call holds ONE request whose status word is clean (multi-request calls only look up).  Synchronises the device.
+ */
+enum { MS_COMPOSE_CACHE_ALL = 1u };
+ms_status memstore_compose_cache(memstore_t* store, size_t budget_bytes, int32_t max_tokens_per_segment, uint32_t flags);
 
 /*
  * Size every scratch buffer ahead of serving (no counterpart in the paper; Sec. 3.3 / 3.4 only ask that the serving

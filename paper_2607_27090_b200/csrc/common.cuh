@@ -25,10 +25,16 @@ constexpr int kTileTokens = 8;
 // and is read over PCIe by the copy kernel; both arenas hold fewer than 2^30 tokens.
 constexpr int32_t kHostTierBit = 0x40000000;
 
+// A source token index with this bit set lives in the composition cache (see CcSlot): keys stored there are already
+// rotated for the positions of the cached segment, so the copy kernel copies them as they are.
+constexpr int32_t kCacheTierBit = 0x20000000;
+constexpr int32_t kNoFill = (int32_t)0x80000000;  // TileDesc::fill_tok0 of a tile that is not recorded in the composition cache
+
 // Work description of one tile, written by the plan kernel and read by the copy kernel.
 struct __align__(16) TileDesc {
   int32_t pos0;                 // position of lane 0 (multiple of kTileTokens)
-  int32_t pad[3];
+  int32_t fill_tok0;            // composition-cache token that lane 0's composed token is recorded at, or kNoFill
+  int32_t pad[2];
   int32_t src_tok[kTileTokens]; // arena token of each lane, -1: nothing to do
   int64_t dst_off[kTileTokens]; // element offset block*block_stride + token*token_stride in the cache
 };
@@ -44,6 +50,21 @@ struct InjectCtrl {
   uint32_t work_next;  // work ticket of the staged copy kernel (zeroed by the last planning CTA)
   uint32_t acc;        // tiles claimed so far by the planning CTAs of the running call (zero between calls)
   uint32_t planned;    // planning CTAs that have finished (zero between calls)
+};
+
+// Composition cache (the paper's closing remark of the appendix "Position independence and rotation fidelity": the
+// composed segment is cached across queries that reuse the same memory; it pays where composing is expensive, i.e. for
+// facts of the host tier, Sec. 6.8).  A slot holds the composed K (rotated, bf16) and V of one request, keyed by the
+// request's id list as given, its start position, its placement flags and the instruction prefix it used.
+constexpr int kCcMaxK = 256;     // longest id list a segment can be keyed by
+constexpr int kCcMaxSlots = 64;
+struct CcSlot {
+  uint32_t hash_lo, hash_hi;
+  int32_t k, start, flags, prefix_src, prefix_len, m;
+  uint32_t epoch;     // the store's cache epoch when the slot was filled (a different epoch: the slot is empty)
+  uint32_t last_use;  // injection call that filled or hit the slot last
+  int32_t pad[2];
+  int32_t ids[kCcMaxK];
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {

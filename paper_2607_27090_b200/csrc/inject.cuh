@@ -44,6 +44,15 @@ struct InjectParams {
   uint32_t tiles_capacity;
   InjectCtrl* ctrl;  // control block of the store (see InjectCtrl)
   int32_t layers_per_item;
+  // composition cache (nullptr / 0: none)
+  CcSlot* cc_slots;
+  __nv_bfloat16* cc_k;  // [L][cc_tokens][H][D] rotated keys of the cached segments, slot s at tokens s * cc_slot_tokens ...
+  __nv_bfloat16* cc_v;
+  int64_t cc_tokens;
+  int32_t cc_n_slots, cc_slot_tokens;
+  uint32_t cc_epoch, cc_call;  // current epoch of the store; number of this injection call (for the least-recently-used choice)
+  int32_t cc_fill_all;         // 0: only requests that name a host-tier fact are recorded; 1: every eligible request
+  uint32_t* cc_counters;       // [0] hits, [1] fills
   uint32_t spin_limit;    // 0: the default bound of the staged kernel's waits; else a test's shorter bound
   int32_t mute_producer;  // test aid: the staged kernel's producer role issues nothing
 };
@@ -64,6 +73,8 @@ struct PlanShared {
   int32_t scan[32];  // one partial sum per warp (up to 1024 threads)
   int32_t carry, status;
   uint32_t tile_base;
+  uint32_t cc_hash_lo, cc_hash_hi;  // composition cache: hash of the request's key; slot that may hold it; slot to record into
+  int32_t cc_cand, cc_victim;
 };
 
 // What planning request r needs and what does not depend on the request's ids, fetched ahead of time (all THREADS
@@ -150,6 +161,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     }
   };
   int32_t m;
+  int names_host_fact = 0;  // some placed fact lives in the host tier (the same value in every thread)
   if (n_entries <= THREADS) {
     // at most one entry per thread: one barrier, then every warp combines the warps' totals by a shuffle scan
     const int j = tid;
@@ -177,7 +189,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       s_src[j] = src;
     }
     __syncwarp();
-    __syncthreads();
+    names_host_fact = __syncthreads_or(len > 0 && (src & kHostTierBit) != 0);
   } else {
     // longer lists: chunks of THREADS entries with a running carry
     for (int base = 0; base < n_entries; base += THREADS) {
@@ -203,7 +215,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
       __syncthreads();
       if (tid == THREADS - 1) s_carry = carry + warp_off + x;
       __syncwarp();
-      __syncthreads();
+      names_host_fact |= __syncthreads_or(len > 0 && (src & kHostTierBit) != 0);
     }
     m = s_carry;
   }
@@ -215,6 +227,94 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     if (tid == 0) atomicOr(&s_status, start < 0 ? 64 /*MS_REQ_BAD_START*/ : 16 /*MS_REQ_POSITION_OVERFLOW*/);
     if (p.out_slot_mapping)
       for (int64_t q = tid; q < min((int64_t)m, p.slot_stride); q += THREADS) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = -1;
+  }
+  // ---- composition cache: has this very request been composed before, or should it be recorded now? ------------
+  int32_t hit_base = -1, fill_base = kNoFill;
+  if (p.cc_slots != nullptr && m > 0 && !bad_start && m <= p.cc_slot_tokens && p.k <= kCcMaxK && p.k > 0) {
+    const int32_t* key_ids = p.fact_ids + (int64_t)r * p.k;  // the list as the caller (or the retrieval) wrote it
+    const int32_t key_flags = (int32_t)(p.flags & 3u);
+    if (tid == 0) {
+      ps.cc_hash_lo = 0x9e3779b9u * (uint32_t)(p.k + 1) ^ (uint32_t)start * 0x85ebca6bu ^ (uint32_t)key_flags;
+      ps.cc_hash_hi = 0xc2b2ae35u * (uint32_t)(p.prefix_src + 3) ^ (uint32_t)p.prefix_len;
+      ps.cc_cand = -1;
+      ps.cc_victim = -1;
+    }
+    __syncthreads();
+    for (int t = tid; t < p.k; t += THREADS) {
+      uint32_t h = (uint32_t)key_ids[t] * 0x9e3779b1u + (uint32_t)t * 0x7feb352du;
+      h ^= h >> 15;
+      h *= 0x846ca68bu;
+      h ^= h >> 16;
+      atomicXor(&ps.cc_hash_lo, h);
+      atomicAdd(&ps.cc_hash_hi, h * 0x2c1b3c6du + 1u);
+    }
+    __syncwarp();
+    __syncthreads();
+    if (warp == 0) {
+      // lane l looks at slots l and l + 32: same key fields and hash?  otherwise, how long ago was it used?
+      uint32_t best_age = 0xffffffffu;
+      int best_slot = -1, match = -1;
+      for (int sl = lane; sl < p.cc_n_slots; sl += 32) {
+        const CcSlot& c = p.cc_slots[sl];
+        const bool live = c.epoch == p.cc_epoch;
+        if (live && c.hash_lo == ps.cc_hash_lo && c.hash_hi == ps.cc_hash_hi && c.k == p.k && c.start == start && c.flags == key_flags &&
+            c.prefix_src == p.prefix_src && c.prefix_len == p.prefix_len && c.m == m && match < 0)
+          match = sl;
+        const uint32_t age = live ? c.last_use + 1u : 0u;  // empty slots first, then the least recently used
+        if (age < best_age) {
+          best_age = age;
+          best_slot = sl;
+        }
+      }
+      const unsigned found = __ballot_sync(0xffffffffu, match >= 0);
+      if (found) {
+        const int src_lane = __ffs(found) - 1;
+        const int sl = __shfl_sync(0xffffffffu, match, src_lane);
+        if (lane == 0) ps.cc_cand = sl;
+      }
+      const uint32_t oldest = __reduce_min_sync(0xffffffffu, best_age);
+      const unsigned who = __ballot_sync(0xffffffffu, best_age == oldest && best_slot >= 0);
+      if (who) {
+        const int sl = __shfl_sync(0xffffffffu, best_slot, __ffs(who) - 1);
+        if (lane == 0) ps.cc_victim = sl;
+      }
+    }
+    __syncwarp();
+    __syncthreads();
+    const int cand = ps.cc_cand;
+    int same = 0;
+    if (cand >= 0) {  // equal hashes: compare the id lists themselves
+      bool eq = true;
+      for (int t = tid; t < p.k; t += THREADS) eq = eq && p.cc_slots[cand].ids[t] == key_ids[t];
+      __syncwarp();
+      same = __syncthreads_and(eq);
+    }
+    if (same) {
+      hit_base = cand * p.cc_slot_tokens;
+      if (tid == 0) {
+        p.cc_slots[cand].last_use = p.cc_call;
+        atomicAdd(&p.cc_counters[0], 1u);
+      }
+    } else if (p.nreq == 1 && s_status == 0 && ps.cc_victim >= 0 && (p.cc_fill_all || names_host_fact)) {
+      // record this request (single-request calls only: one planning CTA, so slots are never claimed concurrently)
+      const int v = ps.cc_victim;
+      fill_base = v * p.cc_slot_tokens;
+      CcSlot& c = p.cc_slots[v];
+      for (int t = tid; t < p.k; t += THREADS) c.ids[t] = key_ids[t];
+      if (tid == 0) {
+        c.hash_lo = ps.cc_hash_lo;
+        c.hash_hi = ps.cc_hash_hi;
+        c.k = p.k;
+        c.start = start;
+        c.flags = key_flags;
+        c.prefix_src = p.prefix_src;
+        c.prefix_len = p.prefix_len;
+        c.m = m;
+        c.epoch = p.cc_epoch;
+        c.last_use = p.cc_call;
+        atomicAdd(&p.cc_counters[1], 1u);
+      }
+    }
   }
   const int32_t first_tile_pos = bad_start ? 0 : (start / kTileTokens) * kTileTokens;
   const uint32_t n_tiles = (m > 0 && !bad_start) ? (uint32_t)((start - first_tile_pos + m + kTileTokens - 1) / kTileTokens) : 0u;
@@ -255,7 +355,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
           if (blk < 0 || blk >= p.num_blocks) {
             st = 8;  // MS_REQ_BAD_BLOCK_ID
           } else {
-            src_tok = s_src[i] + (q - s_begin[i]);
+            src_tok = hit_base >= 0 ? (kCacheTierBit | (hit_base + q)) : s_src[i] + (q - s_begin[i]);
             dst = (int64_t)blk * p.block_stride + (int64_t)in_block * p.token_stride;
             slot = (int64_t)blk * bs + in_block;
           }
@@ -266,7 +366,11 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
     }
     if (tile_base + t < p.tiles_capacity) {
       TileDesc* d = p.tiles + tile_base + t;
-      if (ln == 0) d->pos0 = first_tile_pos + (int32_t)(t * kTileTokens);
+      if (ln == 0) {
+        const int32_t pos0 = first_tile_pos + (int32_t)(t * kTileTokens);
+        d->pos0 = pos0;
+        d->fill_tok0 = fill_base == kNoFill ? kNoFill : fill_base + (pos0 - start);
+      }
       d->src_tok[ln] = src_tok;
       d->dst_off[ln] = dst;
     }
@@ -438,11 +542,16 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
     const int64_t dst = d->dst_off[tk];
     const int32_t pos = d->pos0 + tk;
 
-    // source rows: the HBM arena, or (host tier) the pinned host arena read straight over PCIe
-    const bool host = (src & kHostTierBit) != 0;
-    const int64_t src_row = ((int64_t)layer * (host ? p.host_tokens : p.arena_tokens) + (src & ~kHostTierBit)) * (int64_t)(p.n_heads * D);
-    const __nv_bfloat16* ks = (host ? p.k_host : p.k_arena) + src_row;
-    const __nv_bfloat16* vs = (host ? p.v_host : p.v_arena) + src_row;
+    // source rows: the HBM arena, (host tier) the pinned host arena read straight over PCIe, or a segment composed
+    // earlier and kept in the composition cache, whose keys are rotated already
+    const bool host = (src & kHostTierBit) != 0, cached = (src & kCacheTierBit) != 0;
+    const int64_t tier_tokens = cached ? p.cc_tokens : host ? p.host_tokens : p.arena_tokens;
+    const int64_t src_row = ((int64_t)layer * tier_tokens + (src & ~(kHostTierBit | kCacheTierBit))) * (int64_t)(p.n_heads * D);
+    const __nv_bfloat16* ks = (cached ? p.cc_k : host ? p.k_host : p.k_arena) + src_row;
+    const __nv_bfloat16* vs = (cached ? p.cc_v : host ? p.v_host : p.v_arena) + src_row;
+    const bool rotate_now = rotates && !cached;
+    // a request that is being recorded: the composed rows go to the composition cache as well
+    const int32_t fill0 = d->fill_tok0;
     const int64_t dbase = (int64_t)layer * p.layer_stride + dst;
     uint4 ka[kUnitsPerThread], kb[kUnitsPerThread], va[kUnitsPerThread], vb[kUnitsPerThread];
 #pragma unroll
@@ -459,7 +568,7 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
     // cos/sin of (pos, 8 frequencies), evaluated while the loads are in flight
     float sn[8], cs[8];
     const float posf = (float)pos;
-    if (rotates) {
+    if (rotate_now) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) rope_sincos(posf, __ldg(p.inv_freq + 8 * j + i), sn[i], cs[i]);
     }
@@ -468,8 +577,17 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
       const int unit = u0 + u * kThreadsPerToken;
       if (unit < n_units) {
         const int h = unit >> g_shift;
+        if (rotate_now) rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
+        if (fill0 != kNoFill) {
+          const int64_t fill_row = ((int64_t)layer * p.cc_tokens + (fill0 + tk)) * (int64_t)(p.n_heads * D);
+          __nv_bfloat16* ck = p.cc_k + fill_row + h * D;
+          __nv_bfloat16* cv = p.cc_v + fill_row + h * D;
+          st_stream(reinterpret_cast<uint4*>(ck + offA), ka[u]);
+          st_stream(reinterpret_cast<uint4*>(ck + offB), kb[u]);
+          st_stream(reinterpret_cast<uint4*>(cv + offA), va[u]);
+          st_stream(reinterpret_cast<uint4*>(cv + offB), vb[u]);
+        }
         if (!FP8) {
-          if (rotates) rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
           __nv_bfloat16* kd = p.k_cache + dbase + (int64_t)h * p.head_stride;
           st_stream(reinterpret_cast<uint4*>(kd + offA), ka[u]);
           st_stream(reinterpret_cast<uint4*>(kd + offB), kb[u]);
@@ -478,7 +596,6 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
           st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
         } else {
           float fa[8], fb[8];
-          if (rotates) rotate_unit<STYLE>(ka[u], kb[u], sn, cs);
           scaled_floats(ka[u], p.k_scale, fa);
           scaled_floats(kb[u], p.k_scale, fb);
           uint8_t* kd = reinterpret_cast<uint8_t*>(p.k_cache) + dbase + (int64_t)h * p.head_stride;

@@ -91,6 +91,12 @@ struct memstore {
   int64_t prefix_tokens_total = 0;  // arena tokens taken by this and earlier prefixes (not facts)
   int64_t max_user_count = 0;
   int64_t retrieve_calls = 0, inject_calls = 0, kernels_launched = 0;
+  // composition cache (memstore_compose_cache): composed segments of earlier requests, least recently used evicted
+  CcSlot* cc_slots = nullptr;
+  __nv_bfloat16* cc_arena = nullptr;  // K half then V half, each [L][cc_n_slots * cc_slot_tokens][h][d]
+  uint32_t* cc_counters = nullptr;    // [0] hits, [1] fills
+  int32_t cc_n_slots = 0, cc_slot_tokens = 0, cc_fill_all = 0;
+  uint32_t cc_epoch = 1, cc_call = 0;
   uint32_t test_spin_limit = 0;  // memstore_test_hooks
   int test_mute_producers = 0;
   int copy_ctas_per_sm = 1;
@@ -570,6 +576,9 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_n_fixups);
     cudaFree(s->tc_error);
     cudaFree(s->tiles);
+    cudaFree(s->cc_slots);
+    cudaFree(s->cc_arena);
+    cudaFree(s->cc_counters);
     cudaFree(s->graph);
     cudaFree(s->graph_topk);
     cudaFree(s->append_pairs);
@@ -1208,10 +1217,23 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.ctrl = s->ctrl;
   p.spin_limit = s->test_spin_limit;
   p.mute_producer = s->test_mute_producers;
+  if (s->cc_slots) {
+    const int64_t cc_tokens = (int64_t)s->cc_n_slots * s->cc_slot_tokens;
+    p.cc_slots = s->cc_slots;
+    p.cc_k = s->cc_arena;
+    p.cc_v = s->cc_arena + (size_t)c.n_layers * cc_tokens * c.n_kv_heads * c.head_dim;
+    p.cc_tokens = cc_tokens;
+    p.cc_n_slots = s->cc_n_slots;
+    p.cc_slot_tokens = s->cc_slot_tokens;
+    p.cc_epoch = s->cc_epoch;
+    p.cc_call = ++s->cc_call;
+    p.cc_fill_all = s->cc_fill_all;
+    p.cc_counters = s->cc_counters;
+  }
 
   // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
-  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
+  const bool use_tma = s->tma_path && !s->cc_slots && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
   const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
   const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + p.prefix_len + kTileTokens - 1) / kTileTokens * nreq);
   int lpi = 1;
@@ -1226,7 +1248,7 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
   const memstore_config& c = s->cfg;
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
   // the staged kernel serves the plain parameterisation only (whole-head rotation, bf16 cache)
-  const bool use_tma = s->tma_path && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
+  const bool use_tma = s->tma_path && !s->cc_slots && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
   cudaLaunchConfig_t lc{};
   lc.stream = st;
   cudaLaunchAttribute attr[1];
@@ -1451,6 +1473,15 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->kernels_launched = s->kernels_launched;
   out->arena_bytes = (int64_t)memstore_arena_bytes(&s->cfg);
   out->embedding_bytes = (int64_t)s->cfg.n_users * s->cfg.max_facts_per_user * s->cfg.emb_dim * (int64_t)emb_elem_size(s->cfg.emb_dtype);
+  out->compose_cache_hits = out->compose_cache_fills = 0;
+  out->compose_cache_segments = s->cc_n_slots;
+  if (s->cc_counters) {
+    DeviceGuard g(s->cfg.device);
+    uint32_t cnt[2] = {0, 0};
+    MS_CUDA(s, cudaMemcpy(cnt, s->cc_counters, sizeof cnt, cudaMemcpyDeviceToHost));
+    out->compose_cache_hits = cnt[0];
+    out->compose_cache_fills = cnt[1];
+  }
   out->kernel_timeouts = 0;
   out->filter_fixups = 0;
   out->filter_fixup_overflows = 0;
@@ -1464,6 +1495,48 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
     out->filter_fixup_overflows = flags[1];
     out->filter_fixups = fix;
   }
+  return MS_OK;
+}
+
+ms_status memstore_compose_cache(memstore_t* s, size_t budget_bytes, int32_t max_tokens_per_segment, uint32_t flags) {
+  Range range("memstore_compose_cache");
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (flags & ~(uint32_t)MS_COMPOSE_CACHE_ALL) return fail(s, MS_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  DeviceGuard g(c.device);
+  MS_CUDA(s, cudaDeviceSynchronize());
+  cudaFree(s->cc_slots);
+  cudaFree(s->cc_arena);
+  cudaFree(s->cc_counters);
+  s->cc_slots = nullptr;
+  s->cc_arena = nullptr;
+  s->cc_counters = nullptr;
+  s->cc_n_slots = s->cc_slot_tokens = 0;
+  if (budget_bytes == 0) return MS_OK;
+  if (max_tokens_per_segment <= 0) return fail(s, MS_ERR_INVALID_ARG, "max_tokens_per_segment must be positive");
+  const size_t tok_bytes = (size_t)2 * c.n_layers * c.n_kv_heads * c.head_dim * sizeof(__nv_bfloat16);
+  const size_t seg_bytes = tok_bytes * (size_t)max_tokens_per_segment;
+  const int64_t n_slots = std::min<int64_t>(kCcMaxSlots, (int64_t)(budget_bytes / seg_bytes));
+  if (n_slots < 1) return fail(s, MS_ERR_INVALID_ARG, "a budget of %zu bytes holds no segment of %d tokens (%zu bytes)", budget_bytes, max_tokens_per_segment, seg_bytes);
+  if (n_slots * max_tokens_per_segment >= (int64_t)kCacheTierBit) return fail(s, MS_ERR_UNSUPPORTED, "composition cache of 2^29 tokens or more");
+  if (cudaMalloc(&s->cc_arena, (size_t)n_slots * seg_bytes) != cudaSuccess || cudaMalloc(&s->cc_slots, (size_t)n_slots * sizeof(CcSlot)) != cudaSuccess ||
+      cudaMalloc(&s->cc_counters, 2 * sizeof(uint32_t)) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(s->cc_slots);
+    cudaFree(s->cc_arena);
+    cudaFree(s->cc_counters);
+    s->cc_slots = nullptr;
+    s->cc_arena = nullptr;
+    s->cc_counters = nullptr;
+    return fail(s, MS_ERR_OOM, "composition cache of %lld segments", (long long)n_slots);
+  }
+  MS_CUDA(s, cudaMemset(s->cc_slots, 0, (size_t)n_slots * sizeof(CcSlot)));  // epoch 0: every slot is empty
+  MS_CUDA(s, cudaMemset(s->cc_counters, 0, 2 * sizeof(uint32_t)));
+  s->cc_n_slots = (int32_t)n_slots;
+  s->cc_slot_tokens = max_tokens_per_segment;
+  s->cc_fill_all = (flags & MS_COMPOSE_CACHE_ALL) ? 1 : 0;
+  s->cc_epoch++;
   return MS_OK;
 }
 

@@ -132,6 +132,58 @@ def measure_host_tier(iters: int, seed: int = 0, n_facts: int = 400, ks=(5, 10, 
     return lines
 
 
+def measure_compose_cache(iters: int, seed: int = 0, n_facts: int = 400, ks=(5, 10, 20, 50)):
+    """Host-tier store of the Llama-3.1-8B KV shape: a request composed from pinned host memory (miss: rows cross PCIe)
+    against the same request repeated with the composition cache on (hit: an HBM-rate copy of the cached segment)."""
+    s = synth.CONFIGS["llama8b"]
+    dev = torch.device("cuda")
+    lens = synth.fact_lengths(seed, n_facts, s.len_lo, s.len_hi)
+    emb = synth.embeddings(seed, n_facts, s.emb_dim, s.emb_dtype)
+    T = int(lens.sum())
+    store = M.MemStore(n_layers=s.n_layers, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, emb_dim=s.emb_dim,
+                       rope_theta=s.rope_theta, max_facts_per_user=n_facts, max_kv_tokens=0, max_host_kv_tokens=T)  # fmt: skip
+    g = torch.Generator().manual_seed(seed)
+    for a in range(0, n_facts, 50):
+        b = min(n_facts, a + 50)
+        t = int(lens[a:b].sum())
+        kv = torch.randn((2, s.n_layers, t, s.n_kv_heads, s.head_dim), generator=g, dtype=torch.float32).to(torch.bfloat16)
+        store.add_facts_host(torch.from_numpy(emb[a:b]).to(dev), lens[a:b], kv[0].contiguous(), kv[1].contiguous())
+    lines = []
+    rng = np.random.default_rng(seed)
+    stream = torch.cuda.current_stream()
+    for k in ks:
+        per_req = workload.blocks_per_request(s, k)
+        cache = M.PagedCache.allocate(s.n_layers, max(1024, per_req * 4), s.block_size, s.n_kv_heads, s.head_dim, dev)
+        tables = torch.from_numpy(synth.block_tables(seed, cache.num_blocks, per_req, 4)).to(dev)
+        ids = torch.from_numpy(rng.choice(n_facts, k, replace=False).astype(np.int32)[None]).to(dev)
+        m = int(lens[ids.cpu().numpy()[0]].sum())
+        start = torch.full((1,), s.start_pos, dtype=torch.int32, device=dev)
+
+        def timed(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(n):
+                store.inject(ids, start, tables[i % 4 : i % 4 + 1], cache, flags=M.INJECT_REVERSE, stream=stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / n
+
+        store.compose_cache(0)
+        timed(2)
+        miss_us = timed(max(2, iters // 4))
+        store.compose_cache(2 * k * s.len_hi * s.token_bytes, k * s.len_hi)
+        fill_us = timed(1)  # the first repetition records the segment
+        hit_us = timed(iters)
+        st = store.stats()
+        lines.append({"config": "llama8b host tier, repeated request", "k": k, "tokens": m, "miss_us": miss_us, "recording_miss_us": fill_us,
+                      "hit_us": hit_us, "hit_gbs": 2.0 * m * s.token_bytes / (hit_us * 1e-6) / 1e9, "hits": st["compose_cache_hits"],
+                      "fills": st["compose_cache_fills"]})  # fmt: skip
+        del cache
+    store.close()
+    return lines
+
+
 def measure_permuted_chunks(iters: int, seed: int = 0, sizes=(1024, 2048, 4096, 8192, 16384, 32768), chunk: int = 64):
     """The shape of the paper's chunk-order experiment (appendix "Position independence and rotation fidelity") on the
     Llama-3.1-8B KV shape: fixed 64-token chunks injected
@@ -425,6 +477,7 @@ if __name__ == "__main__":
     ap.add_argument("--hot-per-user", type=int, default=None)
     ap.add_argument("--pool-blocks", type=int, default=None)
     ap.add_argument("--retrieve-only", action="store_true", help="embedding-only store, time the batched retrieval alone")
+    ap.add_argument("--compose-cache", action="store_true", help="Llama shape, host-tier store: a repeated request with and without the composition cache")
     ap.add_argument("--host-tier", action="store_true", help="Llama shape with all K/V in the pinned host arena: inject over PCIe")
     ap.add_argument("--variants", action="store_true", help="Llama shape: bf16 cache, e4m3 cache, partial rotary (inject only)")
     ap.add_argument("--ann", type=int, default=0, metavar="ROWS", help="graph index on ROWS structured embedding rows")
@@ -438,6 +491,9 @@ if __name__ == "__main__":
             print(json.dumps(ln))
     elif a.variants:
         for ln in measure_variants(a.iters, a.seed):
+            print(json.dumps(ln))
+    elif a.compose_cache:
+        for ln in measure_compose_cache(a.iters, a.seed):
             print(json.dumps(ln))
     elif a.host_tier:
         for ln in measure_host_tier(a.iters, a.seed):

@@ -25,6 +25,7 @@ INJECT_REVERSE = 1
 INJECT_PREFIX = 2
 RETRIEVE_ANN = 4
 INPUTS_STABLE = 8
+COMPOSE_CACHE_ALL = 1
 CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 STORE_TMA_COPY_PATH = 1
 REQ_KERNEL_TIMEOUT = 32
@@ -63,7 +64,7 @@ class _AnnParams(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "filter_fixup_overflows")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "compose_cache_hits", "compose_cache_fills", "compose_cache_segments", "filter_fixup_overflows")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares
@@ -73,7 +74,7 @@ EXPORTS = (
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
     "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
-    "memstore_test_hooks", "memstore_reserve",
+    "memstore_test_hooks", "memstore_reserve", "memstore_compose_cache",
 )  # fmt: skip
 
 _lib = None
@@ -110,6 +111,8 @@ def load_library() -> C.CDLL:
     L.memstore_build_graph.argtypes = [vp, i32, vp]
     L.memstore_graph_append.restype = i32
     L.memstore_graph_append.argtypes = [vp, vp]
+    L.memstore_compose_cache.restype = i32
+    L.memstore_compose_cache.argtypes = [vp, C.c_size_t, C.c_int32, C.c_uint32]
     L.memstore_reserve.restype = i32
     L.memstore_reserve.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_int32]
     L.memstore_test_hooks.restype = i32
@@ -354,6 +357,10 @@ class MemStore:
     def build_graph(self, degree=64, stream=None) -> None:
         """Exact neighbour graph of all facts present (single-segment stores), built on the device."""
         self._check(self._lib.memstore_build_graph(self._h, degree, _stream_ptr(stream)))
+
+    def compose_cache(self, budget_bytes: int, max_tokens_per_segment: int = 0, cache_all: bool = False) -> None:
+        """Keep composed segments of earlier requests in HBM (``budget_bytes`` = 0 switches the cache off)."""
+        self._check(self._lib.memstore_compose_cache(self._h, int(budget_bytes), int(max_tokens_per_segment), COMPOSE_CACHE_ALL if cache_all else 0))
 
     def reserve(self, nq: int = 0, k: int = 0, nreq: int = 0, max_tokens_per_request: int = 0, max_blocks: int = 0) -> None:
         """Allocate every scratch buffer that calls of these sizes need, so that they allocate nothing later."""

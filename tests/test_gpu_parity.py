@@ -752,6 +752,142 @@ def test_host_tier_facts_are_injected_over_pcie_and_mix_with_hbm_facts():
     ms.close()
 
 
+def mixed_tier_store(hs, **kw):
+    """Even facts in HBM, odd facts in the pinned host arena."""
+    T = int(hs.lens.sum())
+    ms = MemStore(n_layers=hs.L, n_kv_heads=hs.H, head_dim=hs.D, emb_dim=hs.emb_dim, rope_theta=5e5, max_facts_per_user=len(hs.lens),
+                  max_kv_tokens=T, max_host_kv_tokens=T, **kw)  # fmt: skip
+    for f in range(len(hs.lens)):
+        t0, t1 = int(hs.offs[f]), int(hs.offs[f] + hs.lens[f])
+        kf, vf = np.ascontiguousarray(hs.k[:, t0:t1]), np.ascontiguousarray(hs.v[:, t0:t1])
+        if f % 2 == 0:
+            ms.add_facts(to_dev(hs.emb[f : f + 1]), [hs.lens[f]], to_dev(kf), to_dev(vf))
+        else:
+            ms.add_facts_host(to_dev(hs.emb[f : f + 1]), [hs.lens[f]], kf, vf)
+    return ms
+
+
+@pytest.mark.parametrize("fp8", [False, True])
+def test_composition_cache_hits_are_byte_identical_to_composing_again(fp8):
+    """A request that repeats an earlier one (same ids, start, flags) is served from the composition cache: the paged
+    cache it fills is byte for byte what composing again writes, and what the oracle says.  Another start position,
+    another order or another flag is a miss; the least recently used segment makes room; multi-request calls only
+    look up; requests without a host-tier fact are not recorded unless asked."""
+    hs = HostStore(70, 24, 3, 4, 128, 5, 30, 128, "float16")
+    ms = mixed_tier_store(hs)
+    tok_bytes = 2 * hs.L * hs.H * hs.D * 2
+    seg_tokens = 4 * 30
+    ms.compose_cache(2 * seg_tokens * tok_bytes + 100, seg_tokens)  # room for two segments
+    assert ms.stats()["compose_cache_segments"] == 2
+    tables = synth.block_tables(71, 96, 12, 4)
+
+    def cache_for():
+        return PagedCache.allocate(hs.L, 96, 16, hs.H, hs.D, DEV, fill_bits=0x5A if fp8 else SENT, fp8=fp8, k_scale=0.3, v_scale=1.7)
+
+    def run(ids, start, table, flags=M.INJECT_REVERSE):
+        c = cache_for()
+        run_inject_and_check(ms, hs, ids, start, table, c, 5e5, flags=flags, sentinel=0x5A if fp8 else SENT)
+        st = ms.stats()
+        return c, st["compose_cache_hits"], st["compose_cache_fills"]
+
+    # the policy, restated here as a model: a request is a hit when its key is held; a miss that names a host-tier fact
+    # is recorded in an empty slot, else in the slot used longest ago
+    model, clock, hits, fills = {}, 0, 0, 0  # key -> last use
+
+    def expect(ids, start, flags):
+        nonlocal clock, hits, fills
+        clock += 1
+        key = (tuple(ids), start, flags)
+        if key in model:
+            hits += 1
+        elif any(i % 2 == 1 for i in ids):
+            fills += 1
+            if len(model) == 2:
+                del model[min(model, key=model.get)]
+        else:
+            return
+        model[key] = clock
+
+    A, B, Cc = [1, 4, 7, 2], [3, 5, 9], [11, 0, 13, 15]
+    c1, h, f = run(A, 9, tables[0])
+    assert (h, f) == (0, 1)  # composed over PCIe and recorded
+    c2, h, f = run(A, 9, tables[1])  # the same request through another block table: a hit
+    assert (h, f) == (1, 1)
+    m, slots1 = oracle.slots(A[::-1], hs.lens, 9, tables[0], 16, 96)
+    _, slots2 = oracle.slots(A[::-1], hs.lens, 9, tables[1], 16, 96)
+    from parity import gather_cache_rows
+
+    k1, v1 = gather_cache_rows(c1, slots1)
+    k2, v2 = gather_cache_rows(c2, slots2)
+    assert np.array_equal(k1, k2) and np.array_equal(v1, v2)  # the hit wrote exactly the bytes of the miss
+    expect(A, 9, M.INJECT_REVERSE)
+    expect(A, 9, M.INJECT_REVERSE)
+    # another start position, the other order, a repeat, other lists, a list without host-tier facts, a repeat again ...
+    for ids, start, flags, tb in ((A, 10, M.INJECT_REVERSE, 0), (A, 9, 0, 2), (A, 9, M.INJECT_REVERSE, 0), (A, 9, M.INJECT_REVERSE, 3),
+                                  (B, 9, M.INJECT_REVERSE, 0), (Cc, 9, M.INJECT_REVERSE, 1), (A, 9, M.INJECT_REVERSE, 3), (B, 9, M.INJECT_REVERSE, 2),
+                                  ([0, 2, 4], 9, M.INJECT_REVERSE, 0), ([0, 2, 4], 9, M.INJECT_REVERSE, 1), (Cc, 9, M.INJECT_REVERSE, 0)):  # fmt: skip
+        _, h, f = run(ids, start, tables[tb], flags=flags)
+        expect(ids, start, flags)
+        assert (h, f) == (hits, fills), (ids, start, flags, h, f, hits, fills)
+    assert hits >= 2 and fills >= 5  # the sequence exercised hits, evictions and refills
+    # make the first request the most recent entry again for the two-request call below
+    _, h, f = run(A, 9, tables[0])
+    expect(A, 9, M.INJECT_REVERSE)
+    run(A, 9, tables[0])
+    expect(A, 9, M.INJECT_REVERSE)
+    # a call with two requests looks both up (one is cached) and records nothing
+    ids2 = to_dev(np.array([[1, 4, 7, 2], [6, 8, 10, 12]], np.int32))
+    caches = cache_for()
+    n_tok, st2 = ms.inject(ids2, to_dev(np.array([9, 9], np.int32)), to_dev(tables[:2]), caches, flags=M.INJECT_REVERSE)
+    torch.cuda.synchronize()
+    st = ms.stats()
+    assert (st["compose_cache_hits"], st["compose_cache_fills"]) == (hits + 1, fills) and int(st2.abs().sum()) == 0
+    k3, v3 = gather_cache_rows(caches, slots1)
+    assert np.array_equal(k3, k1) and np.array_equal(v3, v1)
+    # recording everything, and switching the cache off
+    ms.compose_cache(3 * seg_tokens * tok_bytes, seg_tokens, cache_all=True)
+    _, h, f = run([0, 2, 4], 9, tables[0])
+    _, h, f = run([0, 2, 4], 9, tables[1])
+    assert (h, f) == (1, 1)
+    ms.compose_cache(0)
+    run(A, 9, tables[0])
+    assert ms.stats()["compose_cache_segments"] == 0
+    with pytest.raises(M.MemStoreError):
+        ms.compose_cache(1000, seg_tokens)  # holds no segment
+    ms.close()
+
+
+def test_composition_cache_through_the_one_call_paths():
+    """retrieve_inject and serve_host look the request up with the ids the retrieval has just written on the device."""
+    hs = HostStore(72, 200, 2, 4, 64, 4, 12, 64, "float16")
+    ms = mixed_tier_store(hs)
+    k, bs, nb = 8, 16, 64
+    ms.compose_cache(1 << 24, k * 12)
+    q = to_dev(synth.queries(73, 1, 64, "float16"))
+    start = to_dev(np.array([5], np.int32))
+    tables = synth.block_tables(74, nb, (5 + k * 12) // bs + 1, 2)
+    ref = make_cache(hs, nb, bs)
+    ids, _ = ms.retrieve(q, k)
+    ms.compose_cache(0)
+    ms.inject(ids, start, to_dev(tables[:1]), ref, flags=M.INJECT_REVERSE)
+    ms.compose_cache(1 << 24, k * 12)
+    outs = []
+    for rep in range(3):
+        c = make_cache(hs, nb, bs)
+        ids_b, n_b, st_b = ms.retrieve_inject(q, k, start, to_dev(tables[:1]), c, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        assert torch.equal(ids_b, ids) and int(st_b[0]) == 0
+        assert torch.equal(c.k.view(torch.int16), ref.k.view(torch.int16)) and torch.equal(c.v.view(torch.int16), ref.v.view(torch.int16))
+        outs.append((ms.stats()["compose_cache_hits"], ms.stats()["compose_cache_fills"]))
+    assert outs == [(0, 1), (1, 1), (2, 1)]
+    out = np.full(k + 2, -5, np.int32)
+    c = make_cache(hs, nb, bs)
+    ms.serve_host(q[0].cpu().numpy(), k, 5, tables[0], c, out, flags=M.INJECT_REVERSE)
+    assert ms.stats()["compose_cache_hits"] == 3 and out[:k].tolist() == ids[0].cpu().tolist()
+    assert torch.equal(c.k.view(torch.int16), ref.k.view(torch.int16))
+    ms.close()
+
+
 def test_serve_host_matches_the_device_calls():
     """memstore_serve_host (host buffers in, host results out) against retrieve + inject on device buffers."""
     hs = HostStore(19, 120, 2, 8, 128, 8, 40, 256, "float16", n_users=2)
