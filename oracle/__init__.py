@@ -90,6 +90,12 @@ def lib() -> C.CDLL:
                      "oracle_e4m3_to_double"):  # fmt: skip
             getattr(L, name).restype = None
             getattr(L, name).argtypes = [p, i64, p]
+        L.oracle_retrieve_masked.restype = i32
+        L.oracle_retrieve_masked.argtypes = [p, i32, i64, i32, p, p, p, i32, i32, p, p, i32]
+        L.oracle_knn_graph_masked.restype = i32
+        L.oracle_knn_graph_masked.argtypes = [p, i32, i64, i32, i32, p, p, i32]
+        L.oracle_ann_search_masked.restype = i32
+        L.oracle_ann_search_masked.argtypes = [p, i32, i64, i32, p, i32, p, i32, i32, i32, i32, i32, i32, p, p, p, p, p, p]
         L.oracle_e4m3_from_scaled_bf16.restype = None
         L.oracle_e4m3_from_scaled_bf16.argtypes = [p, i64, C.c_float, p]
         _lib = L
@@ -174,8 +180,17 @@ def scores(emb: np.ndarray, query: np.ndarray, n_threads: int = 0) -> np.ndarray
     return out
 
 
-def retrieve(emb: np.ndarray, queries: np.ndarray, k: int, row_ids: np.ndarray | None = None, n_threads: int = 0):
-    """Top-k by (score descending, id ascending); returns (ids int32 [nq,k], scores float32 [nq,k])."""
+def _mask(removed, n):
+    if removed is None:
+        return None
+    removed = np.ascontiguousarray(removed).astype(np.uint8)
+    assert removed.size == n
+    return removed
+
+
+def retrieve(emb: np.ndarray, queries: np.ndarray, k: int, row_ids: np.ndarray | None = None, n_threads: int = 0, removed=None):
+    """Top-k by (score descending, id ascending); returns (ids int32 [nq,k], scores float32 [nq,k]).
+    ``removed``: boolean per row; removed rows are never returned."""
     emb = np.ascontiguousarray(emb)
     queries = np.ascontiguousarray(queries, dtype=emb.dtype)
     if queries.ndim == 1:
@@ -187,8 +202,8 @@ def retrieve(emb: np.ndarray, queries: np.ndarray, k: int, row_ids: np.ndarray |
         assert row_ids.size == n
     ids = np.empty((nq, k), dtype=np.int32)
     sc = np.empty((nq, k), dtype=np.float32)
-    rc = lib().oracle_retrieve(
-        _ptr(emb), _emb_dtype(emb), n, e, _ptr(row_ids), _ptr(queries), nq, k, _ptr(ids), _ptr(sc), n_threads
+    rc = lib().oracle_retrieve_masked(
+        _ptr(emb), _emb_dtype(emb), n, e, _ptr(row_ids), _ptr(_mask(removed, n)), _ptr(queries), nq, k, _ptr(ids), _ptr(sc), n_threads
     )
     if rc:
         raise OracleError(rc)
@@ -206,11 +221,13 @@ def scores_f32(emb: np.ndarray, query: np.ndarray) -> np.ndarray:
     return out
 
 
-def knn_graph(emb: np.ndarray, deg: int, n_threads: int = 0) -> np.ndarray:
-    """Exact k-nearest-neighbour graph by inner product: int32 [n, deg], best first, -1 padded."""
+def knn_graph(emb: np.ndarray, deg: int, n_threads: int = 0, removed=None) -> np.ndarray:
+    """Exact k-nearest-neighbour graph by inner product: int32 [n, deg], best first, -1 padded; ``removed`` rows are
+    nobody's neighbours."""
     emb = np.ascontiguousarray(emb)
     out = np.empty((emb.shape[0], deg), dtype=np.int32)
-    rc = lib().oracle_knn_graph(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], deg, _ptr(out), n_threads)
+    rc = lib().oracle_knn_graph_masked(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], deg, _ptr(_mask(removed, emb.shape[0])),
+                                       _ptr(out), n_threads)  # fmt: skip
     if rc:
         raise OracleError(rc)
     return out
@@ -236,7 +253,7 @@ class AnnResult:
 
 
 def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, beam: int = 64, parents: int = 8,
-               n_entry: int = 64, max_iters: int = 32, exact: bool = False) -> AnnResult:  # fmt: skip
+               n_entry: int = 64, max_iters: int = 32, exact: bool = False, removed=None) -> AnnResult:  # fmt: skip
     """Beam search over ``graph`` for each query: ids / scores [nq, k], steps taken and rows scored per query.
     ``exact``: rank by the double-precision inner products (and report the decision margin of every query) instead of
     the binary32 lane sums."""
@@ -249,8 +266,20 @@ def ann_search(emb: np.ndarray, graph: np.ndarray, queries: np.ndarray, k: int, 
     iters = np.zeros(nq, dtype=np.int32)
     scored = np.zeros(nq, dtype=np.int64)
     margin = np.full(nq, np.inf) if exact else None
+    removed = _mask(removed, emb.shape[0])
     for q in range(nq):
         it, ns = C.c_int32(0), C.c_int64(0)
+        if removed is not None:
+            mg = C.c_double(0.0)
+            rc = lib().oracle_ann_search_masked(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(graph), graph.shape[1],
+                                                _ptr(queries[q]), k, beam, parents, n_entry, max_iters, int(exact), _ptr(removed),
+                                                _ptr(ids[q]), _ptr(sc[q]), C.byref(it), C.byref(ns), C.byref(mg))  # fmt: skip
+            if rc:
+                raise OracleError(rc)
+            iters[q], scored[q] = it.value, ns.value
+            if exact:
+                margin[q] = mg.value
+            continue
         if exact:
             mg = C.c_double(0.0)
             rc = lib().oracle_ann_search_exact(_ptr(emb), _emb_dtype(emb), emb.shape[0], emb.shape[1], _ptr(graph), graph.shape[1],

@@ -233,8 +233,24 @@ static int cmp_scored(const void* a, const void* b) {
  * when there are fewer than k facts.  row_ids[f] is the fact id of embedding row f
  * (NULL: the row index is the id).
  */
+int oracle_retrieve_masked(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim, const int32_t* row_ids,
+                           const uint8_t* removed, const void* queries, int nq, int k, int32_t* out_ids, float* out_scores,
+                           int n_threads);
+
 int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim, const int32_t* row_ids,
                     const void* queries, int nq, int k, int32_t* out_ids, float* out_scores, int n_threads) {
+  return oracle_retrieve_masked(emb, emb_dtype, n_facts, emb_dim, row_ids, NULL, queries, nq, k, out_ids, out_scores, n_threads);
+}
+
+/*
+ * The same with removed facts (the paper names deleting and revising facts as future work, "with consistent updates to
+ * both the index and the pre-RoPE KV store"; the rule here is the plain one): removed[f] != 0 takes row f out of the
+ * search - it is never returned, whatever its score - and everything else is as before: the facts that remain are
+ * sorted by (score desc, id asc), the first k are returned, -1 / 0 pad when fewer remain.
+ */
+int oracle_retrieve_masked(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim, const int32_t* row_ids,
+                           const uint8_t* removed, const void* queries, int nq, int k, int32_t* out_ids, float* out_scores,
+                           int n_threads) {
   if (nq < 0 || k < 0 || !out_ids) return ORACLE_ERR_ARG;
   if (n_facts > 0 && (!emb || !queries)) return ORACLE_ERR_ARG;
   size_t esz = emb_dtype == ORACLE_F32 ? 4 : 2;
@@ -255,13 +271,16 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
         return rc;
       }
     }
+    int64_t n_left = 0;
     for (int64_t f = 0; f < n_facts; ++f) {
-      all[f].s = s[f];
-      all[f].id = row_ids ? row_ids[f] : (int32_t)f;
+      if (removed && removed[f]) continue;
+      all[n_left].s = s[f];
+      all[n_left].id = row_ids ? row_ids[f] : (int32_t)f;
+      ++n_left;
     }
-    qsort(all, (size_t)n_facts, sizeof(scored_t), cmp_scored);
+    qsort(all, (size_t)n_left, sizeof(scored_t), cmp_scored);
     for (int r = 0; r < k; ++r) {
-      if (r < n_facts) {
+      if (r < n_left) {
         out_ids[(size_t)q * k + r] = all[r].id;
         if (out_scores) out_scores[(size_t)q * k + r] = (float)all[r].s;
       } else {
@@ -293,7 +312,8 @@ int oracle_retrieve(const void* emb, int emb_dtype, int64_t n_facts, int emb_dim
  *   step     take the first `parents` unexpanded entries of the list in list order (stop when there is none, or
  *            after max_iters steps), mark them expanded; collect their neighbours that are valid rows and
  *            not in V, add them to V, score them, and keep the best L of list + new.
- *   result   the first k entries of the list; -1 / 0 pads.
+ *   result   the first k entries of the list; -1 / 0 pads.  With removed rows: they walk along like any other row
+ *            (scored, listed, expanded) and are passed over when the result is read out.
  */
 
 /*
@@ -336,7 +356,15 @@ int oracle_scores_f32(const void* emb, int emb_dtype, int64_t n_rows, int emb_di
 }
 
 /* Exact k-nearest-neighbour graph by inner product (double scores, full sort per row). */
+int oracle_knn_graph_masked(const void* emb, int emb_dtype, int64_t n, int emb_dim, int deg, const uint8_t* removed, int32_t* out_graph,
+                            int n_threads);
 int oracle_knn_graph(const void* emb, int emb_dtype, int64_t n, int emb_dim, int deg, int32_t* out_graph, int n_threads) {
+  return oracle_knn_graph_masked(emb, emb_dtype, n, emb_dim, deg, NULL, out_graph, n_threads);
+}
+/* A graph built after removals: removed rows are nobody's neighbours (a removed row still gets a list of its own, so
+ * that a walk that reaches it through an older edge can go on). */
+int oracle_knn_graph_masked(const void* emb, int emb_dtype, int64_t n, int emb_dim, int deg, const uint8_t* removed, int32_t* out_graph,
+                            int n_threads) {
   if (!emb || !out_graph || n < 0 || deg <= 0 || emb_dim <= 0) return ORACLE_ERR_ARG;
   size_t esz = emb_dtype == ORACLE_F32 ? 4 : 2;
   int rc_all = ORACLE_OK;
@@ -351,7 +379,7 @@ int oracle_knn_graph(const void* emb, int emb_dtype, int64_t n, int emb_dim, int
     const char* q = (const char*)emb + (size_t)r * emb_dim * esz;
     int64_t m = 0;
     for (int64_t f = 0; f < n; ++f) {
-      if (f == r) continue;
+      if (f == r || (removed && removed[f])) continue;
       double sc = 0.0;
       for (int d = 0; d < emb_dim; ++d) sc += emb_at(q, emb_dtype, d) * emb_at(emb, emb_dtype, f * emb_dim + d);
       all[m].s = sc;
@@ -484,8 +512,8 @@ static double step_margin(const beam_t* list, int len, int L, const void* emb, s
 
 static int ann_search_core(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
                            const void* query, int k, int beam, int parents, int n_entry, int max_iters, int exact,
-                           int32_t* out_ids, float* out_scores, int32_t* out_iters, int64_t* out_scored,
-                           double* out_margin) {
+                           const uint8_t* removed, int32_t* out_ids, float* out_scores, int32_t* out_iters,
+                           int64_t* out_scored, double* out_margin) {
   if (!out_ids || k <= 0 || beam <= 0 || parents <= 0 || n_entry <= 0 || max_iters < 0 || deg <= 0 || n < 0 ||
       emb_dim <= 0 || emb_dim % 8)
     return ORACLE_ERR_ARG;
@@ -545,9 +573,18 @@ static int ann_search_core(const void* emb, int emb_dtype, int64_t n, int emb_di
       if (len > L) len = L;
     }
   }
-  for (int r = 0; r < k; ++r) {
-    out_ids[r] = r < len ? list[r].row : -1;
-    if (out_scores) out_scores[r] = r < len ? (float)list[r].s : 0.0f;
+  /* result: the first k entries of the list; a removed row takes part in the walk like any other (its edges still lead
+   * somewhere) but is passed over here, so it is never returned */
+  int w = 0;
+  for (int i = 0; i < len && w < k; ++i) {
+    if (removed && removed[list[i].row]) continue;
+    out_ids[w] = list[i].row;
+    if (out_scores) out_scores[w] = (float)list[i].s;
+    ++w;
+  }
+  for (; w < k; ++w) {
+    out_ids[w] = -1;
+    if (out_scores) out_scores[w] = 0.0f;
   }
   if (out_iters) *out_iters = iters;
   if (out_scored) *out_scored = scored;
@@ -565,7 +602,7 @@ static int ann_search_core(const void* emb, int emb_dtype, int64_t n, int emb_di
 int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
                       const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
                       float* out_scores, int32_t* out_iters, int64_t* out_scored) {
-  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 0, out_ids,
+  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 0, NULL, out_ids,
                          out_scores, out_iters, out_scored, NULL);
 }
 
@@ -579,8 +616,17 @@ int oracle_ann_search(const void* emb, int emb_dtype, int64_t n, int emb_dim, co
 int oracle_ann_search_exact(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
                             const void* query, int k, int beam, int parents, int n_entry, int max_iters, int32_t* out_ids,
                             float* out_scores, int32_t* out_iters, int64_t* out_scored, double* out_margin) {
-  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 1, out_ids,
+  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, 1, NULL, out_ids,
                          out_scores, out_iters, out_scored, out_margin);
+}
+
+/* Both forms with removed rows (removed[row] != 0, or NULL): exact != 0 ranks by the double scores and reports the margin. */
+int oracle_ann_search_masked(const void* emb, int emb_dtype, int64_t n, int emb_dim, const int32_t* graph, int deg,
+                             const void* query, int k, int beam, int parents, int n_entry, int max_iters, int exact,
+                             const uint8_t* removed, int32_t* out_ids, float* out_scores, int32_t* out_iters,
+                             int64_t* out_scored, double* out_margin) {
+  return ann_search_core(emb, emb_dtype, n, emb_dim, graph, deg, query, k, beam, parents, n_entry, max_iters, exact, removed,
+                         out_ids, out_scores, out_iters, out_scored, out_margin);
 }
 
 /* ---------------------------------------------------------------- RoPE */

@@ -240,3 +240,88 @@ def test_graph_append_rule(oracle_mod):
     assert np.array_equal(oracle_mod.graph_append(emb[:n_old], old), old)
     # a store that starts empty: append equals build
     assert np.array_equal(oracle_mod.graph_append(emb[:50], np.zeros((0, deg), np.int32)), oracle_mod.knn_graph(emb[:50], deg))
+
+
+# ------------------------------------------------------------------------------------------------ removed rows
+def test_retrieval_with_removed_rows_is_retrieval_over_the_rows_that_remain(oracle_mod):
+    """Masked retrieval reduces to the pinned plain routine on the compacted matrix with its row -> id map, and to a
+    brute-force numpy ranking; removed rows never appear, ties still go to the lower id, short stores are padded."""
+    rng = np.random.default_rng(8)
+    for dtype, dim, n in (("float32", 64, 500), ("float16", 136, 300)):
+        emb = synth.embeddings(8, n, dim, dtype)
+        emb[200] = emb[17]
+        emb[250] = emb[17]
+        q = synth.queries(8, 3, dim, dtype)
+        q[0] = emb[17]
+        removed = rng.random(n) < 0.3
+        removed[17] = True  # the best match of query 0 is gone: its copies move up, lower id first
+        removed[[200, 250]] = False
+        keep = np.flatnonzero(~removed)
+        for k in (1, 7, len(keep), len(keep) + 5):
+            ids, sc = oracle_mod.retrieve(emb, q, k, removed=removed)
+            want_ids, want_sc = oracle_mod.retrieve(emb[keep], q, k, row_ids=keep.astype(np.int32))
+            assert np.array_equal(ids, want_ids) and np.array_equal(sc, want_sc)
+            assert not np.isin(ids[ids >= 0], np.flatnonzero(removed)).any()
+        ids, _ = oracle_mod.retrieve(emb, q, 5, removed=removed)
+        assert ids[0, :2].tolist() == [200, 250]
+        s = emb.astype(np.float64) @ q[1].astype(np.float64)
+        s[removed] = -np.inf
+        order = np.lexsort((np.arange(n), -s))[:5]
+        assert np.array_equal(oracle_mod.retrieve(emb, q[1:2], 5, removed=removed)[0][0], order)
+    everything = np.ones(20, bool)
+    ids, sc = oracle_mod.retrieve(emb[:20], q[:1], 3, removed=everything)
+    assert ids.tolist() == [[-1, -1, -1]] and sc.tolist() == [[0.0, 0.0, 0.0]]
+
+
+@pytest.mark.parametrize("exact", [False, True])
+def test_search_walks_through_removed_rows_but_never_returns_them(oracle_mod, exact):
+    # the path graph of the hand-followed walk: rows 64..66, on the way from the entry 61 to the target 70, are removed;
+    # the walk still gets to 70 through them (same steps, same rows scored), and they are missing from the result
+    n = 100
+    emb = arc(n)
+    path = np.array([[i - 1 if i > 0 else -1, i + 1 if i + 1 < n else -1] for i in range(n)], np.int32)
+    q = emb[70:71].copy()
+    removed = np.zeros(n, bool)
+    removed[[64, 65, 66]] = True
+    plain = oracle_mod.ann_search(emb, path, q, 4, beam=8, parents=1, n_entry=1, max_iters=50, exact=exact)
+    gone = oracle_mod.ann_search(emb, path, q, 4, beam=8, parents=1, n_entry=1, max_iters=50, exact=exact, removed=removed)
+    assert gone.iters[0] == plain.iters[0] and gone.scored[0] == plain.scored[0]
+    assert gone.ids[0, 0] == 70 and not np.isin(gone.ids[0], [64, 65, 66]).any()
+    # removing the target itself: the next best rows are returned
+    removed[70] = True
+    res = oracle_mod.ann_search(emb, path, q, 2, beam=8, parents=1, n_entry=1, max_iters=50, exact=exact, removed=removed)
+    assert sorted(res.ids[0].tolist()) == [69, 71]
+    # complete graph and a list as long as the store: the walk sees every row, so the result is the masked exact ranking
+    m, dim, k = 120, 64, 9
+    e2 = synth.embeddings(9, m, dim, "float32")
+    complete = np.array([[c for c in range(m) if c != r] for r in range(m)], np.int32)
+    q2 = synth.queries(9, 3, dim, "float32")
+    rem2 = np.random.default_rng(9).random(m) < 0.25
+    res = oracle_mod.ann_search(e2, complete, q2, k, beam=m, parents=4, n_entry=m, max_iters=3, exact=exact, removed=rem2)
+    want, _ = oracle_mod.retrieve(e2, q2, k, removed=rem2)
+    assert np.array_equal(res.ids, want)
+    # a list shorter than the removed rows in front: fewer than k rows can be returned, the rest is padding
+    rem3 = np.zeros(m, bool)
+    best = oracle_mod.retrieve(e2, q2[:1], 6)[0][0]
+    rem3[best[:5]] = True
+    res = oracle_mod.ann_search(e2, complete, q2[:1], 4, beam=6, parents=4, n_entry=m, max_iters=3, exact=exact, removed=rem3)
+    assert res.ids[0].tolist() == [int(best[5]), -1, -1, -1]
+
+
+def test_recall_after_removing_a_tenth_of_the_rows(oracle_mod):
+    n, dim, k = 3000, 64, 10
+    emb = synth.embeddings_low_rank(10, n, dim, "float32", intrinsic_dim=8)
+    g = oracle_mod.knn_graph(emb, 16)
+    q = synth.queries_near_rows(10, emb, 20)
+    removed = np.random.default_rng(10).random(n) < 0.1
+    want, _ = oracle_mod.retrieve(emb, q, k, removed=removed)
+    got = oracle_mod.ann_search(emb, g, q, k, beam=96, parents=2, n_entry=16, max_iters=200, removed=removed).ids
+    assert not np.isin(got[got >= 0], np.flatnonzero(removed)).any()
+    recall = np.mean([len(set(got[i]) & set(want[i])) / k for i in range(len(q))])
+    assert recall > 0.9
+    # a graph built after the removals lists no removed row; removed rows keep lists of their own
+    g2 = oracle_mod.knn_graph(emb, 16, removed=removed)
+    assert not np.isin(g2, np.flatnonzero(removed)).any() and np.all(g2[np.flatnonzero(removed)[0]] >= 0)
+    keep = np.flatnonzero(~removed)
+    sub = oracle_mod.knn_graph(emb[keep], 16)
+    assert np.array_equal(g2[keep[5]], keep[sub[5]])  # an alive row's list = its list in the compacted store
