@@ -222,8 +222,11 @@ ms_status memstore_retrieve_static(memstore_t* store, const void* queries, const
  *           list expanded, scores their neighbours that were never scored before, and keeps the best; it ends
  *           when no unexpanded row is left or after max_iters steps.  Scores are the fp32 sums of
  *           memstore_retrieve, so a result differs from the exact one only in which rows were looked at.
- * Single-segment stores (n_users = 1) only; rows are fact ids there.  The graph covers the facts present when it
- * was built or set: facts added later are not found until it is rebuilt.
+ * Every user segment has a graph of its own (the evaluation keeps one index per conversation, Sec. 6.7): rows of a
+ * user's graph are rows of that user's segment (= fact ids in a single-segment store), all graphs share one degree, and
+ * a query searches the graph of its user.  A graph covers the facts present when it was built, set or last grown
+ * (memstore_graph_append): facts added later are not found until then.  A removed fact (memstore_remove_fact) stays
+ * in the graph: a walk goes through it like through any row and passes it over when the result is read out.
  */
 typedef struct {
   int32_t beam;      /* list length (the result needs max(beam, k) <= 256); 0 = 64 */
@@ -233,8 +236,9 @@ typedef struct {
                         (about 39,000 rows for 1024-d embeddings); 0 = 32 */
 } ms_ann_params;
 
-/* Build the graph of all facts present (degree <= 255); replaces an earlier graph.  Synchronises the device once
- * (allocation), then enqueues the retrieval calls on `stream`. */
+/* Build the graphs of all segments from the facts present (degree <= 255); replaces earlier graphs.  Removed facts
+ * are nobody's neighbours in a graph built after their removal.  Synchronises the device once (allocation), then
+ * enqueues the retrieval calls on `stream`. */
 ms_status memstore_build_graph(memstore_t* store, int32_t degree, ms_stream stream);
 /*
  * Grow the graph for the facts added since it was built, set or last grown (the paper names online insertion as future
@@ -245,20 +249,45 @@ ms_status memstore_build_graph(memstore_t* store, int32_t degree, ms_stream stre
  * (allocation of the larger graph).  No-op when nothing was added; MS_ERR_INVALID_ARG when there is no graph.
  */
 ms_status memstore_graph_append(memstore_t* store, ms_stream stream);
-/* Install a caller-made graph: device int32 [n_rows][degree], entries are rows of the segment (others are ignored
- * by the search), n_rows <= number of facts.  Copied on `stream`. */
+/* Install a caller-made graph for user 0: device int32 [n_rows][degree], entries are rows of the segment (others are
+ * ignored by the search), n_rows <= number of facts of the segment.  Copied on `stream`.  memstore_set_graph_user does
+ * the same for any user; a degree other than the store's current one starts every segment's graph over. */
 ms_status memstore_set_graph(memstore_t* store, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream);
+ms_status memstore_set_graph_user(memstore_t* store, int32_t user, const int32_t* graph, int64_t n_rows, int32_t degree,
+                                  ms_stream stream);
 /* Copy the graph out: out = device int32 buffer of out_capacity entries or NULL; *out_rows, *out_degree (host,
  * optional) receive its shape.  MS_ERR_CAPACITY when the buffer is too small. */
 ms_status memstore_get_graph(memstore_t* store, int32_t* out, int64_t out_capacity, int64_t* out_rows, int32_t* out_degree,
                              ms_stream stream);
+ms_status memstore_get_graph_user(memstore_t* store, int32_t user, int32_t* out, int64_t out_capacity, int64_t* out_rows,
+                                  int32_t* out_degree, ms_stream stream);
 /*
  * The search.  queries: device [nq][emb_dim]; params NULL = defaults; out_ids device int32 [nq][k] (best first, -1
  * padded), out_scores device fp32 [nq][k] or NULL, out_counters device int32 [nq][2] or NULL: steps taken and rows
- * scored per query.  One CTA per query; asynchronous on `stream`.
+ * scored per query.  One thread-block cluster per query; asynchronous on `stream`.  memstore_retrieve_ann searches user
+ * 0's graph for every query; memstore_retrieve_ann_users takes query_users (device int32 [nq], or NULL = user 0) and
+ * returns fact ids of the query's user.
  */
 ms_status memstore_retrieve_ann(memstore_t* store, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
                                 int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream);
+ms_status memstore_retrieve_ann_users(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                                      const ms_ann_params* params, int32_t* out_ids, float* out_scores, int32_t* out_counters,
+                                      ms_stream stream);
+
+/*
+ * Take a fact out of the store (the paper names "incrementally inserting, revising, and deleting facts, with consistent
+ * updates to both the index and the pre-RoPE KV store" as future work; insertion is memstore_add_fact(s) +
+ * memstore_graph_append, revision is removal + insertion, and the removal rule is this library's):
+ *   - exact retrieval, on every kernel path, never returns the fact again (it scores minus infinity; a list that would
+ *     reach it because fewer than k facts are left is padded with -1 instead);
+ *   - the graph search still walks through its row (its edges lead on) but passes it over when the result is read out;
+ *   - memstore_inject treats its id like that of a fact without K/V: MS_REQ_NOT_RESIDENT, no tokens;
+ *   - composed segments in the composition cache are dropped.
+ * The id is not reused and the fact's arena tokens and embedding row are not reclaimed (the store stays append-only
+ * underneath).  Enqueued on `stream`, ordered after earlier calls on the store.  MS_ERR_INVALID_ARG for an unknown id
+ * or one removed before.
+ */
+ms_status memstore_remove_fact(memstore_t* store, int32_t fact_id, ms_stream stream);
 
 /* element type of the paged cache */
 enum {
@@ -333,7 +362,7 @@ ms_status memstore_set_prefix(memstore_t* store, const void* k_pre, const void* 
  * retrieval kernel, so that the whole path is two launches (Sec. 3.3: search, compose and scatter per request).
  * Arguments as in the two calls; out_ids [nq][k] is both the retrieval output and the injection input.
  * With MS_RETRIEVE_ANN in flags the ids come from the graph search (the paper's own pipeline: index search, compose,
- * scatter), followed by the planning and copy kernels; query_users must then be NULL and k <= 256.
+ * scatter), followed by the planning and copy kernels; k <= 256.
  */
 ms_status memstore_retrieve_inject(memstore_t* store, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
                                    const int32_t* start_pos, const int32_t* block_tables, int32_t max_blocks,
@@ -366,6 +395,7 @@ typedef struct {
   int64_t kernel_timeouts; /* 1 if a bounded wait inside the tensor-core scoring kernel ever ran out (results of that call are invalid) */
   int64_t filter_fixups;   /* queries of the tensor-core retrieve path that were re-scanned exactly because the filter's margin
                               check failed (more groups within rounding of the k-th score than the margin keeps) */
+  int64_t n_removed_facts;  /* facts taken out by memstore_remove_fact */
   int64_t compose_cache_hits, compose_cache_fills; /* requests served from / recorded into the composition cache */
   int64_t compose_cache_segments;                  /* segments the composition cache can hold (0: none) */
   int64_t filter_fixup_overflows; /* 1 if such a re-scan ever met more than 4096 rows within rounding of the k-th score: that

@@ -29,15 +29,20 @@ constexpr int kAnnMaxCand = 512;   // rows scored in one step: parents * degree,
 constexpr uint32_t kAnnEmpty = 0xffffffffu;
 
 struct AnnParams {
-  const void* emb;      // [n][E] rows of user 0
-  const int32_t* graph; // [n][deg]
+  const void* emb;      // [n_users][seg_capacity][E]
+  const int32_t* graph; // [n_users][graph_cap_rows][deg]: rows of a user's graph are rows of that user's segment
   const void* queries;  // [nq][E]
-  int32_t n, emb_dim, deg;
+  const int32_t* query_users;  // [nq] or nullptr (user 0)
+  const int32_t* graph_rows;   // [n_users]: rows each user's graph covers
+  const int32_t* emb_fact_id;  // [n_users][seg_capacity] row -> fact id, or nullptr when the row is the id
+  int64_t seg_capacity, graph_cap_rows;
+  int32_t n_users, emb_dim, deg;
   int32_t k, list_len, parents, n_entry, max_iters;
   uint32_t table_mask;  // visited table: table_mask + 1 slots (a power of two, at least twice the rows ever scored)
   int32_t* out_ids;     // [nq][k]
   float* out_scores;    // [nq][k] or nullptr
   int32_t* out_counters;  // [nq][2] or nullptr: steps taken, rows scored
+  const uint32_t* removed_bits;  // one bit per row, or nullptr: removed rows walk along but are passed over in the result
 };
 
 // key of a list entry: order key of the score, then lower row first, lowest bit = not yet expanded
@@ -135,8 +140,13 @@ __global__ void __launch_bounds__(kAnnThreads, 1) ann_search_kernel(const AnnPar
   uint32_t* table = reinterpret_cast<uint32_t*>(dyn + (size_t)p.emb_dim * sizeof(float));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int q = blockIdx.x / csize;
-  const int E = p.emb_dim, n = p.n, L = p.list_len;
-  const T* seg = reinterpret_cast<const T*>(p.emb);
+  const int user_in = p.query_users ? p.query_users[q] : 0;
+  const bool user_ok = user_in >= 0 && user_in < p.n_users;
+  const int user = user_ok ? user_in : 0;
+  const int E = p.emb_dim, n = user_ok ? p.graph_rows[user] : 0, L = p.list_len;
+  const T* seg = reinterpret_cast<const T*>(p.emb) + (int64_t)user * p.seg_capacity * E;
+  const int32_t* graph = p.graph + (int64_t)user * p.graph_cap_rows * p.deg;
+  const int64_t row_base = (int64_t)user * p.seg_capacity;  // of this user's rows in the per-row tables
   const T* qv = reinterpret_cast<const T*>(p.queries) + (int64_t)q * E;
 
   for (int i = tid; i < E; i += kAnnThreads) s_q[i] = (float)qv[i];
@@ -261,7 +271,7 @@ __global__ void __launch_bounds__(kAnnThreads, 1) ann_search_kernel(const AnnPar
         __syncthreads();
         const int n_slots = (int)min(all, (uint32_t)p.parents) * p.deg;
         if (tid < n_slots) {
-          const int32_t nb = __ldg(p.graph + (int64_t)sm.parent[tid / p.deg] * p.deg + tid % p.deg);
+          const int32_t nb = __ldg(graph + (int64_t)sm.parent[tid / p.deg] * p.deg + tid % p.deg);
           if (nb >= 0 && nb < n) visit(nb);
         }
         if (tid == 0) sm.steps += 1;
@@ -271,11 +281,38 @@ __global__ void __launch_bounds__(kAnnThreads, 1) ann_search_kernel(const AnnPar
   cluster.sync();  // nobody leaves while another CTA may still read rank 0's shared memory
   if (!master) return;
   const int len = (int)sm.len;
-  for (int r = tid; r < p.k; r += kAnnThreads) {
-    const bool ok = r < len;
-    const unsigned long long key = ok ? sm.list[r] : 0ull;
-    p.out_ids[(int64_t)q * p.k + r] = ok ? ann_key_row(key) : -1;
-    if (p.out_scores) p.out_scores[(int64_t)q * p.k + r] = ok ? key_score((uint32_t)(key >> 32)) : 0.f;
+  auto id_of = [&](int32_t row) { return p.emb_fact_id ? __ldg(p.emb_fact_id + row_base + row) : row; };
+  if (p.removed_bits == nullptr) {
+    for (int r = tid; r < p.k; r += kAnnThreads) {
+      const bool ok = r < len;
+      const unsigned long long key = ok ? sm.list[r] : 0ull;
+      p.out_ids[(int64_t)q * p.k + r] = ok ? id_of(ann_key_row(key)) : -1;
+      if (p.out_scores) p.out_scores[(int64_t)q * p.k + r] = ok ? key_score((uint32_t)(key >> 32)) : 0.f;
+    }
+  } else {
+    // the list entries that have not been removed, in list order (the list holds at most 256 entries: 8 warps)
+    const unsigned long long key = tid < len ? sm.list[tid] : 0ull;
+    const int32_t row = ann_key_row(key);
+    const int64_t grow = row_base + row;
+    const bool keep = tid < len && !((__ldg(p.removed_bits + (grow >> 5)) >> (grow & 31)) & 1u);
+    const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) sm.warp_cnt[warp] = __popc(ballot);
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+    for (int w = 0; w < kAnnMaxList / 32; ++w) {
+      const uint32_t c = sm.warp_cnt[w];
+      before += w < warp ? c : 0u;
+      all += c;
+    }
+    const uint32_t pos = before + __popc(ballot & ((1u << lane) - 1u));
+    if (keep && pos < (uint32_t)p.k) {
+      p.out_ids[(int64_t)q * p.k + pos] = id_of(row);
+      if (p.out_scores) p.out_scores[(int64_t)q * p.k + pos] = key_score((uint32_t)(key >> 32));
+    }
+    for (int r = (int)all + tid; r < p.k; r += kAnnThreads) {
+      p.out_ids[(int64_t)q * p.k + r] = -1;
+      if (p.out_scores) p.out_scores[(int64_t)q * p.k + r] = 0.f;
+    }
   }
   if (p.out_counters && tid == 0) {
     p.out_counters[2 * q] = (int32_t)sm.steps;

@@ -78,11 +78,20 @@ struct memstore {
   std::vector<int64_t> user_count;
   int64_t n_facts = 0, n_resident = 0, kv_tokens_used = 0;
   int32_t max_fact_len = 0;
-  // proximity graph of user 0's rows (memstore_build_graph / memstore_set_graph): [graph_rows][graph_deg]
+  // proximity graphs, one per user segment (memstore_build_graph / memstore_set_graph): [n_users][graph_cap_rows][graph_deg],
+  // rows of a user's graph are rows of that user's segment
   int32_t* graph = nullptr;
-  int64_t graph_rows = 0;
-  int64_t graph_cap_rows = 0;  // rows the graph array has room for (memstore_graph_append grows it geometrically)
+  std::vector<int64_t> graph_rows;  // rows each user's graph covers
+  int32_t* graph_rows_d = nullptr;  // the same on the device, [n_users]
+  int32_t* graph_users_d = nullptr; // scratch: a batch of equal user numbers (queries of one user while building)
+  int64_t graph_cap_rows = 0;  // rows per user the graph array has room for (a single-segment store grows it geometrically)
   int32_t graph_deg = 0;
+  // removed facts (memstore_remove_fact): one bit per embedding row, host mirror and device copy (allocated on first removal)
+  std::vector<uint32_t> removed_bits;
+  uint32_t* removed_bits_d = nullptr;
+  int64_t n_removed = 0;
+  struct IdRun { int32_t first_id, n, user; int64_t slot0; };
+  std::vector<IdRun> id_runs;  // which rows the ids of each add call went to (ids are dense in insertion order)
   int32_t* graph_topk = nullptr;  // build scratch: [64][deg + 1] ids
   size_t graph_topk_cap = 0;      // its size in entries
   unsigned long long* append_pairs = nullptr;  // graph_append scratch: sorted (old row, new row) offers, then their count
@@ -275,7 +284,7 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     if (!make_tmap_rows_f16(&tmap_q, qptr, (uint64_t)nqb, (uint64_t)c.emb_dim, kGemmMaxQ))
       return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the query batch");
     GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes,
-                  s->test_spin_limit, s->test_mute_producers};
+                  s->test_spin_limit, s->test_mute_producers, s->removed_bits_d};
     score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
     MS_CUDA(s, cudaGetLastError());
     select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best);
@@ -344,6 +353,29 @@ void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams
     launch_score_topk_threads<T, kFusedThreadsFew, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
   else
     launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
+}
+
+RetrieveParams retrieve_params(const memstore* s, const void* queries, const int32_t* query_users, int nq, int k, float* scores,
+                               int32_t* out_ids, float* out_scores) {
+  const memstore_config& c = s->cfg;
+  RetrieveParams p{};
+  p.emb = s->emb;
+  p.emb_fact_id = s->emb_fact_id;
+  p.user_count = s->user_count_d;
+  p.seg_capacity = c.max_facts_per_user;
+  p.n_users = c.n_users;
+  p.emb_dim = c.emb_dim;
+  p.queries = queries;
+  p.query_users = query_users;
+  p.nq = nq;
+  p.k = k;
+  p.scores = scores;
+  p.score_stride = c.max_facts_per_user;
+  p.out_ids = out_ids;
+  p.out_scores = out_scores;
+  p.removed_bits = s->removed_bits_d;
+  p.return_rows = 0;
+  return p;
 }
 
 // Scratch that grows on first use.  Each helper synchronises the device only when it really has to allocate;
@@ -580,6 +612,9 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->cc_arena);
     cudaFree(s->cc_counters);
     cudaFree(s->graph);
+    cudaFree(s->graph_rows_d);
+    cudaFree(s->graph_users_d);
+    cudaFree(s->removed_bits_d);
     cudaFree(s->graph_topk);
     cudaFree(s->append_pairs);
     cudaFree(s->dev_stage);
@@ -664,6 +699,7 @@ static ms_status add_facts_tier(memstore_t* s, int32_t user, int64_t n, const vo
     s->kernels_launched++;
   }
   if (out_first_id) *out_first_id = (int32_t)s->n_facts;
+  s->id_runs.push_back(memstore::IdRun{(int32_t)s->n_facts, (int32_t)n, user, slot0});
   s->user_count[user] += n;
   if (s->user_count[user] > s->max_user_count) s->max_user_count = s->user_count[user];
   s->n_facts += n;
@@ -722,9 +758,9 @@ ms_status memstore_set_prefix(memstore_t* s, const void* k_pre, const void* v, i
   return MS_OK;
 }
 
-ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
-                            int32_t* out_ids, float* out_scores, ms_stream stream) {
-  Range range("memstore_retrieve");
+// memstore_retrieve; return_rows != 0 (graph building) writes rows of the user's segment instead of fact ids
+static ms_status retrieve_impl(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k, int32_t* out_ids,
+                               float* out_scores, ms_stream stream, int return_rows) {
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
@@ -743,21 +779,8 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
 
-  RetrieveParams p{};
-  p.emb = s->emb;
-  p.emb_fact_id = s->emb_fact_id;
-  p.user_count = s->user_count_d;
-  p.seg_capacity = c.max_facts_per_user;
-  p.n_users = c.n_users;
-  p.emb_dim = c.emb_dim;
-  p.queries = queries;
-  p.query_users = query_users;
-  p.nq = nq;
-  p.k = k;
-  p.scores = s->scores;
-  p.score_stride = c.max_facts_per_user;
-  p.out_ids = out_ids;
-  p.out_scores = out_scores;
+  RetrieveParams p = retrieve_params(s, queries, query_users, nq, k, s->scores, out_ids, out_scores);
+  p.return_rows = return_rows;
 
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
   if (tc) {
@@ -798,64 +821,129 @@ ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* q
   return mark_last(s, st);
 }
 
+ms_status memstore_retrieve(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                            int32_t* out_ids, float* out_scores, ms_stream stream) {
+  Range range("memstore_retrieve");
+  return retrieve_impl(s, queries, query_users, nq, k, out_ids, out_scores, stream, 0);
+}
+
 // ---- graph index -------------------------------------------------------------------------------------------------
-static ms_status graph_alloc(memstore* s, int64_t n_rows, int32_t degree) {
+// (Re)allocates the graph array for `cap_rows` rows per user; every user's graph is empty afterwards.
+static ms_status graph_alloc(memstore* s, int64_t cap_rows, int32_t degree) {
+  const memstore_config& c = s->cfg;
   MS_CUDA(s, cudaDeviceSynchronize());
   cudaFree(s->graph);
   s->graph = nullptr;
-  s->graph_rows = 0;
   s->graph_cap_rows = 0;
   s->graph_deg = 0;
-  if (n_rows > 0) MS_CUDA(s, cudaMalloc(&s->graph, (size_t)n_rows * degree * sizeof(int32_t)));
-  s->graph_rows = n_rows;
-  s->graph_cap_rows = n_rows;
+  s->graph_rows.assign(c.n_users, 0);
+  if (!s->graph_rows_d) MS_CUDA(s, cudaMalloc(&s->graph_rows_d, (size_t)c.n_users * sizeof(int32_t)));
+  if (!s->graph_users_d) MS_CUDA(s, cudaMalloc(&s->graph_users_d, 256 * sizeof(int32_t)));
+  MS_CUDA(s, cudaMemset(s->graph_rows_d, 0, (size_t)c.n_users * sizeof(int32_t)));
+  if (cap_rows > 0) MS_CUDA(s, cudaMalloc(&s->graph, (size_t)c.n_users * cap_rows * degree * sizeof(int32_t)));
+  s->graph_cap_rows = cap_rows;
   s->graph_deg = degree;
   return MS_OK;
 }
 
-static ms_status graph_check_store(memstore* s, int32_t degree) {
-  if (s->cfg.n_users != 1) return fail(s, MS_ERR_UNSUPPORTED, "the graph index serves single-segment stores (n_users = 1)");
+static ms_status graph_publish_rows(memstore* s, cudaStream_t st) {
+  std::vector<int32_t> rows(s->graph_rows.begin(), s->graph_rows.end());
+  MS_CUDA(s, cudaMemcpyAsync(s->graph_rows_d, rows.data(), rows.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  return MS_OK;
+}
+
+static ms_status graph_check_degree(memstore* s, int32_t degree) {
   if (degree < 1 || degree > kAnnMaxCand || degree + 1 > kTcMaxK)
     return fail(s, MS_ERR_INVALID_ARG, "degree %d out of range (1..%d)", degree, kTcMaxK - 1);
   return MS_OK;
+}
+
+// The batch of equal user numbers that accompanies a batch of one user's rows used as queries (multi-user stores only).
+static const int32_t* graph_batch_users(memstore* s, int32_t user, int n, cudaStream_t st) {
+  if (s->cfg.n_users == 1) return nullptr;
+  std::vector<int32_t> u(n, user);
+  if (cudaMemcpyAsync(s->graph_users_d, u.data(), (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) return nullptr;
+  return s->graph_users_d;
+}
+
+// Rows [row0, row1) of `user` get their exact lists (rows of the segment as queries through the exact retrieval kernels)
+// and, when n_old > 0, the rows below n_old are offered the new rows that list them.
+static ms_status graph_link_rows(memstore* s, int32_t user, int64_t row0, int64_t row1, int64_t n_old, ms_stream stream) {
+  const memstore_config& c = s->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int deg = s->graph_deg, k1 = deg + 1;
+  const int batch = std::max(1, std::min(kAppendMaxOffers, kAppendMaxPairs / deg));
+  const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
+  const char* seg = (const char*)s->emb + (size_t)user * c.max_facts_per_user * row_bytes;
+  int32_t* graph_u = s->graph + (size_t)user * s->graph_cap_rows * deg;
+  RetrieveParams p{};
+  p.emb = seg;
+  p.queries = seg;  // the rows are scored against one another
+  p.emb_dim = c.emb_dim;
+  int* n_pairs = s->append_pairs ? reinterpret_cast<int*>(s->append_pairs + kAppendMaxPairs) : nullptr;
+  for (int64_t r0 = row0; r0 < row1; r0 += batch) {
+    const int nb = (int)std::min<int64_t>(batch, row1 - r0);
+    const int32_t* users = graph_batch_users(s, user, nb, st);
+    if (c.n_users > 1 && !users) return fail(s, MS_ERR_CUDA, "staging the user numbers of a graph batch");
+    ms_status rc = retrieve_impl(s, seg + (size_t)r0 * row_bytes, users, nb, k1, s->graph_topk, nullptr, stream, 1);
+    if (rc != MS_OK) return rc;
+    graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, graph_u, deg, r0, nb);
+    s->kernels_launched++;
+    if (n_old > 0) {
+      append_pairs_kernel<<<1, 1024, 0, st>>>(graph_u, deg, r0, nb, n_old, s->append_pairs, n_pairs);
+      const int grid = kAppendMaxPairs / kAppendWarps;
+      if (c.emb_dtype == MS_DTYPE_F16)
+        append_update_kernel<__half><<<grid, kAppendWarps * 32, 0, st>>>(p, graph_u, deg, row1, s->append_pairs, n_pairs);
+      else
+        append_update_kernel<float><<<grid, kAppendWarps * 32, 0, st>>>(p, graph_u, deg, row1, s->append_pairs, n_pairs);
+      s->kernels_launched += 2;
+    }
+    if (cudaGetLastError() != cudaSuccess) return fail(s, MS_ERR_CUDA, "graph kernels failed to launch");
+  }
+  return MS_OK;
+}
+
+static ms_status graph_scratch(memstore* s) {
+  const size_t need = (size_t)kAppendMaxOffers * (s->graph_deg + 1);
+  if (s->graph_topk_cap < need) {
+    MS_CUDA(s, cudaDeviceSynchronize());
+    cudaFree(s->graph_topk);
+    s->graph_topk = nullptr;
+    s->graph_topk_cap = 0;
+    MS_CUDA(s, cudaMalloc(&s->graph_topk, need * sizeof(int32_t)));
+    s->graph_topk_cap = need;
+  }
+  if (!s->append_pairs) MS_CUDA(s, cudaMalloc(&s->append_pairs, (size_t)kAppendMaxPairs * sizeof(unsigned long long) + 16));
+  return MS_OK;
+}
+
+static void graph_drop(memstore* s) {  // a half-made graph must not be searched
+  s->graph_rows.assign(s->cfg.n_users, 0);
+  if (s->graph_rows_d) cudaMemset(s->graph_rows_d, 0, (size_t)s->cfg.n_users * sizeof(int32_t));
+  s->graph_deg = 0;
 }
 
 ms_status memstore_build_graph(memstore_t* s, int32_t degree, ms_stream stream) {
   Range range("memstore_build_graph");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
-  ms_status rc = graph_check_store(s, degree);
+  ms_status rc = graph_check_degree(s, degree);
   if (rc != MS_OK) return rc;
   const memstore_config& c = s->cfg;
   DeviceGuard g(c.device);
-  cudaStream_t st = (cudaStream_t)stream;
-  const int64_t n = s->user_count[0];
-  rc = graph_alloc(s, n, degree);
-  if (rc != MS_OK || n == 0) return rc;
-  constexpr int kBatch = 64;
-  const int k1 = degree + 1;
-  cudaFree(s->graph_topk);
-  s->graph_topk = nullptr;
-  s->graph_topk_cap = 0;
-  MS_CUDA(s, cudaMalloc(&s->graph_topk, (size_t)kBatch * k1 * sizeof(int32_t)));
-  s->graph_topk_cap = (size_t)kBatch * k1;
-  const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
-  for (int64_t row0 = 0; row0 < n; row0 += kBatch) {
-    const int nb = (int)std::min<int64_t>(kBatch, n - row0);
-    // the rows themselves are the queries: exact top-(degree + 1) of each, the row itself among them
-    rc = memstore_retrieve(s, (const char*)s->emb + (size_t)row0 * row_bytes, nullptr, nb, k1, s->graph_topk, nullptr, stream);
-    if (rc == MS_OK) {
-      graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, degree, row0, nb);
-      if (cudaGetLastError() != cudaSuccess) rc = fail(s, MS_ERR_CUDA, "graph_rows_kernel launch failed");
-    }
-    if (rc != MS_OK) {  // a half-built graph must not be searched
-      s->graph_rows = 0;
-      s->graph_deg = 0;
-      return rc;
-    }
-    s->kernels_launched++;
+  // a single segment gets exactly the rows it has (memstore_graph_append grows the array); several segments share one
+  // array with room for every segment's capacity
+  const int64_t cap = c.n_users == 1 ? s->user_count[0] : c.max_facts_per_user;
+  rc = graph_alloc(s, cap, degree);
+  if (rc != MS_OK) return rc;
+  rc = graph_scratch(s);
+  for (int32_t u = 0; rc == MS_OK && u < c.n_users; ++u) {
+    rc = graph_link_rows(s, u, 0, s->user_count[u], 0, stream);
+    if (rc == MS_OK) s->graph_rows[u] = s->user_count[u];
   }
-  return MS_OK;
+  if (rc == MS_OK) rc = graph_publish_rows(s, (cudaStream_t)stream);
+  if (rc != MS_OK) graph_drop(s);
+  return rc;
 }
 
 ms_status memstore_graph_append(memstore_t* s, ms_stream stream) {
@@ -865,13 +953,14 @@ ms_status memstore_graph_append(memstore_t* s, ms_stream stream) {
   if (!s->graph_deg) return fail(s, MS_ERR_INVALID_ARG, "no graph to grow: call memstore_build_graph or memstore_set_graph first");
   const memstore_config& c = s->cfg;
   const int deg = s->graph_deg;
-  const int64_t n_old = s->graph_rows, n = s->user_count[0];
-  if (n == n_old) return MS_OK;
+  bool any = false;
+  for (int32_t u = 0; u < c.n_users; ++u) any = any || s->user_count[u] > s->graph_rows[u];
+  if (!any) return MS_OK;
   DeviceGuard g(c.device);
-  cudaStream_t st = (cudaStream_t)stream;
-  // room for the new rows: the array grows geometrically (to at least 1.5 times its size, at most the segment's
-  // capacity), so that a stream of small appends does not reallocate and copy the whole graph each time
-  if (n > s->graph_cap_rows) {
+  if (c.n_users == 1 && s->user_count[0] > s->graph_cap_rows) {
+    // room for the new rows: the array grows geometrically (to at least 1.5 times its size, at most the segment's
+    // capacity), so that a stream of small appends does not reallocate and copy the whole graph each time
+    const int64_t n = s->user_count[0], n_old = s->graph_rows[0];
     const int64_t cap = std::min<int64_t>(c.max_facts_per_user, std::max<int64_t>(n, s->graph_cap_rows + s->graph_cap_rows / 2 + 1024));
     MS_CUDA(s, cudaDeviceSynchronize());
     int32_t* grown = nullptr;
@@ -887,81 +976,70 @@ ms_status memstore_graph_append(memstore_t* s, ms_stream stream) {
     s->graph = grown;
     s->graph_cap_rows = cap;
   }
-  s->graph_rows = n;  // searches after this call see all rows (a failure below clears the graph)
-  const int k1 = deg + 1;
-  const int batch = std::max(1, std::min(kAppendMaxOffers, kAppendMaxPairs / deg));
-  ms_status rc = MS_OK;
-  if (s->graph_topk_cap < (size_t)kAppendMaxOffers * k1) {
-    MS_CUDA(s, cudaDeviceSynchronize());
-    cudaFree(s->graph_topk);
-    s->graph_topk = nullptr;
-    s->graph_topk_cap = 0;
-    if (cudaMalloc(&s->graph_topk, (size_t)kAppendMaxOffers * k1 * sizeof(int32_t)) != cudaSuccess)
-      rc = fail(s, MS_ERR_OOM, "scratch for growing the graph");
-    else
-      s->graph_topk_cap = (size_t)kAppendMaxOffers * k1;
+  ms_status rc = graph_scratch(s);
+  for (int32_t u = 0; rc == MS_OK && u < c.n_users; ++u) {
+    const int64_t n_old = s->graph_rows[u], n = s->user_count[u];
+    if (n == n_old) continue;
+    rc = graph_link_rows(s, u, n_old, n, n_old, stream);
+    if (rc == MS_OK) s->graph_rows[u] = n;
   }
-  if (rc == MS_OK && !s->append_pairs && cudaMalloc(&s->append_pairs, (size_t)kAppendMaxPairs * sizeof(unsigned long long) + 16) != cudaSuccess)
-    rc = fail(s, MS_ERR_OOM, "scratch for growing the graph");
-  const size_t row_bytes = (size_t)c.emb_dim * emb_elem_size(c.emb_dtype);
-  RetrieveParams p{};
-  p.emb = s->emb;
-  p.queries = s->emb;  // the rows are scored against one another
-  p.emb_dim = c.emb_dim;
-  int* n_pairs = s->append_pairs ? reinterpret_cast<int*>(s->append_pairs + kAppendMaxPairs) : nullptr;
-  for (int64_t row0 = n_old; rc == MS_OK && row0 < n; row0 += batch) {
-    const int nb = (int)std::min<int64_t>(batch, n - row0);
-    rc = memstore_retrieve(s, (const char*)s->emb + (size_t)row0 * row_bytes, nullptr, nb, k1, s->graph_topk, nullptr, stream);
-    if (rc != MS_OK) break;
-    graph_rows_kernel<<<(nb + 7) / 8, dim3(32, 8), 0, st>>>(s->graph_topk, k1, s->graph, deg, row0, nb);
-    if (n_old > 0) {
-      append_pairs_kernel<<<1, 1024, 0, st>>>(s->graph, deg, row0, nb, n_old, s->append_pairs, n_pairs);
-      const int grid = kAppendMaxPairs / kAppendWarps;
-      if (c.emb_dtype == MS_DTYPE_F16)
-        append_update_kernel<__half><<<grid, kAppendWarps * 32, 0, st>>>(p, s->graph, deg, n, s->append_pairs, n_pairs);
-      else
-        append_update_kernel<float><<<grid, kAppendWarps * 32, 0, st>>>(p, s->graph, deg, n, s->append_pairs, n_pairs);
-      s->kernels_launched += 2;
-    }
-    if (cudaGetLastError() != cudaSuccess) rc = fail(s, MS_ERR_CUDA, "graph append kernels failed to launch");
-    s->kernels_launched++;
-  }
-  if (rc != MS_OK) {  // a half-grown graph must not be searched
-    s->graph_rows = 0;
-    s->graph_deg = 0;
-  }
+  if (rc == MS_OK) rc = graph_publish_rows(s, (cudaStream_t)stream);
+  if (rc != MS_OK) graph_drop(s);
   return rc;
 }
 
-ms_status memstore_set_graph(memstore_t* s, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream) {
+ms_status memstore_set_graph_user(memstore_t* s, int32_t user, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream) {
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
-  ms_status rc = graph_check_store(s, degree);
+  const memstore_config& c = s->cfg;
+  if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
+  ms_status rc = graph_check_degree(s, degree);
   if (rc != MS_OK) return rc;
-  if (n_rows < 0 || n_rows > s->user_count[0] || (n_rows > 0 && !graph))
-    return fail(s, MS_ERR_INVALID_ARG, "graph of %lld rows for a segment of %lld", (long long)n_rows, (long long)s->user_count[0]);
+  if (n_rows < 0 || n_rows > s->user_count[user] || (n_rows > 0 && !graph))
+    return fail(s, MS_ERR_INVALID_ARG, "graph of %lld rows for a segment of %lld", (long long)n_rows, (long long)s->user_count[user]);
+  DeviceGuard g(c.device);
+  const int64_t want_cap = c.n_users == 1 ? n_rows : c.max_facts_per_user;
+  if (!s->graph_deg || s->graph_deg != degree || want_cap > s->graph_cap_rows || c.n_users == 1) {
+    // another degree (or the first graph of this store): every segment's graph starts over
+    rc = graph_alloc(s, want_cap, degree);
+    if (rc != MS_OK) return rc;
+  }
+  if (n_rows > 0)
+    MS_CUDA(s, cudaMemcpyAsync(s->graph + (size_t)user * s->graph_cap_rows * degree, graph, (size_t)n_rows * degree * sizeof(int32_t),
+                               cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  s->graph_rows[user] = n_rows;
+  return graph_publish_rows(s, (cudaStream_t)stream);
+}
+
+ms_status memstore_set_graph(memstore_t* s, const int32_t* graph, int64_t n_rows, int32_t degree, ms_stream stream) {
+  return memstore_set_graph_user(s, 0, graph, n_rows, degree, stream);
+}
+
+ms_status memstore_get_graph_user(memstore_t* s, int32_t user, int32_t* out, int64_t out_capacity, int64_t* out_rows, int32_t* out_degree,
+                                  ms_stream stream) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  if (user < 0 || user >= s->cfg.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
+  const int64_t rows = s->graph_deg && !s->graph_rows.empty() ? s->graph_rows[user] : 0;
+  if (out_rows) *out_rows = rows;
+  if (out_degree) *out_degree = s->graph_deg;
+  if (!out) return MS_OK;
+  const int64_t need = rows * s->graph_deg;
+  if (out_capacity < need) return fail(s, MS_ERR_CAPACITY, "graph holds %lld entries, the buffer %lld", (long long)need, (long long)out_capacity);
   DeviceGuard g(s->cfg.device);
-  rc = graph_alloc(s, n_rows, degree);
-  if (rc != MS_OK || n_rows == 0) return rc;
-  MS_CUDA(s, cudaMemcpyAsync(s->graph, graph, (size_t)n_rows * degree * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  if (need)
+    MS_CUDA(s, cudaMemcpyAsync(out, s->graph + (size_t)user * s->graph_cap_rows * s->graph_deg, (size_t)need * sizeof(int32_t),
+                               cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return MS_OK;
 }
 
 ms_status memstore_get_graph(memstore_t* s, int32_t* out, int64_t out_capacity, int64_t* out_rows, int32_t* out_degree, ms_stream stream) {
-  if (!s) return MS_ERR_INVALID_ARG;
-  std::lock_guard<std::recursive_mutex> lock(s->mu);
-  if (out_rows) *out_rows = s->graph_rows;
-  if (out_degree) *out_degree = s->graph_deg;
-  if (!out) return MS_OK;
-  const int64_t need = s->graph_rows * s->graph_deg;
-  if (out_capacity < need) return fail(s, MS_ERR_CAPACITY, "graph holds %lld entries, the buffer %lld", (long long)need, (long long)out_capacity);
-  DeviceGuard g(s->cfg.device);
-  if (need) MS_CUDA(s, cudaMemcpyAsync(out, s->graph, (size_t)need * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
-  return MS_OK;
+  return memstore_get_graph_user(s, 0, out, out_capacity, out_rows, out_degree, stream);
 }
 
-ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
-                                int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream) {
+ms_status memstore_retrieve_ann_users(memstore_t* s, const void* queries, const int32_t* query_users, int32_t nq, int32_t k,
+                                      const ms_ann_params* params, int32_t* out_ids, float* out_scores, int32_t* out_counters,
+                                      ms_stream stream) {
   Range range("memstore_retrieve_ann");
   if (!s) return MS_ERR_INVALID_ARG;
   std::lock_guard<std::recursive_mutex> lock(s->mu);
@@ -993,7 +1071,12 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
   p.emb = s->emb;
   p.graph = s->graph;
   p.queries = queries;
-  p.n = (int32_t)s->graph_rows;
+  p.query_users = query_users;
+  p.graph_rows = s->graph_rows_d;
+  p.emb_fact_id = c.n_users == 1 ? nullptr : s->emb_fact_id;
+  p.seg_capacity = c.max_facts_per_user;
+  p.graph_cap_rows = s->graph_cap_rows;
+  p.n_users = c.n_users;
   p.emb_dim = c.emb_dim;
   p.deg = s->graph_deg;
   p.k = k;
@@ -1005,6 +1088,7 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
   p.out_ids = out_ids;
   p.out_scores = out_scores;
   p.out_counters = out_counters;
+  p.removed_bits = s->removed_bits_d;
   ms_status rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
   // one cluster per query; its size spreads a small batch over the GPU (a single SM cannot pull the candidate rows
@@ -1034,6 +1118,51 @@ ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, 
   MS_CUDA(s, cudaLaunchKernelExC(&lc, fn, args));
   s->kernels_launched++;
   s->retrieve_calls++;
+  return mark_last(s, st);
+}
+
+ms_status memstore_retrieve_ann(memstore_t* s, const void* queries, int32_t nq, int32_t k, const ms_ann_params* params,
+                                int32_t* out_ids, float* out_scores, int32_t* out_counters, ms_stream stream) {
+  return memstore_retrieve_ann_users(s, queries, nullptr, nq, k, params, out_ids, out_scores, out_counters, stream);
+}
+
+// ---- removing a fact ---------------------------------------------------------------------------------------------
+ms_status memstore_remove_fact(memstore_t* s, int32_t fact_id, ms_stream stream) {
+  Range range("memstore_remove_fact");
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  const memstore_config& c = s->cfg;
+  if (fact_id < 0 || fact_id >= s->n_facts) return fail(s, MS_ERR_INVALID_ARG, "fact id %d out of range (0..%lld)", fact_id, (long long)s->n_facts - 1);
+  // the embedding row of the id: ids are dense in insertion order, each add call put a run of them into one segment
+  size_t lo = 0, hi = s->id_runs.size();
+  while (lo + 1 < hi) {
+    const size_t mid = (lo + hi) / 2;
+    if (s->id_runs[mid].first_id <= fact_id) lo = mid; else hi = mid;
+  }
+  const memstore::IdRun& run = s->id_runs[lo];
+  const int64_t grow = (int64_t)run.user * c.max_facts_per_user + run.slot0 + (fact_id - run.first_id);
+  const int64_t n_rows = (int64_t)c.n_users * c.max_facts_per_user;
+  DeviceGuard g(c.device);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!s->removed_bits_d) {
+    const size_t words = (size_t)((n_rows + 31) / 32);
+    MS_CUDA(s, cudaDeviceSynchronize());
+    MS_CUDA(s, cudaMalloc(&s->removed_bits_d, words * sizeof(uint32_t)));
+    MS_CUDA(s, cudaMemset(s->removed_bits_d, 0, words * sizeof(uint32_t)));
+    s->removed_bits.assign(words, 0u);
+  }
+  uint32_t& word = s->removed_bits[(size_t)(grow >> 5)];
+  if ((word >> (grow & 31)) & 1u) return fail(s, MS_ERR_INVALID_ARG, "fact %d has been removed already", fact_id);
+  ms_status rc = order_after_last(s, st);
+  if (rc != MS_OK) return rc;
+  word |= 1u << (grow & 31);
+  // retrieval stops returning the row; injection refuses the id like a fact without K/V (its arena tokens are not reclaimed)
+  MS_CUDA(s, cudaMemcpyAsync(s->removed_bits_d + (grow >> 5), &word, sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+  const int32_t zero = 0;
+  MS_CUDA(s, cudaMemcpyAsync(reinterpret_cast<char*>(s->facts_d + fact_id) + offsetof(FactRec, resident), &zero, sizeof(int32_t),
+                             cudaMemcpyHostToDevice, st));
+  s->n_removed++;
+  s->cc_epoch++;  // composed segments that contain the fact must not be served any more
   return mark_last(s, st);
 }
 
@@ -1087,21 +1216,7 @@ ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int
   // the tickets must start at zero whatever an earlier call (of any store) left behind
   MS_CUDA(s, cudaMemsetAsync(tickets, 0, (size_t)nq * sizeof(uint32_t), st));
 
-  RetrieveParams p{};
-  p.emb = s->emb;
-  p.emb_fact_id = s->emb_fact_id;
-  p.user_count = s->user_count_d;
-  p.seg_capacity = c.max_facts_per_user;
-  p.n_users = c.n_users;
-  p.emb_dim = c.emb_dim;
-  p.queries = queries;
-  p.query_users = query_users;
-  p.nq = nq;
-  p.k = k;
-  p.scores = scores;
-  p.score_stride = c.max_facts_per_user;
-  p.out_ids = out_ids;
-  p.out_scores = out_scores;
+  RetrieveParams p = retrieve_params(s, queries, query_users, nq, k, scores, out_ids, out_scores);
 
   const int64_t n_max = query_users ? s->max_user_count : s->user_count[0];
   const int64_t target_ctas = std::max<int64_t>(1, (int64_t)s->sm_count * 8 / nq);
@@ -1360,8 +1475,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   const int early = (flags & MS_INPUTS_STABLE) ? 1 : 0;
   flags &= ~(uint32_t)MS_INPUTS_STABLE;
   if (flags & MS_RETRIEVE_ANN) {
-    if (query_users) return fail(s, MS_ERR_INVALID_ARG, "MS_RETRIEVE_ANN serves single-segment stores: query_users must be NULL");
-    ms_status rc = memstore_retrieve_ann(s, queries, nq, k, nullptr, out_ids, out_scores, nullptr, stream);
+    ms_status rc = memstore_retrieve_ann_users(s, queries, query_users, nq, k, nullptr, out_ids, out_scores, nullptr, stream);
     if (rc != MS_OK) return rc;
     return memstore_inject(s, out_ids, nq, k, start_pos, block_tables, max_blocks, cache, out_n_tokens, out_status,
                            out_slot_mapping, slot_stride, flags & ~(uint32_t)MS_RETRIEVE_ANN, stream);
@@ -1384,21 +1498,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   rc = order_after_last(s, st);
   if (rc != MS_OK) return rc;
 
-  RetrieveParams p{};
-  p.emb = s->emb;
-  p.emb_fact_id = s->emb_fact_id;
-  p.user_count = s->user_count_d;
-  p.seg_capacity = c.max_facts_per_user;
-  p.n_users = c.n_users;
-  p.emb_dim = c.emb_dim;
-  p.queries = queries;
-  p.query_users = query_users;
-  p.nq = nq;
-  p.k = k;
-  p.scores = s->scores;
-  p.score_stride = c.max_facts_per_user;
-  p.out_ids = out_ids;
-  p.out_scores = out_scores;
+  RetrieveParams p = retrieve_params(s, queries, query_users, nq, k, s->scores, out_ids, out_scores);
   const int keys_cap = (int)std::max<int64_t>(n_max, 1);
   const size_t smem = (size_t)keys_cap * sizeof(uint32_t);
   const int n_host = query_users ? -1 : (int)n_max;
@@ -1466,6 +1566,7 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   out->n_facts = s->n_facts;
   out->n_resident_facts = s->n_resident;
+  out->n_removed_facts = s->n_removed;
   out->kv_tokens_used = s->kv_tokens_used;
   out->host_kv_tokens_used = s->host_tokens_used;
   out->retrieve_calls = s->retrieve_calls;

@@ -20,7 +20,18 @@ struct RetrieveParams {
   int64_t score_stride;
   int32_t* out_ids;
   float* out_scores;
+  const uint32_t* removed_bits;  // one bit per row (row index user * seg_capacity + slot), or nullptr: nothing was ever removed
+  int32_t return_rows;           // 1: results are rows of the segment instead of fact ids (graph building)
 };
+
+// A removed row scores minus infinity, so it sorts behind every row that is left; results that would carry that
+// score are written as "no fact" (id -1, score 0).
+__device__ __forceinline__ bool row_removed(const RetrieveParams& p, int user, int64_t row) {
+  if (p.removed_bits == nullptr) return false;
+  const int64_t g = (int64_t)user * p.seg_capacity + row;
+  return (__ldg(p.removed_bits + (g >> 5)) >> (g & 31)) & 1u;
+}
+constexpr uint32_t kRemovedKey = 0x007fffffu;  // order_key(-infinity)
 
 constexpr int kScoreThreads = 256;
 constexpr int kScoreWarps = kScoreThreads / 32;
@@ -96,7 +107,7 @@ __device__ __forceinline__ void score_rows(const RetrieveParams& p, const float*
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) p.scores[(int64_t)q * p.score_stride + row] = acc + 0.0f;  // -0 -> +0
+    if (lane == 0) p.scores[(int64_t)q * p.score_stride + row] = row_removed(p, user, row) ? -INFINITY : acc + 0.0f;  // -0 -> +0
   }
 }
 
@@ -180,8 +191,8 @@ __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q
       float s0, s1;
       score_two_rows<T>(p, q, seg, row, row + WARPS, s0, s1);
       if (lane == 0) {
-        p.scores[(int64_t)q * p.score_stride + row] = s0 + 0.0f;
-        p.scores[(int64_t)q * p.score_stride + row + WARPS] = s1 + 0.0f;
+        p.scores[(int64_t)q * p.score_stride + row] = row_removed(p, user, row) ? -INFINITY : s0 + 0.0f;
+        p.scores[(int64_t)q * p.score_stride + row + WARPS] = row_removed(p, user, row + WARPS) ? -INFINITY : s1 + 0.0f;
       }
     }
   }
@@ -219,7 +230,7 @@ __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) p.scores[(int64_t)q * p.score_stride + row] = acc + 0.0f;  // -0 -> +0
+    if (lane == 0) p.scores[(int64_t)q * p.score_stride + row] = row_removed(p, user, row) ? -INFINITY : acc + 0.0f;  // -0 -> +0
   }
 }
 
@@ -265,9 +276,10 @@ __device__ __forceinline__ void write_topk(const unsigned long long* cand, int t
     float s = 0.f;
     if (r < take) {
       const unsigned long long c = cand[r];
-      const uint32_t row = 0xffffffffu - (uint32_t)(c & 0xffffffffull);
-      id = ids(row);
-      s = key_score((uint32_t)(c >> 32));
+      if ((uint32_t)(c >> 32) != kRemovedKey) {  // (a removed row that made the list because too few rows are left)
+        id = ids(0xffffffffu - (uint32_t)(c & 0xffffffffull));
+        s = key_score((uint32_t)(c >> 32));
+      }
     }
     out_ids[r] = id;
     if (ids.mirror) ids.mirror[r] = id;
@@ -402,10 +414,11 @@ __device__ __forceinline__ void rank_candidates(unsigned long long* cand, uint32
     rank += __shfl_xor_sync(0xffffffffu, rank, 1);
     rank += __shfl_xor_sync(0xffffffffu, rank, 2);
     if (ci < n_cand && part == 0 && rank < (uint32_t)k) {
-      const int32_t id = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+      const bool gone = (uint32_t)(mine >> 32) == kRemovedKey;
+      const int32_t id = gone ? -1 : ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
       out_ids[rank] = id;
       if (ids.mirror) ids.mirror[rank] = id;
-      if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+      if (out_scores) out_scores[rank] = gone ? 0.f : key_score((uint32_t)(mine >> 32));
     }
     return;
   }
@@ -415,10 +428,11 @@ __device__ __forceinline__ void rank_candidates(unsigned long long* cand, uint32
       uint32_t rank = 0;
       for (uint32_t jj = 0; jj < n_cand; ++jj) rank += cand[jj] > mine;
       if (rank < (uint32_t)k) {
-        const int32_t id = ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+        const bool gone = (uint32_t)(mine >> 32) == kRemovedKey;
+        const int32_t id = gone ? -1 : ids(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
         out_ids[rank] = id;
         if (ids.mirror) ids.mirror[rank] = id;
-        if (out_scores) out_scores[rank] = key_score((uint32_t)(mine >> 32));
+        if (out_scores) out_scores[rank] = gone ? 0.f : key_score((uint32_t)(mine >> 32));
       }
     }
     return;
@@ -528,8 +542,10 @@ __device__ bool topk_sampled(TopkShared& sm, const float* sc, int n, int k, cons
   for (int j = tid; j < kSampleSize; j += THREADS) {
     const float sv = __ldcg(sc + (int64_t)(j / kRun) * stride + (j % kRun));
     samp[j] = sv;
-    flo = fminf(flo, sv);
-    fhi = fmaxf(fhi, sv);
+    if (sv > -INFINITY) {  // removed rows score minus infinity: they take no part in the bucket layout
+      flo = fminf(flo, sv);
+      fhi = fmaxf(fhi, sv);
+    }
   }
   block_min_max<THREADS>(sm, order_key(flo), order_key(fhi));
   const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
@@ -618,8 +634,10 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
     if (!have_minmax) {
       float flo = INFINITY, fhi = -INFINITY;
       sweep([&](int, float sv) {
-        flo = fminf(flo, sv);
-        fhi = fmaxf(fhi, sv);
+        if (sv > -INFINITY) {  // removed rows score minus infinity: they take no part in the bucket layout
+          flo = fminf(flo, sv);
+          fhi = fmaxf(fhi, sv);
+        }
       });
       if (flo <= fhi) {  // this thread saw at least one score
         lo = order_key(flo);
@@ -627,6 +645,14 @@ __device__ void topk_block(TopkShared& sm, const float* sc, const uint32_t* keys
       }
     }
     block_min_max<THREADS>(sm, lo, hi);  // -> sm.kmin, sm.kmax; clears sm.hist
+    if (sm.kmin > sm.kmax) {  // no score at all took part: every row of the segment has been removed
+      for (int r = tid; r < k; r += THREADS) {
+        out_ids[r] = -1;
+        if (ids.mirror) ids.mirror[r] = -1;
+        if (out_scores) out_scores[r] = 0.f;
+      }
+      return;
+    }
     const uint32_t range = sm.kmax - sm.kmin;
     const float smin = key_score(sm.kmin), smax = key_score(sm.kmax);
     // With k much smaller than n only the upper part of the value range can hold the k-th largest, so the first
@@ -923,7 +949,7 @@ __global__ void __launch_bounds__(kTopkThreads, 1) topk_kernel(const RetrievePar
   const bool user_ok = user >= 0 && user < p.n_users;
   const int n = user_ok ? p.user_count[user] : 0;
   topk_block<kTopkThreads>(sm, p.scores + (int64_t)q * p.score_stride, nullptr, n, p.k,
-                           IdMap{nullptr, p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
+                           IdMap{nullptr, p.return_rows ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity},
                            p.out_ids + (int64_t)q * p.k, p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr);
 }
 
@@ -963,7 +989,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
   if (PLAN) plan_prefetch<THREADS>(*ip, q, ps);  // in flight while the ids are being selected
   const float* sc = p.scores + (int64_t)q * p.score_stride;
   // with a single user segment facts are numbered in row order: the row is the fact id
-  const int32_t* row_ids = p.n_users == 1 ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity;
+  const int32_t* row_ids = (p.n_users == 1 || p.return_rows) ? nullptr : p.emb_fact_id + (int64_t)(user_ok ? user : 0) * p.seg_capacity;
   int32_t* out_ids = p.out_ids + (int64_t)q * p.k;
   float* out_scores = p.out_scores ? p.out_scores + (int64_t)q * p.k : nullptr;
   const int k = p.k;
@@ -995,7 +1021,8 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
     if (done) {
       // the thread that holds a rank resolves the fact (store data only) ...
       int32_t id = -1;
-      if (my_rank >= 0) {
+      const bool gone = (uint32_t)(my_key >> 32) == kRemovedKey;  // a removed row that ranks because too few rows are left
+      if (my_rank >= 0 && !gone) {
         const uint32_t row = 0xffffffffu - (uint32_t)my_key;
         id = row_ids ? row_ids[row] : (int32_t)row;
         if (PLAN) {
@@ -1013,7 +1040,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
       if (PLAN && early) grid_dependency_wait();
       if (my_rank >= 0) {
         out_ids[my_rank] = id;
-        if (out_scores) out_scores[my_rank] = key_score((uint32_t)(my_key >> 32));
+        if (out_scores) out_scores[my_rank] = gone ? 0.f : key_score((uint32_t)(my_key >> 32));
       }
       for (int r = n + (int)threadIdx.x; r < k; r += THREADS) pad(r);  // a segment shorter than k: the other ranks are empty
       if (PLAN) {
@@ -1175,6 +1202,9 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
         } else if (ok0) {
           s0 = score_one_row<T>(p, q, seg, row) + 0.0f;
         }
+        // a removed row stays a candidate (the valid candidates must remain a prefix) with the score of a removed row
+        if (ok0 && row_removed(p, 0, row)) s0 = -INFINITY;
+        if (ok1 && row_removed(p, 0, row + 1)) s1 = -INFINITY;
         if (lane == 0) {
           cs[g_idx * 8 + r] = s0;
           cr[g_idx * 8 + r] = ok0 ? (int32_t)row : -1;
@@ -1207,11 +1237,13 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
   for (int i = threadIdx.x; i < n_valid; i += kScoreThreads) {
     const uint32_t kx = order_key(__ldcg(cs + i));
     s_keys[i] = kx;
-    lo = min(lo, kx);
-    hi = max(hi, kx);
+    if (kx != kRemovedKey) {
+      lo = min(lo, kx);
+      hi = max(hi, kx);
+    }
   }
   __syncthreads();
-  topk_block<kScoreThreads, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
+  topk_block<kScoreThreads, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.return_rows ? nullptr : p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
                             scores_out + (int64_t)q * p.k, true, lo, hi);
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -1255,6 +1287,8 @@ __global__ void __launch_bounds__(kScoreThreads) tc_fixup_kernel(const RetrieveP
       s0 = score_one_row<T>(p, q, seg, row);
     }
     s0 += 0.0f;
+    if (row_removed(p, 0, row)) s0 = -INFINITY;
+    if (row + 1 < row_end && row_removed(p, 0, row + 1)) s1 = -INFINITY;
     if (lane == 0) {
       if (s0 >= need) {
         const uint32_t slot = atomicAdd(&counts[q], 1u);
@@ -1291,7 +1325,8 @@ __global__ void __launch_bounds__(kScoreThreads) tc_fixup_kernel(const RetrieveP
   for (int i = threadIdx.x; i < P2; i += kScoreThreads) s_fix[i] = i < (int)n ? __ldcg(mine + i) : 0ull;
   __syncthreads();
   bitonic_sort_desc<kScoreThreads>(s_fix, P2);
-  write_topk<kScoreThreads>(s_fix, p.k, p.k, IdMap{nullptr, p.emb_fact_id}, p.out_ids + (int64_t)q * p.k, scores_out + (int64_t)q * p.k);
+  write_topk<kScoreThreads>(s_fix, p.k, p.k, IdMap{nullptr, p.return_rows ? nullptr : p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
+                            scores_out + (int64_t)q * p.k);
 }
 
 }  // namespace ms

@@ -45,6 +45,7 @@ struct GemmParams {
   uint32_t smem_bytes;  // dynamic shared memory of the launch
   uint32_t spin_limit;  // 0: the default bound of every wait; else a test's shorter bound
   int mute_producer;    // test aid: the producer role issues nothing, so the other roles' waits run out
+  const uint32_t* removed_bits;  // one bit per row of the segment, or nullptr: removed rows take no part in a group's maximum
 };
 
 // Shared memory after the 1 KiB alignment of the base: queries, ring, epilogue staging (4 warps x [4 groups][32
@@ -232,7 +233,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[b]);  // the MMAs of the tile after next may overwrite this buffer
       const int row = tile * kGemmTileRows + quarter * 32 + lane;
-      if (row >= p.n_rows) {
+      bool out = row >= p.n_rows;
+      if (!out && p.removed_bits != nullptr) out = (__ldg(p.removed_bits + (row >> 5)) >> (row & 31)) & 1u;
+      if (out) {
 #pragma unroll
         for (int q = 0; q < kGemmMaxQ; ++q) v[q] = -INFINITY;
       }

@@ -64,7 +64,7 @@ class _AnnParams(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "compose_cache_hits", "compose_cache_fills", "compose_cache_segments", "filter_fixup_overflows")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "n_removed_facts", "compose_cache_hits", "compose_cache_fills", "compose_cache_segments", "filter_fixup_overflows")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares
@@ -74,7 +74,8 @@ EXPORTS = (
     "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
     "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
-    "memstore_test_hooks", "memstore_reserve", "memstore_compose_cache",
+    "memstore_test_hooks", "memstore_reserve", "memstore_compose_cache", "memstore_remove_fact", "memstore_set_graph_user",
+    "memstore_get_graph_user", "memstore_retrieve_ann_users",
 )  # fmt: skip
 
 _lib = None
@@ -123,6 +124,14 @@ def load_library() -> C.CDLL:
     L.memstore_get_graph.argtypes = [vp, vp, i64, C.POINTER(i64), C.POINTER(i32), vp]
     L.memstore_retrieve_ann.restype = i32
     L.memstore_retrieve_ann.argtypes = [vp, vp, i32, i32, C.POINTER(_AnnParams), vp, vp, vp, vp]
+    L.memstore_retrieve_ann_users.restype = i32
+    L.memstore_retrieve_ann_users.argtypes = [vp, vp, vp, i32, i32, C.POINTER(_AnnParams), vp, vp, vp, vp]
+    L.memstore_set_graph_user.restype = i32
+    L.memstore_set_graph_user.argtypes = [vp, i32, vp, i64, i32, vp]
+    L.memstore_get_graph_user.restype = i32
+    L.memstore_get_graph_user.argtypes = [vp, i32, vp, i64, C.POINTER(i64), C.POINTER(i32), vp]
+    L.memstore_remove_fact.restype = i32
+    L.memstore_remove_fact.argtypes = [vp, i32, vp]
     L.memstore_rope_table_llama3.restype = i32
     L.memstore_rope_table_llama3.argtypes = [i32, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_float)]
     L.memstore_set_prefix.restype = i32
@@ -375,20 +384,25 @@ class MemStore:
         """Grow the graph for the facts added since it was built, set or last grown."""
         self._check(self._lib.memstore_graph_append(self._h, _stream_ptr(stream)))
 
-    def set_graph(self, graph: torch.Tensor, stream=None) -> None:
-        """Install a graph: int32 device tensor [n_rows, degree] of row numbers."""
-        self._check(self._lib.memstore_set_graph(self._h, _dev_ptr(graph, torch.int32, "graph"), graph.shape[0], graph.shape[1],
-                                                 _stream_ptr(stream)))  # fmt: skip
+    def set_graph(self, graph: torch.Tensor, user: int = 0, stream=None) -> None:
+        """Install the graph of ``user``'s segment: int32 device tensor [n_rows, degree] of rows of that segment."""
+        self._check(self._lib.memstore_set_graph_user(self._h, user, _dev_ptr(graph, torch.int32, "graph"), graph.shape[0],
+                                                      graph.shape[1], _stream_ptr(stream)))  # fmt: skip
 
-    def get_graph(self, stream=None) -> torch.Tensor:
+    def get_graph(self, user: int = 0, stream=None) -> torch.Tensor:
         rows, deg = C.c_int64(0), C.c_int32(0)
-        self._check(self._lib.memstore_get_graph(self._h, None, 0, C.byref(rows), C.byref(deg), _stream_ptr(stream)))
+        self._check(self._lib.memstore_get_graph_user(self._h, user, None, 0, C.byref(rows), C.byref(deg), _stream_ptr(stream)))
         out = torch.empty((rows.value, deg.value), dtype=torch.int32, device=self.device)
-        self._check(self._lib.memstore_get_graph(self._h, _dev_ptr(out, torch.int32, "out"), out.numel(), None, None, _stream_ptr(stream)))
+        self._check(self._lib.memstore_get_graph_user(self._h, user, _dev_ptr(out, torch.int32, "out"), out.numel(), None, None,
+                                                      _stream_ptr(stream)))  # fmt: skip
         return out
 
+    def remove_fact(self, fact_id: int, stream=None) -> None:
+        """Take a fact out: retrieval never returns it again, injection refuses its id (MS_REQ_NOT_RESIDENT)."""
+        self._check(self._lib.memstore_remove_fact(self._h, int(fact_id), _stream_ptr(stream)))
+
     def retrieve_ann(self, queries, k, beam=0, parents=0, n_entry=0, max_iters=0, out_ids=None, out_scores=None, want_scores=True,
-                     want_counters=False, stream=None):  # fmt: skip
+                     want_counters=False, stream=None, query_users=None):  # fmt: skip
         """Beam search over the graph (0 = the library's default for that parameter).  Returns (ids, scores) or, with
         ``want_counters``, (ids, scores, counters [nq, 2] = steps taken and rows scored)."""
         nq = queries.shape[0]
@@ -398,9 +412,10 @@ class MemStore:
             out_scores = torch.empty((nq, k), dtype=torch.float32, device=queries.device)
         counters = torch.zeros((nq, 2), dtype=torch.int32, device=queries.device) if want_counters else None
         prm = _AnnParams(beam, parents, n_entry, max_iters)
-        rc = self._lib.memstore_retrieve_ann(self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"), nq, k, C.byref(prm),
-                                             _dev_ptr(out_ids, torch.int32, "out_ids"), _dev_ptr(out_scores, torch.float32, "out_scores"),
-                                             _dev_ptr(counters, torch.int32, "counters"), _stream_ptr(stream))  # fmt: skip
+        rc = self._lib.memstore_retrieve_ann_users(self._h, _dev_ptr(queries, self.emb_torch_dtype, "queries"),
+                                                   _dev_ptr(query_users, torch.int32, "query_users"), nq, k, C.byref(prm),
+                                                   _dev_ptr(out_ids, torch.int32, "out_ids"), _dev_ptr(out_scores, torch.float32, "out_scores"),
+                                                   _dev_ptr(counters, torch.int32, "counters"), _stream_ptr(stream))  # fmt: skip
         self._check(rc)
         return (out_ids, out_scores, counters) if want_counters else (out_ids, out_scores)
 

@@ -74,13 +74,14 @@ class HostStore:
         return ms
 
 
-def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None):
-    """Near-tie rule for one query. ``emb``: the rows visible to the query; row_ids: their fact ids."""
+def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None, removed=None):
+    """Near-tie rule for one query. ``emb``: the rows visible to the query; row_ids: their fact ids; removed: boolean per
+    row, rows that must never be returned."""
     n = emb.shape[0]
-    ids_o, sc_o = oracle.retrieve(emb, query, k, row_ids=row_ids)
+    ids_o, sc_o = oracle.retrieve(emb, query, k, row_ids=row_ids, removed=removed)
     ids_o, sc_o = ids_o[0], sc_o[0]
     gpu_ids = np.asarray(gpu_ids)
-    take = min(n, k)
+    take = min(n if removed is None else int(n - np.count_nonzero(removed)), k)
     assert np.all(gpu_ids[take:] == -1), "padding must be -1"
     g = gpu_ids[:take]
     assert len(set(g.tolist())) == take, "duplicate ids"
@@ -91,6 +92,8 @@ def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None):
         lookup = {int(f): i for i, f in enumerate(row_ids)}
         assert all(int(x) in lookup for x in g), "id outside the user's segment"
         rows = np.array([lookup[int(x)] for x in g], dtype=np.int64)
+    if removed is not None:
+        assert not np.asarray(removed)[rows].any(), "a removed fact was returned"
     # the oracle's exact score of every row the GPU chose
     s_gpu_choice = oracle.scores(emb[rows], query).astype(np.float32) if take else np.zeros(0, np.float32)
     diff = np.abs(s_gpu_choice - sc_o[:take])
@@ -106,25 +109,26 @@ def check_ids(gpu_ids, gpu_scores, emb, query, k, row_ids=None):
 ANN_MARGIN = 1e-6  # decisions of a graph search wider than this cannot depend on how a binary32 sum was ordered
 
 
-def check_ann_search(ids, scores, counters, emb, graph, queries, k, **params):
+def check_ann_search(ids, scores, counters, emb, graph, queries, k, removed=None, row_ids=None, **params):
     """Graph search of the CUDA library against the oracle, query by query.  The reference is the oracle's search over
     its double-precision scores: when every decision of that search was wider than ANN_MARGIN the GPU must return the
     same rows after the same number of steps and scored rows, with scores within binary32 accumulation error of the
     exact ones.  Only a query with a closer decision is compared with the oracle's binary32 lane-order search (which
     restates the kernels' summation order), bit for bit.  Returns (queries judged by the exact search, queries)."""
     ids, scores = np.asarray(ids), np.asarray(scores)
-    exact = oracle.ann_search(emb, graph, queries, k, exact=True, **params)
+    exact = oracle.ann_search(emb, graph, queries, k, exact=True, removed=removed, **params)
+    to_ids = (lambda r: r) if row_ids is None else (lambda r: np.where(r >= 0, np.asarray(row_ids)[np.maximum(r, 0)], -1))
     on_exact_side = 0
     for i in range(len(queries)):
         if exact.margin[i] > ANN_MARGIN:
             on_exact_side += 1
-            assert np.array_equal(ids[i], exact.ids[i]), (i, params)
+            assert np.array_equal(ids[i], to_ids(exact.ids[i])), (i, params)
             assert np.all(np.abs(scores[i] - exact.scores[i]) < 2e-6 + 1e-6 * np.abs(exact.scores[i])), (i, params)
             if counters is not None:
                 assert counters[i, 0] == exact.iters[i] and counters[i, 1] == exact.scored[i], (i, params)
         else:
-            lanes = oracle.ann_search(emb, graph, queries[i : i + 1], k, **params)
-            assert np.array_equal(ids[i], lanes.ids[0]), (i, params)
+            lanes = oracle.ann_search(emb, graph, queries[i : i + 1], k, removed=removed, **params)
+            assert np.array_equal(ids[i], to_ids(lanes.ids[0])), (i, params)
             assert np.array_equal(scores[i].view(np.uint32), lanes.scores[0].view(np.uint32)), (i, params)
             if counters is not None:
                 assert counters[i, 0] == lanes.iters[0] and counters[i, 1] == lanes.scored[0], (i, params)

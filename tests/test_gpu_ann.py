@@ -115,6 +115,104 @@ def test_recall_against_exact_retrieval_on_structured_rows():
     ms.close()
 
 
+def test_graph_search_with_removed_rows():
+    """Removed rows stay in the graph: the walk goes through them and the result passes them over (the oracle's rule)."""
+    n, dim, deg = 4000, 128, 16
+    emb = synth.embeddings_low_rank(94, n, dim, "float16", intrinsic_dim=8)
+    q = synth.queries_near_rows(95, emb, 10)
+    ms = emb_store(emb)
+    ms.build_graph(deg)
+    g = ms.get_graph().cpu().numpy()
+    removed = np.random.default_rng(94).random(n) < 0.15
+    first, _ = ms.retrieve_ann(to_dev(q), 5)
+    removed[first[:, 0].cpu().numpy()] = True  # every query loses its best row
+    for f in np.flatnonzero(removed):
+        ms.remove_fact(int(f))
+    for k, beam in ((10, 64), (50, 64), (64, 64), (100, 128)):
+        par = dict(beam=beam, parents=4, n_entry=64, max_iters=32)
+        ids, sc, cnt = ms.retrieve_ann(to_dev(q), k, want_counters=True, **par)
+        torch.cuda.synchronize()
+        ids_np = ids.cpu().numpy()
+        assert not np.isin(ids_np[ids_np >= 0], np.flatnonzero(removed)).any()
+        check_ann_search(ids_np, sc.cpu().numpy(), cnt.cpu().numpy(), emb, g, q, k, removed=removed, **par)
+    # a graph built now lists no removed row
+    ms.build_graph(deg)
+    g2 = ms.get_graph().cpu().numpy()
+    assert not np.isin(g2, np.flatnonzero(removed)).any()
+    ms.close()
+
+
+@pytest.mark.parametrize("dtype,dim,per_user,n_users,deg", [("float16", 128, 400, 5, 16), ("float32", 64, 152, 3, 8)])
+def test_every_user_segment_has_its_own_graph(dtype, dim, per_user, n_users, deg):
+    """Graphs of a multi-user store: built per segment (rows local to the segment), searched for the query's user,
+    results are that user's fact ids; appended rows are linked per user; a caller-made graph can be set per user."""
+    total = per_user * n_users
+    emb = synth.embeddings_low_rank(96, total, dim, dtype, intrinsic_dim=6)
+    tdt = torch.float32 if dtype == "float32" else torch.float16
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=dim, emb_dtype=tdt, rope_theta=1e4, n_users=n_users,
+                  max_facts_per_user=per_user + 40, max_kv_tokens=0)  # fmt: skip
+    # facts arrive interleaved: ids are global, rows are per segment
+    row_ids = [[] for _ in range(n_users)]
+    nxt = 0
+    for chunk in range(4):
+        for u in range(n_users):
+            a = u * per_user + chunk * (per_user // 4)
+            b = a + per_user // 4
+            first = ms.add_facts(to_dev(emb[a:b]), np.zeros(b - a, np.int32), user=u)
+            assert first == nxt
+            row_ids[u].extend(range(nxt, nxt + (b - a)))
+            nxt += b - a
+    ms.build_graph(deg)
+    users = np.array([u % n_users for u in range(2 * n_users)], np.int32)
+    q = np.stack([synth.queries_near_rows(97 + i, emb[u * per_user : (u + 1) * per_user], 1)[0] for i, u in enumerate(users)])
+    par = dict(beam=64, parents=4, n_entry=32, max_iters=20)
+    graphs = []
+    for u in range(n_users):
+        seg = emb[u * per_user : (u + 1) * per_user]
+        g = ms.get_graph(user=u).cpu().numpy()
+        assert g.shape == (per_user, deg) and g.max() < per_user
+        want = oracle.knn_graph(seg, deg)
+        same = 0
+        for r in range(0, per_user, 7):
+            s_got = oracle.scores(seg[g[r]], seg[r]).astype(np.float32)
+            s_want = oracle.scores(seg[want[r]], seg[r]).astype(np.float32)
+            assert np.all(np.abs(s_got - s_want) < 1e-5) and r not in g[r]
+            same += int(np.array_equal(g[r], want[r]))
+        assert same >= 0.8 * len(range(0, per_user, 7))
+        graphs.append(g)
+    ids, sc, cnt = ms.retrieve_ann(to_dev(q), 10, want_counters=True, query_users=to_dev(users), **par)
+    torch.cuda.synchronize()
+    for i, u in enumerate(users):
+        seg = emb[u * per_user : (u + 1) * per_user]
+        check_ann_search(ids[i : i + 1].cpu().numpy(), sc[i : i + 1].cpu().numpy(), cnt[i : i + 1].cpu().numpy(), seg, graphs[u], q[i : i + 1], 10,
+                         row_ids=np.array(row_ids[u], np.int32), **par)
+    # exact and approximate retrieval agree on the best fact of a query that is a stored row
+    probe = emb[2 * per_user + 5 : 2 * per_user + 6]
+    ids_a, _ = ms.retrieve_ann(to_dev(probe), 1, query_users=to_dev(np.array([2], np.int32)))
+    ids_e, _ = ms.retrieve(to_dev(probe), 1, query_users=to_dev(np.array([2], np.int32)))
+    assert int(ids_a[0, 0]) == int(ids_e[0, 0]) == row_ids[2][5]
+    # rows appended to two segments are linked into those segments' graphs
+    extra = synth.embeddings_low_rank(98, 40, dim, dtype, intrinsic_dim=6)
+    ms.add_facts(to_dev(extra[:25]), np.zeros(25, np.int32), user=1)
+    ms.add_facts(to_dev(extra[25:]), np.zeros(15, np.int32), user=n_users - 1)
+    ms.graph_append()
+    assert ms.get_graph(user=1).shape == (per_user + 25, deg) and ms.get_graph(user=0).shape == (per_user, deg)
+    seg1 = np.concatenate([emb[per_user : 2 * per_user], extra[:25]])
+    want1 = oracle.graph_append(seg1, oracle.knn_graph(seg1[:per_user], deg))
+    g1 = ms.get_graph(user=1).cpu().numpy()
+    for r in list(range(per_user, per_user + 25)) + list(range(0, per_user, 11)):
+        s_got = oracle.scores(seg1[g1[r]], seg1[r]).astype(np.float32)
+        s_want = oracle.scores(seg1[want1[r]], seg1[r]).astype(np.float32)
+        assert np.all(np.abs(s_got - s_want) < 1e-5), r
+    # a caller-made graph for one user replaces that user's graph only
+    custom = synth.random_graph(99, per_user, deg)
+    ms.set_graph(to_dev(custom), user=0)
+    assert torch.equal(ms.get_graph(user=0).cpu(), torch.from_numpy(custom)) and ms.get_graph(user=1).shape[0] == per_user + 25
+    ids_c, sc_c = ms.retrieve_ann(to_dev(q[:1]), 5, query_users=to_dev(users[:1]), **par)
+    check_ann_search(ids_c.cpu().numpy(), sc_c.cpu().numpy(), None, emb[:per_user], custom, q[:1], 5, row_ids=np.array(row_ids[0], np.int32), **par)
+    ms.close()
+
+
 def test_graph_index_errors_and_empty_cases():
     emb = synth.embeddings(86, 100, 64, "float16")
     ms = emb_store(emb)
@@ -134,10 +232,9 @@ def test_graph_index_errors_and_empty_cases():
     ids, _ = ms.retrieve_ann(q, 5)  # still usable after the refused calls
     assert bool((ids >= 0).all())
     ms.close()
-    two = emb_store(emb[:50], n_users=2)
     with pytest.raises(MemStoreError):
-        two.build_graph(8)
-    two.close()
+        ms_bad = emb_store(emb[:50])
+        ms_bad.set_graph(torch.zeros((10, 4), dtype=torch.int32, device=DEV), user=1)  # no such user
     empty = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=64, rope_theta=1e4, max_facts_per_user=10, max_kv_tokens=0)
     empty.build_graph(4)
     ids, sc = empty.retrieve_ann(q, 3)

@@ -170,6 +170,82 @@ def test_tensor_core_filter_with_more_tied_groups_than_its_margin(kind):
     ms.close()
 
 
+@pytest.mark.parametrize("dtype,E,n,nq,n_users", [("float16", 256, 700, 3, 1), ("float32", 64, 300, 5, 3), ("float32", 64, 9000, 2, 1),
+                                                   ("float16", 128, 20_000, 9, 1), ("float16", 64, 2500, 2, 1)])  # fmt: skip
+def test_removed_facts_are_never_retrieved(dtype, E, n, nq, n_users):
+    """memstore_remove_fact on every exact retrieval path (one-launch kernels with one and several keys per thread,
+    per-user segments, the unfused CUDA-core kernels, the tensor-core filter with whole groups removed): the results
+    are the oracle's ranking of the facts that are left; short lists are padded; the allocation-free call agrees."""
+    hs = HostStore(90, n, 1, 1, 16, 1, 1, E, dtype, n_users=n_users)
+    total = n * n_users
+    hs.emb[min(900, n - 1)] = hs.emb[17]
+    ms = hs.to_memstore(1e4, batch=4096)
+    q = synth.queries(90, nq, E, dtype)
+    q[0] = hs.emb[17]
+    users = (np.arange(nq) % n_users).astype(np.int32)
+    rng = np.random.default_rng(90)
+    removed = rng.random(total) < 0.25
+    removed[17] = True  # the exact match of query 0 goes; its copy must come first now
+    removed[min(900, n - 1)] = False
+    removed[64:96] = True  # whole groups of 8 rows (and a whole warp's rows) at once
+    for f in np.flatnonzero(removed):
+        ms.remove_fact(int(f))
+    assert ms.stats()["n_removed_facts"] == int(removed.sum())
+    with pytest.raises(RuntimeError):
+        ms.remove_fact(17)  # twice
+    with pytest.raises(RuntimeError):
+        ms.remove_fact(total)
+    alive0 = int((~removed[:n]).sum())
+    for k in sorted({1, 10, 100, 256, min(alive0 + 3, 2048)}):
+        ids, sc = ms.retrieve(to_dev(q), k, query_users=to_dev(users) if n_users > 1 else None)
+        torch.cuda.synchronize()
+        ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+        for i in range(nq):
+            u = int(users[i])
+            rows = np.arange(u * n, (u + 1) * n)
+            check_ids(ids[i], sc[i], hs.emb[rows], q[i], k, row_ids=rows.astype(np.int32) if n_users > 1 else None, removed=removed[rows])
+        if k >= 1:
+            assert ids[0, 0] == min(900, n - 1)
+        if n * nq <= (1 << 20):
+            ids_s, sc_s = ms.retrieve_static(to_dev(q), k, query_users=to_dev(users) if n_users > 1 else None)
+            assert np.array_equal(ids_s.cpu().numpy(), ids) and np.array_equal(sc_s.cpu().numpy(), sc)
+    assert ms.stats()["kernel_timeouts"] == 0
+    # everything of user 0 removed: nothing but padding
+    for f in np.flatnonzero(~removed[:n]):
+        ms.remove_fact(int(f))
+    ids, sc = ms.retrieve(to_dev(q[:1]), 5)
+    assert ids.cpu().tolist() == [[-1] * 5] and sc.cpu().tolist() == [[0.0] * 5]
+    ms.close()
+
+
+def test_removed_facts_are_refused_by_injection_and_skipped_by_the_one_call_path():
+    hs = HostStore(91, 200, 2, 4, 64, 4, 12, 64, "float16")
+    ms = hs.to_memstore(1e4)
+    bs, nb, k = 16, 64, 6
+    q = synth.queries(92, 1, 64, "float16")
+    ids0, _ = ms.retrieve(to_dev(q), k)
+    best = ids0[0].cpu().tolist()
+    ms.remove_fact(best[0])
+    ms.remove_fact(best[2])
+    table = synth.block_tables(93, nb, 8, 1)[0]
+    # the removed ids in an explicit list contribute nothing and raise the status bit; the others are placed
+    cache = make_cache(hs, nb, bs)
+    n_tok, st = ms.inject(to_dev(np.array([best[:4]], np.int32)), to_dev(np.array([3], np.int32)), to_dev(table[None]), cache)
+    torch.cuda.synchronize()
+    assert int(st[0]) == M.REQ_NOT_RESIDENT and int(n_tok[0]) == int(hs.lens[[best[1], best[3]]].sum())
+    run_inject_and_check(ms, hs, [best[1], best[3]], 3, table, make_cache(hs, nb, bs), 1e4)
+    # retrieval + injection in one call: the list no longer contains them, the status is clean
+    removed = np.zeros(200, bool)
+    removed[[best[0], best[2]]] = True
+    cache = make_cache(hs, nb, bs)
+    for rep in range(2):
+        ids_b, n_b, st_b = ms.retrieve_inject(to_dev(q), k, to_dev(np.array([3], np.int32)), to_dev(table[None]), cache, flags=M.INJECT_REVERSE)
+        torch.cuda.synchronize()
+        check_ids(ids_b[0].cpu().numpy(), None, hs.emb, q[0], k, removed=removed)
+        assert int(st_b[0]) == 0 and int(n_b[0]) == int(hs.lens[ids_b[0].cpu().numpy()].sum())
+    ms.close()
+
+
 def test_bounded_waits_report_a_time_out_and_the_store_stays_usable():
     """The staged kernels bound every wait.  With their producer roles silenced (nothing is ever in flight) and the
     bound shortened, the waits run out: the kernels must return, report the time-out, touch nothing outside the
