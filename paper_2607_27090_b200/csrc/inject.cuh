@@ -34,6 +34,7 @@ struct InjectParams {
   int64_t layer_stride, block_stride, token_stride, head_stride, num_blocks;
   int32_t block_size;
   float k_scale, v_scale;  // 8-bit cache: per-tensor scales of K and V (the cache holds value / scale)
+  float k_recip, v_recip;  // their reciprocals, correctly rounded to fp32 (computed by the host in double)
   // outputs
   int32_t* out_n_tokens;
   int32_t* out_status;
@@ -472,14 +473,31 @@ __device__ __forceinline__ uint2 pack_e4m3x8(const float* f) {
   return make_uint2(w[0], w[1]);
 }
 
-// The 8 bf16 values of a 16-byte vector divided by `scale`: IEEE fp32 division, the arithmetic of the serving engines'
-// own 8-bit cache write (they divide the bf16 key or value by the per-tensor scale in fp32 and round once to e4m3).
-__device__ __forceinline__ void scaled_floats(const uint4& a, float scale, float* f) {
+// x / s rounded to nearest in fp32, as IEEE division gives it, from the correctly rounded reciprocal r = RN(1 / s) that
+// the host supplies: two residual corrections with fused multiply-adds (q <- q + (x - q s) r; the residuals are
+// exact).  After the first the quotient is faithful, after the second it is the correctly rounded one (Markstein's
+// theorem on division with a correctly rounded reciprocal; it excludes divisors whose significand is all ones, for
+// which the host asks for the hardware division instead).  Quotients far outside what an e4m3 cache can hold skip the
+// corrections (they saturate or vanish whatever their last bit), which also keeps infinities out of the residuals.
+template <bool HW_DIV>
+__device__ __forceinline__ float div_by_scale(float x, float s, float r) {
+  if (HW_DIV) return __fdiv_rn(x, s);
+  const float q0 = __fmul_rn(x, r);
+  const float q1 = __fmaf_rn(__fmaf_rn(-q0, s, x), r, q0);
+  const float q2 = __fmaf_rn(__fmaf_rn(-q1, s, x), r, q1);
+  const float a = fabsf(q0);
+  return (a < 1e30f && a > 1e-30f) ? q2 : q0;
+}
+
+// The 8 bf16 values of a 16-byte vector divided by `scale` in fp32: the arithmetic of the serving engines' own 8-bit
+// cache write (they divide the bf16 key or value by the per-tensor scale in fp32 and round once to e4m3).
+template <bool HW_DIV>
+__device__ __forceinline__ void scaled_floats(const uint4& a, float scale, float recip, float* f) {
   const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    f[2 * w] = __fdiv_rn(bf16lo(aw[w]), scale);
-    f[2 * w + 1] = __fdiv_rn(bf16hi(aw[w]), scale);
+    f[2 * w] = div_by_scale<HW_DIV>(bf16lo(aw[w]), scale, recip);
+    f[2 * w + 1] = div_by_scale<HW_DIV>(bf16hi(aw[w]), scale, recip);
   }
 }
 
@@ -506,7 +524,8 @@ constexpr int kUnitsPerPart = kThreadsPerToken * kUnitsPerThread;  // units of a
 // bf16 key (rotated and rounded exactly as for a bf16 cache) and the bf16 value are divided by the per-tensor scale in
 // fp32 and rounded once to e4m3, so the cache is byte for byte what an engine's own cache write would make of the
 // bf16 cache contents; a thread then stores two 8-byte vectors per row.
-template <int STYLE, bool FP8>
+// FP8: 0 = bf16 cache, 1 = 8-bit cache, 2 = 8-bit cache with the hardware division (see div_by_scale)
+template <int STYLE, int FP8>
 __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const InjectParams p) {
   const int tid = threadIdx.x;
   const int tk = tid >> 5;  // token of the tile
@@ -596,13 +615,13 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
           st_stream(reinterpret_cast<uint4*>(vd + offB), vb[u]);
         } else {
           float fa[8], fb[8];
-          scaled_floats(ka[u], p.k_scale, fa);
-          scaled_floats(kb[u], p.k_scale, fb);
+          scaled_floats<FP8 == 2>(ka[u], p.k_scale, p.k_recip, fa);
+          scaled_floats<FP8 == 2>(kb[u], p.k_scale, p.k_recip, fb);
           uint8_t* kd = reinterpret_cast<uint8_t*>(p.k_cache) + dbase + (int64_t)h * p.head_stride;
           st_stream8(reinterpret_cast<uint2*>(kd + offA), pack_e4m3x8(fa));
           st_stream8(reinterpret_cast<uint2*>(kd + offB), pack_e4m3x8(fb));
-          scaled_floats(va[u], p.v_scale, fa);
-          scaled_floats(vb[u], p.v_scale, fb);
+          scaled_floats<FP8 == 2>(va[u], p.v_scale, p.v_recip, fa);
+          scaled_floats<FP8 == 2>(vb[u], p.v_scale, p.v_recip, fb);
           uint8_t* vd = reinterpret_cast<uint8_t*>(p.v_cache) + dbase + (int64_t)h * p.head_stride;
           st_stream8(reinterpret_cast<uint2*>(vd + offA), pack_e4m3x8(fa));
           st_stream8(reinterpret_cast<uint2*>(vd + offB), pack_e4m3x8(fb));

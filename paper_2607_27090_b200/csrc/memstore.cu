@@ -567,7 +567,7 @@ ms_status memstore_create(const memstore_config* config, memstore_t** out) {
   s->user_count.assign(config->n_users, 0);
   s->tma_path = (config->flags & MS_STORE_TMA_COPY_PATH) != 0 && config->max_host_kv_tokens == 0;  // HBM arena only
   int occ = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0, false>, kCopyThreads, 0) == cudaSuccess && occ > 0)
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, inject_copy_kernel<0, 0>, kCopyThreads, 0) == cudaSuccess && occ > 0)
     s->copy_ctas_per_sm = occ;
   if (cudaFuncSetAttribute(inject_copy_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(inject_copy_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaSmemBytes) != cudaSuccess) {
@@ -1323,6 +1323,9 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.block_size = cache->block_size;
   p.k_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? cache->k_scale : 1.0f;
   p.v_scale = cache->dtype == MS_CACHE_FP8_E4M3 ? cache->v_scale : 1.0f;
+  // reciprocals rounded once to fp32 (a double quotient rounds to the same float as the exact one)
+  p.k_recip = (float)(1.0 / (double)p.k_scale);
+  p.v_recip = (float)(1.0 / (double)p.v_scale);
   p.out_n_tokens = out_n_tokens;
   p.out_status = out_status;
   p.out_slot_mapping = out_slot_mapping;
@@ -1402,11 +1405,20 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
     lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
     lc.blockDim = dim3(kCopyThreads);
     lc.dynamicSmemBytes = 0;
-    const bool fp8 = cache->dtype == MS_CACHE_FP8_E4M3;
+    // 8-bit caches: a scale whose significand is all ones, or one so extreme that it or its reciprocal is not a normal
+    // number, takes the kernel variant that divides with the hardware routine (see div_by_scale)
+    auto awkward = [](float sc, float rc) {
+      uint32_t u;
+      memcpy(&u, &sc, 4);
+      return (u & 0x7fffffu) == 0x7fffffu || !std::isnormal(rc) || !std::isnormal(sc);
+    };
+    const int fp8 = cache->dtype != MS_CACHE_FP8_E4M3 ? 0 : (awkward(p.k_scale, p.k_recip) || awkward(p.v_scale, p.v_recip)) ? 2 : 1;
     if (c.rope_style == MS_ROPE_HALF_SPLIT)
-      e = fp8 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, true>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<0, false>, p);
+      e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 0>, p)
+          : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 2>, p);
     else
-      e = fp8 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, true>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, false>, p);
+      e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 0>, p)
+          : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 2>, p);
   }
   if (e != cudaSuccess) {
     // (the planning kernel has left the control block clean: nothing to undo)

@@ -430,6 +430,40 @@ def test_inject_into_an_8_bit_e4m3_cache(layout, style, R):
     ms.close()
 
 
+def test_8_bit_cache_division_is_exact_for_every_bf16_value_at_many_scales():
+    """The copy kernel divides by the scale through a reciprocal and two exact-residual corrections; the result must be
+    the IEEE fp32 quotient, so that the e4m3 code equals the oracle's (a real fp32 division) for EVERY bf16 value -
+    here as the V rows of one long fact - at scales picked to be awkward: random ones over twelve octaves, powers of two
+    and their neighbours, significands that are all ones (the hardware-division route) or nearly so."""
+    every = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    as_f = torch.from_numpy(every.view(np.int16)).view(torch.bfloat16).float()
+    every = every[torch.isfinite(as_f).numpy()]  # 65280 values
+    D, H = 16, 1
+    n_tok = every.size // D
+    vals = np.ascontiguousarray(every[: n_tok * D].reshape(1, n_tok, H, D))
+    ms = MemStore(n_layers=1, n_kv_heads=H, head_dim=D, emb_dim=64, rope_theta=1e4, max_facts_per_user=2, max_kv_tokens=n_tok)
+    ms.add_facts(to_dev(synth.embeddings(1, 1, 64, "float16")), [n_tok], to_dev(vals), to_dev(vals))
+    nb = (n_tok + 15) // 16
+    table = to_dev(np.arange(nb, dtype=np.int32)[None])
+    ids, start = to_dev(np.zeros((1, 1), np.int32)), to_dev(np.zeros(1, np.int32))
+    rng = np.random.default_rng(5)
+    scales = list(np.exp(rng.uniform(np.log(2.0**-8), np.log(2.0**4), 160)).astype(np.float32))
+    for e in (-6, -1, 0, 2):
+        one = np.float32(2.0**e)
+        scales += [one, np.nextafter(one, np.float32(0)), np.nextafter(one, np.float32(9)), np.nextafter(np.nextafter(one, np.float32(0)), np.float32(0))]
+    scales += [np.float32(0.3), np.float32(0.9), np.float32(2.7), np.float32(0.0173), np.float32(1e-30), np.float32(3e30)]
+    for sc in scales:
+        cache = PagedCache.allocate(1, nb, 16, H, D, DEV, fill_bits=0x5A, fp8=True, k_scale=1.0, v_scale=float(sc))
+        _, st = ms.inject(ids, start, table, cache)
+        torch.cuda.synchronize()
+        assert int(st[0]) == 0
+        got = cache.v.cpu().numpy().reshape(-1)[: n_tok * D]
+        want = oracle.e4m3_from_scaled_bf16(vals.reshape(-1), float(sc))
+        bad = np.flatnonzero(got != want)
+        assert bad.size == 0, (float(sc), vals.reshape(-1)[bad[:5]], got[bad[:5]], want[bad[:5]])
+    ms.close()
+
+
 def test_inject_inv_freq_override_and_reverse_flag():
     D = 64
     f = (np.linspace(1.0, 0.001, D // 2)).astype(np.float32)
