@@ -400,6 +400,11 @@ typedef struct {
   int64_t compose_cache_segments;                  /* segments the composition cache can hold (0: none) */
   int64_t filter_fixup_overflows; /* 1 if such a re-scan ever met more than 4096 rows within rounding of the k-th score: that
                                      query kept the filter's answer (ids inside the 1e-5 near-tie rule, exact ties unordered) */
+  int64_t filter_list_queries;   /* queries of the tensor-core retrieve path served from the candidate rows the scoring kernel
+                                    listed for them, */
+  int64_t filter_list_rows;      /* the rows it listed for those queries in all (a few hundred to a thousand each), and */
+  int64_t filter_list_fallbacks; /* the queries whose list was too short, too long or tied at its cut and that were served
+                                    from the group maxima instead (same results, slower) */
 } memstore_stats_t;
 ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
 

@@ -88,4 +88,5 @@ __device__ __forceinline__ void st_stream8(uint2* p, const uint2& v) {
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::); }
 
+
 }  // namespace ms

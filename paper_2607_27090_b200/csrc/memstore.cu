@@ -61,6 +61,12 @@ struct memstore {
   uint32_t* tc_fix_tickets = nullptr;
   uint32_t* tc_n_fixups = nullptr;  // queries the fix-up kernel has redone since creation
   int* tc_error = nullptr;
+  // candidate rows emitted by the filter kernel (see score_gemm.cuh)
+  uint32_t* tc_hist = nullptr;      // [64][kHistWords] + thr_used[64] (zero between calls) + cand_cnt[64][kCandMaxSegs]
+  unsigned long long* tc_emit = nullptr;  // [64][kTcCandPlaces]: candidate rows listed by the filter kernel
+  int32_t* tc_sel_rows = nullptr;   // [64][kTcMaxK]
+  int* tc_slow = nullptr;           // [64]: the query's candidate list was unusable, the group maxima serve it
+  unsigned long long* tc_list_stats = nullptr;  // queries served from their candidate list, rows listed for them, fallbacks
   bool tc_ready = false;
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
@@ -223,6 +229,28 @@ constexpr int64_t kTcFewQueriesRows = 131072;  // ... unless the segment is long
 constexpr int kTcMaxK = 256;
 constexpr int kTcGroupMargin = 28;   // groups selected beyond k: slack for tensor-core vs CUDA-core rounding at the k-th score
 constexpr int kTcMaxK2 = kTcMaxK + kTcGroupMargin;
+constexpr int kTcCandPlaces = kTopkThreads * kCandKpl;  // candidate places per query over all CTAs of the filter kernel
+constexpr int kTcCandSeg = 24;                          // places per epilogue warp of the filter kernel and query
+constexpr int kTcMaxCtas = kCandMaxSegs / 4;
+constexpr int kTcRowMargin = 28;     // candidate rows rescored beyond k
+constexpr size_t kTcHistWords = (size_t)kGemmMaxQ * (kHistWords + 1 + kCandMaxSegs);
+
+// Launch as a programmatic dependent of the kernel before it in the stream (the kernel calls griddepcontrol.wait before
+// it touches anything the earlier kernels write).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t lc{};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 bool tc_path_applies(const memstore* s, const int32_t* query_users, int nq, int k, int64_t n_max) {
   const memstore_config& c = s->cfg;
@@ -250,6 +278,14 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_fix_tickets, (size_t)kGemmMaxQ * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_n_fixups, 2 * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_error, 2 * sizeof(int)));
+  MS_CUDA(s, cudaMalloc(&s->tc_hist, kTcHistWords * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_emit, (size_t)kGemmMaxQ * kTcCandPlaces * sizeof(unsigned long long)));
+  MS_CUDA(s, cudaMalloc(&s->tc_sel_rows, (size_t)kGemmMaxQ * kTcMaxK * sizeof(int32_t)));
+  MS_CUDA(s, cudaMalloc(&s->tc_slow, (size_t)kGemmMaxQ * sizeof(int)));
+  MS_CUDA(s, cudaMemset(s->tc_hist, 0, kTcHistWords * sizeof(uint32_t)));
+  MS_CUDA(s, cudaMemset(s->tc_slow, 0, (size_t)kGemmMaxQ * sizeof(int)));
+  MS_CUDA(s, cudaMalloc(&s->tc_list_stats, 3 * sizeof(unsigned long long)));
+  MS_CUDA(s, cudaMemset(s->tc_list_stats, 0, 3 * sizeof(unsigned long long)));
   MS_CUDA(s, cudaMemset(s->tc_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
   MS_CUDA(s, cudaMemset(s->tc_redo, 0, (size_t)kGemmMaxQ * sizeof(int)));
   MS_CUDA(s, cudaMemset(s->tc_fix_counts, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
@@ -259,7 +295,7 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaFuncSetAttribute(tc_fixup_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kFixupCap * sizeof(unsigned long long))));
   MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
   const size_t rs = (size_t)kTcMaxK2 * 8 * sizeof(uint32_t);
-  MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
+  MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
   s->tc_ready = true;
   return MS_OK;
 }
@@ -283,32 +319,53 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     CUtensorMap tmap_q;
     if (!make_tmap_rows_f16(&tmap_q, qptr, (uint64_t)nqb, (uint64_t)c.emb_dim, kGemmMaxQ))
       return fail(s, MS_ERR_CUDA, "cuTensorMapEncodeTiled failed for the query batch");
+    // Candidate rows from the filter kernel itself when k leaves room in the selection that ranks them and the CTAs
+    // have several tiles each (the thresholds need the other CTAs' first tiles); the group maxima serve the rest and
+    // any query whose list turns out unusable.
+    const int k2r = base.k + kTcRowMargin;
+    const int n_ctas = std::min(n_tiles, s->sm_count);
+    const int n_seg = n_ctas * 4;
+    const int seg = std::min(kTcCandSeg, kTcCandPlaces / n_seg);
+    const bool emit = k2r + 1 <= kExtractMaxK && n_tiles >= 2 * s->sm_count && n_rows >= k2r && n_ctas <= kTcMaxCtas && seg >= 8;
+    uint32_t* hist = s->tc_hist;
+    uint32_t* thr_used = hist + (size_t)kGemmMaxQ * kHistWords;
+    uint32_t* cand_cnt = thr_used + kGemmMaxQ;
     GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes,
-                  s->test_spin_limit, s->test_mute_producers, s->removed_bits_d};
-    score_gemm_groupmax_kernel<<<std::min(n_tiles, s->sm_count), kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
-    MS_CUDA(s, cudaGetLastError());
-    select_groups_kernel<<<nqb, kTopkThreads, 0, st>>>(s->tc_gmax, s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best);
+                  s->test_spin_limit, s->test_mute_producers, s->removed_bits_d,
+                  emit ? hist : nullptr, cand_cnt, thr_used, s->tc_emit, seg, k2r};
+    score_gemm_groupmax_kernel<<<n_ctas, kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
     MS_CUDA(s, cudaGetLastError());
     RetrieveParams p = base;
     p.queries = qptr;
     p.nq = nqb;
     p.out_ids = base.out_ids + (int64_t)q0 * base.k;
     p.out_scores = base.out_scores ? base.out_scores + (int64_t)q0 * base.k : nullptr;
-    dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
     float* scores_out = p.out_scores ? p.out_scores : s->tc_scores_out;
-    rescore_topk_kernel<__half><<<grid, kScoreThreads, (size_t)k2 * 8 * sizeof(uint32_t), st>>>(
-        p, s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets, scores_out, s->tc_next_best, s->tc_redo,
-        s->tc_kth);
-    MS_CUDA(s, cudaGetLastError());
+    const int* slow = emit ? s->tc_slow : nullptr;
+    if (emit) {
+      MS_CUDA(s, launch_dependent(select_rows_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const unsigned long long*)s->tc_emit,
+                                  n_seg, seg, (const uint32_t*)cand_cnt, thr_used, hist, kHistWords,
+                                  k2r, s->tc_sel_rows, s->tc_next_best, s->tc_slow, s->tc_list_stats));
+      dim3 rgrid((unsigned)((k2r + kScoreWarps * 8 - 1) / (kScoreWarps * 8)), (unsigned)nqb);
+      MS_CUDA(s, launch_dependent(rescore_topk_kernel<__half, 1>, rgrid, dim3(kScoreThreads), (size_t)k2r * sizeof(uint32_t), st, p,
+                                  (const int32_t*)s->tc_sel_rows, k2r, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets,
+                                  scores_out, (const float*)s->tc_next_best, s->tc_redo, s->tc_kth, slow, 0));
+      s->kernels_launched += 2;
+    }
+    MS_CUDA(s, launch_dependent(select_groups_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const float*)s->tc_gmax,
+                                s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best, slow));
+    dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
+    MS_CUDA(s, launch_dependent(rescore_topk_kernel<__half, 8>, grid, dim3(kScoreThreads), (size_t)k2 * 8 * sizeof(uint32_t), st, p,
+                                (const int32_t*)s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets, scores_out,
+                                (const float*)s->tc_next_best, s->tc_redo, s->tc_kth, slow, 1));
     // the fix-up of the queries whose margin check failed (its CTAs leave at once for all the others, so the grid is
     // kept small: a few CTAs per query, each taking a slice of the segment)
     const int fix_ctas = std::max(1, std::min(8 * s->sm_count / nqb, (int)((n_rows + 2047) / 2048)));
     const int fix_rows = (int)(((n_rows + fix_ctas - 1) / fix_ctas + 1) & ~(int64_t)1);
     dim3 fgrid((unsigned)((n_rows + fix_rows - 1) / fix_rows), (unsigned)nqb);
-    tc_fixup_kernel<__half><<<fgrid, kScoreThreads, kFixupCap * sizeof(unsigned long long), st>>>(
-        p, (int)n_rows, fix_rows, s->tc_redo, s->tc_kth, s->tc_fix_counts, s->tc_fix_keys, s->tc_fix_tickets, scores_out, s->tc_error + 1,
-        s->tc_n_fixups);
-    MS_CUDA(s, cudaGetLastError());
+    MS_CUDA(s, launch_dependent(tc_fixup_kernel<__half>, fgrid, dim3(kScoreThreads), kFixupCap * sizeof(unsigned long long), st, p,
+                                (int)n_rows, fix_rows, s->tc_redo, (const float*)s->tc_kth, s->tc_fix_counts, s->tc_fix_keys,
+                                s->tc_fix_tickets, scores_out, s->tc_error + 1, s->tc_n_fixups));
     s->kernels_launched += 4;
   }
   return MS_OK;
@@ -607,6 +664,11 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_fix_tickets);
     cudaFree(s->tc_n_fixups);
     cudaFree(s->tc_error);
+    cudaFree(s->tc_hist);
+    cudaFree(s->tc_emit);
+    cudaFree(s->tc_sel_rows);
+    cudaFree(s->tc_slow);
+    cudaFree(s->tc_list_stats);
     cudaFree(s->tiles);
     cudaFree(s->cc_slots);
     cudaFree(s->cc_arena);
@@ -1598,6 +1660,7 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
   out->kernel_timeouts = 0;
   out->filter_fixups = 0;
   out->filter_fixup_overflows = 0;
+  out->filter_list_queries = out->filter_list_rows = out->filter_list_fallbacks = 0;
   if (s->tc_error) {
     DeviceGuard g(s->cfg.device);
     int flags[2] = {0, 0};
@@ -1607,6 +1670,11 @@ ms_status memstore_stats(memstore_t* s, memstore_stats_t* out) {
     out->kernel_timeouts = flags[0];
     out->filter_fixup_overflows = flags[1];
     out->filter_fixups = fix;
+    unsigned long long ls[3] = {0, 0, 0};
+    MS_CUDA(s, cudaMemcpy(ls, s->tc_list_stats, sizeof ls, cudaMemcpyDeviceToHost));
+    out->filter_list_queries = (int64_t)ls[0];
+    out->filter_list_rows = (int64_t)ls[1];
+    out->filter_list_fallbacks = (int64_t)ls[2];
   }
   return MS_OK;
 }

@@ -822,9 +822,10 @@ __host__ __device__ __forceinline__ int extract_rounds(int k, int n_warps) { ret
 // in the upper half, 0xffffffff - row in the lower); the other threads get my_rank = -1.  When n < k the ranks from n
 // on have no key.  Returns false otherwise; s_keys holds the n order keys for the fallback either way.
 // `cand` is shared memory for THREADS 64-bit keys.
-template <int THREADS, int KPL>
-__device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long long* cand, const float* __restrict__ sc, uint32_t* s_keys,
-                                             int n, int k, int& my_rank, unsigned long long& my_key) {
+// key_at(i): the order key of place i < n, or 0 for an empty place (no finite score has key 0).
+template <int THREADS, int KPL, class KeyAt>
+__device__ __forceinline__ bool topk_extract_keys(ExtractShared& es, unsigned long long* cand, KeyAt key_at, uint32_t* s_keys, int n, int k,
+                                                  int& my_rank, unsigned long long& my_key) {
   constexpr int NW = THREADS / 32;
   constexpr unsigned kFull = 0xffffffffu;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -833,12 +834,14 @@ __device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long lo
 #pragma unroll
   for (int j = 0; j < KPL; ++j) {
     const int i = j * THREADS + tid;
-    key[j] = i < n ? order_key(__ldcg(sc + i)) : 0u;  // 0 marks an empty place (no finite score has key 0)
+    key[j] = i < n ? key_at(i) : 0u;
   }
+  if (s_keys != nullptr) {  // (the caller's fallback wants them)
 #pragma unroll
-  for (int j = 0; j < KPL; ++j) {
-    const int i = j * THREADS + tid;
-    if (i < n) s_keys[i] = key[j];
+    for (int j = 0; j < KPL; ++j) {
+      const int i = j * THREADS + tid;
+      if (i < n) s_keys[i] = key[j];
+    }
   }
   if (tid == 0) {
     es.bound = 0u;
@@ -923,6 +926,12 @@ __device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long lo
   }
   __syncwarp();
   return true;
+}
+
+template <int THREADS, int KPL>
+__device__ __forceinline__ bool topk_extract(ExtractShared& es, unsigned long long* cand, const float* __restrict__ sc, uint32_t* s_keys,
+                                             int n, int k, int& my_rank, unsigned long long& my_key) {
+  return topk_extract_keys<THREADS, KPL>(es, cand, [&](int i) { return order_key(__ldcg(sc + i)); }, s_keys, n, k, my_rank, my_key);
 }
 
 // Scoring only (large segments): grid = (row groups, nq); dynamic shared memory holds the query as fp32.
@@ -1095,12 +1104,17 @@ __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const Retrieve
 
 // Step 2: per query, the k2 groups with the largest group maximum, written in ASCENDING group order (so that the
 // candidate rows of step 3 are in row order and "lower index first" among equal scores means "lower fact id first").
+// `only` (or nullptr): the queries to serve are those with only[q] != 0 - the ones whose candidate list from the
+// filter kernel was unusable; the others are served by select_rows_kernel.
 __global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
-                                                                    int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/) {
+                                                                    int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/, const int* only) {
   __shared__ TopkShared sm;
   __shared__ int32_t s_sel[512];
   __shared__ float s_val[512];
+  grid_dependency_wait();  // every kernel of this chain is a programmatic dependent of the one before it
+  grid_launch_dependents();
   const int q = blockIdx.x;
+  if (only != nullptr && !only[q]) return;
   int32_t* out = sel + (int64_t)q * k2;
   // one group more than asked for: its maximum is the best score the filter saw among the rows that will NOT be
   // rescored, which the rescoring step compares with the k-th exact score it finds
@@ -1117,6 +1131,85 @@ __global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const fl
       rank += (other < mine) || (other == mine && j < i);
     }
     out[rank] = (int32_t)mine;
+  }
+}
+
+// Step 2 when the filter kernel emitted candidate rows (see score_gemm.cuh): per query, the k2 candidates with the best
+// filter scores, written in ascending row order, and the best filter score among all the rows that will not be
+// rescored: the (k2+1)-th candidate's, or the highest threshold the filter applied (every row it did not emit scored
+// below that), whichever is larger.  The candidates of a query sit in one segment of `seg` places per epilogue warp of the
+// filter kernel, cand_cnt[q][segment] of them used.  Fewer than k2 candidates in all, a warp that found more than its
+// segment holds, or more candidates tied at the cut than the selection ranks, sets slow[q]: select_groups_kernel then
+// serves the query from the group maxima.  The CTA also leaves the query's histogram and threshold record zeroed for
+// the next call.
+constexpr int kCandKpl = 16;       // places of one query over all segments <= kTopkThreads * kCandKpl
+constexpr int kCandMaxSegs = 1024;
+__global__ void __launch_bounds__(kTopkThreads, 1) select_rows_kernel(const unsigned long long* cand, int n_seg, int seg, const uint32_t* cand_cnt,
+                                                                  uint32_t* thr_used, uint32_t* hist, int hist_words, int k2,
+                                                                  int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/, int* slow /*[nq]*/,
+                                                                  unsigned long long* list_stats /*served, rows listed, fallbacks*/) {
+  __shared__ ExtractShared es;
+  __shared__ unsigned long long s_cand[kTopkThreads];
+  __shared__ uint8_t s_used[kCandMaxSegs];  // per segment
+  __shared__ int32_t s_rows[kExtractMaxK];
+  __shared__ float s_next;
+  __shared__ uint32_t s_total;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  const int q = blockIdx.x;
+  const uint32_t tk = thr_used[q];
+  if (threadIdx.x == 0) {
+    s_next = -INFINITY;
+    s_total = 0u;
+  }
+  __syncthreads();
+  int overrun = 0;
+  for (int i = threadIdx.x; i < n_seg && i < kCandMaxSegs; i += kTopkThreads) {
+    const uint32_t c = cand_cnt[(size_t)q * n_seg + i];
+    overrun |= c > (uint32_t)seg;
+    s_used[i] = (uint8_t)min(c, (uint32_t)seg);
+    if (c) atomicAdd(&s_total, min(c, (uint32_t)seg));
+  }
+  overrun = __syncthreads_or(overrun);
+  const uint32_t n = s_total;
+  {  // clean for the next call
+    uint4* hq = reinterpret_cast<uint4*>(hist + (size_t)q * hist_words);  // hist_words is a multiple of 4
+    for (int i = threadIdx.x; i < hist_words / 4; i += kTopkThreads) hq[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (threadIdx.x == 0) thr_used[q] = 0u;
+  }
+  const int n_places = n_seg * seg;
+  bool ok = !overrun && n >= (uint32_t)k2 && k2 + 1 <= kExtractMaxK && n_places <= kTopkThreads * kCandKpl && n_seg <= kCandMaxSegs && seg < 256;
+  int my_rank = -1;
+  unsigned long long my_key = 0ull;
+  const unsigned long long* mine = cand + (size_t)q * n_places;
+  if (ok)
+    ok = topk_extract_keys<kTopkThreads, kCandKpl>(
+        es, s_cand, [&](int i) { return (uint32_t)(i % seg) < (uint32_t)s_used[i / seg] ? (uint32_t)(__ldcg(mine + i) >> 32) : 0u; }, nullptr,
+        n_places, k2 + 1, my_rank, my_key);
+  if (threadIdx.x == 0) {
+    atomicAdd(list_stats + (ok ? 0 : 2), 1ull);
+    if (ok) atomicAdd(list_stats + 1, (unsigned long long)n);
+  }
+  if (!ok) {
+    if (threadIdx.x == 0) slow[q] = 1;
+    return;
+  }
+  if (my_rank >= 0) {
+    if (my_rank < k2) s_rows[my_rank] = (int32_t)(uint32_t)__ldcg(mine + (0xffffffffu - (uint32_t)my_key));
+    else s_next = key_score((uint32_t)(my_key >> 32));
+  }
+  __syncwarp();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    slow[q] = 0;
+    next_best[q] = fmaxf(s_next, tk ? key_score(tk) : -INFINITY);
+  }
+  // ascending row order by counting (the rows are distinct)
+  if (threadIdx.x < k2) {
+    const int32_t mine_row = s_rows[threadIdx.x];
+    int rank = 0;
+    for (int j = 0; j < k2; ++j) rank += s_rows[j] < mine_row;
+    sel[(size_t)q * k2 + rank] = mine_row;
   }
 }
 
@@ -1173,43 +1266,60 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
 // a row outside the selected groups may belong to the top-k: redo[q] is raised and kth[q] tells the fix-up kernel which
 // exact score a row must reach.
 constexpr float kTcFilterRounding = 1e-5f;  // tensor-core fp32 accumulation against the fixed-order CUDA-core sum, times max(1, |score|)
-template <typename T>
+// GROUP = 8: sel holds groups (candidate c of query q is row sel[q][c / 8] * 8 + c % 8); GROUP = 1: sel holds rows
+// (candidate c is row sel[q][c]; n_sel a multiple of 2 or its last candidate is scored alone).  slow / want_slow:
+// when slow != nullptr the kernel serves the queries with (slow[q] != 0) == want_slow and leaves the others alone.
+template <typename T, int GROUP>
 __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const RetrieveParams p, const int32_t* sel, int k2, int n_rows,
                                                                      float* cand_scores, int32_t* cand_rows, uint32_t* tickets,
-                                                                     float* scores_out, const float* next_best, int* redo, float* kth) {
+                                                                     float* scores_out, const float* next_best, int* redo, float* kth,
+                                                                     const int* slow, int want_slow) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ int s_last;
+  grid_dependency_wait();
+  grid_launch_dependents();
   const int q = blockIdx.y;
-  const int n_cand = k2 * 8;
+  if (slow != nullptr && (slow[q] != 0) != (want_slow != 0)) return;
+  const int n_cand = k2 * GROUP;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const T* seg = reinterpret_cast<const T*>(p.emb);  // user 0
   float* cs = cand_scores + (int64_t)q * n_cand;
   int32_t* cr = cand_rows + (int64_t)q * n_cand;
-  const int c0 = blockIdx.x * kScoreWarps * 8;  // one group of 8 candidate rows per warp
-  {
-    const int g_idx = c0 / 8 + warp;
-    if (g_idx < k2) {
-      const int32_t g = sel[(int64_t)q * k2 + g_idx];
-      for (int r = 0; r < 8; r += 2) {  // two rows of the group in flight at a time
-        const int64_t row = (int64_t)g * 8 + r;
-        const bool ok0 = g >= 0 && row < n_rows, ok1 = g >= 0 && row + 1 < n_rows;
-        float s0 = -INFINITY, s1 = -INFINITY;
-        if (ok1) {
-          score_two_rows<T>(p, q, seg, row, row + 1, s0, s1);
-          s0 += 0.0f;
-          s1 += 0.0f;
-        } else if (ok0) {
-          s0 = score_one_row<T>(p, q, seg, row) + 0.0f;
+  const int c0 = (blockIdx.x * kScoreWarps + warp) * 8;  // eight candidate rows per warp
+  if (c0 < n_cand) {
+    for (int r = 0; r < 8; r += 2) {  // two rows in flight at a time
+      int64_t row0 = -1, row1 = -1;
+      if (GROUP == 8) {
+        const int32_t g = sel[(int64_t)q * k2 + c0 / 8];
+        if (g >= 0) {
+          row0 = (int64_t)g * 8 + r;
+          row1 = row0 + 1;
         }
-        // a removed row stays a candidate (the valid candidates must remain a prefix) with the score of a removed row
-        if (ok0 && row_removed(p, 0, row)) s0 = -INFINITY;
-        if (ok1 && row_removed(p, 0, row + 1)) s1 = -INFINITY;
-        if (lane == 0) {
-          cs[g_idx * 8 + r] = s0;
-          cr[g_idx * 8 + r] = ok0 ? (int32_t)row : -1;
-          cs[g_idx * 8 + r + 1] = s1;
-          cr[g_idx * 8 + r + 1] = ok1 ? (int32_t)(row + 1) : -1;
+      } else {
+        if (c0 + r < n_cand) row0 = sel[(int64_t)q * k2 + c0 + r];
+        if (c0 + r + 1 < n_cand) row1 = sel[(int64_t)q * k2 + c0 + r + 1];
+      }
+      const bool ok0 = row0 >= 0 && row0 < n_rows, ok1 = row1 >= 0 && row1 < n_rows;
+      float s0 = -INFINITY, s1 = -INFINITY;
+      if (ok0 && ok1) {
+        score_two_rows<T>(p, q, seg, row0, row1, s0, s1);
+        s0 += 0.0f;
+        s1 += 0.0f;
+      } else if (ok0) {
+        s0 = score_one_row<T>(p, q, seg, row0) + 0.0f;
+      }
+      // a removed row stays a candidate (the valid candidates must remain a prefix) with the score of a removed row
+      if (ok0 && row_removed(p, 0, row0)) s0 = -INFINITY;
+      if (ok1 && row_removed(p, 0, row1)) s1 = -INFINITY;
+      if (lane == 0) {
+        if (c0 + r < n_cand) {
+          cs[c0 + r] = s0;
+          cr[c0 + r] = ok0 ? (int32_t)row0 : -1;
+        }
+        if (c0 + r + 1 < n_cand) {
+          cs[c0 + r + 1] = s1;
+          cr[c0 + r + 1] = ok1 ? (int32_t)row1 : -1;
         }
       }
     }
@@ -1271,6 +1381,7 @@ __global__ void __launch_bounds__(kScoreThreads) tc_fixup_kernel(const RetrieveP
                                                                  uint32_t* tickets, float* scores_out, int* overflow, uint32_t* n_fixups) {
   extern __shared__ unsigned long long s_fix[];  // kFixupCap keys
   __shared__ int s_last;
+  grid_dependency_wait();
   const int q = blockIdx.y;
   if (!redo[q]) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

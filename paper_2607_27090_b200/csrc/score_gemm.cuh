@@ -7,6 +7,23 @@
 // best groups per query and rescores their rows with the exact CUDA-core routine, so tensor-core rounding never
 // decides a rank; it only has to keep every top-k row inside a selected group.
 //
+// With candidate emission on (GemmParams::hist) the kernel ALSO hands the later steps a short list of candidate ROWS per
+// query, so that they need not sweep the group maxima nor rescore whole groups: the epilogue keeps, per query, a
+// histogram of the group maxima seen so far by all CTAs (buckets = the top 13 bits of the order-preserving key:
+// sign, exponent, 4 significand bits; with two coarser levels over the top 9 and the top 5 bits, so that a reader
+// finds its bucket with three loads of one line each), from which any warp can read a
+// threshold - the lower edge of the bucket in which the count of maxima from the top reaches k2.  At least k2 rows
+// score at or above it (group maxima are scores of distinct rows), so a row below it is not among the k2 best; every
+// row at or above the current threshold is appended to the query's candidate list (row, filter score).  The
+// threshold only rises and a stale one only lets more rows through: the histogram is updated with fire-and-forget
+// atomics, a seventh warp of every CTA does nothing but read it and keep the CTA's 64 thresholds in shared memory, and
+// the epilogue warps never wait for global memory: a warp appends to its OWN segment of every query's list
+// ([query][CTA][warp][cand_seg] places, counted in registers) and publishes its counts when it ends.  The first tile of a
+// CTA is computed before any threshold exists; its accumulator stays parked in tensor memory and its rows are emitted
+// after the CTA's last tile.  The list's consumer checks the counts (at least k2 rows in all, no segment overrun) and
+// falls back to the group maxima otherwise.  (Same-address atomics drain at about 8 ns each: the first tiles of all
+// CTAs arrive together, so a warp counts one maximum per query for them - that of its 32 rows - not four.)
+//
 // Tiling: facts on M (128 rows per tile = the 128 TMEM lanes), queries on N (64), K = E in chunks of 64 fp16
 // (one 128-byte swizzle row).  All queries stay in shared memory for the kernel's lifetime (E/64 chunks of 8 KiB);
 // embedding tiles stream through a 4-stage ring of 16 KiB TMA boxes.  Accumulators are double-buffered in TMEM
@@ -14,6 +31,7 @@
 //   warp 0     TMA producer (one elected lane)
 //   warp 1     TMEM allocation, tcgen05.mma issue (one elected lane), tcgen05.commit -> mbarriers
 //   warps 2-5  epilogue: tcgen05.ld of the warp's 32 TMEM lanes, row mask, 8-row max by shuffles, 16-byte stores
+//   warp 6     thresholds of the candidate emission (idle without it)
 // Every mbarrier wait is bounded; a time-out sets *error_flag, the roles stop, TMEM is released and the CTA leaves.
 #pragma once
 #include <cuda.h>
@@ -29,8 +47,14 @@ constexpr size_t kGemmSmemBytes = 232448;  // all the dynamic shared memory a CT
 constexpr int kGemmMaxQ = 64;
 constexpr int kGemmGroupRows = 8;
 constexpr int kGemmGroupsPerTile = kGemmTileRows / kGemmGroupRows;  // 16
-constexpr int kGemmThreads = 192;
-constexpr int kGemmTmemCols = 128;
+constexpr int kGemmThreads = 224;
+constexpr int kGemmTmemCols = 512;    // all of an SM's tensor memory (one CTA per SM, and an allocation is a power of two)
+constexpr int kGemmAccBufs = 4;       // working accumulators of 64 columns: the MMAs may run this many tiles ahead of the epilogue
+constexpr int kGemmParked = 2;        // first tiles of a CTA whose accumulators stay in tensor memory (candidate emission only)
+constexpr int kHistFine = 8192;       // order key >> 19
+constexpr int kHistMid = 512;         // order key >> 23: 16 fine buckets each
+constexpr int kHistCoarse = 32;       // order key >> 27: 16 middle buckets each
+constexpr int kHistWords = kHistCoarse + kHistMid + kHistFine;  // one query's counters: [coarse][middle][fine]
 constexpr int kGemmABytes = kGemmTileRows * kGemmKChunk * 2;  // 16 KiB
 constexpr int kGemmQBytes = kGemmMaxQ * kGemmKChunk * 2;      // 8 KiB per chunk
 constexpr int kGemmMaxE = 1024;
@@ -46,12 +70,75 @@ struct GemmParams {
   uint32_t spin_limit;  // 0: the default bound of every wait; else a test's shorter bound
   int mute_producer;    // test aid: the producer role issues nothing, so the other roles' waits run out
   const uint32_t* removed_bits;  // one bit per row of the segment, or nullptr: removed rows take no part in a group's maximum
+  // candidate emission (hist == nullptr: off).  All counters are zero when the kernel starts.
+  uint32_t* hist;         // [kGemmMaxQ][kHistWords]
+  uint32_t* cand_cnt;     // [kGemmMaxQ][gridDim.x * 4]: rows the warp found for the query (beyond cand_seg: the surplus was dropped)
+  uint32_t* thr_used;     // [kGemmMaxQ]: order key of the highest threshold any CTA applied (0: none)
+  unsigned long long* cand;  // [kGemmMaxQ][gridDim.x * 4][cand_seg]: (order key of the filter score << 32) | row
+  int cand_seg;
+  int k2;                 // group maxima the threshold keeps at or above it
 };
+
+__device__ __forceinline__ uint32_t gemm_order_key(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float gemm_key_value(uint32_t kx) {
+  return __uint_as_float((kx & 0x80000000u) ? (kx & 0x7fffffffu) : ~kx);
+}
+
+// One level of the threshold search, for two queries at once (the loads of both are issued together): counters
+// c[0..N) of each, scanned from the top; `cum` counts the maxima above the bucket that is returned, the first one from
+// the top at which the running count reaches `need` (-1: not reached).
+template <int NVEC>
+__device__ __forceinline__ void hist_scan2(const uint32_t* a, const uint32_t* b, uint32_t need, uint32_t& cum_a, uint32_t& cum_b, int& at_a,
+                                           int& at_b) {
+  uint4 ca[NVEC], cb[NVEC];
+#pragma unroll
+  for (int i = 0; i < NVEC; ++i) {
+    ca[i] = __ldcg(reinterpret_cast<const uint4*>(a) + i);
+    cb[i] = __ldcg(reinterpret_cast<const uint4*>(b) + i);
+  }
+  at_a = at_b = -1;
+  auto scan1 = [&](uint32_t x, int idx, uint32_t& cum, int& at) {
+    if (at < 0) {
+      if (cum + x >= need) at = idx;
+      else cum += x;
+    }
+  };
+#pragma unroll
+  for (int i = NVEC - 1; i >= 0; --i) {
+    scan1(ca[i].w, 4 * i + 3, cum_a, at_a);
+    scan1(ca[i].z, 4 * i + 2, cum_a, at_a);
+    scan1(ca[i].y, 4 * i + 1, cum_a, at_a);
+    scan1(ca[i].x, 4 * i, cum_a, at_a);
+    scan1(cb[i].w, 4 * i + 3, cum_b, at_b);
+    scan1(cb[i].z, 4 * i + 2, cum_b, at_b);
+    scan1(cb[i].y, 4 * i + 1, cum_b, at_b);
+    scan1(cb[i].x, 4 * i, cum_b, at_b);
+  }
+}
+
+// The thresholds of two queries from their histograms (ha, hb: the queries' kHistWords counters).  -infinity while
+// fewer than `need` maxima have been published.  A coarser counter may run ahead of the finer ones for a moment; the
+// search then stops at the coarser bucket's lower edge, which is lower and therefore still valid.
+__device__ __forceinline__ void hist_thresholds2(const uint32_t* ha, const uint32_t* hb, uint32_t need, float& ta, float& tb) {
+  uint32_t cum_a = 0, cum_b = 0;
+  int ca, cb, ma, mb, fa, fb;
+  hist_scan2<kHistCoarse / 4>(ha, hb, need, cum_a, cum_b, ca, cb);
+  const int ca0 = ca < 0 ? 0 : ca, cb0 = cb < 0 ? 0 : cb;
+  hist_scan2<4>(ha + kHistCoarse + ca0 * 16, hb + kHistCoarse + cb0 * 16, need, cum_a, cum_b, ma, mb);
+  const int ma0 = ca0 * 16 + (ma < 0 ? 0 : ma), mb0 = cb0 * 16 + (mb < 0 ? 0 : mb);
+  hist_scan2<4>(ha + kHistCoarse + kHistMid + ma0 * 16, hb + kHistCoarse + kHistMid + mb0 * 16, need, cum_a, cum_b, fa, fb);
+  const uint32_t bucket_a = (uint32_t)ma0 * 16u + (uint32_t)(fa < 0 ? 0 : fa), bucket_b = (uint32_t)mb0 * 16u + (uint32_t)(fb < 0 ? 0 : fb);
+  ta = ca < 0 ? -INFINITY : gemm_key_value(bucket_a << 19);
+  tb = cb < 0 ? -INFINITY : gemm_key_value(bucket_b << 19);
+}
 
 // Shared memory after the 1 KiB alignment of the base: queries, ring, epilogue staging (4 warps x [4 groups][32
 // queries] floats), barriers.
 constexpr uint32_t kGemmStagingBytes = 4 * 4 * 32 * sizeof(float);
-constexpr uint32_t kGemmBarrierBytes = 256;
+constexpr uint32_t kGemmBarrierBytes = 512;  // barriers and flags (< 256 bytes), 64 thresholds
 __host__ __device__ constexpr int gemm_stages(uint32_t usable_bytes, int emb_dim) {
   const int64_t left = (int64_t)usable_bytes - (int64_t)(emb_dim / kGemmKChunk) * kGemmQBytes - kGemmStagingBytes - kGemmBarrierBytes;
   const int64_t n = left / kGemmABytes;
@@ -110,6 +197,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* r) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Count one maximum in the three levels of its query's histogram (lanes with `mine` false do nothing).
+__device__ __forceinline__ void hist_publish(uint32_t* hq, float gx, bool mine) {
+  if (mine && gx > -INFINITY) {
+    const uint32_t bucket = gemm_order_key(gx) >> 19;
+    atomicAdd(hq + kHistCoarse + kHistMid + bucket, 1u);
+    atomicAdd(hq + kHistCoarse + (bucket >> 4), 1u);
+    atomicAdd(hq + (bucket >> 8), 1u);
+  }
+}
+
+// One column of the warp's 32 tensor-memory lanes; the value is there after tmem_ld_wait().
+__device__ __forceinline__ uint32_t tmem_ld1_issue(uint32_t taddr) {
+  uint32_t u;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(u) : "r"(taddr) : "memory");
+  return u;
+}
+__device__ __forceinline__ float4 lds_volatile_f4(const volatile float* p) {
+  float4 r;
+  asm volatile("ld.volatile.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(smem_u32(const_cast<const float*>(p))));
+  return r;
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
     score_gemm_groupmax_kernel(const __grid_constant__ CUtensorMap tmap_emb, const __grid_constant__ CUtensorMap tmap_q,
                                const GemmParams p) {
@@ -126,9 +235,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   uint64_t* full = bars + 1;
   uint64_t* empty = full + kGemmMaxStages;
   uint64_t* acc_full = empty + kGemmMaxStages;
-  uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* acc_empty = acc_full + kGemmAccBufs + kGemmParked;  // acc_full[kGemmAccBufs + j]: parked tile j
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + kGemmAccBufs);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* thr_ready = abort_flag + 1;  // every query of the batch has a threshold
+  volatile int* epi_done = abort_flag + 2;   // epilogue warps that have finished
+  volatile float* s_thr = reinterpret_cast<volatile float*>(reinterpret_cast<uint8_t*>(bars) + 256);  // [64]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (n_stages < 2) {  // cannot happen with the launch this library makes; nothing has been set up yet
@@ -141,14 +253,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kGemmAccBufs; ++b) {
       mbar_init(&acc_full[b], 1);
       mbar_init(&acc_empty[b], 4);
     }
+    for (int j = 0; j < kGemmParked; ++j) mbar_init(&acc_full[kGemmAccBufs + j], 1);
     *abort_flag = 0;
+    *thr_ready = 0;
+    *epi_done = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (threadIdx.x < kGemmMaxQ) s_thr[threadIdx.x] = -INFINITY;
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kGemmTmemCols)
                  : "memory");
@@ -161,6 +277,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 
   const int n_tiles = (p.n_rows + kGemmTileRows - 1) / kGemmTileRows;
   const uint32_t limit = p.spin_limit ? p.spin_limit : kSpinLimit;
+  const bool emitting = p.hist != nullptr;
+  const int n_parked = emitting ? kGemmParked : 0;
+  grid_launch_dependents();  // the kernels that follow are programmatic dependents: they are placed as SMs free up and wait for this grid
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -191,9 +310,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       uint32_t ph = 0;
       int it = 0;
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++it) {
-        const int b = it & 1;
-        ok = mbar_wait(&acc_empty[b], (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag, limit);
-        if (!ok) break;
+        // with emission on, the CTA's first tiles go to the parked columns (nobody reuses them); the others take the
+        // working buffers in turn
+        const bool parked = it < n_parked;
+        const int wi = it - n_parked;
+        const int b = parked ? kGemmAccBufs + it : wi % kGemmAccBufs;
+        if (!parked) {
+          ok = mbar_wait(&acc_empty[b], (uint32_t)((wi / kGemmAccBufs) & 1) ^ 1u, abort_flag, limit);
+          if (!ok) break;
+        }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * kGemmMaxQ);
         for (int kc = 0; kc < nkc; ++kc) {
@@ -215,26 +340,164 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       }
     }
     __syncwarp();
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ thresholds (candidate emission only)
+    // Reads the histogram over and over (three loads of a line per query and round, two queries per lane) and raises
+    // the thresholds in shared memory; ends when the four epilogue warps have, or after a bounded number of rounds.
+    if (emitting) {
+      const int qa = lane < p.nq ? lane : 0, qb = lane + 32 < p.nq ? lane + 32 : 0;
+      float mine_a = -INFINITY, mine_b = -INFINITY;
+      int settled = 0;  // rounds since every query has had a threshold
+      for (uint32_t round = 0; round < limit && *epi_done < 4 && !*abort_flag; ++round) {
+        float ta, tb;
+        hist_thresholds2(p.hist + (size_t)qa * kHistWords, p.hist + (size_t)qb * kHistWords, (uint32_t)p.k2, ta, tb);
+        if (lane < p.nq && ta > mine_a) {
+          mine_a = ta;
+          s_thr[lane] = ta;
+          atomicMax(p.thr_used + lane, gemm_order_key(ta));
+        }
+        if (lane + 32 < p.nq && tb > mine_b) {
+          mine_b = tb;
+          s_thr[lane + 32] = tb;
+          atomicMax(p.thr_used + lane + 32, gemm_order_key(tb));
+        }
+        const bool have = (lane >= p.nq || mine_a > -INFINITY) && (lane + 32 >= p.nq || mine_b > -INFINITY);
+        if (__all_sync(0xffffffffu, have) && lane == 0) *thr_ready = 1;
+        // the thresholds settle within the first few tiles: read quickly at first, then every 16 us or so (every round
+        // costs the L2 a line per level and query); asleep in short naps so that the end of the CTA is noticed at once
+        if (*thr_ready) ++settled;
+        const int naps = settled < 7 ? (settled ? 1 << (settled - 1) : 1) : 64;
+        for (int w = 0; w < naps && *epi_done < 4 && !*abort_flag; ++w) __nanosleep(256);
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue
+    constexpr unsigned kFull = 0xffffffffu;
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
     float* my_stage = stage_f + (size_t)(warp - 2) * 4 * 32;
-    int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const int b = it & 1;
-      if (!mbar_wait(&acc_full[b], (uint32_t)((it >> 1) & 1), abort_flag, limit)) break;
+    const uint32_t lane_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    // Which of the thread's 64 scores (its row against every query) reach the query's threshold: one bit per query.
+    // Kept short (the rest of the work is done only for the few queries with a bit set in some lane of the warp).
+    auto passes = [&](const float (&v)[kGemmMaxQ], bool out, uint32_t& m_lo, uint32_t& m_hi) {
+      m_lo = m_hi = 0u;
+#pragma unroll
+      for (int q4 = 0; q4 < kGemmMaxQ / 4; ++q4) {
+        const float4 t = lds_volatile_f4(s_thr + 4 * q4);
+        const uint32_t bits = (v[4 * q4] >= t.x ? 1u : 0u) | (v[4 * q4 + 1] >= t.y ? 2u : 0u) | (v[4 * q4 + 2] >= t.z ? 4u : 0u) |
+                              (v[4 * q4 + 3] >= t.w ? 8u : 0u);
+        if (q4 < 8) m_lo |= bits << (4 * (q4 & 7));
+        else m_hi |= bits << (4 * (q4 & 7));
+      }
+      if (out) m_lo = m_hi = 0u;
+      if (p.nq < 32) {
+        m_lo &= (1u << p.nq) - 1u;
+        m_hi = 0u;
+      } else if (p.nq < 64) {
+        m_hi &= (1u << (p.nq - 32)) - 1u;
+      }
+    };
+    // For every query with a bit set somewhere in the warp (two of them at a time, so that their chains of dependent
+    // instructions overlap): the score is read again from tensor memory (a dynamic column; the 64 values in registers can
+    // only be indexed at compile time).  Rows whose bit is set join the query's candidate list, in this warp's own
+    // segment of it (lane l counts the rows found for queries l and l + 32).  publish: the best of the warp's rows for
+    // the query is counted in the histogram (it reaches the threshold; lower values could not raise it): one lane per
+    // level, both queries in one instruction.
+    uint32_t cnt_lo = 0u, cnt_hi = 0u;
+    const size_t my_seg = (size_t)blockIdx.x * 4 + (size_t)(warp - 2);
+    const size_t n_seg = (size_t)gridDim.x * 4;
+    auto serve = [&](uint32_t taddr, int row, uint32_t m_lo, uint32_t m_hi, bool publish) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t m = h ? m_hi : m_lo;
+        uint32_t& cnt = h ? cnt_hi : cnt_lo;
+        uint32_t any = __reduce_or_sync(kFull, m);
+        while (any) {
+          const int qa = __ffs(any) - 1;
+          any &= any - 1u;
+          const bool two = any != 0u;
+          const int qb = two ? __ffs(any) - 1 : qa;
+          if (two) any &= any - 1u;
+          const uint32_t ua = tmem_ld1_issue(taddr + (uint32_t)(qa + 32 * h)), ub = tmem_ld1_issue(taddr + (uint32_t)(qb + 32 * h));
+          tmem_ld_wait();
+          const uint32_t ka = gemm_order_key(__uint_as_float(ua)), kb = gemm_order_key(__uint_as_float(ub));
+          const bool pa = (m >> qa) & 1u, pb = two && ((m >> qb) & 1u);  // (no bit is set for a row that is masked out)
+          const unsigned va = __ballot_sync(kFull, pa), vb = __ballot_sync(kFull, pb);
+          const uint32_t base_a = __shfl_sync(kFull, cnt, qa), base_b = __shfl_sync(kFull, cnt, qb);
+          if (lane == qa) cnt += (uint32_t)__popc(va);
+          if (two && lane == qb) cnt += (uint32_t)__popc(vb);
+          const unsigned below = (1u << lane) - 1u;
+          const uint32_t slot_a = base_a + (uint32_t)__popc(va & below), slot_b = base_b + (uint32_t)__popc(vb & below);
+          if (pa && slot_a < (uint32_t)p.cand_seg)
+            p.cand[((size_t)(qa + 32 * h) * n_seg + my_seg) * p.cand_seg + slot_a] = ((unsigned long long)ka << 32) | (uint32_t)row;
+          if (pb && slot_b < (uint32_t)p.cand_seg)
+            p.cand[((size_t)(qb + 32 * h) * n_seg + my_seg) * p.cand_seg + slot_b] = ((unsigned long long)kb << 32) | (uint32_t)row;
+          if (publish) {
+            const uint32_t best_a = __reduce_max_sync(kFull, pa ? ka : 0u), best_b = __reduce_max_sync(kFull, pb ? kb : 0u);
+            if (lane < (two ? 6 : 3)) {
+              const bool second = lane >= 3;
+              const int level = second ? lane - 3 : lane;
+              const uint32_t bucket = (second ? best_b : best_a) >> 19;
+              uint32_t* hq = p.hist + (size_t)((second ? qb : qa) + 32 * h) * kHistWords;
+              atomicAdd(level == 0 ? hq + kHistCoarse + kHistMid + bucket : level == 1 ? hq + kHistCoarse + (bucket >> 4) : hq + (bucket >> 8), 1u);
+            }
+          }
+        }
+      }
+      __syncwarp();
+    };
+    auto row_of = [&](int tile, bool& out) {
+      const int row = tile * kGemmTileRows + quarter * 32 + lane;
+      out = row >= p.n_rows;
+      if (!out && p.removed_bits != nullptr) out = (__ldg(p.removed_bits + (row >> 5)) >> (row & 31)) & 1u;
+      return row;
+    };
+    // The rows of parked tile j (the CTA's j-th tile) against the thresholds as they stand now.
+    auto emit_parked = [&](int j) {
       tc_fence_after();
       float v[kGemmMaxQ];
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * kGemmMaxQ);
+      const uint32_t taddr = lane_taddr + (uint32_t)((kGemmAccBufs + j) * kGemmMaxQ);
       tmem_ld32(taddr, v);
       tmem_ld32(taddr + 32, v + 32);
       tmem_ld_wait();
+      bool out;
+      const int row = row_of((int)blockIdx.x + j * (int)gridDim.x, out);
+      uint32_t m_lo, m_hi;
+      passes(v, out, m_lo, m_hi);
+      serve(taddr, row, m_lo, m_hi, false);
+      tc_fence_before();
+    };
+    // Before the first rows are compared with thresholds: give the threshold warp a moment to see the first tiles of
+    // the other CTAs (bounded; without thresholds every row would be listed).  The MMAs go on meanwhile.
+    auto await_thresholds = [&]() {
+      for (int w = 0; w < 512 && !*thr_ready && !*abort_flag; ++w) __nanosleep(128);
+    };
+    int it = 0, parked_emitted = 0;
+    bool complete = true;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+      const bool parked = it < n_parked;
+      const int wi = it - n_parked;
+      const int b = parked ? kGemmAccBufs + it : wi % kGemmAccBufs;
+      if (emitting && it == n_parked) await_thresholds();  // the first tile whose rows are compared with thresholds
+      if (!mbar_wait(&acc_full[b], parked ? 0u : (uint32_t)((wi / kGemmAccBufs) & 1), abort_flag, limit)) {
+        complete = false;
+        break;
+      }
+      tc_fence_after();
+      float v[kGemmMaxQ];
+      const uint32_t taddr = lane_taddr + (uint32_t)(b * kGemmMaxQ);
+      tmem_ld32(taddr, v);
+      tmem_ld32(taddr + 32, v + 32);
+      tmem_ld_wait();
+      bool out;
+      const int row = row_of(tile, out);
+      if (emitting && !parked) {
+        uint32_t m_lo, m_hi;
+        passes(v, out, m_lo, m_hi);
+        serve(taddr, row, m_lo, m_hi, true);
+      }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[b]);  // the MMAs of the tile after next may overwrite this buffer
-      const int row = tile * kGemmTileRows + quarter * 32 + lane;
-      bool out = row >= p.n_rows;
-      if (!out && p.removed_bits != nullptr) out = (__ldg(p.removed_bits + (row >> 5)) >> (row & 31)) & 1u;
+      if (!parked && lane == 0) mbar_arrive(&acc_empty[b]);  // the MMAs of a later tile may overwrite this buffer
       if (out) {
 #pragma unroll
         for (int q = 0; q < kGemmMaxQ; ++q) v[q] = -INFINITY;
@@ -242,9 +505,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 #pragma unroll
       for (int q = 0; q < kGemmMaxQ; ++q) {
         float x = v[q];
-        x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
-        x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
-        x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
+        x = fmaxf(x, __shfl_xor_sync(kFull, x, 1));
+        x = fmaxf(x, __shfl_xor_sync(kFull, x, 2));
+        x = fmaxf(x, __shfl_xor_sync(kFull, x, 4));
         v[q] = x;
       }
       // transpose through shared memory, 32 queries at a time: lane q then owns the four group maxima of query q
@@ -262,10 +525,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
         if (q < p.nq) {
           const float4 g = make_float4(my_stage[lane], my_stage[32 + lane], my_stage[64 + lane], my_stage[96 + lane]);
           *reinterpret_cast<float4*>(p.gmax + (int64_t)q * p.gmax_stride + col) = g;
+          // a parked tile is computed before any threshold exists: the best of the warp's 32 rows feeds the histogram,
+          // and the rows are looked at again later
+          if (parked) hist_publish(p.hist + (size_t)q * kHistWords, fmaxf(fmaxf(g.x, g.y), fmaxf(g.z, g.w)), true);
         }
         __syncwarp();
       }
+      // the parked tiles' rows, once the thresholds have seen a few tiles of every CTA, in time the epilogue would
+      // otherwise spend waiting for the next accumulator
+      if (parked_emitted < n_parked && it >= n_parked + 3 + 2 * parked_emitted) emit_parked(parked_emitted++);
     }
+    if (complete && parked_emitted < n_parked && parked_emitted < it) {  // a CTA with few tiles
+      if (it <= n_parked) await_thresholds();
+      while (parked_emitted < n_parked && parked_emitted < it) emit_parked(parked_emitted++);
+    }
+    if (emitting) {
+      if (lane < p.nq) p.cand_cnt[(size_t)lane * n_seg + my_seg] = cnt_lo;
+      if (lane + 32 < p.nq) p.cand_cnt[(size_t)(lane + 32) * n_seg + my_seg] = cnt_hi;
+    }
+    __syncwarp();
+    if (lane == 0) atomicAdd(const_cast<int*>(epi_done), 1);
   }
 
   tc_fence_before();

@@ -81,6 +81,10 @@ def measure_retrieve_only(name: str, iters: int, seed: int = 0):
     line = {"config": name, "mode": "retrieve only", "queries_per_call": s.nq, "k": s.k, "facts_scanned": total,
             "retrieve_us": us, "retrieve_emb_gbs": workload.emb_bytes_scanned(s, total) / (us * 1e-6) / 1e9,
             "kernel_timeouts": store.stats()["kernel_timeouts"]}  # fmt: skip
+    st = store.stats()
+    if st["filter_list_queries"] + st["filter_list_fallbacks"]:
+        line["filter_list"] = {"queries": st["filter_list_queries"], "fallbacks": st["filter_list_fallbacks"],
+                               "rows_per_query": st["filter_list_rows"] / max(1, st["filter_list_queries"])}  # fmt: skip
     store.close()
     return line
 

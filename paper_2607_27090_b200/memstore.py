@@ -64,7 +64,7 @@ class _AnnParams(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_facts", "n_resident_facts", "kv_tokens_used", "retrieve_calls", "inject_calls", "kernels_launched",
-        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "n_removed_facts", "compose_cache_hits", "compose_cache_fills", "compose_cache_segments", "filter_fixup_overflows")]  # fmt: skip
+        "arena_bytes", "embedding_bytes", "host_kv_tokens_used", "kernel_timeouts", "filter_fixups", "n_removed_facts", "compose_cache_hits", "compose_cache_fills", "compose_cache_segments", "filter_fixup_overflows", "filter_list_queries", "filter_list_rows", "filter_list_fallbacks")]  # fmt: skip
 
 
 # every symbol include/memstore.h declares

@@ -122,6 +122,64 @@ def test_retrieve_many_queries_tensor_core_path(n, E, nq):
     ms.close()
 
 
+@pytest.mark.parametrize("n,E,nq", [(70_000, 256, 64), (40_000, 1024, 9), (45_001, 64, 33)])
+def test_tensor_core_filter_candidate_rows(n, E, nq):
+    """Segments long enough that every CTA of the filter kernel has several tiles: the kernel lists candidate rows per
+    query (thresholds from the shared histogram of group maxima, first tile parked in tensor memory) and the later steps
+    select and rescore those rows instead of sweeping the group maxima.  Results must be what every other path gives:
+    the oracle's ranking, and bit-identical scores to the CUDA-core kernels; k beyond what the list serves goes through
+    the group maxima; removed rows are never listed."""
+    hs = HostStore(31, n, 1, 1, 16, 1, 1, E, "float16")
+    hs.emb[n - 1] = hs.emb[17]  # duplicates: first tile of CTA 0, a middle tile, the ragged last tile
+    hs.emb[n // 2 + 3] = hs.emb[17]
+    ms = hs.to_memstore(1e4, batch=8192)
+    q = synth.queries(31, nq, E, "float16")
+    q[0] = hs.emb[17]
+    q[nq - 1] = hs.emb[n - 2]  # the best row of this query sits in the last tile
+    for k in (1, 10, 100, 227, 228):
+        before = ms.stats()
+        ids, sc = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        after = ms.stats()
+        ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+        assert after["kernel_timeouts"] == 0
+        served = after["filter_list_queries"] - before["filter_list_queries"]
+        fell_back = after["filter_list_fallbacks"] - before["filter_list_fallbacks"]
+        if k <= 227:
+            # every query is looked up in its list; on these inputs all lists are usable and short
+            assert served + fell_back == nq and fell_back == 0, (k, served, fell_back)
+            rows_listed = after["filter_list_rows"] - before["filter_list_rows"]
+            assert (k + 28) * nq <= rows_listed <= 3000 * nq, (k, rows_listed / nq)
+        else:
+            assert served == 0 and fell_back == 0  # k + 29 exceeds what the list's selection ranks: group maxima
+        if k >= 3:
+            assert ids[0, :3].tolist() == [17, n // 2 + 3, n - 1] and sc[0, 0] == sc[0, 1] == sc[0, 2]
+        assert ids[nq - 1, 0] == n - 2
+        for i in list(range(0, nq, 7)) + [nq - 1]:
+            check_ids(ids[i], sc[i], hs.emb, q[i], k)
+    ids_tc, sc_tc = ms.retrieve(to_dev(q), 50)
+    for i in (0, 1, nq - 1):
+        ids_1, sc_1 = ms.retrieve(to_dev(q[i : i + 1]), 50)
+        assert torch.equal(ids_1[0], ids_tc[i]) and torch.equal(sc_1[0], sc_tc[i])
+    # removal: the copies of row 17 go one by one, whole tiles go
+    removed = np.zeros(n, bool)
+    removed[[17, n - 1]] = True
+    removed[256:512] = True
+    removed[n - 300 : n - 2] = True
+    for f in np.flatnonzero(removed):
+        ms.remove_fact(int(f))
+    ids, sc = ms.retrieve(to_dev(q), 100)
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    assert ids[0, 0] == n // 2 + 3 and not np.isin(ids, np.flatnonzero(removed)).any()
+    for i in (0, 1, nq - 1):
+        check_ids(ids[i], sc[i], hs.emb, q[i], 100, removed=removed)
+    # twice the same call: identical (the lists' order depends on timing, the results do not)
+    ids2, sc2 = ms.retrieve(to_dev(q), 100)
+    assert np.array_equal(ids2.cpu().numpy(), ids) and np.array_equal(sc2.cpu().numpy(), sc)
+    assert ms.stats()["filter_list_fallbacks"] == 0
+    ms.close()
+
+
 @pytest.mark.parametrize("kind", ["exact_copies", "near_copies", "too_many_exact_copies"])
 def test_tensor_core_filter_with_more_tied_groups_than_its_margin(kind):
     """The filter keeps k + 28 groups.  400 rows that tie with (or sit within rounding of) the best score, spread over 400
