@@ -64,8 +64,7 @@ struct memstore {
   // candidate rows emitted by the filter kernel (see score_gemm.cuh)
   uint32_t* tc_hist = nullptr;      // [64][kHistWords] + thr_used[64] (zero between calls) + cand_cnt[64][kCandMaxSegs]
   unsigned long long* tc_emit = nullptr;  // [64][kTcCandPlaces]: candidate rows listed by the filter kernel
-  int32_t* tc_sel_rows = nullptr;   // [64][kTcMaxK]
-  int* tc_slow = nullptr;           // [64]: the query's candidate list was unusable, the group maxima serve it
+  float* tc_exact = nullptr;        // [64][kTcMaxK]: exact scores of the listed rows that were rescored, by filter rank
   unsigned long long* tc_list_stats = nullptr;  // queries served from their candidate list, rows listed for them, fallbacks
   bool tc_ready = false;
   int64_t scores_nq = 0;
@@ -229,7 +228,7 @@ constexpr int64_t kTcFewQueriesRows = 131072;  // ... unless the segment is long
 constexpr int kTcMaxK = 256;
 constexpr int kTcGroupMargin = 28;   // groups selected beyond k: slack for tensor-core vs CUDA-core rounding at the k-th score
 constexpr int kTcMaxK2 = kTcMaxK + kTcGroupMargin;
-constexpr int kTcCandPlaces = kTopkThreads * kCandKpl;  // candidate places per query over all CTAs of the filter kernel
+constexpr int kTcCandPlaces = 16384;  // candidate places per query over all epilogue warps of the filter kernel
 constexpr int kTcCandSeg = 24;                          // places per epilogue warp of the filter kernel and query
 constexpr int kTcMaxCtas = kCandMaxSegs / 4;
 constexpr int kTcRowMargin = 28;     // candidate rows rescored beyond k
@@ -280,10 +279,8 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_error, 2 * sizeof(int)));
   MS_CUDA(s, cudaMalloc(&s->tc_hist, kTcHistWords * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_emit, (size_t)kGemmMaxQ * kTcCandPlaces * sizeof(unsigned long long)));
-  MS_CUDA(s, cudaMalloc(&s->tc_sel_rows, (size_t)kGemmMaxQ * kTcMaxK * sizeof(int32_t)));
-  MS_CUDA(s, cudaMalloc(&s->tc_slow, (size_t)kGemmMaxQ * sizeof(int)));
+  MS_CUDA(s, cudaMalloc(&s->tc_exact, (size_t)kGemmMaxQ * kTcMaxK * sizeof(float)));
   MS_CUDA(s, cudaMemset(s->tc_hist, 0, kTcHistWords * sizeof(uint32_t)));
-  MS_CUDA(s, cudaMemset(s->tc_slow, 0, (size_t)kGemmMaxQ * sizeof(int)));
   MS_CUDA(s, cudaMalloc(&s->tc_list_stats, 3 * sizeof(unsigned long long)));
   MS_CUDA(s, cudaMemset(s->tc_list_stats, 0, 3 * sizeof(unsigned long long)));
   MS_CUDA(s, cudaMemset(s->tc_tickets, 0, (size_t)kGemmMaxQ * sizeof(uint32_t)));
@@ -295,7 +292,7 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaFuncSetAttribute(tc_fixup_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kFixupCap * sizeof(unsigned long long))));
   MS_CUDA(s, cudaFuncSetAttribute(score_gemm_groupmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes));
   const size_t rs = (size_t)kTcMaxK2 * 8 * sizeof(uint32_t);
-  MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
+  MS_CUDA(s, cudaFuncSetAttribute(rescore_topk_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs));
   s->tc_ready = true;
   return MS_OK;
 }
@@ -333,31 +330,30 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes,
                   s->test_spin_limit, s->test_mute_producers, s->removed_bits_d,
                   emit ? hist : nullptr, cand_cnt, thr_used, s->tc_emit, seg, k2r};
-    score_gemm_groupmax_kernel<<<n_ctas, kGemmThreads, kGemmSmemBytes, st>>>(tmap_emb, tmap_q, gp);
-    MS_CUDA(s, cudaGetLastError());
+    MS_CUDA(s, launch_dependent(score_gemm_groupmax_kernel, dim3((unsigned)n_ctas), dim3(kGemmThreads), kGemmSmemBytes, st, tmap_emb, tmap_q, gp));
     RetrieveParams p = base;
     p.queries = qptr;
     p.nq = nqb;
     p.out_ids = base.out_ids + (int64_t)q0 * base.k;
     p.out_scores = base.out_scores ? base.out_scores + (int64_t)q0 * base.k : nullptr;
     float* scores_out = p.out_scores ? p.out_scores : s->tc_scores_out;
-    const int* slow = emit ? s->tc_slow : nullptr;
     if (emit) {
-      MS_CUDA(s, launch_dependent(select_rows_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const unsigned long long*)s->tc_emit,
-                                  n_seg, seg, (const uint32_t*)cand_cnt, thr_used, hist, kHistWords,
-                                  k2r, s->tc_sel_rows, s->tc_next_best, s->tc_slow, s->tc_list_stats));
-      dim3 rgrid((unsigned)((k2r + kScoreWarps * 8 - 1) / (kScoreWarps * 8)), (unsigned)nqb);
-      MS_CUDA(s, launch_dependent(rescore_topk_kernel<__half, 1>, rgrid, dim3(kScoreThreads), (size_t)k2r * sizeof(uint32_t), st, p,
-                                  (const int32_t*)s->tc_sel_rows, k2r, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets,
-                                  scores_out, (const float*)s->tc_next_best, s->tc_redo, s->tc_kth, slow, 0));
+      // one launch selects among the listed rows, rescores them and writes the top-k (a query whose list is unusable is
+      // served from the group maxima by one CTA of the same launch)
+      MS_CUDA(s, launch_dependent(list_topk_kernel<__half>, dim3(kListCtas, (unsigned)nqb), dim3(kListThreads), (size_t)k2 * 8 * sizeof(uint32_t),
+                                  st, p, (const unsigned long long*)s->tc_emit, n_seg, seg, (const uint32_t*)cand_cnt, thr_used, hist, kHistWords,
+                                  k2r, s->tc_exact, s->tc_tickets, scores_out, s->tc_redo, s->tc_kth, s->tc_list_stats, (const float*)s->tc_gmax,
+                                  s->tc_gmax_stride, n_groups, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows));
+      s->kernels_launched += 1;
+    } else {
+      MS_CUDA(s, launch_dependent(select_groups_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const float*)s->tc_gmax,
+                                  s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best));
+      dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
+      MS_CUDA(s, launch_dependent(rescore_topk_kernel<__half>, grid, dim3(kScoreThreads), (size_t)k2 * 8 * sizeof(uint32_t), st, p,
+                                  (const int32_t*)s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets, scores_out,
+                                  (const float*)s->tc_next_best, s->tc_redo, s->tc_kth));
       s->kernels_launched += 2;
     }
-    MS_CUDA(s, launch_dependent(select_groups_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const float*)s->tc_gmax,
-                                s->tc_gmax_stride, n_groups, k2, s->tc_sel, s->tc_next_best, slow));
-    dim3 grid((unsigned)((k2 + kScoreWarps - 1) / kScoreWarps), (unsigned)nqb);
-    MS_CUDA(s, launch_dependent(rescore_topk_kernel<__half, 8>, grid, dim3(kScoreThreads), (size_t)k2 * 8 * sizeof(uint32_t), st, p,
-                                (const int32_t*)s->tc_sel, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, s->tc_tickets, scores_out,
-                                (const float*)s->tc_next_best, s->tc_redo, s->tc_kth, slow, 1));
     // the fix-up of the queries whose margin check failed (its CTAs leave at once for all the others, so the grid is
     // kept small: a few CTAs per query, each taking a slice of the segment)
     const int fix_ctas = std::max(1, std::min(8 * s->sm_count / nqb, (int)((n_rows + 2047) / 2048)));
@@ -366,7 +362,7 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     MS_CUDA(s, launch_dependent(tc_fixup_kernel<__half>, fgrid, dim3(kScoreThreads), kFixupCap * sizeof(unsigned long long), st, p,
                                 (int)n_rows, fix_rows, s->tc_redo, (const float*)s->tc_kth, s->tc_fix_counts, s->tc_fix_keys,
                                 s->tc_fix_tickets, scores_out, s->tc_error + 1, s->tc_n_fixups));
-    s->kernels_launched += 4;
+    s->kernels_launched += 2;
   }
   return MS_OK;
 }
@@ -666,8 +662,7 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_error);
     cudaFree(s->tc_hist);
     cudaFree(s->tc_emit);
-    cudaFree(s->tc_sel_rows);
-    cudaFree(s->tc_slow);
+    cudaFree(s->tc_exact);
     cudaFree(s->tc_list_stats);
     cudaFree(s->tiles);
     cudaFree(s->cc_slots);

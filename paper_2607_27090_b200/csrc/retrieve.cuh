@@ -171,6 +171,50 @@ __device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, c
   s1 = a1;
 }
 
+// Two fp16 rows at once against a query held in shared memory as fp32 (the values of the fp16 query, exactly): the
+// same products in the same order as score_two_rows, with 16 registers fewer (for kernels of 1024 threads).
+__device__ __forceinline__ void score_two_rows_sq(const float* s_q, int E, const __half* seg, int64_t row0, int64_t row1, float& s0, float& s1) {
+  const int lane = threadIdx.x & 31;
+  const uint4* r0 = reinterpret_cast<const uint4*>(seg + row0 * E);
+  const uint4* r1 = reinterpret_cast<const uint4*>(seg + row1 * E);
+  const int nvec = E / 8;
+  float a0 = 0.f, a1 = 0.f;
+  for (int v0 = 0; v0 < nvec; v0 += 128) {
+    uint4 x[4], z[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        x[u] = __ldg(r0 + v);
+        z[u] = __ldg(r1 + v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * 32 + lane;
+      if (v < nvec) {
+        float f[8], h[8];
+        unpack8(x[u], f);
+        unpack8(z[u], h);
+        const float4 g0 = *reinterpret_cast<const float4*>(s_q + 8 * v), g1 = *reinterpret_cast<const float4*>(s_q + 8 * v + 4);
+        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          a0 = fmaf(f[i], g[i], a0);
+          a1 = fmaf(h[i], g[i], a1);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+  }
+  s0 = a0;
+  s1 = a1;
+}
+
 // The same scoring with the query read straight from global memory (through L1) next to the row, so that one
 // memory round trip serves both and no shared-memory staging or barrier is needed.  Same lane layout and
 // summation order as score_rows.
@@ -1104,17 +1148,14 @@ __global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const Retrieve
 
 // Step 2: per query, the k2 groups with the largest group maximum, written in ASCENDING group order (so that the
 // candidate rows of step 3 are in row order and "lower index first" among equal scores means "lower fact id first").
-// `only` (or nullptr): the queries to serve are those with only[q] != 0 - the ones whose candidate list from the
-// filter kernel was unusable; the others are served by select_rows_kernel.
 __global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const float* gmax, int64_t gmax_stride, int n_groups, int k2,
-                                                                    int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/, const int* only) {
+                                                                    int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/) {
   __shared__ TopkShared sm;
   __shared__ int32_t s_sel[512];
   __shared__ float s_val[512];
   grid_dependency_wait();  // every kernel of this chain is a programmatic dependent of the one before it
   grid_launch_dependents();
   const int q = blockIdx.x;
-  if (only != nullptr && !only[q]) return;
   int32_t* out = sel + (int64_t)q * k2;
   // one group more than asked for: its maximum is the best score the filter saw among the rows that will NOT be
   // rescored, which the rescoring step compares with the k-th exact score it finds
@@ -1131,85 +1172,6 @@ __global__ void __launch_bounds__(kTopkThreads, 1) select_groups_kernel(const fl
       rank += (other < mine) || (other == mine && j < i);
     }
     out[rank] = (int32_t)mine;
-  }
-}
-
-// Step 2 when the filter kernel emitted candidate rows (see score_gemm.cuh): per query, the k2 candidates with the best
-// filter scores, written in ascending row order, and the best filter score among all the rows that will not be
-// rescored: the (k2+1)-th candidate's, or the highest threshold the filter applied (every row it did not emit scored
-// below that), whichever is larger.  The candidates of a query sit in one segment of `seg` places per epilogue warp of the
-// filter kernel, cand_cnt[q][segment] of them used.  Fewer than k2 candidates in all, a warp that found more than its
-// segment holds, or more candidates tied at the cut than the selection ranks, sets slow[q]: select_groups_kernel then
-// serves the query from the group maxima.  The CTA also leaves the query's histogram and threshold record zeroed for
-// the next call.
-constexpr int kCandKpl = 16;       // places of one query over all segments <= kTopkThreads * kCandKpl
-constexpr int kCandMaxSegs = 1024;
-__global__ void __launch_bounds__(kTopkThreads, 1) select_rows_kernel(const unsigned long long* cand, int n_seg, int seg, const uint32_t* cand_cnt,
-                                                                  uint32_t* thr_used, uint32_t* hist, int hist_words, int k2,
-                                                                  int32_t* sel /*[nq][k2]*/, float* next_best /*[nq]*/, int* slow /*[nq]*/,
-                                                                  unsigned long long* list_stats /*served, rows listed, fallbacks*/) {
-  __shared__ ExtractShared es;
-  __shared__ unsigned long long s_cand[kTopkThreads];
-  __shared__ uint8_t s_used[kCandMaxSegs];  // per segment
-  __shared__ int32_t s_rows[kExtractMaxK];
-  __shared__ float s_next;
-  __shared__ uint32_t s_total;
-  grid_dependency_wait();
-  grid_launch_dependents();
-  const int q = blockIdx.x;
-  const uint32_t tk = thr_used[q];
-  if (threadIdx.x == 0) {
-    s_next = -INFINITY;
-    s_total = 0u;
-  }
-  __syncthreads();
-  int overrun = 0;
-  for (int i = threadIdx.x; i < n_seg && i < kCandMaxSegs; i += kTopkThreads) {
-    const uint32_t c = cand_cnt[(size_t)q * n_seg + i];
-    overrun |= c > (uint32_t)seg;
-    s_used[i] = (uint8_t)min(c, (uint32_t)seg);
-    if (c) atomicAdd(&s_total, min(c, (uint32_t)seg));
-  }
-  overrun = __syncthreads_or(overrun);
-  const uint32_t n = s_total;
-  {  // clean for the next call
-    uint4* hq = reinterpret_cast<uint4*>(hist + (size_t)q * hist_words);  // hist_words is a multiple of 4
-    for (int i = threadIdx.x; i < hist_words / 4; i += kTopkThreads) hq[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (threadIdx.x == 0) thr_used[q] = 0u;
-  }
-  const int n_places = n_seg * seg;
-  bool ok = !overrun && n >= (uint32_t)k2 && k2 + 1 <= kExtractMaxK && n_places <= kTopkThreads * kCandKpl && n_seg <= kCandMaxSegs && seg < 256;
-  int my_rank = -1;
-  unsigned long long my_key = 0ull;
-  const unsigned long long* mine = cand + (size_t)q * n_places;
-  if (ok)
-    ok = topk_extract_keys<kTopkThreads, kCandKpl>(
-        es, s_cand, [&](int i) { return (uint32_t)(i % seg) < (uint32_t)s_used[i / seg] ? (uint32_t)(__ldcg(mine + i) >> 32) : 0u; }, nullptr,
-        n_places, k2 + 1, my_rank, my_key);
-  if (threadIdx.x == 0) {
-    atomicAdd(list_stats + (ok ? 0 : 2), 1ull);
-    if (ok) atomicAdd(list_stats + 1, (unsigned long long)n);
-  }
-  if (!ok) {
-    if (threadIdx.x == 0) slow[q] = 1;
-    return;
-  }
-  if (my_rank >= 0) {
-    if (my_rank < k2) s_rows[my_rank] = (int32_t)(uint32_t)__ldcg(mine + (0xffffffffu - (uint32_t)my_key));
-    else s_next = key_score((uint32_t)(my_key >> 32));
-  }
-  __syncwarp();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    slow[q] = 0;
-    next_best[q] = fmaxf(s_next, tk ? key_score(tk) : -INFINITY);
-  }
-  // ascending row order by counting (the rows are distinct)
-  if (threadIdx.x < k2) {
-    const int32_t mine_row = s_rows[threadIdx.x];
-    int rank = 0;
-    for (int j = 0; j < k2; ++j) rank += s_rows[j] < mine_row;
-    sel[(size_t)q * k2 + rank] = mine_row;
   }
 }
 
@@ -1257,73 +1219,102 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
   return acc;
 }
 
-// Step 3: rescore the rows of the selected groups exactly (fp32 CUDA-core sums, the same arithmetic as the other
-// retrieve kernels) and take the top-k of these candidates.  grid = (candidate groups of 8 rows per warp..., nq);
-// candidate c of query q is row sel[q][c / 8] * 8 + c % 8.  The last CTA of a query (wait-free ticket) selects.
-// Dynamic shared memory: n_cand uint32 keys.
-// The margin check: `scores_out` ([nq][k], never NULL) receives the exact scores by rank; when the k-th of them does not
-// beat next_best[q] (the filter's best score among the rows that were not rescored) by more than the filter's rounding,
-// a row outside the selected groups may belong to the top-k: redo[q] is raised and kth[q] tells the fix-up kernel which
-// exact score a row must reach.
 constexpr float kTcFilterRounding = 1e-5f;  // tensor-core fp32 accumulation against the fixed-order CUDA-core sum, times max(1, |score|)
-// GROUP = 8: sel holds groups (candidate c of query q is row sel[q][c / 8] * 8 + c % 8); GROUP = 1: sel holds rows
-// (candidate c is row sel[q][c]; n_sel a multiple of 2 or its last candidate is scored alone).  slow / want_slow:
-// when slow != nullptr the kernel serves the queries with (slow[q] != 0) == want_slow and leaves the others alone.
-template <typename T, int GROUP>
+// The exact scores of the rows of the chosen groups: candidate c of the query is row sel[c / 8] * 8 + c % 8 (sel: the
+// query's k2 groups in ascending order, -1 padded).  The calling warp takes the groups first, first + step, ...; two rows
+// in flight at a time.  cs / cr: the query's candidate scores and rows ([k2 * 8], cr = -1 for an absent row).
+template <typename T>
+__device__ __forceinline__ void rescore_groups(const RetrieveParams& p, int q, const int32_t* sel, int k2, int n_rows, float* cs, int32_t* cr,
+                                               int first, int step) {
+  const int lane = threadIdx.x & 31;
+  const T* seg = reinterpret_cast<const T*>(p.emb);  // user 0
+  for (int g_idx = first; g_idx < k2; g_idx += step) {
+    const int32_t g = sel[g_idx];
+    for (int r = 0; r < 8; r += 2) {
+      const int64_t row = (int64_t)g * 8 + r;
+      const bool ok0 = g >= 0 && row < n_rows, ok1 = g >= 0 && row + 1 < n_rows;
+      float s0 = -INFINITY, s1 = -INFINITY;
+      if (ok1) {
+        score_two_rows<T>(p, q, seg, row, row + 1, s0, s1);
+        s0 += 0.0f;
+        s1 += 0.0f;
+      } else if (ok0) {
+        s0 = score_one_row<T>(p, q, seg, row) + 0.0f;
+      }
+      // a removed row stays a candidate (the valid candidates must remain a prefix) with the score of a removed row
+      if (ok0 && row_removed(p, 0, row)) s0 = -INFINITY;
+      if (ok1 && row_removed(p, 0, row + 1)) s1 = -INFINITY;
+      if (lane == 0) {
+        cs[g_idx * 8 + r] = s0;
+        cr[g_idx * 8 + r] = ok0 ? (int32_t)row : -1;
+        cs[g_idx * 8 + r + 1] = s1;
+        cr[g_idx * 8 + r + 1] = ok1 ? (int32_t)(row + 1) : -1;
+      }
+    }
+  }
+}
+
+// The top-k of a query's rescored candidates (all THREADS threads of the CTA call, after the candidates have been
+// written and made visible), and the margin check: when the k-th exact score does not beat `best_unscored` (the
+// filter's best score among the rows that were not rescored) by more than the filter's rounding, a row outside the
+// selected groups may belong to the top-k: redo[q] is raised and kth[q] tells the fix-up kernel which exact score a row
+// must reach.  s_keys: shared memory for n_cand keys.
+template <int THREADS>
+__device__ __forceinline__ void rescore_select(const RetrieveParams& p, int q, TopkShared& sm, uint32_t* s_keys, const float* cs,
+                                               const int32_t* cr, int n_cand, float* scores_out, float best_unscored, int* redo, float* kth) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // Candidates are in ascending row order with every absent one (padding group, row beyond the segment) at the
+  // end, so the valid candidates are a prefix: count them and select among those only.
+  int mine = 0;
+  for (int i = threadIdx.x; i < n_cand; i += THREADS) mine += __ldcg(cr + i) >= 0;
+  mine = __reduce_add_sync(0xffffffffu, mine);
+  if (lane == 0) sm.warp_cnt[warp] = (uint32_t)mine;
+  __syncthreads();
+  int n_valid = 0;
+  for (int w = 0; w < THREADS / 32; ++w) n_valid += (int)sm.warp_cnt[w];
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for (int i = threadIdx.x; i < n_valid; i += THREADS) {
+    const uint32_t kx = order_key(__ldcg(cs + i));
+    s_keys[i] = kx;
+    if (kx != kRemovedKey) {
+      lo = min(lo, kx);
+      hi = max(hi, kx);
+    }
+  }
+  __syncthreads();
+  topk_block<THREADS, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.return_rows ? nullptr : p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
+                             scores_out + (int64_t)q * p.k, true, lo, hi);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int again = 0;
+    float need = 0.f;
+    if (n_valid >= p.k) {
+      need = __ldcg(scores_out + (int64_t)q * p.k + p.k - 1);
+      again = best_unscored >= need - kTcFilterRounding * fmaxf(1.f, fabsf(need));
+    }
+    redo[q] = again;
+    kth[q] = need;
+  }
+}
+
+// Step 3: grid = (groups of the query / warps per CTA, nq); a warp rescores one chosen group, the last CTA of a query
+// (wait-free ticket) selects.  Dynamic shared memory: k2 * 8 uint32 keys.  `scores_out` ([nq][k], never NULL) receives
+// the exact scores by rank.
+template <typename T>
 __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const RetrieveParams p, const int32_t* sel, int k2, int n_rows,
                                                                      float* cand_scores, int32_t* cand_rows, uint32_t* tickets,
-                                                                     float* scores_out, const float* next_best, int* redo, float* kth,
-                                                                     const int* slow, int want_slow) {
+                                                                     float* scores_out, const float* next_best, int* redo, float* kth) {
   extern __shared__ uint32_t s_keys[];
   __shared__ TopkShared sm;
   __shared__ int s_last;
   grid_dependency_wait();
   grid_launch_dependents();
   const int q = blockIdx.y;
-  if (slow != nullptr && (slow[q] != 0) != (want_slow != 0)) return;
-  const int n_cand = k2 * GROUP;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const T* seg = reinterpret_cast<const T*>(p.emb);  // user 0
+  const int n_cand = k2 * 8;
   float* cs = cand_scores + (int64_t)q * n_cand;
   int32_t* cr = cand_rows + (int64_t)q * n_cand;
-  const int c0 = (blockIdx.x * kScoreWarps + warp) * 8;  // eight candidate rows per warp
-  if (c0 < n_cand) {
-    for (int r = 0; r < 8; r += 2) {  // two rows in flight at a time
-      int64_t row0 = -1, row1 = -1;
-      if (GROUP == 8) {
-        const int32_t g = sel[(int64_t)q * k2 + c0 / 8];
-        if (g >= 0) {
-          row0 = (int64_t)g * 8 + r;
-          row1 = row0 + 1;
-        }
-      } else {
-        if (c0 + r < n_cand) row0 = sel[(int64_t)q * k2 + c0 + r];
-        if (c0 + r + 1 < n_cand) row1 = sel[(int64_t)q * k2 + c0 + r + 1];
-      }
-      const bool ok0 = row0 >= 0 && row0 < n_rows, ok1 = row1 >= 0 && row1 < n_rows;
-      float s0 = -INFINITY, s1 = -INFINITY;
-      if (ok0 && ok1) {
-        score_two_rows<T>(p, q, seg, row0, row1, s0, s1);
-        s0 += 0.0f;
-        s1 += 0.0f;
-      } else if (ok0) {
-        s0 = score_one_row<T>(p, q, seg, row0) + 0.0f;
-      }
-      // a removed row stays a candidate (the valid candidates must remain a prefix) with the score of a removed row
-      if (ok0 && row_removed(p, 0, row0)) s0 = -INFINITY;
-      if (ok1 && row_removed(p, 0, row1)) s1 = -INFINITY;
-      if (lane == 0) {
-        if (c0 + r < n_cand) {
-          cs[c0 + r] = s0;
-          cr[c0 + r] = ok0 ? (int32_t)row0 : -1;
-        }
-        if (c0 + r + 1 < n_cand) {
-          cs[c0 + r + 1] = s1;
-          cr[c0 + r + 1] = ok1 ? (int32_t)row1 : -1;
-        }
-      }
-    }
-  }
+  rescore_groups<T>(p, q, sel + (int64_t)q * k2, k2, n_rows, cs, cr, (int)blockIdx.x * kScoreWarps + (int)(threadIdx.x >> 5),
+                    (int)gridDim.x * kScoreWarps);
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -1334,36 +1325,189 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // Candidates are in ascending row order with every absent one (padding group, row beyond the segment) at the
-  // end, so the valid candidates are a prefix: count them and select among those only.
-  int mine = 0;
-  for (int i = threadIdx.x; i < n_cand; i += kScoreThreads) mine += __ldcg(cr + i) >= 0;
-  mine = __reduce_add_sync(0xffffffffu, mine);
-  if (lane == 0) sm.warp_cnt[warp] = (uint32_t)mine;
+  rescore_select<kScoreThreads>(p, q, sm, s_keys, cs, cr, n_cand, scores_out, next_best[q], redo, kth);
+}
+
+// Steps 2 and 3 in one launch when the filter kernel listed candidate rows (see score_gemm.cuh); grid = (kListCtas, nq).
+// The candidates of a query sit in one segment of `seg` places per epilogue warp of the filter kernel, cand_cnt[q][segment]
+// of them used, each (order key of the filter score << 32) | row.  EVERY CTA of a query gathers the used places into a
+// dense list and takes the k2 candidates with the best filter scores (the same work in each: the list is a few hundred
+// entries and nothing has to be exchanged); then the CTAs share the exact rescoring of those rows - the CUDA-core
+// routine of the other kernels, a warp per two rows, so that the k2 scattered 2 KiB reads of a query come from several
+// SMs at once - and the CTA that finishes last (a wait-free ticket) ranks them by (exact score, lower row first) and
+// writes the top-k.  The margin check is that of rescore_topk_kernel; the best filter score among the rows that were
+// NOT rescored is the (k2+1)-th candidate's or the highest threshold the filter applied (every row it did not list
+// scored below that), whichever is larger.
+// Fewer than k2 candidates in all, a warp that found more than its segment holds, a list longer than kListMaxRows, or
+// more candidates tied at the cut than the selection ranks: the list is unusable and CTA 0 alone serves the query from
+// the group maxima (the bodies of select_groups_kernel and rescore_topk_kernel: slower, about 0.1 ms, and rare).  The
+// histogram and the threshold record of the query are left zeroed for the next call.  Dynamic shared memory: k2g * 8
+// uint32 keys.
+constexpr int kListThreads = 512;
+constexpr int kListCtas = 4;
+constexpr int kListMaxRows = 2048;
+constexpr int kCandMaxSegs = 1024;
+template <typename T>
+__global__ void __launch_bounds__(kListThreads, 1)
+    list_topk_kernel(const RetrieveParams p, const unsigned long long* cand, int n_seg, int seg, const uint32_t* cand_cnt, uint32_t* thr_used,
+                     uint32_t* hist, int hist_words, int k2, float* exact /*[nq][k2]*/, uint32_t* tickets, float* scores_out, int* redo,
+                     float* kth, unsigned long long* list_stats /*served, rows listed, fallbacks*/, const float* gmax, int64_t gmax_stride,
+                     int n_groups, int k2g, int n_rows, float* cand_scores /*[nq][k2g * 8]*/, int32_t* cand_rows) {
+  extern __shared__ uint32_t s_dyn[];
+  __shared__ ExtractShared es;
+  __shared__ TopkShared sm;  // (the group selection of an unusable list; its candidate array also serves the row selection)
+  __shared__ uint16_t s_list[kListMaxRows];  // the used places, segment by segment
+  __shared__ int32_t s_rows[512];            // the chosen rows by filter rank (or the chosen groups)
+  __shared__ float s_val[512];               // their exact scores (or the groups' maxima)
+  __shared__ unsigned long long s_key[kExtractMaxK];
+  __shared__ uint32_t s_wtot[kListThreads / 32];
+  __shared__ float s_next, s_kth;
+  __shared__ int s_last;
+  constexpr unsigned kFull = 0xffffffffu;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  const int q = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    s_next = -INFINITY;
+    s_kth = 0.f;
+  }
+  // ---- the used places of all segments, densely (block-wide exclusive scan of the segments' counts)
+  uint32_t n = 0;
+  int overrun = 0;
+  for (int c0 = 0; c0 < n_seg; c0 += kListThreads) {
+    const int i = c0 + tid;
+    uint32_t c = i < n_seg ? cand_cnt[(size_t)q * n_seg + i] : 0u;
+    overrun |= c > (uint32_t)seg;
+    c = min(c, (uint32_t)seg);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(kFull, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_wtot[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0, total = 0;
+    for (int w = 0; w < kListThreads / 32; ++w) {
+      const uint32_t t = s_wtot[w];
+      before += w < warp ? t : 0u;
+      total += t;
+    }
+    const uint32_t at = n + before + incl - c;
+    for (uint32_t j = 0; j < c; ++j)
+      if (at + j < (uint32_t)kListMaxRows) s_list[at + j] = (uint16_t)(i * seg + (int)j);
+    n += total;
+    __syncthreads();
+  }
+  overrun = __syncthreads_or(overrun);
+  if (blockIdx.x == 0) {  // clean for the next call (only this kernel's CTA 0 of the query touches the histogram)
+    uint4* hq = reinterpret_cast<uint4*>(hist + (size_t)q * hist_words);  // hist_words is a multiple of 4
+    for (int i = tid; i < hist_words / 4; i += kListThreads) hq[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  const int n_places = n_seg * seg;
+  bool ok = !overrun && n >= (uint32_t)k2 && n <= (uint32_t)kListMaxRows && k2 + 1 <= kExtractMaxK && n_places <= 65536 && k2 <= 2 * kListThreads / 4;
+  int my_rank = -1;
+  unsigned long long my_key = 0ull;
+  const unsigned long long* mine = cand + (size_t)q * n_places;
+  if (ok) {
+    auto key_at = [&](int i) { return (uint32_t)(__ldcg(mine + s_list[i]) >> 32); };
+    if (n <= (uint32_t)kListThreads) ok = topk_extract_keys<kListThreads, 1>(es, sm.cand, key_at, nullptr, (int)n, k2 + 1, my_rank, my_key);
+    else if (n <= 2u * kListThreads) ok = topk_extract_keys<kListThreads, 2>(es, sm.cand, key_at, nullptr, (int)n, k2 + 1, my_rank, my_key);
+    else ok = topk_extract_keys<kListThreads, 4>(es, sm.cand, key_at, nullptr, (int)n, k2 + 1, my_rank, my_key);
+  }
+  if (!ok) {
+    // ---- the list is unusable: CTA 0 serves the query from the group maxima
+    if (blockIdx.x != 0) return;
+    __syncthreads();
+    topk_block<kListThreads>(sm, gmax + (int64_t)q * gmax_stride, nullptr, n_groups, k2g + 1, IdMap{nullptr, nullptr}, s_rows, s_val);
+    __syncthreads();
+    const float best_unscored = n_groups > k2g ? s_val[k2g] : -INFINITY;
+    if (tid == 0) {
+      atomicAdd(list_stats + 2, 1ull);
+      thr_used[q] = 0u;
+    }
+    __syncthreads();
+    int32_t* groups = reinterpret_cast<int32_t*>(s_val);  // the chosen groups in ascending order (by counting, as select_groups_kernel)
+    for (int i = tid; i < k2g; i += kListThreads) {
+      const uint32_t me = (uint32_t)s_rows[i];
+      int rank = 0;
+      for (int j = 0; j < k2g; ++j) {
+        const uint32_t other = (uint32_t)s_rows[j];
+        rank += (other < me) || (other == me && j < i);
+      }
+      groups[rank] = (int32_t)me;
+    }
+    __syncthreads();
+    float* cs = cand_scores + (int64_t)q * k2g * 8;
+    int32_t* cr = cand_rows + (int64_t)q * k2g * 8;
+    rescore_groups<T>(p, q, groups, k2g, n_rows, cs, cr, warp, kListThreads / 32);
+    __syncthreads();
+    rescore_select<kListThreads>(p, q, sm, s_dyn, cs, cr, k2g * 8, scores_out, best_unscored, redo, kth);
+    return;
+  }
+  if (my_rank >= 0) {
+    if (my_rank < k2) s_rows[my_rank] = (int32_t)(uint32_t)__ldcg(mine + s_list[0xffffffffu - (uint32_t)my_key]);
+    else s_next = key_score((uint32_t)(my_key >> 32));
+  }
+  __syncwarp();
   __syncthreads();
-  int n_valid = 0;
-  for (int w = 0; w < kScoreThreads / 32; ++w) n_valid += (int)sm.warp_cnt[w];
-  uint32_t lo = 0xffffffffu, hi = 0u;
-  for (int i = threadIdx.x; i < n_valid; i += kScoreThreads) {
-    const uint32_t kx = order_key(__ldcg(cs + i));
-    s_keys[i] = kx;
-    if (kx != kRemovedKey) {
-      lo = min(lo, kx);
-      hi = max(hi, kx);
+  // ---- exact scores: this CTA takes the ranks blockIdx.x, blockIdx.x + kListCtas, ...; a warp two of them at a time
+  const T* seg_rows = reinterpret_cast<const T*>(p.emb);  // user 0
+  float* ex = exact + (int64_t)q * k2;
+  constexpr int kWarps = kListThreads / 32;
+  for (int j = warp; (int)blockIdx.x + kListCtas * j < k2; j += 2 * kWarps) {
+    const int ra = (int)blockIdx.x + kListCtas * j, rb = ra + kListCtas * kWarps;
+    float s0, s1 = 0.f;
+    if (rb < k2) score_two_rows<T>(p, q, seg_rows, (int64_t)s_rows[ra], (int64_t)s_rows[rb], s0, s1);
+    else s0 = score_one_row<T>(p, q, seg_rows, (int64_t)s_rows[ra]);
+    if (lane == 0) {
+      ex[ra] = s0 + 0.0f;
+      if (rb < k2) ex[rb] = s1 + 0.0f;
     }
   }
+  __syncwarp();
   __syncthreads();
-  topk_block<kScoreThreads, false>(sm, cs, s_keys, n_valid, p.k, IdMap{cr, p.return_rows ? nullptr : p.emb_fact_id}, p.out_ids + (int64_t)q * p.k,
-                            scores_out + (int64_t)q * p.k, true, lo, hi);
+  if (tid == 0) {
+    __threadfence();
+    const uint32_t t = atomicAdd(&tickets[q], 1u);
+    s_last = t == gridDim.x - 1;
+    if (s_last) tickets[q] = 0;
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int again = 0;
-    float need = 0.f;
-    if (n_valid >= p.k) {
-      need = __ldcg(scores_out + (int64_t)q * p.k + p.k - 1);
-      again = next_best[q] >= need - kTcFilterRounding * fmaxf(1.f, fabsf(need));
+  if (!s_last) return;
+  __threadfence();
+  if (tid < k2) {
+    const float sc = __ldcg(ex + tid);
+    s_val[tid] = sc;
+    s_key[tid] = ((unsigned long long)order_key(sc) << 32) | (0xffffffffu - (uint32_t)s_rows[tid]);
+  }
+  const uint32_t tk = thr_used[q];
+  __syncthreads();
+  // ---- rank by counting, two lanes per candidate (the rows are distinct, so the keys are)
+  {
+    const int ci = tid >> 1, part = tid & 1;
+    const unsigned long long me = ci < k2 ? s_key[ci] : 0ull;
+    uint32_t rank = 0;
+    if (ci < k2)
+      for (int j = part; j < k2; j += 2) rank += s_key[j] > me;
+    rank += __shfl_xor_sync(kFull, rank, 1);
+    if (ci < k2 && part == 0 && rank < (uint32_t)p.k) {
+      const int32_t row = s_rows[ci];
+      p.out_ids[(int64_t)q * p.k + rank] = (p.return_rows || p.emb_fact_id == nullptr) ? row : p.emb_fact_id[row];
+      scores_out[(int64_t)q * p.k + rank] = s_val[ci];
+      if (rank == (uint32_t)p.k - 1u) s_kth = s_val[ci];
     }
-    redo[q] = again;
+  }
+  __syncwarp();
+  __syncthreads();
+  if (tid == 0) {
+    const float need = s_kth;
+    const float nb = fmaxf(s_next, tk ? key_score(tk) : -INFINITY);
+    atomicAdd(list_stats, 1ull);
+    atomicAdd(list_stats + 1, (unsigned long long)n);
+    thr_used[q] = 0u;
+    redo[q] = nb >= need - kTcFilterRounding * fmaxf(1.f, fabsf(need));
     kth[q] = need;
   }
 }

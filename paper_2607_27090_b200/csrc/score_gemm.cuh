@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   const uint32_t limit = p.spin_limit ? p.spin_limit : kSpinLimit;
   const bool emitting = p.hist != nullptr;
   const int n_parked = emitting ? kGemmParked : 0;
+  grid_dependency_wait();    // launched as a programmatic dependent itself: the set-up above overlaps the end of the preceding kernel
   grid_launch_dependents();  // the kernels that follow are programmatic dependents: they are placed as SMs free up and wait for this grid
 
   if (warp == 0) {
