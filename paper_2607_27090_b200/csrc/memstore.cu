@@ -323,7 +323,7 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     const int n_ctas = std::min(n_tiles, s->sm_count);
     const int n_seg = n_ctas * 4;
     const int seg = std::min(kTcCandSeg, kTcCandPlaces / n_seg);
-    const bool emit = k2r + 1 <= kExtractMaxK && n_tiles >= 2 * s->sm_count && n_rows >= k2r && n_ctas <= kTcMaxCtas && seg >= 8;
+    const bool emit = k2r <= kListMaxK2 && n_tiles >= 2 * s->sm_count && n_rows >= k2r && n_ctas <= kTcMaxCtas && seg >= 8;
     uint32_t* hist = s->tc_hist;
     uint32_t* thr_used = hist + (size_t)kGemmMaxQ * kHistWords;
     uint32_t* cand_cnt = thr_used + kGemmMaxQ;
@@ -375,7 +375,9 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
   // enough CTAs to fill the GPU, at least one row per warp
   constexpr int64_t kWarps = THREADS / 32;
   // (a 1024-thread CTA fills an SM: more CTAs than SMs would only queue behind the first wave)
-  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * (THREADS >= 1024 ? 1 : 8) / nq);
+  // (256-thread CTAs are held to 64 registers so that four of them share an SM: as many CTAs as fit at once, so that the
+  // whole grid is one wave and nothing waits for an SM to be refilled)
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * (THREADS >= 1024 ? 1 : 4) / nq);
   int64_t rows = std::max<int64_t>(kWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
   rows = (rows + kWarps - 1) / kWarps * kWarps;
   const int rows_per_cta = (int)rows;

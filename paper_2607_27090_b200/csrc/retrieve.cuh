@@ -1125,7 +1125,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
 // keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
 // of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
 template <typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
+__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
                                                                          uint32_t* tickets, int keys_capacity, int n_host) {
   score_topk_body<T, THREADS, false>(p, rows_per_cta, tickets, keys_capacity, n_host, nullptr);
 }
@@ -1136,7 +1136,7 @@ __global__ void __launch_bounds__(THREADS) score_topk_fused_kernel(const Retriev
 // this library's copy kernel, they run on the SMs it vacates while it drains - and only the last CTA of a query waits,
 // right before it writes the ids and the plan.
 template <typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
+__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
                                                                         uint32_t* tickets, int keys_capacity, int n_host,
                                                                         const __grid_constant__ InjectParams ip, int early) {
   if (!early) grid_dependency_wait();  // launched as a programmatic dependent: nothing is touched before the preceding grid is done
@@ -1346,6 +1346,7 @@ __global__ void __launch_bounds__(kScoreThreads) rescore_topk_kernel(const Retri
 constexpr int kListThreads = 512;
 constexpr int kListCtas = 4;
 constexpr int kListMaxRows = 2048;
+constexpr int kListMaxK2 = 288;  // rows rescored per query: the largest k of the filter path (256) and the margin
 constexpr int kCandMaxSegs = 1024;
 template <typename T>
 __global__ void __launch_bounds__(kListThreads, 1)
@@ -1359,7 +1360,7 @@ __global__ void __launch_bounds__(kListThreads, 1)
   __shared__ uint16_t s_list[kListMaxRows];  // the used places, segment by segment
   __shared__ int32_t s_rows[512];            // the chosen rows by filter rank (or the chosen groups)
   __shared__ float s_val[512];               // their exact scores (or the groups' maxima)
-  __shared__ unsigned long long s_key[kExtractMaxK];
+  __shared__ unsigned long long s_key[kListMaxK2];
   __shared__ uint32_t s_wtot[kListThreads / 32];
   __shared__ float s_next, s_kth;
   __shared__ int s_last;
@@ -1406,7 +1407,7 @@ __global__ void __launch_bounds__(kListThreads, 1)
     for (int i = tid; i < hist_words / 4; i += kListThreads) hq[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   const int n_places = n_seg * seg;
-  bool ok = !overrun && n >= (uint32_t)k2 && n <= (uint32_t)kListMaxRows && k2 + 1 <= kExtractMaxK && n_places <= 65536 && k2 <= 2 * kListThreads / 4;
+  bool ok = !overrun && n >= (uint32_t)k2 && n <= (uint32_t)kListMaxRows && k2 <= kListMaxK2 && n_places <= 65536;
   int my_rank = -1;
   unsigned long long my_key = 0ull;
   const unsigned long long* mine = cand + (size_t)q * n_places;
@@ -1484,14 +1485,15 @@ __global__ void __launch_bounds__(kListThreads, 1)
   }
   const uint32_t tk = thr_used[q];
   __syncthreads();
-  // ---- rank by counting, two lanes per candidate (the rows are distinct, so the keys are)
+  // ---- rank by counting, two lanes per candidate when the threads allow (the rows are distinct, so the keys are)
   {
-    const int ci = tid >> 1, part = tid & 1;
+    const int per = 2 * k2 <= kListThreads ? 2 : 1;
+    const int ci = per == 2 ? tid >> 1 : tid, part = per == 2 ? tid & 1 : 0;
     const unsigned long long me = ci < k2 ? s_key[ci] : 0ull;
     uint32_t rank = 0;
     if (ci < k2)
-      for (int j = part; j < k2; j += 2) rank += s_key[j] > me;
-    rank += __shfl_xor_sync(kFull, rank, 1);
+      for (int j = part; j < k2; j += per) rank += s_key[j] > me;
+    if (per == 2) rank += __shfl_xor_sync(kFull, rank, 1);
     if (ci < k2 && part == 0 && rank < (uint32_t)p.k) {
       const int32_t row = s_rows[ci];
       p.out_ids[(int64_t)q * p.k + rank] = (p.return_rows || p.emb_fact_id == nullptr) ? row : p.emb_fact_id[row];
