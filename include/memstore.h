@@ -82,8 +82,10 @@ enum {
                              began (a serving loop whose next query is ready before the previous injection is enqueued).
                              The scoring and selection of this call may then overlap the tail of the preceding kernel -
                              typically the previous request's copy kernel, whose draining SMs they use; ids, plan and
-                             cache are still written strictly after it.  Without the flag the call orders itself after
-                             all preceding work, as any launch does.  Results are the same either way. */
+                             cache are still written strictly after it.  Without the flag - and for the first such
+                             call after the store itself was changed (facts added or removed, a new prefix) - the call
+                             orders itself after all preceding work, as any launch does.  Results are the same either
+                             way. */
 };
 /* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
  * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */

@@ -69,6 +69,7 @@ struct memstore {
   bool tc_ready = false;
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
+  bool store_changed = false;  // facts, prefix or removals enqueued since the last serving call: that call must order itself after them
   uint32_t tiles_capacity = 0;
   InjectCtrl* ctrl = nullptr;  // one control block, kept clean by the planning kernels themselves
   cudaEvent_t last_done = nullptr;
@@ -693,6 +694,7 @@ static ms_status add_facts_tier(memstore_t* s, int32_t user, int64_t n, const vo
   const memstore_config& c = s->cfg;
   if (user < 0 || user >= c.n_users) return fail(s, MS_ERR_INVALID_ARG, "user %d out of range", user);
   if (n < 0 || (n > 0 && (!embs || !n_tokens))) return fail(s, MS_ERR_INVALID_ARG, "null embeddings or lengths");
+  s->store_changed = true;
   if (n == 0) {
     if (out_first_id) *out_first_id = (int32_t)s->n_facts;
     return MS_OK;
@@ -791,6 +793,7 @@ ms_status memstore_set_prefix(memstore_t* s, const void* k_pre, const void* v, i
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (n_tokens < 0) return fail(s, MS_ERR_INVALID_ARG, "negative token count");
+  s->store_changed = true;
   if (n_tokens == 0) {
     s->prefix_len = 0;
     return MS_OK;
@@ -1192,6 +1195,7 @@ ms_status memstore_remove_fact(memstore_t* s, int32_t fact_id, ms_stream stream)
   std::lock_guard<std::recursive_mutex> lock(s->mu);
   const memstore_config& c = s->cfg;
   if (fact_id < 0 || fact_id >= s->n_facts) return fail(s, MS_ERR_INVALID_ARG, "fact id %d out of range (0..%lld)", fact_id, (long long)s->n_facts - 1);
+  s->store_changed = true;
   // the embedding row of the id: ids are dense in insertion order, each add call put a run of them into one segment
   size_t lo = 0, hi = s->id_runs.size();
   while (lo + 1 < hi) {
@@ -1543,7 +1547,8 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   if ((uintptr_t)queries & 15) return fail(s, MS_ERR_INVALID_ARG, "queries must be 16-byte aligned");
   // MS_INPUTS_STABLE only matters to the one-launch retrieval + planning kernel below; every other route orders itself
   // after the preceding work of the stream as an ordinary launch does
-  const int early = (flags & MS_INPUTS_STABLE) ? 1 : 0;
+  // (not right after the store itself was changed on the stream: the kernels read its tables)
+  const int early = ((flags & MS_INPUTS_STABLE) && !s->store_changed) ? 1 : 0;
   flags &= ~(uint32_t)MS_INPUTS_STABLE;
   if (flags & MS_RETRIEVE_ANN) {
     ms_status rc = memstore_retrieve_ann_users(s, queries, query_users, nq, k, nullptr, out_ids, out_scores, nullptr, stream);
@@ -1583,6 +1588,7 @@ ms_status memstore_retrieve_inject(memstore_t* s, const void* queries, const int
   s->retrieve_calls++;
   rc = launch_copy(s, ip, cache, tiles_needed, st);
   if (rc != MS_OK) return rc;
+  s->store_changed = false;  // this call's kernels waited for everything before them (the plan kernel always does before it ends)
   return mark_last(s, st);
 }
 

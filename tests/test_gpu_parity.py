@@ -725,6 +725,45 @@ def test_inputs_stable_flag_overlaps_requests_without_changing_results():
     ms.close()
 
 
+def test_inputs_stable_flag_after_a_change_of_the_store():
+    """The flag vouches for the caller's inputs, not for the store: a fact added, or removed, on the stream right before a
+    flagged request (no host synchronisation in between) must be seen by it - the first flagged call after a change of
+    the store orders itself like an ordinary launch."""
+    hs = HostStore(46, 600, 2, 2, 64, 4, 12, 128, "float16")
+    ms = MemStore(n_layers=hs.L, n_kv_heads=hs.H, head_dim=hs.D, emb_dim=128, emb_dtype=torch.float16, rope_theta=1e4,
+                  max_facts_per_user=700, max_kv_tokens=int(hs.lens.sum()) + 4000)  # fmt: skip
+    first, extra = 500, 100
+    t1 = int(hs.offs[first - 1] + hs.lens[first - 1])
+    ms.add_facts(to_dev(hs.emb[:first]), hs.lens[:first], to_dev(hs.k[:, :t1]), to_dev(hs.v[:, :t1]))
+    bs, k = 16, 8
+    q = synth.queries(47, 6, 128, "float16")
+    per_req = (k * int(hs.lens.max())) // bs + 2
+    tables = to_dev(synth.block_tables(48, per_req * 6, per_req, 6))
+    start = to_dev(np.zeros(1, np.int32))
+    cache = make_cache(hs, per_req * 6, bs)
+    ids = torch.empty((6, k), dtype=torch.int32, device=DEV)
+    flags = M.INJECT_REVERSE | M.INPUTS_STABLE
+    for i in range(3):  # warm: scratch sized, the flagged path in use
+        ms.retrieve_inject(to_dev(q[i : i + 1]), k, start, tables[i : i + 1], cache, out_ids=ids[i : i + 1], flags=flags)
+    # the new facts: the first of them is query 3 itself, so it must come out on top of request 3
+    emb2 = hs.emb[first : first + extra].copy()
+    emb2[0] = q[3]
+    t2 = int(hs.offs[first + extra - 1] + hs.lens[first + extra - 1])
+    ms.add_facts(to_dev(emb2), hs.lens[first : first + extra], to_dev(hs.k[:, t1:t2]), to_dev(hs.v[:, t1:t2]))
+    ms.retrieve_inject(to_dev(q[3:4]), k, start, tables[3:4], cache, out_ids=ids[3:4], flags=flags)
+    ms.remove_fact(first)
+    ms.retrieve_inject(to_dev(q[3:4]), k, start, tables[4:5], cache, out_ids=ids[4:5], flags=flags)
+    torch.cuda.synchronize()
+    emb_all = np.concatenate([hs.emb[:first], emb2])
+    assert int(ids[3, 0]) == first
+    check_ids(ids[3].cpu().numpy(), None, emb_all, q[3], k)
+    removed = np.zeros(first + extra, bool)
+    removed[first] = True
+    assert first not in ids[4].tolist()
+    check_ids(ids[4].cpu().numpy(), None, emb_all, q[3], k, removed=removed)
+    ms.close()
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_inject_with_instruction_prefix(path):
     """The stored instruction prefix leads the composed segment (pre-RoPE keys rotated at the positions it gets), in
