@@ -418,6 +418,14 @@ ms_status memstore_stats(memstore_t* store, memstore_stats_t* out);
  * (NULL, NULL) when timing whole calls.  The caller owns the events.
  */
 ms_status memstore_set_profile_events(memstore_t* store, void* before_copy, void* after_copy);
+/*
+ * Measurement aid, with the events above: while they are set, every memstore_inject launches its direct
+ * gather/rotate/scatter kernel n times in a row on the same plan (the writes are the same every time), as ordinary
+ * launches - each starts when the one before it has ended - between the two event records.  (after - before) / n is then
+ * the duration of one launch with the cost of the event records (a few microseconds: nothing of a kernel launch overlaps
+ * an event record) spread over n launches.  n = 1 restores one launch per call.  1 <= n <= 1024.
+ */
+ms_status memstore_set_profile_repeats(memstore_t* store, int32_t n);
 
 /*
  * The composition cache (appendix "Position independence and rotation fidelity", closing remark: the one-time

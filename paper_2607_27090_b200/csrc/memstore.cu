@@ -69,6 +69,7 @@ struct memstore {
   bool tc_ready = false;
   int64_t scores_nq = 0;
   TileDesc* tiles = nullptr;
+  int prof_repeats = 1;        // measurement aid: launches of the copy kernel per inject call while profile events are set
   bool store_changed = false;  // facts, prefix or removals enqueued since the last serving call: that call must order itself after them
   uint32_t tiles_capacity = 0;
   InjectCtrl* ctrl = nullptr;  // one control block, kept clean by the planning kernels themselves
@@ -1443,52 +1444,57 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
     MS_CUDA(s, cudaEventRecord(s->prof_before, st));
   }
   cudaError_t e = cudaSuccess;
-  if (use_tma) {
-    // bulk-async staged kernel: one persistent CTA per SM
-    int ts = kTileTokens;
-    while (ts > 1 && ts * row_bytes > kTmaAreaBytes) ts >>= 1;
-    const int v_rows = cache->head_stride == c.head_dim ? 1 : 0;
-    lc.gridDim = dim3((unsigned)s->sm_count);
-    lc.blockDim = dim3(kTmaThreads);
-    lc.dynamicSmemBytes = kTmaSmemBytes;
-    if (c.rope_style == MS_ROPE_HALF_SPLIT)
-      e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<0>, p, ts, v_rows);
-    else
-      e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<1>, p, ts, v_rows);
-  } else {
-    // direct kernel: one CTA per (tile, layer, row part).  The ids are on the device, so the host sizes the grid
-    // from the mean length of the resident facts (plus a ragged tile per request and 3 %); the kernel's
-    // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
-    const int units = c.n_kv_heads * (c.head_dim / 16);
-    const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used - s->prefix_tokens_total + s->host_tokens_used) / (double)s->n_resident : 0.0;
-    int64_t est_tiles_grid = (int64_t)((((double)p.k * mean_len + p.prefix_len) / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
-    est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
-    const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
-    if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
-    lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
-    lc.blockDim = dim3(kCopyThreads);
-    lc.dynamicSmemBytes = 0;
-    // 8-bit caches: a scale whose significand is all ones, or one so extreme that it or its reciprocal is not a normal
-    // number, takes the kernel variant that divides with the hardware routine (see div_by_scale)
-    auto awkward = [](float sc, float rc) {
-      uint32_t u;
-      memcpy(&u, &sc, 4);
-      return (u & 0x7fffffu) == 0x7fffffu || !std::isnormal(rc) || !std::isnormal(sc);
-    };
-    const int fp8 = cache->dtype != MS_CACHE_FP8_E4M3 ? 0 : (awkward(p.k_scale, p.k_recip) || awkward(p.v_scale, p.v_recip)) ? 2 : 1;
-    if (c.rope_style == MS_ROPE_HALF_SPLIT)
-      e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 0>, p)
-          : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 2>, p);
-    else
-      e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 0>, p)
-          : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 2>, p);
+  // (measurement aid: the direct kernel may be launched several times in a row on the same plan - its writes are the same
+  // every time - as ordinary launches, each after the one before it has ended)
+  const int repeats = (prof && !use_tma) ? std::max(1, s->prof_repeats) : 1;
+  for (int rep = 0; rep < repeats && e == cudaSuccess; ++rep) {
+    if (use_tma) {
+      // bulk-async staged kernel: one persistent CTA per SM
+      int ts = kTileTokens;
+      while (ts > 1 && ts * row_bytes > kTmaAreaBytes) ts >>= 1;
+      const int v_rows = cache->head_stride == c.head_dim ? 1 : 0;
+      lc.gridDim = dim3((unsigned)s->sm_count);
+      lc.blockDim = dim3(kTmaThreads);
+      lc.dynamicSmemBytes = kTmaSmemBytes;
+      if (c.rope_style == MS_ROPE_HALF_SPLIT)
+        e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<0>, p, ts, v_rows);
+      else
+        e = cudaLaunchKernelEx(&lc, inject_copy_tma_kernel<1>, p, ts, v_rows);
+    } else {
+      // direct kernel: one CTA per (tile, layer, row part).  The ids are on the device, so the host sizes the grid
+      // from the mean length of the resident facts (plus a ragged tile per request and 3 %); the kernel's
+      // grid-stride loop makes any grid correct, and the worst case (every fact of maximal length) bounds it.
+      const int units = c.n_kv_heads * (c.head_dim / 16);
+      const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used - s->prefix_tokens_total + s->host_tokens_used) / (double)s->n_resident : 0.0;
+      int64_t est_tiles_grid = (int64_t)((((double)p.k * mean_len + p.prefix_len) / kTileTokens + 2.0) * p.nreq * 1.03) + 1;
+      est_tiles_grid = std::min(est_tiles_grid, tiles_needed);
+      const int64_t items = std::max<int64_t>(1, est_tiles_grid) * c.n_layers;
+      if (items > 0x7fffffff) return fail(s, MS_ERR_UNSUPPORTED, "request batch too large");
+      lc.gridDim = dim3((unsigned)items, (unsigned)((units + kUnitsPerPart - 1) / kUnitsPerPart));
+      lc.blockDim = dim3(kCopyThreads);
+      lc.dynamicSmemBytes = 0;
+      // 8-bit caches: a scale whose significand is all ones, or one so extreme that it or its reciprocal is not a normal
+      // number, takes the kernel variant that divides with the hardware routine (see div_by_scale)
+      auto awkward = [](float sc, float rc) {
+        uint32_t u;
+        memcpy(&u, &sc, 4);
+        return (u & 0x7fffffu) == 0x7fffffu || !std::isnormal(rc) || !std::isnormal(sc);
+      };
+      const int fp8 = cache->dtype != MS_CACHE_FP8_E4M3 ? 0 : (awkward(p.k_scale, p.k_recip) || awkward(p.v_scale, p.v_recip)) ? 2 : 1;
+      if (c.rope_style == MS_ROPE_HALF_SPLIT)
+        e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 0>, p)
+            : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<0, 2>, p);
+      else
+        e = fp8 == 0 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 0>, p)
+            : fp8 == 1 ? cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 1>, p) : cudaLaunchKernelEx(&lc, inject_copy_kernel<1, 2>, p);
+    }
   }
   if (e != cudaSuccess) {
     // (the planning kernel has left the control block clean: nothing to undo)
     return fail(s, MS_ERR_CUDA, "copy kernel launch: %s", cudaGetErrorString(e));
   }
   if (prof) MS_CUDA(s, cudaEventRecord(s->prof_after, st));
-  s->kernels_launched++;
+  s->kernels_launched += repeats;
   s->inject_calls++;
   return MS_OK;
 }
@@ -1767,6 +1773,14 @@ ms_status memstore_test_hooks(memstore_t* s, uint32_t wait_poll_limit, int32_t m
     DeviceGuard g(s->cfg.device);
     MS_CUDA(s, cudaMemset(s->tc_error, 0, sizeof(int)));
   }
+  return MS_OK;
+}
+
+ms_status memstore_set_profile_repeats(memstore_t* s, int32_t n) {
+  if (!s) return MS_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> lock(s->mu);
+  if (n < 1 || n > 1024) return fail(s, MS_ERR_INVALID_ARG, "repeats %d out of range (1..1024)", n);
+  s->prof_repeats = n;
   return MS_OK;
 }
 

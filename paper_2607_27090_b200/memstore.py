@@ -71,7 +71,7 @@ class _Stats(C.Structure):
 EXPORTS = (
     "memstore_version", "memstore_arena_bytes", "memstore_create", "memstore_destroy", "memstore_add_fact",
     "memstore_add_facts", "memstore_retrieve", "memstore_inject", "memstore_stats", "memstore_last_error",
-    "memstore_set_profile_events", "memstore_retrieve_static", "memstore_serve_host",
+    "memstore_set_profile_events", "memstore_set_profile_repeats", "memstore_retrieve_static", "memstore_serve_host",
     "memstore_retrieve_inject", "memstore_add_facts_host", "memstore_set_prefix", "memstore_rope_table_llama3",
     "memstore_build_graph", "memstore_set_graph", "memstore_get_graph", "memstore_retrieve_ann", "memstore_graph_append",
     "memstore_test_hooks", "memstore_reserve", "memstore_compose_cache", "memstore_remove_fact", "memstore_set_graph_user",
@@ -149,6 +149,8 @@ def load_library() -> C.CDLL:
     L.memstore_stats.argtypes = [vp, C.POINTER(_Stats)]
     L.memstore_set_profile_events.restype = i32
     L.memstore_set_profile_events.argtypes = [vp, vp, vp]
+    L.memstore_set_profile_repeats.restype = i32
+    L.memstore_set_profile_repeats.argtypes = [vp, i32]
     L.memstore_last_error.restype = C.c_char_p
     L.memstore_last_error.argtypes = [vp]
     _lib = L
@@ -510,6 +512,10 @@ class MemStore:
             return
         self._prof = (before_copy, after_copy)
         self._check(self._lib.memstore_set_profile_events(self._h, C.c_void_p(before_copy.cuda_event), C.c_void_p(after_copy.cuda_event)))
+
+    def set_profile_repeats(self, n: int):
+        """Measurement aid: launches of the copy kernel per inject call while profile events are set (see the header)."""
+        self._check(self._lib.memstore_set_profile_repeats(self._h, int(n)))
 
     def stats(self) -> dict:
         st = _Stats()
