@@ -122,7 +122,7 @@ def test_retrieve_many_queries_tensor_core_path(n, E, nq):
     ms.close()
 
 
-@pytest.mark.parametrize("n,E,nq", [(70_000, 256, 64), (40_000, 1024, 9), (45_001, 64, 33)])
+@pytest.mark.parametrize("n,E,nq", [(70_000, 256, 64), (40_000, 1024, 9), (45_001, 64, 33), (38_000, 512, 17)])
 def test_tensor_core_filter_candidate_rows(n, E, nq):
     """Segments long enough that every CTA of the filter kernel has several tiles: the kernel lists candidate rows per
     query (thresholds from the shared histogram of group maxima, first tile parked in tensor memory) and the later steps
@@ -318,30 +318,31 @@ def test_bounded_waits_report_a_time_out_and_the_store_stays_usable():
     ms.test_hooks()
     run_inject_and_check(ms, hs, [3, 1, 7], 5, table, make_cache(hs, 32, 16), 1e4)
     ms.close()
-    # (2) the tensor-core scoring kernel
-    n_rows, E, nq, k = 9000, 128, 8, 10
-    emb = synth.embeddings(53, n_rows, E, "float16")
-    q = synth.queries(53, nq, E, "float16")
-    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float16, rope_theta=1e4,
-                  max_facts_per_user=n_rows, max_kv_tokens=0)  # fmt: skip
-    ms.add_facts(to_dev(emb), np.zeros(n_rows, np.int32))
-    ids, _ = ms.retrieve(to_dev(q), k)  # a normal call first: sizes the scratch
-    torch.cuda.synchronize()
-    assert ms.stats()["kernel_timeouts"] == 0
-    ms.test_hooks(wait_poll_limit=4000, mute_producers=True)
-    bad_ids, _ = ms.retrieve(to_dev(q), k)
-    torch.cuda.synchronize()
-    assert ms.stats()["kernel_timeouts"] == 1
-    bad = bad_ids.cpu().numpy()
-    assert np.all((bad >= -1) & (bad < n_rows))  # unspecified, but ids of this store or padding
-    ms.test_hooks()
-    assert ms.stats()["kernel_timeouts"] == 0
-    ids2, sc2 = ms.retrieve(to_dev(q), k)
-    torch.cuda.synchronize()
-    assert torch.equal(ids, ids2)
-    for i in range(nq):
-        check_ids(ids2[i].cpu().numpy(), sc2[i].cpu().numpy(), emb, q[i], k)
-    ms.close()
+    # (2) the tensor-core scoring kernel: a segment it only filters, and one long enough that it lists candidate rows
+    # (more roles wait there: the threshold warp, the parked first tiles)
+    for n_rows, E, nq, k in ((9000, 128, 8, 10), (40_000, 128, 12, 10)):
+        emb = synth.embeddings(53, n_rows, E, "float16")
+        q = synth.queries(53, nq, E, "float16")
+        ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float16, rope_theta=1e4,
+                      max_facts_per_user=n_rows, max_kv_tokens=0)  # fmt: skip
+        ms.add_facts(to_dev(emb), np.zeros(n_rows, np.int32))
+        ids, _ = ms.retrieve(to_dev(q), k)  # a normal call first: sizes the scratch
+        torch.cuda.synchronize()
+        assert ms.stats()["kernel_timeouts"] == 0
+        ms.test_hooks(wait_poll_limit=4000, mute_producers=True)
+        bad_ids, _ = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        assert ms.stats()["kernel_timeouts"] == 1
+        bad = bad_ids.cpu().numpy()
+        assert np.all((bad >= -1) & (bad < n_rows))  # unspecified, but ids of this store or padding
+        ms.test_hooks()
+        assert ms.stats()["kernel_timeouts"] == 0
+        ids2, sc2 = ms.retrieve(to_dev(q), k)
+        torch.cuda.synchronize()
+        assert torch.equal(ids, ids2)
+        for i in range(nq):
+            check_ids(ids2[i].cpu().numpy(), sc2[i].cpu().numpy(), emb, q[i], k)
+        ms.close()
 
 
 @pytest.mark.parametrize("case", ["plain", "too_many_candidates", "biased_sample"])
