@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(kAnnThreads, 1) ann_search_kernel(const AnnPar
     if (tid < p.n_entry) visit((int32_t)(((unsigned long long)(tid + 1) * 2654435761ull) % (unsigned long long)n));
   }
   for (;;) {
-    cluster.sync();  // rank 0's candidate list (or its verdict that the search is over) is complete
+    cluster.sync();  // rank 0's candidate list (or its decision that the search is over) is complete
     if (m->done) break;
     // ---- every CTA: score its share of the candidates into rank 0's merge array ----
     {
