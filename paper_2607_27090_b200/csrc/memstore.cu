@@ -64,7 +64,7 @@ struct memstore {
   // candidate rows emitted by the filter kernel (see score_gemm.cuh)
   uint32_t* tc_hist = nullptr;      // [64][kHistWords] + thr_used[64] (zero between calls) + cand_cnt[64][kCandMaxSegs]
   unsigned long long* tc_emit = nullptr;  // [64][kTcCandPlaces]: candidate rows listed by the filter kernel
-  float* tc_exact = nullptr;        // [64][kTcMaxK]: exact scores of the listed rows that were rescored, by filter rank
+  float* tc_exact = nullptr;        // [64][kListMaxK2]: exact scores of the listed rows that were rescored, by filter rank
   unsigned long long* tc_list_stats = nullptr;  // queries served from their candidate list, rows listed for them, fallbacks
   bool tc_ready = false;
   int64_t scores_nq = 0;
@@ -234,6 +234,7 @@ constexpr int kTcCandPlaces = 16384;  // candidate places per query over all epi
 constexpr int kTcCandSeg = 24;                          // places per epilogue warp of the filter kernel and query
 constexpr int kTcMaxCtas = kCandMaxSegs / 4;
 constexpr int kTcRowMargin = 28;     // candidate rows rescored beyond k
+static_assert(kTcMaxK + kTcRowMargin <= kListMaxK2, "the list kernel's per-query arrays hold k + margin rows");
 constexpr size_t kTcHistWords = (size_t)kGemmMaxQ * (kHistWords + 1 + kCandMaxSegs);
 
 // Launch as a programmatic dependent of the kernel before it in the stream (the kernel calls griddepcontrol.wait before
@@ -281,7 +282,7 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_error, 2 * sizeof(int)));
   MS_CUDA(s, cudaMalloc(&s->tc_hist, kTcHistWords * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_emit, (size_t)kGemmMaxQ * kTcCandPlaces * sizeof(unsigned long long)));
-  MS_CUDA(s, cudaMalloc(&s->tc_exact, (size_t)kGemmMaxQ * kTcMaxK * sizeof(float)));
+  MS_CUDA(s, cudaMalloc(&s->tc_exact, (size_t)kGemmMaxQ * kListMaxK2 * sizeof(float)));
   MS_CUDA(s, cudaMemset(s->tc_hist, 0, kTcHistWords * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_list_stats, 3 * sizeof(unsigned long long)));
   MS_CUDA(s, cudaMemset(s->tc_list_stats, 0, 3 * sizeof(unsigned long long)));

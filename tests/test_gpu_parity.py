@@ -122,7 +122,7 @@ def test_retrieve_many_queries_tensor_core_path(n, E, nq):
     ms.close()
 
 
-@pytest.mark.parametrize("n,E,nq", [(70_000, 256, 64), (40_000, 1024, 9), (45_001, 64, 33), (38_000, 512, 17)])
+@pytest.mark.parametrize("n,E,nq", [(70_000, 256, 64), (40_000, 1024, 9), (45_001, 64, 33), (38_000, 512, 17), (50_000, 128, 100)])
 def test_tensor_core_filter_candidate_rows(n, E, nq):
     """Segments long enough that every CTA of the filter kernel has several tiles: the kernel lists candidate rows per
     query (thresholds from the shared histogram of group maxima, first tile parked in tensor memory) and the later steps
