@@ -177,6 +177,51 @@ def test_tensor_core_filter_candidate_rows(n, E, nq):
     ms.close()
 
 
+@pytest.mark.parametrize("kind", ["all_negative", "all_equal", "huge_and_tiny"])
+def test_tensor_core_filter_candidate_rows_on_degenerate_scores(kind):
+    """The thresholds of the candidate lists come from a histogram over the bits of the scores: segments whose scores are
+    all negative, all exactly equal, or spread over many binades must give the oracle's ranking like any other (lists
+    that cannot be used fall back to the group maxima and, for ties beyond the margin, to the exact re-scan)."""
+    n, E, nq, k = 40_000, 128, 9, 50
+    rng = np.random.default_rng(77)
+    emb = synth.embeddings(77, n, E, "float16").astype(np.float32)
+    q = synth.queries(77, nq, E, "float16").astype(np.float32)
+    if kind == "all_negative":
+        base = emb[0].copy()
+        emb = base[None, :] + 0.3 * emb
+        emb /= np.linalg.norm(emb, axis=1, keepdims=True)
+        q = -(base[None, :] + 0.3 * q)
+        q /= np.linalg.norm(q, axis=1, keepdims=True)
+    elif kind == "all_equal":
+        emb[:] = emb[0]
+    else:
+        emb *= np.exp2(rng.integers(-12, 4, n)).astype(np.float32)[:, None]  # row norms from 2^-12 to 8
+    emb, q = emb.astype(np.float16), q.astype(np.float16)
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float16, rope_theta=1e4,
+                  max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+    ms.add_facts(to_dev(emb), np.zeros(n, np.int32))
+    ids, sc = ms.retrieve(to_dev(q), k)
+    torch.cuda.synchronize()
+    st = ms.stats()
+    assert st["kernel_timeouts"] == 0
+    ids, sc = ids.cpu().numpy(), sc.cpu().numpy()
+    if kind == "all_negative":
+        assert np.all(sc < 0) and st["filter_list_fallbacks"] == 0
+    if kind == "all_equal":
+        assert np.all(sc == sc[:, :1])  # (which 50 of the 40,000 tied rows come back is not fixed beyond the re-scan's capacity)
+        assert st["filter_fixup_overflows"] == 1
+        for i in range(nq):
+            assert len(set(ids[i].tolist())) == k and ids[i].min() >= 0 and ids[i].max() < n
+    else:
+        for i in range(nq):
+            check_ids(ids[i], sc[i], emb, q[i], k)
+    # the same through the CUDA-core kernels, one query at a time
+    ids_1, sc_1 = ms.retrieve(to_dev(q[:1]), k)
+    if kind != "all_equal":
+        assert np.array_equal(ids_1.cpu().numpy()[0], ids[0]) and np.array_equal(sc_1.cpu().numpy()[0], sc[0])
+    ms.close()
+
+
 @pytest.mark.parametrize("kind", ["exact_copies", "near_copies", "too_many_exact_copies"])
 def test_tensor_core_filter_with_more_tied_groups_than_its_margin(kind):
     """The filter keeps k + 28 groups.  400 rows that tie with (or sit within rounding of) the best score, spread over 400
