@@ -63,6 +63,7 @@ struct memstore {
   int* tc_error = nullptr;
   // candidate rows emitted by the filter kernel (see score_gemm.cuh)
   uint32_t* tc_hist = nullptr;      // [64][kHistWords] + thr_used[64] (zero between calls) + cand_cnt[64][kCandMaxSegs]
+  float* tc_raw = nullptr;                // [64][32 * kRawPerLane]: the table the thresholds of the lists are calibrated from
   unsigned long long* tc_emit = nullptr;  // [64][kTcCandPlaces]: candidate rows listed by the filter kernel
   float* tc_exact = nullptr;        // [64][kListMaxK2]: exact scores of the listed rows that were rescored, by filter rank
   unsigned long long* tc_list_stats = nullptr;  // queries served from their candidate list, rows listed for them, fallbacks
@@ -235,7 +236,7 @@ constexpr int kTcCandSeg = 24;                          // places per epilogue w
 constexpr int kTcMaxCtas = kCandMaxSegs / 4;
 constexpr int kTcRowMargin = 28;     // candidate rows rescored beyond k
 static_assert(kTcMaxK + kTcRowMargin <= kListMaxK2, "the list kernel's per-query arrays hold k + margin rows");
-constexpr size_t kTcHistWords = (size_t)kGemmMaxQ * (kHistWords + 1 + kCandMaxSegs);
+constexpr size_t kTcHistWords = (size_t)kGemmMaxQ * (kHistWords + kCalibWords + 1 + kCandMaxSegs);
 
 // Launch as a programmatic dependent of the kernel before it in the stream (the kernel calls griddepcontrol.wait before
 // it touches anything the earlier kernels write).
@@ -282,6 +283,8 @@ ms_status tc_prepare(memstore* s) {
   MS_CUDA(s, cudaMalloc(&s->tc_error, 2 * sizeof(int)));
   MS_CUDA(s, cudaMalloc(&s->tc_hist, kTcHistWords * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_emit, (size_t)kGemmMaxQ * kTcCandPlaces * sizeof(unsigned long long)));
+  MS_CUDA(s, cudaMalloc(&s->tc_raw, (size_t)kGemmMaxQ * 32 * kRawPerLane * sizeof(float)));
+  MS_CUDA(s, cudaMemset(s->tc_raw, 0xff, (size_t)kGemmMaxQ * 32 * kRawPerLane * sizeof(float)));  // every word kRawEmpty
   MS_CUDA(s, cudaMalloc(&s->tc_exact, (size_t)kGemmMaxQ * kListMaxK2 * sizeof(float)));
   MS_CUDA(s, cudaMemset(s->tc_hist, 0, kTcHistWords * sizeof(uint32_t)));
   MS_CUDA(s, cudaMalloc(&s->tc_list_stats, 3 * sizeof(unsigned long long)));
@@ -326,13 +329,15 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
     const int n_ctas = std::min(n_tiles, s->sm_count);
     const int n_seg = n_ctas * 4;
     const int seg = std::min(kTcCandSeg, kTcCandPlaces / n_seg);
-    const bool emit = k2r <= kListMaxK2 && n_tiles >= 2 * s->sm_count && n_rows >= k2r && n_ctas <= kTcMaxCtas && seg >= 8;
+    const bool emit = k2r <= kListMaxK2 && n_tiles >= kGemmParked * s->sm_count && n_rows >= k2r && n_ctas <= kTcMaxCtas && seg >= 8 &&
+                      n_ctas >= nqb && n_ctas * 4 * kGemmParked <= 32 * kRawPerLane && n_ctas * 4 * kGemmParked >= k2r;
     uint32_t* hist = s->tc_hist;
-    uint32_t* thr_used = hist + (size_t)kGemmMaxQ * kHistWords;
+    uint32_t* calib = hist + (size_t)kGemmMaxQ * kHistWords;  // (the list kernel zeroes a query's counters and calibration as one run of words)
+    uint32_t* thr_used = calib + (size_t)kGemmMaxQ * kCalibWords;
     uint32_t* cand_cnt = thr_used + kGemmMaxQ;
     GemmParams gp{(int)n_rows, c.emb_dim, nqb, s->tc_gmax, s->tc_gmax_stride, s->tc_error, (uint32_t)kGemmSmemBytes,
                   s->test_spin_limit, s->test_mute_producers, s->removed_bits_d,
-                  emit ? hist : nullptr, cand_cnt, thr_used, s->tc_emit, seg, k2r};
+                  emit ? hist : nullptr, calib, s->tc_raw, cand_cnt, thr_used, s->tc_emit, seg, k2r};
     MS_CUDA(s, launch_dependent(score_gemm_groupmax_kernel, dim3((unsigned)n_ctas), dim3(kGemmThreads), kGemmSmemBytes, st, tmap_emb, tmap_q, gp));
     RetrieveParams p = base;
     p.queries = qptr;
@@ -344,9 +349,10 @@ ms_status retrieve_tensor_core(memstore* s, const RetrieveParams& base, int64_t 
       // one launch selects among the listed rows, rescores them and writes the top-k (a query whose list is unusable is
       // served from the group maxima by one CTA of the same launch)
       MS_CUDA(s, launch_dependent(list_topk_kernel<__half>, dim3(kListCtas, (unsigned)nqb), dim3(kListThreads), (size_t)k2 * 8 * sizeof(uint32_t),
-                                  st, p, (const unsigned long long*)s->tc_emit, n_seg, seg, (const uint32_t*)cand_cnt, thr_used, hist, kHistWords,
+                                  st, p, (const unsigned long long*)s->tc_emit, n_seg, seg, (const uint32_t*)cand_cnt, thr_used, hist, kHistWords, calib,
                                   k2r, s->tc_exact, s->tc_tickets, scores_out, s->tc_redo, s->tc_kth, s->tc_list_stats, (const float*)s->tc_gmax,
-                                  s->tc_gmax_stride, n_groups, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows));
+                                  s->tc_gmax_stride, n_groups, k2, (int)n_rows, s->tc_cand_scores, s->tc_cand_rows, reinterpret_cast<uint32_t*>(s->tc_raw),
+                                  32 * kRawPerLane, n_ctas * 4 * kGemmParked));
       s->kernels_launched += 1;
     } else {
       MS_CUDA(s, launch_dependent(select_groups_kernel, dim3((unsigned)nqb), dim3(kTopkThreads), 0, st, (const float*)s->tc_gmax,
@@ -667,6 +673,7 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->tc_error);
     cudaFree(s->tc_hist);
     cudaFree(s->tc_emit);
+    cudaFree(s->tc_raw);
     cudaFree(s->tc_exact);
     cudaFree(s->tc_list_stats);
     cudaFree(s->tiles);

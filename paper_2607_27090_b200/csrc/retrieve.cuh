@@ -1351,9 +1351,10 @@ constexpr int kCandMaxSegs = 1024;
 template <typename T>
 __global__ void __launch_bounds__(kListThreads, 1)
     list_topk_kernel(const RetrieveParams p, const unsigned long long* cand, int n_seg, int seg, const uint32_t* cand_cnt, uint32_t* thr_used,
-                     uint32_t* hist, int hist_words, int k2, float* exact /*[nq][k2]*/, uint32_t* tickets, float* scores_out, int* redo,
+                     uint32_t* hist, int hist_words, uint32_t* calib, int k2, float* exact /*[nq][k2]*/, uint32_t* tickets, float* scores_out, int* redo,
                      float* kth, unsigned long long* list_stats /*served, rows listed, fallbacks*/, const float* gmax, int64_t gmax_stride,
-                     int n_groups, int k2g, int n_rows, float* cand_scores /*[nq][k2g * 8]*/, int32_t* cand_rows) {
+                     int n_groups, int k2g, int n_rows, float* cand_scores /*[nq][k2g * 8]*/, int32_t* cand_rows, uint32_t* raw,
+                     int raw_stride, int n_raw) {
   extern __shared__ uint32_t s_dyn[];
   __shared__ ExtractShared es;
   __shared__ TopkShared sm;  // (the group selection of an unusable list; its candidate array also serves the row selection)
@@ -1405,6 +1406,8 @@ __global__ void __launch_bounds__(kListThreads, 1)
   if (blockIdx.x == 0) {  // clean for the next call (only this kernel's CTA 0 of the query touches the histogram)
     uint4* hq = reinterpret_cast<uint4*>(hist + (size_t)q * hist_words);  // hist_words is a multiple of 4
     for (int i = tid; i < hist_words / 4; i += kListThreads) hq[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < n_raw; i += kListThreads) raw[(size_t)q * raw_stride + i] = 0xffffffffu;  // the calibration table: empty
+    if (tid < 4) calib[(size_t)q * 4 + tid] = 0u;
   }
   const int n_places = n_seg * seg;
   bool ok = !overrun && n >= (uint32_t)k2 && n <= (uint32_t)kListMaxRows && k2 <= kListMaxK2 && n_places <= 65536;

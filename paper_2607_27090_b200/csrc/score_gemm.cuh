@@ -8,21 +8,26 @@
 // decides a rank; it only has to keep every top-k row inside a selected group.
 //
 // With candidate emission on (GemmParams::hist) the kernel ALSO hands the later steps a short list of candidate ROWS per
-// query, so that they need not sweep the group maxima nor rescore whole groups: the epilogue keeps, per query, a
-// histogram of the group maxima seen so far by all CTAs (buckets = the top 13 bits of the order-preserving key:
-// sign, exponent, 4 significand bits; with two coarser levels over the top 9 and the top 5 bits, so that a reader
-// finds its bucket with three loads of one line each), from which any warp can read a
-// threshold - the lower edge of the bucket in which the count of maxima from the top reaches k2.  At least k2 rows
-// score at or above it (group maxima are scores of distinct rows), so a row below it is not among the k2 best; every
-// row at or above the current threshold is appended to the query's candidate list (row, filter score).  The
-// threshold only rises and a stale one only lets more rows through: the histogram is updated with fire-and-forget
-// atomics, a seventh warp of every CTA does nothing but read it and keep the CTA's 64 thresholds in shared memory, and
-// the epilogue warps never wait for global memory: a warp appends to its OWN segment of every query's list
-// ([query][CTA][warp][cand_seg] places, counted in registers) and publishes its counts when it ends.  The first tile of a
-// CTA is computed before any threshold exists; its accumulator stays parked in tensor memory and its rows are emitted
-// after the CTA's last tile.  The list's consumer checks the counts (at least k2 rows in all, no segment overrun) and
-// falls back to the group maxima otherwise.  (Same-address atomics drain at about 8 ns each: the first tiles of all
-// CTAs arrive together, so a warp counts one maximum per query for them - that of its 32 rows - not four.)
+// query, so that they need not sweep the group maxima nor rescore whole groups.  Every row whose score reaches the
+// query's current THRESHOLD is appended to the query's list (row, filter score).  A threshold is valid when at least k2
+// rows of the segment score at or above it (then no row below it is among the k2 best), and thresholds only rise:
+//  - the first two tiles of every CTA are computed before any threshold exists; their accumulators stay PARKED in tensor
+//    memory, and every epilogue warp only writes the best score of its 32 rows per query to a global table;
+//  - when all CTAs have done so (the table is filled with a pattern that is no score between calls, so an entry is its
+//    own arrival flag; every CTA is resident, one per SM), the seventh warp of CTA q CALIBRATES query q: the exact k2-th largest of the table's values (a bitwise search on the order-preserving keys, in
+//    registers) is the first threshold, and the span from it to the largest value fixes 256 LINEAR buckets for the
+//    query's histogram - linear in the score and as wide as the query's own top region, so that the resolution does
+//    not depend on the magnitude of the scores (buckets over the bits of the floats resolve 6 %: useless when all the
+//    best scores lie within 1 % of one another);
+//  - from then on a warp that lists rows for a query also counts the best of them in the query's histogram
+//    (fire-and-forget atomics: one per level), and the seventh warp of every CTA keeps reading the histograms (two loads
+//    of one line per query) and raises the CTA's 64 thresholds in shared memory to the lower edge of the bucket at which
+//    the count from the top reaches k2.  A stale threshold only lets more rows through.
+// The epilogue warps never wait for global memory: a warp appends to its OWN segment of every query's list
+// ([query][CTA][warp][cand_seg] places, counted in registers) and publishes its counts when it ends.  The parked tiles'
+// rows are compared with the thresholds later, in time the epilogue would otherwise spend waiting.  The list's consumer
+// checks the counts (at least k2 rows in all, no segment overrun) and falls back to the group maxima otherwise.  Every
+// wait (for the arrivals, for the calibrations) is bounded; when one runs out nothing is listed and the fallback serves.
 //
 // Tiling: facts on M (128 rows per tile = the 128 TMEM lanes), queries on N (64), K = E in chunks of 64 fp16
 // (one 128-byte swizzle row).  All queries stay in shared memory for the kernel's lifetime (E/64 chunks of 8 KiB);
@@ -51,10 +56,12 @@ constexpr int kGemmThreads = 224;
 constexpr int kGemmTmemCols = 512;    // all of an SM's tensor memory (one CTA per SM, and an allocation is a power of two)
 constexpr int kGemmAccBufs = 4;       // working accumulators of 64 columns: the MMAs may run this many tiles ahead of the epilogue
 constexpr int kGemmParked = 2;        // first tiles of a CTA whose accumulators stay in tensor memory (candidate emission only)
-constexpr int kHistFine = 8192;       // order key >> 19
-constexpr int kHistMid = 512;         // order key >> 23: 16 fine buckets each
-constexpr int kHistCoarse = 32;       // order key >> 27: 16 middle buckets each
-constexpr int kHistWords = kHistCoarse + kHistMid + kHistFine;  // one query's counters: [coarse][middle][fine]
+constexpr int kHistFine = 256;        // linear buckets over the query's calibrated span
+constexpr int kHistCoarse = 16;       // 16 fine buckets each
+constexpr int kHistWords = kHistCoarse + kHistFine;  // one query's counters: [coarse][fine]
+constexpr int kCalibWords = 4;        // one query's calibration: {lowest score, buckets per unit, ready, -}, 16 bytes that a reader loads at once
+constexpr int kRawPerLane = 40;       // parked-tile maxima per query <= 32 * this (2 tiles x 4 warps x CTAs)
+constexpr uint32_t kRawEmpty = 0xffffffffu;  // (a NaN pattern: never a score)
 constexpr int kGemmABytes = kGemmTileRows * kGemmKChunk * 2;  // 16 KiB
 constexpr int kGemmQBytes = kGemmMaxQ * kGemmKChunk * 2;      // 8 KiB per chunk
 constexpr int kGemmMaxE = 1024;
@@ -72,6 +79,9 @@ struct GemmParams {
   const uint32_t* removed_bits;  // one bit per row of the segment, or nullptr: removed rows take no part in a group's maximum
   // candidate emission (hist == nullptr: off).  All counters are zero when the kernel starts.
   uint32_t* hist;         // [kGemmMaxQ][kHistWords]
+  uint32_t* calib;        // [kGemmMaxQ][kCalibWords], zero when the kernel starts (kept apart from the counters: every CTA polls it)
+  float* raw;             // [kGemmMaxQ][32 * kRawPerLane]: the best score of every epilogue warp's rows in its parked tiles;
+                          // every word is kRawEmpty when the kernel starts
   uint32_t* cand_cnt;     // [kGemmMaxQ][gridDim.x * 4]: rows the warp found for the query (beyond cand_seg: the surplus was dropped)
   uint32_t* thr_used;     // [kGemmMaxQ]: order key of the highest threshold any CTA applied (0: none)
   unsigned long long* cand;  // [kGemmMaxQ][gridDim.x * 4][cand_seg]: (order key of the filter score << 32) | row
@@ -87,52 +97,63 @@ __device__ __forceinline__ float gemm_key_value(uint32_t kx) {
   return __uint_as_float((kx & 0x80000000u) ? (kx & 0x7fffffffu) : ~kx);
 }
 
-// One level of the threshold search, for two queries at once (the loads of both are issued together): counters
-// c[0..N) of each, scanned from the top; `cum` counts the maxima above the bucket that is returned, the first one from
-// the top at which the running count reaches `need` (-1: not reached).
-template <int NVEC>
-__device__ __forceinline__ void hist_scan2(const uint32_t* a, const uint32_t* b, uint32_t need, uint32_t& cum_a, uint32_t& cum_b, int& at_a,
-                                           int& at_b) {
-  uint4 ca[NVEC], cb[NVEC];
-#pragma unroll
-  for (int i = 0; i < NVEC; ++i) {
-    ca[i] = __ldcg(reinterpret_cast<const uint4*>(a) + i);
-    cb[i] = __ldcg(reinterpret_cast<const uint4*>(b) + i);
-  }
-  at_a = at_b = -1;
-  auto scan1 = [&](uint32_t x, int idx, uint32_t& cum, int& at) {
-    if (at < 0) {
-      if (cum + x >= need) at = idx;
-      else cum += x;
-    }
-  };
-#pragma unroll
-  for (int i = NVEC - 1; i >= 0; --i) {
-    scan1(ca[i].w, 4 * i + 3, cum_a, at_a);
-    scan1(ca[i].z, 4 * i + 2, cum_a, at_a);
-    scan1(ca[i].y, 4 * i + 1, cum_a, at_a);
-    scan1(ca[i].x, 4 * i, cum_a, at_a);
-    scan1(cb[i].w, 4 * i + 3, cum_b, at_b);
-    scan1(cb[i].z, 4 * i + 2, cum_b, at_b);
-    scan1(cb[i].y, 4 * i + 1, cum_b, at_b);
-    scan1(cb[i].x, 4 * i, cum_b, at_b);
-  }
+// The bucket of a score in a query's calibrated histogram.
+__device__ __forceinline__ int hist_bucket(float x, float lo, float per_unit) {
+  const float b = (x - lo) * per_unit;
+  return b >= (float)(kHistFine - 1) ? kHistFine - 1 : b > 0.f ? (int)b : 0;
 }
 
-// The thresholds of two queries from their histograms (ha, hb: the queries' kHistWords counters).  -infinity while
-// fewer than `need` maxima have been published.  A coarser counter may run ahead of the finer ones for a moment; the
-// search then stops at the coarser bucket's lower edge, which is lower and therefore still valid.
-__device__ __forceinline__ void hist_thresholds2(const uint32_t* ha, const uint32_t* hb, uint32_t need, float& ta, float& tb) {
+// The threshold of a query from its histogram: the lower edge (a quarter of a bucket further down, so that float rounding
+// at an edge cannot matter) of the bucket at which the count from the top reaches `need`; `lo` while it does not.
+// Two queries at once: the loads of both are issued together.
+__device__ __forceinline__ void hist_thresholds2(const uint32_t* ha, const uint32_t* hb, uint32_t need, float lo_a, float pu_a, float lo_b,
+                                                 float pu_b, float& ta, float& tb) {
+  auto scan16 = [&](const uint4 (&c)[4], uint32_t& cum, int& at) {
+    at = -1;
+    auto one = [&](uint32_t x, int idx) {
+      if (at < 0) {
+        if (cum + x >= need) at = idx;
+        else cum += x;
+      }
+    };
+#pragma unroll
+    for (int i = 3; i >= 0; --i) {
+      one(c[i].w, 4 * i + 3);
+      one(c[i].z, 4 * i + 2);
+      one(c[i].y, 4 * i + 1);
+      one(c[i].x, 4 * i);
+    }
+  };
+  uint4 ca[4], cb[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    ca[i] = __ldcg(reinterpret_cast<const uint4*>(ha) + i);
+    cb[i] = __ldcg(reinterpret_cast<const uint4*>(hb) + i);
+  }
   uint32_t cum_a = 0, cum_b = 0;
-  int ca, cb, ma, mb, fa, fb;
-  hist_scan2<kHistCoarse / 4>(ha, hb, need, cum_a, cum_b, ca, cb);
-  const int ca0 = ca < 0 ? 0 : ca, cb0 = cb < 0 ? 0 : cb;
-  hist_scan2<4>(ha + kHistCoarse + ca0 * 16, hb + kHistCoarse + cb0 * 16, need, cum_a, cum_b, ma, mb);
-  const int ma0 = ca0 * 16 + (ma < 0 ? 0 : ma), mb0 = cb0 * 16 + (mb < 0 ? 0 : mb);
-  hist_scan2<4>(ha + kHistCoarse + kHistMid + ma0 * 16, hb + kHistCoarse + kHistMid + mb0 * 16, need, cum_a, cum_b, fa, fb);
-  const uint32_t bucket_a = (uint32_t)ma0 * 16u + (uint32_t)(fa < 0 ? 0 : fa), bucket_b = (uint32_t)mb0 * 16u + (uint32_t)(fb < 0 ? 0 : fb);
-  ta = ca < 0 ? -INFINITY : gemm_key_value(bucket_a << 19);
-  tb = cb < 0 ? -INFINITY : gemm_key_value(bucket_b << 19);
+  int at_a, at_b, fa, fb;
+  scan16(ca, cum_a, at_a);
+  scan16(cb, cum_b, at_b);
+  const int a0 = at_a < 0 ? 0 : at_a, b0 = at_b < 0 ? 0 : at_b;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    ca[i] = __ldcg(reinterpret_cast<const uint4*>(ha + kHistCoarse + a0 * 16) + i);
+    cb[i] = __ldcg(reinterpret_cast<const uint4*>(hb + kHistCoarse + b0 * 16) + i);
+  }
+  scan16(ca, cum_a, fa);  // (a coarse counter may run ahead of its fine ones for a moment: then the coarse bucket's edge)
+  scan16(cb, cum_b, fb);
+  const float ea = (float)(a0 * 16 + (fa < 0 ? 0 : fa)) - 0.25f, eb = (float)(b0 * 16 + (fb < 0 ? 0 : fb)) - 0.25f;
+  ta = (at_a < 0 || !(pu_a > 0.f)) ? lo_a : fmaxf(lo_a, lo_a + ea / pu_a);
+  tb = (at_b < 0 || !(pu_b > 0.f)) ? lo_b : fmaxf(lo_b, lo_b + eb / pu_b);
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // Shared memory after the 1 KiB alignment of the base: queries, ring, epilogue staging (4 warps x [4 groups][32
@@ -196,16 +217,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Count one maximum in the three levels of its query's histogram (lanes with `mine` false do nothing).
-__device__ __forceinline__ void hist_publish(uint32_t* hq, float gx, bool mine) {
-  if (mine && gx > -INFINITY) {
-    const uint32_t bucket = gemm_order_key(gx) >> 19;
-    atomicAdd(hq + kHistCoarse + kHistMid + bucket, 1u);
-    atomicAdd(hq + kHistCoarse + (bucket >> 4), 1u);
-    atomicAdd(hq + (bucket >> 8), 1u);
-  }
-}
 
 // One column of the warp's 32 tensor-memory lanes; the value is there after tmem_ld_wait().
 __device__ __forceinline__ uint32_t tmem_ld1_issue(uint32_t taddr) {
@@ -343,31 +354,122 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     __syncwarp();
   } else if (warp == 6) {
     // ------------------------------------------------------------------ thresholds (candidate emission only)
-    // Reads the histogram over and over (three loads of a line per query and round, two queries per lane) and raises
-    // the thresholds in shared memory; ends when the four epilogue warps have, or after a bounded number of rounds.
     if (emitting) {
+      constexpr unsigned kFull = 0xffffffffu;
+      const int n_raw = (int)(gridDim.x * 4u * (uint32_t)kGemmParked);  // values per query in the table: epilogue warps x parked tiles
+      // (a) the warp of CTA q calibrates query q once the parked tiles of all CTAs are in the table
+      if ((int)blockIdx.x < p.nq) {
+        const int q = blockIdx.x;
+        float lo = INFINITY, per_unit = 0.f;  // (nothing reaches +infinity: no row is listed and the group maxima serve the query)
+        bool ok = false;
+        uint32_t key[kRawPerLane];
+        if (n_raw <= 32 * kRawPerLane && n_raw >= p.k2) {
+          const uint32_t* rq = reinterpret_cast<const uint32_t*>(p.raw) + (size_t)q * (32 * kRawPerLane);
+          for (uint32_t w = 0; w < limit && !*abort_flag && !ok; ++w) {  // until every entry has been written
+            bool full = true;
+#pragma unroll
+            for (int j = 0; j < kRawPerLane; ++j) {
+              const int i = j * 32 + lane;
+              const uint32_t bits = i < n_raw ? __ldcg(rq + i) : 0u;
+              full = full && bits != kRawEmpty;
+              key[j] = i < n_raw ? gemm_order_key(__uint_as_float(bits)) : 0u;
+            }
+            ok = __all_sync(kFull, full);
+            if (!ok) __nanosleep(256);
+          }
+        }
+        if (ok) {
+          // the k2-th largest key, two bits at a time: the largest value that at least k2 keys reach
+          uint32_t kth = 0u, top = 0u;
+          for (int bit = 30; bit >= 0; bit -= 2) {
+            const uint32_t c1 = kth | (1u << bit), c2 = kth | (2u << bit), c3 = kth | (3u << bit);
+            int n1 = 0, n2 = 0, n3 = 0;
+#pragma unroll
+            for (int j = 0; j < kRawPerLane; ++j) {
+              n1 += key[j] >= c1;
+              n2 += key[j] >= c2;
+              n3 += key[j] >= c3;
+            }
+            n1 = __reduce_add_sync(kFull, n1);
+            n2 = __reduce_add_sync(kFull, n2);
+            n3 = __reduce_add_sync(kFull, n3);
+            kth = n3 >= p.k2 ? c3 : n2 >= p.k2 ? c2 : n1 >= p.k2 ? c1 : kth;
+          }
+#pragma unroll
+          for (int j = 0; j < kRawPerLane; ++j) top = max(top, key[j]);
+          top = __reduce_max_sync(kFull, top);
+          const float t0 = gemm_key_value(kth), hi = gemm_key_value(top);
+          if (t0 > -INFINITY && hi < INFINITY) {
+            lo = t0;
+            const float span = 2.f * (hi - t0);  // room above the best score seen so far; scores beyond it share the last bucket
+            per_unit = span > 1e-30f ? (float)kHistFine / span : 0.f;
+            // (The table's own values are not counted in the histogram: until k2 later maxima have reached the threshold
+            // it stays where it is, and afterwards it is read from those alone - lower than with the table's values
+            // counted too, never invalid.  Counting them costs atomics on a few addresses right when every warp of the
+            // GPU waits for this calibration: same-address atomics take 50 - 100 ns each while the embeddings stream.)
+          }
+        }
+        __syncwarp();
+        if (lane == 0) {
+          uint32_t* cq = p.calib + (size_t)q * kCalibWords;
+          cq[0] = __float_as_uint(lo);
+          cq[1] = __float_as_uint(per_unit);
+          __threadfence();  // the two words above before the flag
+          st_release_u32(cq + 2, 1u);
+        }
+      }
+      // (b) the calibration of every query: lane l looks after queries l and l + 32
       const int qa = lane < p.nq ? lane : 0, qb = lane + 32 < p.nq ? lane + 32 : 0;
-      float mine_a = -INFINITY, mine_b = -INFINITY;
-      int settled = 0;  // rounds since every query has had a threshold
-      for (uint32_t round = 0; round < limit && *epi_done < 4 && !*abort_flag; ++round) {
+      const uint32_t* ha = p.hist + (size_t)qa * kHistWords;
+      const uint32_t* hb = p.hist + (size_t)qb * kHistWords;
+      // (one 16-byte load per query and poll, every half microsecond: 148 CTAs poll the same 64 entries)
+      bool have = false;
+      uint4 ca = make_uint4(0u, 0u, 0u, 0u), cb = ca;
+      for (uint32_t w = 0; w < limit && !*abort_flag && *epi_done < 4; ++w) {
+        ca = __ldcg(reinterpret_cast<const uint4*>(p.calib + (size_t)qa * kCalibWords));
+        cb = __ldcg(reinterpret_cast<const uint4*>(p.calib + (size_t)qb * kCalibWords));
+        have = ca.z != 0u && cb.z != 0u;
+        if (__all_sync(kFull, have)) break;
+        __nanosleep(512);
+      }
+      have = __all_sync(kFull, have);
+      __threadfence();
+      float lo_a = INFINITY, pu_a = 0.f, lo_b = INFINITY, pu_b = 0.f;
+      if (have) {
+        lo_a = __uint_as_float(ca.x);
+        pu_a = __uint_as_float(ca.y);
+        lo_b = __uint_as_float(cb.x);
+        pu_b = __uint_as_float(cb.y);
+      }
+      float mine_a = lo_a, mine_b = lo_b;
+      if (lane < p.nq) {
+        s_thr[lane] = mine_a;
+        if (mine_a < INFINITY) atomicMax(p.thr_used + lane, gemm_order_key(mine_a));
+      }
+      if (lane + 32 < p.nq) {
+        s_thr[lane + 32] = mine_b;
+        if (mine_b < INFINITY) atomicMax(p.thr_used + lane + 32, gemm_order_key(mine_b));
+      }
+      __syncwarp();
+      __threadfence_block();
+      if (lane == 0) *thr_ready = 1;
+      // (c) the histograms, over and over: two loads of a line per query and round.  The thresholds settle within the first
+      // few tiles: read quickly at first, then every 16 us or so; asleep in short naps so that the end of the CTA is
+      // noticed at once.  Ends when the four epilogue warps have, or after a bounded number of rounds.
+      for (uint32_t round = 0; have && round < limit && *epi_done < 4 && !*abort_flag; ++round) {
         float ta, tb;
-        hist_thresholds2(p.hist + (size_t)qa * kHistWords, p.hist + (size_t)qb * kHistWords, (uint32_t)p.k2, ta, tb);
-        if (lane < p.nq && ta > mine_a) {
+        hist_thresholds2(ha, hb, (uint32_t)p.k2, lo_a, pu_a, lo_b, pu_b, ta, tb);
+        if (lane < p.nq && ta > mine_a && ta < INFINITY) {
           mine_a = ta;
           s_thr[lane] = ta;
           atomicMax(p.thr_used + lane, gemm_order_key(ta));
         }
-        if (lane + 32 < p.nq && tb > mine_b) {
+        if (lane + 32 < p.nq && tb > mine_b && tb < INFINITY) {
           mine_b = tb;
           s_thr[lane + 32] = tb;
           atomicMax(p.thr_used + lane + 32, gemm_order_key(tb));
         }
-        const bool have = (lane >= p.nq || mine_a > -INFINITY) && (lane + 32 >= p.nq || mine_b > -INFINITY);
-        if (__all_sync(0xffffffffu, have) && lane == 0) *thr_ready = 1;
-        // the thresholds settle within the first few tiles: read quickly at first, then every 16 us or so (every round
-        // costs the L2 a line per level and query); asleep in short naps so that the end of the CTA is noticed at once
-        if (*thr_ready) ++settled;
-        const int naps = settled < 7 ? (settled ? 1 << (settled - 1) : 1) : 64;
+        const int naps = round < 6 ? 1 << round : 64;
         for (int w = 0; w < naps && *epi_done < 4 && !*abort_flag; ++w) __nanosleep(256);
       }
     }
@@ -404,6 +506,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     // the query is counted in the histogram (it reaches the threshold; lower values could not raise it): one lane per
     // level, both queries in one instruction.
     uint32_t cnt_lo = 0u, cnt_hi = 0u;
+    float cal_lo_lo = INFINITY, cal_pu_lo = 0.f, cal_lo_hi = INFINITY, cal_pu_hi = 0.f;  // lane l: the calibrations of queries l and l + 32
     const size_t my_seg = (size_t)blockIdx.x * 4 + (size_t)(warp - 2);
     const size_t n_seg = (size_t)gridDim.x * 4;
     auto serve = [&](uint32_t taddr, int row, uint32_t m_lo, uint32_t m_hi, bool publish) {
@@ -434,12 +537,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
             p.cand[((size_t)(qb + 32 * h) * n_seg + my_seg) * p.cand_seg + slot_b] = ((unsigned long long)kb << 32) | (uint32_t)row;
           if (publish) {
             const uint32_t best_a = __reduce_max_sync(kFull, pa ? ka : 0u), best_b = __reduce_max_sync(kFull, pb ? kb : 0u);
-            if (lane < (two ? 6 : 3)) {
-              const bool second = lane >= 3;
-              const int level = second ? lane - 3 : lane;
-              const uint32_t bucket = (second ? best_b : best_a) >> 19;
-              uint32_t* hq = p.hist + (size_t)((second ? qb : qa) + 32 * h) * kHistWords;
-              atomicAdd(level == 0 ? hq + kHistCoarse + kHistMid + bucket : level == 1 ? hq + kHistCoarse + (bucket >> 4) : hq + (bucket >> 8), 1u);
+            const float lo_a = __shfl_sync(kFull, h ? cal_lo_hi : cal_lo_lo, qa), pu_a = __shfl_sync(kFull, h ? cal_pu_hi : cal_pu_lo, qa);
+            const float lo_b = __shfl_sync(kFull, h ? cal_lo_hi : cal_lo_lo, qb), pu_b = __shfl_sync(kFull, h ? cal_pu_hi : cal_pu_lo, qb);
+            if (lane < (two ? 4 : 2)) {  // lanes 0, 1: the two levels of query a; lanes 2, 3: of query b
+              const bool second = lane >= 2;
+              const float lo = second ? lo_b : lo_a;
+              if (lo < INFINITY) {
+                const int b = hist_bucket(gemm_key_value(second ? best_b : best_a), lo, second ? pu_b : pu_a);
+                uint32_t* hq = p.hist + (size_t)((second ? qb : qa) + 32 * h) * kHistWords;
+                atomicAdd((lane & 1) ? hq + (b >> 4) : hq + kHistCoarse + b, 1u);
+              }
             }
           }
         }
@@ -470,7 +577,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     // Before the first rows are compared with thresholds: give the threshold warp a moment to see the first tiles of
     // the other CTAs (bounded; without thresholds every row would be listed).  The MMAs go on meanwhile.
     auto await_thresholds = [&]() {
-      for (int w = 0; w < 512 && !*thr_ready && !*abort_flag; ++w) __nanosleep(128);
+      for (int w = 0; w < 1024 && !*thr_ready && !*abort_flag; ++w) __nanosleep(128);
+      if (*thr_ready) {  // the calibrations are published: this lane's two, for the histogram updates
+        const uint32_t* ha = p.calib + (size_t)(lane < p.nq ? lane : 0) * kCalibWords;
+        const uint32_t* hb = p.calib + (size_t)(lane + 32 < p.nq ? lane + 32 : 0) * kCalibWords;
+        // (the threshold warp saw every calibration's flag before it raised thr_ready, and these loads go to the L2)
+        __threadfence();
+        const uint4 ca = __ldcg(reinterpret_cast<const uint4*>(ha)), cb = __ldcg(reinterpret_cast<const uint4*>(hb));
+        if (ca.z != 0u) {
+          cal_lo_lo = __uint_as_float(ca.x);
+          cal_pu_lo = __uint_as_float(ca.y);
+        }
+        if (cb.z != 0u) {
+          cal_lo_hi = __uint_as_float(cb.x);
+          cal_pu_hi = __uint_as_float(cb.y);
+        }
+      }
     };
     int it = 0, parked_emitted = 0;
     bool complete = true;
@@ -526,9 +648,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
         if (q < p.nq) {
           const float4 g = make_float4(my_stage[lane], my_stage[32 + lane], my_stage[64 + lane], my_stage[96 + lane]);
           *reinterpret_cast<float4*>(p.gmax + (int64_t)q * p.gmax_stride + col) = g;
-          // a parked tile is computed before any threshold exists: the best of the warp's 32 rows feeds the histogram,
-          // and the rows are looked at again later
-          if (parked) hist_publish(p.hist + (size_t)q * kHistWords, fmaxf(fmaxf(g.x, g.y), fmaxf(g.z, g.w)), true);
+          // a parked tile is computed before any threshold exists: the best of the warp's 32 rows goes to the table the
+          // thresholds are calibrated from, and the rows are looked at again later
+          if (parked) p.raw[(size_t)q * (32 * kRawPerLane) + (my_seg * kGemmParked + (size_t)it)] = fmaxf(fmaxf(g.x, g.y), fmaxf(g.z, g.w));
         }
         __syncwarp();
       }
