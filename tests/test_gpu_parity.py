@@ -177,7 +177,7 @@ def test_tensor_core_filter_candidate_rows(n, E, nq):
     ms.close()
 
 
-@pytest.mark.parametrize("kind", ["all_negative", "all_equal", "huge_and_tiny"])
+@pytest.mark.parametrize("kind", ["all_negative", "all_equal", "huge_and_tiny", "best_rows_last"])
 def test_tensor_core_filter_candidate_rows_on_degenerate_scores(kind):
     """The thresholds of the candidate lists come from a histogram over the bits of the scores: segments whose scores are
     all negative, all exactly equal, or spread over many binades must give the oracle's ranking like any other (lists
@@ -194,6 +194,10 @@ def test_tensor_core_filter_candidate_rows_on_degenerate_scores(kind):
         q /= np.linalg.norm(q, axis=1, keepdims=True)
     elif kind == "all_equal":
         emb[:] = emb[0]
+    elif kind == "best_rows_last":
+        # rows in ascending order of their score with query 0: the thresholds calibrated on the first tiles are far too low
+        # for that query (its list may overrun and fall back), and every other query sees an ordinary segment
+        emb = emb[np.argsort(emb @ q[0], kind="stable")]
     else:
         emb *= np.exp2(rng.integers(-12, 4, n)).astype(np.float32)[:, None]  # row norms from 2^-12 to 8
     emb, q = emb.astype(np.float16), q.astype(np.float16)
