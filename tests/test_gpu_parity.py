@@ -942,6 +942,45 @@ def test_calls_captured_in_a_cuda_graph_replay_correctly(n_calls):
     ms.close()
 
 
+@pytest.mark.parametrize("n", [12_000, 40_000])
+def test_tensor_core_retrieve_captured_in_a_cuda_graph(n):
+    """The tensor-core retrieve path (scoring kernel and the kernels after it, launched as programmatic dependents of one
+    another) recorded into a CUDA graph gives the eager results on every replay - with group maxima only (short segment)
+    and with candidate lists, whose counters, table and thresholds must be left clean by every replay for the next."""
+    E, nq, k = 128, 12, 40
+    emb = synth.embeddings(98, n, E, "float16")
+    q = to_dev(synth.queries(98, nq, E, "float16"))
+    ms = MemStore(n_layers=1, n_kv_heads=1, head_dim=16, emb_dim=E, emb_dtype=torch.float16, rope_theta=1e4,
+                  max_facts_per_user=n, max_kv_tokens=0)  # fmt: skip
+    ms.add_facts(to_dev(emb), np.zeros(n, np.int32))
+    ids_e, sc_e = ms.retrieve(q, k)  # (also sizes the scratch: nothing is allocated during the capture)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    ids_g = torch.empty((nq, k), dtype=torch.int32, device=DEV)
+    sc_g = torch.empty((nq, k), dtype=torch.float32, device=DEV)
+    with torch.cuda.stream(side):
+        ms.retrieve(q, k, out_ids=ids_g, out_scores=sc_g, stream=side)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            ms.retrieve(q, k, out_ids=ids_g, out_scores=sc_g, stream=side)
+            ms.retrieve(q, k, out_ids=ids_g, out_scores=sc_g, stream=side)  # twice in one graph: the second finds clean scratch
+    torch.cuda.synchronize()
+    for rep in range(3):
+        ids_g.fill_(-7)
+        sc_g.fill_(-7.0)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(ids_g, ids_e) and torch.equal(sc_g, sc_e)
+        ids_x, sc_x = ms.retrieve(q, k)  # an eager call between replays
+        assert torch.equal(ids_x, ids_e) and torch.equal(sc_x, sc_e)
+    st = ms.stats()
+    assert st["kernel_timeouts"] == 0 and st["filter_list_fallbacks"] == 0
+    for i in (0, nq - 1):
+        check_ids(ids_e[i].cpu().numpy(), sc_e[i].cpu().numpy(), emb, q[i].cpu().numpy(), k)
+    ms.close()
+
+
 def test_head_sharded_stores_reproduce_the_unsharded_cache():
     """Tensor-parallel serving: each shard holds a slice of the KV heads (and all embeddings), retrieves the same ids and
     fills its own cache; together the shard caches are the unsharded cache, bit for bit.  (Shards run one after the
