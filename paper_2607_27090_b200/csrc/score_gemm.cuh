@@ -14,8 +14,9 @@
 //  - the first two tiles of every CTA are computed before any threshold exists; their accumulators stay PARKED in tensor
 //    memory, and every epilogue warp only writes the best score of its 32 rows per query to a global table;
 //  - when all CTAs have done so (the table is filled with a pattern that is no score between calls, so an entry is its
-//    own arrival flag; every CTA is resident, one per SM), the seventh warp of CTA q CALIBRATES query q: the exact k2-th largest of the table's values (a bitwise search on the order-preserving keys, in
-//    registers) is the first threshold, and the span from it to the largest value fixes 256 LINEAR buckets for the
+//    own arrival flag; every CTA is resident, one per SM), the seventh warp of CTA q CALIBRATES query q: the exact
+//    k2-th largest of the table's values (a search on the order-preserving keys, two bits at a time, in registers) is the
+//    first threshold, and the span from it to the largest value fixes 256 LINEAR buckets for the
 //    query's histogram - linear in the score and as wide as the query's own top region, so that the resolution does
 //    not depend on the magnitude of the scores (buckets over the bits of the floats resolve 6 %: useless when all the
 //    best scores lie within 1 % of one another);
@@ -31,8 +32,9 @@
 //
 // Tiling: facts on M (128 rows per tile = the 128 TMEM lanes), queries on N (64), K = E in chunks of 64 fp16
 // (one 128-byte swizzle row).  All queries stay in shared memory for the kernel's lifetime (E/64 chunks of 8 KiB);
-// embedding tiles stream through a 4-stage ring of 16 KiB TMA boxes.  Accumulators are double-buffered in TMEM
-// (2 x 64 columns) so that the epilogue of a tile overlaps the MMAs of the next.
+// embedding tiles stream through a ring of 16 KiB TMA boxes that takes the rest of the shared memory (6 stages at
+// E = 1024).  Four working accumulators of 64 columns live in tensor memory (plus the parked ones), so that the MMAs -
+// and with them the loads, which a stalled MMA lane stalls - can run several tiles ahead of the epilogue.
 //   warp 0     TMA producer (one elected lane)
 //   warp 1     TMEM allocation, tcgen05.mma issue (one elected lane), tcgen05.commit -> mbarriers
 //   warps 2-5  epilogue: tcgen05.ld of the warp's 32 TMEM lanes, row mask, 8-row max by shuffles, 16-byte stores
