@@ -489,6 +489,30 @@ __device__ __forceinline__ float div_by_scale(float x, float s, float r) {
   return (a < 1e30f && a > 1e-30f) ? q2 : q0;
 }
 
+// Two quotients at once with the packed fp32 instructions of this architecture (mul / fma .f32x2: each half is the
+// IEEE operation of the scalar instruction, so the results are those of div_by_scale bit for bit, in half the
+// instructions).
+__device__ __forceinline__ unsigned long long pack_f32x2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void div_by_scale_x2(float x0, float x1, float s, float r, float& o0, float& o1) {
+  const unsigned long long X = pack_f32x2(x0, x1), NS = pack_f32x2(-s, -s), R = pack_f32x2(r, r);
+  unsigned long long Q0, T, Q1, Q2;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(Q0) : "l"(X), "l"(R));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(T) : "l"(Q0), "l"(NS), "l"(X));  // x - q0 s, exactly
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(Q1) : "l"(T), "l"(R), "l"(Q0));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(T) : "l"(Q1), "l"(NS), "l"(X));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(Q2) : "l"(T), "l"(R), "l"(Q1));
+  float a0, a1, b0, b1;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(Q0));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(Q2));
+  const float m0 = fabsf(a0), m1 = fabsf(a1);
+  o0 = (m0 < 1e30f && m0 > 1e-30f) ? b0 : a0;
+  o1 = (m1 < 1e30f && m1 > 1e-30f) ? b1 : a1;
+}
+
 // The 8 bf16 values of a 16-byte vector divided by `scale` in fp32: the arithmetic of the serving engines' own 8-bit
 // cache write (they divide the bf16 key or value by the per-tensor scale in fp32 and round once to e4m3).
 template <bool HW_DIV>
@@ -496,8 +520,12 @@ __device__ __forceinline__ void scaled_floats(const uint4& a, float scale, float
   const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    f[2 * w] = div_by_scale<HW_DIV>(bf16lo(aw[w]), scale, recip);
-    f[2 * w + 1] = div_by_scale<HW_DIV>(bf16hi(aw[w]), scale, recip);
+    if (HW_DIV) {
+      f[2 * w] = div_by_scale<true>(bf16lo(aw[w]), scale, recip);
+      f[2 * w + 1] = div_by_scale<true>(bf16hi(aw[w]), scale, recip);
+    } else {
+      div_by_scale_x2(bf16lo(aw[w]), bf16hi(aw[w]), scale, recip, f[2 * w], f[2 * w + 1]);
+    }
   }
 }
 
