@@ -53,6 +53,26 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   }
 }
 
+// acc + x[0] y[0] + ... + x[7] y[7] for the 8 fp16 values of two 16-byte vectors, added in index order with the
+// mixed-precision FMA of this architecture (fma.rn.f32.f16: fp16 factors, fp32 addend and result, the exact product
+// rounded once with the sum) - bit for bit what fmaf gives on the converted values, without the sixteen conversions.
+__device__ __forceinline__ float dot8_f16(const uint4& x, const uint4& y, float acc) {
+  const uint32_t* xw = reinterpret_cast<const uint32_t*>(&x);
+  const uint32_t* yw = reinterpret_cast<const uint32_t*>(&y);
+#pragma unroll
+  for (int w = 0; w < 4; ++w)
+    asm("{\n\t"
+        ".reg .b16 xl, xh, yl, yh;\n\t"
+        "mov.b32 {xl, xh}, %1;\n\t"
+        "mov.b32 {yl, yh}, %2;\n\t"
+        "fma.rn.f32.f16 %0, xl, yl, %0;\n\t"
+        "fma.rn.f32.f16 %0, xh, yh, %0;\n\t"
+        "}"
+        : "+f"(acc)
+        : "r"(xw[w]), "r"(yw[w]));
+  return acc;
+}
+
 // fp32 score -> unsigned key that orders like the float
 __device__ __forceinline__ uint32_t order_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -140,15 +160,8 @@ __device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, c
       const int v = v0 + u * 32 + lane;
       if (v < nvec) {
         if (sizeof(T) == 2) {
-          float f[8], h[8], g[8];
-          unpack8(x[u], f);
-          unpack8(z[u], h);
-          unpack8(y[u], g);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            a0 = fmaf(f[i], g[i], a0);
-            a1 = fmaf(h[i], g[i], a1);
-          }
+          a0 = dot8_f16(x[u], y[u], a0);
+          a1 = dot8_f16(z[u], y[u], a1);
         } else {
           const float* f = reinterpret_cast<const float*>(&x[u]);
           const float* h = reinterpret_cast<const float*>(&z[u]);
@@ -158,50 +171,6 @@ __device__ __forceinline__ void score_two_rows(const RetrieveParams& p, int q, c
             a0 = fmaf(f[i], g[i], a0);
             a1 = fmaf(h[i], g[i], a1);
           }
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    a0 += __shfl_xor_sync(0xffffffffu, a0, o);
-    a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-  }
-  s0 = a0;
-  s1 = a1;
-}
-
-// Two fp16 rows at once against a query held in shared memory as fp32 (the values of the fp16 query, exactly): the
-// same products in the same order as score_two_rows, with 16 registers fewer (for kernels of 1024 threads).
-__device__ __forceinline__ void score_two_rows_sq(const float* s_q, int E, const __half* seg, int64_t row0, int64_t row1, float& s0, float& s1) {
-  const int lane = threadIdx.x & 31;
-  const uint4* r0 = reinterpret_cast<const uint4*>(seg + row0 * E);
-  const uint4* r1 = reinterpret_cast<const uint4*>(seg + row1 * E);
-  const int nvec = E / 8;
-  float a0 = 0.f, a1 = 0.f;
-  for (int v0 = 0; v0 < nvec; v0 += 128) {
-    uint4 x[4], z[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int v = v0 + u * 32 + lane;
-      if (v < nvec) {
-        x[u] = __ldg(r0 + v);
-        z[u] = __ldg(r1 + v);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int v = v0 + u * 32 + lane;
-      if (v < nvec) {
-        float f[8], h[8];
-        unpack8(x[u], f);
-        unpack8(z[u], h);
-        const float4 g0 = *reinterpret_cast<const float4*>(s_q + 8 * v), g1 = *reinterpret_cast<const float4*>(s_q + 8 * v + 4);
-        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          a0 = fmaf(f[i], g[i], a0);
-          a1 = fmaf(h[i], g[i], a1);
         }
       }
     }
@@ -258,11 +227,7 @@ __device__ __forceinline__ void score_rows_direct(const RetrieveParams& p, int q
         const int v = v0 + u * 32 + lane;
         if (v < nvec) {
           if (sizeof(T) == 2) {
-            float f[8], g[8];
-            unpack8(x[u], f);
-            unpack8(y[u], g);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc = fmaf(f[i], g[i], acc);
+            acc = dot8_f16(x[u], y[u], acc);
           } else {
             const float* f = reinterpret_cast<const float*>(&x[u]);
             const float* g = reinterpret_cast<const float*>(&y[u]);
@@ -1200,11 +1165,7 @@ __device__ __forceinline__ float score_one_row(const RetrieveParams& p, int q, c
       const int v = v0 + u * 32 + lane;
       if (v < nvec) {
         if (sizeof(T) == 2) {
-          float f[8], g[8];
-          unpack8(x[u], f);
-          unpack8(y[u], g);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) acc = fmaf(f[i], g[i], acc);
+          acc = dot8_f16(x[u], y[u], acc);
         } else {
           const float* f = reinterpret_cast<const float*>(&x[u]);
           const float* g = reinterpret_cast<const float*>(&y[u]);
