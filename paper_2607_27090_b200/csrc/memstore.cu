@@ -407,8 +407,11 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
     lc.attrs = attr;
     lc.numAttrs = 1;
     cudaLaunchKernelEx(&lc, score_topk_plan_kernel<T, THREADS>, p, rows_per_cta, tickets, keys_cap, n_host, *ip, early);
-  } else
-    score_topk_fused_kernel<T, THREADS><<<grid, THREADS, smem, st>>>(p, rows_per_cta, tickets, keys_cap, n_host);
+  } else {
+    // (a programmatic dependent as well: when retrieve calls follow one another, a call's CTAs are placed while the
+    // call before it drains; the kernel waits for the preceding grid before it touches anything)
+    launch_dependent(score_topk_fused_kernel<T, THREADS>, grid, dim3(THREADS), smem, st, p, rows_per_cta, tickets, keys_cap, n_host);
+  }
 }
 template <typename T, bool PLAN>
 void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,

@@ -1092,6 +1092,8 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
 template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
                                                                          uint32_t* tickets, int keys_capacity, int n_host) {
+  grid_dependency_wait();    // launched as a programmatic dependent: nothing is touched before the preceding grid is done
+  grid_launch_dependents();  // a kernel that follows as a programmatic dependent may be placed while this one drains
   score_topk_body<T, THREADS, false>(p, rows_per_cta, tickets, keys_capacity, n_host, nullptr);
 }
 
