@@ -214,6 +214,8 @@ cudaError_t ensure_fused_smem(int device, size_t bytes) {
   if (bytes <= set_bytes[d]) return cudaSuccess;
   cudaError_t e = cudaSuccess;
   const void* fns[] = {(const void*)score_topk_fused_kernel<__half, kFusedThreadsFew>, (const void*)score_topk_fused_kernel<float, kFusedThreadsFew>,
+                       (const void*)score_topk_fused_kernel<__half, kFusedThreadsBig>, (const void*)score_topk_fused_kernel<float, kFusedThreadsBig>,
+                       (const void*)score_topk_plan_kernel<__half, kFusedThreadsBig>, (const void*)score_topk_plan_kernel<float, kFusedThreadsBig>,
                        (const void*)score_topk_fused_kernel<__half, kFusedThreadsMany>, (const void*)score_topk_fused_kernel<float, kFusedThreadsMany>,
                        (const void*)score_topk_plan_kernel<__half, kFusedThreadsFew>, (const void*)score_topk_plan_kernel<float, kFusedThreadsFew>,
                        (const void*)score_topk_plan_kernel<__half, kFusedThreadsMany>, (const void*)score_topk_plan_kernel<float, kFusedThreadsMany>};
@@ -386,7 +388,7 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
   // (a 1024-thread CTA fills an SM: more CTAs than SMs would only queue behind the first wave)
   // (256-thread CTAs are held to 64 registers so that four of them share an SM: as many CTAs as fit at once, so that the
   // whole grid is one wave and nothing waits for an SM to be refilled)
-  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * (THREADS >= 1024 ? 1 : 4) / nq);
+  const int64_t target_ctas = std::max<int64_t>(1, (int64_t)sm_count * (THREADS >= 1024 ? 1 : THREADS >= 512 ? 2 : 4) / nq);
   int64_t rows = std::max<int64_t>(kWarps, (std::max<int64_t>(n_max, 1) + target_ctas - 1) / target_ctas);
   rows = (rows + kWarps - 1) / kWarps * kWarps;
   const int rows_per_cta = (int)rows;
@@ -416,7 +418,9 @@ void launch_score_topk_threads(int sm_count, int nq, int64_t n_max, const Retrie
 template <typename T, bool PLAN>
 void launch_score_topk(int sm_count, int nq, int64_t n_max, const RetrieveParams& p, uint32_t* tickets, int keys_cap, int n_host,
                        const InjectParams* ip, size_t smem, cudaStream_t st, int early = 0) {
-  if (nq <= kFusedFewQueries)
+  if (nq <= kFusedFewQueries && (n_max > (int64_t)kFusedThreadsFew * kExtractMaxKpl || (PLAN && p.k > kFusedPlanBigK)))
+    launch_score_topk_threads<T, kFusedThreadsBig, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
+  else if (nq <= kFusedFewQueries)
     launch_score_topk_threads<T, kFusedThreadsFew, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);
   else
     launch_score_topk_threads<T, kFusedThreadsMany, PLAN>(sm_count, nq, n_max, p, tickets, keys_cap, n_host, ip, smem, st, early);

@@ -38,9 +38,11 @@ constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkMaxK = 2048;
 constexpr int kFusedMaxRows = 8192;  // largest segment whose top-k runs inside the scoring kernel
-// CTA size of the one-launch scoring + top-k (+ plan) kernels: the last CTA of a query does the selection and the
-// planning alone, which want many threads when there are few queries; with many queries smaller CTAs fill the GPU better
-constexpr int kFusedThreadsFew = 1024, kFusedThreadsMany = 256, kFusedFewQueries = 8;
+// CTA size of the one-launch scoring + top-k (+ plan) kernels.  The last CTA of a query does the selection and the
+// planning alone.  Few queries: 512 threads (two CTAs per SM; they find room on an SM sooner than a CTA that needs all
+// of it, and their barriers are cheaper), 1024 threads when the planning has many tokens to lay out (k above
+// kFusedPlanBigK) or the segment is too long for the 512-thread selection.  Many queries: 256 threads fill the GPU better.
+constexpr int kFusedThreadsFew = 512, kFusedThreadsBig = 1024, kFusedThreadsMany = 256, kFusedFewQueries = 8, kFusedPlanBigK = 32;
 static_assert(2 * kTopkMaxK * sizeof(int32_t) <= kTopkMaxK * sizeof(unsigned long long), "plan arrays reuse the candidate buffer");
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
@@ -1090,7 +1092,7 @@ __device__ __forceinline__ void score_topk_body(const RetrieveParams& p, int row
 // keys held in shared memory (dynamic shared memory: keys_capacity uint32 keys).  n_host >= 0 is the row count
 // of user 0 known to the host (no per-query users): it saves the dependent load of the device-side count.
 template <typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
+__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : THREADS >= 512 ? 2 : 4) score_topk_fused_kernel(const RetrieveParams p, int rows_per_cta,
                                                                          uint32_t* tickets, int keys_capacity, int n_host) {
   grid_dependency_wait();    // launched as a programmatic dependent: nothing is touched before the preceding grid is done
   grid_launch_dependents();  // a kernel that follows as a programmatic dependent may be placed while this one drains
@@ -1103,7 +1105,7 @@ __global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_f
 // this library's copy kernel, they run on the SMs it vacates while it drains - and only the last CTA of a query waits,
 // right before it writes the ids and the plan.
 template <typename T, int THREADS>
-__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : 4) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
+__global__ void __launch_bounds__(THREADS, THREADS >= 1024 ? 1 : THREADS >= 512 ? 2 : 4) score_topk_plan_kernel(const RetrieveParams p, int rows_per_cta,
                                                                         uint32_t* tickets, int keys_capacity, int n_host,
                                                                         const __grid_constant__ InjectParams ip, int early) {
   if (!early) grid_dependency_wait();  // launched as a programmatic dependent: nothing is touched before the preceding grid is done
