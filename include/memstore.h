@@ -86,6 +86,12 @@ enum {
                              call after the store itself was changed (facts added or removed, a new prefix) - the call
                              orders itself after all preceding work, as any launch does.  Results are the same either
                              way. */
+  ,
+  MS_SERVE_EARLY_RETURN = 16u /* memstore_serve_host only: return as soon as the ids, the token count and the status
+                             have reached the host - they are final once the request is planned - instead of waiting
+                             for the stream; the copy of K and V into the cache completes in stream order, as after any
+                             asynchronous call (later work on the same stream sees the injected tokens; the host
+                             synchronises the stream before it reads the cache itself) */
 };
 /* store flag: inject through the bulk-async (TMA) staged copy kernel instead of the direct one (kept for
  * comparison; it is slower on B200 and serves rows of at most 16 KiB, larger rows fall back to the direct kernel) */
@@ -376,8 +382,8 @@ ms_status memstore_retrieve_inject(memstore_t* store, const void* queries, const
  * One request end to end from HOST buffers, for a caller that holds its query and block table in host memory
  * (Sec. 3.3 and 3.4 in one call: search, compose, scatter).  Copies the query, the start position and the block table
  * to the device in one transfer (through a pinned staging buffer owned by the store, allocated on first use),
- * retrieves the k best facts of `user`, injects them (flags: MS_INJECT_*), copies ids, token count and status
- * back in one transfer and waits for the stream.
+ * retrieves the k best facts of `user`, injects them (flags: MS_INJECT_*), has the kernels write ids, token count and
+ * status into pinned host memory and waits for the stream (with MS_SERVE_EARLY_RETURN: only for those results).
  *   query        host, [emb_dim] in emb_dtype          block_table  host int32 [max_blocks]
  *   out_ids      host int32 [k] (best first, -1 padded) out_n_tokens, out_status  host, optional
  * The paged cache itself stays on the device.  Not thread-safe against other calls on the same store.

@@ -56,6 +56,11 @@ struct InjectParams {
   uint32_t* cc_counters;       // [0] hits, [1] fills
   uint32_t spin_limit;    // 0: the default bound of the staged kernel's waits; else a test's shorter bound
   int32_t mute_producer;  // test aid: the staged kernel's producer role issues nothing
+  // memstore_serve_host with MS_SERVE_EARLY_RETURN (one request): a word of pinned host memory, through its device
+  // address, that takes host_seq once the request's ids, token count and status - which the kernels write into pinned
+  // host memory too - are final; nullptr otherwise
+  uint32_t* host_flag;
+  uint32_t host_seq;
 };
 
 constexpr int kPlanThreads = 256;
@@ -381,6 +386,12 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   if (tid == 0) {
     if (p.out_n_tokens) p.out_n_tokens[r] = m;
     if (p.out_status) p.out_status[r] = s_status;
+    if (p.host_flag != nullptr) {
+      // the ids (written before the barriers above, by this CTA or an earlier kernel) and the two words above reach the
+      // host before the flag does
+      __threadfence_system();
+      *reinterpret_cast<volatile uint32_t*>(p.host_flag) = p.host_seq;
+    }
     // the last planning CTA of the call hands the control block to the copy kernel and leaves it clean
     if (p.nreq == 1) {
       p.ctrl->n_tiles = n_tiles;

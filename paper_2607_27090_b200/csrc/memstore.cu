@@ -3,6 +3,8 @@
 // device memory and enqueues launches.  There is no CPU implementation of any step.
 #include "../../include/memstore.h"
 
+#include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -61,6 +63,8 @@ struct memstore {
   uint32_t* tc_fix_tickets = nullptr;
   uint32_t* tc_n_fixups = nullptr;  // queries the fix-up kernel has redone since creation
   int* tc_error = nullptr;
+  uint32_t* serve_flag_dev = nullptr;  // memstore_serve_host, early return: device address of the pinned flag word, while its call runs
+  uint32_t serve_seq = 0;              // value the flag takes for the current request
   // candidate rows emitted by the filter kernel (see score_gemm.cuh)
   uint32_t* tc_hist = nullptr;      // [64][kHistWords] + thr_used[64] (zero between calls) + cand_cnt[64][kCandMaxSegs]
   float* tc_raw = nullptr;                // [64][32 * kRawPerLane]: the table the thresholds of the lists are calibrated from
@@ -78,6 +82,7 @@ struct memstore {
   cudaEvent_t prof_before = nullptr, prof_after = nullptr;  // caller-owned, optional
   // memstore_serve_host staging: one pinned host buffer and one device buffer, inputs first, outputs after
   unsigned char* host_stage = nullptr;
+  cudaStream_t serve_stream = nullptr;  // memstore_serve_host, early return: the inputs go up on this stream
   unsigned char* dev_stage = nullptr;
   size_t stage_bytes = 0;
   cudaStream_t last_stream = nullptr;
@@ -489,6 +494,7 @@ ms_status ensure_stage(memstore* s, size_t bytes) {
   const size_t want = bytes * 2;
   MS_CUDA(s, cudaMalloc(&s->dev_stage, want));
   MS_CUDA(s, cudaHostAlloc(&s->host_stage, want, cudaHostAllocMapped));
+  if (!s->serve_stream) MS_CUDA(s, cudaStreamCreateWithFlags(&s->serve_stream, cudaStreamNonBlocking));
   s->stage_bytes = want;
   return MS_OK;
 }
@@ -497,7 +503,7 @@ ms_status ensure_stage(memstore* s, size_t bytes) {
 void serve_host_layout(const memstore_config& c, int32_t max_blocks, int32_t k, size_t* q_bytes, size_t* in_bytes, size_t* out_bytes) {
   *q_bytes = ((size_t)c.emb_dim * emb_elem_size(c.emb_dtype) + 15) & ~(size_t)15;
   *in_bytes = *q_bytes + 16 + (((size_t)max_blocks * 4 + 15) & ~(size_t)15);
-  *out_bytes = (((size_t)k + 2) * 4 + 15) & ~(size_t)15;
+  *out_bytes = ((((size_t)k + 2) * 4 + 15) & ~(size_t)15) + 16;  // (the last 16 bytes: the flag word of an early return)
 }
 
 // Serialise use of the shared scratch across streams without a host sync: when a call arrives on another
@@ -695,6 +701,7 @@ ms_status memstore_destroy(memstore_t* s) {
     cudaFree(s->append_pairs);
     cudaFree(s->dev_stage);
     if (s->host_stage) cudaFreeHost(s->host_stage);
+    if (s->serve_stream) cudaStreamDestroy(s->serve_stream);
     if (s->last_done) cudaEventDestroy(s->last_done);
     cudaGetLastError();
   }
@@ -1414,6 +1421,8 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.ctrl = s->ctrl;
   p.spin_limit = s->test_spin_limit;
   p.mute_producer = s->test_mute_producers;
+  p.host_flag = nreq == 1 ? s->serve_flag_dev : nullptr;  // (set by memstore_serve_host for the one call it makes)
+  p.host_seq = s->serve_seq;
   if (s->cc_slots) {
     const int64_t cc_tokens = (int64_t)s->cc_n_slots * s->cc_slot_tokens;
     p.cc_slots = s->cc_slots;
@@ -1640,18 +1649,49 @@ ms_status memstore_serve_host(memstore_t* s, const void* query, int32_t user, in
   hdr[0] = start_pos;
   hdr[1] = user;
   memcpy(h + q_bytes + 16, block_table, (size_t)max_blocks * 4);
-  MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, st));
+  const bool early_return = (flags & MS_SERVE_EARLY_RETURN) != 0;
+  flags &= ~(uint32_t)MS_SERVE_EARLY_RETURN;
+  if (early_return) {
+    // The previous request's planning is over (its call saw the results), so the staging buffer on the device is free
+    // although that request's copy kernel may still run: the inputs go up beside it on a stream of their own and the
+    // host waits for them here.  They are then complete before this request is launched, which is all the early
+    // scoring of MS_INPUTS_STABLE needs: the retrieval runs while the previous copy kernel drains.
+    MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, s->serve_stream));
+    MS_CUDA(s, cudaStreamSynchronize(s->serve_stream));
+    flags |= MS_INPUTS_STABLE;
+  } else {
+    MS_CUDA(s, cudaMemcpyAsync(d, h, in_bytes, cudaMemcpyHostToDevice, st));
+  }
   int32_t* d_hdr = reinterpret_cast<int32_t*>(d + q_bytes);
   // The results (k ids, token count, status: a few hundred bytes) are written by the kernels straight into the pinned
   // host buffer through its device address, so that no copy back has to be queued behind the copy kernel.
   void* res_dev = nullptr;
   MS_CUDA(s, cudaHostGetDevicePointer(&res_dev, h + in_bytes, 0));
   int32_t* d_ids = static_cast<int32_t*>(res_dev);
+  volatile uint32_t* flag_host = reinterpret_cast<volatile uint32_t*>(h + in_bytes + out_bytes - 16);
+  if (early_return) {
+    s->serve_seq += 1;
+    if (s->serve_seq == 0) s->serve_seq = 1;
+    *flag_host = 0;
+    s->serve_flag_dev = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(res_dev) + out_bytes - 16);
+  }
   ms_status rc = memstore_retrieve_inject(s, d, c.n_users > 1 ? d_hdr + 1 : nullptr, 1, k, d_hdr,
                                           reinterpret_cast<const int32_t*>(d + q_bytes + 16), max_blocks, cache, d_ids, nullptr,
                                           d_ids + k, d_ids + k + 1, nullptr, 0, flags, stream);
+  s->serve_flag_dev = nullptr;
   if (rc != MS_OK) return rc;
-  MS_CUDA(s, cudaStreamSynchronize(st));
+  bool seen = false;
+  if (early_return) {
+    // the planning CTA writes the flag after the results; a launch that failed, or a device that is busy with other
+    // work for long, ends the wait and the stream is synchronised as usual
+    const auto t0 = std::chrono::steady_clock::now();
+    for (uint32_t spins = 1; !seen; ++spins) {
+      seen = *flag_host == s->serve_seq;
+      if (!seen && (spins & 1023u) == 0 && std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(200)) break;
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+  }
+  if (!seen) MS_CUDA(s, cudaStreamSynchronize(st));
   const int32_t* res = reinterpret_cast<const int32_t*>(h + in_bytes);
   memcpy(out_ids, res, (size_t)k * 4);
   if (out_n_tokens) *out_n_tokens = res[k];

@@ -25,6 +25,7 @@ INJECT_REVERSE = 1
 INJECT_PREFIX = 2
 RETRIEVE_ANN = 4
 INPUTS_STABLE = 8
+SERVE_EARLY_RETURN = 16
 COMPOSE_CACHE_ALL = 1
 CACHE_BF16, CACHE_FP8_E4M3 = 0, 1
 STORE_TMA_COPY_PATH = 1

@@ -1203,6 +1203,43 @@ def test_serve_host_matches_the_device_calls():
     ms.close()
 
 
+def test_serve_host_early_return():
+    """MS_SERVE_EARLY_RETURN: the call comes back once ids, token count and status are on the host; they equal those of
+    the waiting call, and after a stream synchronise so does the cache.  Several requests in a row without a
+    synchronise in between (the staging buffers and the flag word are reused), a request with a data error, and a
+    segment long enough for the separate planning kernel."""
+    for n_facts, E in ((120, 256), (9000, 64)):
+        hs = HostStore(23, n_facts, 2, 4, 64, 8, 40, E, "float16", lens=None if n_facts < 1000 else [8 + (i % 9) for i in range(n_facts)])
+        ms = hs.to_memstore(5e5)
+        bs, nb, k = 16, 96, 6
+        ca, cb = make_cache(hs, nb, bs), make_cache(hs, nb, bs)
+        reqs = []
+        for i in range(5):
+            q = synth.queries(40 + i, 1, E, "float16")[0]
+            table = synth.block_tables(50 + i, nb, 32, 1)[0]
+            reqs.append((q, 3 + 16 * i, table))
+        waited = []
+        for q, start, table in reqs:
+            out = np.full(k + 2, -5, np.int32)
+            ms.serve_host(q, k, start, table, ca, out, flags=M.INJECT_REVERSE)
+            waited.append(out)
+        early = []
+        for q, start, table in reqs:  # no synchronise between the calls
+            out = np.full(k + 2, -5, np.int32)
+            ms.serve_host(q, k, start, table, cb, out, flags=M.INJECT_REVERSE | M.SERVE_EARLY_RETURN)
+            early.append(out.copy())  # final when the call returns
+        torch.cuda.synchronize()
+        for a, b in zip(waited, early):
+            assert a.tolist() == b.tolist() and b[k + 1] == 0 and b[k] > 0
+        assert torch.equal(ca.k.view(torch.int16), cb.k.view(torch.int16)) and torch.equal(ca.v.view(torch.int16), cb.v.view(torch.int16))
+        # a block table that is too short: the status word arrives with the early return as well
+        out = np.full(k + 2, -5, np.int32)
+        ms.serve_host(reqs[0][0], k, 3, reqs[0][2][:1].copy(), cb, out, flags=M.SERVE_EARLY_RETURN)
+        assert out[k + 1] & M.REQ_BLOCK_TABLE_SHORT and out[:k].tolist() == waited[0][:k].tolist()
+        torch.cuda.synchronize()
+        ms.close()
+
+
 # ------------------------------------------------------------------------------------------------ safety
 def test_inject_data_errors_set_status_and_skip():
     lens = [4, 6, 0, 5]
