@@ -77,16 +77,17 @@ enum {
   MS_INJECT_PREFIX = 2u,  /* place the store's instruction prefix (memstore_set_prefix) before the facts */
   MS_RETRIEVE_ANN = 4u,   /* memstore_retrieve_inject / memstore_serve_host only: retrieve through the graph index
                              (memstore_retrieve_ann with its default parameters) instead of the exact scan */
-  MS_INPUTS_STABLE = 8u   /* memstore_retrieve_inject only: the caller vouches that queries, query_users, start_pos and
+  MS_INPUTS_STABLE = 8u,  /* memstore_retrieve_inject only: the caller vouches that queries, query_users, start_pos and
                              block_tables were completely written before the work that precedes this call in the stream
-                             began (a serving loop whose next query is ready before the previous injection is enqueued).
+                             began (a serving loop whose next query is ready before the previous injection is enqueued),
+                             or that the host has seen them complete before it makes this call (a transfer on another
+                             stream that the host waited for).
                              The scoring and selection of this call may then overlap the tail of the preceding kernel -
                              typically the previous request's copy kernel, whose draining SMs they use; ids, plan and
                              cache are still written strictly after it.  Without the flag - and for the first such
                              call after the store itself was changed (facts added or removed, a new prefix) - the call
                              orders itself after all preceding work, as any launch does.  Results are the same either
                              way. */
-  ,
   MS_SERVE_EARLY_RETURN = 16u /* memstore_serve_host only: return as soon as the ids, the token count and the status
                              have reached the host - they are final once the request is planned - instead of waiting
                              for the stream; the copy of K and V into the cache completes in stream order, as after any
