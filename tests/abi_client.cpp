@@ -108,6 +108,20 @@ int main() {
   for (size_t i = 0; i < cache_elems; ++i) still += vc[i] == 0x1111;
   CHECK(still == cache_elems - touched);
 
+  // the same request from host buffers, waited for and with an early return: the same id, token count and status, and
+  // (after a synchronise) the same cache
+  {
+    for (uint32_t flags : {0u, (uint32_t)MS_SERVE_EARLY_RETURN}) {
+      int32_t h_id = -9, h_n = -9, h_st = -9;
+      CHECK(memstore_serve_host(store, emb1.data(), 0, 1, 0, table, 2, &cache, flags, &h_id, &h_n, &h_st, nullptr) == MS_OK);
+      CHECK(h_id == 1 && h_n == T && h_st == 0);
+      CHECK(cudaDeviceSynchronize() == cudaSuccess);
+      std::vector<uint16_t> vc2(cache_elems);
+      cudaMemcpy(vc2.data(), d_vc, cache_elems * 2, cudaMemcpyDeviceToHost);
+      CHECK(vc2 == vc);
+    }
+  }
+
   memstore_stats_t st;
   CHECK(memstore_stats(store, &st) == MS_OK && st.n_facts == 2 && st.kv_tokens_used == T);
   CHECK(memstore_inject(store, d_ids, 1, 1, d_start, d_table, -1, &cache, nullptr, nullptr, nullptr, 0, 0, nullptr) == MS_ERR_INVALID_ARG);
