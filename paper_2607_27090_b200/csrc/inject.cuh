@@ -61,6 +61,8 @@ struct InjectParams {
   // host memory too - are final; nullptr otherwise
   uint32_t* host_flag;
   uint32_t host_seq;
+  int32_t host_flag_in_copy;  // 1: the direct copy kernel raises the flag when it starts (the planning kernel is then spared the
+                              // system-wide fence at its end, which the copy kernel would have to wait out); 0: the planning does
 };
 
 constexpr int kPlanThreads = 256;
@@ -386,7 +388,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   if (tid == 0) {
     if (p.out_n_tokens) p.out_n_tokens[r] = m;
     if (p.out_status) p.out_status[r] = s_status;
-    if (p.host_flag != nullptr) {
+    if (p.host_flag != nullptr && !p.host_flag_in_copy) {
       // the ids (written before the barriers above, by this CTA or an earlier kernel) and the two words above reach the
       // host before the flag does
       __threadfence_system();
@@ -586,6 +588,12 @@ __global__ void __launch_bounds__(kCopyThreads, 3) inject_copy_kernel(const Inje
   // SMs once every CTA of this grid has got this far; it waits for this grid's completion before it does anything.
   grid_launch_dependents();
 
+  if (p.host_flag != nullptr && p.host_flag_in_copy && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
+    // early return of memstore_serve_host: the planning grid is complete, so the request's ids, token count and status
+    // are final; they reach the host before the flag does
+    __threadfence_system();
+    *reinterpret_cast<volatile uint32_t*>(p.host_flag) = p.host_seq;
+  }
   const uint32_t n_tiles = min(p.ctrl->n_tiles, p.tiles_capacity);
   const uint32_t n_items = n_tiles * (uint32_t)p.n_layers;
   // items in (layer, tile) order: CTAs that run together stream neighbouring rows of one layer.  The grid is the

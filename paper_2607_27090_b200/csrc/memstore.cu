@@ -1338,6 +1338,13 @@ ms_status memstore_retrieve_static(memstore_t* s, const void* queries, const int
 namespace {
 
 // Validation, scratch sizing and parameter block shared by memstore_inject and memstore_retrieve_inject.
+// the staged (bulk-async) copy kernel serves the plain parameterisation only (whole-head rotation, bf16 cache)
+bool copy_uses_tma(const memstore* s, const ms_paged_cache* cache) {
+  const memstore_config& c = s->cfg;
+  const int row_bytes = c.n_kv_heads * c.head_dim * 2;
+  return s->tma_path && !s->cc_slots && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
+}
+
 ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int32_t k, const int32_t* start_pos,
                          const int32_t* block_tables, int32_t max_blocks, const ms_paged_cache* cache, int32_t* out_n_tokens,
                          int32_t* out_status, int64_t* out_slot_mapping, int64_t slot_stride, uint32_t flags, cudaStream_t st,
@@ -1423,6 +1430,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
   p.mute_producer = s->test_mute_producers;
   p.host_flag = nreq == 1 ? s->serve_flag_dev : nullptr;  // (set by memstore_serve_host for the one call it makes)
   p.host_seq = s->serve_seq;
+  p.host_flag_in_copy = copy_uses_tma(s, cache) ? 0 : 1;
   if (s->cc_slots) {
     const int64_t cc_tokens = (int64_t)s->cc_n_slots * s->cc_slot_tokens;
     p.cc_slots = s->cc_slots;
@@ -1439,7 +1447,7 @@ ms_status prepare_inject(memstore* s, const int32_t* fact_ids, int32_t nreq, int
 
   // layers per work item (bulk-async kernel): the largest power of two that still leaves every CTA about 16 items
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
-  const bool use_tma = s->tma_path && !s->cc_slots && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
+  const bool use_tma = copy_uses_tma(s, cache);
   const int resident_ctas = use_tma ? s->sm_count : s->sm_count * s->copy_ctas_per_sm;
   const int64_t est_tiles = std::max<int64_t>(1, ((int64_t)k * (s->max_fact_len + 1) / 2 + p.prefix_len + kTileTokens - 1) / kTileTokens * nreq);
   int lpi = 1;
@@ -1454,7 +1462,7 @@ ms_status launch_copy(memstore* s, const InjectParams& p, const ms_paged_cache* 
   const memstore_config& c = s->cfg;
   const int row_bytes = c.n_kv_heads * c.head_dim * 2;
   // the staged kernel serves the plain parameterisation only (whole-head rotation, bf16 cache)
-  const bool use_tma = s->tma_path && !s->cc_slots && row_bytes <= kTmaAreaBytes && c.rotary_dim == c.head_dim && cache->dtype == MS_CACHE_BF16;
+  const bool use_tma = copy_uses_tma(s, cache);
   cudaLaunchConfig_t lc{};
   lc.stream = st;
   cudaLaunchAttribute attr[1];

@@ -1206,11 +1206,12 @@ def test_serve_host_matches_the_device_calls():
 def test_serve_host_early_return():
     """MS_SERVE_EARLY_RETURN: the call comes back once ids, token count and status are on the host; they equal those of
     the waiting call, and after a stream synchronise so does the cache.  Several requests in a row without a
-    synchronise in between (the staging buffers and the flag word are reused), a request with a data error, and a
-    segment long enough for the separate planning kernel."""
-    for n_facts, E in ((120, 256), (9000, 64)):
+    synchronise in between (the staging buffers and the flag word are reused), a request with a data error, a
+    segment long enough for the separate planning kernel, and a store that copies with the staged kernel."""
+    for n_facts, E, store_flags in ((120, 256, 0), (9000, 64, 0), (120, 256, M.STORE_TMA_COPY_PATH)):
+        # (with the staged copy kernel the planning kernel raises the flag, otherwise the copy kernel does when it starts)
         hs = HostStore(23, n_facts, 2, 4, 64, 8, 40, E, "float16", lens=None if n_facts < 1000 else [8 + (i % 9) for i in range(n_facts)])
-        ms = hs.to_memstore(5e5)
+        ms = hs.to_memstore(5e5, flags=store_flags)
         bs, nb, k = 16, 96, 6
         ca, cb = make_cache(hs, nb, bs), make_cache(hs, nb, bs)
         reqs = []
