@@ -400,17 +400,19 @@ def measure(name: str, iters: int, seed: int = 0, hot_per_user: int | None = Non
     torch.cuda.synchronize()
     assert int(status.abs().sum()) == 0, "a request named a fact without K/V: the hot set was chosen too small"
     m_total = int(n_tok.sum())
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-    t_r, t_i = [], []
+    # retrieve and inject alternate on the stream without a host synchronise in between (the GPU stays busy, as in a
+    # serving loop: an event pair around a call issued to an idle GPU would also time the host's launch path)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(iters)]
     for i in range(iters):
-        ev[0].record(stream)
+        evs[i][0].record(stream)
         retrieve()
-        ev[1].record(stream)
+        evs[i][1].record(stream)
         inject(i)
-        ev[2].record(stream)
-        torch.cuda.synchronize()
-        t_r.append(ev[0].elapsed_time(ev[1]) * 1e3)
-        t_i.append(ev[1].elapsed_time(ev[2]) * 1e3)
+        evs[i][2].record(stream)
+    torch.cuda.synchronize()
+    t_r = [e[0].elapsed_time(e[1]) * 1e3 for e in evs]
+    t_i = [e[1].elapsed_time(e[2]) * 1e3 for e in evs]
+    ev = evs[0]
     # the retrieval call alone, back to back (no injection between two calls): a few calls first, so that the timed ones
     # start in the steady state, and enough of them that the first one's lone start does not weigh
     n_b2b = max(iters, 100)
