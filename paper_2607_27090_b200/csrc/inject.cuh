@@ -65,7 +65,8 @@ struct InjectParams {
                               // system-wide fence at its end, which the copy kernel would have to wait out); 0: the planning does
 };
 
-constexpr int kPlanThreads = 256;
+constexpr int kPlanThreads = 256;      // planning CTA when a call holds more requests than the GPU has SMs
+constexpr int kPlanThreadsWide = 1024;  // otherwise: the tile descriptors are laid out one token per thread and pass
 constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by the plan kernel
 
 // ------------------------------------------------------------------------------------------------
@@ -410,13 +411,14 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   }
 }
 
-__global__ void __launch_bounds__(kPlanThreads) inject_plan_kernel(const InjectParams p) {
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) inject_plan_kernel(const InjectParams p) {
   __shared__ int32_t s_begin[kPlanMaxK];  // b_i: first composed token of placed fact i
   __shared__ int32_t s_src[kPlanMaxK];    // arena token of the fact's first token
   __shared__ PlanShared ps;
   grid_dependency_wait();    // launched as a programmatic dependent (of the previous call's copy kernel, typically)
   grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
-  plan_request<kPlanThreads>(p, blockIdx.x, s_begin, s_src, ps);
+  plan_request<THREADS>(p, blockIdx.x, s_begin, s_src, ps);
 }
 
 // ------------------------------------------------------------------------------------------------
