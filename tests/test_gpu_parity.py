@@ -606,6 +606,35 @@ def test_inject_batch_of_requests_shares_one_cache():
     assert untouched_mask_ok(cache, np.concatenate(all_slots), SENT)
 
 
+def test_inject_more_requests_than_sms():
+    """A call with more requests than the GPU has SMs takes the 256-thread planning kernel and an ordinary launch of the
+    copy kernel (fewer requests: 1024-thread planning CTAs and a programmatic launch): 300 short requests in one cache."""
+    hs = HostStore(15, 60, 2, 2, 64, 1, 6, 64, "float16")
+    ms = hs.to_memstore(1e4)
+    nreq, k, bs = 300, 4, 16
+    rng = np.random.default_rng(1)
+    ids = rng.integers(-1, 60, size=(nreq, k)).astype(np.int32)
+    starts = rng.integers(0, 40, nreq).astype(np.int32)
+    per = (40 + k * 6 + bs - 1) // bs + 1
+    nb = per * nreq + 2
+    tables = synth.block_tables(16, nb, per, nreq)
+    cache = make_cache(hs, nb, bs)
+    n_tok, status = ms.inject(to_dev(ids), to_dev(starts), to_dev(tables), cache, flags=M.INJECT_REVERSE)
+    torch.cuda.synchronize()
+    from parity import check_k, gather_cache_rows
+
+    all_slots = []
+    for r in range(nreq):
+        res = oracle.inject(np.ascontiguousarray(ids[r][::-1]), hs.offs, hs.lens, hs.k, hs.v, 1e4, int(starts[r]), tables[r], bs, nb)
+        assert int(n_tok[r]) == res.m and int(status[r]) == 0, r
+        if res.m:
+            kb, vb = gather_cache_rows(cache, res.slots)
+            assert np.array_equal(vb, res.v)
+            check_k(kb, res.k_ref)
+            all_slots.append(res.slots)
+    assert untouched_mask_ok(cache, np.concatenate(all_slots), SENT)
+
+
 def test_inject_at_the_largest_sizes():
     """The longest id list (4096 entries, repeats allowed), one entry too many, and the last representable positions
     (2^24 - 1 is the largest position that is exact in fp32; tokens beyond max_position are refused)."""
