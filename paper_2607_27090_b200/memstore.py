@@ -241,12 +241,20 @@ class PagedCache:
         return self.k.dtype == torch.uint8
 
     def _struct(self) -> _PagedCache:
+        # (made once per state of the cache object: the calls of a serving loop pass the same cache every time)
+        key = (self.k.data_ptr(), self.v.data_ptr(), self.layer_stride, self.block_stride, self.token_stride, self.head_stride,
+               self.num_blocks, self.block_size, self.fp8, self.k_scale, self.v_scale)  # fmt: skip
+        made = getattr(self, "_made", None)
+        if made is not None and made[0] == key:
+            return made[1]
         for t, n in ((self.k, "k"), (self.v, "v")):
             if not t.is_cuda or t.dtype not in (torch.bfloat16, torch.uint8) or t.dtype != self.k.dtype:
                 raise TypeError(f"cache.{n} must be a CUDA bfloat16 (or, for an 8-bit cache, uint8) tensor")
-        return _PagedCache(self.k.data_ptr(), self.v.data_ptr(), self.layer_stride, self.block_stride,
-                           self.token_stride, self.head_stride, self.num_blocks, self.block_size,
-                           CACHE_FP8_E4M3 if self.fp8 else CACHE_BF16, self.k_scale, self.v_scale)  # fmt: skip
+        cs = _PagedCache(self.k.data_ptr(), self.v.data_ptr(), self.layer_stride, self.block_stride,
+                         self.token_stride, self.head_stride, self.num_blocks, self.block_size,
+                         CACHE_FP8_E4M3 if self.fp8 else CACHE_BF16, self.k_scale, self.v_scale)  # fmt: skip
+        self._made = (key, cs)
+        return cs
 
 
 class MemStore:
