@@ -66,6 +66,7 @@ struct InjectParams {
 };
 
 constexpr int kPlanThreads = 256;      // planning CTA when a call holds more requests than the GPU has SMs
+constexpr int kPlanMaxParts = 16;       // CTAs that plan one long request together
 constexpr int kPlanThreadsWide = 1024;  // otherwise: the tile descriptors are laid out one token per thread and pass
 constexpr int kPlanMaxK = 4096;  // facts per request held in shared memory by the plan kernel
 
@@ -107,9 +108,13 @@ __device__ __forceinline__ void plan_prefetch(const InjectParams& p, const int r
 // been called for this request by the same threads.  PREFILLED: the caller has resolved the facts already - s_begin[j]
 // holds the LENGTH and s_src[j] the source token of entry j (placement order, entry 0 left for the prefix when there
 // is one), data errors of the lookup are in ps.status, and a block barrier separates those writes from this call.
+// parts > 1 (a call of ONE long request without a composition cache): `parts` CTAs plan the request together.  Each
+// resolves the facts and scans the lengths itself (cheap), they share the per-token work - every CTA takes every
+// parts-th pass of THREADS tokens - and the last one to finish (a ticket in the control block, whose `acc` word gathers
+// the status bits meanwhile) writes the token count, the status and the tile count.
 template <int THREADS, bool PREFETCHED = false, bool PREFILLED = false>
 __device__ __forceinline__ void plan_request(const InjectParams& p, const int r, int32_t* s_begin, int32_t* s_src, PlanShared& ps,
-                                             const int32_t* ids_smem = nullptr) {
+                                             const int32_t* ids_smem = nullptr, const uint32_t part = 0, const uint32_t parts = 1) {
   int32_t* const s_scan = ps.scan;
   int32_t& s_carry = ps.carry;
   int32_t& s_status = ps.status;
@@ -235,7 +240,8 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   if (bad_start && m > 0) {
     if (tid == 0) atomicOr(&s_status, start < 0 ? 64 /*MS_REQ_BAD_START*/ : 16 /*MS_REQ_POSITION_OVERFLOW*/);
     if (p.out_slot_mapping)
-      for (int64_t q = tid; q < min((int64_t)m, p.slot_stride); q += THREADS) p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = -1;
+      for (int64_t q = (int64_t)part * THREADS + tid; q < min((int64_t)m, p.slot_stride); q += (int64_t)parts * THREADS)
+        p.out_slot_mapping[(int64_t)r * p.slot_stride + q] = -1;
   }
   // ---- composition cache: has this very request been composed before, or should it be recorded now? ------------
   int32_t hit_base = -1, fill_base = kNoFill;
@@ -336,7 +342,7 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
 
   const int bs = p.block_size;
   const int bs_shift = (bs & (bs - 1)) == 0 ? 31 - __clz(bs) : -1;  // block sizes are powers of two in practice
-  for (uint32_t e = tid; e < n_tiles * kTileTokens; e += THREADS) {
+  for (uint32_t e = part * THREADS + tid; e < n_tiles * kTileTokens; e += parts * THREADS) {
     const uint32_t t = e / kTileTokens, ln = e % kTileTokens;
     const int32_t pos = first_tile_pos + (int32_t)e;
     const int32_t q = pos - start;  // index in the composed segment
@@ -386,7 +392,24 @@ __device__ __forceinline__ void plan_request(const InjectParams& p, const int r,
   }
   __syncwarp();
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && parts > 1) {
+    // one request planned by several CTAs: the last of them publishes
+    if (s_status) atomicOr(&p.ctrl->acc, (uint32_t)s_status);
+    __threadfence();  // this CTA's descriptors and status bits are visible before its arrival is
+    if (atomicAdd(&p.ctrl->planned, 1u) == parts - 1u) {
+      __threadfence();
+      const int32_t st_all = (int32_t)atomicExch(&p.ctrl->acc, 0u);
+      if (p.out_n_tokens) p.out_n_tokens[r] = m;
+      if (p.out_status) p.out_status[r] = st_all;
+      if (p.host_flag != nullptr && !p.host_flag_in_copy) {
+        __threadfence_system();
+        *reinterpret_cast<volatile uint32_t*>(p.host_flag) = p.host_seq;
+      }
+      p.ctrl->n_tiles = n_tiles;
+      p.ctrl->work_next = 0;
+      p.ctrl->planned = 0;
+    }
+  } else if (tid == 0) {
     if (p.out_n_tokens) p.out_n_tokens[r] = m;
     if (p.out_status) p.out_status[r] = s_status;
     if (p.host_flag != nullptr && !p.host_flag_in_copy) {
@@ -418,7 +441,7 @@ __global__ void __launch_bounds__(THREADS) inject_plan_kernel(const InjectParams
   __shared__ PlanShared ps;
   grid_dependency_wait();    // launched as a programmatic dependent (of the previous call's copy kernel, typically)
   grid_launch_dependents();  // the copy kernel may start its prologue now; it waits before reading the plan
-  plan_request<THREADS>(p, blockIdx.x, s_begin, s_src, ps);
+  plan_request<THREADS>(p, blockIdx.x, s_begin, s_src, ps, nullptr, blockIdx.y, gridDim.y);
 }
 
 // ------------------------------------------------------------------------------------------------

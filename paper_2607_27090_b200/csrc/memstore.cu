@@ -1565,6 +1565,12 @@ ms_status memstore_inject(memstore_t* s, const int32_t* fact_ids, int32_t nreq, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.gridDim = dim3((unsigned)nreq);
     const bool wide = nreq <= s->sm_count;  // every planning CTA has an SM to itself
+    // one long request (and no composition cache, whose bookkeeping one CTA does): several CTAs share its per-token work,
+    // one per 1024 tokens (one pass of a CTA) the request is expected to hold
+    const double mean_len = s->n_resident > 0 ? (double)(s->kv_tokens_used - s->prefix_tokens_total + s->host_tokens_used) / (double)s->n_resident : 0.0;
+    const int64_t est_tokens = (int64_t)((double)k * mean_len) + p.prefix_len;
+    const int parts = (nreq == 1 && !s->cc_slots) ? (int)std::max<int64_t>(1, std::min<int64_t>(kPlanMaxParts, est_tokens / 1024)) : 1;
+    lc.gridDim = dim3((unsigned)nreq, (unsigned)parts);
     lc.blockDim = dim3(wide ? kPlanThreadsWide : kPlanThreads);
     lc.stream = st;
     lc.attrs = attr;

@@ -651,6 +651,18 @@ def test_inject_at_the_largest_sizes():
     cache = make_cache(hs, nb, bs)
     out = run_inject_and_check(ms, hs, ids, 7, table, cache, 1e4, flags=M.INJECT_REVERSE)
     assert out["m"] == m and out["exact_frac"] > 0.99
+    # (a request this long is planned by several CTAs together.)  The same request with half the block table: the CTAs
+    # that plan the later tokens find the table short, the status word gathers their bit, the token count is the
+    # composed length all the same, and the blocks of the first half hold what the full run wrote there
+    half = len(table) // 2
+    cache_h = make_cache(hs, nb, bs)
+    n_tok_h, status_h = ms.inject(to_dev(ids[None]), to_dev(np.array([7], np.int32)), to_dev(table[None, :half].copy()), cache_h,
+                                  flags=M.INJECT_REVERSE)  # fmt: skip
+    torch.cuda.synchronize()
+    assert int(n_tok_h[0]) == m and int(status_h[0]) == M.REQ_BLOCK_TABLE_SHORT
+    blocks = torch.from_numpy(table[:half].astype(np.int64)).to(DEV)
+    for full, part in ((cache.k, cache_h.k), (cache.v, cache_h.v)):
+        assert torch.equal(full.view(torch.int16)[:, blocks], part.view(torch.int16)[:, blocks])
     with pytest.raises(RuntimeError):
         ms.inject(to_dev(np.zeros((1, 4097), np.int32)), to_dev(np.array([0], np.int32)), to_dev(table[None]), cache)
     # the end of the position range: 31 tokens placed from 2^24 - 20; the last 11 are refused
